@@ -1,0 +1,206 @@
+/*
+ * kdn.h -- C ABI of libkdn: the data-movement hot path of a Knowledge Delivery
+ * Network (KDN) on one NVIDIA B200 (sm_100a).
+ *
+ * A KDN keeps precomputed KV caches apart from the serving engine and hands
+ * them back on demand (paper Sec. 3.1: storage, delivery and blending
+ * modules).  The engine talks to it through two calls, "store the KV cache"
+ * and "retrieve the KV cache" (Sec. 3.2, "Interface with LLM serving
+ * engines"), and a retrieved context may be put together from several stored
+ * pieces (Sec. 3.1 blending module; Sec. 3.2 "KV-cache blending").  This
+ * library is that path between an engine's paged GPU KV pool and compact
+ * per-chunk buffers:
+ *
+ *   kdn_store     paged pool  -> chunk buffers   (gather, optional int8 coding)
+ *   kdn_retrieve  chunk buffers -> paged pool    (optional decoding, scatter)
+ *   kdn_compose   several chunks -> one request's blocks at new positions,
+ *                 keys re-rotated by the rotary-embedding position shift
+ *
+ * Every step runs in CUDA kernels on the caller's stream.  There is no CPU
+ * fallback: without a usable CUDA device kdn_create fails.
+ *
+ * ---------------------------------------------------------------- layouts --
+ * Pool (engine-owned device memory), for every layer l and for K and V
+ * separately:            bf16 pool[n_blocks][block_size][n_kv_heads][head_dim]
+ * Block table (device):  int32 table[n_table_blocks]; request position p lives
+ *                        in block table[p / block_size], slot p % block_size.
+ * Chunk, T tokens, L layers, H heads, D head_dim, kv 0 = K, 1 = V:
+ *   KDN_CODEC_RAW_BF16   bf16 data[L][2][T][H][D]               4*L*T*H*D bytes
+ *   KDN_CODEC_INT8_G64   int8 codes[L][2][T][H][D] followed by
+ *                        fp32 scales[L][2][T][H*D/64]           2*L*T*H*D*(1+4/64) bytes
+ *   No header, no padding, little endian.  A chunk does not record where it
+ *   sat in the pool; it can be retrieved into any blocks of any request.
+ * int8 coding: group = 64 consecutive head_dim elements of one token-head row;
+ *   a = max|x|, scale = a/127 in fp32; scale < FLT_MIN -> scale 0, codes 0;
+ *   else code = round_half_even(x * (127/a)) in fp32, in [-127, 127];
+ *   decode = bf16_round_nearest_even((float)code * scale).
+ * Key re-rotation in kdn_compose: the stored keys of a part carry rotary
+ *   position embedding for positions base_pos + t; placing the part at
+ *   dst_pos rotates each pair (k[i], k[i + D/2]) of every head by
+ *   (dst_pos - base_pos) * theta^(-2i/D).  Angles are evaluated in fp64 on the
+ *   device, the rotation itself in fp32.  Values are copied unchanged.
+ *
+ * -------------------------------------------------------------- ownership --
+ * The caller owns pools, block tables, chunk buffers and streams.  The
+ * library owns only the context: a status word, a small ring of launch
+ * descriptors, a rotation table, and (on first use of pinned-host chunks) two
+ * staging slabs.  It never frees or reallocates caller memory.
+ *
+ * ----------------------------------------------------------------- errors --
+ * Argument errors are returned at once and nothing is enqueued.  Otherwise a
+ * call returns after enqueueing its work; it does not wait for the GPU.
+ * Errors found on the device (a block id outside the pool, a copy that never
+ * completed) skip the affected tile, never fault, and are reported by
+ * kdn_status_sync.  A context is not thread safe; use one per thread.
+ */
+#ifndef KDN_H
+#define KDN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct kdn_ctx kdn_ctx;   /* opaque */
+
+typedef enum {
+    KDN_OK = 0,
+    KDN_E_INVAL = 1,        /* null pointer, negative count, unknown enum value */
+    KDN_E_SHAPE = 2,        /* chunk.bytes or n_tokens does not match the pool's shape */
+    KDN_E_ALIGN = 3,        /* a pointer is not 16-byte aligned, or H*D*2 is not a multiple of 16 */
+    KDN_E_RANGE = 4,        /* token range beyond the block table; block id outside the pool (device) */
+    KDN_E_UNSUPPORTED = 5,  /* int8 with head_dim % 64 != 0; rotation with head_dim % 16 != 0; ... */
+    KDN_E_CUDA = 6,         /* a CUDA runtime call failed */
+    KDN_E_NOMEM = 7,        /* context scratch could not be allocated */
+    KDN_E_TIMEOUT = 8       /* a bounded wait inside a kernel gave up (device) */
+} kdn_status;
+
+typedef enum { KDN_CODEC_RAW_BF16 = 0, KDN_CODEC_INT8_G64 = 1 } kdn_codec;
+typedef enum { KDN_MEM_DEVICE = 0, KDN_MEM_PINNED_HOST = 1 } kdn_mem;
+
+/* An engine's paged KV pool (Sec. 3.2 names vLLM's paged memory).  k_layers and v_layers are HOST
+ * arrays of n_layers DEVICE pointers, each to bf16 [n_blocks][block_size][n_kv_heads][head_dim],
+ * 16-byte aligned.  The arrays are copied at registration; the pool memory stays the caller's. */
+typedef struct {
+    int32_t n_layers, n_kv_heads, head_dim, block_size;
+    int64_t n_blocks;
+    void *const *k_layers;
+    void *const *v_layers;
+} kdn_pool_desc;
+
+/* One stored chunk: the KV cache of n_tokens consecutive tokens (Sec. 3.1 storage module).
+ * data: 16-byte aligned; device memory (mem = KDN_MEM_DEVICE) or page-locked host memory
+ * (KDN_MEM_PINNED_HOST).  bytes must equal kdn_chunk_bytes(pool, n_tokens, codec).
+ * base_pos: the absolute position of token 0 when its keys were computed; only kdn_compose reads it. */
+typedef struct {
+    void   *data;
+    size_t  bytes;
+    int32_t n_tokens;
+    int32_t codec;      /* kdn_codec */
+    int32_t mem;        /* kdn_mem */
+    int32_t reserved;   /* 0 */
+    int64_t base_pos;
+} kdn_chunk;
+
+/* One transfer between a request's blocks and one chunk.  Chunk token t <-> request position
+ * token_offset + t.  block_table: DEVICE int32 [n_table_blocks] in the request's logical order.
+ * Needs token_offset >= 0 and token_offset + n_tokens <= n_table_blocks * block_size.  Neither
+ * token_offset nor n_tokens need be a multiple of block_size. */
+typedef struct {
+    const int32_t *block_table;
+    int32_t  n_table_blocks;
+    int32_t  reserved;  /* 0 */
+    int64_t  token_offset;
+    kdn_chunk chunk;
+} kdn_xfer_op;
+
+/* One composed request (Sec. 3.1 blending module): part j is written at request positions
+ * part_dst_pos[j] + t.  parts and part_dst_pos are HOST arrays of n_parts entries.  Parts must not
+ * overlap each other; positions no part covers keep their contents.
+ * rope_style 0 = pairs (i, i + head_dim/2); no other style is implemented. */
+typedef struct {
+    const int32_t  *block_table;     /* device */
+    int32_t         n_table_blocks;
+    int32_t         n_parts;
+    const kdn_chunk *parts;
+    const int64_t  *part_dst_pos;
+    double          rope_theta;
+    int32_t         rope_style;
+    int32_t         reserved;        /* 0 */
+} kdn_compose_req;
+
+/* Launch shape of the tile pipeline.  0 in a field keeps the built-in default.  tile_bytes: bf16
+ * bytes moved per pipeline slot (multiple of 128); stages: slots per CTA; ctas_per_sm: persistent
+ * CTAs per SM.  Settings that do not fit in shared memory are rejected with KDN_E_UNSUPPORTED. */
+typedef struct {
+    int32_t tile_bytes;
+    int32_t stages;
+    int32_t ctas_per_sm;
+    int32_t reserved;   /* 0 */
+} kdn_tuning;
+
+/* Create a context on CUDA device `device` (makes it current for the call).  KDN_E_CUDA when no
+ * such device can be used. */
+kdn_status kdn_create(kdn_ctx **out, int device);
+/* Wait for the context's own streams and free its scratch.  NULL is allowed. */
+void kdn_destroy(kdn_ctx *ctx);
+
+/* Register a pool (Sec. 3.2: the engine's paged memory); *pool_id is the handle for later calls. */
+kdn_status kdn_pool_register(kdn_ctx *ctx, const kdn_pool_desc *pool, int *pool_id);
+
+/* Bytes of one chunk of n_tokens tokens for this pool's shape; 0 if the codec cannot hold the
+ * shape.  Pure host arithmetic; reads only the shape fields of *pool. */
+size_t kdn_chunk_bytes(const kdn_pool_desc *pool, int32_t n_tokens, int32_t codec);
+
+/* Host-side argument check shared by kdn_store / kdn_retrieve (same status they would return);
+ * touches no device.  Pointers are only compared and tested for alignment, never dereferenced,
+ * except the host arrays ops[]. */
+kdn_status kdn_validate_xfer(const kdn_pool_desc *pool, const kdn_xfer_op *ops, int n_ops);
+/* Same for kdn_compose; reads reqs[], parts[] and part_dst_pos[]. */
+kdn_status kdn_validate_compose(const kdn_pool_desc *pool, const kdn_compose_req *reqs, int n_reqs);
+
+/* Sec. 3.2 call (i), store: for each op gather the chunk's tokens out of the pool blocks its table
+ * names and write the chunk (int8-coded if chunk.codec says so).  One kernel launch covers the
+ * whole batch.  Source blocks may repeat; chunk buffers of one call must not overlap.
+ * A KDN_MEM_PINNED_HOST chunk is written to a staging slab and copied out on side_stream. */
+kdn_status kdn_store(kdn_ctx *ctx, int pool_id, const kdn_xfer_op *ops, int n_ops,
+                     void *cuda_stream, void *side_stream);
+
+/* Sec. 3.2 call (ii), retrieve, with Sec. 3.1's decompression on the GPU: the inverse of
+ * kdn_store.  Writes exactly the n_tokens addressed token slots of each op; every other byte of
+ * the pool keeps its value.  Destination slots of one call must be pairwise distinct (otherwise
+ * the overlapped slots hold one of the written values, unspecified which).  KDN_MEM_PINNED_HOST
+ * chunks are copied to the device on side_stream (NULL = a stream the context owns), layer range by
+ * layer range through two staging slabs, while the kernel of the previous range runs on
+ * cuda_stream. */
+kdn_status kdn_retrieve(kdn_ctx *ctx, int pool_id, const kdn_xfer_op *ops, int n_ops,
+                        void *cuda_stream, void *side_stream);
+
+/* Sec. 3.1 blending module: compose every request's parts into its blocks; keys of parts whose
+ * part_dst_pos differs from base_pos are re-rotated (see the top of this file).  A part with equal
+ * positions, and every value plane, is written exactly as kdn_retrieve writes it. */
+kdn_status kdn_compose(kdn_ctx *ctx, int pool_id, const kdn_compose_req *reqs, int n_reqs,
+                       void *cuda_stream, void *side_stream);
+
+/* Wait for cuda_stream (and the context's side stream) and return the first error a kernel of this
+ * context recorded since the last call of this function, or KDN_OK. */
+kdn_status kdn_status_sync(kdn_ctx *ctx, void *cuda_stream);
+
+/* Change the launch shape for later calls.  NULL restores the defaults. */
+kdn_status kdn_set_tuning(kdn_ctx *ctx, const kdn_tuning *tuning);
+/* Bytes of each of the two staging slabs used for pinned-host chunks (default 256 MiB, allocated
+ * on first use).  Takes effect at the next pinned-host call; frees slabs already allocated. */
+kdn_status kdn_set_staging_bytes(kdn_ctx *ctx, size_t bytes_per_slab);
+
+/* Kernels this context has launched so far (for accounting; never reset). */
+uint64_t kdn_launch_count(const kdn_ctx *ctx);
+
+/* Static string for a status code. */
+const char *kdn_strerror(kdn_status status);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* KDN_H */

@@ -1,0 +1,192 @@
+"""CPU oracle for the KDN store / retrieve / compose path (test infrastructure).
+
+The arithmetic lives in ``kdn_oracle.c`` (plain scalar C, one loop nest per
+definition).  This module compiles it with gcc on first use and exposes it to
+numpy.  Only tests, the smoke check and the benchmark's CPU-baseline leg may
+import this package; the CUDA library and its Python binding never do.
+
+Array conventions (all host, C-contiguous numpy):
+  pool    uint16 [L][2][n_blocks][block_size][H][D]   bf16 bit patterns, kv 0 = K, 1 = V
+  table   int32  [n_table_blocks]
+  chunk   uint8  [chunk_bytes]  raw: bf16 [L][2][T][H][D];
+                                int8: int8 codes [L][2][T][H][D] then fp32 scales [L][2][T][H*D/64]
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+import subprocess
+import threading
+
+import numpy as np
+
+RAW_BF16 = 0
+INT8_G64 = 1
+GROUP = 64
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_SRC = os.path.join(_HERE, "kdn_oracle.c")
+_LIB = os.path.join(_HERE, "libkdn_oracle.so")
+_lock = threading.Lock()
+_lib = None
+
+
+def build(force: bool = False) -> str:
+    """Compile the oracle (no fast-math, no fused multiply-add contraction)."""
+    if force or not os.path.exists(_LIB) or os.path.getmtime(_LIB) < os.path.getmtime(_SRC):
+        tmp = _LIB + ".%d.tmp" % os.getpid()
+        cmd = ["gcc", "-std=c99", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared",
+               "-Wall", "-Wextra", "-o", tmp, _SRC, "-lm"]
+        subprocess.run(cmd, check=True)
+        os.replace(tmp, _LIB)
+    return _LIB
+
+
+def lib():
+    global _lib
+    with _lock:
+        if _lib is None:
+            L = C.CDLL(build())
+            i32, i64, f64, sz = C.c_int, C.c_int64, C.c_double, C.c_size_t
+            vp = C.c_void_p
+            L.kdn_oracle_bf16_to_f32.restype = C.c_float
+            L.kdn_oracle_bf16_to_f32.argtypes = [C.c_uint16]
+            L.kdn_oracle_f32_to_bf16.restype = C.c_uint16
+            L.kdn_oracle_f32_to_bf16.argtypes = [C.c_float]
+            L.kdn_oracle_f64_to_bf16.restype = C.c_uint16
+            L.kdn_oracle_f64_to_bf16.argtypes = [f64]
+            L.kdn_oracle_chunk_bytes.restype = sz
+            L.kdn_oracle_chunk_bytes.argtypes = [i32, i32, i32, i32, i32]
+            L.kdn_oracle_quant_group.restype = None
+            L.kdn_oracle_quant_group.argtypes = [vp, vp, vp]
+            L.kdn_oracle_dequant.restype = C.c_uint16
+            L.kdn_oracle_dequant.argtypes = [C.c_int8, C.c_float]
+            L.kdn_oracle_rope_angle.restype = f64
+            L.kdn_oracle_rope_angle.argtypes = [i64, f64, i32, i32]
+            L.kdn_oracle_rotate_pair.restype = None
+            L.kdn_oracle_rotate_pair.argtypes = [f64, f64, f64, C.POINTER(f64), C.POINTER(f64)]
+            xfer = [vp, i32, i32, i32, i32, i64, vp, i32, i64, i32, i32, vp]
+            L.kdn_oracle_store.restype = i32
+            L.kdn_oracle_store.argtypes = xfer
+            L.kdn_oracle_retrieve.restype = i32
+            L.kdn_oracle_retrieve.argtypes = xfer
+            L.kdn_oracle_compose.restype = i32
+            L.kdn_oracle_compose.argtypes = [vp, i32, i32, i32, i32, i64, vp, i32, i32,
+                                             vp, vp, vp, vp, vp, f64, vp, vp]
+            _lib = L
+    return _lib
+
+
+def _ptr(a: np.ndarray):
+    return a.ctypes.data_as(C.c_void_p)
+
+
+def _check_pool(pool: np.ndarray):
+    if pool.dtype != np.uint16 or pool.ndim != 6 or pool.shape[1] != 2 or not pool.flags.c_contiguous:
+        raise ValueError("pool must be C-contiguous uint16 [L][2][n_blocks][block_size][H][D]")
+    L, _, nb, bs, H, D = pool.shape
+    return L, H, D, bs, nb
+
+
+def _check_table(table: np.ndarray):
+    if table.dtype != np.int32 or table.ndim != 1 or not table.flags.c_contiguous:
+        raise ValueError("table must be C-contiguous int32 [n_table_blocks]")
+
+
+def chunk_bytes(L: int, H: int, D: int, T: int, codec: int) -> int:
+    return int(lib().kdn_oracle_chunk_bytes(L, H, D, T, codec))
+
+
+def store(pool: np.ndarray, table: np.ndarray, token_offset: int, n_tokens: int, codec: int) -> np.ndarray:
+    """Gather ``n_tokens`` tokens at request positions ``token_offset + t`` into a new chunk."""
+    L, H, D, bs, nb = _check_pool(pool)
+    _check_table(table)
+    chunk = np.zeros(chunk_bytes(L, H, D, n_tokens, codec), dtype=np.uint8)
+    rc = lib().kdn_oracle_store(_ptr(pool), L, H, D, bs, nb, _ptr(table), len(table),
+                                int(token_offset), int(n_tokens), int(codec), _ptr(chunk))
+    if rc:
+        raise ValueError("oracle store: bad arguments (code %d)" % rc)
+    return chunk
+
+
+def retrieve(pool: np.ndarray, table: np.ndarray, token_offset: int, n_tokens: int, codec: int,
+             chunk: np.ndarray) -> None:
+    """Scatter ``chunk`` into ``pool`` in place at request positions ``token_offset + t``."""
+    L, H, D, bs, nb = _check_pool(pool)
+    _check_table(table)
+    if chunk.dtype != np.uint8 or chunk.size != chunk_bytes(L, H, D, n_tokens, codec):
+        raise ValueError("chunk has the wrong size for this shape / codec")
+    chunk = np.ascontiguousarray(chunk)
+    rc = lib().kdn_oracle_retrieve(_ptr(pool), L, H, D, bs, nb, _ptr(table), len(table),
+                                   int(token_offset), int(n_tokens), int(codec), _ptr(chunk))
+    if rc:
+        raise ValueError("oracle retrieve: bad arguments (code %d)" % rc)
+
+
+def compose(pool: np.ndarray, table: np.ndarray, parts, theta: float, want_ref: bool = False):
+    """Compose ``parts`` into ``pool`` in place.
+
+    ``parts`` is a list of ``(chunk, n_tokens, codec, base_pos, dst_pos)``.
+    With ``want_ref`` returns ``(kref, kmag)``: fp64 ``[L][n_table*bs][H][D]`` arrays holding the
+    unrounded key result (NaN where no part wrote) and ``|u| + |w|`` of each rotated pair.
+    """
+    L, H, D, bs, nb = _check_pool(pool)
+    _check_table(table)
+    n = len(parts)
+    chunks = [np.ascontiguousarray(p[0]) for p in parts]
+    for ch, p in zip(chunks, parts):
+        if ch.dtype != np.uint8 or ch.size != chunk_bytes(L, H, D, p[1], p[2]):
+            raise ValueError("part chunk has the wrong size for this shape / codec")
+    ptrs = (C.c_void_p * max(n, 1))(*[c.ctypes.data for c in chunks])
+    Ts = np.array([p[1] for p in parts], dtype=np.int32)
+    codecs = np.array([p[2] for p in parts], dtype=np.int32)
+    base = np.array([p[3] for p in parts], dtype=np.int64)
+    dst = np.array([p[4] for p in parts], dtype=np.int64)
+    kref = kmag = None
+    if want_ref:
+        kref = np.full((L, len(table) * bs, H, D), np.nan, dtype=np.float64)
+        kmag = np.zeros((L, len(table) * bs, H, D), dtype=np.float64)
+    rc = lib().kdn_oracle_compose(_ptr(pool), L, H, D, bs, nb, _ptr(table), len(table), n,
+                                  C.cast(ptrs, C.c_void_p), _ptr(Ts), _ptr(codecs), _ptr(base), _ptr(dst),
+                                  float(theta), _ptr(kref) if want_ref else None,
+                                  _ptr(kmag) if want_ref else None)
+    if rc:
+        raise ValueError("oracle compose: bad arguments (code %d)" % rc)
+    return (kref, kmag) if want_ref else None
+
+
+def quant_group(x_bf16: np.ndarray):
+    """Encode one group of 64 bf16 bit patterns -> (int8 codes [64], fp32 scale)."""
+    x = np.ascontiguousarray(x_bf16, dtype=np.uint16)
+    if x.shape != (GROUP,):
+        raise ValueError("a group is 64 values")
+    q = np.zeros(GROUP, dtype=np.int8)
+    s = np.zeros(1, dtype=np.float32)
+    lib().kdn_oracle_quant_group(_ptr(x), _ptr(q), _ptr(s))
+    return q, s[0]
+
+
+def dequant(q: int, scale) -> int:
+    return int(lib().kdn_oracle_dequant(int(q), float(np.float32(scale))))
+
+
+def f32_to_bf16(f) -> int:
+    return int(lib().kdn_oracle_f32_to_bf16(float(np.float32(f))))
+
+
+def f64_to_bf16(x: float) -> int:
+    return int(lib().kdn_oracle_f64_to_bf16(float(x)))
+
+
+def bf16_to_f32(b: int) -> float:
+    return float(lib().kdn_oracle_bf16_to_f32(int(b)))
+
+
+def rope_angle(delta: int, theta: float, i: int, D: int) -> float:
+    return float(lib().kdn_oracle_rope_angle(int(delta), float(theta), int(i), int(D)))
+
+
+def rotate_pair(u: float, w: float, phi: float):
+    a, b = C.c_double(), C.c_double()
+    lib().kdn_oracle_rotate_pair(float(u), float(w), float(phi), C.byref(a), C.byref(b))
+    return a.value, b.value

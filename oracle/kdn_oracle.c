@@ -1,0 +1,396 @@
+/*
+ * CPU oracle for the KV-cache store / retrieve / compose path of a Knowledge
+ * Delivery Network (paper Sec. 3.1: storage, delivery and blending modules;
+ * Sec. 3.2 "Interface with LLM serving engines": the two calls (i) store and
+ * (ii) retrieve).
+ *
+ * THIS FILE IS TEST INFRASTRUCTURE.  It is a plain, slow, scalar statement of
+ * what the path computes.  It shares no code, header, table or constant with
+ * the CUDA library, and the CUDA library never calls it.  Only the tests, the
+ * smoke check and the benchmark's CPU-baseline leg may load it.
+ *
+ * The paper states the problem (store KV caches apart from the engine's paged
+ * memory, deliver them compressed and decompress on the GPU, compose several
+ * of them in one query's context, reuse a chunk at another position) but
+ * prints no layout, codec, formula or number for it.  The concrete readings
+ * taken here, each one stated where it is used:
+ *
+ *   R1  paged pool   per layer l and kv in {0 = K, 1 = V}:
+ *                    pool[l][kv][block][slot][head][d], bf16
+ *                    (Sec. 3.2 names "paged memory" only).
+ *   R2  chunk        raw : bf16  chunk[l][kv][t][head][d]
+ *                    int8: int8  codes[l][kv][t][head][d] followed by
+ *                          fp32  scales[l][kv][t][head*D/64 + g]
+ *                    no header, no padding, little endian.
+ *   R3  mapping      request position p sits in block table[p / bs], slot
+ *                    p % bs; chunk token t of an op with token_offset s is
+ *                    position p = s + t.
+ *   R4  int8 codec   group = 64 consecutive d of one (l, kv, t, head);
+ *                    a = max|x|; scale = a / 127 (fp32 divide);
+ *                    scale below FLT_MIN (zero or subnormal) -> scale 0, codes 0;
+ *                    else inv = 127 / a (fp32 divide),
+ *                    q = clamp(round_half_even(x * inv), -127, 127), the
+ *                    product being one fp32 multiply.
+ *   R5  decode       x^ = bf16_rne((float)q * scale), one fp32 multiply.
+ *   R6  re-rotation  stored keys carry rotary position embedding at absolute
+ *                    positions base_pos + t (what an engine's pool holds), so
+ *                    reuse at dst_pos (Sec. 3.2 "KV-cache blending": a
+ *                    segment's cache reused at different positions) rotates
+ *                    every pair (k[i], k[i + D/2]) of every head by
+ *                    phi_i = delta * theta^(-2 i / D), delta = dst_pos - base_pos,
+ *                    evaluated in fp64.  Values are copied.  delta == 0 keys
+ *                    take the decode path unchanged.
+ *
+ * Parity pins (tests/test_oracle_*.py, all CPU): brute force against an
+ * independent index-by-index formulation on tiny shapes; contiguous table
+ * reduces store to a slice copy; store-then-retrieve identity on raw bf16 for
+ * all bit-pattern classes; placement invariance; hand-worked codec groups
+ * (tests/golden/); |x - q*scale| <= scale/2 bound; a second round-half-even
+ * formulation; exhaustive-class bf16 rounding against torch; rotation
+ * composition R(a)R(b) = R(a+b), norm preservation, quarter/half turns, and
+ * rotary-from-scratch at p then re-rotation by delta equals rotary at p+delta.
+ * End-to-end values: parity unpinned by the paper (it prints no value on this
+ * path); every pin above comes from the definitions and from mathematics.
+ */
+#include <float.h>
+#include <math.h>
+#include <stddef.h>
+#include <stdint.h>
+#include <string.h>
+
+#define KDN_ORACLE_RAW_BF16 0
+#define KDN_ORACLE_INT8_G64 1
+#define KDN_ORACLE_GROUP 64
+
+/* ---------------------------------------------------------------- bf16 -- */
+
+float kdn_oracle_bf16_to_f32(uint16_t b)
+{
+    uint32_t u = (uint32_t)b << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return f;
+}
+
+/* fp32 -> bf16, round to nearest, ties to even.  NaN stays NaN (quiet). */
+uint16_t kdn_oracle_f32_to_bf16(float f)
+{
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    if ((u & 0x7fffffffu) > 0x7f800000u)          /* NaN */
+        return (uint16_t)((u >> 16) | 0x0040u);
+    uint32_t keep = u >> 16;
+    uint32_t rest = u & 0xffffu;
+    if (rest > 0x8000u || (rest == 0x8000u && (keep & 1u)))
+        keep += 1u;                                /* may carry into inf: correct */
+    return (uint16_t)keep;
+}
+
+/* fp64 -> bf16, round to nearest even in ONE rounding (no trip through fp32):
+ * take the bf16 at or below |x| and its upper neighbour, keep the nearer one,
+ * the even one on a tie. */
+uint16_t kdn_oracle_f64_to_bf16(double x)
+{
+    if (x != x) return 0x7fc0u;
+    uint16_t sign = (uint16_t)(signbit(x) ? 0x8000u : 0u);
+    double a = fabs(x);
+    if (isinf(a)) return (uint16_t)(sign | 0x7f80u);
+    /* largest bf16 magnitude <= a, by bisection over the 0..0x7f80 codes
+     * (bf16 magnitudes are monotone in their bit pattern) */
+    uint32_t lo = 0, hi = 0x7f80u;                 /* value(lo) <= a < value(hi)=inf */
+    while (hi - lo > 1u) {
+        uint32_t mid = (lo + hi) / 2u;
+        if ((double)kdn_oracle_bf16_to_f32((uint16_t)mid) <= a) lo = mid; else hi = mid;
+    }
+    double vlo = (double)kdn_oracle_bf16_to_f32((uint16_t)lo);
+    if (hi == 0x7f80u) {
+        /* above the largest finite bf16: round to inf only past the half-way
+         * point to the next (unrepresentable) step 2^128 */
+        double step = ldexp(1.0, 127 - 7);
+        double half = vlo + step / 2.0;
+        uint32_t r = (a > half || (a == half && (lo & 1u))) ? hi : lo;
+        return (uint16_t)(sign | r);
+    }
+    double vhi = (double)kdn_oracle_bf16_to_f32((uint16_t)hi);
+    double dlo = a - vlo, dhi = vhi - a;           /* exact: all three are close doubles */
+    uint32_t r;
+    if (dlo < dhi) r = lo; else if (dhi < dlo) r = hi; else r = (lo & 1u) ? hi : lo;
+    return (uint16_t)(sign | r);
+}
+
+/* --------------------------------------------------------------- sizes -- */
+
+/* R2: bytes of one chunk of T tokens.  0 when the codec cannot hold the shape. */
+size_t kdn_oracle_chunk_bytes(int L, int H, int D, int T, int codec)
+{
+    if (L <= 0 || H <= 0 || D <= 0 || T < 0) return 0;
+    size_t elems = (size_t)L * 2u * (size_t)T * (size_t)H * (size_t)D;
+    if (codec == KDN_ORACLE_RAW_BF16) return 2u * elems;
+    if (codec == KDN_ORACLE_INT8_G64) {
+        if (D % KDN_ORACLE_GROUP) return 0;
+        return elems + 4u * (elems / KDN_ORACLE_GROUP);
+    }
+    return 0;
+}
+
+/* ------------------------------------------------------------ int8 codec -- */
+
+/* R4: encode one group of 64 bf16 values. */
+void kdn_oracle_quant_group(const uint16_t *x_bf16, int8_t *q, float *scale_out)
+{
+    float a = 0.0f;
+    for (int i = 0; i < KDN_ORACLE_GROUP; ++i) {
+        float v = fabsf(kdn_oracle_bf16_to_f32(x_bf16[i]));
+        if (v > a) a = v;
+    }
+    volatile float scale = a / 127.0f;             /* volatile: one fp32 divide, stored as fp32 */
+    if (!(scale >= FLT_MIN)) {
+        *scale_out = 0.0f;
+        for (int i = 0; i < KDN_ORACLE_GROUP; ++i) q[i] = 0;
+        return;
+    }
+    volatile float inv = 127.0f / a;
+    for (int i = 0; i < KDN_ORACLE_GROUP; ++i) {
+        volatile float prod = kdn_oracle_bf16_to_f32(x_bf16[i]) * inv;   /* one fp32 multiply */
+        float r = rintf(prod);                     /* default rounding mode: ties to even */
+        if (r > 127.0f) r = 127.0f;
+        if (r < -127.0f) r = -127.0f;
+        q[i] = (int8_t)(int)r;
+    }
+    *scale_out = scale;
+}
+
+/* R5: decode one code. */
+uint16_t kdn_oracle_dequant(int8_t q, float scale)
+{
+    volatile float prod = (float)q * scale;
+    return kdn_oracle_f32_to_bf16(prod);
+}
+
+/* ------------------------------------------------------------- rotation -- */
+
+/* R6: angle of frequency index i (0 <= i < D/2) for a position shift delta. */
+double kdn_oracle_rope_angle(int64_t delta, double theta, int i, int D)
+{
+    double inv_freq = pow(theta, -2.0 * (double)i / (double)D);
+    return (double)delta * inv_freq;
+}
+
+/* R6: rotate the pair (u, w) = (k[i], k[i + D/2]) by phi. */
+void kdn_oracle_rotate_pair(double u, double w, double phi, double *u_out, double *w_out)
+{
+    double c = cos(phi), s = sin(phi);
+    *u_out = u * c - w * s;
+    *w_out = w * c + u * s;
+}
+
+/* ------------------------------------------------------- index helpers -- */
+
+typedef struct {
+    int L, H, D, bs;
+    int64_t nb;
+} shape_t;
+
+/* R1: element offset of pool[l][kv][block][slot][h][d]. */
+static size_t pool_index(const shape_t *s, int l, int kv, int64_t block, int slot, int h, int d)
+{
+    size_t i = (size_t)l;
+    i = i * 2u + (size_t)kv;
+    i = i * (size_t)s->nb + (size_t)block;
+    i = i * (size_t)s->bs + (size_t)slot;
+    i = i * (size_t)s->H + (size_t)h;
+    i = i * (size_t)s->D + (size_t)d;
+    return i;
+}
+
+/* R2: element offset of chunk[l][kv][t][h][d] for a chunk of T tokens. */
+static size_t chunk_index(const shape_t *s, int T, int l, int kv, int t, int h, int d)
+{
+    size_t i = (size_t)l;
+    i = i * 2u + (size_t)kv;
+    i = i * (size_t)T + (size_t)t;
+    i = i * (size_t)s->H + (size_t)h;
+    i = i * (size_t)s->D + (size_t)d;
+    return i;
+}
+
+static int check_args(const shape_t *s, const int32_t *table, int n_table, int64_t off, int T, int codec)
+{
+    if (s->L <= 0 || s->H <= 0 || s->D <= 0 || s->bs <= 0 || s->nb <= 0) return 1;
+    if (T < 0 || off < 0 || n_table < 0) return 1;
+    if (off + (int64_t)T > (int64_t)n_table * (int64_t)s->bs) return 2;
+    if (codec != KDN_ORACLE_RAW_BF16 && codec != KDN_ORACLE_INT8_G64) return 3;
+    if (codec == KDN_ORACLE_INT8_G64 && s->D % KDN_ORACLE_GROUP) return 3;
+    for (int64_t p = off; p < off + T; ++p) {
+        int32_t b = table[p / s->bs];
+        if (b < 0 || (int64_t)b >= s->nb) return 4;
+    }
+    return 0;
+}
+
+/* ---------------------------------------------------------------- store -- */
+
+/* Sec. 3.2 call (i): gather T tokens starting at request position `off` out
+ * of the paged pool (R1, R3) into one chunk (R2), optionally int8-coded (R4).
+ * Returns 0, or a small positive code for bad arguments (nothing written). */
+int kdn_oracle_store(const uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
+                     const int32_t *table, int n_table, int64_t off, int T, int codec,
+                     uint8_t *chunk)
+{
+    shape_t s = { L, H, D, bs, nb };
+    int rc = check_args(&s, table, n_table, off, T, codec);
+    if (rc) return rc;
+    size_t elems = (size_t)L * 2u * (size_t)T * (size_t)H * (size_t)D;
+    uint16_t *raw = (uint16_t *)chunk;
+    int8_t *codes = (int8_t *)chunk;
+    float *scales = (float *)(chunk + elems);
+    for (int l = 0; l < L; ++l)
+        for (int kv = 0; kv < 2; ++kv)
+            for (int t = 0; t < T; ++t) {
+                int64_t p = off + t;
+                int64_t block = table[p / bs];
+                int slot = (int)(p % bs);
+                for (int h = 0; h < H; ++h) {
+                    if (codec == KDN_ORACLE_RAW_BF16) {
+                        for (int d = 0; d < D; ++d)
+                            raw[chunk_index(&s, T, l, kv, t, h, d)] =
+                                pool[pool_index(&s, l, kv, block, slot, h, d)];
+                    } else {
+                        for (int g = 0; g < D / KDN_ORACLE_GROUP; ++g) {
+                            size_t src = pool_index(&s, l, kv, block, slot, h, g * KDN_ORACLE_GROUP);
+                            size_t dst = chunk_index(&s, T, l, kv, t, h, g * KDN_ORACLE_GROUP);
+                            kdn_oracle_quant_group(pool + src, codes + dst, scales + dst / KDN_ORACLE_GROUP);
+                        }
+                    }
+                }
+            }
+    return 0;
+}
+
+/* ------------------------------------------------------------- retrieve -- */
+
+/* Sec. 3.2 call (ii) with Sec. 3.1's "decompresses them in GPU": scatter a
+ * chunk back into the pool blocks the table names, decoding int8 (R5).  Only
+ * the T addressed token slots are written. */
+int kdn_oracle_retrieve(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
+                        const int32_t *table, int n_table, int64_t off, int T, int codec,
+                        const uint8_t *chunk)
+{
+    shape_t s = { L, H, D, bs, nb };
+    int rc = check_args(&s, table, n_table, off, T, codec);
+    if (rc) return rc;
+    size_t elems = (size_t)L * 2u * (size_t)T * (size_t)H * (size_t)D;
+    const uint16_t *raw = (const uint16_t *)chunk;
+    const int8_t *codes = (const int8_t *)chunk;
+    const float *scales = (const float *)(chunk + elems);
+    for (int l = 0; l < L; ++l)
+        for (int kv = 0; kv < 2; ++kv)
+            for (int t = 0; t < T; ++t) {
+                int64_t p = off + t;
+                int64_t block = table[p / bs];
+                int slot = (int)(p % bs);
+                for (int h = 0; h < H; ++h)
+                    for (int d = 0; d < D; ++d) {
+                        size_t c = chunk_index(&s, T, l, kv, t, h, d);
+                        size_t o = pool_index(&s, l, kv, block, slot, h, d);
+                        pool[o] = (codec == KDN_ORACLE_RAW_BF16)
+                                      ? raw[c]
+                                      : kdn_oracle_dequant(codes[c], scales[c / KDN_ORACLE_GROUP]);
+                    }
+            }
+    return 0;
+}
+
+/* -------------------------------------------------------------- compose -- */
+
+/* Sec. 3.1 blending module / Sec. 3.2 "KV-cache blending": place n_parts
+ * chunks into one request's blocks, part j at positions dst_pos[j] + t, and
+ * re-rotate the keys of every part whose delta = dst_pos - base_pos is not
+ * zero (R6).  Values, and keys with delta == 0, are exactly a retrieve.
+ *
+ * For rotated keys the result is computed in fp64 from the stored value (raw
+ * bf16, or the UNROUNDED product q * scale for int8) and written to the pool
+ * rounded once to bf16.  When kref / kmag are not NULL they receive, for every
+ * key element of every part (rotated or not), the fp64 result and |u| + |w| of
+ * its pair, laid out [l][position][h][d] over the n_table * bs request
+ * positions; entries no part covers are left as the caller set them.
+ */
+int kdn_oracle_compose(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
+                       const int32_t *table, int n_table, int n_parts,
+                       const uint8_t *const *chunks, const int32_t *part_T, const int32_t *part_codec,
+                       const int64_t *base_pos, const int64_t *dst_pos, double theta,
+                       double *kref, double *kmag)
+{
+    shape_t s = { L, H, D, bs, nb };
+    if (n_parts < 0) return 1;
+    if (D % 2) return 3;
+    for (int j = 0; j < n_parts; ++j) {
+        int rc = check_args(&s, table, n_table, dst_pos[j], part_T[j], part_codec[j]);
+        if (rc) return rc;
+    }
+    int64_t P = (int64_t)n_table * bs;
+    int half = D / 2;
+    for (int j = 0; j < n_parts; ++j) {
+        int T = part_T[j];
+        int codec = part_codec[j];
+        int64_t delta = dst_pos[j] - base_pos[j];
+        size_t elems = (size_t)L * 2u * (size_t)T * (size_t)H * (size_t)D;
+        const uint16_t *raw = (const uint16_t *)chunks[j];
+        const int8_t *codes = (const int8_t *)chunks[j];
+        const float *scales = (const float *)(chunks[j] + elems);
+        for (int l = 0; l < L; ++l)
+            for (int kv = 0; kv < 2; ++kv)
+                for (int t = 0; t < T; ++t) {
+                    int64_t p = dst_pos[j] + t;
+                    int64_t block = table[p / bs];
+                    int slot = (int)(p % bs);
+                    for (int h = 0; h < H; ++h) {
+                        int rotate = (kv == 0 && delta != 0);
+                        if (!rotate) {
+                            for (int d = 0; d < D; ++d) {
+                                size_t c = chunk_index(&s, T, l, kv, t, h, d);
+                                size_t o = pool_index(&s, l, kv, block, slot, h, d);
+                                pool[o] = (codec == KDN_ORACLE_RAW_BF16)
+                                              ? raw[c]
+                                              : kdn_oracle_dequant(codes[c], scales[c / KDN_ORACLE_GROUP]);
+                                if (kv == 0 && kref) {
+                                    size_t r = (((size_t)l * (size_t)P + (size_t)p) * (size_t)H + (size_t)h) * (size_t)D + (size_t)d;
+                                    kref[r] = (double)kdn_oracle_bf16_to_f32(pool[o]);
+                                    if (kmag) kmag[r] = 0.0;
+                                }
+                            }
+                            continue;
+                        }
+                        for (int i = 0; i < half; ++i) {
+                            size_t cu = chunk_index(&s, T, l, 0, t, h, i);
+                            size_t cw = chunk_index(&s, T, l, 0, t, h, i + half);
+                            double u, w;
+                            if (codec == KDN_ORACLE_RAW_BF16) {
+                                u = (double)kdn_oracle_bf16_to_f32(raw[cu]);
+                                w = (double)kdn_oracle_bf16_to_f32(raw[cw]);
+                            } else {
+                                u = (double)codes[cu] * (double)scales[cu / KDN_ORACLE_GROUP];
+                                w = (double)codes[cw] * (double)scales[cw / KDN_ORACLE_GROUP];
+                            }
+                            double phi = kdn_oracle_rope_angle(delta, theta, i, D);
+                            double u2, w2;
+                            kdn_oracle_rotate_pair(u, w, phi, &u2, &w2);
+                            size_t ou = pool_index(&s, l, 0, block, slot, h, i);
+                            size_t ow = pool_index(&s, l, 0, block, slot, h, i + half);
+                            pool[ou] = kdn_oracle_f64_to_bf16(u2);
+                            pool[ow] = kdn_oracle_f64_to_bf16(w2);
+                            if (kref) {
+                                size_t r = (((size_t)l * (size_t)P + (size_t)p) * (size_t)H + (size_t)h) * (size_t)D;
+                                kref[r + (size_t)i] = u2;
+                                kref[r + (size_t)i + (size_t)half] = w2;
+                                if (kmag) {
+                                    kmag[r + (size_t)i] = fabs(u) + fabs(w);
+                                    kmag[r + (size_t)i + (size_t)half] = fabs(u) + fabs(w);
+                                }
+                            }
+                        }
+                    }
+                }
+    }
+    return 0;
+}
