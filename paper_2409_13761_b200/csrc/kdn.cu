@@ -1,0 +1,653 @@
+// Host side of libkdn: the C ABI declared in include/kdn.h.  Validates arguments, turns ops into
+// 64-byte device records, and launches the tile pipeline of kdn_kernels.cuh on the caller's stream.
+// Paper anchors: Sec. 3.2 "Interface with LLM serving engines" (store / retrieve), Sec. 3.1 (storage,
+// delivery and blending modules).
+#include "kdn.h"
+#include "kdn_kernels.cuh"
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+using namespace kdn;
+
+namespace {
+
+constexpr int kRing = 8;                   // launches that may be queued before the host has to wait
+constexpr int kMaxOpsPerLaunch = 4096;
+constexpr unsigned kMaxTilesPerLaunch = 0x7fff0000u;
+constexpr size_t kDefaultSlabBytes = (size_t)256 << 20;
+
+struct Pool {
+    int L, H, D, bs;
+    long long nb;
+    void **d_k = nullptr;                   // device copies of the per-layer pointer arrays
+    void **d_v = nullptr;
+};
+
+struct RingSlot {
+    DevOp *h_ops = nullptr;                 // pinned
+    DevOp *d_ops = nullptr;
+    RopeParam *h_rope = nullptr;            // pinned
+    RopeParam *d_rope = nullptr;
+    float2 *d_table = nullptr;
+    size_t table_rows_cap = 0;
+    int table_half = 0;
+    cudaEvent_t done = nullptr;
+    bool used = false;
+};
+
+struct HostOp {                             // one op (or one layer range of one) before tiling
+    DevOp op;
+    bool rotate = false;
+    RopeParam rp{};
+};
+
+struct Piece {                              // host <-> slab copies belonging to a staged op
+    unsigned char *host;
+    size_t slab_off;
+    size_t bytes;
+};
+
+}  // namespace
+
+struct kdn_ctx {
+    int device = 0;
+    int sm_count = 0;
+    int smem_optin = 0;
+    std::vector<Pool> pools;
+    RingSlot ring[kRing];
+    unsigned ring_next = 0;
+    int *d_status = nullptr;
+    int *h_status = nullptr;                // pinned
+    cudaStream_t own_side = nullptr;
+    unsigned char *slab[2] = { nullptr, nullptr };
+    size_t slab_bytes = kDefaultSlabBytes;
+    cudaEvent_t slab_free[2] = { nullptr, nullptr };   // last consumer of the slab has finished
+    cudaEvent_t slab_ready[2] = { nullptr, nullptr };  // the slab's producer has finished
+    unsigned slab_next = 0;
+    uint64_t launches = 0;
+    kdn_tuning tuning{};
+};
+
+namespace {
+
+#define KDN_CUDA(call)                                                                  \
+    do {                                                                                \
+        cudaError_t e_ = (call);                                                        \
+        if (e_ != cudaSuccess) return e_ == cudaErrorMemoryAllocation ? KDN_E_NOMEM : KDN_E_CUDA; \
+    } while (0)
+
+bool shape_ok(const kdn_pool_desc *p)
+{
+    return p && p->n_layers > 0 && p->n_kv_heads > 0 && p->head_dim > 0 && p->block_size > 0 && p->n_blocks > 0;
+}
+
+kdn_status check_shape(const kdn_pool_desc *p)
+{
+    if (!shape_ok(p)) return KDN_E_INVAL;
+    if (((long long)p->n_kv_heads * p->head_dim * 2) % 16) return KDN_E_ALIGN;
+    if ((long long)p->n_kv_heads * p->head_dim > (1 << 24) || p->block_size > (1 << 20)) return KDN_E_UNSUPPORTED;
+    return KDN_OK;
+}
+
+kdn_status check_chunk(const kdn_pool_desc *p, const kdn_chunk *c)
+{
+    if (c->n_tokens < 0) return KDN_E_INVAL;
+    if (c->codec != KDN_CODEC_RAW_BF16 && c->codec != KDN_CODEC_INT8_G64) return KDN_E_INVAL;
+    if (c->mem != KDN_MEM_DEVICE && c->mem != KDN_MEM_PINNED_HOST) return KDN_E_INVAL;
+    if (c->codec == KDN_CODEC_INT8_G64 && p->head_dim % 64) return KDN_E_UNSUPPORTED;
+    if (c->bytes != kdn_chunk_bytes(p, c->n_tokens, c->codec)) return KDN_E_SHAPE;
+    if (c->n_tokens > 0) {
+        if (!c->data) return KDN_E_INVAL;
+        if ((uintptr_t)c->data % 16) return KDN_E_ALIGN;
+    }
+    return KDN_OK;
+}
+
+kdn_status check_range(const kdn_pool_desc *p, const int32_t *table, int32_t n_table, int64_t off, int32_t T)
+{
+    if (n_table < 0 || off < 0) return KDN_E_INVAL;
+    if (T > 0 && !table) return KDN_E_INVAL;
+    if (off + (int64_t)T > (int64_t)n_table * p->block_size) return KDN_E_RANGE;
+    return KDN_OK;
+}
+
+unsigned gcd_u(unsigned a, unsigned b) { while (b) { unsigned t = a % b; a = b; b = t; } return a; }
+unsigned lcm_u(unsigned a, unsigned b) { return a / gcd_u(a, b) * b; }
+
+kdn_status ensure_side(kdn_ctx *ctx)
+{
+    if (!ctx->own_side) KDN_CUDA(cudaStreamCreateWithFlags(&ctx->own_side, cudaStreamNonBlocking));
+    return KDN_OK;
+}
+
+kdn_status ensure_slabs(kdn_ctx *ctx)
+{
+    for (int i = 0; i < 2; ++i) {
+        if (!ctx->slab[i]) KDN_CUDA(cudaMalloc((void **)&ctx->slab[i], ctx->slab_bytes));
+        if (!ctx->slab_free[i]) KDN_CUDA(cudaEventCreateWithFlags(&ctx->slab_free[i], cudaEventDisableTiming));
+        if (!ctx->slab_ready[i]) KDN_CUDA(cudaEventCreateWithFlags(&ctx->slab_ready[i], cudaEventDisableTiming));
+    }
+    return KDN_OK;
+}
+
+template <typename K>
+kdn_status launch_kernel(K kernel, int threads, unsigned grid, size_t smem, cudaStream_t stream, const Launch &lp)
+{
+    KDN_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    kernel<<<grid, threads, smem, stream>>>(lp);
+    KDN_CUDA(cudaGetLastError());
+    return KDN_OK;
+}
+
+// Tile one batch of host ops (at most kMaxOpsPerLaunch, all on the device side) and launch it.
+kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *hops, int n, cudaStream_t stream)
+{
+    if (n <= 0) return KDN_OK;
+    bool any_int8 = false, any_rot = false;
+    for (int i = 0; i < n; ++i) {
+        any_int8 |= hops[i].op.codec == KDN_CODEC_INT8_G64;
+        any_rot |= hops[i].rotate;
+    }
+    const bool compute = any_int8 || any_rot;
+    const unsigned row_elems = (unsigned)pool.H * (unsigned)pool.D;
+
+    // tile size: whole 16-byte units; whole 64-element groups with int8; whole head rows with rotation
+    unsigned unit = 8;
+    if (any_int8) unit = lcm_u(unit, 64);
+    if (any_rot) unit = lcm_u(unit, (unsigned)pool.D);
+    int tile_bytes = ctx->tuning.tile_bytes > 0 ? ctx->tuning.tile_bytes : (compute ? 8192 : 16384);
+    unsigned tile_elems = (unsigned)tile_bytes / 2u / unit * unit;
+    if (tile_elems < unit) tile_elems = unit;
+    const unsigned long long block_elems = (unsigned long long)pool.bs * row_elems;
+    if (tile_elems > block_elems) tile_elems = (unsigned)((block_elems + unit - 1) / unit * unit);
+    const unsigned tpb = (unsigned)((block_elems + tile_elems - 1) / tile_elems);
+
+    const unsigned a_bytes = (tile_elems * 2u + 127u) & ~127u;
+    const unsigned b_bytes = compute ? ((tile_elems + 127u) & ~127u) : 0u;
+    const unsigned s_bytes = compute ? ((tile_elems / 16u + 127u) & ~127u) : 0u;
+    const unsigned stage_bytes = a_bytes + b_bytes + s_bytes;
+    int ctas_per_sm = ctx->tuning.ctas_per_sm > 0 ? ctx->tuning.ctas_per_sm : 2;
+    int stages = ctx->tuning.stages > 0 ? ctx->tuning.stages : (compute ? 8 : 6);
+    if (stages > kMaxStages) stages = kMaxStages;
+    if (stages < kStoreLag + 2) stages = kStoreLag + 2;
+    const size_t smem_limit = (size_t)ctx->smem_optin;
+    if (ctx->tuning.stages <= 0)
+        while (stages > kStoreLag + 2 && smem_bytes(stages, stage_bytes) * (size_t)ctas_per_sm > smem_limit - 1024u * (size_t)ctas_per_sm)
+            --stages;
+    const size_t smem = smem_bytes(stages, stage_bytes);
+    if (smem > smem_limit) return KDN_E_UNSUPPORTED;
+
+    RingSlot &slot = ctx->ring[ctx->ring_next++ % kRing];
+    if (slot.used) KDN_CUDA(cudaEventSynchronize(slot.done));
+
+    unsigned long long tiles = 0;
+    int n_rope = 0;
+    for (int i = 0; i < n; ++i) {
+        DevOp op = hops[i].op;
+        op.tile_begin = (unsigned)tiles;
+        op.rope = -1;
+        if (hops[i].rotate) {
+            slot.h_rope[n_rope] = hops[i].rp;
+            op.rope = n_rope++;
+        }
+        slot.h_ops[i] = op;
+        tiles += (unsigned long long)op.nl * 2ull * (unsigned long long)op.nblk * tpb;
+        if (tiles > kMaxTilesPerLaunch) return KDN_E_UNSUPPORTED;
+    }
+    if (tiles == 0) return KDN_OK;
+
+    KDN_CUDA(cudaMemcpyAsync(slot.d_ops, slot.h_ops, sizeof(DevOp) * (size_t)n, cudaMemcpyHostToDevice, stream));
+    const int half = pool.D / 2;
+    if (n_rope) {
+        if (slot.table_rows_cap < (size_t)n_rope || slot.table_half != half) {
+            KDN_CUDA(cudaEventSynchronize(slot.done));
+            if (slot.d_table) KDN_CUDA(cudaFree(slot.d_table));
+            slot.d_table = nullptr;
+            size_t rows = (size_t)n_rope < 64 ? 64 : (size_t)n_rope;
+            KDN_CUDA(cudaMalloc((void **)&slot.d_table, rows * (size_t)half * sizeof(float2)));
+            slot.table_rows_cap = rows;
+            slot.table_half = half;
+        }
+        KDN_CUDA(cudaMemcpyAsync(slot.d_rope, slot.h_rope, sizeof(RopeParam) * (size_t)n_rope, cudaMemcpyHostToDevice, stream));
+        const long long total = (long long)n_rope * half;
+        kdn_rope_table_kernel<<<(unsigned)((total + 127) / 128), 128, 0, stream>>>(slot.d_rope, n_rope, pool.D, slot.d_table);
+        KDN_CUDA(cudaGetLastError());
+        ctx->launches++;
+    }
+
+    Launch lp{};
+    lp.ops = slot.d_ops;
+    lp.n_ops = n;
+    lp.n_tiles = (unsigned)tiles;
+    lp.k_layers = pool.d_k;
+    lp.v_layers = pool.d_v;
+    lp.n_blocks = pool.nb;
+    lp.bs = pool.bs;
+    lp.D = pool.D;
+    lp.row_elems = row_elems;
+    lp.tile_elems = tile_elems;
+    lp.tpb = tpb;
+    lp.rope = slot.d_table;
+    lp.status = ctx->d_status;
+    lp.stages = stages;
+    lp.stage_bytes = stage_bytes;
+    lp.off_b = a_bytes;
+    lp.off_s = a_bytes + b_bytes;
+
+    unsigned long long want = (unsigned long long)ctx->sm_count * (unsigned)ctas_per_sm;
+    const unsigned grid = (unsigned)(tiles < want ? tiles : want);
+    kdn_status st;
+    if (compute) {
+        if (OP == OP_STORE) st = launch_kernel(kdn_store_kernel<true>, kThreadsCompute, grid, smem, stream, lp);
+        else if (OP == OP_RETRIEVE) st = launch_kernel(kdn_retrieve_kernel<true>, kThreadsCompute, grid, smem, stream, lp);
+        else st = launch_kernel(kdn_compose_kernel<true>, kThreadsCompute, grid, smem, stream, lp);
+    } else {
+        if (OP == OP_STORE) st = launch_kernel(kdn_store_kernel<false>, kThreadsCopy, grid, smem, stream, lp);
+        else if (OP == OP_RETRIEVE) st = launch_kernel(kdn_retrieve_kernel<false>, kThreadsCopy, grid, smem, stream, lp);
+        else st = launch_kernel(kdn_compose_kernel<false>, kThreadsCopy, grid, smem, stream, lp);
+    }
+    if (st != KDN_OK) return st;
+    ctx->launches++;
+    KDN_CUDA(cudaEventRecord(slot.done, stream));
+    slot.used = true;
+    return KDN_OK;
+}
+
+kdn_status launch_all(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<HostOp> &hops, cudaStream_t stream)
+{
+    for (size_t i = 0; i < hops.size(); i += kMaxOpsPerLaunch) {
+        size_t n = hops.size() - i < (size_t)kMaxOpsPerLaunch ? hops.size() - i : (size_t)kMaxOpsPerLaunch;
+        kdn_status st = launch_batch(ctx, pool, OP, hops.data() + i, (int)n, stream);
+        if (st != KDN_OK) return st;
+    }
+    return KDN_OK;
+}
+
+// The device record of an op that covers all layers of a device-resident chunk.
+HostOp make_host_op(const Pool &pool, const int32_t *table, int64_t off, const kdn_chunk &c)
+{
+    HostOp h;
+    std::memset(&h.op, 0, sizeof h.op);
+    h.op.table = table;
+    h.op.data = (unsigned char *)c.data;
+    h.op.off = off;
+    h.op.T = c.n_tokens;
+    h.op.codec = c.codec;
+    h.op.j0 = (int)(off / pool.bs);
+    h.op.nblk = c.n_tokens > 0 ? (int)((off + c.n_tokens - 1) / pool.bs - off / pool.bs + 1) : 0;
+    h.op.rope = -1;
+    h.op.l0 = 0;
+    h.op.nl = pool.L;
+    return h;
+}
+
+// Ops whose chunk lives in pinned host memory go through the two staging slabs in layer ranges:
+//   retrieve / compose: side stream copies host -> slab, main stream runs the kernel on the slab;
+//   store:              main stream runs the kernel into the slab, side stream copies slab -> host.
+// While one slab is being copied the kernel works on the other.
+kdn_status run_staged(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<HostOp> &hops,
+                      cudaStream_t stream, cudaStream_t side)
+{
+    kdn_status st = ensure_slabs(ctx);
+    if (st != KDN_OK) return st;
+    const size_t row = (size_t)pool.H * pool.D;
+    std::vector<HostOp> batch;
+    std::vector<Piece> pieces;
+    size_t used = 0;
+
+    auto flush = [&]() -> kdn_status {
+        if (batch.empty()) return KDN_OK;
+        const unsigned s = ctx->slab_next++ & 1u;
+        if (OP == OP_STORE) {
+            KDN_CUDA(cudaStreamWaitEvent(stream, ctx->slab_free[s], 0));
+            kdn_status r = launch_all(ctx, pool, OP, batch, stream);
+            if (r != KDN_OK) return r;
+            KDN_CUDA(cudaEventRecord(ctx->slab_ready[s], stream));
+            KDN_CUDA(cudaStreamWaitEvent(side, ctx->slab_ready[s], 0));
+            for (const Piece &p : pieces)
+                KDN_CUDA(cudaMemcpyAsync(p.host, ctx->slab[s] + p.slab_off, p.bytes, cudaMemcpyDeviceToHost, side));
+            KDN_CUDA(cudaEventRecord(ctx->slab_free[s], side));
+        } else {
+            KDN_CUDA(cudaStreamWaitEvent(side, ctx->slab_free[s], 0));
+            for (const Piece &p : pieces)
+                KDN_CUDA(cudaMemcpyAsync(ctx->slab[s] + p.slab_off, p.host, p.bytes, cudaMemcpyHostToDevice, side));
+            KDN_CUDA(cudaEventRecord(ctx->slab_ready[s], side));
+            KDN_CUDA(cudaStreamWaitEvent(stream, ctx->slab_ready[s], 0));
+            kdn_status r = launch_all(ctx, pool, OP, batch, stream);
+            if (r != KDN_OK) return r;
+            KDN_CUDA(cudaEventRecord(ctx->slab_free[s], stream));
+        }
+        batch.clear();
+        pieces.clear();
+        used = 0;
+        return KDN_OK;
+    };
+
+    for (const HostOp &h : hops) {
+        const size_t T = (size_t)h.op.T;
+        if (T == 0) continue;
+        const bool int8 = h.op.codec == KDN_CODEC_INT8_G64;
+        const size_t codes_per_layer = 2 * T * row * (int8 ? 1 : 2);
+        const size_t scales_per_layer = int8 ? 2 * T * (row / 64) * 4 : 0;
+        const size_t per_layer = ((codes_per_layer + 255) & ~(size_t)255) + ((scales_per_layer + 255) & ~(size_t)255);
+        if (per_layer > ctx->slab_bytes) return KDN_E_UNSUPPORTED;
+        unsigned char *host = h.op.data;
+        const size_t host_codes_total = (size_t)pool.L * codes_per_layer;
+        int l = 0;
+        while (l < pool.L) {
+            size_t room = ctx->slab_bytes - used;
+            if (room < per_layer) {
+                st = flush();
+                if (st != KDN_OK) return st;
+                room = ctx->slab_bytes;
+            }
+            int nl = (int)(room / per_layer);
+            if (nl > pool.L - l) nl = pool.L - l;
+            // a piece is laid out exactly like a chunk of nl layers: codes, then scales
+            const size_t base = used;
+            const size_t cbytes = (size_t)nl * codes_per_layer;
+            const size_t sbytes = (size_t)nl * scales_per_layer;
+            HostOp sub = h;
+            sub.op.l0 = l;
+            sub.op.nl = nl;
+            const unsigned s = ctx->slab_next & 1u;
+            sub.op.data = ctx->slab[s] + base;
+            pieces.push_back(Piece{ host + (size_t)l * codes_per_layer, base, cbytes });
+            if (sbytes) pieces.push_back(Piece{ host + host_codes_total + (size_t)l * scales_per_layer, base + cbytes, sbytes });
+            batch.push_back(sub);
+            used = (base + cbytes + sbytes + 255) & ~(size_t)255;
+            l += nl;
+        }
+    }
+    return flush();
+}
+
+kdn_status run_ops(kdn_ctx *ctx, int pool_id, int OP, std::vector<HostOp> &dev_ops, std::vector<HostOp> &host_ops,
+                   void *cuda_stream, void *side_stream)
+{
+    const Pool &pool = ctx->pools[(size_t)pool_id];
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    kdn_status st = launch_all(ctx, pool, OP, dev_ops, stream);
+    if (st != KDN_OK) return st;
+    if (!host_ops.empty()) {
+        cudaStream_t side = (cudaStream_t)side_stream;
+        if (!side) {
+            st = ensure_side(ctx);
+            if (st != KDN_OK) return st;
+            side = ctx->own_side;
+        }
+        st = run_staged(ctx, pool, OP, host_ops, stream, side);
+    }
+    return st;
+}
+
+kdn_pool_desc shape_of(const Pool &p)
+{
+    kdn_pool_desc d{};
+    d.n_layers = p.L; d.n_kv_heads = p.H; d.head_dim = p.D; d.block_size = p.bs; d.n_blocks = p.nb;
+    return d;
+}
+
+kdn_status xfer(kdn_ctx *ctx, int pool_id, int OP, const kdn_xfer_op *ops, int n_ops, void *cuda_stream, void *side_stream)
+{
+    if (!ctx || pool_id < 0 || (size_t)pool_id >= ctx->pools.size()) return KDN_E_INVAL;
+    const Pool &pool = ctx->pools[(size_t)pool_id];
+    const kdn_pool_desc shape = shape_of(pool);
+    kdn_status st = kdn_validate_xfer(&shape, ops, n_ops);
+    if (st != KDN_OK) return st;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return KDN_E_CUDA;
+    std::vector<HostOp> dev_ops, host_ops;
+    for (int i = 0; i < n_ops; ++i) {
+        if (ops[i].chunk.n_tokens == 0) continue;
+        HostOp h = make_host_op(pool, ops[i].block_table, ops[i].token_offset, ops[i].chunk);
+        (ops[i].chunk.mem == KDN_MEM_PINNED_HOST ? host_ops : dev_ops).push_back(h);
+    }
+    return run_ops(ctx, pool_id, OP, dev_ops, host_ops, cuda_stream, side_stream);
+}
+
+}  // namespace
+
+extern "C" {
+
+size_t kdn_chunk_bytes(const kdn_pool_desc *pool, int32_t n_tokens, int32_t codec)
+{
+    if (!shape_ok(pool) || n_tokens < 0) return 0;
+    const size_t elems = (size_t)pool->n_layers * 2u * (size_t)n_tokens * (size_t)pool->n_kv_heads * (size_t)pool->head_dim;
+    if (codec == KDN_CODEC_RAW_BF16) return elems * 2u;
+    if (codec == KDN_CODEC_INT8_G64) return pool->head_dim % 64 ? 0 : elems + elems / 64u * 4u;
+    return 0;
+}
+
+kdn_status kdn_validate_xfer(const kdn_pool_desc *pool, const kdn_xfer_op *ops, int n_ops)
+{
+    kdn_status st = check_shape(pool);
+    if (st != KDN_OK) return st;
+    if (n_ops < 0 || (n_ops > 0 && !ops)) return KDN_E_INVAL;
+    for (int i = 0; i < n_ops; ++i) {
+        st = check_chunk(pool, &ops[i].chunk);
+        if (st != KDN_OK) return st;
+        st = check_range(pool, ops[i].block_table, ops[i].n_table_blocks, ops[i].token_offset, ops[i].chunk.n_tokens);
+        if (st != KDN_OK) return st;
+    }
+    return KDN_OK;
+}
+
+kdn_status kdn_validate_compose(const kdn_pool_desc *pool, const kdn_compose_req *reqs, int n_reqs)
+{
+    kdn_status st = check_shape(pool);
+    if (st != KDN_OK) return st;
+    if (n_reqs < 0 || (n_reqs > 0 && !reqs)) return KDN_E_INVAL;
+    for (int r = 0; r < n_reqs; ++r) {
+        const kdn_compose_req &q = reqs[r];
+        if (q.n_parts < 0 || (q.n_parts > 0 && (!q.parts || !q.part_dst_pos))) return KDN_E_INVAL;
+        if (q.rope_style != 0) return KDN_E_UNSUPPORTED;
+        bool rotates = false;
+        for (int j = 0; j < q.n_parts; ++j) {
+            st = check_chunk(pool, &q.parts[j]);
+            if (st != KDN_OK) return st;
+            st = check_range(pool, q.block_table, q.n_table_blocks, q.part_dst_pos[j], q.parts[j].n_tokens);
+            if (st != KDN_OK) return st;
+            rotates |= q.parts[j].n_tokens > 0 && q.part_dst_pos[j] != q.parts[j].base_pos;
+        }
+        if (rotates) {
+            if (!(q.rope_theta > 0.0) || q.rope_theta != q.rope_theta || q.rope_theta > 1e300) return KDN_E_INVAL;
+            if (pool->head_dim % 16) return KDN_E_UNSUPPORTED;
+        }
+        // parts of one request must not overlap
+        for (int a = 0; a < q.n_parts; ++a)
+            for (int b = a + 1; b < q.n_parts; ++b) {
+                const int64_t a0 = q.part_dst_pos[a], a1 = a0 + q.parts[a].n_tokens;
+                const int64_t b0 = q.part_dst_pos[b], b1 = b0 + q.parts[b].n_tokens;
+                if (a0 < b1 && b0 < a1) return KDN_E_RANGE;
+            }
+    }
+    return KDN_OK;
+}
+
+kdn_status kdn_create(kdn_ctx **out, int device)
+{
+    if (!out) return KDN_E_INVAL;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return KDN_E_CUDA;
+    if (cudaSetDevice(device) != cudaSuccess) return KDN_E_CUDA;
+    kdn_ctx *ctx = new (std::nothrow) kdn_ctx();
+    if (!ctx) return KDN_E_NOMEM;
+    ctx->device = device;
+    kdn_status st = KDN_OK;
+    auto fail = [&](kdn_status s) { kdn_destroy(ctx); return s; };
+    int major = 0;
+    if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess) return fail(KDN_E_CUDA);
+    if (major < 10) return fail(KDN_E_UNSUPPORTED);       // the kernels are built for sm_100a only
+    if (cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return fail(KDN_E_CUDA);
+    if (cudaDeviceGetAttribute(&ctx->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess) return fail(KDN_E_CUDA);
+    if (cudaMalloc((void **)&ctx->d_status, sizeof(int)) != cudaSuccess) return fail(KDN_E_NOMEM);
+    if (cudaMemset(ctx->d_status, 0, sizeof(int)) != cudaSuccess) return fail(KDN_E_CUDA);
+    if (cudaMallocHost((void **)&ctx->h_status, sizeof(int)) != cudaSuccess) return fail(KDN_E_NOMEM);
+    for (int i = 0; i < kRing; ++i) {
+        RingSlot &s = ctx->ring[i];
+        if (cudaMallocHost((void **)&s.h_ops, sizeof(DevOp) * kMaxOpsPerLaunch) != cudaSuccess) return fail(KDN_E_NOMEM);
+        if (cudaMalloc((void **)&s.d_ops, sizeof(DevOp) * kMaxOpsPerLaunch) != cudaSuccess) return fail(KDN_E_NOMEM);
+        if (cudaMallocHost((void **)&s.h_rope, sizeof(RopeParam) * kMaxOpsPerLaunch) != cudaSuccess) return fail(KDN_E_NOMEM);
+        if (cudaMalloc((void **)&s.d_rope, sizeof(RopeParam) * kMaxOpsPerLaunch) != cudaSuccess) return fail(KDN_E_NOMEM);
+        if (cudaEventCreateWithFlags(&s.done, cudaEventDisableTiming) != cudaSuccess) return fail(KDN_E_CUDA);
+    }
+    *out = ctx;
+    return st;
+}
+
+void kdn_destroy(kdn_ctx *ctx)
+{
+    if (!ctx) return;
+    cudaSetDevice(ctx->device);
+    cudaDeviceSynchronize();
+    for (int i = 0; i < kRing; ++i) {
+        RingSlot &s = ctx->ring[i];
+        if (s.h_ops) cudaFreeHost(s.h_ops);
+        if (s.d_ops) cudaFree(s.d_ops);
+        if (s.h_rope) cudaFreeHost(s.h_rope);
+        if (s.d_rope) cudaFree(s.d_rope);
+        if (s.d_table) cudaFree(s.d_table);
+        if (s.done) cudaEventDestroy(s.done);
+    }
+    for (Pool &p : ctx->pools) {
+        if (p.d_k) cudaFree(p.d_k);
+        if (p.d_v) cudaFree(p.d_v);
+    }
+    for (int i = 0; i < 2; ++i) {
+        if (ctx->slab[i]) cudaFree(ctx->slab[i]);
+        if (ctx->slab_free[i]) cudaEventDestroy(ctx->slab_free[i]);
+        if (ctx->slab_ready[i]) cudaEventDestroy(ctx->slab_ready[i]);
+    }
+    if (ctx->own_side) cudaStreamDestroy(ctx->own_side);
+    if (ctx->d_status) cudaFree(ctx->d_status);
+    if (ctx->h_status) cudaFreeHost(ctx->h_status);
+    delete ctx;
+}
+
+kdn_status kdn_pool_register(kdn_ctx *ctx, const kdn_pool_desc *pool, int *pool_id)
+{
+    if (!ctx || !pool_id) return KDN_E_INVAL;
+    kdn_status st = check_shape(pool);
+    if (st != KDN_OK) return st;
+    if (!pool->k_layers || !pool->v_layers) return KDN_E_INVAL;
+    for (int l = 0; l < pool->n_layers; ++l) {
+        if (!pool->k_layers[l] || !pool->v_layers[l]) return KDN_E_INVAL;
+        if ((uintptr_t)pool->k_layers[l] % 16 || (uintptr_t)pool->v_layers[l] % 16) return KDN_E_ALIGN;
+    }
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return KDN_E_CUDA;
+    Pool p;
+    p.L = pool->n_layers; p.H = pool->n_kv_heads; p.D = pool->head_dim; p.bs = pool->block_size; p.nb = pool->n_blocks;
+    const size_t bytes = sizeof(void *) * (size_t)p.L;
+    KDN_CUDA(cudaMalloc((void **)&p.d_k, bytes));
+    if (cudaMalloc((void **)&p.d_v, bytes) != cudaSuccess) { cudaFree(p.d_k); return KDN_E_NOMEM; }
+    if (cudaMemcpy(p.d_k, pool->k_layers, bytes, cudaMemcpyHostToDevice) != cudaSuccess ||
+        cudaMemcpy(p.d_v, pool->v_layers, bytes, cudaMemcpyHostToDevice) != cudaSuccess) {
+        cudaFree(p.d_k); cudaFree(p.d_v);
+        return KDN_E_CUDA;
+    }
+    ctx->pools.push_back(p);
+    *pool_id = (int)ctx->pools.size() - 1;
+    return KDN_OK;
+}
+
+kdn_status kdn_store(kdn_ctx *ctx, int pool_id, const kdn_xfer_op *ops, int n_ops, void *cuda_stream, void *side_stream)
+{
+    return xfer(ctx, pool_id, OP_STORE, ops, n_ops, cuda_stream, side_stream);
+}
+
+kdn_status kdn_retrieve(kdn_ctx *ctx, int pool_id, const kdn_xfer_op *ops, int n_ops, void *cuda_stream, void *side_stream)
+{
+    return xfer(ctx, pool_id, OP_RETRIEVE, ops, n_ops, cuda_stream, side_stream);
+}
+
+kdn_status kdn_compose(kdn_ctx *ctx, int pool_id, const kdn_compose_req *reqs, int n_reqs, void *cuda_stream, void *side_stream)
+{
+    if (!ctx || pool_id < 0 || (size_t)pool_id >= ctx->pools.size()) return KDN_E_INVAL;
+    const Pool &pool = ctx->pools[(size_t)pool_id];
+    const kdn_pool_desc shape = shape_of(pool);
+    kdn_status st = kdn_validate_compose(&shape, reqs, n_reqs);
+    if (st != KDN_OK) return st;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return KDN_E_CUDA;
+    std::vector<HostOp> dev_ops, host_ops;
+    for (int r = 0; r < n_reqs; ++r) {
+        const kdn_compose_req &q = reqs[r];
+        for (int j = 0; j < q.n_parts; ++j) {
+            const kdn_chunk &c = q.parts[j];
+            if (c.n_tokens == 0) continue;
+            HostOp h = make_host_op(pool, q.block_table, q.part_dst_pos[j], c);
+            const long long delta = (long long)(q.part_dst_pos[j] - c.base_pos);
+            if (delta != 0) {
+                h.rotate = true;
+                h.rp.delta = delta;
+                h.rp.theta = q.rope_theta;
+            }
+            (c.mem == KDN_MEM_PINNED_HOST ? host_ops : dev_ops).push_back(h);
+        }
+    }
+    return run_ops(ctx, pool_id, OP_COMPOSE, dev_ops, host_ops, cuda_stream, side_stream);
+}
+
+kdn_status kdn_status_sync(kdn_ctx *ctx, void *cuda_stream)
+{
+    if (!ctx) return KDN_E_INVAL;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return KDN_E_CUDA;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    KDN_CUDA(cudaStreamSynchronize(stream));
+    if (ctx->own_side) KDN_CUDA(cudaStreamSynchronize(ctx->own_side));
+    KDN_CUDA(cudaStreamSynchronize(stream));              // work the side stream released onto `stream`
+    KDN_CUDA(cudaMemcpyAsync(ctx->h_status, ctx->d_status, sizeof(int), cudaMemcpyDeviceToHost, stream));
+    KDN_CUDA(cudaMemsetAsync(ctx->d_status, 0, sizeof(int), stream));
+    KDN_CUDA(cudaStreamSynchronize(stream));
+    const int s = *ctx->h_status;
+    return (s >= KDN_OK && s <= KDN_E_TIMEOUT) ? (kdn_status)s : KDN_E_CUDA;
+}
+
+kdn_status kdn_set_tuning(kdn_ctx *ctx, const kdn_tuning *tuning)
+{
+    if (!ctx) return KDN_E_INVAL;
+    if (!tuning) { ctx->tuning = kdn_tuning{}; return KDN_OK; }
+    if (tuning->tile_bytes < 0 || tuning->stages < 0 || tuning->ctas_per_sm < 0) return KDN_E_INVAL;
+    if (tuning->tile_bytes % 128) return KDN_E_INVAL;
+    if (tuning->stages && (tuning->stages < kStoreLag + 2 || tuning->stages > kMaxStages)) return KDN_E_UNSUPPORTED;
+    if (tuning->ctas_per_sm > 32) return KDN_E_UNSUPPORTED;
+    if (tuning->tile_bytes > ctx->smem_optin) return KDN_E_UNSUPPORTED;
+    ctx->tuning = *tuning;
+    return KDN_OK;
+}
+
+kdn_status kdn_set_staging_bytes(kdn_ctx *ctx, size_t bytes_per_slab)
+{
+    if (!ctx || bytes_per_slab < 4096) return KDN_E_INVAL;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return KDN_E_CUDA;
+    KDN_CUDA(cudaDeviceSynchronize());
+    for (int i = 0; i < 2; ++i) {
+        if (ctx->slab[i]) KDN_CUDA(cudaFree(ctx->slab[i]));
+        ctx->slab[i] = nullptr;
+    }
+    ctx->slab_bytes = bytes_per_slab & ~(size_t)255;
+    return KDN_OK;
+}
+
+uint64_t kdn_launch_count(const kdn_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+const char *kdn_strerror(kdn_status status)
+{
+    switch (status) {
+    case KDN_OK: return "ok";
+    case KDN_E_INVAL: return "invalid argument";
+    case KDN_E_SHAPE: return "chunk size does not match the pool shape";
+    case KDN_E_ALIGN: return "pointer or row size not 16-byte aligned";
+    case KDN_E_RANGE: return "token range or block id out of range";
+    case KDN_E_UNSUPPORTED: return "unsupported shape, codec or setting";
+    case KDN_E_CUDA: return "CUDA runtime error";
+    case KDN_E_NOMEM: return "out of memory";
+    case KDN_E_TIMEOUT: return "a bounded wait inside a kernel expired";
+    }
+    return "unknown status";
+}
+
+}  // extern "C"

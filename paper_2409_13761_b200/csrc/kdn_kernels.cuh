@@ -1,0 +1,613 @@
+// Device side of libkdn: one persistent, warp-specialised tile pipeline for sm_100a, instantiated
+// as the three kernels of the path (paper Sec. 3.1: storage -> kdn_store_kernel, delivery with
+// decompression on the GPU -> kdn_retrieve_kernel, blending -> kdn_compose_kernel).
+//
+// Work decomposition.  A chunk of T tokens and a paged pool meet in runs: for one (layer, K|V)
+// plane and one logical block of the request, the tokens of that block that belong to the chunk
+// are contiguous both in the pool block and in the chunk plane.  A run is cut into tiles of at most
+// tile_elems elements; tile g of the launch is handled by CTA g % gridDim.x.  Nothing in a tile
+// depends on another tile, so there is no inter-CTA synchronisation.
+//
+// Pipeline inside a CTA (S slots of shared memory, all hand-offs through mbarriers):
+//   loader warp   decodes tiles 32 at a time (one per lane: op lookup, block-table entry, addresses),
+//                 then issues each tile's bulk async copies global -> shared
+//   compute warps (4) int8 coding / decoding and key rotation, shared -> shared
+//   storer thread issues the bulk async copy shared -> global and recycles the slot
+// Tiles that are a pure copy (raw bf16 without rotation) never touch the compute warps' ALUs.
+// Every mbarrier wait is bounded by a wall-clock limit; on expiry the CTA records KDN_E_TIMEOUT,
+// drains its own copies with bounded waits and returns.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <cuda_bf16.h>
+#include <stdint.h>
+
+namespace kdn {
+
+constexpr int kLoaderWarp = 0;
+constexpr int kComputeWarps = 4;
+constexpr int kComputeThreads = kComputeWarps * 32;
+constexpr int kThreadsCompute = 32 + kComputeThreads + 32;   // loader + compute + storer
+constexpr int kThreadsCopy = 64;                             // loader + storer
+constexpr int kMaxStages = 32;
+constexpr int kStoreLag = 2;              // bulk stores allowed to be still reading shared memory
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+enum : uint32_t { TF_INT8 = 1u, TF_ROTATE = 2u, TF_SCALES_PLAIN = 4u };
+enum : int { OP_STORE = 0, OP_RETRIEVE = 1, OP_COMPOSE = 2 };
+
+// Status values mirrored from kdn.h (kept numeric here so device code has no host header).
+constexpr int kStatusRange = 4;
+constexpr int kStatusTimeout = 8;
+
+struct __align__(16) DevOp {
+    const int32_t *table;     // device block table of the request
+    unsigned char *data;      // chunk bytes for layers [l0, l0 + nl): raw bf16, or codes then scales
+    long long off;            // request position of chunk token 0
+    int T;                    // tokens
+    int codec;                // 0 raw bf16, 1 int8 group-64
+    int j0;                   // first logical block touched: off / block_size
+    int nblk;                 // logical blocks touched
+    unsigned tile_begin;      // index of this op's first tile in the launch
+    int rope;                 // row of the rotation table, -1: keys are copied
+    int l0;                   // first pool layer
+    int nl;                   // layers held in data
+    long long reserved;
+};
+static_assert(sizeof(DevOp) == 64, "DevOp is copied as 64-byte records");
+
+struct RopeParam {            // one row of the rotation table to fill
+    long long delta;          // dst_pos - base_pos
+    double theta;
+};
+
+struct Launch {
+    const DevOp *ops;
+    int n_ops;
+    unsigned n_tiles;
+    void *const *k_layers;    // device arrays of per-layer pool pointers
+    void *const *v_layers;
+    long long n_blocks;
+    int bs;
+    int D;
+    unsigned row_elems;       // H * D
+    unsigned tile_elems;
+    unsigned tpb;             // tiles per logical block
+    const float2 *rope;       // [rows][D/2] (cos, sin)
+    int *status;
+    int stages;
+    unsigned stage_bytes;
+    unsigned off_b;           // offset of the code buffer inside a stage (compute launches)
+    unsigned off_s;           // offset of the scale buffer inside a stage
+};
+
+struct __align__(16) TileDesc {
+    unsigned long long g_pool;    // bf16 address in the pool
+    unsigned long long g_chunk;   // chunk side: bf16 (raw) or codes (int8)
+    unsigned long long g_scales;  // chunk side: scales (int8)
+    unsigned n;                   // elements; 0: nothing to do
+    unsigned flags;
+    int rope;
+    int reserved;
+};
+
+// ------------------------------------------------------------------ PTX --
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar)
+{
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+// Bounded wait: true when the phase completed; false when the CTA is aborting or the limit passed.
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    unsigned long long t0 = global_timer_ns();
+    for (uint32_t n = 1;; ++n) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((n & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
+        }
+    }
+}
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    return mbar_wait_slow(bar, parity, abort_flag);
+}
+// Bulk async copy global -> this CTA's shared memory, completion counted on an mbarrier.
+// (No cluster is launched: the CTA's own shared window is the cluster window.)
+__device__ __forceinline__ void bulk_g2s(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void bulk_s2g(void *dst, uint32_t src, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(dst), "r"(src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+template <int N> __device__ __forceinline__ void bulk_wait_read()
+{
+    asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+__device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void compute_bar_sync()
+{
+    asm volatile("bar.sync 1, %0;" ::"n"(kComputeThreads) : "memory");
+}
+
+__device__ __forceinline__ uint4 lds128(const void *p) { return *reinterpret_cast<const uint4 *>(p); }
+__device__ __forceinline__ uint2 lds64(const void *p) { return *reinterpret_cast<const uint2 *>(p); }
+__device__ __forceinline__ void sts128(void *p, uint4 v) { *reinterpret_cast<uint4 *>(p) = v; }
+__device__ __forceinline__ void sts64(void *p, uint2 v) { *reinterpret_cast<uint2 *>(p) = v; }
+
+// ----------------------------------------------------------- arithmetic --
+
+__device__ __forceinline__ float bf16_lo(uint32_t w) { return __uint_as_float(w << 16); }
+__device__ __forceinline__ float bf16_hi(uint32_t w) { return __uint_as_float(w & 0xffff0000u); }
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
+{
+    __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);     // round to nearest even, lo in the low half
+    return *reinterpret_cast<uint32_t *>(&v);
+}
+
+// round_half_even(x * inv) as the low byte of the fp32 sum with 1.5 * 2^23: for |x * inv| < 2^22 the
+// sum is rounded to an integer by the adder itself (ties to even) and its low mantissa bits are the
+// two's-complement integer.  The product and the sum are two separately rounded fp32 operations.
+__device__ __forceinline__ uint32_t code_bits(float x, float inv)
+{
+    return __float_as_uint(__fadd_rn(__fmul_rn(x, inv), 12582912.0f));
+}
+__device__ __forceinline__ uint32_t pack_codes4(uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3)
+{
+    uint32_t a = __byte_perm(r0, r1, 0x0040);             // r0.b0, r1.b0
+    uint32_t b = __byte_perm(r2, r3, 0x0040);
+    return __byte_perm(a, b, 0x5410);
+}
+// (float)code for byte k of w, where w holds four codes already XORed with 0x80: 2^23 + (code + 128)
+// built in the mantissa, minus 2^23 + 128.  Exact.
+template <int K> __device__ __forceinline__ float code_to_float(uint32_t w_biased)
+{
+    return __fsub_rn(__uint_as_float(__byte_perm(w_biased, 0x4B000000u, 0x7650 + K)), 8388736.0f);
+}
+
+// Encode n elements (a multiple of 64) of bf16 at A into int8 codes at B and one fp32 scale per 64
+// elements (to shared S, or straight to global when the destination is not 16-byte aligned).
+// 8 lanes share a group; the absmax is reduced with three shuffles.
+__device__ __forceinline__ void quantise_tile(const unsigned char *A, unsigned char *B, float *S, float *g_scales,
+                                              unsigned n, int ct)
+{
+    const unsigned nvec = n >> 3;
+    const unsigned lane = (unsigned)ct & 31u;
+    for (unsigned vb = (unsigned)ct & ~31u; vb < nvec; vb += kComputeThreads) {
+        const unsigned v = vb + lane;
+        const bool act = v < nvec;
+        uint4 x = act ? lds128(A + (size_t)v * 16u) : make_uint4(0u, 0u, 0u, 0u);
+        float f[8] = { bf16_lo(x.x), bf16_hi(x.x), bf16_lo(x.y), bf16_hi(x.y),
+                       bf16_lo(x.z), bf16_hi(x.z), bf16_lo(x.w), bf16_hi(x.w) };
+        float a = 0.0f;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) a = fmaxf(a, fabsf(f[k]));
+        a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
+        a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 2));
+        a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 4));
+        float scale = __fdiv_rn(a, 127.0f);
+        const bool ok = scale >= 1.17549435e-38f;         // smallest normal fp32; false for NaN too
+        const float inv = ok ? __fdiv_rn(127.0f, a) : 0.0f;
+        scale = ok ? scale : 0.0f;
+        if (act) {
+            uint2 q;
+            q.x = pack_codes4(code_bits(f[0], inv), code_bits(f[1], inv), code_bits(f[2], inv), code_bits(f[3], inv));
+            q.y = pack_codes4(code_bits(f[4], inv), code_bits(f[5], inv), code_bits(f[6], inv), code_bits(f[7], inv));
+            sts64(B + (size_t)v * 8u, q);
+            if ((lane & 7u) == 0u) {
+                if (g_scales) g_scales[v >> 3] = scale; else S[v >> 3] = scale;
+            }
+        }
+    }
+}
+
+// Decode n int8 codes at B with scales S into bf16 at A: one fp32 product, rounded to bf16.
+__device__ __forceinline__ void dequantise_tile(const unsigned char *B, const float *S, unsigned char *A,
+                                                unsigned n, int ct)
+{
+    const unsigned nvec = n >> 4;
+    for (unsigned v = (unsigned)ct; v < nvec; v += kComputeThreads) {
+        const uint4 c = lds128(B + (size_t)v * 16u);
+        const float sc = S[v >> 2];
+        const uint32_t w[4] = { c.x ^ 0x80808080u, c.y ^ 0x80808080u, c.z ^ 0x80808080u, c.w ^ 0x80808080u };
+        uint32_t o[8];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            o[2 * j] = pack_bf16x2(__fmul_rn(code_to_float<0>(w[j]), sc), __fmul_rn(code_to_float<1>(w[j]), sc));
+            o[2 * j + 1] = pack_bf16x2(__fmul_rn(code_to_float<2>(w[j]), sc), __fmul_rn(code_to_float<3>(w[j]), sc));
+        }
+        sts128(A + (size_t)v * 32u, make_uint4(o[0], o[1], o[2], o[3]));
+        sts128(A + (size_t)v * 32u + 16u, make_uint4(o[4], o[5], o[6], o[7]));
+    }
+}
+
+// Rotation coefficients a thread keeps in registers: (cos, sin) for 8 consecutive frequencies.
+struct RotCoef {
+    float c[8], s[8];
+    int rope;      // table row they belong to
+    unsigned col;  // first frequency index
+};
+
+__device__ __forceinline__ void load_coef(RotCoef &rc, const float2 *table, int rope, unsigned col, unsigned half)
+{
+    if (rc.rope == rope && rc.col == col) return;
+    const float4 *p = reinterpret_cast<const float4 *>(table + (size_t)rope * half + col);
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        float4 v = __ldg(p + k);
+        rc.c[2 * k] = v.x; rc.s[2 * k] = v.y; rc.c[2 * k + 1] = v.z; rc.s[2 * k + 1] = v.w;
+    }
+    rc.rope = rope; rc.col = col;
+}
+
+__device__ __forceinline__ void rotate8(const float *u, const float *w, const RotCoef &rc, uint4 &lo, uint4 &hi)
+{
+    float u2[8], w2[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) {
+        u2[k] = __fmaf_rn(u[k], rc.c[k], -__fmul_rn(w[k], rc.s[k]));
+        w2[k] = __fmaf_rn(w[k], rc.c[k], __fmul_rn(u[k], rc.s[k]));
+    }
+    lo = make_uint4(pack_bf16x2(u2[0], u2[1]), pack_bf16x2(u2[2], u2[3]), pack_bf16x2(u2[4], u2[5]), pack_bf16x2(u2[6], u2[7]));
+    hi = make_uint4(pack_bf16x2(w2[0], w2[1]), pack_bf16x2(w2[2], w2[3]), pack_bf16x2(w2[4], w2[5]), pack_bf16x2(w2[6], w2[7]));
+}
+
+// Rotate a tile of whole head rows (n a multiple of D, D a multiple of 16).  One work item is 8
+// frequencies of one head row: elements [col, col+8) and [D/2 + col, D/2 + col + 8).
+// kInt8 = false: bf16 at A, in place.  kInt8 = true: codes at B and scales at S -> bf16 at A.
+template <bool kInt8>
+__device__ __forceinline__ void rotate_tile(unsigned char *A, const unsigned char *B, const float *S, unsigned n,
+                                            unsigned D, const float2 *table, int rope, RotCoef &rc, int ct)
+{
+    const unsigned half = D >> 1;
+    const unsigned per_row = D >> 4;                      // work items per head row
+    const unsigned items = n >> 4;
+    for (unsigned it = (unsigned)ct; it < items; it += kComputeThreads) {
+        const unsigned r = it / per_row;
+        const unsigned col = (it - r * per_row) << 3;
+        load_coef(rc, table, rope, col, half);
+        const unsigned e_lo = r * D + col, e_hi = e_lo + half;
+        float u[8], w[8];
+        if (kInt8) {
+            const uint2 cl = lds64(B + e_lo), ch = lds64(B + e_hi);
+            const float sl = S[e_lo >> 6], sh = S[e_hi >> 6];
+            const uint32_t l0 = cl.x ^ 0x80808080u, l1 = cl.y ^ 0x80808080u;
+            const uint32_t h0 = ch.x ^ 0x80808080u, h1 = ch.y ^ 0x80808080u;
+            u[0] = __fmul_rn(code_to_float<0>(l0), sl); u[1] = __fmul_rn(code_to_float<1>(l0), sl);
+            u[2] = __fmul_rn(code_to_float<2>(l0), sl); u[3] = __fmul_rn(code_to_float<3>(l0), sl);
+            u[4] = __fmul_rn(code_to_float<0>(l1), sl); u[5] = __fmul_rn(code_to_float<1>(l1), sl);
+            u[6] = __fmul_rn(code_to_float<2>(l1), sl); u[7] = __fmul_rn(code_to_float<3>(l1), sl);
+            w[0] = __fmul_rn(code_to_float<0>(h0), sh); w[1] = __fmul_rn(code_to_float<1>(h0), sh);
+            w[2] = __fmul_rn(code_to_float<2>(h0), sh); w[3] = __fmul_rn(code_to_float<3>(h0), sh);
+            w[4] = __fmul_rn(code_to_float<0>(h1), sh); w[5] = __fmul_rn(code_to_float<1>(h1), sh);
+            w[6] = __fmul_rn(code_to_float<2>(h1), sh); w[7] = __fmul_rn(code_to_float<3>(h1), sh);
+        } else {
+            const uint4 xl = lds128(A + (size_t)e_lo * 2u), xh = lds128(A + (size_t)e_hi * 2u);
+            u[0] = bf16_lo(xl.x); u[1] = bf16_hi(xl.x); u[2] = bf16_lo(xl.y); u[3] = bf16_hi(xl.y);
+            u[4] = bf16_lo(xl.z); u[5] = bf16_hi(xl.z); u[6] = bf16_lo(xl.w); u[7] = bf16_hi(xl.w);
+            w[0] = bf16_lo(xh.x); w[1] = bf16_hi(xh.x); w[2] = bf16_lo(xh.y); w[3] = bf16_hi(xh.y);
+            w[4] = bf16_lo(xh.z); w[5] = bf16_hi(xh.z); w[6] = bf16_lo(xh.w); w[7] = bf16_hi(xh.w);
+        }
+        uint4 lo, hi;
+        rotate8(u, w, rc, lo, hi);
+        sts128(A + (size_t)e_lo * 2u, lo);
+        sts128(A + (size_t)e_hi * 2u, hi);
+    }
+}
+
+// ---------------------------------------------------------- tile decode --
+
+// Address resolution (request position -> block-table entry -> pool address) and chunk addressing
+// for tile g.  Records KDN_E_RANGE and yields an empty tile for a block id outside the pool.
+template <int OP>
+__device__ __forceinline__ void decode_tile(const Launch &P, unsigned g, TileDesc &d)
+{
+    d.n = 0; d.flags = 0; d.rope = -1; d.reserved = 0;
+    d.g_pool = 0; d.g_chunk = 0; d.g_scales = 0;
+    if (g >= P.n_tiles) return;                             // lanes past this CTA's last tile
+    int lo = 0, hi = P.n_ops - 1;
+    while (lo < hi) {                                       // last op with tile_begin <= g
+        int mid = (lo + hi + 1) >> 1;
+        if (__ldg(&P.ops[mid].tile_begin) <= g) lo = mid; else hi = mid - 1;
+    }
+    const DevOp op = P.ops[lo];
+    const unsigned gl = g - op.tile_begin;
+    const unsigned per_plane = (unsigned)op.nblk * P.tpb;
+    const unsigned plane = gl / per_plane;
+    const unsigned rem = gl - plane * per_plane;
+    const unsigned j = rem / P.tpb;
+    const unsigned k = rem - j * P.tpb;
+    const int kv = (int)(plane & 1u);
+    const int l = op.l0 + (int)(plane >> 1);
+    const long long blk_start = ((long long)op.j0 + j) * P.bs;
+    const long long p_lo = op.off > blk_start ? op.off : blk_start;
+    const long long p_end = op.off + op.T;
+    const long long p_hi = p_end < blk_start + P.bs ? p_end : blk_start + P.bs;
+    if (p_hi <= p_lo) return;
+    const unsigned long long run = (unsigned long long)(p_hi - p_lo) * P.row_elems;
+    const unsigned long long e0 = (unsigned long long)k * P.tile_elems;
+    if (e0 >= run) return;
+    const unsigned n = (unsigned)((run - e0) < (unsigned long long)P.tile_elems ? (run - e0) : P.tile_elems);
+    const long long id = __ldg(op.table + op.j0 + j);
+    if (id < 0 || id >= P.n_blocks) { atomicCAS(P.status, 0, kStatusRange); return; }
+    const unsigned char *base = reinterpret_cast<const unsigned char *>(kv ? P.v_layers[l] : P.k_layers[l]);
+    d.g_pool = (unsigned long long)(base + (((unsigned long long)id * P.bs + (unsigned long long)(p_lo - blk_start)) * P.row_elems + e0) * 2ull);
+    const unsigned long long ce = ((unsigned long long)plane * op.T + (unsigned long long)(p_lo - op.off)) * P.row_elems + e0;
+    if (op.codec == 0) {
+        d.g_chunk = (unsigned long long)(op.data + ce * 2ull);
+    } else {
+        d.flags |= TF_INT8;
+        d.g_chunk = (unsigned long long)(op.data + ce);
+        const unsigned long long codes_bytes = (unsigned long long)op.nl * 2ull * op.T * P.row_elems;
+        d.g_scales = (unsigned long long)(op.data + codes_bytes + (ce >> 6) * 4ull);
+        if ((d.g_scales & 15ull) || ((n >> 6) & 3u)) d.flags |= TF_SCALES_PLAIN;
+    }
+    if (OP == OP_COMPOSE && kv == 0 && op.rope >= 0) { d.flags |= TF_ROTATE; d.rope = op.rope; }
+    d.n = n;
+}
+
+// ------------------------------------------------------------- pipeline --
+
+struct Smem {
+    unsigned char *stage0;
+    uint32_t full, empty, ready;      // shared addresses of the barrier arrays (8 bytes per stage)
+    TileDesc *desc;
+    volatile int *abort_flag;
+};
+
+__device__ __forceinline__ Smem carve(const Launch &P, unsigned char *smem)
+{
+    Smem s;
+    s.stage0 = smem;
+    unsigned char *p = smem + (size_t)P.stages * P.stage_bytes;
+    s.full = smem_u32(p);
+    s.empty = s.full + 8u * (uint32_t)P.stages;
+    s.ready = s.empty + 8u * (uint32_t)P.stages;
+    p += 24u * (size_t)P.stages;
+    p = (unsigned char *)(((uintptr_t)p + 15u) & ~(uintptr_t)15u);
+    s.desc = reinterpret_cast<TileDesc *>(p);
+    s.abort_flag = reinterpret_cast<volatile int *>(p + sizeof(TileDesc) * (size_t)P.stages);
+    return s;
+}
+
+// Bytes of shared memory a launch needs (host mirrors this).
+__host__ __device__ inline size_t smem_bytes(int stages, unsigned stage_bytes)
+{
+    return (size_t)stages * stage_bytes + 24u * (size_t)stages + 16u + sizeof(TileDesc) * (size_t)stages + 16u;
+}
+
+template <int OP, bool kCompute>
+__device__ __forceinline__ void tile_pipeline(const Launch &P)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const Smem sm = carve(P, smem_raw);
+    const int S = P.stages;
+    const int tid = (int)threadIdx.x;
+    const int warp = tid >> 5;
+    const int lane = tid & 31;
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(sm.full + 8u * s, 1u);
+            mbar_init(sm.empty + 8u * s, 1u);
+            mbar_init(sm.ready + 8u * s, (uint32_t)kComputeWarps);
+        }
+        *sm.abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_async_smem();
+    }
+    __syncthreads();
+
+    const unsigned grid = gridDim.x, bid = blockIdx.x;
+    const unsigned n_my = P.n_tiles > bid ? (P.n_tiles - bid + grid - 1u) / grid : 0u;
+    const int storer_warp = kCompute ? 1 + kComputeWarps : 1;
+
+    if (warp == kLoaderWarp) {
+        // ------------------------------------------------------------ loader
+        unsigned issued = 0;
+        bool aborted = false;
+        TileDesc cur;
+        decode_tile<OP>(P, (unsigned)lane < n_my ? bid + (unsigned)lane * grid : 0xffffffffu, cur);
+        for (unsigned base = 0; base < n_my && !aborted; base += 32u) {
+            TileDesc nxt;
+            decode_tile<OP>(P, base + 32u + lane < n_my ? bid + (base + 32u + lane) * grid : 0xffffffffu, nxt);
+            const unsigned cnt = n_my - base < 32u ? n_my - base : 32u;
+            for (unsigned t = 0; t < cnt; ++t) {
+                if ((unsigned)lane == t) {
+                    const unsigned slot = base + t;
+                    const unsigned st = slot % (unsigned)S;
+                    const uint32_t ph = (slot / (unsigned)S) & 1u;
+                    if (mbar_wait(sm.empty + 8u * st, ph ^ 1u, sm.abort_flag)) {
+                        sm.desc[st] = cur;
+                        const uint32_t bar = sm.full + 8u * st;
+                        unsigned char *A = sm.stage0 + (size_t)st * P.stage_bytes;
+                        if (cur.n == 0u) {
+                            mbar_arrive(bar);
+                        } else if (OP == OP_STORE) {
+                            mbar_arrive_expect_tx(bar, cur.n * 2u);
+                            bulk_g2s(smem_u32(A), (const void *)cur.g_pool, cur.n * 2u, bar);
+                        } else if (!(cur.flags & TF_INT8)) {
+                            mbar_arrive_expect_tx(bar, cur.n * 2u);
+                            bulk_g2s(smem_u32(A), (const void *)cur.g_chunk, cur.n * 2u, bar);
+                        } else if (cur.flags & TF_SCALES_PLAIN) {
+                            mbar_arrive_expect_tx(bar, cur.n);
+                            bulk_g2s(smem_u32(A + P.off_b), (const void *)cur.g_chunk, cur.n, bar);
+                        } else {
+                            mbar_arrive_expect_tx(bar, cur.n + (cur.n >> 4));
+                            bulk_g2s(smem_u32(A + P.off_b), (const void *)cur.g_chunk, cur.n, bar);
+                            bulk_g2s(smem_u32(A + P.off_s), (const void *)cur.g_scales, cur.n >> 4, bar);
+                        }
+                    }
+                }
+                __syncwarp();
+                if (__any_sync(0xffffffffu, *sm.abort_flag != 0)) { aborted = true; break; }
+                ++issued;
+            }
+            cur = nxt;
+        }
+        if (aborted && lane == 0) {
+            atomicCAS(P.status, 0, kStatusTimeout);
+            // bounded drain of the copies this warp issued into the last S slots
+            const unsigned first = issued > (unsigned)S ? issued - (unsigned)S : 0u;
+            for (unsigned slot = first; slot < issued; ++slot) {
+                unsigned long long t0 = global_timer_ns();
+                while (!mbar_try_wait(sm.full + 8u * (slot % (unsigned)S), (slot / (unsigned)S) & 1u))
+                    if (global_timer_ns() - t0 > kWaitLimitNs) break;
+            }
+        }
+    } else if (warp == storer_warp) {
+        // ------------------------------------------------------------ storer
+        if (lane == 0) {
+            unsigned done = 0;                                // slots whose store group was committed
+            for (unsigned slot = 0; slot < n_my; ++slot) {
+                const unsigned st = slot % (unsigned)S;
+                const uint32_t ph = (slot / (unsigned)S) & 1u;
+                if (!mbar_wait(sm.full + 8u * st, ph, sm.abort_flag)) break;
+                const TileDesc d = sm.desc[st];
+                unsigned char *A = sm.stage0 + (size_t)st * P.stage_bytes;
+                if (d.n != 0u) {
+                    const bool computed = kCompute && (OP == OP_STORE ? (d.flags & TF_INT8) != 0u
+                                                                       : (d.flags & (TF_INT8 | TF_ROTATE)) != 0u);
+                    if (computed && !mbar_wait(sm.ready + 8u * st, ph, sm.abort_flag)) break;
+                    if (OP == OP_STORE) {
+                        if (d.flags & TF_INT8) {
+                            bulk_s2g((void *)d.g_chunk, smem_u32(A + P.off_b), d.n);
+                            if (!(d.flags & TF_SCALES_PLAIN))
+                                bulk_s2g((void *)d.g_scales, smem_u32(A + P.off_s), d.n >> 4);
+                        } else {
+                            bulk_s2g((void *)d.g_chunk, smem_u32(A), d.n * 2u);
+                        }
+                    } else {
+                        bulk_s2g((void *)d.g_pool, smem_u32(A), d.n * 2u);
+                    }
+                }
+                bulk_commit();
+                ++done;
+                // recycle the slot committed kStoreLag slots ago: its store has read shared memory,
+                // and every compute warp has moved past it
+                bulk_wait_read<kStoreLag>();
+                if (slot >= (unsigned)kStoreLag) {
+                    const unsigned old = slot - (unsigned)kStoreLag;
+                    const unsigned st2 = old % (unsigned)S;
+                    if (kCompute && !mbar_wait(sm.ready + 8u * st2, (old / (unsigned)S) & 1u, sm.abort_flag)) break;
+                    mbar_arrive(sm.empty + 8u * st2);
+                }
+            }
+            bulk_wait_read<0>();
+            for (unsigned slot = done > (unsigned)kStoreLag ? done - kStoreLag : 0u; slot < done; ++slot)
+                mbar_arrive(sm.empty + 8u * (slot % (unsigned)S));
+            bulk_wait_all();
+            if (done != n_my) atomicCAS(P.status, 0, kStatusTimeout);
+        }
+    } else if (kCompute) {
+        // ----------------------------------------------------------- compute
+        const int ct = tid - 32;
+        RotCoef rc;
+        rc.rope = -1; rc.col = 0xffffffffu;
+        for (unsigned slot = 0; slot < n_my; ++slot) {
+            const unsigned st = slot % (unsigned)S;
+            const uint32_t ph = (slot / (unsigned)S) & 1u;
+            if (!mbar_wait(sm.full + 8u * st, ph, sm.abort_flag)) break;
+            const unsigned n = sm.desc[st].n;
+            const unsigned flags = sm.desc[st].flags;
+            unsigned char *A = sm.stage0 + (size_t)st * P.stage_bytes;
+            unsigned char *B = A + P.off_b;
+            float *Sc = reinterpret_cast<float *>(A + P.off_s);
+            bool computed = false;
+            if (n != 0u) {
+                if (OP == OP_STORE) {
+                    if (flags & TF_INT8) {
+                        float *gs = (flags & TF_SCALES_PLAIN) ? reinterpret_cast<float *>(sm.desc[st].g_scales) : nullptr;
+                        quantise_tile(A, B, Sc, gs, n, ct);
+                        computed = true;
+                    }
+                } else if (flags & TF_INT8) {
+                    if (flags & TF_SCALES_PLAIN) {
+                        const float *gs = reinterpret_cast<const float *>(sm.desc[st].g_scales);
+                        for (unsigned i = (unsigned)ct; i < (n >> 6); i += kComputeThreads) Sc[i] = __ldg(gs + i);
+                        compute_bar_sync();
+                    }
+                    if (OP == OP_COMPOSE && (flags & TF_ROTATE))
+                        rotate_tile<true>(A, B, Sc, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct);
+                    else
+                        dequantise_tile(B, Sc, A, n, ct);
+                    computed = true;
+                } else if (OP == OP_COMPOSE && (flags & TF_ROTATE)) {
+                    rotate_tile<false>(A, nullptr, nullptr, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct);
+                    computed = true;
+                }
+            }
+            // one arrival per warp and slot: "this warp's shared-memory writes are visible to the
+            // bulk store, and it no longer reads the slot"
+            if (computed) fence_async_smem();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(sm.ready + 8u * st);
+        }
+    }
+    __syncthreads();
+}
+
+// Sec. 3.2 call (i) store, Sec. 3.1 storage module: paged pool -> chunk, optional int8 coding.
+template <bool kCompute>
+__global__ void __launch_bounds__(kCompute ? kThreadsCompute : kThreadsCopy)
+kdn_store_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_STORE, kCompute>(P); }
+
+// Sec. 3.2 call (ii) retrieve, Sec. 3.1 delivery module (decompression on the GPU): chunk -> pool.
+template <bool kCompute>
+__global__ void __launch_bounds__(kCompute ? kThreadsCompute : kThreadsCopy)
+kdn_retrieve_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_RETRIEVE, kCompute>(P); }
+
+// Sec. 3.1 blending module: parts -> request blocks at new positions, keys re-rotated.
+template <bool kCompute>
+__global__ void __launch_bounds__(kCompute ? kThreadsCompute : kThreadsCopy)
+kdn_compose_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_COMPOSE, kCompute>(P); }
+
+// Rotation table: row r, frequency i -> (cos, sin) of delta_r * theta_r^(-2i/D), evaluated in fp64 and
+// rounded once to fp32 (an fp32 angle would lose more than half a bf16 ulp at large position shifts).
+__global__ void kdn_rope_table_kernel(const RopeParam *params, int n_rows, int D, float2 *table)
+{
+    const int half = D >> 1;
+    const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= (long long)n_rows * half) return;
+    const int r = (int)(idx / half), i = (int)(idx - (long long)r * half);
+    const double inv_freq = pow(params[r].theta, -2.0 * (double)i / (double)D);
+    const double phi = (double)params[r].delta * inv_freq;
+    double s, c;
+    sincos(phi, &s, &c);
+    table[idx] = make_float2((float)c, (float)s);
+}
+
+}  // namespace kdn

@@ -1,0 +1,235 @@
+"""ctypes binding of libkdn.so: the functions of include/kdn.h under the same names.
+
+Argument marshalling only.  Every step of store / retrieve / compose runs in the library's CUDA
+kernels; there is no Python or CPU implementation behind these calls.  Importing this module fails
+if libkdn.so is absent and cannot be built.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from dataclasses import dataclass
+from typing import List, Optional, Sequence
+
+from . import build as _build
+
+KDN_OK, KDN_E_INVAL, KDN_E_SHAPE, KDN_E_ALIGN, KDN_E_RANGE, KDN_E_UNSUPPORTED, KDN_E_CUDA, KDN_E_NOMEM, \
+    KDN_E_TIMEOUT = range(9)
+KDN_CODEC_RAW_BF16, KDN_CODEC_INT8_G64 = 0, 1
+KDN_MEM_DEVICE, KDN_MEM_PINNED_HOST = 0, 1
+
+EXPORTS = ["kdn_create", "kdn_destroy", "kdn_pool_register", "kdn_chunk_bytes", "kdn_validate_xfer",
+           "kdn_validate_compose", "kdn_store", "kdn_retrieve", "kdn_compose", "kdn_status_sync",
+           "kdn_set_tuning", "kdn_set_staging_bytes", "kdn_launch_count", "kdn_strerror"]
+
+
+class kdn_pool_desc(C.Structure):
+    _fields_ = [("n_layers", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
+                ("block_size", C.c_int32), ("n_blocks", C.c_int64),
+                ("k_layers", C.POINTER(C.c_void_p)), ("v_layers", C.POINTER(C.c_void_p))]
+
+
+class kdn_chunk(C.Structure):
+    _fields_ = [("data", C.c_void_p), ("bytes", C.c_size_t), ("n_tokens", C.c_int32), ("codec", C.c_int32),
+                ("mem", C.c_int32), ("reserved", C.c_int32), ("base_pos", C.c_int64)]
+
+
+class kdn_xfer_op(C.Structure):
+    _fields_ = [("block_table", C.c_void_p), ("n_table_blocks", C.c_int32), ("reserved", C.c_int32),
+                ("token_offset", C.c_int64), ("chunk", kdn_chunk)]
+
+
+class kdn_compose_req(C.Structure):
+    _fields_ = [("block_table", C.c_void_p), ("n_table_blocks", C.c_int32), ("n_parts", C.c_int32),
+                ("parts", C.POINTER(kdn_chunk)), ("part_dst_pos", C.POINTER(C.c_int64)),
+                ("rope_theta", C.c_double), ("rope_style", C.c_int32), ("reserved", C.c_int32)]
+
+
+class kdn_tuning(C.Structure):
+    _fields_ = [("tile_bytes", C.c_int32), ("stages", C.c_int32), ("ctas_per_sm", C.c_int32),
+                ("reserved", C.c_int32)]
+
+
+def _load() -> C.CDLL:
+    path = _build.LIB
+    if not _build.up_to_date():
+        try:
+            _build.build()
+        except Exception as exc:                      # no nvcc, or the compile failed
+            if not os.path.exists(path):
+                raise ImportError("libkdn.so is missing and could not be built: %s" % exc) from exc
+    lib = C.CDLL(path)
+    vp, i32 = C.c_void_p, C.c_int
+    lib.kdn_create.restype = i32
+    lib.kdn_create.argtypes = [C.POINTER(vp), i32]
+    lib.kdn_destroy.restype = None
+    lib.kdn_destroy.argtypes = [vp]
+    lib.kdn_pool_register.restype = i32
+    lib.kdn_pool_register.argtypes = [vp, C.POINTER(kdn_pool_desc), C.POINTER(i32)]
+    lib.kdn_chunk_bytes.restype = C.c_size_t
+    lib.kdn_chunk_bytes.argtypes = [C.POINTER(kdn_pool_desc), C.c_int32, C.c_int32]
+    lib.kdn_validate_xfer.restype = i32
+    lib.kdn_validate_xfer.argtypes = [C.POINTER(kdn_pool_desc), C.POINTER(kdn_xfer_op), i32]
+    lib.kdn_validate_compose.restype = i32
+    lib.kdn_validate_compose.argtypes = [C.POINTER(kdn_pool_desc), C.POINTER(kdn_compose_req), i32]
+    for name in ("kdn_store", "kdn_retrieve"):
+        fn = getattr(lib, name)
+        fn.restype = i32
+        fn.argtypes = [vp, i32, C.POINTER(kdn_xfer_op), i32, vp, vp]
+    lib.kdn_compose.restype = i32
+    lib.kdn_compose.argtypes = [vp, i32, C.POINTER(kdn_compose_req), i32, vp, vp]
+    lib.kdn_status_sync.restype = i32
+    lib.kdn_status_sync.argtypes = [vp, vp]
+    lib.kdn_set_tuning.restype = i32
+    lib.kdn_set_tuning.argtypes = [vp, C.POINTER(kdn_tuning)]
+    lib.kdn_set_staging_bytes.restype = i32
+    lib.kdn_set_staging_bytes.argtypes = [vp, C.c_size_t]
+    lib.kdn_launch_count.restype = C.c_uint64
+    lib.kdn_launch_count.argtypes = [vp]
+    lib.kdn_strerror.restype = C.c_char_p
+    lib.kdn_strerror.argtypes = [i32]
+    return lib
+
+
+lib = _load()
+
+
+class KdnError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = int(status)
+        super().__init__("%s: %s (status %d)" % (where, kdn_strerror(status), status))
+
+
+def _check(status: int, where: str) -> None:
+    if status != KDN_OK:
+        raise KdnError(status, where)
+
+
+# ------------------------------------------------------------ Python-side argument records --
+
+@dataclass
+class Chunk:
+    data: int                  # address: device memory, or page-locked host memory with mem=KDN_MEM_PINNED_HOST
+    bytes: int
+    n_tokens: int
+    codec: int = KDN_CODEC_RAW_BF16
+    mem: int = KDN_MEM_DEVICE
+    base_pos: int = 0
+
+    def c(self) -> kdn_chunk:
+        return kdn_chunk(self.data, self.bytes, self.n_tokens, self.codec, self.mem, 0, self.base_pos)
+
+
+@dataclass
+class XferOp:
+    block_table: int           # device address of int32 [n_table_blocks]
+    n_table_blocks: int
+    token_offset: int
+    chunk: Chunk
+
+
+@dataclass
+class ComposeReq:
+    block_table: int
+    n_table_blocks: int
+    parts: Sequence[Chunk]
+    part_dst_pos: Sequence[int]
+    rope_theta: float
+    rope_style: int = 0
+
+
+def pool_desc(n_layers: int, n_kv_heads: int, head_dim: int, block_size: int, n_blocks: int,
+              k_layers: Optional[Sequence[int]] = None, v_layers: Optional[Sequence[int]] = None) -> kdn_pool_desc:
+    """Build a kdn_pool_desc; the pointer arrays are kept alive on the returned object."""
+    d = kdn_pool_desc(n_layers, n_kv_heads, head_dim, block_size, n_blocks, None, None)
+    if k_layers is not None:
+        ka = (C.c_void_p * len(k_layers))(*k_layers)
+        va = (C.c_void_p * len(v_layers))(*v_layers)
+        d.k_layers = C.cast(ka, C.POINTER(C.c_void_p))
+        d.v_layers = C.cast(va, C.POINTER(C.c_void_p))
+        d._keep = (ka, va)
+    return d
+
+
+def xfer_array(ops: Sequence[XferOp]):
+    arr = (kdn_xfer_op * max(1, len(ops)))()
+    for i, o in enumerate(ops):
+        arr[i] = kdn_xfer_op(o.block_table, o.n_table_blocks, 0, o.token_offset, o.chunk.c())
+    return arr
+
+
+def compose_array(reqs: Sequence[ComposeReq]):
+    arr = (kdn_compose_req * max(1, len(reqs)))()
+    keep = []
+    for i, r in enumerate(reqs):
+        n = len(r.parts)
+        parts = (kdn_chunk * max(1, n))(*[p.c() for p in r.parts])
+        pos = (C.c_int64 * max(1, n))(*[int(x) for x in r.part_dst_pos])
+        keep.append((parts, pos))
+        arr[i] = kdn_compose_req(r.block_table, r.n_table_blocks, n, C.cast(parts, C.POINTER(kdn_chunk)),
+                                 C.cast(pos, C.POINTER(C.c_int64)), float(r.rope_theta), r.rope_style, 0)
+    arr._keep = keep
+    return arr
+
+
+# ------------------------------------------------------------------------- the C ABI's calls --
+
+def kdn_strerror(status: int) -> str:
+    return lib.kdn_strerror(int(status)).decode()
+
+
+def kdn_create(device: int = 0) -> C.c_void_p:
+    ctx = C.c_void_p()
+    _check(lib.kdn_create(C.byref(ctx), int(device)), "kdn_create")
+    return ctx
+
+
+def kdn_destroy(ctx) -> None:
+    lib.kdn_destroy(ctx)
+
+
+def kdn_pool_register(ctx, desc: kdn_pool_desc) -> int:
+    pid = C.c_int(-1)
+    _check(lib.kdn_pool_register(ctx, C.byref(desc), C.byref(pid)), "kdn_pool_register")
+    return pid.value
+
+
+def kdn_chunk_bytes(desc: kdn_pool_desc, n_tokens: int, codec: int) -> int:
+    return int(lib.kdn_chunk_bytes(C.byref(desc), int(n_tokens), int(codec)))
+
+
+def kdn_validate_xfer(desc: kdn_pool_desc, ops: Sequence[XferOp]) -> int:
+    return int(lib.kdn_validate_xfer(C.byref(desc), xfer_array(ops), len(ops)))
+
+
+def kdn_validate_compose(desc: kdn_pool_desc, reqs: Sequence[ComposeReq]) -> int:
+    return int(lib.kdn_validate_compose(C.byref(desc), compose_array(reqs), len(reqs)))
+
+
+def kdn_store(ctx, pool_id: int, ops: Sequence[XferOp], stream: int = 0, side_stream: int = 0) -> None:
+    _check(lib.kdn_store(ctx, pool_id, xfer_array(ops), len(ops), stream, side_stream), "kdn_store")
+
+
+def kdn_retrieve(ctx, pool_id: int, ops: Sequence[XferOp], stream: int = 0, side_stream: int = 0) -> None:
+    _check(lib.kdn_retrieve(ctx, pool_id, xfer_array(ops), len(ops), stream, side_stream), "kdn_retrieve")
+
+
+def kdn_compose(ctx, pool_id: int, reqs: Sequence[ComposeReq], stream: int = 0, side_stream: int = 0) -> None:
+    _check(lib.kdn_compose(ctx, pool_id, compose_array(reqs), len(reqs), stream, side_stream), "kdn_compose")
+
+
+def kdn_status_sync(ctx, stream: int = 0) -> int:
+    return int(lib.kdn_status_sync(ctx, stream))
+
+
+def kdn_set_tuning(ctx, tile_bytes: int = 0, stages: int = 0, ctas_per_sm: int = 0) -> None:
+    t = kdn_tuning(tile_bytes, stages, ctas_per_sm, 0)
+    _check(lib.kdn_set_tuning(ctx, C.byref(t)), "kdn_set_tuning")
+
+
+def kdn_set_staging_bytes(ctx, bytes_per_slab: int) -> None:
+    _check(lib.kdn_set_staging_bytes(ctx, int(bytes_per_slab)), "kdn_set_staging_bytes")
+
+
+def kdn_launch_count(ctx) -> int:
+    return int(lib.kdn_launch_count(ctx))
