@@ -199,6 +199,12 @@ def run_gpu(args) -> None:
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
     shape = synth.LLAMA3_8B
+    global N_CHUNKS, N_PARTS
+    reduced = bool(args.pool_blocks or args.chunks or args.parts)
+    if args.pool_blocks:
+        shape = shape.with_(n_blocks=args.pool_blocks)
+    N_CHUNKS = args.chunks or N_CHUNKS
+    N_PARTS = args.parts or N_PARTS
 
     # ---- inputs (untimed): pool, tables, chunk buffers; every rank has its own copy of the same workload
     k, v = synth.make_pool(shape, dev, seed=synth.SEED_VALUES + rank)
@@ -314,6 +320,12 @@ def run_gpu(args) -> None:
              for i, n in enumerate(names)}
 
     # ---- end to end: the same step with every chunk in page-locked host memory
+    if args.no_e2e:
+        if rank == 0:
+            print(json.dumps({"note": "profiling run, not a bench record", "ops_ms": op_ms,
+                              "ops_gbs": {n: op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 for n in names}}))
+        K.kdn_destroy(ctx)
+        return
     host_sets = make_sets(True)
     for codec in (RAW, INT8):
         K.kdn_store(ctx, pid, host_sets[codec]["part_store"], s)
@@ -375,7 +387,7 @@ def run_gpu(args) -> None:
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16/int8 (fp32 codec and rotation, fp64 angles)", "data": "synthetic",
-            "config": {"workload": WORKLOAD, "l2": "inputs larger than L2 (every op streams >= 1.9 GB once)",
+            "config": {"workload": WORKLOAD if not reduced else "REDUCED (%d chunks, %d parts, %d blocks): not the bench workload" % (N_CHUNKS, N_PARTS, shape.n_blocks), "l2": "inputs larger than L2 (every op streams >= 1.9 GB once)",
                        "bytes_per_step": step_bytes},
             "tokens_per_s_reloaded": world * reload_tokens / (sum(op_ms[n] for n in names if not n.startswith("store")) * 1e-3),
             "ops": ops,
@@ -408,6 +420,10 @@ def main() -> None:
     ap.add_argument("--impl", default="kdn", choices=["kdn", "reference"])
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true", help="skip the host-link leg (profiling runs)")
+    ap.add_argument("--pool-blocks", type=int, default=0, help="smaller pool for profiler captures (default 16384)")
+    ap.add_argument("--chunks", type=int, default=0, help="chunks per store/retrieve batch (default 64)")
+    ap.add_argument("--parts", type=int, default=0, help="parts per composed request (default 10)")
     args = ap.parse_args()
     args.warmup = max(3, args.warmup) if args.impl == "kdn" else args.warmup
     if args.impl == "reference":
