@@ -184,6 +184,48 @@ kdn_status kdn_retrieve(kdn_ctx *ctx, int pool_id, const kdn_xfer_op *ops, int n
 kdn_status kdn_compose(kdn_ctx *ctx, int pool_id, const kdn_compose_req *reqs, int n_reqs,
                        void *cuda_stream, void *side_stream);
 
+/* Limits of kdn_compose_static: one call may carry at most KDN_STATIC_MAX_PARTS parts (summed over
+ * its requests), on a pool of at most KDN_STATIC_MAX_LAYERS layers and head_dim <= KDN_STATIC_MAX_HEAD_DIM.
+ * The fixed device array behind it is KDN_STATIC_SCRATCH_BYTES bytes. */
+#define KDN_STATIC_MAX_PARTS     128
+#define KDN_STATIC_MAX_LAYERS    128
+#define KDN_STATIC_MAX_HEAD_DIM  512
+#define KDN_STATIC_SCRATCH_BYTES 274688
+
+/* kdn_compose for callers that must not allocate device memory.  (The paper has no counterpart to
+ * this call; it exists for integration reasons only.)
+ *
+ * Who needs it: an engine that handed all of the GPU's memory to its own allocator at start-up, so a
+ * cudaMalloc from a library would fail; a thread that runs while another thread captures a CUDA graph
+ * in global capture mode, where cudaMalloc is an error; a latency-critical loop that cannot take the
+ * device-wide synchronisation cudaMalloc and cudaFree may imply.  kdn_create and kdn_pool_register
+ * allocate (descriptor ring, pointer arrays, rotation table), so such callers cannot use a context.
+ *
+ * This call needs no context and calls no cudaMalloc, cudaFree or other allocating routine.  Its
+ * scratch -- the device copies of the pool's layer pointers, the part records, the rotation table and
+ * a status word -- lives in one fixed array inside the library's device image.  Every GPU that loads
+ * the library holds those KDN_STATIC_SCRATCH_BYTES bytes until the process exits.
+ *
+ * Arguments are those of kdn_pool_register (pool) and kdn_compose (reqs, n_reqs, cuda_stream), with
+ * the same layouts, preconditions and results: a part whose position is unchanged is written exactly
+ * as kdn_retrieve writes it, so the call also serves as a retrieve.  device is the CUDA device that
+ * owns the pool; it is made current.  Only KDN_MEM_DEVICE parts are accepted (staging slabs would
+ * have to be allocated).  Sizes beyond the limits above return KDN_E_UNSUPPORTED and enqueue nothing.
+ * The built-in launch shape is used; kdn_set_tuning does not apply.
+ *
+ * wait != 0: the call waits for cuda_stream and returns the first error the kernels recorded
+ * (KDN_E_RANGE for a block id outside the pool, ...), or KDN_OK.  wait == 0: the call returns after
+ * enqueueing; errors found on the device by that call are then not reported.
+ *
+ * The first call on each device looks up the array's device address (a one-time set-up step);
+ * make that first call before any stream capture begins.  All calls on a device share the one array,
+ * and it still holds the previous call's records when the next call starts: each call rewrites the
+ * records it uses and clears the status word, on cuda_stream, before its kernels run.  Two calls
+ * whose work can overlap on the GPU (different streams without an ordering between them) therefore
+ * race on the array and corrupt each other; issue them on one stream or order them yourself. */
+kdn_status kdn_compose_static(int device, const kdn_pool_desc *pool, const kdn_compose_req *reqs, int n_reqs,
+                              void *cuda_stream, int wait);
+
 /* Wait for cuda_stream (and the context's side stream) and return the first error a kernel of this
  * context recorded since the last call of this function, or KDN_OK. */
 kdn_status kdn_status_sync(kdn_ctx *ctx, void *cuda_stream);

@@ -7,6 +7,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -651,3 +652,192 @@ const char *kdn_strerror(kdn_status status)
 }
 
 }  // extern "C"
+
+// ------------------------------------------------------------------------------------------------
+// kdn_compose_static: compose without any device allocation (no paper counterpart; see kdn.h).
+// Its scratch is this fixed array in the library's device image.  Layout (byte offsets):
+//   0      int status                      (256 bytes reserved)
+//   256    void *k_layers[128]
+//   1280   void *v_layers[128]
+//   2304   DevOp ops[128]
+//   10496  RopeParam rope[128]
+//   12544  float2 table[128 * 256]         (rows x head_dim/2, packed by the call's head_dim)
+// In host code `g_static_scratch` is only a handle for cudaGetSymbolAddress, never an address to
+// hand to a kernel.
+static __device__ __align__(256) unsigned char g_static_scratch[KDN_STATIC_SCRATCH_BYTES];
+
+namespace {
+
+constexpr size_t kStOffK = 256, kStOffV = 1280, kStOffOps = 2304, kStOffRope = 10496, kStOffTable = 12544;
+constexpr size_t kStHeadBytes = kStOffTable;                 // everything the host uploads per call
+constexpr int kStMaxDevices = 64;
+static_assert(kStOffTable + sizeof(float2) * KDN_STATIC_MAX_PARTS * (KDN_STATIC_MAX_HEAD_DIM / 2) == KDN_STATIC_SCRATCH_BYTES,
+              "scratch layout and KDN_STATIC_SCRATCH_BYTES disagree");
+static_assert(kStOffRope - kStOffOps == sizeof(DevOp) * KDN_STATIC_MAX_PARTS, "ops area");
+static_assert(kStOffTable - kStOffRope == sizeof(RopeParam) * KDN_STATIC_MAX_PARTS, "rope area");
+
+struct StaticDev {
+    unsigned char *base = nullptr;          // device address of g_static_scratch on this device
+    int sm_count = 0;
+    int smem_optin = 0;
+};
+StaticDev g_static_dev[kStMaxDevices];
+std::mutex g_static_mutex;
+
+// One-time set-up per device, with that device current: resolve the array's device address.
+kdn_status static_setup(int device, StaticDev **out)
+{
+    if (device < 0 || device >= kStMaxDevices) return KDN_E_UNSUPPORTED;
+    std::lock_guard<std::mutex> lock(g_static_mutex);
+    StaticDev &d = g_static_dev[device];
+    if (!d.base) {
+        int major = 0;
+        KDN_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device));
+        if (major < 10) return KDN_E_UNSUPPORTED;
+        KDN_CUDA(cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, device));
+        KDN_CUDA(cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device));
+        void *ptr = nullptr;
+        KDN_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
+        if (!ptr) return KDN_E_CUDA;
+        d.base = (unsigned char *)ptr;
+    }
+    *out = &d;
+    return KDN_OK;
+}
+
+}  // namespace
+
+extern "C" kdn_status kdn_compose_static(int device, const kdn_pool_desc *pool, const kdn_compose_req *reqs, int n_reqs,
+                                         void *cuda_stream, int wait)
+{
+    kdn_status st = kdn_validate_compose(pool, reqs, n_reqs);
+    if (st != KDN_OK) return st;
+    if (!pool->k_layers || !pool->v_layers) return KDN_E_INVAL;
+    if (pool->n_layers > KDN_STATIC_MAX_LAYERS || pool->head_dim > KDN_STATIC_MAX_HEAD_DIM) return KDN_E_UNSUPPORTED;
+    long long n_parts = 0;
+    for (int r = 0; r < n_reqs; ++r) {
+        for (int j = 0; j < reqs[r].n_parts; ++j) {
+            if (reqs[r].parts[j].n_tokens == 0) continue;
+            if (reqs[r].parts[j].mem != KDN_MEM_DEVICE) return KDN_E_UNSUPPORTED;
+            ++n_parts;
+        }
+        if (n_parts > KDN_STATIC_MAX_PARTS) return KDN_E_UNSUPPORTED;
+    }
+    for (int l = 0; l < pool->n_layers; ++l) {
+        if (!pool->k_layers[l] || !pool->v_layers[l]) return KDN_E_INVAL;
+        if ((uintptr_t)pool->k_layers[l] % 16 || (uintptr_t)pool->v_layers[l] % 16) return KDN_E_ALIGN;
+    }
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) return KDN_E_CUDA;
+    KDN_CUDA(cudaSetDevice(device));
+    StaticDev *sd = nullptr;
+    st = static_setup(device, &sd);
+    if (st != KDN_OK) return st;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+
+    Pool p;
+    p.L = pool->n_layers; p.H = pool->n_kv_heads; p.D = pool->head_dim; p.bs = pool->block_size; p.nb = pool->n_blocks;
+    const unsigned row_elems = (unsigned)p.H * (unsigned)p.D;
+
+    // host image of the scratch head: status word (zero), layer pointers, part records, rotation rows
+    alignas(16) unsigned char head[kStHeadBytes];
+    std::memset(head, 0, sizeof head);
+    std::memcpy(head + kStOffK, pool->k_layers, sizeof(void *) * (size_t)p.L);
+    std::memcpy(head + kStOffV, pool->v_layers, sizeof(void *) * (size_t)p.L);
+    DevOp *ops = reinterpret_cast<DevOp *>(head + kStOffOps);
+    RopeParam *rope = reinterpret_cast<RopeParam *>(head + kStOffRope);
+
+    // launch shape: the library defaults for a compose launch
+    bool any_int8 = false, any_rot = false;
+    for (int r = 0; r < n_reqs; ++r)
+        for (int j = 0; j < reqs[r].n_parts; ++j) {
+            if (reqs[r].parts[j].n_tokens == 0) continue;
+            any_int8 |= reqs[r].parts[j].codec == KDN_CODEC_INT8_G64;
+            any_rot |= reqs[r].part_dst_pos[j] != reqs[r].parts[j].base_pos;
+        }
+    const bool compute = any_int8 || any_rot;
+    unsigned unit = 8;
+    if (any_int8) unit = lcm_u(unit, 64);
+    if (any_rot) unit = lcm_u(unit, (unsigned)p.D);
+    unsigned tile_elems = (compute ? 8192u : 16384u) / 2u / unit * unit;
+    if (tile_elems < unit) tile_elems = unit;
+    const unsigned long long block_elems = (unsigned long long)p.bs * row_elems;
+    if (tile_elems > block_elems) tile_elems = (unsigned)((block_elems + unit - 1) / unit * unit);
+    const unsigned tpb = (unsigned)((block_elems + tile_elems - 1) / tile_elems);
+    const unsigned a_bytes = (tile_elems * 2u + 127u) & ~127u;
+    const unsigned b_bytes = compute ? ((tile_elems + 127u) & ~127u) : 0u;
+    const unsigned s_bytes = compute ? ((tile_elems / 16u + 127u) & ~127u) : 0u;
+    const unsigned stage_bytes = a_bytes + b_bytes + s_bytes;
+    const int ctas_per_sm = 2;
+    int stages = compute ? 8 : 6;
+    const size_t smem_limit = (size_t)sd->smem_optin;
+    while (stages > kStoreLag + 2 && smem_bytes(stages, stage_bytes) * (size_t)ctas_per_sm > smem_limit - 1024u * (size_t)ctas_per_sm)
+        --stages;
+    const size_t smem = smem_bytes(stages, stage_bytes);
+    if (smem > smem_limit) return KDN_E_UNSUPPORTED;
+
+    unsigned long long tiles = 0;
+    int n = 0, n_rope = 0;
+    for (int r = 0; r < n_reqs; ++r) {
+        const kdn_compose_req &q = reqs[r];
+        for (int j = 0; j < q.n_parts; ++j) {
+            const kdn_chunk &c = q.parts[j];
+            if (c.n_tokens == 0) continue;
+            HostOp h = make_host_op(p, q.block_table, q.part_dst_pos[j], c);
+            DevOp op = h.op;
+            op.tile_begin = (unsigned)tiles;
+            const long long delta = (long long)(q.part_dst_pos[j] - c.base_pos);
+            if (delta != 0) {
+                rope[n_rope].delta = delta;
+                rope[n_rope].theta = q.rope_theta;
+                op.rope = n_rope++;
+            }
+            ops[n++] = op;
+            tiles += (unsigned long long)op.nl * 2ull * (unsigned long long)op.nblk * tpb;
+            if (tiles > kMaxTilesPerLaunch) return KDN_E_UNSUPPORTED;
+        }
+    }
+    const int half = p.D / 2;
+    if ((size_t)n_rope * (size_t)half > (size_t)KDN_STATIC_MAX_PARTS * (KDN_STATIC_MAX_HEAD_DIM / 2)) return KDN_E_UNSUPPORTED;
+
+    // upload the head (this also clears the status word); the source is ordinary host memory, so the
+    // runtime has taken its copy of `head` by the time the call returns
+    KDN_CUDA(cudaMemcpyAsync(sd->base, head, kStHeadBytes, cudaMemcpyHostToDevice, stream));
+    if (tiles != 0) {
+        float2 *d_table = reinterpret_cast<float2 *>(sd->base + kStOffTable);
+        if (n_rope) {
+            const long long total = (long long)n_rope * half;
+            kdn_rope_table_kernel<<<(unsigned)((total + 127) / 128), 128, 0, stream>>>(
+                reinterpret_cast<const RopeParam *>(sd->base + kStOffRope), n_rope, p.D, d_table);
+            KDN_CUDA(cudaGetLastError());
+        }
+        Launch lp{};
+        lp.ops = reinterpret_cast<const DevOp *>(sd->base + kStOffOps);
+        lp.n_ops = n;
+        lp.n_tiles = (unsigned)tiles;
+        lp.k_layers = reinterpret_cast<void *const *>(sd->base + kStOffK);
+        lp.v_layers = reinterpret_cast<void *const *>(sd->base + kStOffV);
+        lp.n_blocks = p.nb;
+        lp.bs = p.bs;
+        lp.D = p.D;
+        lp.row_elems = row_elems;
+        lp.tile_elems = tile_elems;
+        lp.tpb = tpb;
+        lp.rope = d_table;
+        lp.status = reinterpret_cast<int *>(sd->base);
+        lp.stages = stages;
+        lp.stage_bytes = stage_bytes;
+        lp.off_b = a_bytes;
+        lp.off_s = a_bytes + b_bytes;
+        const unsigned long long want = (unsigned long long)sd->sm_count * (unsigned)ctas_per_sm;
+        const unsigned grid = (unsigned)(tiles < want ? tiles : want);
+        st = compute ? launch_kernel(kdn_compose_kernel<true>, kThreadsCompute, grid, smem, stream, lp)
+                     : launch_kernel(kdn_compose_kernel<false>, kThreadsCopy, grid, smem, stream, lp);
+        if (st != KDN_OK) return st;
+    }
+    if (!wait) return KDN_OK;
+    KDN_CUDA(cudaStreamSynchronize(stream));
+    int dev_status = 0;
+    KDN_CUDA(cudaMemcpy(&dev_status, sd->base, sizeof(int), cudaMemcpyDeviceToHost));
+    return (dev_status >= KDN_OK && dev_status <= KDN_E_TIMEOUT) ? (kdn_status)dev_status : KDN_E_CUDA;
+}

@@ -20,7 +20,8 @@ KDN_MEM_DEVICE, KDN_MEM_PINNED_HOST = 0, 1
 
 EXPORTS = ["kdn_create", "kdn_destroy", "kdn_pool_register", "kdn_chunk_bytes", "kdn_validate_xfer",
            "kdn_validate_compose", "kdn_store", "kdn_retrieve", "kdn_compose", "kdn_status_sync",
-           "kdn_set_tuning", "kdn_set_staging_bytes", "kdn_launch_count", "kdn_strerror"]
+           "kdn_set_tuning", "kdn_set_staging_bytes", "kdn_launch_count", "kdn_strerror",
+           "kdn_compose_static"]
 
 
 class kdn_pool_desc(C.Structure):
@@ -78,6 +79,8 @@ def _load() -> C.CDLL:
         fn.argtypes = [vp, i32, C.POINTER(kdn_xfer_op), i32, vp, vp]
     lib.kdn_compose.restype = i32
     lib.kdn_compose.argtypes = [vp, i32, C.POINTER(kdn_compose_req), i32, vp, vp]
+    lib.kdn_compose_static.restype = i32
+    lib.kdn_compose_static.argtypes = [i32, C.POINTER(kdn_pool_desc), C.POINTER(kdn_compose_req), i32, vp, i32]
     lib.kdn_status_sync.restype = i32
     lib.kdn_status_sync.argtypes = [vp, vp]
     lib.kdn_set_tuning.restype = i32
@@ -216,6 +219,14 @@ def kdn_retrieve(ctx, pool_id: int, ops: Sequence[XferOp], stream: int = 0, side
 
 def kdn_compose(ctx, pool_id: int, reqs: Sequence[ComposeReq], stream: int = 0, side_stream: int = 0) -> None:
     _check(lib.kdn_compose(ctx, pool_id, compose_array(reqs), len(reqs), stream, side_stream), "kdn_compose")
+
+
+def kdn_compose_static(device: int, desc: kdn_pool_desc, reqs: Sequence[ComposeReq], stream: int = 0,
+                       wait: bool = True) -> int:
+    """kdn_compose without a context and without any device allocation (fixed scratch inside the library).
+
+    Returns the status code instead of raising: an argument error, or (with ``wait``) what the kernels recorded."""
+    return int(lib.kdn_compose_static(int(device), C.byref(desc), compose_array(reqs), len(reqs), stream, 1 if wait else 0))
 
 
 def kdn_status_sync(ctx, stream: int = 0) -> int:
