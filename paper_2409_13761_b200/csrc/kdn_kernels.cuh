@@ -11,7 +11,8 @@
 // Pipeline inside a CTA (S slots of shared memory, all hand-offs through mbarriers):
 //   loader warp   decodes tiles 32 at a time (one per lane: op lookup, block-table entry, addresses),
 //                 then issues each tile's bulk async copies global -> shared
-//   compute warps (4) int8 coding / decoding and key rotation, shared -> shared
+//   compute warps (2 groups of 4; group g owns slots g, g+2, ...) int8 coding / decoding and key
+//                 rotation, shared -> shared
 //   storer thread issues the bulk async copy shared -> global and recycles the slot
 // Tiles that are a pure copy (raw bf16 without rotation) never touch the compute warps' ALUs.
 // Every mbarrier wait is bounded by a wall-clock limit; on expiry the CTA records KDN_E_TIMEOUT,
@@ -25,7 +26,10 @@
 namespace kdn {
 
 constexpr int kLoaderWarp = 0;
-constexpr int kComputeWarps = 4;
+constexpr int kGroupWarps = 4;                // warps that work together on one tile
+constexpr int kGroupThreads = kGroupWarps * 32;
+constexpr int kComputeGroups = 2;             // groups take alternate pipeline slots (group_bar_sync knows two)
+constexpr int kComputeWarps = kGroupWarps * kComputeGroups;
 constexpr int kComputeThreads = kComputeWarps * 32;
 constexpr int kThreadsCompute = 32 + kComputeThreads + 32;   // loader + compute + storer
 constexpr int kThreadsCopy = 64;                             // loader + storer
@@ -158,9 +162,10 @@ template <int N> __device__ __forceinline__ void bulk_wait_read()
 }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void compute_bar_sync()
+__device__ __forceinline__ void group_bar_sync(int group)
 {
-    asm volatile("bar.sync 1, %0;" ::"n"(kComputeThreads) : "memory");
+    if (group == 0) asm volatile("bar.sync 1, %0;" ::"n"(kGroupThreads) : "memory");
+    else            asm volatile("bar.sync 2, %0;" ::"n"(kGroupThreads) : "memory");
 }
 
 __device__ __forceinline__ uint4 lds128(const void *p) { return *reinterpret_cast<const uint4 *>(p); }
@@ -200,35 +205,56 @@ template <int K> __device__ __forceinline__ float code_to_float(uint32_t w_biase
 
 // Encode n elements (a multiple of 64) of bf16 at A into int8 codes at B and one fp32 scale per 64
 // elements (to shared S, or straight to global when the destination is not 16-byte aligned).
-// 8 lanes share a group; the absmax is reduced with three shuffles.
+// Two lanes share a group, 32 elements each, read as four 128-bit shared loads in a lane-rotated
+// order (bank-conflict free); the absmax is reduced with one shuffle; the two IEEE divides are
+// issued once per 32 elements.  ct is the thread's index inside its compute group.
 __device__ __forceinline__ void quantise_tile(const unsigned char *A, unsigned char *B, float *S, float *g_scales,
                                               unsigned n, int ct)
 {
-    const unsigned nvec = n >> 3;
+    const unsigned nhalf = n >> 5;                         // 32-element half groups
     const unsigned lane = (unsigned)ct & 31u;
-    for (unsigned vb = (unsigned)ct & ~31u; vb < nvec; vb += kComputeThreads) {
-        const unsigned v = vb + lane;
-        const bool act = v < nvec;
-        uint4 x = act ? lds128(A + (size_t)v * 16u) : make_uint4(0u, 0u, 0u, 0u);
-        float f[8] = { bf16_lo(x.x), bf16_hi(x.x), bf16_lo(x.y), bf16_hi(x.y),
-                       bf16_lo(x.z), bf16_hi(x.z), bf16_lo(x.w), bf16_hi(x.w) };
-        float a = 0.0f;
+    const unsigned rot = (lane >> 1) & 3u;
+    for (unsigned hb = (unsigned)ct & ~31u; hb < nhalf; hb += kGroupThreads) {
+        const unsigned h = hb + lane;
+        const bool act = h < nhalf;
+        const unsigned char *src = A + (size_t)h * 64u;
+        uint4 x[4];
 #pragma unroll
-        for (int k = 0; k < 8; ++k) a = fmaxf(a, fabsf(f[k]));
+        for (int j = 0; j < 4; ++j)
+            x[j] = act ? lds128(src + (((unsigned)j + rot) & 3u) * 16u) : make_uint4(0u, 0u, 0u, 0u);
+        float f[32];
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            f[8 * j + 0] = bf16_lo(x[j].x); f[8 * j + 1] = bf16_hi(x[j].x);
+            f[8 * j + 2] = bf16_lo(x[j].y); f[8 * j + 3] = bf16_hi(x[j].y);
+            f[8 * j + 4] = bf16_lo(x[j].z); f[8 * j + 5] = bf16_hi(x[j].z);
+            f[8 * j + 6] = bf16_lo(x[j].w); f[8 * j + 7] = bf16_hi(x[j].w);
+        }
+        float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
+#pragma unroll
+        for (int k = 0; k < 32; k += 4) {
+            a0 = fmaxf(a0, fabsf(f[k])); a1 = fmaxf(a1, fabsf(f[k + 1]));
+            a2 = fmaxf(a2, fabsf(f[k + 2])); a3 = fmaxf(a3, fabsf(f[k + 3]));
+        }
+        float a = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3));
         a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
-        a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 2));
-        a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 4));
         float scale = __fdiv_rn(a, 127.0f);
         const bool ok = scale >= 1.17549435e-38f;         // smallest normal fp32; false for NaN too
         const float inv = ok ? __fdiv_rn(127.0f, a) : 0.0f;
         scale = ok ? scale : 0.0f;
         if (act) {
-            uint2 q;
-            q.x = pack_codes4(code_bits(f[0], inv), code_bits(f[1], inv), code_bits(f[2], inv), code_bits(f[3], inv));
-            q.y = pack_codes4(code_bits(f[4], inv), code_bits(f[5], inv), code_bits(f[6], inv), code_bits(f[7], inv));
-            sts64(B + (size_t)v * 8u, q);
-            if ((lane & 7u) == 0u) {
-                if (g_scales) g_scales[v >> 3] = scale; else S[v >> 3] = scale;
+            unsigned char *dst = B + (size_t)h * 32u;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                uint2 q;
+                q.x = pack_codes4(code_bits(f[8 * j + 0], inv), code_bits(f[8 * j + 1], inv),
+                                  code_bits(f[8 * j + 2], inv), code_bits(f[8 * j + 3], inv));
+                q.y = pack_codes4(code_bits(f[8 * j + 4], inv), code_bits(f[8 * j + 5], inv),
+                                  code_bits(f[8 * j + 6], inv), code_bits(f[8 * j + 7], inv));
+                sts64(dst + (((unsigned)j + rot) & 3u) * 8u, q);
+            }
+            if ((lane & 1u) == 0u) {
+                if (g_scales) g_scales[h >> 1] = scale; else S[h >> 1] = scale;
             }
         }
     }
@@ -239,7 +265,7 @@ __device__ __forceinline__ void dequantise_tile(const unsigned char *B, const fl
                                                 unsigned n, int ct)
 {
     const unsigned nvec = n >> 4;
-    for (unsigned v = (unsigned)ct; v < nvec; v += kComputeThreads) {
+    for (unsigned v = (unsigned)ct; v < nvec; v += kGroupThreads) {
         const uint4 c = lds128(B + (size_t)v * 16u);
         const float sc = S[v >> 2];
         const uint32_t w[4] = { c.x ^ 0x80808080u, c.y ^ 0x80808080u, c.z ^ 0x80808080u, c.w ^ 0x80808080u };
@@ -294,9 +320,11 @@ __device__ __forceinline__ void rotate_tile(unsigned char *A, const unsigned cha
 {
     const unsigned half = D >> 1;
     const unsigned per_row = D >> 4;                      // work items per head row
+    const bool pow2 = (per_row & (per_row - 1u)) == 0u;
+    const unsigned shift = 31u - (unsigned)__clz(per_row);
     const unsigned items = n >> 4;
-    for (unsigned it = (unsigned)ct; it < items; it += kComputeThreads) {
-        const unsigned r = it / per_row;
+    for (unsigned it = (unsigned)ct; it < items; it += kGroupThreads) {
+        const unsigned r = pow2 ? it >> shift : it / per_row;
         const unsigned col = (it - r * per_row) << 3;
         load_coef(rc, table, rope, col, half);
         const unsigned e_lo = r * D + col, e_hi = e_lo + half;
@@ -423,7 +451,7 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
         for (int s = 0; s < S; ++s) {
             mbar_init(sm.full + 8u * s, 1u);
             mbar_init(sm.empty + 8u * s, 1u);
-            mbar_init(sm.ready + 8u * s, (uint32_t)kComputeWarps);
+            mbar_init(sm.ready + 8u * s, (uint32_t)kGroupWarps);
         }
         *sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -534,10 +562,11 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
         }
     } else if (kCompute) {
         // ----------------------------------------------------------- compute
-        const int ct = tid - 32;
+        const int group = (tid - 32) / kGroupThreads;       // this group owns slots group, group + 2, ...
+        const int ct = (tid - 32) % kGroupThreads;
         RotCoef rc;
         rc.rope = -1; rc.col = 0xffffffffu;
-        for (unsigned slot = 0; slot < n_my; ++slot) {
+        for (unsigned slot = (unsigned)group; slot < n_my; slot += (unsigned)kComputeGroups) {
             const unsigned st = slot % (unsigned)S;
             const uint32_t ph = (slot / (unsigned)S) & 1u;
             if (!mbar_wait(sm.full + 8u * st, ph, sm.abort_flag)) break;
@@ -557,8 +586,8 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                 } else if (flags & TF_INT8) {
                     if (flags & TF_SCALES_PLAIN) {
                         const float *gs = reinterpret_cast<const float *>(sm.desc[st].g_scales);
-                        for (unsigned i = (unsigned)ct; i < (n >> 6); i += kComputeThreads) Sc[i] = __ldg(gs + i);
-                        compute_bar_sync();
+                        for (unsigned i = (unsigned)ct; i < (n >> 6); i += kGroupThreads) Sc[i] = __ldg(gs + i);
+                        group_bar_sync(group);
                     }
                     if (OP == OP_COMPOSE && (flags & TF_ROTATE))
                         rotate_tile<true>(A, B, Sc, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct);
