@@ -133,11 +133,16 @@ typedef struct {
 
 /* Launch shape of the tile pipeline.  0 in a field keeps the built-in default.  tile_bytes: bf16
  * bytes moved per pipeline slot (multiple of 128); stages: slots per CTA; ctas_per_sm: persistent
- * CTAs per SM.  Settings that do not fit in shared memory are rejected with KDN_E_UNSUPPORTED. */
+ * CTAs per SM; compute_groups: groups of four compute warps per CTA in launches that code, decode or
+ * rotate (1, 2, 3, 4 or 6); store_lag: how many shared-to-global copies may still be draining before
+ * the storer waits (1..4).  stages is raised to store_lag + 2 and rounded down to a multiple of
+ * compute_groups.  Settings that do not fit in shared memory are rejected with KDN_E_UNSUPPORTED. */
 typedef struct {
     int32_t tile_bytes;
     int32_t stages;
     int32_t ctas_per_sm;
+    int32_t compute_groups;
+    int32_t store_lag;
     int32_t reserved;   /* 0 */
 } kdn_tuning;
 

@@ -143,6 +143,50 @@ kdn_status launch_kernel(K kernel, int threads, unsigned grid, size_t smem, cuda
     return KDN_OK;
 }
 
+// Built-in launch shapes, from sweeps on 8B-shaped KV with fully fragmented tables on B200.  The copy
+// form runs best with about two tiles of loads and two of stores in flight per SM; deeper queues lose
+// 3-4 % of bandwidth.  The coding forms want more compute warps per SM than the copy form needs.
+struct Shape { int tile_bytes, stages, ctas_per_sm, groups, lag; };
+Shape default_shape(int OP, bool any_int8, bool any_rot)
+{
+    if (!any_int8 && !any_rot) return Shape{ 32768, 4, 1, 0, 2 };
+    if (OP == OP_STORE) return Shape{ 16384, 9, 1, 3, 2 };
+    if (OP == OP_RETRIEVE || !any_rot) return Shape{ 8192, 6, 3, 2, 2 };
+    if (!any_int8) return Shape{ 8192, 6, 2, 2, 2 };
+    return Shape{ 16384, 9, 1, 3, 2 };
+}
+
+// Pipeline slots: at least lag + 2, a multiple of the compute groups (a slot must always belong to the
+// same group), and, unless the caller fixed the count, few enough for ctas_per_sm CTAs to share an SM.
+kdn_status fit_stages(int &stages, int groups, int lag, bool shrink, unsigned stage_bytes, int ctas_per_sm, size_t smem_limit)
+{
+    const int g = groups > 0 ? groups : 1;
+    if (stages > kMaxStages) stages = kMaxStages;
+    int min_stages = (lag + 2 + g - 1) / g * g;
+    if (stages < min_stages) stages = min_stages;
+    stages = stages / g * g;
+    if (shrink)
+        while (stages - g >= min_stages &&
+               smem_bytes(stages, stage_bytes) * (size_t)ctas_per_sm > smem_limit - 1024u * (size_t)ctas_per_sm)
+            stages -= g;
+    return smem_bytes(stages, stage_bytes) > smem_limit ? KDN_E_UNSUPPORTED : KDN_OK;
+}
+
+// Launch the instantiation for (OP, compute groups); groups = 0 is the pure-copy form.
+kdn_status launch_tiles(int OP, int groups, unsigned grid, size_t smem, cudaStream_t stream, const Launch &lp)
+{
+#define KDN_CASE(G)                                                                                         \
+    case G:                                                                                                 \
+        if (OP == OP_STORE) return launch_kernel(kdn_store_kernel<G>, threads_for(G), grid, smem, stream, lp);      \
+        if (OP == OP_RETRIEVE) return launch_kernel(kdn_retrieve_kernel<G>, threads_for(G), grid, smem, stream, lp); \
+        return launch_kernel(kdn_compose_kernel<G>, threads_for(G), grid, smem, stream, lp);
+    switch (groups) {
+        KDN_CASE(0) KDN_CASE(1) KDN_CASE(2) KDN_CASE(3) KDN_CASE(4) KDN_CASE(6)
+    }
+#undef KDN_CASE
+    return KDN_E_UNSUPPORTED;
+}
+
 // Tile one batch of host ops (at most kMaxOpsPerLaunch, all on the device side) and launch it.
 kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *hops, int n, cudaStream_t stream)
 {
@@ -159,7 +203,8 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     unsigned unit = 8;
     if (any_int8) unit = lcm_u(unit, 64);
     if (any_rot) unit = lcm_u(unit, (unsigned)pool.D);
-    int tile_bytes = ctx->tuning.tile_bytes > 0 ? ctx->tuning.tile_bytes : (compute ? 8192 : 16384);
+    const Shape def = default_shape(OP, any_int8, any_rot);
+    int tile_bytes = ctx->tuning.tile_bytes > 0 ? ctx->tuning.tile_bytes : def.tile_bytes;
     unsigned tile_elems = (unsigned)tile_bytes / 2u / unit * unit;
     if (tile_elems < unit) tile_elems = unit;
     const unsigned long long block_elems = (unsigned long long)pool.bs * row_elems;
@@ -170,16 +215,15 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     const unsigned b_bytes = compute ? ((tile_elems + 127u) & ~127u) : 0u;
     const unsigned s_bytes = compute ? ((tile_elems / 16u + 127u) & ~127u) : 0u;
     const unsigned stage_bytes = a_bytes + b_bytes + s_bytes;
-    int ctas_per_sm = ctx->tuning.ctas_per_sm > 0 ? ctx->tuning.ctas_per_sm : 2;
-    int stages = ctx->tuning.stages > 0 ? ctx->tuning.stages : (compute ? 8 : 6);
-    if (stages > kMaxStages) stages = kMaxStages;
-    if (stages < kStoreLag + 2) stages = kStoreLag + 2;
+    int groups = 0;
+    if (compute) groups = ctx->tuning.compute_groups > 0 ? ctx->tuning.compute_groups : def.groups;
+    const int lag = ctx->tuning.store_lag > 0 ? ctx->tuning.store_lag : def.lag;
+    int ctas_per_sm = ctx->tuning.ctas_per_sm > 0 ? ctx->tuning.ctas_per_sm : def.ctas_per_sm;
+    int stages = ctx->tuning.stages > 0 ? ctx->tuning.stages : def.stages;
     const size_t smem_limit = (size_t)ctx->smem_optin;
-    if (ctx->tuning.stages <= 0)
-        while (stages > kStoreLag + 2 && smem_bytes(stages, stage_bytes) * (size_t)ctas_per_sm > smem_limit - 1024u * (size_t)ctas_per_sm)
-            --stages;
+    kdn_status fit = fit_stages(stages, groups, lag, ctx->tuning.stages <= 0, stage_bytes, ctas_per_sm, smem_limit);
+    if (fit != KDN_OK) return fit;
     const size_t smem = smem_bytes(stages, stage_bytes);
-    if (smem > smem_limit) return KDN_E_UNSUPPORTED;
 
     RingSlot &slot = ctx->ring[ctx->ring_next++ % kRing];
     if (slot.used) KDN_CUDA(cudaEventSynchronize(slot.done));
@@ -237,19 +281,11 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     lp.stage_bytes = stage_bytes;
     lp.off_b = a_bytes;
     lp.off_s = a_bytes + b_bytes;
+    lp.store_lag = lag;
 
     unsigned long long want = (unsigned long long)ctx->sm_count * (unsigned)ctas_per_sm;
     const unsigned grid = (unsigned)(tiles < want ? tiles : want);
-    kdn_status st;
-    if (compute) {
-        if (OP == OP_STORE) st = launch_kernel(kdn_store_kernel<true>, kThreadsCompute, grid, smem, stream, lp);
-        else if (OP == OP_RETRIEVE) st = launch_kernel(kdn_retrieve_kernel<true>, kThreadsCompute, grid, smem, stream, lp);
-        else st = launch_kernel(kdn_compose_kernel<true>, kThreadsCompute, grid, smem, stream, lp);
-    } else {
-        if (OP == OP_STORE) st = launch_kernel(kdn_store_kernel<false>, kThreadsCopy, grid, smem, stream, lp);
-        else if (OP == OP_RETRIEVE) st = launch_kernel(kdn_retrieve_kernel<false>, kThreadsCopy, grid, smem, stream, lp);
-        else st = launch_kernel(kdn_compose_kernel<false>, kThreadsCopy, grid, smem, stream, lp);
-    }
+    kdn_status st = launch_tiles(OP, groups, grid, smem, stream, lp);
     if (st != KDN_OK) return st;
     ctx->launches++;
     KDN_CUDA(cudaEventRecord(slot.done, stream));
@@ -613,8 +649,12 @@ kdn_status kdn_set_tuning(kdn_ctx *ctx, const kdn_tuning *tuning)
     if (!tuning) { ctx->tuning = kdn_tuning{}; return KDN_OK; }
     if (tuning->tile_bytes < 0 || tuning->stages < 0 || tuning->ctas_per_sm < 0) return KDN_E_INVAL;
     if (tuning->tile_bytes % 128) return KDN_E_INVAL;
-    if (tuning->stages && (tuning->stages < kStoreLag + 2 || tuning->stages > kMaxStages)) return KDN_E_UNSUPPORTED;
+    if (tuning->stages > kMaxStages) return KDN_E_UNSUPPORTED;
+    if (tuning->store_lag < 0) return KDN_E_INVAL;
+    if (tuning->store_lag > kMaxStoreLag) return KDN_E_UNSUPPORTED;
     if (tuning->ctas_per_sm > 32) return KDN_E_UNSUPPORTED;
+    if (tuning->compute_groups < 0) return KDN_E_INVAL;
+    if (tuning->compute_groups > kMaxGroups || tuning->compute_groups == 5) return KDN_E_UNSUPPORTED;
     if (tuning->tile_bytes > ctx->smem_optin) return KDN_E_UNSUPPORTED;
     ctx->tuning = *tuning;
     return KDN_OK;
@@ -759,7 +799,8 @@ extern "C" kdn_status kdn_compose_static(int device, const kdn_pool_desc *pool, 
     unsigned unit = 8;
     if (any_int8) unit = lcm_u(unit, 64);
     if (any_rot) unit = lcm_u(unit, (unsigned)p.D);
-    unsigned tile_elems = (compute ? 8192u : 16384u) / 2u / unit * unit;
+    const Shape def = default_shape(OP_COMPOSE, any_int8, any_rot);
+    unsigned tile_elems = (unsigned)def.tile_bytes / 2u / unit * unit;
     if (tile_elems < unit) tile_elems = unit;
     const unsigned long long block_elems = (unsigned long long)p.bs * row_elems;
     if (tile_elems > block_elems) tile_elems = (unsigned)((block_elems + unit - 1) / unit * unit);
@@ -768,13 +809,12 @@ extern "C" kdn_status kdn_compose_static(int device, const kdn_pool_desc *pool, 
     const unsigned b_bytes = compute ? ((tile_elems + 127u) & ~127u) : 0u;
     const unsigned s_bytes = compute ? ((tile_elems / 16u + 127u) & ~127u) : 0u;
     const unsigned stage_bytes = a_bytes + b_bytes + s_bytes;
-    const int ctas_per_sm = 2;
-    int stages = compute ? 8 : 6;
+    const int ctas_per_sm = def.ctas_per_sm;
+    int stages = def.stages;
     const size_t smem_limit = (size_t)sd->smem_optin;
-    while (stages > kStoreLag + 2 && smem_bytes(stages, stage_bytes) * (size_t)ctas_per_sm > smem_limit - 1024u * (size_t)ctas_per_sm)
-        --stages;
+    st = fit_stages(stages, def.groups, def.lag, true, stage_bytes, ctas_per_sm, smem_limit);
+    if (st != KDN_OK) return st;
     const size_t smem = smem_bytes(stages, stage_bytes);
-    if (smem > smem_limit) return KDN_E_UNSUPPORTED;
 
     unsigned long long tiles = 0;
     int n = 0, n_rope = 0;
@@ -829,10 +869,10 @@ extern "C" kdn_status kdn_compose_static(int device, const kdn_pool_desc *pool, 
         lp.stage_bytes = stage_bytes;
         lp.off_b = a_bytes;
         lp.off_s = a_bytes + b_bytes;
+        lp.store_lag = def.lag;
         const unsigned long long want = (unsigned long long)sd->sm_count * (unsigned)ctas_per_sm;
         const unsigned grid = (unsigned)(tiles < want ? tiles : want);
-        st = compute ? launch_kernel(kdn_compose_kernel<true>, kThreadsCompute, grid, smem, stream, lp)
-                     : launch_kernel(kdn_compose_kernel<false>, kThreadsCopy, grid, smem, stream, lp);
+        st = launch_tiles(OP_COMPOSE, def.groups, grid, smem, stream, lp);
         if (st != KDN_OK) return st;
     }
     if (!wait) return KDN_OK;

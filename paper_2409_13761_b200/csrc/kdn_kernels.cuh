@@ -11,7 +11,7 @@
 // Pipeline inside a CTA (S slots of shared memory, all hand-offs through mbarriers):
 //   loader warp   decodes tiles 32 at a time (one per lane: op lookup, block-table entry, addresses),
 //                 then issues each tile's bulk async copies global -> shared
-//   compute warps (2 groups of 4; group g owns slots g, g+2, ...) int8 coding / decoding and key
+//   compute warps (G groups of 4; group g owns slots g, g+G, ...) int8 coding / decoding and key
 //                 rotation, shared -> shared
 //   storer thread issues the bulk async copy shared -> global and recycles the slot
 // Tiles that are a pure copy (raw bf16 without rotation) never touch the compute warps' ALUs.
@@ -28,13 +28,11 @@ namespace kdn {
 constexpr int kLoaderWarp = 0;
 constexpr int kGroupWarps = 4;                // warps that work together on one tile
 constexpr int kGroupThreads = kGroupWarps * 32;
-constexpr int kComputeGroups = 2;             // groups take alternate pipeline slots (group_bar_sync knows two)
-constexpr int kComputeWarps = kGroupWarps * kComputeGroups;
-constexpr int kComputeThreads = kComputeWarps * 32;
-constexpr int kThreadsCompute = 32 + kComputeThreads + 32;   // loader + compute + storer
+constexpr int kMaxGroups = 6;                 // compute groups per CTA; group g owns slots g, g + G, ...
+__host__ __device__ constexpr int threads_for(int groups) { return 32 + groups * kGroupThreads + 32; }  // loader + compute + storer
 constexpr int kThreadsCopy = 64;                             // loader + storer
 constexpr int kMaxStages = 32;
-constexpr int kStoreLag = 2;              // bulk stores allowed to be still reading shared memory
+constexpr int kMaxStoreLag = 4;           // most bulk-store groups allowed to be still reading shared memory
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 enum : uint32_t { TF_INT8 = 1u, TF_ROTATE = 2u, TF_SCALES_PLAIN = 4u };
@@ -83,6 +81,7 @@ struct Launch {
     unsigned stage_bytes;
     unsigned off_b;           // offset of the code buffer inside a stage (compute launches)
     unsigned off_s;           // offset of the scale buffer inside a stage
+    int store_lag;            // bulk-store groups that may still be reading shared memory (1..kMaxStoreLag)
 };
 
 struct __align__(16) TileDesc {
@@ -160,12 +159,27 @@ template <int N> __device__ __forceinline__ void bulk_wait_read()
 {
     asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
 }
+__device__ __forceinline__ void bulk_wait_read_n(int n)      // the instruction takes an immediate
+{
+    switch (n) {
+    case 1: bulk_wait_read<1>(); break;
+    case 2: bulk_wait_read<2>(); break;
+    case 3: bulk_wait_read<3>(); break;
+    default: bulk_wait_read<4>(); break;
+    }
+}
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void group_bar_sync(int group)
 {
-    if (group == 0) asm volatile("bar.sync 1, %0;" ::"n"(kGroupThreads) : "memory");
-    else            asm volatile("bar.sync 2, %0;" ::"n"(kGroupThreads) : "memory");
+    switch (group) {                                       // immediate ids: only kMaxGroups barriers are reserved
+    case 0: asm volatile("bar.sync 1, %0;" ::"n"(kGroupThreads) : "memory"); break;
+    case 1: asm volatile("bar.sync 2, %0;" ::"n"(kGroupThreads) : "memory"); break;
+    case 2: asm volatile("bar.sync 3, %0;" ::"n"(kGroupThreads) : "memory"); break;
+    case 3: asm volatile("bar.sync 4, %0;" ::"n"(kGroupThreads) : "memory"); break;
+    case 4: asm volatile("bar.sync 5, %0;" ::"n"(kGroupThreads) : "memory"); break;
+    default: asm volatile("bar.sync 6, %0;" ::"n"(kGroupThreads) : "memory"); break;
+    }
 }
 
 __device__ __forceinline__ uint4 lds128(const void *p) { return *reinterpret_cast<const uint4 *>(p); }
@@ -437,9 +451,10 @@ __host__ __device__ inline size_t smem_bytes(int stages, unsigned stage_bytes)
     return (size_t)stages * stage_bytes + 24u * (size_t)stages + 16u + sizeof(TileDesc) * (size_t)stages + 16u;
 }
 
-template <int OP, bool kCompute>
+template <int OP, int kGroups>
 __device__ __forceinline__ void tile_pipeline(const Launch &P)
 {
+    constexpr bool kCompute = kGroups > 0;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const Smem sm = carve(P, smem_raw);
     const int S = P.stages;
@@ -461,7 +476,7 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
 
     const unsigned grid = gridDim.x, bid = blockIdx.x;
     const unsigned n_my = P.n_tiles > bid ? (P.n_tiles - bid + grid - 1u) / grid : 0u;
-    const int storer_warp = kCompute ? 1 + kComputeWarps : 1;
+    const int storer_warp = 1 + kGroups * kGroupWarps;
 
     if (warp == kLoaderWarp) {
         // ------------------------------------------------------------ loader
@@ -544,18 +559,18 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                 }
                 bulk_commit();
                 ++done;
-                // recycle the slot committed kStoreLag slots ago: its store has read shared memory,
+                // recycle the slot committed store_lag slots ago: its store has read shared memory,
                 // and every compute warp has moved past it
-                bulk_wait_read<kStoreLag>();
-                if (slot >= (unsigned)kStoreLag) {
-                    const unsigned old = slot - (unsigned)kStoreLag;
+                bulk_wait_read_n(P.store_lag);
+                if (slot >= (unsigned)P.store_lag) {
+                    const unsigned old = slot - (unsigned)P.store_lag;
                     const unsigned st2 = old % (unsigned)S;
                     if (kCompute && !mbar_wait(sm.ready + 8u * st2, (old / (unsigned)S) & 1u, sm.abort_flag)) break;
                     mbar_arrive(sm.empty + 8u * st2);
                 }
             }
             bulk_wait_read<0>();
-            for (unsigned slot = done > (unsigned)kStoreLag ? done - kStoreLag : 0u; slot < done; ++slot)
+            for (unsigned slot = done > (unsigned)P.store_lag ? done - (unsigned)P.store_lag : 0u; slot < done; ++slot)
                 mbar_arrive(sm.empty + 8u * (slot % (unsigned)S));
             bulk_wait_all();
             if (done != n_my) atomicCAS(P.status, 0, kStatusTimeout);
@@ -566,7 +581,7 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
         const int ct = (tid - 32) % kGroupThreads;
         RotCoef rc;
         rc.rope = -1; rc.col = 0xffffffffu;
-        for (unsigned slot = (unsigned)group; slot < n_my; slot += (unsigned)kComputeGroups) {
+        for (unsigned slot = (unsigned)group; slot < n_my; slot += (unsigned)kGroups) {
             const unsigned st = slot % (unsigned)S;
             const uint32_t ph = (slot / (unsigned)S) & 1u;
             if (!mbar_wait(sm.full + 8u * st, ph, sm.abort_flag)) break;
@@ -609,20 +624,23 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
     __syncthreads();
 }
 
+// kGroups = 0 is the pure-copy form (loader + storer only); kGroups > 0 adds that many compute groups.
+// The host keeps stages a multiple of kGroups, so a pipeline slot always belongs to the same group and
+// every waiter visits a barrier once per phase (a parity wait cannot tell phases two apart).
 // Sec. 3.2 call (i) store, Sec. 3.1 storage module: paged pool -> chunk, optional int8 coding.
-template <bool kCompute>
-__global__ void __launch_bounds__(kCompute ? kThreadsCompute : kThreadsCopy)
-kdn_store_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_STORE, kCompute>(P); }
+template <int kGroups>
+__global__ void __launch_bounds__(threads_for(kGroups))
+kdn_store_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_STORE, kGroups>(P); }
 
 // Sec. 3.2 call (ii) retrieve, Sec. 3.1 delivery module (decompression on the GPU): chunk -> pool.
-template <bool kCompute>
-__global__ void __launch_bounds__(kCompute ? kThreadsCompute : kThreadsCopy)
-kdn_retrieve_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_RETRIEVE, kCompute>(P); }
+template <int kGroups>
+__global__ void __launch_bounds__(threads_for(kGroups))
+kdn_retrieve_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_RETRIEVE, kGroups>(P); }
 
 // Sec. 3.1 blending module: parts -> request blocks at new positions, keys re-rotated.
-template <bool kCompute>
-__global__ void __launch_bounds__(kCompute ? kThreadsCompute : kThreadsCopy)
-kdn_compose_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_COMPOSE, kCompute>(P); }
+template <int kGroups>
+__global__ void __launch_bounds__(threads_for(kGroups))
+kdn_compose_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_COMPOSE, kGroups>(P); }
 
 // Rotation table: row r, frequency i -> (cos, sin) of delta_r * theta_r^(-2i/D), evaluated in fp64 and
 // rounded once to fp32 (an fp32 angle would lose more than half a bf16 ulp at large position shifts).

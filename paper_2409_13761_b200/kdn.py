@@ -48,7 +48,7 @@ class kdn_compose_req(C.Structure):
 
 class kdn_tuning(C.Structure):
     _fields_ = [("tile_bytes", C.c_int32), ("stages", C.c_int32), ("ctas_per_sm", C.c_int32),
-                ("reserved", C.c_int32)]
+                ("compute_groups", C.c_int32), ("store_lag", C.c_int32), ("reserved", C.c_int32)]
 
 
 def _load() -> C.CDLL:
@@ -233,8 +233,9 @@ def kdn_status_sync(ctx, stream: int = 0) -> int:
     return int(lib.kdn_status_sync(ctx, stream))
 
 
-def kdn_set_tuning(ctx, tile_bytes: int = 0, stages: int = 0, ctas_per_sm: int = 0) -> None:
-    t = kdn_tuning(tile_bytes, stages, ctas_per_sm, 0)
+def kdn_set_tuning(ctx, tile_bytes: int = 0, stages: int = 0, ctas_per_sm: int = 0, compute_groups: int = 0,
+                   store_lag: int = 0) -> None:
+    t = kdn_tuning(tile_bytes, stages, ctas_per_sm, compute_groups, store_lag, 0)
     _check(lib.kdn_set_tuning(ctx, C.byref(t)), "kdn_set_tuning")
 
 

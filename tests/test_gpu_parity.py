@@ -372,13 +372,14 @@ def test_tuning_shapes_give_identical_results():
         tab = np.random.default_rng(2).permutation(64)[:20].astype(np.int32)
         T, off = 300, 7
         want = {c: oracle.store(host, tab, off, T, c) for c in (RAW, INT8)}
-        for tile, stages, ctas in [(0, 0, 0), (2048, 4, 1), (4096, 12, 3), (32768, 4, 1), (16384, 5, 2), (1024, 16, 4)]:
-            K.kdn_set_tuning(dev.ctx, tile, stages, ctas)
+        for tile, stages, ctas, groups, lag in [(0, 0, 0, 0, 0), (2048, 4, 1, 1, 1), (4096, 12, 3, 3, 2), (32768, 4, 1, 4, 2),
+                                                (16384, 5, 2, 2, 3), (1024, 16, 4, 6, 4), (8192, 3, 2, 3, 1), (8192, 7, 1, 6, 1)]:
+            K.kdn_set_tuning(dev.ctx, tile, stages, ctas, groups, lag)
             for c in (RAW, INT8):
                 buf = dev.chunk_buf(T, c)
                 dev.store([dev.op(dev.table(tab), off, buf, T, c)])
                 assert dev.sync() == 0
-                assert np.array_equal(to_np(buf), want[c]), (tile, stages, ctas, c)
+                assert np.array_equal(to_np(buf), want[c]), (tile, stages, ctas, groups, lag, c)
         with pytest.raises(K.KdnError):
             K.kdn_set_tuning(dev.ctx, 100, 0, 0)                 # not a multiple of 128
     finally:
