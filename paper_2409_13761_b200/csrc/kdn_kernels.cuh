@@ -197,26 +197,72 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi)
     return *reinterpret_cast<uint32_t *>(&v);
 }
 
-// round_half_even(x * inv) as the low byte of the fp32 sum with 1.5 * 2^23: for |x * inv| < 2^22 the
-// sum is rounded to an integer by the adder itself (ties to even) and its low mantissa bits are the
-// two's-complement integer.  The product and the sum are two separately rounded fp32 operations.
-__device__ __forceinline__ uint32_t code_bits(float x, float inv)
+// Two fp32 values in one 64-bit register for the packed fp32 instructions of sm_100 (each half is an
+// ordinary IEEE round-to-nearest operation; nothing is fused unless fma2 is asked for).
+typedef unsigned long long f32x2;
+__device__ __forceinline__ f32x2 pack2(float lo, float hi)
 {
-    return __float_as_uint(__fadd_rn(__fmul_rn(x, inv), 12582912.0f));
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
 }
+__device__ __forceinline__ f32x2 pack2_bits(uint32_t lo, uint32_t hi)
+{
+    f32x2 r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "r"(lo), "r"(hi));
+    return r;
+}
+__device__ __forceinline__ void unpack2(f32x2 v, float &lo, float &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(v));
+}
+__device__ __forceinline__ void unpack2_bits(f32x2 v, uint32_t &lo, uint32_t &hi)
+{
+    asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(v));
+}
+__device__ __forceinline__ f32x2 mul2(f32x2 a, f32x2 b)
+{
+    f32x2 d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2 add2(f32x2 a, f32x2 b)
+{
+    f32x2 d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
+{
+    f32x2 d;
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(a), "l"(b), "l"(c));
+    return d;
+}
+// p + c with its own rounding when p is a product.  The assembler contracts a packed multiply whose only
+// use is a packed add into one fused multiply-add (measured: it does so even though both carry .rn, unlike
+// the scalar forms), which would round x * inv + c once instead of twice.  Written as fma(p, 1, c) the sum
+// is the same correctly rounded p + c and there is nothing left to contract.
+__device__ __forceinline__ f32x2 add2_unfused(f32x2 p, f32x2 c, f32x2 one) { return fma2(p, one, c); }
+// The two bf16 halves of w as a packed fp32 pair (exact).
+__device__ __forceinline__ f32x2 bf16x2_to_f32x2(uint32_t w) { return pack2_bits(w << 16, w & 0xffff0000u); }
+// max(|a|, |b|) on both bf16 halves; the sign of the result is meaningless.
+__device__ __forceinline__ uint32_t maxabs_bf16x2(uint32_t a, uint32_t b)
+{
+    uint32_t d;
+    asm("max.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+    return d;
+}
+
+// Rounding trick used by quantise_tile: round_half_even(x * inv) is the low byte of the fp32 sum of the
+// (already rounded) product with 1.5 * 2^23.  For |x * inv| < 2^22 the adder itself rounds the sum to an
+// integer, ties to even, and the low mantissa bits are the two's-complement integer.  The product and the
+// sum are two separately rounded fp32 operations, as the codec's definition requires.
 __device__ __forceinline__ uint32_t pack_codes4(uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3)
 {
     uint32_t a = __byte_perm(r0, r1, 0x0040);             // r0.b0, r1.b0
     uint32_t b = __byte_perm(r2, r3, 0x0040);
     return __byte_perm(a, b, 0x5410);
 }
-// (float)code for byte k of w, where w holds four codes already XORed with 0x80: 2^23 + (code + 128)
-// built in the mantissa, minus 2^23 + 128.  Exact.
-template <int K> __device__ __forceinline__ float code_to_float(uint32_t w_biased)
-{
-    return __fsub_rn(__uint_as_float(__byte_perm(w_biased, 0x4B000000u, 0x7650 + K)), 8388736.0f);
-}
-
 // Encode n elements (a multiple of 64) of bf16 at A into int8 codes at B and one fp32 scale per 64
 // elements (to shared S, or straight to global when the destination is not 16-byte aligned).
 // Two lanes share a group, 32 elements each, read as four 128-bit shared loads in a lane-rotated
@@ -236,35 +282,36 @@ __device__ __forceinline__ void quantise_tile(const unsigned char *A, unsigned c
 #pragma unroll
         for (int j = 0; j < 4; ++j)
             x[j] = act ? lds128(src + (((unsigned)j + rot) & 3u) * 16u) : make_uint4(0u, 0u, 0u, 0u);
-        float f[32];
+        // absmax on the packed bf16 pairs, two chains
+        uint32_t m0 = maxabs_bf16x2(x[0].x, x[0].y), m1 = maxabs_bf16x2(x[0].z, x[0].w);
 #pragma unroll
-        for (int j = 0; j < 4; ++j) {
-            f[8 * j + 0] = bf16_lo(x[j].x); f[8 * j + 1] = bf16_hi(x[j].x);
-            f[8 * j + 2] = bf16_lo(x[j].y); f[8 * j + 3] = bf16_hi(x[j].y);
-            f[8 * j + 4] = bf16_lo(x[j].z); f[8 * j + 5] = bf16_hi(x[j].z);
-            f[8 * j + 6] = bf16_lo(x[j].w); f[8 * j + 7] = bf16_hi(x[j].w);
+        for (int j = 1; j < 4; ++j) {
+            m0 = maxabs_bf16x2(m0, x[j].x); m1 = maxabs_bf16x2(m1, x[j].y);
+            m0 = maxabs_bf16x2(m0, x[j].z); m1 = maxabs_bf16x2(m1, x[j].w);
         }
-        float a0 = 0.0f, a1 = 0.0f, a2 = 0.0f, a3 = 0.0f;
-#pragma unroll
-        for (int k = 0; k < 32; k += 4) {
-            a0 = fmaxf(a0, fabsf(f[k])); a1 = fmaxf(a1, fabsf(f[k + 1]));
-            a2 = fmaxf(a2, fabsf(f[k + 2])); a3 = fmaxf(a3, fabsf(f[k + 3]));
-        }
-        float a = fmaxf(fmaxf(a0, a1), fmaxf(a2, a3));
+        m0 = maxabs_bf16x2(m0, m1);
+        float a = fmaxf(__uint_as_float((m0 << 16) & 0x7fffffffu), __uint_as_float(m0 & 0x7fff0000u));
         a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
         float scale = __fdiv_rn(a, 127.0f);
         const bool ok = scale >= 1.17549435e-38f;         // smallest normal fp32; false for NaN too
         const float inv = ok ? __fdiv_rn(127.0f, a) : 0.0f;
         scale = ok ? scale : 0.0f;
         if (act) {
+            const f32x2 inv2 = pack2(inv, inv);
+            const f32x2 magic2 = pack2(12582912.0f, 12582912.0f);
+            const f32x2 one2 = pack2(1.0f, 1.0f);
             unsigned char *dst = B + (size_t)h * 32u;
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
+                // per pair: one rounded product, one rounded sum with 1.5 * 2^23 (see above)
+                uint32_t r[8];
+                unpack2_bits(add2_unfused(mul2(bf16x2_to_f32x2(x[j].x), inv2), magic2, one2), r[0], r[1]);
+                unpack2_bits(add2_unfused(mul2(bf16x2_to_f32x2(x[j].y), inv2), magic2, one2), r[2], r[3]);
+                unpack2_bits(add2_unfused(mul2(bf16x2_to_f32x2(x[j].z), inv2), magic2, one2), r[4], r[5]);
+                unpack2_bits(add2_unfused(mul2(bf16x2_to_f32x2(x[j].w), inv2), magic2, one2), r[6], r[7]);
                 uint2 q;
-                q.x = pack_codes4(code_bits(f[8 * j + 0], inv), code_bits(f[8 * j + 1], inv),
-                                  code_bits(f[8 * j + 2], inv), code_bits(f[8 * j + 3], inv));
-                q.y = pack_codes4(code_bits(f[8 * j + 4], inv), code_bits(f[8 * j + 5], inv),
-                                  code_bits(f[8 * j + 6], inv), code_bits(f[8 * j + 7], inv));
+                q.x = pack_codes4(r[0], r[1], r[2], r[3]);
+                q.y = pack_codes4(r[4], r[5], r[6], r[7]);
                 sts64(dst + (((unsigned)j + rot) & 3u) * 8u, q);
             }
             if ((lane & 1u) == 0u) {
@@ -274,29 +321,46 @@ __device__ __forceinline__ void quantise_tile(const unsigned char *A, unsigned c
     }
 }
 
-// Decode n int8 codes at B with scales S into bf16 at A: one fp32 product, rounded to bf16.
+// (float)code for bytes K and K+1 of w (four codes already XORed with 0x80) as a packed pair: each
+// byte is placed in the mantissa of 2^23 (giving 2^23 + code + 128) and 2^23 + 128 is subtracted. Exact.
+template <int K> __device__ __forceinline__ f32x2 codes_to_f32x2(uint32_t w_biased, f32x2 minus_bias)
+{
+    return add2(pack2_bits(__byte_perm(w_biased, 0x4B000000u, 0x7650 + K),
+                           __byte_perm(w_biased, 0x4B000000u, 0x7650 + K + 1)), minus_bias);
+}
+__device__ __forceinline__ uint32_t pack_bf16x2(f32x2 v)
+{
+    float lo, hi;
+    unpack2(v, lo, hi);
+    return pack_bf16x2(lo, hi);
+}
+
+// Decode n int8 codes at B with scales S into bf16 at A: one fp32 product per element, rounded to bf16.
 __device__ __forceinline__ void dequantise_tile(const unsigned char *B, const float *S, unsigned char *A,
                                                 unsigned n, int ct)
 {
     const unsigned nvec = n >> 4;
+    const f32x2 minus_bias = pack2(-8388736.0f, -8388736.0f);
     for (unsigned v = (unsigned)ct; v < nvec; v += kGroupThreads) {
         const uint4 c = lds128(B + (size_t)v * 16u);
         const float sc = S[v >> 2];
+        const f32x2 sc2 = pack2(sc, sc);
         const uint32_t w[4] = { c.x ^ 0x80808080u, c.y ^ 0x80808080u, c.z ^ 0x80808080u, c.w ^ 0x80808080u };
         uint32_t o[8];
 #pragma unroll
         for (int j = 0; j < 4; ++j) {
-            o[2 * j] = pack_bf16x2(__fmul_rn(code_to_float<0>(w[j]), sc), __fmul_rn(code_to_float<1>(w[j]), sc));
-            o[2 * j + 1] = pack_bf16x2(__fmul_rn(code_to_float<2>(w[j]), sc), __fmul_rn(code_to_float<3>(w[j]), sc));
+            o[2 * j] = pack_bf16x2(mul2(codes_to_f32x2<0>(w[j], minus_bias), sc2));
+            o[2 * j + 1] = pack_bf16x2(mul2(codes_to_f32x2<2>(w[j], minus_bias), sc2));
         }
         sts128(A + (size_t)v * 32u, make_uint4(o[0], o[1], o[2], o[3]));
         sts128(A + (size_t)v * 32u + 16u, make_uint4(o[4], o[5], o[6], o[7]));
     }
 }
 
-// Rotation coefficients a thread keeps in registers: (cos, sin) for 8 consecutive frequencies.
+// Rotation coefficients a thread keeps in registers: (cos, sin, -sin) for 8 consecutive frequencies,
+// as four packed pairs each.
 struct RotCoef {
-    float c[8], s[8];
+    f32x2 c[4], s[4], ns[4];
     int rope;      // table row they belong to
     unsigned col;  // first frequency index
 };
@@ -307,22 +371,26 @@ __device__ __forceinline__ void load_coef(RotCoef &rc, const float2 *table, int 
     const float4 *p = reinterpret_cast<const float4 *>(table + (size_t)rope * half + col);
 #pragma unroll
     for (int k = 0; k < 4; ++k) {
-        float4 v = __ldg(p + k);
-        rc.c[2 * k] = v.x; rc.s[2 * k] = v.y; rc.c[2 * k + 1] = v.z; rc.s[2 * k + 1] = v.w;
+        const float4 v = __ldg(p + k);                     // (cos, sin) of frequencies 2k and 2k + 1
+        rc.c[k] = pack2(v.x, v.z);
+        rc.s[k] = pack2(v.y, v.w);
+        rc.ns[k] = pack2(-v.y, -v.w);
     }
     rc.rope = rope; rc.col = col;
 }
 
-__device__ __forceinline__ void rotate8(const float *u, const float *w, const RotCoef &rc, uint4 &lo, uint4 &hi)
+// u' = u cos - w sin, w' = w cos + u sin for four packed pairs of (u, w); each result is one rounded
+// product folded into one fused multiply-add.
+__device__ __forceinline__ void rotate8(const f32x2 *u, const f32x2 *w, const RotCoef &rc, uint4 &lo, uint4 &hi)
 {
-    float u2[8], w2[8];
+    uint32_t ou[4], ow[4];
 #pragma unroll
-    for (int k = 0; k < 8; ++k) {
-        u2[k] = __fmaf_rn(u[k], rc.c[k], -__fmul_rn(w[k], rc.s[k]));
-        w2[k] = __fmaf_rn(w[k], rc.c[k], __fmul_rn(u[k], rc.s[k]));
+    for (int k = 0; k < 4; ++k) {
+        ou[k] = pack_bf16x2(fma2(u[k], rc.c[k], mul2(w[k], rc.ns[k])));
+        ow[k] = pack_bf16x2(fma2(w[k], rc.c[k], mul2(u[k], rc.s[k])));
     }
-    lo = make_uint4(pack_bf16x2(u2[0], u2[1]), pack_bf16x2(u2[2], u2[3]), pack_bf16x2(u2[4], u2[5]), pack_bf16x2(u2[6], u2[7]));
-    hi = make_uint4(pack_bf16x2(w2[0], w2[1]), pack_bf16x2(w2[2], w2[3]), pack_bf16x2(w2[4], w2[5]), pack_bf16x2(w2[6], w2[7]));
+    lo = make_uint4(ou[0], ou[1], ou[2], ou[3]);
+    hi = make_uint4(ow[0], ow[1], ow[2], ow[3]);
 }
 
 // Rotate a tile of whole head rows (n a multiple of D, D a multiple of 16).  One work item is 8
@@ -337,31 +405,27 @@ __device__ __forceinline__ void rotate_tile(unsigned char *A, const unsigned cha
     const bool pow2 = (per_row & (per_row - 1u)) == 0u;
     const unsigned shift = 31u - (unsigned)__clz(per_row);
     const unsigned items = n >> 4;
+    const f32x2 minus_bias = pack2(-8388736.0f, -8388736.0f);
     for (unsigned it = (unsigned)ct; it < items; it += kGroupThreads) {
         const unsigned r = pow2 ? it >> shift : it / per_row;
         const unsigned col = (it - r * per_row) << 3;
         load_coef(rc, table, rope, col, half);
         const unsigned e_lo = r * D + col, e_hi = e_lo + half;
-        float u[8], w[8];
+        f32x2 u[4], w[4];
         if (kInt8) {
             const uint2 cl = lds64(B + e_lo), ch = lds64(B + e_hi);
             const float sl = S[e_lo >> 6], sh = S[e_hi >> 6];
+            const f32x2 sl2 = pack2(sl, sl), sh2 = pack2(sh, sh);
             const uint32_t l0 = cl.x ^ 0x80808080u, l1 = cl.y ^ 0x80808080u;
             const uint32_t h0 = ch.x ^ 0x80808080u, h1 = ch.y ^ 0x80808080u;
-            u[0] = __fmul_rn(code_to_float<0>(l0), sl); u[1] = __fmul_rn(code_to_float<1>(l0), sl);
-            u[2] = __fmul_rn(code_to_float<2>(l0), sl); u[3] = __fmul_rn(code_to_float<3>(l0), sl);
-            u[4] = __fmul_rn(code_to_float<0>(l1), sl); u[5] = __fmul_rn(code_to_float<1>(l1), sl);
-            u[6] = __fmul_rn(code_to_float<2>(l1), sl); u[7] = __fmul_rn(code_to_float<3>(l1), sl);
-            w[0] = __fmul_rn(code_to_float<0>(h0), sh); w[1] = __fmul_rn(code_to_float<1>(h0), sh);
-            w[2] = __fmul_rn(code_to_float<2>(h0), sh); w[3] = __fmul_rn(code_to_float<3>(h0), sh);
-            w[4] = __fmul_rn(code_to_float<0>(h1), sh); w[5] = __fmul_rn(code_to_float<1>(h1), sh);
-            w[6] = __fmul_rn(code_to_float<2>(h1), sh); w[7] = __fmul_rn(code_to_float<3>(h1), sh);
+            u[0] = mul2(codes_to_f32x2<0>(l0, minus_bias), sl2); u[1] = mul2(codes_to_f32x2<2>(l0, minus_bias), sl2);
+            u[2] = mul2(codes_to_f32x2<0>(l1, minus_bias), sl2); u[3] = mul2(codes_to_f32x2<2>(l1, minus_bias), sl2);
+            w[0] = mul2(codes_to_f32x2<0>(h0, minus_bias), sh2); w[1] = mul2(codes_to_f32x2<2>(h0, minus_bias), sh2);
+            w[2] = mul2(codes_to_f32x2<0>(h1, minus_bias), sh2); w[3] = mul2(codes_to_f32x2<2>(h1, minus_bias), sh2);
         } else {
             const uint4 xl = lds128(A + (size_t)e_lo * 2u), xh = lds128(A + (size_t)e_hi * 2u);
-            u[0] = bf16_lo(xl.x); u[1] = bf16_hi(xl.x); u[2] = bf16_lo(xl.y); u[3] = bf16_hi(xl.y);
-            u[4] = bf16_lo(xl.z); u[5] = bf16_hi(xl.z); u[6] = bf16_lo(xl.w); u[7] = bf16_hi(xl.w);
-            w[0] = bf16_lo(xh.x); w[1] = bf16_hi(xh.x); w[2] = bf16_lo(xh.y); w[3] = bf16_hi(xh.y);
-            w[4] = bf16_lo(xh.z); w[5] = bf16_hi(xh.z); w[6] = bf16_lo(xh.w); w[7] = bf16_hi(xh.w);
+            u[0] = bf16x2_to_f32x2(xl.x); u[1] = bf16x2_to_f32x2(xl.y); u[2] = bf16x2_to_f32x2(xl.z); u[3] = bf16x2_to_f32x2(xl.w);
+            w[0] = bf16x2_to_f32x2(xh.x); w[1] = bf16x2_to_f32x2(xh.y); w[2] = bf16x2_to_f32x2(xh.z); w[3] = bf16x2_to_f32x2(xh.w);
         }
         uint4 lo, hi;
         rotate8(u, w, rc, lo, hi);

@@ -132,6 +132,9 @@ def test_unaligned_ragged_batched_mixed_codecs(shape):
         dev.close()
 
 
+FUSION_WITNESS_ABSMAX = [21.25, 38.5, 46.0, 84.0, 23.0, 25.75]
+
+
 def special_pool(shape):
     """Pool whose groups hit the codec's special cases: zeros, -0, subnormal scales, ties, big outliers, NaN-free."""
     rng = np.random.default_rng(99)
@@ -152,6 +155,11 @@ def special_pool(shape):
     flat[5::11] = f((g.view(np.uint32) & 0xffff0000).view(np.float32))    # tiny but normal
     g = np.full(64, 2.0 ** 120, dtype=np.float32); g[::2] *= -1
     flat[6::11] = f(g)                                                    # huge magnitudes
+    # products that round TO a tie: x = a/2 with fl(127/a) below 127/a, so fl(x * inv) = 63.5 -> 64 while
+    # a single-rounding fused multiply-add would give 63 (see tests/test_oracle_codec.py)
+    for k, a in enumerate(FUSION_WITNESS_ABSMAX):
+        g = np.zeros(64, dtype=np.float32); g[0] = a; g[1] = a / 2; g[2] = -a / 2; g[33] = -a; g[40] = a / 2
+        flat[7 + 11 * k::11 * len(FUSION_WITNESS_ABSMAX)] = f(g)
     return pool
 
 

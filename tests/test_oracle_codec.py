@@ -234,3 +234,17 @@ def test_f64_to_bf16_single_rounding():
     xs = rng.standard_normal(3000) * 10.0 ** rng.integers(-6, 6, 3000)
     for x in xs:
         assert oracle.f64_to_bf16(float(x)) == nearest_bf16_by_search(float(x))
+
+
+def test_double_rounding_witnesses():
+    """Groups where the codec's two roundings matter: x = a/2 and fl(127/a) < 127/a, so the exact product is just
+    below 63.5 but the fp32 product IS 63.5, a tie that goes to 64.  One fused rounding would give 63."""
+    from fractions import Fraction
+    for a in [21.25, 38.5, 46.0, 84.0, 23.0, 25.75]:
+        inv = np.float32(127.0) / np.float32(a)
+        x = np.float32(a / 2)
+        exact = Fraction(float(x)) * Fraction(float(inv))
+        assert exact < Fraction(127, 2) and np.float32(x * inv) == np.float32(63.5)
+        g = np.zeros(64, dtype=np.float32); g[0] = a; g[1] = x; g[2] = -x
+        q, _ = oracle.quant_group(bf16_bits(g))
+        assert (q[0], q[1], q[2]) == (127, 64, -64)
