@@ -150,8 +150,7 @@ struct Shape { int tile_bytes, stages, ctas_per_sm, groups, lag; };
 Shape default_shape(int OP, bool any_int8, bool any_rot)
 {
     if (!any_int8 && !any_rot) return Shape{ 32768, 4, 1, 0, 2 };
-    if (OP == OP_STORE) return Shape{ 16384, 9, 1, 3, 2 };
-    if (OP == OP_RETRIEVE || !any_rot) return Shape{ 8192, 6, 3, 2, 2 };
+    if (OP != OP_COMPOSE || !any_rot) return Shape{ 8192, 6, 3, 2, 2 };
     if (!any_int8) return Shape{ 8192, 6, 2, 2, 2 };
     return Shape{ 16384, 9, 1, 3, 2 };
 }
