@@ -100,7 +100,7 @@ def check_rotated_keys(got_bits: np.ndarray, kref: np.ndarray, kmag: np.ndarray,
     |got - ref64| <= 2^-8 |ref64| + 2^-21 (|u| + |w|): one bf16 ulp relative to the fp64 result, plus a
     floor for results that cancel to almost nothing, where the fp32 rounding of the table and of the
     products (each <= 2^-24 relative to |u| or |w|) is all that is left.  Also: at most one bf16 step
-    from the oracle's own rounding, and almost always equal to it.
+    from the oracle's own rounding wherever the result did not cancel, and almost always equal to it.
     """
     got = bits_to_f64(got_bits)
     err = np.abs(got - kref)
@@ -109,7 +109,11 @@ def check_rotated_keys(got_bits: np.ndarray, kref: np.ndarray, kmag: np.ndarray,
     assert not bad.any(), "%d rotated key elements out of tolerance, worst %.3g vs %.3g" % (
         int(bad.sum()), float(err[bad].max()), float(tol[bad].max()))
     d = bf16_ulp_distance(got_bits, oracle_bits)
-    assert d.max() <= 1, "rotated key differs from the rounded fp64 result by %d bf16 steps" % int(d.max())
+    # where the result did not cancel (|ref| >= 2^-12 (|u|+|w|)) the fp32 error is far below a bf16 step, so the
+    # kernel may differ from the oracle's rounding by one step at most (a near-tie); cancelled results are
+    # covered by the absolute floor above only
+    solid = np.abs(kref) >= 2.0 ** -12 * kmag
+    assert d[solid].max(initial=0) <= 1, "rotated key differs from the rounded fp64 result by %d bf16 steps" % int(d[solid].max())
     frac_equal = float((d == 0).mean())
     assert frac_equal > 0.995, "only %.4f of rotated keys equal the rounded fp64 result" % frac_equal
     return frac_equal
