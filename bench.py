@@ -185,7 +185,7 @@ NCU_SMALL_CASE_BYTES = {"store_raw": (536.894720e6 + 485.936384e6, 8), "retrieve
                         "retrieve_int8": (285.241600e6 + 483.000064e6, 8), "compose_int8": (142.639616e6 + 213.129216e6, 2)}
 
 
-def measured_traffic(op: str, units: int):
+def measured_traffic(op: str, units: float):
     import hashlib
     try:
         with open(os.path.join(ROOT, "paper_2409_13761_b200", "csrc", "kdn_kernels.cuh"), "rb") as fh:
@@ -206,26 +206,45 @@ def measured_hbm_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
+def make_workload(args, synth):
+    """Sizes of one step.  llama3-8b is the benchmark workload; llama3-70b is the batched-retrieve configuration."""
+    if args.workload == "llama3-70b":
+        shape = synth.LLAMA3_70B
+        assign = synth.assign_chunks(32, 4, 16)                       # 32 requests x 4 chunks out of a library of 16
+        w = dict(name="llama3-70b", shape=shape, lib=16, chunk_tokens=2048, retr=assign.reshape(-1), part_lib=16,
+                 part_tokens=2048, reqs=[list(map(int, row)) for row in assign], suffix=0, exclusive=False,
+                 text=("llama3-70b KV (L80 H8 D128 bf16, block_size 16, 16384-block pool): store a library of 16x2048 "
+                       "tokens, retrieve 32 requests x 4 chunks (fills the pool), compose the same 32x4 at cumulative "
+                       "offsets; raw bf16 and int8-g64, fully fragmented tables"))
+    else:
+        shape = synth.LLAMA3_8B
+        n_chunks, n_parts = args.chunks or N_CHUNKS, args.parts or N_PARTS
+        if args.pool_blocks:
+            shape = shape.with_(n_blocks=args.pool_blocks)
+        w = dict(name="llama3-8b", shape=shape, lib=n_chunks, chunk_tokens=CHUNK_TOKENS, retr=np.arange(n_chunks),
+                 part_lib=n_parts, part_tokens=PART_TOKENS, reqs=[list(range(n_parts))], suffix=SUFFIX_TOKENS,
+                 exclusive=True, text=WORKLOAD)
+        if args.pool_blocks or args.chunks or args.parts:
+            w["text"] = "REDUCED (%d chunks, %d parts, %d blocks): not the bench workload" % (n_chunks, n_parts, shape.n_blocks)
+    return w
+
+
 def run_gpu(args) -> None:
     import torch
-    from paper_2409_13761_b200 import kdn as K, synth
+    from paper_2409_13761_b200 import kdn as K, shard, synth
 
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    rank = int(os.environ.get("RANK", "0"))
-    local = int(os.environ.get("LOCAL_RANK", "0"))
+    rank, world, local = shard.rank_env()
     dist = None
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    shape = synth.LLAMA3_8B
-    global N_CHUNKS, N_PARTS
-    reduced = bool(args.pool_blocks or args.chunks or args.parts)
-    if args.pool_blocks:
-        shape = shape.with_(n_blocks=args.pool_blocks)
-    N_CHUNKS = args.chunks or N_CHUNKS
-    N_PARTS = args.parts or N_PARTS
+    W = make_workload(args, synth)
+    shape = W["shape"]
+    T, PT, bs = W["chunk_tokens"], W["part_tokens"], shape.block_size
+    n_lib, n_retr, n_plib = W["lib"], len(W["retr"]), W["part_lib"]
+    n_parts_total = sum(len(r) for r in W["reqs"])
 
     # ---- inputs (untimed): pool, tables, chunk buffers; every rank has its own copy of the same workload
     k, v = synth.make_pool(shape, dev, seed=synth.SEED_VALUES + rank)
@@ -235,46 +254,60 @@ def run_gpu(args) -> None:
     pid = K.kdn_pool_register(ctx, desc)
     stream = torch.cuda.Stream(device=dev)
     s = stream.cuda_stream
-    bs = shape.block_size
-    blocks_per_chunk = CHUNK_TOKENS // bs
-    blocks_per_part = PART_TOKENS // bs
-    req_blocks = (N_PARTS * PART_TOKENS + SUFFIX_TOKENS) // bs
-    all_src = synth.make_table(N_CHUNKS * blocks_per_chunk, shape.n_blocks, 1, synth.SEED_TABLES)
-    all_dst = synth.make_table(N_CHUNKS * blocks_per_chunk, shape.n_blocks, 1, synth.SEED_TABLES + 1, exclude=all_src)
-    part_src = synth.make_table(N_PARTS * blocks_per_part, shape.n_blocks, 1, synth.SEED_TABLES + 2,
-                                exclude=np.concatenate([all_src, all_dst]))
-    req_tab = synth.make_table(req_blocks, shape.n_blocks, 1, synth.SEED_TABLES + 3,
-                               exclude=np.concatenate([all_src, all_dst, part_src]))
-    d_src = torch.from_numpy(all_src).to(dev)
-    d_dst = torch.from_numpy(all_dst).to(dev)
-    d_part_src = torch.from_numpy(part_src).to(dev)
-    d_req = torch.from_numpy(req_tab).to(dev)
+    bpc, bpp = T // bs, PT // bs
+    req_blocks = [(len(r) * PT + W["suffix"]) // bs for r in W["reqs"]]
+    taken = np.zeros(0, dtype=np.int64)
+
+    def table(n, seed):
+        nonlocal taken
+        t = synth.make_table(n, shape.n_blocks, 1, seed, exclude=taken if W["exclusive"] else None)
+        if W["exclusive"]:
+            taken = np.concatenate([taken, t])
+        return torch.from_numpy(t).to(dev)
+
+    d_src = table(n_lib * bpc, synth.SEED_TABLES)                 # where the library chunks are gathered from
+    d_dst = table(n_retr * bpc, synth.SEED_TABLES + 1)            # where retrievals land
+    d_part_src = table(n_plib * bpp, synth.SEED_TABLES + 2)
+    d_req = table(sum(req_blocks), synth.SEED_TABLES + 3)         # all composed requests, back to back
     i32 = 4
 
-    def make_sets(pinned: bool):
-        """Chunk buffers and the op lists of one step, per codec."""
+    def make_sets(pinned_lib, pinned_retr=()):
+        """Chunk buffers and the op lists of one step, per codec.  pinned_lib: the whole library lives in page-locked
+        host memory; pinned_retr: only these retrievals read a host copy of their chunk."""
         sets = {}
         for codec in (RAW, INT8):
-            cb = K.kdn_chunk_bytes(desc, CHUNK_TOKENS, codec)
-            pb = K.kdn_chunk_bytes(desc, PART_TOKENS, codec)
-            if pinned:
-                chunks = torch.empty(N_CHUNKS * cb, dtype=torch.uint8).pin_memory()
-                parts = torch.empty(N_PARTS * pb, dtype=torch.uint8).pin_memory()
+            cb, pb = K.kdn_chunk_bytes(desc, T, codec), K.kdn_chunk_bytes(desc, PT, codec)
+            if pinned_lib:
+                chunks = torch.empty(n_lib * cb, dtype=torch.uint8).pin_memory()
+                parts = torch.empty(n_plib * pb, dtype=torch.uint8).pin_memory()
                 mem = K.KDN_MEM_PINNED_HOST
             else:
-                chunks = torch.empty(N_CHUNKS * cb, dtype=torch.uint8, device=dev)
-                parts = torch.empty(N_PARTS * pb, dtype=torch.uint8, device=dev)
+                chunks = torch.empty(n_lib * cb, dtype=torch.uint8, device=dev)
+                parts = torch.empty(n_plib * pb, dtype=torch.uint8, device=dev)
                 mem = K.KDN_MEM_DEVICE
-            st_ops = [K.XferOp(d_src.data_ptr() + i * blocks_per_chunk * i32, blocks_per_chunk, 0,
-                               K.Chunk(chunks.data_ptr() + i * cb, cb, CHUNK_TOKENS, codec, mem)) for i in range(N_CHUNKS)]
-            rt_ops = [K.XferOp(d_dst.data_ptr() + i * blocks_per_chunk * i32, blocks_per_chunk, 0,
-                               K.Chunk(chunks.data_ptr() + i * cb, cb, CHUNK_TOKENS, codec, mem)) for i in range(N_CHUNKS)]
-            part_store = [K.XferOp(d_part_src.data_ptr() + j * blocks_per_part * i32, blocks_per_part, 0,
-                                   K.Chunk(parts.data_ptr() + j * pb, pb, PART_TOKENS, codec, mem)) for j in range(N_PARTS)]
-            req = K.ComposeReq(d_req.data_ptr(), req_blocks,
-                               [K.Chunk(parts.data_ptr() + j * pb, pb, PART_TOKENS, codec, mem, 0) for j in range(N_PARTS)],
-                               [j * PART_TOKENS for j in range(N_PARTS)], shape.rope_theta)
-            sets[codec] = dict(chunks=chunks, parts=parts, store=st_ops, retrieve=rt_ops, part_store=part_store, req=req)
+            host_copy = {}
+            for r in pinned_retr:
+                c = int(W["retr"][r])
+                if c not in host_copy:
+                    host_copy[c] = torch.empty(cb, dtype=torch.uint8).pin_memory()
+            st_ops = [K.XferOp(d_src.data_ptr() + c * bpc * i32, bpc, 0,
+                               K.Chunk(chunks.data_ptr() + c * cb, cb, T, codec, mem)) for c in range(n_lib)]
+            rt_ops = []
+            for r, c in enumerate(W["retr"]):
+                c = int(c)
+                ch = (K.Chunk(host_copy[c].data_ptr(), cb, T, codec, K.KDN_MEM_PINNED_HOST) if r in pinned_retr
+                      else K.Chunk(chunks.data_ptr() + c * cb, cb, T, codec, mem))
+                rt_ops.append(K.XferOp(d_dst.data_ptr() + r * bpc * i32, bpc, 0, ch))
+            part_store = [K.XferOp(d_part_src.data_ptr() + j * bpp * i32, bpp, 0,
+                                   K.Chunk(parts.data_ptr() + j * pb, pb, PT, codec, mem)) for j in range(n_plib)]
+            reqs, first = [], 0
+            for ids, nb_req in zip(W["reqs"], req_blocks):
+                reqs.append(K.ComposeReq(d_req.data_ptr() + first * i32, nb_req,
+                                         [K.Chunk(parts.data_ptr() + j * pb, pb, PT, codec, mem, 0) for j in ids],
+                                         [i * PT for i in range(len(ids))], shape.rope_theta))
+                first += nb_req
+            sets[codec] = dict(chunks=chunks, parts=parts, host_copy=host_copy, store=st_ops, retrieve=rt_ops,
+                               part_store=part_store, reqs=reqs)
         return sets
 
     dev_sets = make_sets(False)
@@ -283,30 +316,30 @@ def run_gpu(args) -> None:
     assert K.kdn_status_sync(ctx, s) == K.KDN_OK
 
     names = ["store_raw", "retrieve_raw", "compose_raw", "store_int8", "retrieve_int8", "compose_int8"]
-    chunk_elems = N_CHUNKS * CHUNK_TOKENS * shape.elems_per_token
-    part_elems = N_PARTS * PART_TOKENS * shape.elems_per_token
-    op_bytes = {"store_raw": chunk_elems * bytes_per_elem(RAW), "retrieve_raw": chunk_elems * bytes_per_elem(RAW),
-                "compose_raw": part_elems * bytes_per_elem(RAW), "store_int8": chunk_elems * bytes_per_elem(INT8),
-                "retrieve_int8": chunk_elems * bytes_per_elem(INT8), "compose_int8": part_elems * bytes_per_elem(INT8)}
-    op_tokens = {n: (N_CHUNKS * CHUNK_TOKENS if "compose" not in n else N_PARTS * PART_TOKENS) for n in names}
+    E = shape.elems_per_token
+    tokens_of = {"store": n_lib * T, "retrieve": n_retr * T, "compose": n_parts_total * PT}
+    op_tokens = {n: tokens_of[n.split("_")[0]] for n in names}
+    op_bytes = {n: op_tokens[n] * E * bytes_per_elem(INT8 if n.endswith("int8") else RAW) for n in names}
     step_bytes = float(sum(op_bytes.values()))
     reload_tokens = sum(op_tokens[n] for n in names if not n.startswith("store"))
-    kernel_of = {"store_raw": "kdn_store_kernel<false>", "retrieve_raw": "kdn_retrieve_kernel<false>",
-                 "compose_raw": "kdn_compose_kernel<true>", "store_int8": "kdn_store_kernel<true>",
-                 "retrieve_int8": "kdn_retrieve_kernel<true>", "compose_int8": "kdn_compose_kernel<true>"}
+    kernel_of = {"store_raw": "kdn_store_kernel<0>", "retrieve_raw": "kdn_retrieve_kernel<0>",
+                 "compose_raw": "kdn_compose_kernel<2>", "store_int8": "kdn_store_kernel<2>",
+                 "retrieve_int8": "kdn_retrieve_kernel<2>", "compose_int8": "kdn_compose_kernel<3>"}
 
-    def step(sets, events=None):
+    def step(sets, events=None, kinds=("store", "retrieve", "compose")):
         i = 0
         for codec in (RAW, INT8):
             for kind in ("store", "retrieve", "compose"):
                 if events is not None:
                     events[i].record(stream)
-                if kind == "store":
+                if kind not in kinds:
+                    pass
+                elif kind == "store":
                     K.kdn_store(ctx, pid, sets[codec]["store"], s)
                 elif kind == "retrieve":
                     K.kdn_retrieve(ctx, pid, sets[codec]["retrieve"], s)
                 else:
-                    K.kdn_compose(ctx, pid, [sets[codec]["req"]], s)
+                    K.kdn_compose(ctx, pid, sets[codec]["reqs"], s)
                 i += 1
         if events is not None:
             events[i].record(stream)
@@ -340,35 +373,57 @@ def run_gpu(args) -> None:
     op_ms = {n: float(np.mean([ev[it][i].elapsed_time(ev[it][i + 1]) for it in range(args.steps)]))
              for i, n in enumerate(names)}
 
-    # ---- end to end: the same step with every chunk in page-locked host memory
     if args.no_e2e:
         if rank == 0:
             print(json.dumps({"note": "profiling run, not a bench record", "ops_ms": op_ms,
                               "ops_gbs": {n: op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 for n in names}}))
         K.kdn_destroy(ctx)
         return
-    host_sets = make_sets(True)
-    for codec in (RAW, INT8):
-        K.kdn_store(ctx, pid, host_sets[codec]["part_store"], s)
-    assert K.kdn_status_sync(ctx, s) == K.KDN_OK
+
+    # ---- end to end: chunks in page-locked host memory, every byte crosses the host link inside the timed region
     e2e_steps = max(1, min(args.steps, args.e2e_steps))
-    step(host_sets)
+    if W["name"] == "llama3-8b":
+        # the whole step with the entire library on the host
+        del dev_sets
+        torch.cuda.empty_cache()
+        host_sets = make_sets(True)
+        e2e_kinds = ("store", "retrieve", "compose")
+        for codec in (RAW, INT8):
+            K.kdn_store(ctx, pid, host_sets[codec]["part_store"], s)
+        e2e_bytes = step_bytes
+        d2h = sum(K.kdn_chunk_bytes(desc, T, c) * n_lib for c in (RAW, INT8)) + 4
+        h2d = sum(K.kdn_chunk_bytes(desc, T, c) * n_retr + K.kdn_chunk_bytes(desc, PT, c) * n_parts_total for c in (RAW, INT8))
+        e2e_what = "whole step, every chunk in page-locked host memory"
+    else:
+        # the batched retrieve with four of its chunks on the host, copied in on the side stream while the
+        # device-resident retrievals run
+        pinned_retr = (5, 50, 90, 120)
+        host_sets = make_sets(False, pinned_retr)
+        for codec in (RAW, INT8):
+            host_sets[codec]["chunks"].copy_(dev_sets[codec]["chunks"])
+            for c, hb in host_sets[codec]["host_copy"].items():
+                cb = hb.numel()
+                hb.copy_(dev_sets[codec]["chunks"][c * cb:(c + 1) * cb])
+        e2e_kinds = ("retrieve",)
+        e2e_bytes = op_bytes["retrieve_raw"] + op_bytes["retrieve_int8"]
+        d2h = 4
+        h2d = sum(K.kdn_chunk_bytes(desc, T, c) * len(pinned_retr) for c in (RAW, INT8))
+        e2e_what = "batched retrieve, 4 of %d chunks in page-locked host memory (side stream)" % n_retr
+    assert K.kdn_status_sync(ctx, s) == K.KDN_OK
+    step(host_sets, kinds=e2e_kinds)
     assert K.kdn_status_sync(ctx, s) == K.KDN_OK
     barrier()
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
-        step(host_sets)
+        step(host_sets, kinds=e2e_kinds)
         st = K.kdn_status_sync(ctx, s)            # the step's result is read back: device status + all copies landed
         assert st == K.KDN_OK
     barrier()
     e2e_ms = (time.perf_counter() - t0) * 1e3
-    d2h = sum(K.kdn_chunk_bytes(desc, CHUNK_TOKENS, c) * N_CHUNKS for c in (RAW, INT8)) + 4
-    h2d = sum(K.kdn_chunk_bytes(desc, CHUNK_TOKENS, c) * N_CHUNKS + K.kdn_chunk_bytes(desc, PART_TOKENS, c) * N_PARTS
-              for c in (RAW, INT8))
 
     # ---- host-link ceiling, same run: one large pinned cudaMemcpyAsync each way
-    probe = host_sets[RAW]["chunks"][: 1 << 30]
-    dprobe = dev_sets[RAW]["chunks"][: 1 << 30]
+    probe = torch.empty(1 << 30, dtype=torch.uint8).pin_memory()
+    dprobe = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
     link = {}
     for name, (dst_t, src_t) in {"h2d": (dprobe, probe), "d2h": (probe, dprobe)}.items():
         best = 0.0
@@ -383,36 +438,35 @@ def run_gpu(args) -> None:
         link[name + "_gbs"] = best
 
     # ---- reduce over ranks (max time), print on rank 0
-    times = torch.tensor([elapsed_ms, e2e_ms] + [op_ms[n] for n in names], dtype=torch.float64, device=dev)
-    if dist is not None:
-        dist.all_reduce(times, op=dist.ReduceOp.MAX)
-    times = times.cpu().numpy()
+    times = shard.max_over_ranks([elapsed_ms, e2e_ms] + [op_ms[n] for n in names], device=dev)
     elapsed_ms, e2e_ms = float(times[0]), float(times[1])
     op_ms = {n: float(times[2 + i]) for i, n in enumerate(names)}
     if rank == 0:
         peak, peak_kind = measured_hbm_peak()
         ms_per_step = elapsed_ms / args.steps
-        value = world * step_bytes / (ms_per_step * 1e-3) / 1e9
+        value = shard.job_throughput(step_bytes, world, ms_per_step * 1e-3) / 1e9
         ops = {n: {"ms": op_ms[n], "gbs": op_bytes[n] / (op_ms[n] * 1e-3) / 1e9,
                    "frac_of_%s_copy_peak" % peak_kind: op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 / peak,
                    "frac_of_8000": op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 / 8000.0,
                    "tokens_per_s": op_tokens[n] / (op_ms[n] * 1e-3), "kernel": kernel_of[n]} for n in names}
         top = max(names, key=lambda n: op_ms[n])
-        traffic = measured_traffic(top, N_CHUNKS if "compose" not in top else N_PARTS)
+        units = {"store": n_lib * T / CHUNK_TOKENS, "retrieve": n_retr * T / CHUNK_TOKENS,
+                 "compose": n_parts_total * PT / PART_TOKENS}[top.split("_")[0]]
+        traffic = measured_traffic(top, units) if shape.elems_per_token == 65536 else None
         rec = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16/int8 (fp32 codec and rotation, fp64 angles)", "data": "synthetic",
-            "config": {"workload": WORKLOAD if not reduced else "REDUCED (%d chunks, %d parts, %d blocks): not the bench workload" % (N_CHUNKS, N_PARTS, shape.n_blocks), "l2": "inputs larger than L2 (every op streams >= 1.9 GB once)",
+            "config": {"workload": W["text"], "l2": "inputs larger than L2 (every op streams >= 1.9 GB once)",
                        "bytes_per_step": step_bytes},
             "tokens_per_s_reloaded": world * reload_tokens / (sum(op_ms[n] for n in names if not n.startswith("store")) * 1e-3),
             "ops": ops,
             "roofline": {"bound": "hbm", "kernel": kernel_of[top], "op": top, "achieved": ops[top]["gbs"], "peak": peak,
                          "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": ops[top]["gbs"] / peak,
                          "frac_of_nominal_8000": ops[top]["gbs"] / 8000.0, "traffic": traffic},
-            "e2e": {"value": world * step_bytes / (e2e_ms / e2e_steps * 1e-3) / 1e9, "unit": UNIT,
+            "e2e": {"value": world * e2e_bytes / (e2e_ms / e2e_steps * 1e-3) / 1e9, "unit": UNIT,
                     "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps,
-                    "ms_per_step": e2e_ms / e2e_steps,
+                    "ms_per_step": e2e_ms / e2e_steps, "what": e2e_what,
                     "host_link_gbs": (h2d + d2h) / (e2e_ms / e2e_steps * 1e-3) / 1e9, "host_link_peak": link},
             "gpu_launches": int(launches), "clocks": clocks,
         }
@@ -437,6 +491,8 @@ def main() -> None:
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-link leg (profiling runs)")
+    ap.add_argument("--workload", default="llama3-8b", choices=["llama3-8b", "llama3-70b"],
+                    help="llama3-8b is the benchmark workload; llama3-70b is the batched-retrieve configuration")
     ap.add_argument("--pool-blocks", type=int, default=0, help="smaller pool for profiler captures (default 16384)")
     ap.add_argument("--chunks", type=int, default=0, help="chunks per store/retrieve batch (default 64)")
     ap.add_argument("--parts", type=int, default=0, help="parts per composed request (default 10)")
