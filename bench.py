@@ -482,6 +482,69 @@ def run_gpu(args) -> None:
         dist.destroy_process_group()
 
 
+def run_sweep(args) -> None:
+    """GB/s against chunk length on the 8B shape: chunk length 128-8192 tokens x block_size {16, 32} x codec x block-table
+    fragmentation (runs of all / 64 / 8 / 1 consecutive physical blocks), store and retrieve, each point batching enough
+    distinct chunks to move at least 2 GiB.  Prints one JSON line per point and a final line with all of them."""
+    import torch
+    from paper_2409_13761_b200 import kdn as K, synth
+
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+    shape16 = synth.LLAMA3_8B
+    k, v = synth.make_pool(shape16, dev)
+    ctx = K.kdn_create(0)
+    pools = {}
+    for bs in (16, 32):
+        nb = shape16.n_blocks * 16 // bs
+        d = K.pool_desc(shape16.n_layers, shape16.n_kv_heads, shape16.head_dim, bs, nb,
+                        [t.data_ptr() for t in k], [t.data_ptr() for t in v])           # same memory, other block size
+        pools[bs] = (d, K.kdn_pool_register(ctx, d), nb)
+    stream = torch.cuda.Stream(device=dev)
+    s = stream.cuda_stream
+    E = shape16.elems_per_token
+    arena = torch.empty((2 << 30) + (256 << 20), dtype=torch.uint8, device=dev)
+    peak, peak_kind = measured_hbm_peak()
+    points = []
+    for bs in (16, 32):
+        desc, pid, nb = pools[bs]
+        for T in (128, 256, 512, 1024, 2048, 4096, 8192):
+            for codec in (RAW, INT8):
+                bpe = bytes_per_elem(codec)
+                n = max(1, -(-(2 << 30) // int(T * E * bpe)))
+                cb = K.kdn_chunk_bytes(desc, T, codec)
+                blocks = -(-T // bs)
+                for run in (None, 64, 8, 1):
+                    r = blocks if run is None else run
+                    src = synth.make_table(n * blocks, nb, r, synth.SEED_TABLES)
+                    dst = synth.make_table(n * blocks, nb, r, synth.SEED_TABLES + 1, exclude=src)
+                    d_src, d_dst = torch.from_numpy(src).to(dev), torch.from_numpy(dst).to(dev)
+                    ops = {"store": [K.XferOp(d_src.data_ptr() + i * blocks * 4, blocks, 0,
+                                               K.Chunk(arena.data_ptr() + i * cb, cb, T, codec)) for i in range(n)],
+                           "retrieve": [K.XferOp(d_dst.data_ptr() + i * blocks * 4, blocks, 0,
+                                                  K.Chunk(arena.data_ptr() + i * cb, cb, T, codec)) for i in range(n)]}
+                    row = {"block_size": bs, "chunk_tokens": T, "codec": "int8-g64" if codec else "raw", "chunks": n,
+                           "run_blocks": "all" if run is None else run, "gib_moved": n * T * E * bpe / 2 ** 30}
+                    for name, fn in (("store", K.kdn_store), ("retrieve", K.kdn_retrieve)):
+                        for _ in range(3):
+                            fn(ctx, pid, ops[name], s)
+                        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                        a.record(stream)
+                        for _ in range(args.steps):
+                            fn(ctx, pid, ops[name], s)
+                        b.record(stream)
+                        torch.cuda.synchronize()
+                        ms = a.elapsed_time(b) / args.steps
+                        row[name + "_gbs"] = n * T * E * bpe / (ms * 1e-3) / 1e9
+                        row[name + "_us"] = ms * 1e3
+                    assert K.kdn_status_sync(ctx, s) == K.KDN_OK
+                    points.append(row)
+                    print(json.dumps(row), flush=True)
+    K.kdn_destroy(ctx)
+    print(json.dumps({"sweep": "llama3-8b chunk length x block_size x codec x fragmentation", "peak_gbs": peak,
+                      "peak_kind": peak_kind, "reps": args.steps, "points": points}))
+
+
 def main() -> None:
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -491,6 +554,7 @@ def main() -> None:
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-link leg (profiling runs)")
+    ap.add_argument("--sweep", action="store_true", help="chunk-length / block-size / codec / fragmentation sweep (1 GPU)")
     ap.add_argument("--workload", default="llama3-8b", choices=["llama3-8b", "llama3-70b"],
                     help="llama3-8b is the benchmark workload; llama3-70b is the batched-retrieve configuration")
     ap.add_argument("--pool-blocks", type=int, default=0, help="smaller pool for profiler captures (default 16384)")
@@ -500,6 +564,8 @@ def main() -> None:
     args.warmup = max(3, args.warmup) if args.impl == "kdn" else args.warmup
     if args.impl == "reference":
         run_reference(args)
+    elif args.sweep:
+        run_sweep(args)
     else:
         run_gpu(args)
 
