@@ -7,8 +7,10 @@
 
 #include <cstdio>
 #include <cstring>
+#include <map>
 #include <mutex>
 #include <new>
+#include <utility>
 #include <vector>
 
 using namespace kdn;
@@ -134,10 +136,24 @@ kdn_status ensure_slabs(kdn_ctx *ctx)
     return KDN_OK;
 }
 
+// Largest dynamic shared-memory size already granted to each kernel on each device (setting the attribute on
+// every launch costs about a microsecond of host time).
+std::mutex g_attr_mutex;
+std::map<std::pair<int, const void *>, size_t> g_attr_granted;
+
 template <typename K>
 kdn_status launch_kernel(K kernel, int threads, unsigned grid, size_t smem, cudaStream_t stream, const Launch &lp)
 {
-    KDN_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+    {
+        int device = 0;
+        KDN_CUDA(cudaGetDevice(&device));
+        std::lock_guard<std::mutex> lock(g_attr_mutex);
+        size_t &granted = g_attr_granted[std::make_pair(device, (const void *)kernel)];
+        if (granted < smem) {
+            KDN_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+            granted = smem;
+        }
+    }
     kernel<<<grid, threads, smem, stream>>>(lp);
     KDN_CUDA(cudaGetLastError());
     return KDN_OK;
@@ -224,8 +240,18 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     if (fit != KDN_OK) return fit;
     const size_t smem = smem_bytes(stages, stage_bytes);
 
-    RingSlot &slot = ctx->ring[ctx->ring_next++ % kRing];
-    if (slot.used) KDN_CUDA(cudaEventSynchronize(slot.done));
+    // Few ops travel as kernel parameters; otherwise through a ring slot (pinned staging + device copy).  A ring
+    // slot is also what owns the rotation table.
+    const bool inl = n <= kInlineOps;
+    RingSlot *slot = nullptr;
+    if (!inl || any_rot) {
+        slot = &ctx->ring[ctx->ring_next++ % kRing];
+        if (slot->used) KDN_CUDA(cudaEventSynchronize(slot->done));
+    }
+    Launch lp{};
+    RopeInline rope_inl{};
+    DevOp *h_ops = inl ? lp.inline_ops : slot->h_ops;
+    RopeParam *h_rope = inl ? rope_inl.p : (slot ? slot->h_rope : nullptr);
 
     unsigned long long tiles = 0;
     int n_rope = 0;
@@ -234,36 +260,36 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
         op.tile_begin = (unsigned)tiles;
         op.rope = -1;
         if (hops[i].rotate) {
-            slot.h_rope[n_rope] = hops[i].rp;
+            h_rope[n_rope] = hops[i].rp;
             op.rope = n_rope++;
         }
-        slot.h_ops[i] = op;
+        h_ops[i] = op;
         tiles += (unsigned long long)op.nl * 2ull * (unsigned long long)op.nblk * tpb;
         if (tiles > kMaxTilesPerLaunch) return KDN_E_UNSUPPORTED;
     }
     if (tiles == 0) return KDN_OK;
 
-    KDN_CUDA(cudaMemcpyAsync(slot.d_ops, slot.h_ops, sizeof(DevOp) * (size_t)n, cudaMemcpyHostToDevice, stream));
+    if (!inl) KDN_CUDA(cudaMemcpyAsync(slot->d_ops, slot->h_ops, sizeof(DevOp) * (size_t)n, cudaMemcpyHostToDevice, stream));
     const int half = pool.D / 2;
     if (n_rope) {
-        if (slot.table_rows_cap < (size_t)n_rope || slot.table_half != half) {
-            KDN_CUDA(cudaEventSynchronize(slot.done));
-            if (slot.d_table) KDN_CUDA(cudaFree(slot.d_table));
-            slot.d_table = nullptr;
+        if (slot->table_rows_cap < (size_t)n_rope || slot->table_half != half) {
+            KDN_CUDA(cudaEventSynchronize(slot->done));
+            if (slot->d_table) KDN_CUDA(cudaFree(slot->d_table));
+            slot->d_table = nullptr;
             size_t rows = (size_t)n_rope < 64 ? 64 : (size_t)n_rope;
-            KDN_CUDA(cudaMalloc((void **)&slot.d_table, rows * (size_t)half * sizeof(float2)));
-            slot.table_rows_cap = rows;
-            slot.table_half = half;
+            KDN_CUDA(cudaMalloc((void **)&slot->d_table, rows * (size_t)half * sizeof(float2)));
+            slot->table_rows_cap = rows;
+            slot->table_half = half;
         }
-        KDN_CUDA(cudaMemcpyAsync(slot.d_rope, slot.h_rope, sizeof(RopeParam) * (size_t)n_rope, cudaMemcpyHostToDevice, stream));
+        if (!inl) KDN_CUDA(cudaMemcpyAsync(slot->d_rope, slot->h_rope, sizeof(RopeParam) * (size_t)n_rope, cudaMemcpyHostToDevice, stream));
         const long long total = (long long)n_rope * half;
-        kdn_rope_table_kernel<<<(unsigned)((total + 127) / 128), 128, 0, stream>>>(slot.d_rope, n_rope, pool.D, slot.d_table);
+        kdn_rope_table_kernel<<<(unsigned)((total + 127) / 128), 128, 0, stream>>>(inl ? nullptr : slot->d_rope, rope_inl, n_rope,
+                                                                              pool.D, slot->d_table);
         KDN_CUDA(cudaGetLastError());
         ctx->launches++;
     }
 
-    Launch lp{};
-    lp.ops = slot.d_ops;
+    lp.ops = inl ? nullptr : slot->d_ops;
     lp.n_ops = n;
     lp.n_tiles = (unsigned)tiles;
     lp.k_layers = pool.d_k;
@@ -274,7 +300,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     lp.row_elems = row_elems;
     lp.tile_elems = tile_elems;
     lp.tpb = tpb;
-    lp.rope = slot.d_table;
+    lp.rope = slot ? slot->d_table : nullptr;
     lp.status = ctx->d_status;
     lp.stages = stages;
     lp.stage_bytes = stage_bytes;
@@ -287,8 +313,10 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     kdn_status st = launch_tiles(OP, groups, grid, smem, stream, lp);
     if (st != KDN_OK) return st;
     ctx->launches++;
-    KDN_CUDA(cudaEventRecord(slot.done, stream));
-    slot.used = true;
+    if (slot) {
+        KDN_CUDA(cudaEventRecord(slot->done, stream));
+        slot->used = true;
+    }
     return KDN_OK;
 }
 
@@ -847,7 +875,7 @@ extern "C" kdn_status kdn_compose_static(int device, const kdn_pool_desc *pool, 
         if (n_rope) {
             const long long total = (long long)n_rope * half;
             kdn_rope_table_kernel<<<(unsigned)((total + 127) / 128), 128, 0, stream>>>(
-                reinterpret_cast<const RopeParam *>(sd->base + kStOffRope), n_rope, p.D, d_table);
+                reinterpret_cast<const RopeParam *>(sd->base + kStOffRope), RopeInline{}, n_rope, p.D, d_table);
             KDN_CUDA(cudaGetLastError());
         }
         Launch lp{};

@@ -63,8 +63,10 @@ struct RopeParam {            // one row of the rotation table to fill
     double theta;
 };
 
+constexpr int kInlineOps = 8;             // launches of up to this many ops carry them as kernel parameters
+
 struct Launch {
-    const DevOp *ops;
+    const DevOp *ops;         // device array of n_ops records, or nullptr: the records are in inline_ops
     int n_ops;
     unsigned n_tiles;
     void *const *k_layers;    // device arrays of per-layer pool pointers
@@ -82,6 +84,7 @@ struct Launch {
     unsigned off_b;           // offset of the code buffer inside a stage (compute launches)
     unsigned off_s;           // offset of the scale buffer inside a stage
     int store_lag;            // bulk-store groups that may still be reading shared memory (1..kMaxStoreLag)
+    DevOp inline_ops[kInlineOps];
 };
 
 struct __align__(16) TileDesc {
@@ -444,12 +447,13 @@ __device__ __forceinline__ void decode_tile(const Launch &P, unsigned g, TileDes
     d.n = 0; d.flags = 0; d.rope = -1; d.reserved = 0;
     d.g_pool = 0; d.g_chunk = 0; d.g_scales = 0;
     if (g >= P.n_tiles) return;                             // lanes past this CTA's last tile
+    const DevOp *ops = P.ops ? P.ops : P.inline_ops;       // global memory, or the kernel's parameter space
     int lo = 0, hi = P.n_ops - 1;
     while (lo < hi) {                                       // last op with tile_begin <= g
         int mid = (lo + hi + 1) >> 1;
-        if (__ldg(&P.ops[mid].tile_begin) <= g) lo = mid; else hi = mid - 1;
+        if (ops[mid].tile_begin <= g) lo = mid; else hi = mid - 1;
     }
-    const DevOp op = P.ops[lo];
+    const DevOp op = ops[lo];
     const unsigned gl = g - op.tile_begin;
     const unsigned per_plane = (unsigned)op.nblk * P.tpb;
     const unsigned plane = gl / per_plane;
@@ -708,8 +712,12 @@ kdn_compose_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_COMPOSE,
 
 // Rotation table: row r, frequency i -> (cos, sin) of delta_r * theta_r^(-2i/D), evaluated in fp64 and
 // rounded once to fp32 (an fp32 angle would lose more than half a bf16 ulp at large position shifts).
-__global__ void kdn_rope_table_kernel(const RopeParam *params, int n_rows, int D, float2 *table)
+struct RopeInline { RopeParam p[kInlineOps]; };
+
+__global__ void kdn_rope_table_kernel(const RopeParam *params, const __grid_constant__ RopeInline inl, int n_rows, int D,
+                                      float2 *table)
 {
+    if (!params) params = inl.p;                           // few rows: passed as kernel parameters
     const int half = D >> 1;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
     if (idx >= (long long)n_rows * half) return;
