@@ -131,7 +131,7 @@ class ClockSampler:
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, index: int):
+    def __init__(self, index):
         self.index = index
         self.proc = None
         self.lines = []
@@ -354,7 +354,11 @@ def run_gpu(args) -> None:
         step(dev_sets)
     assert K.kdn_status_sync(ctx, s) == K.KDN_OK
     ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(names) + 1)] for _ in range(args.steps)]
-    sampler = ClockSampler(torch.cuda.current_device() if "CUDA_VISIBLE_DEVICES" not in os.environ else local)
+    try:                                            # address the GPU by UUID: indices shift under CUDA_VISIBLE_DEVICES
+        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(local).uuid)
+    except Exception:
+        gpu_id = str(local)
+    sampler = ClockSampler(gpu_id)
     barrier()
     sampler.start()
     launches0 = K.kdn_launch_count(ctx)

@@ -392,3 +392,35 @@ def test_tuning_shapes_give_identical_results():
             K.kdn_set_tuning(dev.ctx, 100, 0, 0)                 # not a multiple of 128
     finally:
         dev.close()
+
+
+def test_more_ops_than_one_launch_carries():
+    """7000 tiny ops in one call: the library splits them over several launches; every chunk must still be right."""
+    shape = synth.TOY.with_(n_layers=1, n_kv_heads=1, head_dim=64, block_size=4, n_blocks=512)
+    dev = Device(shape, seed=8)
+    try:
+        K = dev.K
+        rng = np.random.default_rng(3)
+        host = dev.pool_np()
+        n = 7000
+        Ts = rng.integers(0, 4, n)                              # 0..3 tokens, some empty
+        offs = rng.integers(0, 4, n)
+        codecs = rng.integers(0, 2, n)
+        tabs = rng.integers(0, 512, (n, 2)).astype(np.int32)     # two blocks each, repeats allowed as a source
+        d_tabs = dev.table(tabs.reshape(-1))
+        sizes = [K.kdn_chunk_bytes(dev.desc, int(t), int(c)) for t, c in zip(Ts, codecs)]
+        starts = np.concatenate([[0], np.cumsum([(sz + 255) // 256 * 256 for sz in sizes])])
+        arena = torch.full((int(starts[-1]) + 256,), 0xA5, dtype=torch.uint8, device=dev.dev)
+        ops = [K.XferOp(d_tabs.data_ptr() + i * 8, 2, int(offs[i]),
+                        K.Chunk(arena.data_ptr() + int(starts[i]), sizes[i], int(Ts[i]), int(codecs[i]))) for i in range(n)]
+        n0 = K.kdn_launch_count(dev.ctx)
+        dev.store(ops)
+        assert dev.sync() == 0
+        assert K.kdn_launch_count(dev.ctx) - n0 >= 2
+        got = to_np(arena)
+        for i in range(n):
+            want = oracle.store(host, tabs[i], int(offs[i]), int(Ts[i]), int(codecs[i]))
+            assert np.array_equal(got[starts[i]:starts[i] + sizes[i]], want), i
+            assert np.all(got[starts[i] + sizes[i]:starts[i + 1]] == 0xA5)       # gaps between chunks untouched
+    finally:
+        dev.close()
