@@ -416,6 +416,28 @@ def run_gpu(args) -> None:
     assert K.kdn_status_sync(ctx, s) == K.KDN_OK
     step(host_sets, kinds=e2e_kinds)
     assert K.kdn_status_sync(ctx, s) == K.KDN_OK
+    layerwise = None
+    if W["name"] != "llama3-8b":
+        # layer-wise delivery of one host-resident chunk: when is the first layer range usable, when the last?
+        layerwise = {}
+        r0 = pinned_retr[0]
+        for codec, cname in ((RAW, "raw"), (INT8, "int8")):
+            op = [host_sets[codec]["retrieve"][r0]]
+            for mode, lps in (("whole", shape.n_layers), ("by_8_layers", 8)):
+                evs = [torch.cuda.Event(enable_timing=True) for _ in range(shape.n_layers)]
+                t_start = torch.cuda.Event(enable_timing=True)
+                for e in evs + [t_start]:
+                    e.record(stream)
+                torch.cuda.synchronize()
+                K.kdn_retrieve_layerwise(ctx, pid, op, lps, s, 0, [e.cuda_event for e in evs])   # warm
+                torch.cuda.synchronize()
+                t_start.record(stream)
+                K.kdn_retrieve_layerwise(ctx, pid, op, lps, s, 0, [e.cuda_event for e in evs])
+                torch.cuda.synchronize()
+                layerwise["%s_%s" % (cname, mode)] = {"first_layers_ready_ms": t_start.elapsed_time(evs[min(lps, shape.n_layers) - 1]),
+                                                      "all_layers_ready_ms": t_start.elapsed_time(evs[-1]),
+                                                      "chunk_bytes": K.kdn_chunk_bytes(desc, T, codec)}
+        assert K.kdn_status_sync(ctx, s) == K.KDN_OK
     barrier()
     t0 = time.perf_counter()
     for _ in range(e2e_steps):
@@ -471,7 +493,8 @@ def run_gpu(args) -> None:
             "e2e": {"value": world * e2e_bytes / (e2e_ms / e2e_steps * 1e-3) / 1e9, "unit": UNIT,
                     "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps,
                     "ms_per_step": e2e_ms / e2e_steps, "what": e2e_what,
-                    "host_link_gbs": (h2d + d2h) / (e2e_ms / e2e_steps * 1e-3) / 1e9, "host_link_peak": link},
+                    "host_link_gbs": (h2d + d2h) / (e2e_ms / e2e_steps * 1e-3) / 1e9, "host_link_peak": link,
+                    "layerwise_one_host_chunk": layerwise},
             "gpu_launches": int(launches), "clocks": clocks,
         }
         if not args.no_cpu_baseline and world == 1:

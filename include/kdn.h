@@ -183,6 +183,16 @@ kdn_status kdn_store(kdn_ctx *ctx, int pool_id, const kdn_xfer_op *ops, int n_op
 kdn_status kdn_retrieve(kdn_ctx *ctx, int pool_id, const kdn_xfer_op *ops, int n_ops,
                         void *cuda_stream, void *side_stream);
 
+/* Layer-wise delivery (Sec. 3.1 delivery module; Sec. 3 names the bandwidth of loading KV caches into GPU memory
+ * as the constraint once they live outside it): kdn_retrieve issued in steps of layers_per_step layers, first
+ * layers first, so that the engine can run layer l while later layers are still crossing the host link.
+ * layer_ready: NULL, or a HOST array of n_layers CUDA events (cudaEvent_t, entries may be NULL) owned by the
+ * caller; layer_ready[l] is recorded on cuda_stream once layers 0..l of every op of the call have been written.
+ * Results are exactly those of kdn_retrieve.  Each step is one launch (plus staged copies for pinned-host
+ * chunks), so small steps on small chunks cost launch overhead. */
+kdn_status kdn_retrieve_layerwise(kdn_ctx *ctx, int pool_id, const kdn_xfer_op *ops, int n_ops, int layers_per_step,
+                                  void *cuda_stream, void *side_stream, void *const *layer_ready);
+
 /* Sec. 3.1 blending module: compose every request's parts into its blocks; keys of parts whose
  * part_dst_pos differs from base_pos are re-rotated (see the top of this file).  A part with equal
  * positions, and every value plane, is written exactly as kdn_retrieve writes it. */

@@ -345,6 +345,8 @@ HostOp make_host_op(const Pool &pool, const int32_t *table, int64_t off, const k
     h.op.rope = -1;
     h.op.l0 = 0;
     h.op.nl = pool.L;
+    if (c.codec == KDN_CODEC_INT8_G64)
+        h.op.scales = (unsigned char *)c.data + (size_t)pool.L * 2u * (size_t)c.n_tokens * (size_t)pool.H * (size_t)pool.D;
     return h;
 }
 
@@ -400,8 +402,9 @@ kdn_status run_staged(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<
         if (per_layer > ctx->slab_bytes) return KDN_E_UNSUPPORTED;
         unsigned char *host = h.op.data;
         const size_t host_codes_total = (size_t)pool.L * codes_per_layer;
-        int l = 0;
-        while (l < pool.L) {
+        int l = h.op.l0;                                    // the op's own layer range (the whole chunk unless layer-wise)
+        const int l_end = h.op.l0 + h.op.nl;
+        while (l < l_end) {
             size_t room = ctx->slab_bytes - used;
             if (room < per_layer) {
                 st = flush();
@@ -409,7 +412,7 @@ kdn_status run_staged(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<
                 room = ctx->slab_bytes;
             }
             int nl = (int)(room / per_layer);
-            if (nl > pool.L - l) nl = pool.L - l;
+            if (nl > l_end - l) nl = l_end - l;
             // a piece is laid out exactly like a chunk of nl layers: codes, then scales
             const size_t base = used;
             const size_t cbytes = (size_t)nl * codes_per_layer;
@@ -419,6 +422,7 @@ kdn_status run_staged(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<
             sub.op.nl = nl;
             const unsigned s = ctx->slab_next & 1u;
             sub.op.data = ctx->slab[s] + base;
+            sub.op.scales = sbytes ? ctx->slab[s] + base + cbytes : nullptr;
             pieces.push_back(Piece{ host + (size_t)l * codes_per_layer, base, cbytes });
             if (sbytes) pieces.push_back(Piece{ host + host_codes_total + (size_t)l * scales_per_layer, base + cbytes, sbytes });
             batch.push_back(sub);
@@ -446,6 +450,22 @@ kdn_status run_ops(kdn_ctx *ctx, int pool_id, int OP, std::vector<HostOp> &dev_o
         st = run_staged(ctx, pool, OP, host_ops, stream, side);
     }
     return st;
+}
+
+// The record of `h` restricted to layers [l0, l0 + nl) of a device-resident chunk.
+HostOp layer_range(const Pool &pool, const HostOp &h, int l0, int nl)
+{
+    HostOp sub = h;
+    const size_t plane = 2u * (size_t)h.op.T * (size_t)pool.H * (size_t)pool.D;     // elements of one layer
+    sub.op.l0 = l0;
+    sub.op.nl = nl;
+    if (h.op.codec == KDN_CODEC_INT8_G64) {
+        sub.op.data = h.op.data + (size_t)l0 * plane;
+        sub.op.scales = h.op.scales + (size_t)l0 * (plane / 64u) * 4u;
+    } else {
+        sub.op.data = h.op.data + (size_t)l0 * plane * 2u;
+    }
+    return sub;
 }
 
 kdn_pool_desc shape_of(const Pool &p)
@@ -626,6 +646,37 @@ kdn_status kdn_store(kdn_ctx *ctx, int pool_id, const kdn_xfer_op *ops, int n_op
 kdn_status kdn_retrieve(kdn_ctx *ctx, int pool_id, const kdn_xfer_op *ops, int n_ops, void *cuda_stream, void *side_stream)
 {
     return xfer(ctx, pool_id, OP_RETRIEVE, ops, n_ops, cuda_stream, side_stream);
+}
+
+kdn_status kdn_retrieve_layerwise(kdn_ctx *ctx, int pool_id, const kdn_xfer_op *ops, int n_ops, int layers_per_step,
+                                  void *cuda_stream, void *side_stream, void *const *layer_ready)
+{
+    if (!ctx || pool_id < 0 || (size_t)pool_id >= ctx->pools.size() || layers_per_step < 1) return KDN_E_INVAL;
+    const Pool &pool = ctx->pools[(size_t)pool_id];
+    const kdn_pool_desc shape = shape_of(pool);
+    kdn_status st = kdn_validate_xfer(&shape, ops, n_ops);
+    if (st != KDN_OK) return st;
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return KDN_E_CUDA;
+    std::vector<HostOp> dev_all, host_all;
+    for (int i = 0; i < n_ops; ++i) {
+        if (ops[i].chunk.n_tokens == 0) continue;
+        HostOp h = make_host_op(pool, ops[i].block_table, ops[i].token_offset, ops[i].chunk);
+        (ops[i].chunk.mem == KDN_MEM_PINNED_HOST ? host_all : dev_all).push_back(h);
+    }
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    for (int l0 = 0; l0 < pool.L; l0 += layers_per_step) {
+        const int nl = pool.L - l0 < layers_per_step ? pool.L - l0 : layers_per_step;
+        std::vector<HostOp> dev_ops, host_ops;
+        for (const HostOp &h : dev_all) dev_ops.push_back(layer_range(pool, h, l0, nl));
+        // a host-resident chunk keeps its full-chunk addresses; run_staged cuts out the layer range itself
+        for (const HostOp &h : host_all) { HostOp sub = h; sub.op.l0 = l0; sub.op.nl = nl; host_ops.push_back(sub); }
+        st = run_ops(ctx, pool_id, OP_RETRIEVE, dev_ops, host_ops, cuda_stream, side_stream);
+        if (st != KDN_OK) return st;
+        if (layer_ready)
+            for (int l = l0; l < l0 + nl; ++l)
+                if (layer_ready[l]) KDN_CUDA(cudaEventRecord((cudaEvent_t)layer_ready[l], stream));
+    }
+    return KDN_OK;
 }
 
 kdn_status kdn_compose(kdn_ctx *ctx, int pool_id, const kdn_compose_req *reqs, int n_reqs, void *cuda_stream, void *side_stream)

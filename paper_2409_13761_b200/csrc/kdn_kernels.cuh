@@ -44,7 +44,7 @@ constexpr int kStatusTimeout = 8;
 
 struct __align__(16) DevOp {
     const int32_t *table;     // device block table of the request
-    unsigned char *data;      // chunk bytes for layers [l0, l0 + nl): raw bf16, or codes then scales
+    unsigned char *data;      // layers [l0, l0 + nl) of the chunk: raw bf16, or int8 codes
     long long off;            // request position of chunk token 0
     int T;                    // tokens
     int codec;                // 0 raw bf16, 1 int8 group-64
@@ -54,7 +54,7 @@ struct __align__(16) DevOp {
     int rope;                 // row of the rotation table, -1: keys are copied
     int l0;                   // first pool layer
     int nl;                   // layers held in data
-    long long reserved;
+    unsigned char *scales;    // int8: fp32 scales of the same layers; raw: unused
 };
 static_assert(sizeof(DevOp) == 64, "DevOp is copied as 64-byte records");
 
@@ -481,8 +481,7 @@ __device__ __forceinline__ void decode_tile(const Launch &P, unsigned g, TileDes
     } else {
         d.flags |= TF_INT8;
         d.g_chunk = (unsigned long long)(op.data + ce);
-        const unsigned long long codes_bytes = (unsigned long long)op.nl * 2ull * op.T * P.row_elems;
-        d.g_scales = (unsigned long long)(op.data + codes_bytes + (ce >> 6) * 4ull);
+        d.g_scales = (unsigned long long)(op.scales + (ce >> 6) * 4ull);
         if ((d.g_scales & 15ull) || ((n >> 6) & 3u)) d.flags |= TF_SCALES_PLAIN;
     }
     if (OP == OP_COMPOSE && kv == 0 && op.rope >= 0) { d.flags |= TF_ROTATE; d.rope = op.rope; }

@@ -21,7 +21,7 @@ KDN_MEM_DEVICE, KDN_MEM_PINNED_HOST = 0, 1
 EXPORTS = ["kdn_create", "kdn_destroy", "kdn_pool_register", "kdn_chunk_bytes", "kdn_validate_xfer",
            "kdn_validate_compose", "kdn_store", "kdn_retrieve", "kdn_compose", "kdn_status_sync",
            "kdn_set_tuning", "kdn_set_staging_bytes", "kdn_launch_count", "kdn_strerror",
-           "kdn_compose_static"]
+           "kdn_compose_static", "kdn_retrieve_layerwise"]
 
 
 class kdn_pool_desc(C.Structure):
@@ -77,6 +77,8 @@ def _load() -> C.CDLL:
         fn = getattr(lib, name)
         fn.restype = i32
         fn.argtypes = [vp, i32, C.POINTER(kdn_xfer_op), i32, vp, vp]
+    lib.kdn_retrieve_layerwise.restype = i32
+    lib.kdn_retrieve_layerwise.argtypes = [vp, i32, C.POINTER(kdn_xfer_op), i32, i32, vp, vp, C.POINTER(vp)]
     lib.kdn_compose.restype = i32
     lib.kdn_compose.argtypes = [vp, i32, C.POINTER(kdn_compose_req), i32, vp, vp]
     lib.kdn_compose_static.restype = i32
@@ -215,6 +217,16 @@ def kdn_store(ctx, pool_id: int, ops: Sequence[XferOp], stream: int = 0, side_st
 
 def kdn_retrieve(ctx, pool_id: int, ops: Sequence[XferOp], stream: int = 0, side_stream: int = 0) -> None:
     _check(lib.kdn_retrieve(ctx, pool_id, xfer_array(ops), len(ops), stream, side_stream), "kdn_retrieve")
+
+
+def kdn_retrieve_layerwise(ctx, pool_id: int, ops: Sequence[XferOp], layers_per_step: int, stream: int = 0,
+                           side_stream: int = 0, layer_ready: Optional[Sequence[int]] = None) -> None:
+    """layer_ready: one cudaEvent_t handle (int, 0 = none) per layer, or None."""
+    ev = None
+    if layer_ready is not None:
+        ev = (C.c_void_p * len(layer_ready))(*[int(e) if e else None for e in layer_ready])
+    _check(lib.kdn_retrieve_layerwise(ctx, pool_id, xfer_array(ops), len(ops), int(layers_per_step), stream, side_stream,
+                                      ev), "kdn_retrieve_layerwise")
 
 
 def kdn_compose(ctx, pool_id: int, reqs: Sequence[ComposeReq], stream: int = 0, side_stream: int = 0) -> None:

@@ -424,3 +424,40 @@ def test_more_ops_than_one_launch_carries():
             assert np.all(got[starts[i] + sizes[i]:starts[i + 1]] == 0xA5)       # gaps between chunks untouched
     finally:
         dev.close()
+
+
+@pytest.mark.parametrize("codec", [RAW, INT8])
+def test_layerwise_retrieve_equals_retrieve_and_events_order_layers(codec):
+    """Layer-wise delivery: same bits as a plain retrieve; after waiting for layer l's event, layers 0..l are complete
+    (checked while later layers may still be in flight); device and pinned-host chunks mixed in one call."""
+    shape = synth.TOY.with_(n_layers=7, n_kv_heads=2, head_dim=64, block_size=16, n_blocks=64)
+    dev = Device(shape, seed=19)
+    try:
+        K = dev.K
+        K.kdn_set_staging_bytes(dev.ctx, 64 * 1024)
+        host = dev.pool_np()
+        perm = np.random.default_rng(9).permutation(64).astype(np.int32)
+        T1, T2 = 70, 33
+        b1, b2 = dev.chunk_buf(T1, codec), dev.chunk_buf(T2, codec, pinned=True)
+        dev.store([dev.op(dev.table(perm[:5]), 3, b1, T1, codec), dev.op(dev.table(perm[5:8]), 0, b2, T2, codec)])
+        assert dev.sync() == 0
+        ops = [dev.op(dev.table(perm[20:25]), 9, b1, T1, codec), dev.op(dev.table(perm[30:33]), 2, b2, T2, codec)]
+        ref = host.copy()
+        oracle.retrieve(ref, perm[20:25], 9, T1, codec, oracle.store(host, perm[:5], 3, T1, codec))
+        oracle.retrieve(ref, perm[30:33], 2, T2, codec, oracle.store(host, perm[5:8], 0, T2, codec))
+        events = [torch.cuda.Event() for _ in range(shape.n_layers)]
+        for e in events:
+            e.record(dev.stream)                                  # creates the underlying CUDA event
+        torch.cuda.synchronize()
+        K.kdn_retrieve_layerwise(dev.ctx, dev.pool_id, ops, 3, dev.stream.cuda_stream, 0, [e.cuda_event for e in events])
+        for l in range(shape.n_layers):
+            events[l].synchronize()
+            got_k = dev.k[l].view(torch.int16).cpu().numpy().view(np.uint16)
+            got_v = dev.v[l].view(torch.int16).cpu().numpy().view(np.uint16)
+            assert np.array_equal(got_k, ref[l, 0]) and np.array_equal(got_v, ref[l, 1]), l
+        assert dev.sync() == 0
+        assert np.array_equal(dev.pool_np(), ref)
+        with pytest.raises(K.KdnError):
+            K.kdn_retrieve_layerwise(dev.ctx, dev.pool_id, ops, 0, dev.stream.cuda_stream)
+    finally:
+        dev.close()
