@@ -10,6 +10,7 @@ Array conventions (all host, C-contiguous numpy):
   table   int32  [n_table_blocks]
   chunk   uint8  [chunk_bytes]  raw: bf16 [L][2][T][H][D];
                                 int8: int8 codes [L][2][T][H][D] then fp32 scales [L][2][T][H*D/64]
+                                int4: nibbles [L][2][T][H][D/2] bytes (element 2k low, 2k+1 high) then the same scales
 """
 from __future__ import annotations
 
@@ -22,6 +23,7 @@ import numpy as np
 
 RAW_BF16 = 0
 INT8_G64 = 1
+INT4_G64 = 2
 GROUP = 64
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -59,6 +61,8 @@ def lib():
             L.kdn_oracle_chunk_bytes.argtypes = [i32, i32, i32, i32, i32]
             L.kdn_oracle_quant_group.restype = None
             L.kdn_oracle_quant_group.argtypes = [vp, vp, vp]
+            L.kdn_oracle_quant4_group.restype = None
+            L.kdn_oracle_quant4_group.argtypes = [vp, vp, vp]
             L.kdn_oracle_dequant.restype = C.c_uint16
             L.kdn_oracle_dequant.argtypes = [C.c_int8, C.c_float]
             L.kdn_oracle_rope_angle.restype = f64
@@ -163,6 +167,17 @@ def quant_group(x_bf16: np.ndarray):
     q = np.zeros(GROUP, dtype=np.int8)
     s = np.zeros(1, dtype=np.float32)
     lib().kdn_oracle_quant_group(_ptr(x), _ptr(q), _ptr(s))
+    return q, s[0]
+
+
+def quant4_group(x_bf16: np.ndarray):
+    """Encode one group of 64 bf16 bit patterns -> (32 bytes of nibbles, fp32 scale)."""
+    x = np.ascontiguousarray(x_bf16, dtype=np.uint16)
+    if x.shape != (GROUP,):
+        raise ValueError("a group is 64 values")
+    q = np.zeros(GROUP // 2, dtype=np.uint8)
+    s = np.zeros(1, dtype=np.float32)
+    lib().kdn_oracle_quant4_group(_ptr(x), _ptr(q), _ptr(s))
     return q, s[0]
 
 

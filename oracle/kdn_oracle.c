@@ -32,6 +32,11 @@
  *                    q = clamp(round_half_even(x * inv), -127, 127), the
  *                    product being one fp32 multiply.
  *   R5  decode       x^ = bf16_rne((float)q * scale), one fp32 multiply.
+ *   R4' int4 codec   (a stronger codec on the way to the "over 10x" footprint reduction Sec. 3.2 cites; not
+ *                    prescribed by the paper) same as R4 with 7 in place of 127: scale = a / 7, inv = 7 / a,
+ *                    q = clamp(round_half_even(x * inv), -7, 7); two codes per byte as two's-complement
+ *                    nibbles, element 2k in the low nibble and 2k+1 in the high nibble of byte k;
+ *                    chunk = nibbles[l][kv][t][head][D/2] bytes followed by the fp32 scales as in R2.
  *   R6  re-rotation  stored keys carry rotary position embedding at absolute
  *                    positions base_pos + t (what an engine's pool holds), so
  *                    reuse at dst_pos (Sec. 3.2 "KV-cache blending": a
@@ -60,6 +65,7 @@
 
 #define KDN_ORACLE_RAW_BF16 0
 #define KDN_ORACLE_INT8_G64 1
+#define KDN_ORACLE_INT4_G64 2
 #define KDN_ORACLE_GROUP 64
 
 /* ---------------------------------------------------------------- bf16 -- */
@@ -130,34 +136,59 @@ size_t kdn_oracle_chunk_bytes(int L, int H, int D, int T, int codec)
         if (D % KDN_ORACLE_GROUP) return 0;
         return elems + 4u * (elems / KDN_ORACLE_GROUP);
     }
+    if (codec == KDN_ORACLE_INT4_G64) {
+        if (D % KDN_ORACLE_GROUP) return 0;
+        return elems / 2u + 4u * (elems / KDN_ORACLE_GROUP);
+    }
     return 0;
 }
 
 /* ------------------------------------------------------------ int8 codec -- */
 
-/* R4: encode one group of 64 bf16 values. */
-void kdn_oracle_quant_group(const uint16_t *x_bf16, int8_t *q, float *scale_out)
+/* R4 / R4': encode one group of 64 bf16 values with codes in [-qmax, qmax] (127 or 7). */
+static void quant_group_q(const uint16_t *x_bf16, int8_t *q, float *scale_out, float qmax)
 {
     float a = 0.0f;
     for (int i = 0; i < KDN_ORACLE_GROUP; ++i) {
         float v = fabsf(kdn_oracle_bf16_to_f32(x_bf16[i]));
         if (v > a) a = v;
     }
-    volatile float scale = a / 127.0f;             /* volatile: one fp32 divide, stored as fp32 */
+    volatile float scale = a / qmax;               /* volatile: one fp32 divide, stored as fp32 */
     if (!(scale >= FLT_MIN)) {
         *scale_out = 0.0f;
         for (int i = 0; i < KDN_ORACLE_GROUP; ++i) q[i] = 0;
         return;
     }
-    volatile float inv = 127.0f / a;
+    volatile float inv = qmax / a;
     for (int i = 0; i < KDN_ORACLE_GROUP; ++i) {
         volatile float prod = kdn_oracle_bf16_to_f32(x_bf16[i]) * inv;   /* one fp32 multiply */
         float r = rintf(prod);                     /* default rounding mode: ties to even */
-        if (r > 127.0f) r = 127.0f;
-        if (r < -127.0f) r = -127.0f;
+        if (r > qmax) r = qmax;
+        if (r < -qmax) r = -qmax;
         q[i] = (int8_t)(int)r;
     }
     *scale_out = scale;
+}
+
+void kdn_oracle_quant_group(const uint16_t *x_bf16, int8_t *q, float *scale_out)
+{
+    quant_group_q(x_bf16, q, scale_out, 127.0f);
+}
+
+/* R4': 64 values -> 32 bytes of nibbles + one scale. */
+void kdn_oracle_quant4_group(const uint16_t *x_bf16, uint8_t *packed, float *scale_out)
+{
+    int8_t q[KDN_ORACLE_GROUP];
+    quant_group_q(x_bf16, q, scale_out, 7.0f);
+    for (int k = 0; k < KDN_ORACLE_GROUP / 2; ++k)
+        packed[k] = (uint8_t)(((uint8_t)q[2 * k] & 0x0fu) | (((uint8_t)q[2 * k + 1] & 0x0fu) << 4));
+}
+
+/* R4': the code of element i (0 <= i < 64) of a packed group, sign-extended. */
+int kdn_oracle_nibble(const uint8_t *packed, size_t i)
+{
+    int v = (i & 1u) ? (packed[i >> 1] >> 4) : (packed[i >> 1] & 0x0f);
+    return v >= 8 ? v - 16 : v;
 }
 
 /* R5: decode one code. */
@@ -219,8 +250,8 @@ static int check_args(const shape_t *s, const int32_t *table, int n_table, int64
     if (s->L <= 0 || s->H <= 0 || s->D <= 0 || s->bs <= 0 || s->nb <= 0) return 1;
     if (T < 0 || off < 0 || n_table < 0) return 1;
     if (off + (int64_t)T > (int64_t)n_table * (int64_t)s->bs) return 2;
-    if (codec != KDN_ORACLE_RAW_BF16 && codec != KDN_ORACLE_INT8_G64) return 3;
-    if (codec == KDN_ORACLE_INT8_G64 && s->D % KDN_ORACLE_GROUP) return 3;
+    if (codec != KDN_ORACLE_RAW_BF16 && codec != KDN_ORACLE_INT8_G64 && codec != KDN_ORACLE_INT4_G64) return 3;
+    if (codec != KDN_ORACLE_RAW_BF16 && s->D % KDN_ORACLE_GROUP) return 3;
     for (int64_t p = off; p < off + T; ++p) {
         int32_t b = table[p / s->bs];
         if (b < 0 || (int64_t)b >= s->nb) return 4;
@@ -243,7 +274,7 @@ int kdn_oracle_store(const uint16_t *pool, int L, int H, int D, int bs, int64_t 
     size_t elems = (size_t)L * 2u * (size_t)T * (size_t)H * (size_t)D;
     uint16_t *raw = (uint16_t *)chunk;
     int8_t *codes = (int8_t *)chunk;
-    float *scales = (float *)(chunk + elems);
+    float *scales = (float *)(chunk + (codec == KDN_ORACLE_INT4_G64 ? elems / 2u : elems));
     for (int l = 0; l < L; ++l)
         for (int kv = 0; kv < 2; ++kv)
             for (int t = 0; t < T; ++t) {
@@ -251,7 +282,13 @@ int kdn_oracle_store(const uint16_t *pool, int L, int H, int D, int bs, int64_t 
                 int64_t block = table[p / bs];
                 int slot = (int)(p % bs);
                 for (int h = 0; h < H; ++h) {
-                    if (codec == KDN_ORACLE_RAW_BF16) {
+                    if (codec == KDN_ORACLE_INT4_G64) {
+                        for (int g = 0; g < D / KDN_ORACLE_GROUP; ++g) {
+                            size_t src = pool_index(&s, l, kv, block, slot, h, g * KDN_ORACLE_GROUP);
+                            size_t dst = chunk_index(&s, T, l, kv, t, h, g * KDN_ORACLE_GROUP);
+                            kdn_oracle_quant4_group(pool + src, chunk + dst / 2u, scales + dst / KDN_ORACLE_GROUP);
+                        }
+                    } else if (codec == KDN_ORACLE_RAW_BF16) {
                         for (int d = 0; d < D; ++d)
                             raw[chunk_index(&s, T, l, kv, t, h, d)] =
                                 pool[pool_index(&s, l, kv, block, slot, h, d)];
@@ -267,6 +304,28 @@ int kdn_oracle_store(const uint16_t *pool, int L, int H, int D, int bs, int64_t 
     return 0;
 }
 
+/* The stored value of chunk element c before any bf16 rounding: code and scale (raw: the bf16 itself). */
+static void stored_code(const uint8_t *chunk, size_t elems, int codec, size_t c, int *q, float *scale)
+{
+    if (codec == KDN_ORACLE_INT8_G64) {
+        *q = ((const int8_t *)chunk)[c];
+        *scale = ((const float *)(chunk + elems))[c / KDN_ORACLE_GROUP];
+    } else {                                       /* int4 */
+        *q = kdn_oracle_nibble(chunk, c);
+        *scale = ((const float *)(chunk + elems / 2u))[c / KDN_ORACLE_GROUP];
+    }
+}
+
+/* R5: the bf16 a retrieve writes for chunk element c. */
+static uint16_t decoded(const uint8_t *chunk, size_t elems, int codec, size_t c)
+{
+    if (codec == KDN_ORACLE_RAW_BF16) return ((const uint16_t *)chunk)[c];
+    int q;
+    float scale;
+    stored_code(chunk, elems, codec, c, &q, &scale);
+    return kdn_oracle_dequant((int8_t)q, scale);
+}
+
 /* ------------------------------------------------------------- retrieve -- */
 
 /* Sec. 3.2 call (ii) with Sec. 3.1's "decompresses them in GPU": scatter a
@@ -280,9 +339,6 @@ int kdn_oracle_retrieve(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
     int rc = check_args(&s, table, n_table, off, T, codec);
     if (rc) return rc;
     size_t elems = (size_t)L * 2u * (size_t)T * (size_t)H * (size_t)D;
-    const uint16_t *raw = (const uint16_t *)chunk;
-    const int8_t *codes = (const int8_t *)chunk;
-    const float *scales = (const float *)(chunk + elems);
     for (int l = 0; l < L; ++l)
         for (int kv = 0; kv < 2; ++kv)
             for (int t = 0; t < T; ++t) {
@@ -293,9 +349,7 @@ int kdn_oracle_retrieve(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
                     for (int d = 0; d < D; ++d) {
                         size_t c = chunk_index(&s, T, l, kv, t, h, d);
                         size_t o = pool_index(&s, l, kv, block, slot, h, d);
-                        pool[o] = (codec == KDN_ORACLE_RAW_BF16)
-                                      ? raw[c]
-                                      : kdn_oracle_dequant(codes[c], scales[c / KDN_ORACLE_GROUP]);
+                        pool[o] = decoded(chunk, elems, codec, c);
                     }
             }
     return 0;
@@ -336,8 +390,6 @@ int kdn_oracle_compose(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
         int64_t delta = dst_pos[j] - base_pos[j];
         size_t elems = (size_t)L * 2u * (size_t)T * (size_t)H * (size_t)D;
         const uint16_t *raw = (const uint16_t *)chunks[j];
-        const int8_t *codes = (const int8_t *)chunks[j];
-        const float *scales = (const float *)(chunks[j] + elems);
         for (int l = 0; l < L; ++l)
             for (int kv = 0; kv < 2; ++kv)
                 for (int t = 0; t < T; ++t) {
@@ -350,9 +402,7 @@ int kdn_oracle_compose(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
                             for (int d = 0; d < D; ++d) {
                                 size_t c = chunk_index(&s, T, l, kv, t, h, d);
                                 size_t o = pool_index(&s, l, kv, block, slot, h, d);
-                                pool[o] = (codec == KDN_ORACLE_RAW_BF16)
-                                              ? raw[c]
-                                              : kdn_oracle_dequant(codes[c], scales[c / KDN_ORACLE_GROUP]);
+                                pool[o] = decoded(chunks[j], elems, codec, c);
                                 if (kv == 0 && kref) {
                                     size_t r = (((size_t)l * (size_t)P + (size_t)p) * (size_t)H + (size_t)h) * (size_t)D + (size_t)d;
                                     kref[r] = (double)kdn_oracle_bf16_to_f32(pool[o]);
@@ -369,8 +419,12 @@ int kdn_oracle_compose(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
                                 u = (double)kdn_oracle_bf16_to_f32(raw[cu]);
                                 w = (double)kdn_oracle_bf16_to_f32(raw[cw]);
                             } else {
-                                u = (double)codes[cu] * (double)scales[cu / KDN_ORACLE_GROUP];
-                                w = (double)codes[cw] * (double)scales[cw / KDN_ORACLE_GROUP];
+                                int qu, qw;
+                                float su, sw;
+                                stored_code(chunks[j], elems, codec, cu, &qu, &su);
+                                stored_code(chunks[j], elems, codec, cw, &qw, &sw);
+                                u = (double)qu * (double)su;
+                                w = (double)qw * (double)sw;
                             }
                             double phi = kdn_oracle_rope_angle(delta, theta, i, D);
                             double u2, w2;
