@@ -28,12 +28,16 @@
  *   KDN_CODEC_RAW_BF16   bf16 data[L][2][T][H][D]               4*L*T*H*D bytes
  *   KDN_CODEC_INT8_G64   int8 codes[L][2][T][H][D] followed by
  *                        fp32 scales[L][2][T][H*D/64]           2*L*T*H*D*(1+4/64) bytes
+ *   KDN_CODEC_INT4_G64   nibbles[L][2][T][H][D/2] bytes (element 2k in the low, 2k+1 in the high nibble,
+ *                        two's complement) followed by the same fp32 scales       L*T*H*D*(1+1/8) bytes
  *   No header, no padding, little endian.  A chunk does not record where it
  *   sat in the pool; it can be retrieved into any blocks of any request.
  * int8 coding: group = 64 consecutive head_dim elements of one token-head row;
  *   a = max|x|, scale = a/127 in fp32; scale < FLT_MIN -> scale 0, codes 0;
  *   else code = round_half_even(x * (127/a)) in fp32, in [-127, 127];
  *   decode = bf16_round_nearest_even((float)code * scale).
+ * int4 coding: the same with 7 in place of 127 (scale = a/7, code in [-7, 7]); a stronger codec towards the
+ *   "over 10x" footprint reduction Sec. 3.2 ("KV-cache delivery") cites.
  * Key re-rotation in kdn_compose: the stored keys of a part carry rotary
  *   position embedding for positions base_pos + t; placing the part at
  *   dst_pos rotates each pair (k[i], k[i + D/2]) of every head by
@@ -71,13 +75,13 @@ typedef enum {
     KDN_E_SHAPE = 2,        /* chunk.bytes or n_tokens does not match the pool's shape */
     KDN_E_ALIGN = 3,        /* a pointer is not 16-byte aligned, or H*D*2 is not a multiple of 16 */
     KDN_E_RANGE = 4,        /* token range beyond the block table; block id outside the pool (device) */
-    KDN_E_UNSUPPORTED = 5,  /* int8 with head_dim % 64 != 0; rotation with head_dim % 16 != 0; ... */
+    KDN_E_UNSUPPORTED = 5,  /* int8 / int4 with head_dim % 64 != 0; rotation with head_dim % 16 != 0; ... */
     KDN_E_CUDA = 6,         /* a CUDA runtime call failed */
     KDN_E_NOMEM = 7,        /* context scratch could not be allocated */
     KDN_E_TIMEOUT = 8       /* a bounded wait inside a kernel gave up (device) */
 } kdn_status;
 
-typedef enum { KDN_CODEC_RAW_BF16 = 0, KDN_CODEC_INT8_G64 = 1 } kdn_codec;
+typedef enum { KDN_CODEC_RAW_BF16 = 0, KDN_CODEC_INT8_G64 = 1, KDN_CODEC_INT4_G64 = 2 } kdn_codec;
 typedef enum { KDN_MEM_DEVICE = 0, KDN_MEM_PINNED_HOST = 1 } kdn_mem;
 
 /* An engine's paged KV pool (Sec. 3.2 names vLLM's paged memory).  k_layers and v_layers are HOST

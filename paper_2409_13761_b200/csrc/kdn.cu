@@ -98,9 +98,9 @@ kdn_status check_shape(const kdn_pool_desc *p)
 kdn_status check_chunk(const kdn_pool_desc *p, const kdn_chunk *c)
 {
     if (c->n_tokens < 0) return KDN_E_INVAL;
-    if (c->codec != KDN_CODEC_RAW_BF16 && c->codec != KDN_CODEC_INT8_G64) return KDN_E_INVAL;
+    if (c->codec != KDN_CODEC_RAW_BF16 && c->codec != KDN_CODEC_INT8_G64 && c->codec != KDN_CODEC_INT4_G64) return KDN_E_INVAL;
     if (c->mem != KDN_MEM_DEVICE && c->mem != KDN_MEM_PINNED_HOST) return KDN_E_INVAL;
-    if (c->codec == KDN_CODEC_INT8_G64 && p->head_dim % 64) return KDN_E_UNSUPPORTED;
+    if (c->codec != KDN_CODEC_RAW_BF16 && p->head_dim % 64) return KDN_E_UNSUPPORTED;
     if (c->bytes != kdn_chunk_bytes(p, c->n_tokens, c->codec)) return KDN_E_SHAPE;
     if (c->n_tokens > 0) {
         if (!c->data) return KDN_E_INVAL;
@@ -208,7 +208,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     if (n <= 0) return KDN_OK;
     bool any_int8 = false, any_rot = false;
     for (int i = 0; i < n; ++i) {
-        any_int8 |= hops[i].op.codec == KDN_CODEC_INT8_G64;
+        any_int8 |= hops[i].op.codec != KDN_CODEC_RAW_BF16;
         any_rot |= hops[i].rotate;
     }
     const bool compute = any_int8 || any_rot;
@@ -345,8 +345,9 @@ HostOp make_host_op(const Pool &pool, const int32_t *table, int64_t off, const k
     h.op.rope = -1;
     h.op.l0 = 0;
     h.op.nl = pool.L;
-    if (c.codec == KDN_CODEC_INT8_G64)
-        h.op.scales = (unsigned char *)c.data + (size_t)pool.L * 2u * (size_t)c.n_tokens * (size_t)pool.H * (size_t)pool.D;
+    const size_t elems = (size_t)pool.L * 2u * (size_t)c.n_tokens * (size_t)pool.H * (size_t)pool.D;
+    if (c.codec == KDN_CODEC_INT8_G64) h.op.scales = (unsigned char *)c.data + elems;
+    if (c.codec == KDN_CODEC_INT4_G64) h.op.scales = (unsigned char *)c.data + elems / 2u;
     return h;
 }
 
@@ -395,9 +396,9 @@ kdn_status run_staged(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<
     for (const HostOp &h : hops) {
         const size_t T = (size_t)h.op.T;
         if (T == 0) continue;
-        const bool int8 = h.op.codec == KDN_CODEC_INT8_G64;
-        const size_t codes_per_layer = 2 * T * row * (int8 ? 1 : 2);
-        const size_t scales_per_layer = int8 ? 2 * T * (row / 64) * 4 : 0;
+        const bool coded = h.op.codec != KDN_CODEC_RAW_BF16;
+        const size_t codes_per_layer = h.op.codec == KDN_CODEC_INT4_G64 ? T * row : 2 * T * row * (coded ? 1 : 2);
+        const size_t scales_per_layer = coded ? 2 * T * (row / 64) * 4 : 0;
         const size_t per_layer = ((codes_per_layer + 255) & ~(size_t)255) + ((scales_per_layer + 255) & ~(size_t)255);
         if (per_layer > ctx->slab_bytes) return KDN_E_UNSUPPORTED;
         unsigned char *host = h.op.data;
@@ -459,8 +460,8 @@ HostOp layer_range(const Pool &pool, const HostOp &h, int l0, int nl)
     const size_t plane = 2u * (size_t)h.op.T * (size_t)pool.H * (size_t)pool.D;     // elements of one layer
     sub.op.l0 = l0;
     sub.op.nl = nl;
-    if (h.op.codec == KDN_CODEC_INT8_G64) {
-        sub.op.data = h.op.data + (size_t)l0 * plane;
+    if (h.op.codec != KDN_CODEC_RAW_BF16) {
+        sub.op.data = h.op.data + (size_t)l0 * (h.op.codec == KDN_CODEC_INT4_G64 ? plane / 2u : plane);
         sub.op.scales = h.op.scales + (size_t)l0 * (plane / 64u) * 4u;
     } else {
         sub.op.data = h.op.data + (size_t)l0 * plane * 2u;
@@ -502,6 +503,7 @@ size_t kdn_chunk_bytes(const kdn_pool_desc *pool, int32_t n_tokens, int32_t code
     const size_t elems = (size_t)pool->n_layers * 2u * (size_t)n_tokens * (size_t)pool->n_kv_heads * (size_t)pool->head_dim;
     if (codec == KDN_CODEC_RAW_BF16) return elems * 2u;
     if (codec == KDN_CODEC_INT8_G64) return pool->head_dim % 64 ? 0 : elems + elems / 64u * 4u;
+    if (codec == KDN_CODEC_INT4_G64) return pool->head_dim % 64 ? 0 : elems / 2u + elems / 64u * 4u;
     return 0;
 }
 
@@ -870,7 +872,7 @@ extern "C" kdn_status kdn_compose_static(int device, const kdn_pool_desc *pool, 
     for (int r = 0; r < n_reqs; ++r)
         for (int j = 0; j < reqs[r].n_parts; ++j) {
             if (reqs[r].parts[j].n_tokens == 0) continue;
-            any_int8 |= reqs[r].parts[j].codec == KDN_CODEC_INT8_G64;
+            any_int8 |= reqs[r].parts[j].codec != KDN_CODEC_RAW_BF16;
             any_rot |= reqs[r].part_dst_pos[j] != reqs[r].parts[j].base_pos;
         }
     const bool compute = any_int8 || any_rot;

@@ -35,7 +35,7 @@ constexpr int kMaxStages = 32;
 constexpr int kMaxStoreLag = 4;           // most bulk-store groups allowed to be still reading shared memory
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
-enum : uint32_t { TF_INT8 = 1u, TF_ROTATE = 2u, TF_SCALES_PLAIN = 4u };
+enum : uint32_t { TF_CODED = 1u, TF_ROTATE = 2u, TF_SCALES_PLAIN = 4u, TF_INT4 = 8u };   // TF_CODED: int8 or int4
 enum : int { OP_STORE = 0, OP_RETRIEVE = 1, OP_COMPOSE = 2 };
 
 // Status values mirrored from kdn.h (kept numeric here so device code has no host header).
@@ -47,7 +47,7 @@ struct __align__(16) DevOp {
     unsigned char *data;      // layers [l0, l0 + nl) of the chunk: raw bf16, or int8 codes
     long long off;            // request position of chunk token 0
     int T;                    // tokens
-    int codec;                // 0 raw bf16, 1 int8 group-64
+    int codec;                // 0 raw bf16, 1 int8 group-64, 2 int4 group-64
     int j0;                   // first logical block touched: off / block_size
     int nblk;                 // logical blocks touched
     unsigned tile_begin;      // index of this op's first tile in the launch
@@ -271,9 +271,12 @@ __device__ __forceinline__ uint32_t pack_codes4(uint32_t r0, uint32_t r1, uint32
 // Two lanes share a group, 32 elements each, read as four 128-bit shared loads in a lane-rotated
 // order (bank-conflict free); the absmax is reduced with one shuffle; the two IEEE divides are
 // issued once per 32 elements.  ct is the thread's index inside its compute group.
+// kInt4: codes in [-7, 7], two per byte (element 2k in the low nibble), 16 bytes per lane instead of 32.
+template <bool kInt4>
 __device__ __forceinline__ void quantise_tile(const unsigned char *A, unsigned char *B, float *S, float *g_scales,
                                               unsigned n, int ct)
 {
+    const float qmax = kInt4 ? 7.0f : 127.0f;
     const unsigned nhalf = n >> 5;                         // 32-element half groups
     const unsigned lane = (unsigned)ct & 31u;
     const unsigned rot = (lane >> 1) & 3u;
@@ -295,15 +298,16 @@ __device__ __forceinline__ void quantise_tile(const unsigned char *A, unsigned c
         m0 = maxabs_bf16x2(m0, m1);
         float a = fmaxf(__uint_as_float((m0 << 16) & 0x7fffffffu), __uint_as_float(m0 & 0x7fff0000u));
         a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
-        float scale = __fdiv_rn(a, 127.0f);
+        float scale = __fdiv_rn(a, qmax);
         const bool ok = scale >= 1.17549435e-38f;         // smallest normal fp32; false for NaN too
-        const float inv = ok ? __fdiv_rn(127.0f, a) : 0.0f;
+        const float inv = ok ? __fdiv_rn(qmax, a) : 0.0f;
         scale = ok ? scale : 0.0f;
         if (act) {
             const f32x2 inv2 = pack2(inv, inv);
             const f32x2 magic2 = pack2(12582912.0f, 12582912.0f);
             const f32x2 one2 = pack2(1.0f, 1.0f);
-            unsigned char *dst = B + (size_t)h * 32u;
+            unsigned char *dst = B + (size_t)h * (kInt4 ? 16u : 32u);
+            uint32_t nib[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 // per pair: one rounded product, one rounded sum with 1.5 * 2^23 (see above)
@@ -315,7 +319,20 @@ __device__ __forceinline__ void quantise_tile(const unsigned char *A, unsigned c
                 uint2 q;
                 q.x = pack_codes4(r[0], r[1], r[2], r[3]);
                 q.y = pack_codes4(r[4], r[5], r[6], r[7]);
-                sts64(dst + (((unsigned)j + rot) & 3u) * 8u, q);
+                if (kInt4) {
+                    // low nibbles of the eight code bytes -> four bytes: byte k = code 2k | code 2k+1 << 4
+                    const uint32_t t0 = q.x & 0x0f0f0f0fu, t1 = q.y & 0x0f0f0f0fu;
+                    nib[j] = __byte_perm(t0 | (t0 >> 4), t1 | (t1 >> 4), 0x6420);
+                } else {
+                    sts64(dst + (((unsigned)j + rot) & 3u) * 8u, q);
+                }
+            }
+            if (kInt4) {
+                // nib[j] belongs at word (j + rot) & 3: rotate the registers, then one 128-bit store
+                uint32_t o0 = nib[0], o1 = nib[1], o2 = nib[2], o3 = nib[3];
+                if (rot & 1u) { const uint32_t t = o3; o3 = o2; o2 = o1; o1 = o0; o0 = t; }
+                if (rot & 2u) { uint32_t t = o0; o0 = o2; o2 = t; t = o1; o1 = o3; o3 = t; }
+                sts128(dst, make_uint4(o0, o1, o2, o3));
             }
             if ((lane & 1u) == 0u) {
                 if (g_scales) g_scales[h >> 1] = scale; else S[h >> 1] = scale;
@@ -360,6 +377,39 @@ __device__ __forceinline__ void dequantise_tile(const unsigned char *B, const fl
     }
 }
 
+// Eight int4 codes of one word as four packed fp32 pairs (elements 0-1, 2-3, 4-5, 6-7), exact: the nibbles are
+// biased by 8, split into even and odd bytes, and each byte goes through the same 2^23 mantissa trick.
+__device__ __forceinline__ void nibbles_to_f32x2(uint32_t w, f32x2 minus_bias4, f32x2 *out)
+{
+    const uint32_t b = w ^ 0x88888888u;
+    const uint32_t e = b & 0x0f0f0f0fu, o = (b >> 4) & 0x0f0f0f0fu;
+    out[0] = add2(pack2_bits(__byte_perm(e, 0x4B000000u, 0x7650), __byte_perm(o, 0x4B000000u, 0x7650)), minus_bias4);
+    out[1] = add2(pack2_bits(__byte_perm(e, 0x4B000000u, 0x7651), __byte_perm(o, 0x4B000000u, 0x7651)), minus_bias4);
+    out[2] = add2(pack2_bits(__byte_perm(e, 0x4B000000u, 0x7652), __byte_perm(o, 0x4B000000u, 0x7652)), minus_bias4);
+    out[3] = add2(pack2_bits(__byte_perm(e, 0x4B000000u, 0x7653), __byte_perm(o, 0x4B000000u, 0x7653)), minus_bias4);
+}
+
+// Decode n int4 codes (n/2 bytes at B) with scales S into bf16 at A.
+__device__ __forceinline__ void dequantise4_tile(const unsigned char *B, const float *S, unsigned char *A,
+                                                 unsigned n, int ct)
+{
+    const unsigned nvec = n >> 4;                          // 16 codes = 8 bytes per step
+    const f32x2 minus_bias4 = pack2(-8388616.0f, -8388616.0f);   // -(2^23 + 8)
+    for (unsigned v = (unsigned)ct; v < nvec; v += kGroupThreads) {
+        const uint2 c = lds64(B + (size_t)v * 8u);
+        const float sc = S[v >> 2];
+        const f32x2 sc2 = pack2(sc, sc);
+        f32x2 f[8];
+        nibbles_to_f32x2(c.x, minus_bias4, f);
+        nibbles_to_f32x2(c.y, minus_bias4, f + 4);
+        uint32_t o[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) o[k] = pack_bf16x2(mul2(f[k], sc2));
+        sts128(A + (size_t)v * 32u, make_uint4(o[0], o[1], o[2], o[3]));
+        sts128(A + (size_t)v * 32u + 16u, make_uint4(o[4], o[5], o[6], o[7]));
+    }
+}
+
 // Rotation coefficients a thread keeps in registers: (cos, sin, -sin) for 8 consecutive frequencies,
 // as four packed pairs each.
 struct RotCoef {
@@ -398,8 +448,8 @@ __device__ __forceinline__ void rotate8(const f32x2 *u, const f32x2 *w, const Ro
 
 // Rotate a tile of whole head rows (n a multiple of D, D a multiple of 16).  One work item is 8
 // frequencies of one head row: elements [col, col+8) and [D/2 + col, D/2 + col + 8).
-// kInt8 = false: bf16 at A, in place.  kInt8 = true: codes at B and scales at S -> bf16 at A.
-template <bool kInt8>
+// kCodec = 0: bf16 at A, in place.  kCodec = 1 / 2: int8 / int4 codes at B and scales at S -> bf16 at A.
+template <int kCodec>
 __device__ __forceinline__ void rotate_tile(unsigned char *A, const unsigned char *B, const float *S, unsigned n,
                                             unsigned D, const float2 *table, int rope, RotCoef &rc, int ct)
 {
@@ -415,7 +465,17 @@ __device__ __forceinline__ void rotate_tile(unsigned char *A, const unsigned cha
         load_coef(rc, table, rope, col, half);
         const unsigned e_lo = r * D + col, e_hi = e_lo + half;
         f32x2 u[4], w[4];
-        if (kInt8) {
+        if (kCodec == 2) {
+            const uint32_t cl = *reinterpret_cast<const uint32_t *>(B + (e_lo >> 1));
+            const uint32_t ch = *reinterpret_cast<const uint32_t *>(B + (e_hi >> 1));
+            const float sl = S[e_lo >> 6], sh = S[e_hi >> 6];
+            const f32x2 sl2 = pack2(sl, sl), sh2 = pack2(sh, sh);
+            const f32x2 minus_bias4 = pack2(-8388616.0f, -8388616.0f);
+            nibbles_to_f32x2(cl, minus_bias4, u);
+            nibbles_to_f32x2(ch, minus_bias4, w);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) { u[k] = mul2(u[k], sl2); w[k] = mul2(w[k], sh2); }
+        } else if (kCodec == 1) {
             const uint2 cl = lds64(B + e_lo), ch = lds64(B + e_hi);
             const float sl = S[e_lo >> 6], sh = S[e_hi >> 6];
             const f32x2 sl2 = pack2(sl, sl), sh2 = pack2(sh, sh);
@@ -479,8 +539,9 @@ __device__ __forceinline__ void decode_tile(const Launch &P, unsigned g, TileDes
     if (op.codec == 0) {
         d.g_chunk = (unsigned long long)(op.data + ce * 2ull);
     } else {
-        d.flags |= TF_INT8;
-        d.g_chunk = (unsigned long long)(op.data + ce);
+        d.flags |= TF_CODED;
+        if (op.codec == 2) { d.flags |= TF_INT4; d.g_chunk = (unsigned long long)(op.data + (ce >> 1)); }
+        else d.g_chunk = (unsigned long long)(op.data + ce);
         d.g_scales = (unsigned long long)(op.scales + (ce >> 6) * 4ull);
         if ((d.g_scales & 15ull) || ((n >> 6) & 3u)) d.flags |= TF_SCALES_PLAIN;
     }
@@ -569,16 +630,19 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                         } else if (OP == OP_STORE) {
                             mbar_arrive_expect_tx(bar, cur.n * 2u);
                             bulk_g2s(smem_u32(A), (const void *)cur.g_pool, cur.n * 2u, bar);
-                        } else if (!(cur.flags & TF_INT8)) {
+                        } else if (!(cur.flags & TF_CODED)) {
                             mbar_arrive_expect_tx(bar, cur.n * 2u);
                             bulk_g2s(smem_u32(A), (const void *)cur.g_chunk, cur.n * 2u, bar);
-                        } else if (cur.flags & TF_SCALES_PLAIN) {
-                            mbar_arrive_expect_tx(bar, cur.n);
-                            bulk_g2s(smem_u32(A + P.off_b), (const void *)cur.g_chunk, cur.n, bar);
                         } else {
-                            mbar_arrive_expect_tx(bar, cur.n + (cur.n >> 4));
-                            bulk_g2s(smem_u32(A + P.off_b), (const void *)cur.g_chunk, cur.n, bar);
-                            bulk_g2s(smem_u32(A + P.off_s), (const void *)cur.g_scales, cur.n >> 4, bar);
+                            const uint32_t code_bytes = (cur.flags & TF_INT4) ? cur.n >> 1 : cur.n;
+                            if (cur.flags & TF_SCALES_PLAIN) {
+                                mbar_arrive_expect_tx(bar, code_bytes);
+                                bulk_g2s(smem_u32(A + P.off_b), (const void *)cur.g_chunk, code_bytes, bar);
+                            } else {
+                                mbar_arrive_expect_tx(bar, code_bytes + (cur.n >> 4));
+                                bulk_g2s(smem_u32(A + P.off_b), (const void *)cur.g_chunk, code_bytes, bar);
+                                bulk_g2s(smem_u32(A + P.off_s), (const void *)cur.g_scales, cur.n >> 4, bar);
+                            }
                         }
                     }
                 }
@@ -609,12 +673,12 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                 const TileDesc d = sm.desc[st];
                 unsigned char *A = sm.stage0 + (size_t)st * P.stage_bytes;
                 if (d.n != 0u) {
-                    const bool computed = kCompute && (OP == OP_STORE ? (d.flags & TF_INT8) != 0u
-                                                                       : (d.flags & (TF_INT8 | TF_ROTATE)) != 0u);
+                    const bool computed = kCompute && (OP == OP_STORE ? (d.flags & TF_CODED) != 0u
+                                                                       : (d.flags & (TF_CODED | TF_ROTATE)) != 0u);
                     if (computed && !mbar_wait(sm.ready + 8u * st, ph, sm.abort_flag)) break;
                     if (OP == OP_STORE) {
-                        if (d.flags & TF_INT8) {
-                            bulk_s2g((void *)d.g_chunk, smem_u32(A + P.off_b), d.n);
+                        if (d.flags & TF_CODED) {
+                            bulk_s2g((void *)d.g_chunk, smem_u32(A + P.off_b), (d.flags & TF_INT4) ? d.n >> 1 : d.n);
                             if (!(d.flags & TF_SCALES_PLAIN))
                                 bulk_s2g((void *)d.g_scales, smem_u32(A + P.off_s), d.n >> 4);
                         } else {
@@ -660,24 +724,29 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
             bool computed = false;
             if (n != 0u) {
                 if (OP == OP_STORE) {
-                    if (flags & TF_INT8) {
+                    if (flags & TF_CODED) {
                         float *gs = (flags & TF_SCALES_PLAIN) ? reinterpret_cast<float *>(sm.desc[st].g_scales) : nullptr;
-                        quantise_tile(A, B, Sc, gs, n, ct);
+                        if (flags & TF_INT4) quantise_tile<true>(A, B, Sc, gs, n, ct);
+                        else quantise_tile<false>(A, B, Sc, gs, n, ct);
                         computed = true;
                     }
-                } else if (flags & TF_INT8) {
+                } else if (flags & TF_CODED) {
                     if (flags & TF_SCALES_PLAIN) {
                         const float *gs = reinterpret_cast<const float *>(sm.desc[st].g_scales);
                         for (unsigned i = (unsigned)ct; i < (n >> 6); i += kGroupThreads) Sc[i] = __ldg(gs + i);
                         group_bar_sync(group);
                     }
-                    if (OP == OP_COMPOSE && (flags & TF_ROTATE))
-                        rotate_tile<true>(A, B, Sc, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct);
-                    else
+                    if (OP == OP_COMPOSE && (flags & TF_ROTATE)) {
+                        if (flags & TF_INT4) rotate_tile<2>(A, B, Sc, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct);
+                        else rotate_tile<1>(A, B, Sc, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct);
+                    } else if (flags & TF_INT4) {
+                        dequantise4_tile(B, Sc, A, n, ct);
+                    } else {
                         dequantise_tile(B, Sc, A, n, ct);
+                    }
                     computed = true;
                 } else if (OP == OP_COMPOSE && (flags & TF_ROTATE)) {
-                    rotate_tile<false>(A, nullptr, nullptr, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct);
+                    rotate_tile<0>(A, nullptr, nullptr, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct);
                     computed = true;
                 }
             }

@@ -13,7 +13,7 @@ from paper_2409_13761_b200 import synth
 from harness import Device, to_np, check_rotated_keys
 
 pytestmark = pytest.mark.gpu
-RAW, INT8 = oracle.RAW_BF16, oracle.INT8_G64
+RAW, INT8, INT4 = oracle.RAW_BF16, oracle.INT8_G64, oracle.INT4_G64
 
 
 def need_gib(gib):
@@ -27,8 +27,9 @@ def sub_chunk(chunk: np.ndarray, L: int, T: int, H: int, D: int, codec: int, lay
     n = L * 2 * T * H * D
     if codec == RAW:
         return np.ascontiguousarray(chunk.view(np.uint16).reshape(L, -1)[layers]).view(np.uint8).reshape(-1)
-    codes = np.ascontiguousarray(chunk[:n].reshape(L, -1)[layers]).reshape(-1)
-    scales = np.ascontiguousarray(chunk[n:].reshape(L, -1)[layers]).reshape(-1)
+    nc = n // 2 if codec == INT4 else n
+    codes = np.ascontiguousarray(chunk[:nc].reshape(L, -1)[layers]).reshape(-1)
+    scales = np.ascontiguousarray(chunk[nc:].reshape(L, -1)[layers]).reshape(-1)
     return np.concatenate([codes, scales])
 
 
@@ -52,7 +53,7 @@ def test_8b_store_then_retrieve_64_chunks_of_512_tokens():
         d_src, d_dst = dev.table(src.reshape(-1)), dev.table(dst.reshape(-1))
         sample = [0, 29, 63]
         layers = list(range(shape.n_layers))
-        for codec in (RAW, INT8):
+        for codec in (RAW, INT8, INT4):
             cb = dev.K.kdn_chunk_bytes(dev.desc, T, codec)
             big = torch.empty(n_req * cb, dtype=torch.uint8, device=dev.dev)
             K = dev.K
@@ -103,7 +104,7 @@ def test_8b_rag_compose_10_chunks_of_1024_tokens_with_suffix():
         d_src, d_req = dev.table(src.reshape(-1)), dev.table(req)
         layers = [0, 13, 31]
         L, H, D = shape.n_layers, shape.n_kv_heads, shape.head_dim
-        for codec in (RAW, INT8):
+        for codec in (RAW, INT8, INT4):
             pb = K.kdn_chunk_bytes(dev.desc, T, codec)
             parts = torch.empty(n_parts * pb, dtype=torch.uint8, device=dev.dev)
             dev.store([K.XferOp(d_src.data_ptr() + j * nb * 4, nb, 0, K.Chunk(parts.data_ptr() + j * pb, pb, T, codec)) for j in range(n_parts)])

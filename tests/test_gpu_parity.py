@@ -9,7 +9,7 @@ from harness import Device, to_np, bits_to_f64, check_rotated_keys
 
 pytestmark = pytest.mark.gpu
 
-RAW, INT8 = oracle.RAW_BF16, oracle.INT8_G64
+RAW, INT8, INT4 = oracle.RAW_BF16, oracle.INT8_G64, oracle.INT4_G64
 
 
 def gather_positions(pool_np, table, pos):
@@ -30,7 +30,7 @@ def test_toy_config_store_retrieve_compose():
         perm = rng.permutation(shape.n_blocks).astype(np.int32)
         tA, tR, tB, tC = perm[0:16], perm[16:32], perm[32:48], np.concatenate([perm[16:32], perm[48:64]])
         host = dev.pool_np()
-        for codec in (RAW, INT8):
+        for codec in (RAW, INT8, INT4):
             ref = host.copy()
             # store A and B in one batched call
             bufA, bufB = dev.chunk_buf(256, codec), dev.chunk_buf(256, codec)
@@ -76,12 +76,12 @@ def test_toy_config_store_retrieve_compose():
 # ------------------------------------------------------------------------------------ edge cases --
 
 EDGE_SHAPES = [
-    synth.TOY.with_(n_blocks=48, block_size=16),
+    synth.TOY.with_(n_blocks=72, block_size=16),
     synth.TOY.with_(n_blocks=96, block_size=3),
     synth.TOY.with_(n_blocks=200, block_size=1),
-    synth.TOY.with_(n_layers=3, n_kv_heads=8, head_dim=128, block_size=32, n_blocks=24),
-    synth.TOY.with_(n_layers=1, n_kv_heads=1, head_dim=256, block_size=16, n_blocks=24),
-    synth.TOY.with_(n_layers=2, n_kv_heads=3, head_dim=192, block_size=8, n_blocks=32),
+    synth.TOY.with_(n_layers=3, n_kv_heads=8, head_dim=128, block_size=32, n_blocks=72),
+    synth.TOY.with_(n_layers=1, n_kv_heads=1, head_dim=256, block_size=16, n_blocks=72),
+    synth.TOY.with_(n_layers=2, n_kv_heads=3, head_dim=192, block_size=8, n_blocks=72),
 ]
 
 
@@ -97,7 +97,8 @@ def test_unaligned_ragged_batched_mixed_codecs(shape):
         cases = []                                       # (src table, off, T, codec)
         span = 6 * bs
         for off, T, codec in [(0, span, RAW), (1 % span, max(1, span - 2), INT8), (bs // 2, 1, INT8), (span - 1, 1, RAW),
-                              (2 % span, max(1, span // 2), RAW), (0, 0, INT8), (bs - 1 if bs > 1 else 0, bs + 1, INT8)]:
+                              (2 % span, max(1, span // 2), RAW), (0, 0, INT8), (bs - 1 if bs > 1 else 0, bs + 1, INT8),
+                              (3 % span, max(1, span - 5), INT4), (bs // 2, 1, INT4)]:
             tab = np.array([free[i] for i in rng.integers(0, len(free), 6)], dtype=np.int32)   # repeats allowed as a source
             cases.append((tab, off, T, codec))
         bufs, ops = [], []
@@ -132,7 +133,8 @@ def test_unaligned_ragged_batched_mixed_codecs(shape):
         dev.close()
 
 
-FUSION_WITNESS_ABSMAX = [21.25, 38.5, 46.0, 84.0, 23.0, 25.75]
+FUSION_WITNESS_ABSMAX = [21.25, 38.5, 46.0, 84.0, 23.0, 25.75,          # for 127/a (int8) ...
+                         16.125, 17.25, 19.0, 20.0]                     # ... and for 7/a (int4)
 
 
 def special_pool(shape):
@@ -163,7 +165,8 @@ def special_pool(shape):
     return pool
 
 
-def test_codec_special_groups_bit_exact():
+@pytest.mark.parametrize("INT8", [INT8, INT4], ids=["int8", "int4"])
+def test_codec_special_groups_bit_exact(INT8):
     shape = synth.TOY.with_(n_blocks=32, block_size=8)
     pool = special_pool(shape)
     dev = Device(shape, pool_np=pool)
@@ -204,7 +207,8 @@ def test_raw_copy_preserves_every_bit_pattern():
         dev.close()
 
 
-@pytest.mark.parametrize("D,codec", [(64, RAW), (64, INT8), (128, RAW), (128, INT8), (256, INT8), (192, INT8), (192, RAW), (80, RAW)])
+@pytest.mark.parametrize("D,codec", [(64, RAW), (64, INT8), (128, RAW), (128, INT8), (256, INT8), (192, INT8), (192, RAW), (80, RAW),
+                                     (64, INT4), (128, INT4), (192, INT4)])
 def test_compose_unaligned_parts_negative_and_large_deltas(D, codec):
     H = 2 if D != 80 else 1
     shape = synth.TOY.with_(n_layers=2, n_kv_heads=H, head_dim=D, block_size=8, n_blocks=64, rope_theta=500000.0)
@@ -250,7 +254,7 @@ def test_compose_unaligned_parts_negative_and_large_deltas(D, codec):
         dev.close()
 
 
-@pytest.mark.parametrize("codec", [RAW, INT8])
+@pytest.mark.parametrize("codec", [RAW, INT8, INT4])
 def test_compose_with_zero_delta_equals_retrieve(codec):
     shape = synth.TOY.with_(n_blocks=40, block_size=16)
     dev = Device(shape, seed=3)
@@ -327,7 +331,7 @@ def test_argument_errors_launch_nothing():
         dev.close()
 
 
-@pytest.mark.parametrize("codec", [RAW, INT8])
+@pytest.mark.parametrize("codec", [RAW, INT8, INT4])
 def test_pinned_host_chunks_through_small_staging_slabs(codec):
     """Chunks in page-locked host memory: store copies out, retrieve and compose copy in, layer range by layer
     range through staging slabs far smaller than the chunk."""
@@ -379,11 +383,11 @@ def test_tuning_shapes_give_identical_results():
         host = dev.pool_np()
         tab = np.random.default_rng(2).permutation(64)[:20].astype(np.int32)
         T, off = 300, 7
-        want = {c: oracle.store(host, tab, off, T, c) for c in (RAW, INT8)}
+        want = {c: oracle.store(host, tab, off, T, c) for c in (RAW, INT8, INT4)}
         for tile, stages, ctas, groups, lag in [(0, 0, 0, 0, 0), (2048, 4, 1, 1, 1), (4096, 12, 3, 3, 2), (32768, 4, 1, 4, 2),
                                                 (16384, 5, 2, 2, 3), (1024, 16, 4, 6, 4), (8192, 3, 2, 3, 1), (8192, 7, 1, 6, 1)]:
             K.kdn_set_tuning(dev.ctx, tile, stages, ctas, groups, lag)
-            for c in (RAW, INT8):
+            for c in (RAW, INT8, INT4):
                 buf = dev.chunk_buf(T, c)
                 dev.store([dev.op(dev.table(tab), off, buf, T, c)])
                 assert dev.sync() == 0
@@ -405,7 +409,7 @@ def test_more_ops_than_one_launch_carries():
         n = 7000
         Ts = rng.integers(0, 4, n)                              # 0..3 tokens, some empty
         offs = rng.integers(0, 4, n)
-        codecs = rng.integers(0, 2, n)
+        codecs = rng.integers(0, 3, n)
         tabs = rng.integers(0, 512, (n, 2)).astype(np.int32)     # two blocks each, repeats allowed as a source
         d_tabs = dev.table(tabs.reshape(-1))
         sizes = [K.kdn_chunk_bytes(dev.desc, int(t), int(c)) for t, c in zip(Ts, codecs)]
@@ -426,7 +430,7 @@ def test_more_ops_than_one_launch_carries():
         dev.close()
 
 
-@pytest.mark.parametrize("codec", [RAW, INT8])
+@pytest.mark.parametrize("codec", [RAW, INT8, INT4])
 def test_layerwise_retrieve_equals_retrieve_and_events_order_layers(codec):
     """Layer-wise delivery: same bits as a plain retrieve; after waiting for layer l's event, layers 0..l are complete
     (checked while later layers may still be in flight); device and pinned-host chunks mixed in one call."""

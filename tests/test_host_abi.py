@@ -31,7 +31,7 @@ def test_chunk_bytes_matches_oracle():
     for (L, H, D) in [(2, 2, 64), (32, 8, 128), (80, 8, 128), (1, 3, 8), (4, 1, 192), (2, 2, 96)]:
         d = K.pool_desc(L, H, D, 16, 64)
         for T in (0, 1, 17, 512, 2048):
-            for codec in (0, 1):
+            for codec in (0, 1, 2):
                 assert K.kdn_chunk_bytes(d, T, codec) == oracle.chunk_bytes(L, H, D, T, codec), (L, H, D, T, codec)
     d = K.pool_desc(2, 2, 64, 16, 64)
     assert K.kdn_chunk_bytes(d, -1, 0) == 0

@@ -157,3 +157,15 @@ def test_compose_int4_rotates_the_unrounded_stored_value():
     ref = before.copy()
     oracle.retrieve(ref, table, 5, T, oracle.INT4_G64, chunk)
     assert np.array_equal(pool[:, 1], ref[:, 1])                                  # values: a plain retrieve
+
+
+def test_double_rounding_witnesses_int4():
+    """x = a/2 with fl(7/a) < 7/a: the exact product is just below 3.5, the fp32 product IS 3.5 -> tie -> 4."""
+    from fractions import Fraction
+    for a in [16.125, 17.25, 19.0, 20.0, 25.75]:
+        inv = np.float32(7.0) / np.float32(a)
+        x = np.float32(a / 2)
+        assert Fraction(float(x)) * Fraction(float(inv)) < Fraction(7, 2) and np.float32(x * inv) == np.float32(3.5)
+        g = np.zeros(64, dtype=np.float32); g[0] = a; g[1] = x; g[2] = -x
+        q = unpack_nibbles(oracle.quant4_group(bf16_bits(g))[0])
+        assert (q[0], q[1], q[2]) == (7, 4, -4)
