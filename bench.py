@@ -38,13 +38,13 @@ WORKLOAD = ("llama3-8b KV (L32 H8 D128 bf16, block_size 16, 16384-block pool): s
             "compose 10x1024 tokens (+256-token suffix), raw bf16 and int8-g64, fully fragmented tables")
 N_CHUNKS, CHUNK_TOKENS = 64, 512
 N_PARTS, PART_TOKENS, SUFFIX_TOKENS = 10, 1024, 256
-RAW, INT8 = 0, 1
+RAW, INT8, INT4 = 0, 1, 2
 FALLBACK_HBM_GBS = 6650.0
 
 
 def bytes_per_elem(codec: int) -> float:
     """Algorithmic bytes per KV element moved by one op: bf16 on the pool side + the chunk side."""
-    return 4.0 if codec == RAW else 2.0 + 1.0 + 4.0 / 64.0
+    return {RAW: 4.0, INT8: 2.0 + 1.0 + 4.0 / 64.0, INT4: 2.0 + 0.5 + 4.0 / 64.0}[codec]
 
 
 # ------------------------------------------------------------------------------------ CPU oracle leg --
@@ -271,11 +271,11 @@ def run_gpu(args) -> None:
     d_req = table(sum(req_blocks), synth.SEED_TABLES + 3)         # all composed requests, back to back
     i32 = 4
 
-    def make_sets(pinned_lib, pinned_retr=()):
+    def make_sets(pinned_lib, pinned_retr=(), codecs=(RAW, INT8)):
         """Chunk buffers and the op lists of one step, per codec.  pinned_lib: the whole library lives in page-locked
         host memory; pinned_retr: only these retrievals read a host copy of their chunk."""
         sets = {}
-        for codec in (RAW, INT8):
+        for codec in codecs:
             cb, pb = K.kdn_chunk_bytes(desc, T, codec), K.kdn_chunk_bytes(desc, PT, codec)
             if pinned_lib:
                 chunks = torch.empty(n_lib * cb, dtype=torch.uint8).pin_memory()
@@ -377,10 +377,32 @@ def run_gpu(args) -> None:
     op_ms = {n: float(np.mean([ev[it][i].elapsed_time(ev[it][i + 1]) for it in range(args.steps)]))
              for i, n in enumerate(names)}
 
+    # ---- the int4 codec (a widening beyond the benchmark step; timed on its own, not part of `value`)
+    int4_ops = {}
+    i4 = make_sets(False, codecs=(INT4,))[INT4]
+    K.kdn_store(ctx, pid, i4["part_store"], s)
+    for name, fn, arg in (("store_int4", K.kdn_store, i4["store"]), ("retrieve_int4", K.kdn_retrieve, i4["retrieve"]),
+                          ("compose_int4", K.kdn_compose, i4["reqs"])):
+        for _ in range(3):
+            fn(ctx, pid, arg, s)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = max(1, min(args.steps, 20))
+        a.record(stream)
+        for _ in range(reps):
+            fn(ctx, pid, arg, s)
+        b.record(stream)
+        torch.cuda.synchronize()
+        ms = a.elapsed_time(b) / reps
+        nbytes = tokens_of[name.split("_")[0]] * E * bytes_per_elem(INT4)
+        int4_ops[name] = {"ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9, "tokens_per_s": tokens_of[name.split("_")[0]] / (ms * 1e-3)}
+    assert K.kdn_status_sync(ctx, s) == K.KDN_OK
+    del i4
+    torch.cuda.empty_cache()
+
     if args.no_e2e:
         if rank == 0:
             print(json.dumps({"note": "profiling run, not a bench record", "ops_ms": op_ms,
-                              "ops_gbs": {n: op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 for n in names}}))
+                              "ops_gbs": {n: op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 for n in names}, "int4": int4_ops}))
         K.kdn_destroy(ctx)
         return
 
@@ -486,7 +508,7 @@ def run_gpu(args) -> None:
             "config": {"workload": W["text"], "l2": "inputs larger than L2 (every op streams >= 1.9 GB once)",
                        "bytes_per_step": step_bytes},
             "tokens_per_s_reloaded": world * reload_tokens / (sum(op_ms[n] for n in names if not n.startswith("store")) * 1e-3),
-            "ops": ops,
+            "ops": ops, "ops_int4_not_in_value": int4_ops,
             "roofline": {"bound": "hbm", "kernel": kernel_of[top], "op": top, "achieved": ops[top]["gbs"], "peak": peak,
                          "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": ops[top]["gbs"] / peak,
                          "frac_of_nominal_8000": ops[top]["gbs"] / 8000.0, "traffic": traffic},

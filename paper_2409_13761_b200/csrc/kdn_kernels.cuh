@@ -269,8 +269,8 @@ __device__ __forceinline__ uint32_t pack_codes4(uint32_t r0, uint32_t r1, uint32
 // Encode n elements (a multiple of 64) of bf16 at A into int8 codes at B and one fp32 scale per 64
 // elements (to shared S, or straight to global when the destination is not 16-byte aligned).
 // Two lanes share a group, 32 elements each, read as four 128-bit shared loads in a lane-rotated
-// order (bank-conflict free); the absmax is reduced with one shuffle; the two IEEE divides are
-// issued once per 32 elements.  ct is the thread's index inside its compute group.
+// order (bank-conflict free); the absmax is reduced with one shuffle; each lane issues one of the
+// group's two IEEE divides.  ct is the thread's index inside its compute group.
 // kInt4: codes in [-7, 7], two per byte (element 2k in the low nibble), 16 bytes per lane instead of 32.
 template <bool kInt4>
 __device__ __forceinline__ void quantise_tile(const unsigned char *A, unsigned char *B, float *S, float *g_scales,
@@ -298,9 +298,14 @@ __device__ __forceinline__ void quantise_tile(const unsigned char *A, unsigned c
         m0 = maxabs_bf16x2(m0, m1);
         float a = fmaxf(__uint_as_float((m0 << 16) & 0x7fffffffu), __uint_as_float(m0 & 0x7fff0000u));
         a = fmaxf(a, __shfl_xor_sync(0xffffffffu, a, 1));
-        float scale = __fdiv_rn(a, qmax);
+        // the two IEEE divides of the group are shared by its two lanes: the even lane forms a / qmax, the odd
+        // lane qmax / a, and one shuffle swaps them
+        const bool odd = (lane & 1u) != 0u;
+        const float mine = odd ? __fdiv_rn(qmax, a) : __fdiv_rn(a, qmax);
+        const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
+        float scale = odd ? other : mine;
         const bool ok = scale >= 1.17549435e-38f;         // smallest normal fp32; false for NaN too
-        const float inv = ok ? __fdiv_rn(qmax, a) : 0.0f;
+        const float inv = ok ? (odd ? mine : other) : 0.0f;
         scale = ok ? scale : 0.0f;
         if (act) {
             const f32x2 inv2 = pack2(inv, inv);
