@@ -74,6 +74,14 @@ def lib():
             L.kdn_oracle_store.argtypes = xfer
             L.kdn_oracle_retrieve.restype = i32
             L.kdn_oracle_retrieve.argtypes = xfer
+            xs = [vp, i32, i32, i32, i32, i64, vp, i32, i64, i32, i32, vp, vp]
+            L.kdn_oracle_store_sparse.restype = i32
+            L.kdn_oracle_store_sparse.argtypes = xs
+            L.kdn_oracle_retrieve_sparse.restype = i32
+            L.kdn_oracle_retrieve_sparse.argtypes = xs
+            L.kdn_oracle_compose_select.restype = i32
+            L.kdn_oracle_compose_select.argtypes = [vp, i32, i32, i32, i32, i64, vp, i32, i32,
+                                                    vp, vp, vp, vp, vp, f64, vp, vp, vp, vp]
             L.kdn_oracle_compose.restype = i32
             L.kdn_oracle_compose.argtypes = [vp, i32, i32, i32, i32, i64, vp, i32, i32,
                                              vp, vp, vp, vp, vp, f64, vp, vp]
@@ -101,36 +109,55 @@ def chunk_bytes(L: int, H: int, D: int, T: int, codec: int) -> int:
     return int(lib().kdn_oracle_chunk_bytes(L, H, D, T, codec))
 
 
-def store(pool: np.ndarray, table: np.ndarray, token_offset: int, n_tokens: int, codec: int) -> np.ndarray:
-    """Gather ``n_tokens`` tokens at request positions ``token_offset + t`` into a new chunk."""
+def _list(x):
+    a = np.ascontiguousarray(x, dtype=np.int32)
+    if a.ndim != 1:
+        raise ValueError("a token list is one-dimensional")
+    return a
+
+
+def store(pool: np.ndarray, table: np.ndarray, token_offset: int, n_tokens: int, codec: int, keep=None) -> np.ndarray:
+    """Gather tokens into a new chunk: positions ``token_offset + t``, or ``token_offset + keep[t]`` for a keep-list
+    (then ``n_tokens == len(keep)``)."""
     L, H, D, bs, nb = _check_pool(pool)
     _check_table(table)
+    if keep is not None:
+        keep = _list(keep)
+        if len(keep) != n_tokens:
+            raise ValueError("n_tokens must equal len(keep)")
     chunk = np.zeros(chunk_bytes(L, H, D, n_tokens, codec), dtype=np.uint8)
-    rc = lib().kdn_oracle_store(_ptr(pool), L, H, D, bs, nb, _ptr(table), len(table),
-                                int(token_offset), int(n_tokens), int(codec), _ptr(chunk))
+    rc = lib().kdn_oracle_store_sparse(_ptr(pool), L, H, D, bs, nb, _ptr(table), len(table),
+                                       int(token_offset), int(n_tokens), int(codec),
+                                       _ptr(keep) if keep is not None else None, _ptr(chunk))
     if rc:
         raise ValueError("oracle store: bad arguments (code %d)" % rc)
     return chunk
 
 
 def retrieve(pool: np.ndarray, table: np.ndarray, token_offset: int, n_tokens: int, codec: int,
-             chunk: np.ndarray) -> None:
-    """Scatter ``chunk`` into ``pool`` in place at request positions ``token_offset + t``."""
+             chunk: np.ndarray, keep=None) -> None:
+    """Scatter ``chunk`` into ``pool`` in place at request positions ``token_offset + t`` (or ``+ keep[t]``)."""
+    if keep is not None:
+        keep = _list(keep)
+        if len(keep) != n_tokens:
+            raise ValueError("n_tokens must equal len(keep)")
     L, H, D, bs, nb = _check_pool(pool)
     _check_table(table)
     if chunk.dtype != np.uint8 or chunk.size != chunk_bytes(L, H, D, n_tokens, codec):
         raise ValueError("chunk has the wrong size for this shape / codec")
     chunk = np.ascontiguousarray(chunk)
-    rc = lib().kdn_oracle_retrieve(_ptr(pool), L, H, D, bs, nb, _ptr(table), len(table),
-                                   int(token_offset), int(n_tokens), int(codec), _ptr(chunk))
+    rc = lib().kdn_oracle_retrieve_sparse(_ptr(pool), L, H, D, bs, nb, _ptr(table), len(table),
+                                          int(token_offset), int(n_tokens), int(codec),
+                                          _ptr(keep) if keep is not None else None, _ptr(chunk))
     if rc:
         raise ValueError("oracle retrieve: bad arguments (code %d)" % rc)
 
 
-def compose(pool: np.ndarray, table: np.ndarray, parts, theta: float, want_ref: bool = False):
+def compose(pool: np.ndarray, table: np.ndarray, parts, theta: float, want_ref: bool = False, select=None):
     """Compose ``parts`` into ``pool`` in place.
 
-    ``parts`` is a list of ``(chunk, n_tokens, codec, base_pos, dst_pos)``.
+    ``parts`` is a list of ``(chunk, n_tokens, codec, base_pos, dst_pos)``.  ``select``: None, or one entry per part,
+    each None (deliver every token) or a strictly increasing list of the chunk tokens to deliver.
     With ``want_ref`` returns ``(kref, kmag)``: fp64 ``[L][n_table*bs][H][D]`` arrays holding the
     unrounded key result (NaN where no part wrote) and ``|u| + |w|`` of each rotated pair.
     """
@@ -150,10 +177,18 @@ def compose(pool: np.ndarray, table: np.ndarray, parts, theta: float, want_ref: 
     if want_ref:
         kref = np.full((L, len(table) * bs, H, D), np.nan, dtype=np.float64)
         kmag = np.zeros((L, len(table) * bs, H, D), dtype=np.float64)
-    rc = lib().kdn_oracle_compose(_ptr(pool), L, H, D, bs, nb, _ptr(table), len(table), n,
-                                  C.cast(ptrs, C.c_void_p), _ptr(Ts), _ptr(codecs), _ptr(base), _ptr(dst),
-                                  float(theta), _ptr(kref) if want_ref else None,
-                                  _ptr(kmag) if want_ref else None)
+    sel_ptr = nsel_ptr = None
+    if select is not None:
+        if len(select) != n:
+            raise ValueError("select needs one entry per part")
+        sels = [_list(x if x is not None else np.arange(p[1])) for x, p in zip(select, parts)]
+        sel_arr = (C.c_void_p * max(n, 1))(*[a.ctypes.data for a in sels])
+        nsel = np.array([len(a) for a in sels], dtype=np.int32)
+        sel_ptr, nsel_ptr = C.cast(sel_arr, C.c_void_p), _ptr(nsel)
+    rc = lib().kdn_oracle_compose_select(_ptr(pool), L, H, D, bs, nb, _ptr(table), len(table), n,
+                                         C.cast(ptrs, C.c_void_p), _ptr(Ts), _ptr(codecs), _ptr(base), _ptr(dst),
+                                         float(theta), sel_ptr, nsel_ptr, _ptr(kref) if want_ref else None,
+                                         _ptr(kmag) if want_ref else None)
     if rc:
         raise ValueError("oracle compose: bad arguments (code %d)" % rc)
     return (kref, kmag) if want_ref else None

@@ -46,6 +46,14 @@
  *                    evaluated in fp64.  Values are copied.  delta == 0 keys
  *                    take the decode path unchanged.
  *
+ *   R7  token lists  (Sec. 3.2 "KV-cache delivery" cites dropping tokens and KV elements by importance; Sec. 3.2
+ *                    "KV-cache blending" cites recomputing a fraction of the tokens after blending.  The scoring
+ *                    is not part of this path; moving only the listed tokens is.)
+ *                    keep-list: a chunk may hold only some tokens of a span: chunk token t is the request position
+ *                    off + keep[t], keep strictly increasing; store gathers those, retrieve writes only those.
+ *                    select-list: compose may deliver only some tokens of a part: for each listed chunk token c
+ *                    (strictly increasing) it writes position dst_pos + c and leaves the other positions alone.
+ *
  * Parity pins (tests/test_oracle_*.py, all CPU): brute force against an
  * independent index-by-index formulation on tiny shapes; contiguous table
  * reduces store to a slice copy; store-then-retrieve identity on raw bf16 for
@@ -245,14 +253,20 @@ static size_t chunk_index(const shape_t *s, int T, int l, int kv, int t, int h, 
     return i;
 }
 
-static int check_args(const shape_t *s, const int32_t *table, int n_table, int64_t off, int T, int codec)
+/* Validate one transfer of n listed tokens: token i sits at position off + (list ? list[i] : i). */
+static int check_args_list(const shape_t *s, const int32_t *table, int n_table, int64_t off, int n, int codec,
+                           const int32_t *list, int list_bound)
 {
     if (s->L <= 0 || s->H <= 0 || s->D <= 0 || s->bs <= 0 || s->nb <= 0) return 1;
-    if (T < 0 || off < 0 || n_table < 0) return 1;
-    if (off + (int64_t)T > (int64_t)n_table * (int64_t)s->bs) return 2;
+    if (n < 0 || off < 0 || n_table < 0) return 1;
     if (codec != KDN_ORACLE_RAW_BF16 && codec != KDN_ORACLE_INT8_G64 && codec != KDN_ORACLE_INT4_G64) return 3;
     if (codec != KDN_ORACLE_RAW_BF16 && s->D % KDN_ORACLE_GROUP) return 3;
-    for (int64_t p = off; p < off + T; ++p) {
+    for (int i = 0; i < n; ++i) {
+        int64_t rel = list ? list[i] : i;
+        if (rel < 0 || (list && i > 0 && list[i] <= list[i - 1])) return 5;       /* strictly increasing */
+        if (list_bound >= 0 && rel >= list_bound) return 5;
+        int64_t p = off + rel;
+        if (p >= (int64_t)n_table * (int64_t)s->bs) return 2;
         int32_t b = table[p / s->bs];
         if (b < 0 || (int64_t)b >= s->nb) return 4;
     }
@@ -264,12 +278,12 @@ static int check_args(const shape_t *s, const int32_t *table, int n_table, int64
 /* Sec. 3.2 call (i): gather T tokens starting at request position `off` out
  * of the paged pool (R1, R3) into one chunk (R2), optionally int8-coded (R4).
  * Returns 0, or a small positive code for bad arguments (nothing written). */
-int kdn_oracle_store(const uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
-                     const int32_t *table, int n_table, int64_t off, int T, int codec,
-                     uint8_t *chunk)
+int kdn_oracle_store_sparse(const uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
+                            const int32_t *table, int n_table, int64_t off, int T, int codec,
+                            const int32_t *keep, uint8_t *chunk)
 {
     shape_t s = { L, H, D, bs, nb };
-    int rc = check_args(&s, table, n_table, off, T, codec);
+    int rc = check_args_list(&s, table, n_table, off, T, codec, keep, -1);
     if (rc) return rc;
     size_t elems = (size_t)L * 2u * (size_t)T * (size_t)H * (size_t)D;
     uint16_t *raw = (uint16_t *)chunk;
@@ -278,7 +292,7 @@ int kdn_oracle_store(const uint16_t *pool, int L, int H, int D, int bs, int64_t 
     for (int l = 0; l < L; ++l)
         for (int kv = 0; kv < 2; ++kv)
             for (int t = 0; t < T; ++t) {
-                int64_t p = off + t;
+                int64_t p = off + (keep ? keep[t] : t);             /* R3, R7 */
                 int64_t block = table[p / bs];
                 int slot = (int)(p % bs);
                 for (int h = 0; h < H; ++h) {
@@ -302,6 +316,14 @@ int kdn_oracle_store(const uint16_t *pool, int L, int H, int D, int bs, int64_t 
                 }
             }
     return 0;
+}
+
+/* Sec. 3.2 call (i) for a whole span: every token, in order. */
+int kdn_oracle_store(const uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
+                     const int32_t *table, int n_table, int64_t off, int T, int codec,
+                     uint8_t *chunk)
+{
+    return kdn_oracle_store_sparse(pool, L, H, D, bs, nb, table, n_table, off, T, codec, NULL, chunk);
 }
 
 /* The stored value of chunk element c before any bf16 rounding: code and scale (raw: the bf16 itself). */
@@ -331,18 +353,18 @@ static uint16_t decoded(const uint8_t *chunk, size_t elems, int codec, size_t c)
 /* Sec. 3.2 call (ii) with Sec. 3.1's "decompresses them in GPU": scatter a
  * chunk back into the pool blocks the table names, decoding int8 (R5).  Only
  * the T addressed token slots are written. */
-int kdn_oracle_retrieve(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
-                        const int32_t *table, int n_table, int64_t off, int T, int codec,
-                        const uint8_t *chunk)
+int kdn_oracle_retrieve_sparse(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
+                               const int32_t *table, int n_table, int64_t off, int T, int codec,
+                               const int32_t *keep, const uint8_t *chunk)
 {
     shape_t s = { L, H, D, bs, nb };
-    int rc = check_args(&s, table, n_table, off, T, codec);
+    int rc = check_args_list(&s, table, n_table, off, T, codec, keep, -1);
     if (rc) return rc;
     size_t elems = (size_t)L * 2u * (size_t)T * (size_t)H * (size_t)D;
     for (int l = 0; l < L; ++l)
         for (int kv = 0; kv < 2; ++kv)
             for (int t = 0; t < T; ++t) {
-                int64_t p = off + t;
+                int64_t p = off + (keep ? keep[t] : t);
                 int64_t block = table[p / bs];
                 int slot = (int)(p % bs);
                 for (int h = 0; h < H; ++h)
@@ -353,6 +375,13 @@ int kdn_oracle_retrieve(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
                     }
             }
     return 0;
+}
+
+int kdn_oracle_retrieve(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
+                        const int32_t *table, int n_table, int64_t off, int T, int codec,
+                        const uint8_t *chunk)
+{
+    return kdn_oracle_retrieve_sparse(pool, L, H, D, bs, nb, table, n_table, off, T, codec, NULL, chunk);
 }
 
 /* -------------------------------------------------------------- compose -- */
@@ -369,17 +398,19 @@ int kdn_oracle_retrieve(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
  * its pair, laid out [l][position][h][d] over the n_table * bs request
  * positions; entries no part covers are left as the caller set them.
  */
-int kdn_oracle_compose(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
-                       const int32_t *table, int n_table, int n_parts,
-                       const uint8_t *const *chunks, const int32_t *part_T, const int32_t *part_codec,
-                       const int64_t *base_pos, const int64_t *dst_pos, double theta,
-                       double *kref, double *kmag)
+int kdn_oracle_compose_select(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
+                              const int32_t *table, int n_table, int n_parts,
+                              const uint8_t *const *chunks, const int32_t *part_T, const int32_t *part_codec,
+                              const int64_t *base_pos, const int64_t *dst_pos, double theta,
+                              const int32_t *const *part_sel, const int32_t *part_nsel,
+                              double *kref, double *kmag)
 {
     shape_t s = { L, H, D, bs, nb };
     if (n_parts < 0) return 1;
     if (D % 2) return 3;
     for (int j = 0; j < n_parts; ++j) {
-        int rc = check_args(&s, table, n_table, dst_pos[j], part_T[j], part_codec[j]);
+        const int32_t *sel = part_sel ? part_sel[j] : NULL;
+        int rc = check_args_list(&s, table, n_table, dst_pos[j], sel ? part_nsel[j] : part_T[j], part_codec[j], sel, part_T[j]);
         if (rc) return rc;
     }
     int64_t P = (int64_t)n_table * bs;
@@ -390,9 +421,12 @@ int kdn_oracle_compose(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
         int64_t delta = dst_pos[j] - base_pos[j];
         size_t elems = (size_t)L * 2u * (size_t)T * (size_t)H * (size_t)D;
         const uint16_t *raw = (const uint16_t *)chunks[j];
+        const int32_t *sel = part_sel ? part_sel[j] : NULL;
+        int n_deliver = sel ? part_nsel[j] : T;
         for (int l = 0; l < L; ++l)
             for (int kv = 0; kv < 2; ++kv)
-                for (int t = 0; t < T; ++t) {
+                for (int i_sel = 0; i_sel < n_deliver; ++i_sel) {
+                    int t = sel ? sel[i_sel] : i_sel;                 /* R7: only the listed chunk tokens */
                     int64_t p = dst_pos[j] + t;
                     int64_t block = table[p / bs];
                     int slot = (int)(p % bs);
@@ -447,4 +481,14 @@ int kdn_oracle_compose(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
                 }
     }
     return 0;
+}
+
+int kdn_oracle_compose(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
+                       const int32_t *table, int n_table, int n_parts,
+                       const uint8_t *const *chunks, const int32_t *part_T, const int32_t *part_codec,
+                       const int64_t *base_pos, const int64_t *dst_pos, double theta,
+                       double *kref, double *kmag)
+{
+    return kdn_oracle_compose_select(pool, L, H, D, bs, nb, table, n_table, n_parts, chunks, part_T, part_codec,
+                                     base_pos, dst_pos, theta, NULL, NULL, kref, kmag);
 }
