@@ -399,10 +399,40 @@ def run_gpu(args) -> None:
     del i4
     torch.cuda.empty_cache()
 
+    # ---- keep-lists: every chunk holds a seeded random half of its span's tokens (timed on its own, not in `value`)
+    sparse_ops = {}
+    rng = np.random.default_rng(synth.SEED_ASSIGN)
+    n_keep = T // 2
+    keep_np = np.stack([np.sort(rng.choice(T, n_keep, replace=False)) for _ in range(n_lib)]).astype(np.int32)
+    d_keep = torch.from_numpy(keep_np).to(dev)
+    for codec, cname in ((RAW, "raw"), (INT8, "int8")):
+        cb = K.kdn_chunk_bytes(desc, n_keep, codec)
+        buf = torch.empty(n_lib * cb, dtype=torch.uint8, device=dev)
+        keeps = [d_keep.data_ptr() + c * n_keep * i32 for c in range(n_lib)]
+        st_ops = [K.XferOp(d_src.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(buf.data_ptr() + c * cb, cb, n_keep, codec)) for c in range(n_lib)]
+        rt_ops = [K.XferOp(d_dst.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(buf.data_ptr() + c * cb, cb, n_keep, codec)) for c in range(n_lib)]
+        for name, fn, arg in (("store_sparse_" + cname, K.kdn_store_sparse, st_ops), ("retrieve_sparse_" + cname, K.kdn_retrieve_sparse, rt_ops)):
+            for _ in range(3):
+                fn(ctx, pid, arg, keeps, s)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            reps = max(1, min(args.steps, 20))
+            a.record(stream)
+            for _ in range(reps):
+                fn(ctx, pid, arg, keeps, s)
+            b.record(stream)
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / reps
+            nbytes = n_lib * n_keep * E * bytes_per_elem(codec)
+            sparse_ops[name] = {"ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9, "tokens_per_s": n_lib * n_keep / (ms * 1e-3),
+                                "kept": "%d of %d tokens per chunk, seeded random" % (n_keep, T)}
+        assert K.kdn_status_sync(ctx, s) == K.KDN_OK
+        del buf
+    torch.cuda.empty_cache()
+
     if args.no_e2e:
         if rank == 0:
             print(json.dumps({"note": "profiling run, not a bench record", "ops_ms": op_ms,
-                              "ops_gbs": {n: op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 for n in names}, "int4": int4_ops}))
+                              "ops_gbs": {n: op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 for n in names}, "int4": int4_ops, "sparse": sparse_ops}))
         K.kdn_destroy(ctx)
         return
 
@@ -508,7 +538,7 @@ def run_gpu(args) -> None:
             "config": {"workload": W["text"], "l2": "inputs larger than L2 (every op streams >= 1.9 GB once)",
                        "bytes_per_step": step_bytes},
             "tokens_per_s_reloaded": world * reload_tokens / (sum(op_ms[n] for n in names if not n.startswith("store")) * 1e-3),
-            "ops": ops, "ops_int4_not_in_value": int4_ops,
+            "ops": ops, "ops_int4_not_in_value": int4_ops, "ops_keep_list_not_in_value": sparse_ops,
             "roofline": {"bound": "hbm", "kernel": kernel_of[top], "op": top, "achieved": ops[top]["gbs"], "peak": peak,
                          "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": ops[top]["gbs"] / peak,
                          "frac_of_nominal_8000": ops[top]["gbs"] / 8000.0, "traffic": traffic},

@@ -135,11 +135,34 @@ typedef struct {
     int32_t         reserved;        /* 0 */
 } kdn_compose_req;
 
+/* Token lists.  Sec. 3.2 "KV-cache delivery" cites dropping tokens or KV elements by importance (LLMLingua, H2O)
+ * and "KV-cache blending" cites recomputing a fraction of the tokens after composing (CacheBlend); deciding
+ * which tokens is the engine's business, moving only those is this library's.
+ *
+ * Keep-list: the chunk of a kdn_sparse_op holds exactly op.chunk.n_tokens tokens, and chunk token i is request
+ * position op.token_offset + keep[i].  keep: DEVICE int32 [op.chunk.n_tokens], non-negative, strictly
+ * increasing.  The chunk's layout is the ordinary one for n_tokens tokens, so a sparse chunk can later be
+ * retrieved or composed densely, and a dense chunk retrieved sparsely is not supported (store it sparsely). */
+typedef struct {
+    kdn_xfer_op    op;
+    const int32_t *keep;
+} kdn_sparse_op;
+
+/* Select-lists for kdn_compose_select: part j of the request delivers only its chunk tokens
+ * part_select[j][0 .. part_n_select[j]) (DEVICE int32 lists, strictly increasing, each < the part's n_tokens);
+ * token c still lands at part_dst_pos[j] + c and the positions of unlisted tokens keep their contents, e.g.
+ * for the engine to recompute.  part_select: HOST array [n_parts] (NULL, or NULL entries, = deliver every
+ * token); part_n_select: HOST array [n_parts]. */
+typedef struct {
+    const int32_t *const *part_select;
+    const int32_t        *part_n_select;
+} kdn_select;
+
 /* Launch shape of the tile pipeline.  0 in a field keeps the built-in default.  tile_bytes: bf16
  * bytes moved per pipeline slot (multiple of 128); stages: slots per CTA; ctas_per_sm: persistent
  * CTAs per SM; compute_groups: groups of four compute warps per CTA in launches that code, decode or
- * rotate (1, 2, 3, 4 or 6); store_lag: how many shared-to-global copies may still be draining before
- * the storer waits (1..4).  stages is raised to store_lag + 2 and rounded down to a multiple of
+ * rotate; group_warps: warps per group, 4 (groups 1, 2, 3, 4 or 6) or 1 (groups 2, 4 or 8); store_lag: how many shared-to-global copies may still be draining before
+ * the storer waits (1..16).  stages is raised to store_lag + 2 and rounded down to a multiple of
  * compute_groups.  Settings that do not fit in shared memory are rejected with KDN_E_UNSUPPORTED. */
 typedef struct {
     int32_t tile_bytes;
@@ -147,7 +170,7 @@ typedef struct {
     int32_t ctas_per_sm;
     int32_t compute_groups;
     int32_t store_lag;
-    int32_t reserved;   /* 0 */
+    int32_t group_warps;
 } kdn_tuning;
 
 /* Create a context on CUDA device `device` (makes it current for the call).  KDN_E_CUDA when no
@@ -209,7 +232,7 @@ kdn_status kdn_compose(kdn_ctx *ctx, int pool_id, const kdn_compose_req *reqs, i
 #define KDN_STATIC_MAX_PARTS     128
 #define KDN_STATIC_MAX_LAYERS    128
 #define KDN_STATIC_MAX_HEAD_DIM  512
-#define KDN_STATIC_SCRATCH_BYTES 274688
+#define KDN_STATIC_SCRATCH_BYTES 278784
 
 /* kdn_compose for callers that must not allocate device memory.  (The paper has no counterpart to
  * this call; it exists for integration reasons only.)
@@ -244,6 +267,19 @@ kdn_status kdn_compose(kdn_ctx *ctx, int pool_id, const kdn_compose_req *reqs, i
  * race on the array and corrupt each other; issue them on one stream or order them yourself. */
 kdn_status kdn_compose_static(int device, const kdn_pool_desc *pool, const kdn_compose_req *reqs, int n_reqs,
                               void *cuda_stream, int wait);
+
+/* kdn_store / kdn_retrieve for chunks that hold only the tokens of a keep-list (see kdn_sparse_op).  One tile per
+ * listed token row; list entries that point outside the block table are skipped and reported as KDN_E_RANGE by
+ * kdn_status_sync.  kdn_retrieve_sparse writes exactly the listed positions. */
+kdn_status kdn_store_sparse(kdn_ctx *ctx, int pool_id, const kdn_sparse_op *ops, int n_ops,
+                            void *cuda_stream, void *side_stream);
+kdn_status kdn_retrieve_sparse(kdn_ctx *ctx, int pool_id, const kdn_sparse_op *ops, int n_ops,
+                               void *cuda_stream, void *side_stream);
+
+/* kdn_compose that delivers only selected tokens of each part (see kdn_select); selects[r] belongs to reqs[r].
+ * Rotation, codecs and everything else are as in kdn_compose. */
+kdn_status kdn_compose_select(kdn_ctx *ctx, int pool_id, const kdn_compose_req *reqs, const kdn_select *selects,
+                              int n_reqs, void *cuda_stream, void *side_stream);
 
 /* Wait for cuda_stream (and the context's side stream) and return the first error a kernel of this
  * context recorded since the last call of this function, or KDN_OK. */

@@ -162,7 +162,7 @@ kdn_status launch_kernel(K kernel, int threads, unsigned grid, size_t smem, cuda
 // Built-in launch shapes, from sweeps on 8B-shaped KV with fully fragmented tables on B200.  The copy
 // form runs best with about two tiles of loads and two of stores in flight per SM; deeper queues lose
 // 3-4 % of bandwidth.  The coding forms want more compute warps per SM than the copy form needs.
-struct Shape { int tile_bytes, stages, ctas_per_sm, groups, lag; };
+struct Shape { int tile_bytes, stages, ctas_per_sm, groups, lag; int gw = 4; };
 Shape default_shape(int OP, bool any_int8, bool any_rot)
 {
     if (!any_int8 && !any_rot) return Shape{ 32768, 4, 1, 0, 2 };
@@ -187,17 +187,17 @@ kdn_status fit_stages(int &stages, int groups, int lag, bool shrink, unsigned st
     return smem_bytes(stages, stage_bytes) > smem_limit ? KDN_E_UNSUPPORTED : KDN_OK;
 }
 
-// Launch the instantiation for (OP, compute groups); groups = 0 is the pure-copy form.
-kdn_status launch_tiles(int OP, int groups, unsigned grid, size_t smem, cudaStream_t stream, const Launch &lp)
+// Launch the instantiation for (OP, compute groups, warps per group); groups = 0 is the pure-copy form.
+kdn_status launch_tiles(int OP, int groups, int gw, unsigned grid, size_t smem, cudaStream_t stream, const Launch &lp)
 {
-#define KDN_CASE(G)                                                                                         \
-    case G:                                                                                                 \
-        if (OP == OP_STORE) return launch_kernel(kdn_store_kernel<G>, threads_for(G), grid, smem, stream, lp);      \
-        if (OP == OP_RETRIEVE) return launch_kernel(kdn_retrieve_kernel<G>, threads_for(G), grid, smem, stream, lp); \
-        return launch_kernel(kdn_compose_kernel<G>, threads_for(G), grid, smem, stream, lp);
-    switch (groups) {
-        KDN_CASE(0) KDN_CASE(1) KDN_CASE(2) KDN_CASE(3) KDN_CASE(4) KDN_CASE(6)
+#define KDN_CASE(G, W)                                                                                             \
+    if (groups == G && (G == 0 || gw == W)) {                                                                      \
+        if (OP == OP_STORE) return launch_kernel(kdn_store_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp);      \
+        if (OP == OP_RETRIEVE) return launch_kernel(kdn_retrieve_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp); \
+        return launch_kernel(kdn_compose_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp);                        \
     }
+    KDN_CASE(0, 4) KDN_CASE(1, 4) KDN_CASE(2, 4) KDN_CASE(3, 4) KDN_CASE(4, 4) KDN_CASE(6, 4)
+    KDN_CASE(2, 1) KDN_CASE(4, 1) KDN_CASE(8, 1)
 #undef KDN_CASE
     return KDN_E_UNSUPPORTED;
 }
@@ -206,10 +206,12 @@ kdn_status launch_tiles(int OP, int groups, unsigned grid, size_t smem, cudaStre
 kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *hops, int n, cudaStream_t stream)
 {
     if (n <= 0) return KDN_OK;
-    bool any_int8 = false, any_rot = false;
+    bool any_int8 = false, any_rot = false, any_list = false, all_list = true;
     for (int i = 0; i < n; ++i) {
         any_int8 |= hops[i].op.codec != KDN_CODEC_RAW_BF16;
         any_rot |= hops[i].rotate;
+        any_list |= hops[i].op.list_mode != 0;
+        all_list &= hops[i].op.list_mode != 0;
     }
     const bool compute = any_int8 || any_rot;
     const unsigned row_elems = (unsigned)pool.H * (unsigned)pool.D;
@@ -218,12 +220,23 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     unsigned unit = 8;
     if (any_int8) unit = lcm_u(unit, 64);
     if (any_rot) unit = lcm_u(unit, (unsigned)pool.D);
-    const Shape def = default_shape(OP, any_int8, any_rot);
+    Shape def = default_shape(OP, any_int8, any_rot);
     int tile_bytes = ctx->tuning.tile_bytes > 0 ? ctx->tuning.tile_bytes : def.tile_bytes;
     unsigned tile_elems = (unsigned)tile_bytes / 2u / unit * unit;
     if (tile_elems < unit) tile_elems = unit;
     const unsigned long long block_elems = (unsigned long long)pool.bs * row_elems;
     if (tile_elems > block_elems) tile_elems = (unsigned)((block_elems + unit - 1) / unit * unit);
+    // a token-list op moves one token row per tile: the tile must hold a row; a launch of only such ops uses
+    // row-sized slots and as many of them as fit, to keep enough bytes in flight
+    if (any_list && tile_elems < row_elems) tile_elems = row_elems;
+    if (all_list) {
+        // row-sized tiles are bound by the per-CTA loader and storer, not by bytes in flight per CTA: measured on
+        // the 8B shape (2 KiB rows), throughput grows with CTAs per SM up to 8 (copy form 3.0 -> 6.4 TB/s)
+        tile_elems = row_elems;
+        if (!any_int8 && !any_rot) def = Shape{ 0, 4, 8, 0, 1 };
+        else if (OP == OP_STORE) def = Shape{ 0, 8, 8, 2, 2, 1 };      // two single-warp groups: a row is one warp's work
+        else def = Shape{ 0, 8, 6, 1, 2 };
+    }
     const unsigned tpb = (unsigned)((block_elems + tile_elems - 1) / tile_elems);
 
     const unsigned a_bytes = (tile_elems * 2u + 127u) & ~127u;
@@ -264,7 +277,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
             op.rope = n_rope++;
         }
         h_ops[i] = op;
-        tiles += (unsigned long long)op.nl * 2ull * (unsigned long long)op.nblk * tpb;
+        tiles += (unsigned long long)op.nl * 2ull * (op.list_mode ? (unsigned long long)op.n_list : (unsigned long long)op.nblk * tpb);
         if (tiles > kMaxTilesPerLaunch) return KDN_E_UNSUPPORTED;
     }
     if (tiles == 0) return KDN_OK;
@@ -310,7 +323,8 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
 
     unsigned long long want = (unsigned long long)ctx->sm_count * (unsigned)ctas_per_sm;
     const unsigned grid = (unsigned)(tiles < want ? tiles : want);
-    kdn_status st = launch_tiles(OP, groups, grid, smem, stream, lp);
+    const int gw = ctx->tuning.group_warps > 0 ? ctx->tuning.group_warps : def.gw;
+    kdn_status st = launch_tiles(OP, groups, gw, grid, smem, stream, lp);
     if (st != KDN_OK) return st;
     ctx->launches++;
     if (slot) {
@@ -331,7 +345,7 @@ kdn_status launch_all(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<
 }
 
 // The device record of an op that covers all layers of a device-resident chunk.
-HostOp make_host_op(const Pool &pool, const int32_t *table, int64_t off, const kdn_chunk &c)
+HostOp make_host_op(const Pool &pool, const int32_t *table, int32_t n_table, int64_t off, const kdn_chunk &c)
 {
     HostOp h;
     std::memset(&h.op, 0, sizeof h.op);
@@ -345,6 +359,7 @@ HostOp make_host_op(const Pool &pool, const int32_t *table, int64_t off, const k
     h.op.rope = -1;
     h.op.l0 = 0;
     h.op.nl = pool.L;
+    h.op.pos_end = (long long)n_table * pool.bs;
     const size_t elems = (size_t)pool.L * 2u * (size_t)c.n_tokens * (size_t)pool.H * (size_t)pool.D;
     if (c.codec == KDN_CODEC_INT8_G64) h.op.scales = (unsigned char *)c.data + elems;
     if (c.codec == KDN_CODEC_INT4_G64) h.op.scales = (unsigned char *)c.data + elems / 2u;
@@ -487,8 +502,40 @@ kdn_status xfer(kdn_ctx *ctx, int pool_id, int OP, const kdn_xfer_op *ops, int n
     std::vector<HostOp> dev_ops, host_ops;
     for (int i = 0; i < n_ops; ++i) {
         if (ops[i].chunk.n_tokens == 0) continue;
-        HostOp h = make_host_op(pool, ops[i].block_table, ops[i].token_offset, ops[i].chunk);
+        HostOp h = make_host_op(pool, ops[i].block_table, ops[i].n_table_blocks, ops[i].token_offset, ops[i].chunk);
         (ops[i].chunk.mem == KDN_MEM_PINNED_HOST ? host_ops : dev_ops).push_back(h);
+    }
+    return run_ops(ctx, pool_id, OP, dev_ops, host_ops, cuda_stream, side_stream);
+}
+
+// Keep-list transfers: the chunk holds only the listed tokens (chunk token i <-> token_offset + keep[i]).
+kdn_status xfer_sparse(kdn_ctx *ctx, int pool_id, int OP, const kdn_sparse_op *ops, int n_ops, void *cuda_stream, void *side_stream)
+{
+    if (!ctx || pool_id < 0 || (size_t)pool_id >= ctx->pools.size()) return KDN_E_INVAL;
+    if (n_ops < 0 || (n_ops > 0 && !ops)) return KDN_E_INVAL;
+    const Pool &pool = ctx->pools[(size_t)pool_id];
+    const kdn_pool_desc shape = shape_of(pool);
+    kdn_status st = check_shape(&shape);
+    if (st != KDN_OK) return st;
+    for (int i = 0; i < n_ops; ++i) {
+        const kdn_xfer_op &o = ops[i].op;
+        st = check_chunk(&shape, &o.chunk);
+        if (st != KDN_OK) return st;
+        if (o.n_table_blocks < 0 || o.token_offset < 0) return KDN_E_INVAL;
+        if (o.chunk.n_tokens > 0 && (!o.block_table || !ops[i].keep)) return KDN_E_INVAL;
+        // the listed tokens are distinct positions below the end of the table, so there cannot be more of them
+        if ((int64_t)o.chunk.n_tokens > (int64_t)o.n_table_blocks * pool.bs - o.token_offset) return KDN_E_RANGE;
+    }
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return KDN_E_CUDA;
+    std::vector<HostOp> dev_ops, host_ops;
+    for (int i = 0; i < n_ops; ++i) {
+        const kdn_xfer_op &o = ops[i].op;
+        if (o.chunk.n_tokens == 0) continue;
+        HostOp h = make_host_op(pool, o.block_table, o.n_table_blocks, o.token_offset, o.chunk);
+        h.op.list = ops[i].keep;
+        h.op.n_list = o.chunk.n_tokens;
+        h.op.list_mode = 1;
+        (o.chunk.mem == KDN_MEM_PINNED_HOST ? host_ops : dev_ops).push_back(h);
     }
     return run_ops(ctx, pool_id, OP, dev_ops, host_ops, cuda_stream, side_stream);
 }
@@ -662,7 +709,7 @@ kdn_status kdn_retrieve_layerwise(kdn_ctx *ctx, int pool_id, const kdn_xfer_op *
     std::vector<HostOp> dev_all, host_all;
     for (int i = 0; i < n_ops; ++i) {
         if (ops[i].chunk.n_tokens == 0) continue;
-        HostOp h = make_host_op(pool, ops[i].block_table, ops[i].token_offset, ops[i].chunk);
+        HostOp h = make_host_op(pool, ops[i].block_table, ops[i].n_table_blocks, ops[i].token_offset, ops[i].chunk);
         (ops[i].chunk.mem == KDN_MEM_PINNED_HOST ? host_all : dev_all).push_back(h);
     }
     cudaStream_t stream = (cudaStream_t)cuda_stream;
@@ -681,7 +728,33 @@ kdn_status kdn_retrieve_layerwise(kdn_ctx *ctx, int pool_id, const kdn_xfer_op *
     return KDN_OK;
 }
 
+static kdn_status compose_impl(kdn_ctx *ctx, int pool_id, const kdn_compose_req *reqs, const kdn_select *selects, int n_reqs,
+                               void *cuda_stream, void *side_stream);
+
 kdn_status kdn_compose(kdn_ctx *ctx, int pool_id, const kdn_compose_req *reqs, int n_reqs, void *cuda_stream, void *side_stream)
+{
+    return compose_impl(ctx, pool_id, reqs, nullptr, n_reqs, cuda_stream, side_stream);
+}
+
+kdn_status kdn_compose_select(kdn_ctx *ctx, int pool_id, const kdn_compose_req *reqs, const kdn_select *selects, int n_reqs,
+                              void *cuda_stream, void *side_stream)
+{
+    if (n_reqs > 0 && !selects) return KDN_E_INVAL;
+    return compose_impl(ctx, pool_id, reqs, selects, n_reqs, cuda_stream, side_stream);
+}
+
+kdn_status kdn_store_sparse(kdn_ctx *ctx, int pool_id, const kdn_sparse_op *ops, int n_ops, void *cuda_stream, void *side_stream)
+{
+    return xfer_sparse(ctx, pool_id, OP_STORE, ops, n_ops, cuda_stream, side_stream);
+}
+
+kdn_status kdn_retrieve_sparse(kdn_ctx *ctx, int pool_id, const kdn_sparse_op *ops, int n_ops, void *cuda_stream, void *side_stream)
+{
+    return xfer_sparse(ctx, pool_id, OP_RETRIEVE, ops, n_ops, cuda_stream, side_stream);
+}
+
+static kdn_status compose_impl(kdn_ctx *ctx, int pool_id, const kdn_compose_req *reqs, const kdn_select *selects, int n_reqs,
+                               void *cuda_stream, void *side_stream)
 {
     if (!ctx || pool_id < 0 || (size_t)pool_id >= ctx->pools.size()) return KDN_E_INVAL;
     const Pool &pool = ctx->pools[(size_t)pool_id];
@@ -695,12 +768,20 @@ kdn_status kdn_compose(kdn_ctx *ctx, int pool_id, const kdn_compose_req *reqs, i
         for (int j = 0; j < q.n_parts; ++j) {
             const kdn_chunk &c = q.parts[j];
             if (c.n_tokens == 0) continue;
-            HostOp h = make_host_op(pool, q.block_table, q.part_dst_pos[j], c);
+            HostOp h = make_host_op(pool, q.block_table, q.n_table_blocks, q.part_dst_pos[j], c);
             const long long delta = (long long)(q.part_dst_pos[j] - c.base_pos);
             if (delta != 0) {
                 h.rotate = true;
                 h.rp.delta = delta;
                 h.rp.theta = q.rope_theta;
+            }
+            if (selects && selects[r].part_select && selects[r].part_select[j]) {
+                if (!selects[r].part_n_select || selects[r].part_n_select[j] < 0 || selects[r].part_n_select[j] > c.n_tokens)
+                    return KDN_E_INVAL;
+                if (selects[r].part_n_select[j] == 0) continue;          // nothing of this part is delivered
+                h.op.list = selects[r].part_select[j];
+                h.op.n_list = selects[r].part_n_select[j];
+                h.op.list_mode = 2;
             }
             (c.mem == KDN_MEM_PINNED_HOST ? host_ops : dev_ops).push_back(h);
         }
@@ -734,7 +815,8 @@ kdn_status kdn_set_tuning(kdn_ctx *ctx, const kdn_tuning *tuning)
     if (tuning->store_lag > kMaxStoreLag) return KDN_E_UNSUPPORTED;
     if (tuning->ctas_per_sm > 32) return KDN_E_UNSUPPORTED;
     if (tuning->compute_groups < 0) return KDN_E_INVAL;
-    if (tuning->compute_groups > kMaxGroups || tuning->compute_groups == 5) return KDN_E_UNSUPPORTED;
+    if (tuning->compute_groups > kMaxGroups) return KDN_E_UNSUPPORTED;
+    if (tuning->group_warps != 0 && tuning->group_warps != 1 && tuning->group_warps != 4) return KDN_E_UNSUPPORTED;
     if (tuning->tile_bytes > ctx->smem_optin) return KDN_E_UNSUPPORTED;
     ctx->tuning = *tuning;
     return KDN_OK;
@@ -780,15 +862,15 @@ const char *kdn_strerror(kdn_status status)
 //   256    void *k_layers[128]
 //   1280   void *v_layers[128]
 //   2304   DevOp ops[128]
-//   10496  RopeParam rope[128]
-//   12544  float2 table[128 * 256]         (rows x head_dim/2, packed by the call's head_dim)
+//   14592  RopeParam rope[128]
+//   16640  float2 table[128 * 256]         (rows x head_dim/2, packed by the call's head_dim)
 // In host code `g_static_scratch` is only a handle for cudaGetSymbolAddress, never an address to
 // hand to a kernel.
 static __device__ __align__(256) unsigned char g_static_scratch[KDN_STATIC_SCRATCH_BYTES];
 
 namespace {
 
-constexpr size_t kStOffK = 256, kStOffV = 1280, kStOffOps = 2304, kStOffRope = 10496, kStOffTable = 12544;
+constexpr size_t kStOffK = 256, kStOffV = 1280, kStOffOps = 2304, kStOffRope = 14592, kStOffTable = 16640;
 constexpr size_t kStHeadBytes = kStOffTable;                 // everything the host uploads per call
 constexpr int kStMaxDevices = 64;
 static_assert(kStOffTable + sizeof(float2) * KDN_STATIC_MAX_PARTS * (KDN_STATIC_MAX_HEAD_DIM / 2) == KDN_STATIC_SCRATCH_BYTES,
@@ -903,7 +985,7 @@ extern "C" kdn_status kdn_compose_static(int device, const kdn_pool_desc *pool, 
         for (int j = 0; j < q.n_parts; ++j) {
             const kdn_chunk &c = q.parts[j];
             if (c.n_tokens == 0) continue;
-            HostOp h = make_host_op(p, q.block_table, q.part_dst_pos[j], c);
+            HostOp h = make_host_op(p, q.block_table, q.n_table_blocks, q.part_dst_pos[j], c);
             DevOp op = h.op;
             op.tile_begin = (unsigned)tiles;
             const long long delta = (long long)(q.part_dst_pos[j] - c.base_pos);
@@ -952,7 +1034,7 @@ extern "C" kdn_status kdn_compose_static(int device, const kdn_pool_desc *pool, 
         lp.store_lag = def.lag;
         const unsigned long long want = (unsigned long long)sd->sm_count * (unsigned)ctas_per_sm;
         const unsigned grid = (unsigned)(tiles < want ? tiles : want);
-        st = launch_tiles(OP_COMPOSE, def.groups, grid, smem, stream, lp);
+        st = launch_tiles(OP_COMPOSE, def.groups, def.gw, grid, smem, stream, lp);
         if (st != KDN_OK) return st;
     }
     if (!wait) return KDN_OK;

@@ -6,12 +6,13 @@
 // plane and one logical block of the request, the tokens of that block that belong to the chunk
 // are contiguous both in the pool block and in the chunk plane.  A run is cut into tiles of at most
 // tile_elems elements; tile g of the launch is handled by CTA g % gridDim.x.  Nothing in a tile
-// depends on another tile, so there is no inter-CTA synchronisation.
+// depends on another tile, so there is no inter-CTA synchronisation.  Ops with a token list (keep-list,
+// select-list) are cut into one tile per listed token row instead.
 //
 // Pipeline inside a CTA (S slots of shared memory, all hand-offs through mbarriers):
 //   loader warp   decodes tiles 32 at a time (one per lane: op lookup, block-table entry, addresses),
 //                 then issues each tile's bulk async copies global -> shared
-//   compute warps (G groups of 4; group g owns slots g, g+G, ...) int8 coding / decoding and key
+//   compute warps (G groups of 4 warps, or of 1 warp for row-sized tiles; group g owns slots g, g+G, ...) int8 coding / decoding and key
 //                 rotation, shared -> shared
 //   storer thread issues the bulk async copy shared -> global and recycles the slot
 // Tiles that are a pure copy (raw bf16 without rotation) never touch the compute warps' ALUs.
@@ -26,13 +27,12 @@
 namespace kdn {
 
 constexpr int kLoaderWarp = 0;
-constexpr int kGroupWarps = 4;                // warps that work together on one tile
-constexpr int kGroupThreads = kGroupWarps * 32;
-constexpr int kMaxGroups = 6;                 // compute groups per CTA; group g owns slots g, g + G, ...
-__host__ __device__ constexpr int threads_for(int groups) { return 32 + groups * kGroupThreads + 32; }  // loader + compute + storer
+constexpr int kMaxGroups = 8;                 // compute groups per CTA; group g owns slots g, g + G, ...
+// A compute group is kGW warps (4 for ordinary tiles, 1 for row-sized tiles) that work together on one tile.
+__host__ __device__ constexpr int threads_for(int groups, int group_warps) { return 32 + groups * group_warps * 32 + 32; }  // loader + compute + storer
 constexpr int kThreadsCopy = 64;                             // loader + storer
 constexpr int kMaxStages = 32;
-constexpr int kMaxStoreLag = 4;           // most bulk-store groups allowed to be still reading shared memory
+constexpr int kMaxStoreLag = 16;          // most bulk-store groups allowed to be still reading shared memory
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 enum : uint32_t { TF_CODED = 1u, TF_ROTATE = 2u, TF_SCALES_PLAIN = 4u, TF_INT4 = 8u };   // TF_CODED: int8 or int4
@@ -54,9 +54,15 @@ struct __align__(16) DevOp {
     int rope;                 // row of the rotation table, -1: keys are copied
     int l0;                   // first pool layer
     int nl;                   // layers held in data
-    unsigned char *scales;    // int8: fp32 scales of the same layers; raw: unused
+    unsigned char *scales;    // int8 / int4: fp32 scales of the same layers; raw: unused
+    const int32_t *list;      // device token list (list_mode != 0): relative request positions, increasing
+    int n_list;               // listed tokens
+    int list_mode;            // 0: every token; 1 keep-list: chunk token i <-> off + list[i];
+                              // 2 select-list: chunk token list[i] <-> off + list[i]
+    long long pos_end;        // request positions >= pos_end are outside the block table
+    long long reserved;
 };
-static_assert(sizeof(DevOp) == 64, "DevOp is copied as 64-byte records");
+static_assert(sizeof(DevOp) == 96, "DevOp is copied as 96-byte records");
 
 struct RopeParam {            // one row of the rotation table to fill
     long long delta;          // dst_pos - base_pos
@@ -168,20 +174,34 @@ __device__ __forceinline__ void bulk_wait_read_n(int n)      // the instruction 
     case 1: bulk_wait_read<1>(); break;
     case 2: bulk_wait_read<2>(); break;
     case 3: bulk_wait_read<3>(); break;
-    default: bulk_wait_read<4>(); break;
+    case 4: bulk_wait_read<4>(); break;
+    case 5: bulk_wait_read<5>(); break;
+    case 6: bulk_wait_read<6>(); break;
+    case 7: bulk_wait_read<7>(); break;
+    case 8: bulk_wait_read<8>(); break;
+    case 9: bulk_wait_read<9>(); break;
+    case 10: bulk_wait_read<10>(); break;
+    case 11: bulk_wait_read<11>(); break;
+    case 12: bulk_wait_read<12>(); break;
+    case 13: bulk_wait_read<13>(); break;
+    case 14: bulk_wait_read<14>(); break;
+    case 15: bulk_wait_read<15>(); break;
+    default: bulk_wait_read<16>(); break;
     }
 }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 __device__ __forceinline__ void fence_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
-__device__ __forceinline__ void group_bar_sync(int group)
+__device__ __forceinline__ void group_bar_sync(int group, unsigned gthreads)
 {
     switch (group) {                                       // immediate ids: only kMaxGroups barriers are reserved
-    case 0: asm volatile("bar.sync 1, %0;" ::"n"(kGroupThreads) : "memory"); break;
-    case 1: asm volatile("bar.sync 2, %0;" ::"n"(kGroupThreads) : "memory"); break;
-    case 2: asm volatile("bar.sync 3, %0;" ::"n"(kGroupThreads) : "memory"); break;
-    case 3: asm volatile("bar.sync 4, %0;" ::"n"(kGroupThreads) : "memory"); break;
-    case 4: asm volatile("bar.sync 5, %0;" ::"n"(kGroupThreads) : "memory"); break;
-    default: asm volatile("bar.sync 6, %0;" ::"n"(kGroupThreads) : "memory"); break;
+    case 0: asm volatile("bar.sync 1, %0;" ::"r"(gthreads) : "memory"); break;
+    case 1: asm volatile("bar.sync 2, %0;" ::"r"(gthreads) : "memory"); break;
+    case 2: asm volatile("bar.sync 3, %0;" ::"r"(gthreads) : "memory"); break;
+    case 3: asm volatile("bar.sync 4, %0;" ::"r"(gthreads) : "memory"); break;
+    case 4: asm volatile("bar.sync 5, %0;" ::"r"(gthreads) : "memory"); break;
+    case 5: asm volatile("bar.sync 6, %0;" ::"r"(gthreads) : "memory"); break;
+    case 6: asm volatile("bar.sync 7, %0;" ::"r"(gthreads) : "memory"); break;
+    default: asm volatile("bar.sync 8, %0;" ::"r"(gthreads) : "memory"); break;
     }
 }
 
@@ -274,13 +294,13 @@ __device__ __forceinline__ uint32_t pack_codes4(uint32_t r0, uint32_t r1, uint32
 // kInt4: codes in [-7, 7], two per byte (element 2k in the low nibble), 16 bytes per lane instead of 32.
 template <bool kInt4>
 __device__ __forceinline__ void quantise_tile(const unsigned char *A, unsigned char *B, float *S, float *g_scales,
-                                              unsigned n, int ct)
+                                              unsigned n, int ct, unsigned gthreads)
 {
     const float qmax = kInt4 ? 7.0f : 127.0f;
     const unsigned nhalf = n >> 5;                         // 32-element half groups
     const unsigned lane = (unsigned)ct & 31u;
     const unsigned rot = (lane >> 1) & 3u;
-    for (unsigned hb = (unsigned)ct & ~31u; hb < nhalf; hb += kGroupThreads) {
+    for (unsigned hb = (unsigned)ct & ~31u; hb < nhalf; hb += gthreads) {
         const unsigned h = hb + lane;
         const bool act = h < nhalf;
         const unsigned char *src = A + (size_t)h * 64u;
@@ -362,11 +382,11 @@ __device__ __forceinline__ uint32_t pack_bf16x2(f32x2 v)
 
 // Decode n int8 codes at B with scales S into bf16 at A: one fp32 product per element, rounded to bf16.
 __device__ __forceinline__ void dequantise_tile(const unsigned char *B, const float *S, unsigned char *A,
-                                                unsigned n, int ct)
+                                                unsigned n, int ct, unsigned gthreads)
 {
     const unsigned nvec = n >> 4;
     const f32x2 minus_bias = pack2(-8388736.0f, -8388736.0f);
-    for (unsigned v = (unsigned)ct; v < nvec; v += kGroupThreads) {
+    for (unsigned v = (unsigned)ct; v < nvec; v += gthreads) {
         const uint4 c = lds128(B + (size_t)v * 16u);
         const float sc = S[v >> 2];
         const f32x2 sc2 = pack2(sc, sc);
@@ -396,11 +416,11 @@ __device__ __forceinline__ void nibbles_to_f32x2(uint32_t w, f32x2 minus_bias4, 
 
 // Decode n int4 codes (n/2 bytes at B) with scales S into bf16 at A.
 __device__ __forceinline__ void dequantise4_tile(const unsigned char *B, const float *S, unsigned char *A,
-                                                 unsigned n, int ct)
+                                                 unsigned n, int ct, unsigned gthreads)
 {
     const unsigned nvec = n >> 4;                          // 16 codes = 8 bytes per step
     const f32x2 minus_bias4 = pack2(-8388616.0f, -8388616.0f);   // -(2^23 + 8)
-    for (unsigned v = (unsigned)ct; v < nvec; v += kGroupThreads) {
+    for (unsigned v = (unsigned)ct; v < nvec; v += gthreads) {
         const uint2 c = lds64(B + (size_t)v * 8u);
         const float sc = S[v >> 2];
         const f32x2 sc2 = pack2(sc, sc);
@@ -456,7 +476,7 @@ __device__ __forceinline__ void rotate8(const f32x2 *u, const f32x2 *w, const Ro
 // kCodec = 0: bf16 at A, in place.  kCodec = 1 / 2: int8 / int4 codes at B and scales at S -> bf16 at A.
 template <int kCodec>
 __device__ __forceinline__ void rotate_tile(unsigned char *A, const unsigned char *B, const float *S, unsigned n,
-                                            unsigned D, const float2 *table, int rope, RotCoef &rc, int ct)
+                                            unsigned D, const float2 *table, int rope, RotCoef &rc, int ct, unsigned gthreads)
 {
     const unsigned half = D >> 1;
     const unsigned per_row = D >> 4;                      // work items per head row
@@ -464,7 +484,7 @@ __device__ __forceinline__ void rotate_tile(unsigned char *A, const unsigned cha
     const unsigned shift = 31u - (unsigned)__clz(per_row);
     const unsigned items = n >> 4;
     const f32x2 minus_bias = pack2(-8388736.0f, -8388736.0f);
-    for (unsigned it = (unsigned)ct; it < items; it += kGroupThreads) {
+    for (unsigned it = (unsigned)ct; it < items; it += gthreads) {
         const unsigned r = pow2 ? it >> shift : it / per_row;
         const unsigned col = (it - r * per_row) << 3;
         load_coef(rc, table, rope, col, half);
@@ -520,27 +540,47 @@ __device__ __forceinline__ void decode_tile(const Launch &P, unsigned g, TileDes
     }
     const DevOp op = ops[lo];
     const unsigned gl = g - op.tile_begin;
-    const unsigned per_plane = (unsigned)op.nblk * P.tpb;
-    const unsigned plane = gl / per_plane;
-    const unsigned rem = gl - plane * per_plane;
-    const unsigned j = rem / P.tpb;
-    const unsigned k = rem - j * P.tpb;
+    unsigned plane, n;
+    long long id_index;                                     // block-table entry of the tile
+    unsigned long long pool_elem;                           // element offset of the tile inside its pool block
+    unsigned long long ce;                                  // element offset of the tile inside the chunk
+    if (op.list_mode != 0) {
+        // one listed token (one row of H * D elements) per tile
+        plane = gl / (unsigned)op.n_list;
+        const unsigned i = gl - plane * (unsigned)op.n_list;
+        const long long rel = __ldg(op.list + i);
+        const long long c = op.list_mode == 2 ? rel : (long long)i;      // chunk token
+        const long long p = op.off + rel;
+        if (rel < 0 || p >= op.pos_end || c >= op.T) { atomicCAS(P.status, 0, kStatusRange); return; }
+        id_index = p / P.bs;
+        pool_elem = (unsigned long long)(p - id_index * P.bs) * P.row_elems;
+        ce = ((unsigned long long)plane * op.T + (unsigned long long)c) * P.row_elems;
+        n = P.row_elems;
+    } else {
+        const unsigned per_plane = (unsigned)op.nblk * P.tpb;
+        plane = gl / per_plane;
+        const unsigned rem = gl - plane * per_plane;
+        const unsigned j = rem / P.tpb;
+        const unsigned k = rem - j * P.tpb;
+        const long long blk_start = ((long long)op.j0 + j) * P.bs;
+        const long long p_lo = op.off > blk_start ? op.off : blk_start;
+        const long long p_end = op.off + op.T;
+        const long long p_hi = p_end < blk_start + P.bs ? p_end : blk_start + P.bs;
+        if (p_hi <= p_lo) return;
+        const unsigned long long run = (unsigned long long)(p_hi - p_lo) * P.row_elems;
+        const unsigned long long e0 = (unsigned long long)k * P.tile_elems;
+        if (e0 >= run) return;
+        n = (unsigned)((run - e0) < (unsigned long long)P.tile_elems ? (run - e0) : P.tile_elems);
+        id_index = (long long)op.j0 + j;
+        pool_elem = (unsigned long long)(p_lo - blk_start) * P.row_elems + e0;
+        ce = ((unsigned long long)plane * op.T + (unsigned long long)(p_lo - op.off)) * P.row_elems + e0;
+    }
     const int kv = (int)(plane & 1u);
     const int l = op.l0 + (int)(plane >> 1);
-    const long long blk_start = ((long long)op.j0 + j) * P.bs;
-    const long long p_lo = op.off > blk_start ? op.off : blk_start;
-    const long long p_end = op.off + op.T;
-    const long long p_hi = p_end < blk_start + P.bs ? p_end : blk_start + P.bs;
-    if (p_hi <= p_lo) return;
-    const unsigned long long run = (unsigned long long)(p_hi - p_lo) * P.row_elems;
-    const unsigned long long e0 = (unsigned long long)k * P.tile_elems;
-    if (e0 >= run) return;
-    const unsigned n = (unsigned)((run - e0) < (unsigned long long)P.tile_elems ? (run - e0) : P.tile_elems);
-    const long long id = __ldg(op.table + op.j0 + j);
+    const long long id = __ldg(op.table + id_index);
     if (id < 0 || id >= P.n_blocks) { atomicCAS(P.status, 0, kStatusRange); return; }
     const unsigned char *base = reinterpret_cast<const unsigned char *>(kv ? P.v_layers[l] : P.k_layers[l]);
-    d.g_pool = (unsigned long long)(base + (((unsigned long long)id * P.bs + (unsigned long long)(p_lo - blk_start)) * P.row_elems + e0) * 2ull);
-    const unsigned long long ce = ((unsigned long long)plane * op.T + (unsigned long long)(p_lo - op.off)) * P.row_elems + e0;
+    d.g_pool = (unsigned long long)(base + ((unsigned long long)id * P.bs * P.row_elems + pool_elem) * 2ull);
     if (op.codec == 0) {
         d.g_chunk = (unsigned long long)(op.data + ce * 2ull);
     } else {
@@ -584,10 +624,11 @@ __host__ __device__ inline size_t smem_bytes(int stages, unsigned stage_bytes)
     return (size_t)stages * stage_bytes + 24u * (size_t)stages + 16u + sizeof(TileDesc) * (size_t)stages + 16u;
 }
 
-template <int OP, int kGroups>
+template <int OP, int kGroups, int kGW>
 __device__ __forceinline__ void tile_pipeline(const Launch &P)
 {
     constexpr bool kCompute = kGroups > 0;
+    constexpr unsigned kGT = (unsigned)kGW * 32u;           // threads of one compute group
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const Smem sm = carve(P, smem_raw);
     const int S = P.stages;
@@ -599,7 +640,7 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
         for (int s = 0; s < S; ++s) {
             mbar_init(sm.full + 8u * s, 1u);
             mbar_init(sm.empty + 8u * s, 1u);
-            mbar_init(sm.ready + 8u * s, (uint32_t)kGroupWarps);
+            mbar_init(sm.ready + 8u * s, (uint32_t)kGW);
         }
         *sm.abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -609,7 +650,7 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
 
     const unsigned grid = gridDim.x, bid = blockIdx.x;
     const unsigned n_my = P.n_tiles > bid ? (P.n_tiles - bid + grid - 1u) / grid : 0u;
-    const int storer_warp = 1 + kGroups * kGroupWarps;
+    const int storer_warp = 1 + kGroups * kGW;
 
     if (warp == kLoaderWarp) {
         // ------------------------------------------------------------ loader
@@ -713,8 +754,8 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
         }
     } else if (kCompute) {
         // ----------------------------------------------------------- compute
-        const int group = (tid - 32) / kGroupThreads;       // this group owns slots group, group + 2, ...
-        const int ct = (tid - 32) % kGroupThreads;
+        const int group = (tid - 32) / (int)kGT;            // this group owns slots group, group + kGroups, ...
+        const int ct = (tid - 32) % (int)kGT;
         RotCoef rc;
         rc.rope = -1; rc.col = 0xffffffffu;
         for (unsigned slot = (unsigned)group; slot < n_my; slot += (unsigned)kGroups) {
@@ -731,27 +772,27 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                 if (OP == OP_STORE) {
                     if (flags & TF_CODED) {
                         float *gs = (flags & TF_SCALES_PLAIN) ? reinterpret_cast<float *>(sm.desc[st].g_scales) : nullptr;
-                        if (flags & TF_INT4) quantise_tile<true>(A, B, Sc, gs, n, ct);
-                        else quantise_tile<false>(A, B, Sc, gs, n, ct);
+                        if (flags & TF_INT4) quantise_tile<true>(A, B, Sc, gs, n, ct, kGT);
+                        else quantise_tile<false>(A, B, Sc, gs, n, ct, kGT);
                         computed = true;
                     }
                 } else if (flags & TF_CODED) {
                     if (flags & TF_SCALES_PLAIN) {
                         const float *gs = reinterpret_cast<const float *>(sm.desc[st].g_scales);
-                        for (unsigned i = (unsigned)ct; i < (n >> 6); i += kGroupThreads) Sc[i] = __ldg(gs + i);
-                        group_bar_sync(group);
+                        for (unsigned i = (unsigned)ct; i < (n >> 6); i += kGT) Sc[i] = __ldg(gs + i);
+                        group_bar_sync(group, kGT);
                     }
                     if (OP == OP_COMPOSE && (flags & TF_ROTATE)) {
-                        if (flags & TF_INT4) rotate_tile<2>(A, B, Sc, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct);
-                        else rotate_tile<1>(A, B, Sc, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct);
+                        if (flags & TF_INT4) rotate_tile<2>(A, B, Sc, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct, kGT);
+                        else rotate_tile<1>(A, B, Sc, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct, kGT);
                     } else if (flags & TF_INT4) {
-                        dequantise4_tile(B, Sc, A, n, ct);
+                        dequantise4_tile(B, Sc, A, n, ct, kGT);
                     } else {
-                        dequantise_tile(B, Sc, A, n, ct);
+                        dequantise_tile(B, Sc, A, n, ct, kGT);
                     }
                     computed = true;
                 } else if (OP == OP_COMPOSE && (flags & TF_ROTATE)) {
-                    rotate_tile<0>(A, nullptr, nullptr, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct);
+                    rotate_tile<0>(A, nullptr, nullptr, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct, kGT);
                     computed = true;
                 }
             }
@@ -769,19 +810,19 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
 // The host keeps stages a multiple of kGroups, so a pipeline slot always belongs to the same group and
 // every waiter visits a barrier once per phase (a parity wait cannot tell phases two apart).
 // Sec. 3.2 call (i) store, Sec. 3.1 storage module: paged pool -> chunk, optional int8 coding.
-template <int kGroups>
-__global__ void __launch_bounds__(threads_for(kGroups))
-kdn_store_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_STORE, kGroups>(P); }
+template <int kGroups, int kGW>
+__global__ void __launch_bounds__(threads_for(kGroups, kGW))
+kdn_store_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_STORE, kGroups, kGW>(P); }
 
 // Sec. 3.2 call (ii) retrieve, Sec. 3.1 delivery module (decompression on the GPU): chunk -> pool.
-template <int kGroups>
-__global__ void __launch_bounds__(threads_for(kGroups))
-kdn_retrieve_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_RETRIEVE, kGroups>(P); }
+template <int kGroups, int kGW>
+__global__ void __launch_bounds__(threads_for(kGroups, kGW))
+kdn_retrieve_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_RETRIEVE, kGroups, kGW>(P); }
 
 // Sec. 3.1 blending module: parts -> request blocks at new positions, keys re-rotated.
-template <int kGroups>
-__global__ void __launch_bounds__(threads_for(kGroups))
-kdn_compose_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_COMPOSE, kGroups>(P); }
+template <int kGroups, int kGW>
+__global__ void __launch_bounds__(threads_for(kGroups, kGW))
+kdn_compose_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_COMPOSE, kGroups, kGW>(P); }
 
 // Rotation table: row r, frequency i -> (cos, sin) of delta_r * theta_r^(-2i/D), evaluated in fp64 and
 // rounded once to fp32 (an fp32 angle would lose more than half a bf16 ulp at large position shifts).

@@ -21,7 +21,8 @@ KDN_MEM_DEVICE, KDN_MEM_PINNED_HOST = 0, 1
 EXPORTS = ["kdn_create", "kdn_destroy", "kdn_pool_register", "kdn_chunk_bytes", "kdn_validate_xfer",
            "kdn_validate_compose", "kdn_store", "kdn_retrieve", "kdn_compose", "kdn_status_sync",
            "kdn_set_tuning", "kdn_set_staging_bytes", "kdn_launch_count", "kdn_strerror",
-           "kdn_compose_static", "kdn_retrieve_layerwise"]
+           "kdn_compose_static", "kdn_retrieve_layerwise",
+           "kdn_store_sparse", "kdn_retrieve_sparse", "kdn_compose_select"]
 
 
 class kdn_pool_desc(C.Structure):
@@ -46,9 +47,17 @@ class kdn_compose_req(C.Structure):
                 ("rope_theta", C.c_double), ("rope_style", C.c_int32), ("reserved", C.c_int32)]
 
 
+class kdn_sparse_op(C.Structure):
+    _fields_ = [("op", kdn_xfer_op), ("keep", C.c_void_p)]
+
+
+class kdn_select(C.Structure):
+    _fields_ = [("part_select", C.POINTER(C.c_void_p)), ("part_n_select", C.POINTER(C.c_int32))]
+
+
 class kdn_tuning(C.Structure):
     _fields_ = [("tile_bytes", C.c_int32), ("stages", C.c_int32), ("ctas_per_sm", C.c_int32),
-                ("compute_groups", C.c_int32), ("store_lag", C.c_int32), ("reserved", C.c_int32)]
+                ("compute_groups", C.c_int32), ("store_lag", C.c_int32), ("group_warps", C.c_int32)]
 
 
 def _load() -> C.CDLL:
@@ -79,6 +88,12 @@ def _load() -> C.CDLL:
         fn.argtypes = [vp, i32, C.POINTER(kdn_xfer_op), i32, vp, vp]
     lib.kdn_retrieve_layerwise.restype = i32
     lib.kdn_retrieve_layerwise.argtypes = [vp, i32, C.POINTER(kdn_xfer_op), i32, i32, vp, vp, C.POINTER(vp)]
+    for name in ("kdn_store_sparse", "kdn_retrieve_sparse"):
+        fn = getattr(lib, name)
+        fn.restype = i32
+        fn.argtypes = [vp, i32, C.POINTER(kdn_sparse_op), i32, vp, vp]
+    lib.kdn_compose_select.restype = i32
+    lib.kdn_compose_select.argtypes = [vp, i32, C.POINTER(kdn_compose_req), C.POINTER(kdn_select), i32, vp, vp]
     lib.kdn_compose.restype = i32
     lib.kdn_compose.argtypes = [vp, i32, C.POINTER(kdn_compose_req), i32, vp, vp]
     lib.kdn_compose_static.restype = i32
@@ -229,6 +244,35 @@ def kdn_retrieve_layerwise(ctx, pool_id: int, ops: Sequence[XferOp], layers_per_
                                       ev), "kdn_retrieve_layerwise")
 
 
+def sparse_array(ops: Sequence[XferOp], keeps: Sequence[int]):
+    arr = (kdn_sparse_op * max(1, len(ops)))()
+    for i, (o, kp) in enumerate(zip(ops, keeps)):
+        arr[i] = kdn_sparse_op(kdn_xfer_op(o.block_table, o.n_table_blocks, 0, o.token_offset, o.chunk.c()), kp)
+    return arr
+
+
+def kdn_store_sparse(ctx, pool_id: int, ops: Sequence[XferOp], keeps: Sequence[int], stream: int = 0, side_stream: int = 0) -> None:
+    """keeps[i]: device address of the int32 keep-list of ops[i] (ops[i].chunk.n_tokens entries)."""
+    _check(lib.kdn_store_sparse(ctx, pool_id, sparse_array(ops, keeps), len(ops), stream, side_stream), "kdn_store_sparse")
+
+
+def kdn_retrieve_sparse(ctx, pool_id: int, ops: Sequence[XferOp], keeps: Sequence[int], stream: int = 0, side_stream: int = 0) -> None:
+    _check(lib.kdn_retrieve_sparse(ctx, pool_id, sparse_array(ops, keeps), len(ops), stream, side_stream), "kdn_retrieve_sparse")
+
+
+def kdn_compose_select(ctx, pool_id: int, reqs: Sequence[ComposeReq], selects, stream: int = 0, side_stream: int = 0) -> None:
+    """selects[r]: list with one entry per part of reqs[r]: None (every token) or (device address, count)."""
+    arr = (kdn_select * max(1, len(reqs)))()
+    keep = []
+    for r, sel in enumerate(selects):
+        n = len(sel)
+        ptrs = (C.c_void_p * max(1, n))(*[(x[0] if x else None) for x in sel])
+        cnts = (C.c_int32 * max(1, n))(*[(x[1] if x else 0) for x in sel])
+        keep.append((ptrs, cnts))
+        arr[r] = kdn_select(C.cast(ptrs, C.POINTER(C.c_void_p)), C.cast(cnts, C.POINTER(C.c_int32)))
+    _check(lib.kdn_compose_select(ctx, pool_id, compose_array(reqs), arr, len(reqs), stream, side_stream), "kdn_compose_select")
+
+
 def kdn_compose(ctx, pool_id: int, reqs: Sequence[ComposeReq], stream: int = 0, side_stream: int = 0) -> None:
     _check(lib.kdn_compose(ctx, pool_id, compose_array(reqs), len(reqs), stream, side_stream), "kdn_compose")
 
@@ -246,8 +290,8 @@ def kdn_status_sync(ctx, stream: int = 0) -> int:
 
 
 def kdn_set_tuning(ctx, tile_bytes: int = 0, stages: int = 0, ctas_per_sm: int = 0, compute_groups: int = 0,
-                   store_lag: int = 0) -> None:
-    t = kdn_tuning(tile_bytes, stages, ctas_per_sm, compute_groups, store_lag, 0)
+                   store_lag: int = 0, group_warps: int = 0) -> None:
+    t = kdn_tuning(tile_bytes, stages, ctas_per_sm, compute_groups, store_lag, group_warps)
     _check(lib.kdn_set_tuning(ctx, C.byref(t)), "kdn_set_tuning")
 
 
