@@ -179,10 +179,10 @@ class ClockSampler:
 # DRAM bytes (read + write) per launch from the committed ncu capture of a reduced case (8 chunks per
 # store/retrieve launch, 2 parts per compose launch; profiles/ncu_full_small_case_llama3_8b.md), scaled by the
 # units a bench launch processes.  Valid only for the kernel source the capture was taken from.
-NCU_KERNEL_SHA = "59ec05579632cb7b"
-NCU_SMALL_CASE_BYTES = {"store_raw": (536.894720e6 + 485.936384e6, 8), "retrieve_raw": (536.895744e6 + 490.880256e6, 8),
-                        "compose_raw": (268.468992e6 + 221.113088e6, 2), "store_int8": (536.903680e6 + 252.184576e6, 8),
-                        "retrieve_int8": (285.241600e6 + 483.000064e6, 8), "compose_int8": (142.639616e6 + 213.129216e6, 2)}
+NCU_KERNEL_SHA = "34fb2edbebe6ef81"
+NCU_SMALL_CASE_BYTES = {"store_raw": (536.902400e6 + 491.561984e6, 8), "retrieve_raw": (536.900608e6 + 491.330048e6, 8),
+                        "compose_raw": (268.481024e6 + 224.729088e6, 2), "store_int8": (536.914432e6 + 252.475136e6, 8),
+                        "retrieve_int8": (285.250048e6 + 482.733056e6, 8), "compose_int8": (142.692352e6 + 214.896640e6, 2)}
 
 
 def measured_traffic(op: str, units: float):
