@@ -85,6 +85,12 @@ def lib():
             L.kdn_oracle_compose.restype = i32
             L.kdn_oracle_compose.argtypes = [vp, i32, i32, i32, i32, i64, vp, i32, i32,
                                              vp, vp, vp, vp, vp, f64, vp, vp]
+            L.kdn_oracle_fnv1a.restype = C.c_uint64
+            L.kdn_oracle_fnv1a.argtypes = [vp, sz]
+            L.kdn_oracle_key_hash.restype = C.c_uint64
+            L.kdn_oracle_key_hash.argtypes = [vp, sz]
+            L.kdn_oracle_checksum.restype = C.c_uint64
+            L.kdn_oracle_checksum.argtypes = [vp, sz]
             _lib = L
     return _lib
 
@@ -240,3 +246,21 @@ def rotate_pair(u: float, w: float, phi: float):
     a, b = C.c_double(), C.c_double()
     lib().kdn_oracle_rotate_pair(float(u), float(w), float(phi), C.byref(a), C.byref(b))
     return a.value, b.value
+
+
+def fnv1a(data: bytes) -> int:
+    a = np.frombuffer(data, dtype=np.uint8) if len(data) else np.zeros(0, dtype=np.uint8)
+    a = np.ascontiguousarray(a)
+    return int(lib().kdn_oracle_fnv1a(_ptr(a) if a.size else None, a.size))
+
+
+def key_hash(tokens) -> int:
+    a = np.ascontiguousarray(tokens, dtype=np.int32)
+    return int(lib().kdn_oracle_key_hash(_ptr(a) if a.size else None, a.size))
+
+
+def checksum(payload: np.ndarray) -> int:
+    a = np.ascontiguousarray(payload, dtype=np.uint8)
+    if a.size % 4:
+        raise ValueError("payload must be a multiple of 4 bytes")
+    return int(lib().kdn_oracle_checksum(_ptr(a) if a.size else None, a.size))

@@ -54,6 +54,12 @@
  *                    select-list: compose may deliver only some tokens of a part: for each listed chunk token c
  *                    (strictly increasing) it writes position dst_pos + c and leaves the other positions alone.
  *
+ *   R8  storage shell (Sec. 3.1 storage module: "stores the KV caches keyed by various texts"; Sec. 3.2 interface:
+ *                    store "with the associated text", retrieve "using some text".)  key = FNV-1a 64-bit hash of the
+ *                    text's token ids taken as little-endian 32-bit integers; payload checksum =
+ *                    sum_i ((w_i XOR 0x9E3779B9) * ((2 i + 1) mod 2^32)) mod 2^64 over the payload's little-endian
+ *                    32-bit words w_i.  Neither is prescribed by the paper.
+ *
  * Parity pins (tests/test_oracle_*.py, all CPU): brute force against an
  * independent index-by-index formulation on tiny shapes; contiguous table
  * reduces store to a slice copy; store-then-retrieve identity on raw bf16 for
@@ -491,4 +497,45 @@ int kdn_oracle_compose(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,
 {
     return kdn_oracle_compose_select(pool, L, H, D, bs, nb, table, n_table, n_parts, chunks, part_T, part_codec,
                                      base_pos, dst_pos, theta, NULL, NULL, kref, kmag);
+}
+
+/* ------------------------------------------------------- storage shell -- */
+
+/* R8: FNV-1a, 64 bit, over n bytes. */
+uint64_t kdn_oracle_fnv1a(const uint8_t *bytes, size_t n)
+{
+    uint64_t h = 0xcbf29ce484222325ull;
+    for (size_t i = 0; i < n; ++i) {
+        h ^= bytes[i];
+        h *= 0x100000001b3ull;
+    }
+    return h;
+}
+
+/* R8: key of a text given as token ids (each id hashed as its four little-endian bytes). */
+uint64_t kdn_oracle_key_hash(const int32_t *tokens, size_t n)
+{
+    uint64_t h = 0xcbf29ce484222325ull;
+    for (size_t i = 0; i < n; ++i) {
+        uint32_t t = (uint32_t)tokens[i];
+        for (int b = 0; b < 4; ++b) {
+            h ^= (t >> (8 * b)) & 0xffu;
+            h *= 0x100000001b3ull;
+        }
+    }
+    return h;
+}
+
+/* R8: payload checksum; bytes must be a multiple of 4 (every chunk layout is). */
+uint64_t kdn_oracle_checksum(const uint8_t *payload, size_t bytes)
+{
+    uint64_t c = 0;
+    for (size_t i = 0; i < bytes / 4; ++i) {
+        uint32_t w = (uint32_t)payload[4 * i] | ((uint32_t)payload[4 * i + 1] << 8) |
+                     ((uint32_t)payload[4 * i + 2] << 16) | ((uint32_t)payload[4 * i + 3] << 24);
+        uint32_t a = w ^ 0x9E3779B9u;
+        uint32_t m = (uint32_t)(2u * (uint32_t)i + 1u);
+        c += (uint64_t)a * (uint64_t)m;
+    }
+    return c;
 }
