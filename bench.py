@@ -377,6 +377,21 @@ def run_gpu(args) -> None:
     op_ms = {n: float(np.mean([ev[it][i].elapsed_time(ev[it][i + 1]) for it in range(args.steps)]))
              for i, n in enumerate(names)}
 
+    # ---- storage shell: payload checksum over the raw chunk library (read-only stream; not part of `value`)
+    lib_buf = dev_sets[RAW]["chunks"]
+    csum_out = torch.zeros(1, dtype=torch.int64, device=dev)
+    for _ in range(3):
+        K.kdn_checksum(local, lib_buf.data_ptr(), lib_buf.numel(), csum_out.data_ptr(), s)
+    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    reps = max(1, min(args.steps, 20))
+    a.record(stream)
+    for _ in range(reps):
+        K.kdn_checksum(local, lib_buf.data_ptr(), lib_buf.numel(), csum_out.data_ptr(), s)
+    b.record(stream)
+    torch.cuda.synchronize()
+    shell_ops = {"checksum_raw_library": {"ms": a.elapsed_time(b) / reps, "bytes": lib_buf.numel(),
+                                          "gbs": lib_buf.numel() / (a.elapsed_time(b) / reps * 1e-3) / 1e9}}
+
     # ---- the int4 codec (a widening beyond the benchmark step; timed on its own, not part of `value`)
     int4_ops = {}
     i4 = make_sets(False, codecs=(INT4,))[INT4]
@@ -432,7 +447,7 @@ def run_gpu(args) -> None:
     if args.no_e2e:
         if rank == 0:
             print(json.dumps({"note": "profiling run, not a bench record", "ops_ms": op_ms,
-                              "ops_gbs": {n: op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 for n in names}, "int4": int4_ops, "sparse": sparse_ops}))
+                              "ops_gbs": {n: op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 for n in names}, "int4": int4_ops, "sparse": sparse_ops, "shell": shell_ops}))
         K.kdn_destroy(ctx)
         return
 
@@ -538,7 +553,7 @@ def run_gpu(args) -> None:
             "config": {"workload": W["text"], "l2": "inputs larger than L2 (every op streams >= 1.9 GB once)",
                        "bytes_per_step": step_bytes},
             "tokens_per_s_reloaded": world * reload_tokens / (sum(op_ms[n] for n in names if not n.startswith("store")) * 1e-3),
-            "ops": ops, "ops_int4_not_in_value": int4_ops, "ops_keep_list_not_in_value": sparse_ops,
+            "ops": ops, "ops_int4_not_in_value": int4_ops, "ops_keep_list_not_in_value": sparse_ops, "ops_shell_not_in_value": shell_ops,
             "roofline": {"bound": "hbm", "kernel": kernel_of[top], "op": top, "achieved": ops[top]["gbs"], "peak": peak,
                          "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": ops[top]["gbs"] / peak,
                          "frac_of_nominal_8000": ops[top]["gbs"] / 8000.0, "traffic": traffic},

@@ -78,7 +78,9 @@ typedef enum {
     KDN_E_UNSUPPORTED = 5,  /* int8 / int4 with head_dim % 64 != 0; rotation with head_dim % 16 != 0; ... */
     KDN_E_CUDA = 6,         /* a CUDA runtime call failed */
     KDN_E_NOMEM = 7,        /* context scratch could not be allocated */
-    KDN_E_TIMEOUT = 8       /* a bounded wait inside a kernel gave up (device) */
+    KDN_E_TIMEOUT = 8,      /* a bounded wait inside a kernel gave up (device) */
+    KDN_E_NOTFOUND = 9,     /* kdn_index_get / kdn_index_remove: no chunk under this key */
+    KDN_E_CHECKSUM = 10     /* kdn_header_check: the payload does not match the header's checksum */
 } kdn_status;
 
 typedef enum { KDN_CODEC_RAW_BF16 = 0, KDN_CODEC_INT8_G64 = 1, KDN_CODEC_INT4_G64 = 2 } kdn_codec;
@@ -293,6 +295,62 @@ kdn_status kdn_set_staging_bytes(kdn_ctx *ctx, size_t bytes_per_slab);
 
 /* Kernels this context has launched so far (for accounting; never reset). */
 uint64_t kdn_launch_count(const kdn_ctx *ctx);
+
+/* ------------------------------------------------------------------------------------------------
+ * Storage-module shell (Sec. 3.1: the storage module "stores the KV caches keyed by various texts"; Sec. 3.2:
+ * the engine stores a KV cache "with the associated text" and retrieves it "using some text").  The paper fixes
+ * neither a key, a header nor an eviction rule; these are this library's choices.  The shell owns no chunk
+ * memory: it maps keys to the caller's chunk descriptors and says which ones to drop. */
+
+/* Key of a text: FNV-1a (64 bit) over its token ids, each taken as four little-endian bytes.  Host arithmetic. */
+uint64_t kdn_key_hash(const int32_t *token_ids, size_t n);
+
+/* Payload checksum, computed on the GPU: sum over the payload's little-endian 32-bit words w_i of
+ * (w_i XOR 0x9E3779B9) * ((2 i + 1) mod 2^32), modulo 2^64.  payload: DEVICE memory, 4-byte aligned (16 for full
+ * speed), bytes a multiple of 4 (every chunk layout is).  The result is written to *device_out (DEVICE uint64,
+ * 8-byte aligned) by work enqueued on cuda_stream; read it after synchronising.  Needs no context. */
+kdn_status kdn_checksum(int device, const void *payload, size_t bytes, uint64_t *device_out, void *cuda_stream);
+
+/* Self-describing header a caller can keep in front of (or beside) a stored chunk: 128 bytes, little endian. */
+typedef struct {
+    char     magic[8];        /* "KDNCHNK1" */
+    uint32_t header_bytes;    /* 128 */
+    uint32_t codec;           /* kdn_codec */
+    int32_t  n_layers, n_kv_heads, head_dim, n_tokens;
+    int64_t  base_pos;
+    uint64_t payload_bytes;
+    uint64_t key;
+    uint64_t checksum;
+    uint8_t  reserved[64];    /* 0 */
+} kdn_chunk_header;
+
+/* Fill *out for `chunk` of a pool of this shape.  KDN_E_SHAPE if chunk.bytes does not fit shape, tokens and codec. */
+kdn_status kdn_header_fill(const kdn_pool_desc *pool, const kdn_chunk *chunk, uint64_t key, uint64_t checksum,
+                           kdn_chunk_header *out);
+/* Check a header read back from storage against the pool's shape and against the checksum the caller computed over
+ * the payload it read (kdn_checksum).  KDN_E_INVAL: not a header; KDN_E_SHAPE: another model shape or inconsistent
+ * sizes; KDN_E_CHECKSUM: payload damaged.  On KDN_OK and out != NULL, fills out->bytes, n_tokens, codec, base_pos
+ * (data and mem stay the caller's to set). */
+kdn_status kdn_header_check(const kdn_pool_desc *pool, const kdn_chunk_header *header, uint64_t checksum_of_payload,
+                            kdn_chunk *out);
+
+/* Index from key to chunk descriptor with least-recently-used eviction under a byte budget.  Not thread safe. */
+typedef struct kdn_index kdn_index;
+typedef struct { size_t capacity_bytes, bytes, entries; uint64_t hits, misses, evictions; } kdn_index_info;
+
+kdn_status kdn_index_create(kdn_index **out, size_t capacity_bytes);
+void kdn_index_destroy(kdn_index *index);
+/* Insert `chunk` under `key` as the most recently used entry.  A chunk already stored under the key is replaced and
+ * handed back first in evicted[]; then least-recently-used entries are dropped until the budget holds, each handed
+ * back in evicted[] (the caller frees or reuses their memory).  If more than max_evicted descriptors would have to be
+ * handed back, or the chunk alone exceeds the budget, nothing changes and KDN_E_NOMEM is returned. */
+kdn_status kdn_index_put(kdn_index *index, uint64_t key, const kdn_chunk *chunk, kdn_chunk *evicted, int max_evicted,
+                         int *n_evicted);
+/* Look a key up (KDN_E_NOTFOUND if absent) and mark it most recently used. */
+kdn_status kdn_index_get(kdn_index *index, uint64_t key, kdn_chunk *out);
+/* Drop a key; its descriptor is returned in *out (may be NULL). */
+kdn_status kdn_index_remove(kdn_index *index, uint64_t key, kdn_chunk *out);
+void kdn_index_stats(const kdn_index *index, kdn_index_info *out);
 
 /* Static string for a status code. */
 const char *kdn_strerror(kdn_status status);

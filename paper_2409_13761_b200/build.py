@@ -10,7 +10,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libkdn.so")
-SOURCES = [os.path.join(CSRC, "kdn.cu")]
+SOURCES = [os.path.join(CSRC, "kdn.cu"), os.path.join(CSRC, "kdn_shell.cu")]
 DEPS = SOURCES + [os.path.join(CSRC, "kdn_kernels.cuh"), os.path.join(ROOT, "include", "kdn.h")]
 
 

@@ -849,6 +849,8 @@ const char *kdn_strerror(kdn_status status)
     case KDN_E_CUDA: return "CUDA runtime error";
     case KDN_E_NOMEM: return "out of memory";
     case KDN_E_TIMEOUT: return "a bounded wait inside a kernel expired";
+    case KDN_E_NOTFOUND: return "no chunk under this key";
+    case KDN_E_CHECKSUM: return "payload does not match the header's checksum";
     }
     return "unknown status";
 }

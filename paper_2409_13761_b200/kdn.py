@@ -14,7 +14,7 @@ from typing import List, Optional, Sequence
 from . import build as _build
 
 KDN_OK, KDN_E_INVAL, KDN_E_SHAPE, KDN_E_ALIGN, KDN_E_RANGE, KDN_E_UNSUPPORTED, KDN_E_CUDA, KDN_E_NOMEM, \
-    KDN_E_TIMEOUT = range(9)
+    KDN_E_TIMEOUT, KDN_E_NOTFOUND, KDN_E_CHECKSUM = range(11)
 KDN_CODEC_RAW_BF16, KDN_CODEC_INT8_G64, KDN_CODEC_INT4_G64 = 0, 1, 2
 KDN_MEM_DEVICE, KDN_MEM_PINNED_HOST = 0, 1
 
@@ -22,7 +22,9 @@ EXPORTS = ["kdn_create", "kdn_destroy", "kdn_pool_register", "kdn_chunk_bytes", 
            "kdn_validate_compose", "kdn_store", "kdn_retrieve", "kdn_compose", "kdn_status_sync",
            "kdn_set_tuning", "kdn_set_staging_bytes", "kdn_launch_count", "kdn_strerror",
            "kdn_compose_static", "kdn_retrieve_layerwise",
-           "kdn_store_sparse", "kdn_retrieve_sparse", "kdn_compose_select"]
+           "kdn_store_sparse", "kdn_retrieve_sparse", "kdn_compose_select",
+           "kdn_key_hash", "kdn_checksum", "kdn_header_fill", "kdn_header_check", "kdn_index_create", "kdn_index_destroy",
+           "kdn_index_put", "kdn_index_get", "kdn_index_remove", "kdn_index_stats"]
 
 
 class kdn_pool_desc(C.Structure):
@@ -53,6 +55,18 @@ class kdn_sparse_op(C.Structure):
 
 class kdn_select(C.Structure):
     _fields_ = [("part_select", C.POINTER(C.c_void_p)), ("part_n_select", C.POINTER(C.c_int32))]
+
+
+class kdn_chunk_header(C.Structure):
+    _fields_ = [("magic", C.c_char * 8), ("header_bytes", C.c_uint32), ("codec", C.c_uint32),
+                ("n_layers", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32), ("n_tokens", C.c_int32),
+                ("base_pos", C.c_int64), ("payload_bytes", C.c_uint64), ("key", C.c_uint64), ("checksum", C.c_uint64),
+                ("reserved", C.c_uint8 * 64)]
+
+
+class kdn_index_info(C.Structure):
+    _fields_ = [("capacity_bytes", C.c_size_t), ("bytes", C.c_size_t), ("entries", C.c_size_t),
+                ("hits", C.c_uint64), ("misses", C.c_uint64), ("evictions", C.c_uint64)]
 
 
 class kdn_tuning(C.Structure):
@@ -106,6 +120,26 @@ def _load() -> C.CDLL:
     lib.kdn_set_staging_bytes.argtypes = [vp, C.c_size_t]
     lib.kdn_launch_count.restype = C.c_uint64
     lib.kdn_launch_count.argtypes = [vp]
+    lib.kdn_key_hash.restype = C.c_uint64
+    lib.kdn_key_hash.argtypes = [vp, C.c_size_t]
+    lib.kdn_checksum.restype = i32
+    lib.kdn_checksum.argtypes = [i32, vp, C.c_size_t, vp, vp]
+    lib.kdn_header_fill.restype = i32
+    lib.kdn_header_fill.argtypes = [C.POINTER(kdn_pool_desc), C.POINTER(kdn_chunk), C.c_uint64, C.c_uint64, C.POINTER(kdn_chunk_header)]
+    lib.kdn_header_check.restype = i32
+    lib.kdn_header_check.argtypes = [C.POINTER(kdn_pool_desc), C.POINTER(kdn_chunk_header), C.c_uint64, C.POINTER(kdn_chunk)]
+    lib.kdn_index_create.restype = i32
+    lib.kdn_index_create.argtypes = [C.POINTER(vp), C.c_size_t]
+    lib.kdn_index_destroy.restype = None
+    lib.kdn_index_destroy.argtypes = [vp]
+    lib.kdn_index_put.restype = i32
+    lib.kdn_index_put.argtypes = [vp, C.c_uint64, C.POINTER(kdn_chunk), C.POINTER(kdn_chunk), i32, C.POINTER(i32)]
+    lib.kdn_index_get.restype = i32
+    lib.kdn_index_get.argtypes = [vp, C.c_uint64, C.POINTER(kdn_chunk)]
+    lib.kdn_index_remove.restype = i32
+    lib.kdn_index_remove.argtypes = [vp, C.c_uint64, C.POINTER(kdn_chunk)]
+    lib.kdn_index_stats.restype = None
+    lib.kdn_index_stats.argtypes = [vp, C.POINTER(kdn_index_info)]
     lib.kdn_strerror.restype = C.c_char_p
     lib.kdn_strerror.argtypes = [i32]
     return lib
@@ -301,3 +335,69 @@ def kdn_set_staging_bytes(ctx, bytes_per_slab: int) -> None:
 
 def kdn_launch_count(ctx) -> int:
     return int(lib.kdn_launch_count(ctx))
+
+
+# ------------------------------------------------------------------------ storage-module shell --
+
+def _chunk_from_c(c: kdn_chunk) -> Chunk:
+    return Chunk(c.data or 0, c.bytes, c.n_tokens, c.codec, c.mem, c.base_pos)
+
+
+def kdn_key_hash(token_ids) -> int:
+    arr = (C.c_int32 * max(1, len(token_ids)))(*[int(t) for t in token_ids])
+    return int(lib.kdn_key_hash(arr, len(token_ids)))
+
+
+def kdn_checksum(device: int, payload: int, nbytes: int, device_out: int, stream: int = 0) -> None:
+    _check(lib.kdn_checksum(int(device), payload, int(nbytes), device_out, stream), "kdn_checksum")
+
+
+def kdn_header_fill(desc: kdn_pool_desc, chunk: Chunk, key: int, checksum: int) -> kdn_chunk_header:
+    h = kdn_chunk_header()
+    c = chunk.c()
+    _check(lib.kdn_header_fill(C.byref(desc), C.byref(c), key, checksum, C.byref(h)), "kdn_header_fill")
+    return h
+
+
+def kdn_header_check(desc: kdn_pool_desc, header: kdn_chunk_header, checksum_of_payload: int):
+    """Returns (status, Chunk or None); the Chunk has bytes, n_tokens, codec, base_pos filled in."""
+    c = kdn_chunk()
+    st = int(lib.kdn_header_check(C.byref(desc), C.byref(header), checksum_of_payload, C.byref(c)))
+    return st, (_chunk_from_c(c) if st == KDN_OK else None)
+
+
+def kdn_index_create(capacity_bytes: int) -> C.c_void_p:
+    idx = C.c_void_p()
+    _check(lib.kdn_index_create(C.byref(idx), int(capacity_bytes)), "kdn_index_create")
+    return idx
+
+
+def kdn_index_destroy(idx) -> None:
+    lib.kdn_index_destroy(idx)
+
+
+def kdn_index_put(idx, key: int, chunk: Chunk, max_evicted: int = 64):
+    """Returns (status, [evicted Chunks])."""
+    ev = (kdn_chunk * max(1, max_evicted))()
+    n = C.c_int(0)
+    c = chunk.c()
+    st = int(lib.kdn_index_put(idx, key, C.byref(c), ev, max_evicted, C.byref(n)))
+    return st, [_chunk_from_c(ev[i]) for i in range(n.value)]
+
+
+def kdn_index_get(idx, key: int):
+    c = kdn_chunk()
+    st = int(lib.kdn_index_get(idx, key, C.byref(c)))
+    return st, (_chunk_from_c(c) if st == KDN_OK else None)
+
+
+def kdn_index_remove(idx, key: int):
+    c = kdn_chunk()
+    st = int(lib.kdn_index_remove(idx, key, C.byref(c)))
+    return st, (_chunk_from_c(c) if st == KDN_OK else None)
+
+
+def kdn_index_stats(idx) -> kdn_index_info:
+    info = kdn_index_info()
+    lib.kdn_index_stats(idx, C.byref(info))
+    return info
