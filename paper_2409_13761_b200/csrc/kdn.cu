@@ -7,6 +7,7 @@
 
 #include <cstdio>
 #include <cstring>
+#include <functional>
 #include <map>
 #include <mutex>
 #include <new>
@@ -334,10 +335,11 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     return KDN_OK;
 }
 
-kdn_status launch_all(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<HostOp> &hops, cudaStream_t stream)
+kdn_status launch_all(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<HostOp> &hops, cudaStream_t stream,
+                      size_t max_ops = kMaxOpsPerLaunch)
 {
-    for (size_t i = 0; i < hops.size(); i += kMaxOpsPerLaunch) {
-        size_t n = hops.size() - i < (size_t)kMaxOpsPerLaunch ? hops.size() - i : (size_t)kMaxOpsPerLaunch;
+    for (size_t i = 0; i < hops.size(); i += max_ops) {
+        size_t n = hops.size() - i < max_ops ? hops.size() - i : max_ops;
         kdn_status st = launch_batch(ctx, pool, OP, hops.data() + i, (int)n, stream);
         if (st != KDN_OK) return st;
     }
@@ -370,8 +372,10 @@ HostOp make_host_op(const Pool &pool, const int32_t *table, int32_t n_table, int
 //   retrieve / compose: side stream copies host -> slab, main stream runs the kernel on the slab;
 //   store:              main stream runs the kernel into the slab, side stream copies slab -> host.
 // While one slab is being copied the kernel works on the other.
+// `between` is called once per slab hand-over, at the point where the main stream would otherwise only wait for the
+// host link: the caller uses it to enqueue a share of its device-resident work there.
 kdn_status run_staged(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<HostOp> &hops,
-                      cudaStream_t stream, cudaStream_t side)
+                      cudaStream_t stream, cudaStream_t side, const std::function<kdn_status()> &between)
 {
     kdn_status st = ensure_slabs(ctx);
     if (st != KDN_OK) return st;
@@ -392,13 +396,17 @@ kdn_status run_staged(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<
             for (const Piece &p : pieces)
                 KDN_CUDA(cudaMemcpyAsync(p.host, ctx->slab[s] + p.slab_off, p.bytes, cudaMemcpyDeviceToHost, side));
             KDN_CUDA(cudaEventRecord(ctx->slab_free[s], side));
+            r = between();                                       // device-resident work runs while the slab drains
+            if (r != KDN_OK) return r;
         } else {
             KDN_CUDA(cudaStreamWaitEvent(side, ctx->slab_free[s], 0));
             for (const Piece &p : pieces)
                 KDN_CUDA(cudaMemcpyAsync(ctx->slab[s] + p.slab_off, p.host, p.bytes, cudaMemcpyHostToDevice, side));
             KDN_CUDA(cudaEventRecord(ctx->slab_ready[s], side));
+            kdn_status r = between();                            // device-resident work runs while the slab fills
+            if (r != KDN_OK) return r;
             KDN_CUDA(cudaStreamWaitEvent(stream, ctx->slab_ready[s], 0));
-            kdn_status r = launch_all(ctx, pool, OP, batch, stream);
+            r = launch_all(ctx, pool, OP, batch, stream);
             if (r != KDN_OK) return r;
             KDN_CUDA(cudaEventRecord(ctx->slab_free[s], stream));
         }
@@ -449,22 +457,51 @@ kdn_status run_staged(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<
     return flush();
 }
 
+// Bytes of the chunk side of one op (what crosses the host link when the chunk is host resident).
+size_t chunk_side_bytes(const Pool &pool, const HostOp &h)
+{
+    const size_t elems = (size_t)h.op.nl * 2u * (size_t)h.op.T * (size_t)pool.H * (size_t)pool.D;
+    if (h.op.codec == KDN_CODEC_RAW_BF16) return elems * 2u;
+    return (h.op.codec == KDN_CODEC_INT4_G64 ? elems / 2u : elems) + elems / 64u * 4u;
+}
+
 kdn_status run_ops(kdn_ctx *ctx, int pool_id, int OP, std::vector<HostOp> &dev_ops, std::vector<HostOp> &host_ops,
                    void *cuda_stream, void *side_stream)
 {
     const Pool &pool = ctx->pools[(size_t)pool_id];
     cudaStream_t stream = (cudaStream_t)cuda_stream;
-    kdn_status st = launch_all(ctx, pool, OP, dev_ops, stream);
-    if (st != KDN_OK) return st;
-    if (!host_ops.empty()) {
-        cudaStream_t side = (cudaStream_t)side_stream;
-        if (!side) {
-            st = ensure_side(ctx);
-            if (st != KDN_OK) return st;
-            side = ctx->own_side;
-        }
-        st = run_staged(ctx, pool, OP, host_ops, stream, side);
+    if (host_ops.empty()) return launch_all(ctx, pool, OP, dev_ops, stream);
+    cudaStream_t side = (cudaStream_t)side_stream;
+    if (!side) {
+        kdn_status st = ensure_side(ctx);
+        if (st != KDN_OK) return st;
+        side = ctx->own_side;
     }
+    // Host-resident chunks cross the link slab by slab.  The device-resident ops of the same call are cut into about
+    // as many launches as there are slab hand-overs and enqueued between them, so the GPU works on them while the
+    // link is busy instead of before it (one stream: a single big launch up front would leave the link idle behind it).
+    size_t staged = 0;
+    for (const HostOp &h : host_ops) staged += chunk_side_bytes(pool, h);
+    size_t n_parts = staged / ctx->slab_bytes + 1;
+    if (n_parts > dev_ops.size()) n_parts = dev_ops.size();
+    size_t dev_total = 0;
+    for (const HostOp &h : dev_ops) dev_total += chunk_side_bytes(pool, h);
+    size_t next = 0, done_bytes = 0, part = 0;
+    auto between = [&]() -> kdn_status {
+        if (next >= dev_ops.size()) return KDN_OK;
+        ++part;
+        const size_t target = part >= n_parts ? dev_total : dev_total / n_parts * part;
+        std::vector<HostOp> share;
+        while (next < dev_ops.size() && (share.empty() || done_bytes < target)) {
+            done_bytes += chunk_side_bytes(pool, dev_ops[next]);
+            share.push_back(dev_ops[next++]);
+        }
+        // at most kInlineOps ops per launch: their records then travel as kernel parameters.  A descriptor copy
+        // would queue on the copy engine behind the slab transfer in flight and hold the launch back by a whole slab.
+        return launch_all(ctx, pool, OP, share, stream, (size_t)kInlineOps);
+    };
+    kdn_status st = run_staged(ctx, pool, OP, host_ops, stream, side, between);
+    while (st == KDN_OK && next < dev_ops.size()) st = between();
     return st;
 }
 

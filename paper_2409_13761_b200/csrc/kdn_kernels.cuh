@@ -69,7 +69,7 @@ struct RopeParam {            // one row of the rotation table to fill
     double theta;
 };
 
-constexpr int kInlineOps = 8;             // launches of up to this many ops carry them as kernel parameters
+constexpr int kInlineOps = 32;            // launches of up to this many ops carry them as kernel parameters (3 KiB)
 
 struct Launch {
     const DevOp *ops;         // device array of n_ops records, or nullptr: the records are in inline_ops
