@@ -134,13 +134,24 @@ __device__ __forceinline__ unsigned long long global_timer_ns()
     asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
     return t;
 }
+// The same test, but the hardware may park the thread for up to `hint_ns` before answering "not yet" (it answers
+// at once when the phase completes), so a waiting warp does not eat issue slots that working warps need.
+__device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t parity, uint32_t hint_ns)
+{
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\t"
+                 "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+                 "selp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity), "r"(hint_ns) : "memory");
+    return ok != 0;
+}
 // Bounded wait: true when the phase completed; false when the CTA is aborting or the limit passed.
 __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag)
 {
     unsigned long long t0 = global_timer_ns();
     for (uint32_t n = 1;; ++n) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((n & 63u) == 0u) {
+        if (mbar_try_wait_parked(bar, parity, 20000u)) return true;
+        if ((n & 15u) == 0u) {
             if (*abort_flag) return false;
             if (global_timer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
         }
