@@ -235,7 +235,7 @@ def run_gpu(args) -> None:
 
     rank, world, local = shard.rank_env()
     dist = None
-    if world > 1:
+    if world > 1 or "TORCHELASTIC_RUN_ID" in os.environ:        # launched by torch.distributed.run, even with one rank
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     torch.cuda.set_device(local)
