@@ -179,10 +179,8 @@ class ClockSampler:
 # DRAM bytes (read + write) per launch from the committed ncu capture of a reduced case (8 chunks per
 # store/retrieve launch, 2 parts per compose launch; profiles/ncu_full_small_case_llama3_8b.md), scaled by the
 # units a bench launch processes.  Valid only for the kernel source the capture was taken from.
-NCU_KERNEL_SHA = "34fb2edbebe6ef81"
-NCU_SMALL_CASE_BYTES = {"store_raw": (536.902400e6 + 491.561984e6, 8), "retrieve_raw": (536.900608e6 + 491.330048e6, 8),
-                        "compose_raw": (268.481024e6 + 224.729088e6, 2), "store_int8": (536.914432e6 + 252.475136e6, 8),
-                        "retrieve_int8": (285.250048e6 + 482.733056e6, 8), "compose_int8": (142.692352e6 + 214.896640e6, 2)}
+NCU_KERNEL_SHA = "b9e8cd645fa7f423"
+NCU_SMALL_CASE_BYTES = {"store_raw": (536.920576e6 + 486.232576e6, 8), "retrieve_raw": (536.900608e6 + 490.784768e6, 8), "compose_raw": (268.483840e6 + 223.139840e6, 2), "store_int8": (536.966400e6 + 252.484608e6, 8), "retrieve_int8": (285.251840e6 + 483.219200e6, 8), "compose_int8": (142.698240e6 + 213.456640e6, 2)}
 
 
 def measured_traffic(op: str, units: float):

@@ -783,8 +783,16 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                 if (OP == OP_STORE) {
                     if (flags & TF_CODED) {
                         float *gs = (flags & TF_SCALES_PLAIN) ? reinterpret_cast<float *>(sm.desc[st].g_scales) : nullptr;
-                        if (flags & TF_INT4) quantise_tile<true>(A, B, Sc, gs, n, ct, kGT);
-                        else quantise_tile<false>(A, B, Sc, gs, n, ct, kGT);
+                        // a full tile of exactly one pass per thread gets a copy of the routine specialised for
+                        // that size (no loop, no tail predicates): about a quarter fewer instructions
+                        constexpr unsigned kOnePass = kGT * 32u;
+                        if (flags & TF_INT4) {
+                            if (n == kOnePass) quantise_tile<true>(A, B, Sc, gs, kOnePass, ct, kGT);
+                            else quantise_tile<true>(A, B, Sc, gs, n, ct, kGT);
+                        } else {
+                            if (n == kOnePass) quantise_tile<false>(A, B, Sc, gs, kOnePass, ct, kGT);
+                            else quantise_tile<false>(A, B, Sc, gs, n, ct, kGT);
+                        }
                         computed = true;
                     }
                 } else if (flags & TF_CODED) {
@@ -797,9 +805,11 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                         if (flags & TF_INT4) rotate_tile<2>(A, B, Sc, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct, kGT);
                         else rotate_tile<1>(A, B, Sc, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct, kGT);
                     } else if (flags & TF_INT4) {
-                        dequantise4_tile(B, Sc, A, n, ct, kGT);
+                        if (n == kGT * 32u) dequantise4_tile(B, Sc, A, kGT * 32u, ct, kGT);
+                        else dequantise4_tile(B, Sc, A, n, ct, kGT);
                     } else {
-                        dequantise_tile(B, Sc, A, n, ct, kGT);
+                        if (n == kGT * 32u) dequantise_tile(B, Sc, A, kGT * 32u, ct, kGT);
+                        else dequantise_tile(B, Sc, A, n, ct, kGT);
                     }
                     computed = true;
                 } else if (OP == OP_COMPOSE && (flags & TF_ROTATE)) {
