@@ -164,11 +164,11 @@ kdn_status launch_kernel(K kernel, int threads, unsigned grid, size_t smem, cuda
 // form runs best with about two tiles of loads and two of stores in flight per SM; deeper queues lose
 // 3-4 % of bandwidth.  The coding forms want more compute warps per SM than the copy form needs.
 struct Shape { int tile_bytes, stages, ctas_per_sm, groups, lag; int gw = 4; };
-Shape default_shape(int OP, bool any_int8, bool any_rot)
+Shape default_shape(int OP, bool any_coded, bool any_rot)
 {
-    if (!any_int8 && !any_rot) return Shape{ 32768, 4, 1, 0, 2 };
+    if (!any_coded && !any_rot) return Shape{ 32768, 4, 1, 0, 2 };
     if (OP != OP_COMPOSE || !any_rot) return Shape{ 8192, 6, 3, 2, 2 };
-    if (!any_int8) return Shape{ 8192, 6, 2, 2, 2 };
+    if (!any_coded) return Shape{ 8192, 6, 2, 2, 2 };
     return Shape{ 16384, 9, 1, 3, 2 };
 }
 
@@ -207,21 +207,21 @@ kdn_status launch_tiles(int OP, int groups, int gw, unsigned grid, size_t smem, 
 kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *hops, int n, cudaStream_t stream)
 {
     if (n <= 0) return KDN_OK;
-    bool any_int8 = false, any_rot = false, any_list = false, all_list = true;
+    bool any_coded = false, any_rot = false, any_list = false, all_list = true;
     for (int i = 0; i < n; ++i) {
-        any_int8 |= hops[i].op.codec != KDN_CODEC_RAW_BF16;
+        any_coded |= hops[i].op.codec != KDN_CODEC_RAW_BF16;
         any_rot |= hops[i].rotate;
         any_list |= hops[i].op.list_mode != 0;
         all_list &= hops[i].op.list_mode != 0;
     }
-    const bool compute = any_int8 || any_rot;
+    const bool compute = any_coded || any_rot;
     const unsigned row_elems = (unsigned)pool.H * (unsigned)pool.D;
 
-    // tile size: whole 16-byte units; whole 64-element groups with int8; whole head rows with rotation
+    // tile size: whole 16-byte units; whole 64-element groups with int8 / int4; whole head rows with rotation
     unsigned unit = 8;
-    if (any_int8) unit = lcm_u(unit, 64);
+    if (any_coded) unit = lcm_u(unit, 64);
     if (any_rot) unit = lcm_u(unit, (unsigned)pool.D);
-    Shape def = default_shape(OP, any_int8, any_rot);
+    Shape def = default_shape(OP, any_coded, any_rot);
     int tile_bytes = ctx->tuning.tile_bytes > 0 ? ctx->tuning.tile_bytes : def.tile_bytes;
     unsigned tile_elems = (unsigned)tile_bytes / 2u / unit * unit;
     if (tile_elems < unit) tile_elems = unit;
@@ -234,7 +234,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
         // row-sized tiles are bound by the per-CTA loader and storer, not by bytes in flight per CTA: measured on
         // the 8B shape (2 KiB rows), throughput grows with CTAs per SM up to 8 (copy form 3.0 -> 6.4 TB/s)
         tile_elems = row_elems;
-        if (!any_int8 && !any_rot) def = Shape{ 0, 4, 8, 0, 1 };
+        if (!any_coded && !any_rot) def = Shape{ 0, 4, 8, 0, 1 };
         else if (OP == OP_STORE) def = Shape{ 0, 8, 8, 2, 2, 1 };      // two single-warp groups: a row is one warp's work
         else def = Shape{ 0, 8, 6, 1, 2 };
     }
@@ -989,18 +989,18 @@ extern "C" kdn_status kdn_compose_static(int device, const kdn_pool_desc *pool, 
     RopeParam *rope = reinterpret_cast<RopeParam *>(head + kStOffRope);
 
     // launch shape: the library defaults for a compose launch
-    bool any_int8 = false, any_rot = false;
+    bool any_coded = false, any_rot = false;
     for (int r = 0; r < n_reqs; ++r)
         for (int j = 0; j < reqs[r].n_parts; ++j) {
             if (reqs[r].parts[j].n_tokens == 0) continue;
-            any_int8 |= reqs[r].parts[j].codec != KDN_CODEC_RAW_BF16;
+            any_coded |= reqs[r].parts[j].codec != KDN_CODEC_RAW_BF16;
             any_rot |= reqs[r].part_dst_pos[j] != reqs[r].parts[j].base_pos;
         }
-    const bool compute = any_int8 || any_rot;
+    const bool compute = any_coded || any_rot;
     unsigned unit = 8;
-    if (any_int8) unit = lcm_u(unit, 64);
+    if (any_coded) unit = lcm_u(unit, 64);
     if (any_rot) unit = lcm_u(unit, (unsigned)p.D);
-    const Shape def = default_shape(OP_COMPOSE, any_int8, any_rot);
+    const Shape def = default_shape(OP_COMPOSE, any_coded, any_rot);
     unsigned tile_elems = (unsigned)def.tile_bytes / 2u / unit * unit;
     if (tile_elems < unit) tile_elems = unit;
     const unsigned long long block_elems = (unsigned long long)p.bs * row_elems;
