@@ -142,8 +142,11 @@ kdn_status ensure_slabs(kdn_ctx *ctx)
 std::mutex g_attr_mutex;
 std::map<std::pair<int, const void *>, size_t> g_attr_granted;
 
+// `overlap`: the launch may start while the kernel before it in the stream (the rotation-table kernel) still runs;
+// the warps that read that kernel's output wait for it on the device.
 template <typename K>
-kdn_status launch_kernel(K kernel, int threads, unsigned grid, size_t smem, cudaStream_t stream, const Launch &lp)
+kdn_status launch_kernel(K kernel, int threads, unsigned grid, size_t smem, cudaStream_t stream, const Launch &lp,
+                         bool overlap = false)
 {
     {
         int device = 0;
@@ -155,7 +158,21 @@ kdn_status launch_kernel(K kernel, int threads, unsigned grid, size_t smem, cuda
             granted = smem;
         }
     }
-    kernel<<<grid, threads, smem, stream>>>(lp);
+    if (overlap) {
+        cudaLaunchConfig_t cfg{};
+        cfg.gridDim = dim3(grid);
+        cfg.blockDim = dim3((unsigned)threads);
+        cfg.dynamicSmemBytes = smem;
+        cfg.stream = stream;
+        cudaLaunchAttribute attr{};
+        attr.id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr.val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = &attr;
+        cfg.numAttrs = 1;
+        KDN_CUDA(cudaLaunchKernelEx(&cfg, kernel, lp));
+    } else {
+        kernel<<<grid, threads, smem, stream>>>(lp);
+    }
     KDN_CUDA(cudaGetLastError());
     return KDN_OK;
 }
@@ -189,13 +206,14 @@ kdn_status fit_stages(int &stages, int groups, int lag, bool shrink, unsigned st
 }
 
 // Launch the instantiation for (OP, compute groups, warps per group); groups = 0 is the pure-copy form.
-kdn_status launch_tiles(int OP, int groups, int gw, unsigned grid, size_t smem, cudaStream_t stream, const Launch &lp)
+kdn_status launch_tiles(int OP, int groups, int gw, unsigned grid, size_t smem, cudaStream_t stream, const Launch &lp,
+                        bool overlap = false)
 {
 #define KDN_CASE(G, W)                                                                                             \
     if (groups == G && (G == 0 || gw == W)) {                                                                      \
         if (OP == OP_STORE) return launch_kernel(kdn_store_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp);      \
         if (OP == OP_RETRIEVE) return launch_kernel(kdn_retrieve_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp); \
-        return launch_kernel(kdn_compose_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp);                        \
+        return launch_kernel(kdn_compose_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp, overlap);               \
     }
     KDN_CASE(0, 4) KDN_CASE(1, 4) KDN_CASE(2, 4) KDN_CASE(3, 4) KDN_CASE(4, 4) KDN_CASE(6, 4)
     KDN_CASE(2, 1) KDN_CASE(4, 1) KDN_CASE(8, 1)
@@ -325,7 +343,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     unsigned long long want = (unsigned long long)ctx->sm_count * (unsigned)ctas_per_sm;
     const unsigned grid = (unsigned)(tiles < want ? tiles : want);
     const int gw = ctx->tuning.group_warps > 0 ? ctx->tuning.group_warps : def.gw;
-    kdn_status st = launch_tiles(OP, groups, gw, grid, smem, stream, lp);
+    kdn_status st = launch_tiles(OP, groups, gw, grid, smem, stream, lp, OP == OP_COMPOSE && n_rope > 0);
     if (st != KDN_OK) return st;
     ctx->launches++;
     if (slot) {

@@ -216,6 +216,13 @@ __device__ __forceinline__ void group_bar_sync(int group, unsigned gthreads)
     }
 }
 
+// Programmatic dependent launch: a kernel launched with the programmatic-serialisation attribute may start while
+// the kernel before it in the stream still runs; dependency_wait() returns once that kernel has finished and its
+// writes are visible (at once when the launch carried no such attribute).  release_dependents() lets the next
+// kernel start early.
+__device__ __forceinline__ void dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void release_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ uint4 lds128(const void *p) { return *reinterpret_cast<const uint4 *>(p); }
 __device__ __forceinline__ uint2 lds64(const void *p) { return *reinterpret_cast<const uint2 *>(p); }
 __device__ __forceinline__ void sts128(void *p, uint4 v) { *reinterpret_cast<uint4 *>(p) = v; }
@@ -666,6 +673,8 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
     if (warp == kLoaderWarp) {
         // ------------------------------------------------------------ loader
         unsigned issued = 0;
+        unsigned st = 0;                                      // pipeline slot of the next tile, and the phase of its
+        uint32_t ph = 0;                                      // barriers (flips every time the slots wrap around)
         bool aborted = false;
         TileDesc cur;
         decode_tile<OP>(P, (unsigned)lane < n_my ? bid + (unsigned)lane * grid : 0xffffffffu, cur);
@@ -675,9 +684,6 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
             const unsigned cnt = n_my - base < 32u ? n_my - base : 32u;
             for (unsigned t = 0; t < cnt; ++t) {
                 if ((unsigned)lane == t) {
-                    const unsigned slot = base + t;
-                    const unsigned st = slot % (unsigned)S;
-                    const uint32_t ph = (slot / (unsigned)S) & 1u;
                     if (mbar_wait(sm.empty + 8u * st, ph ^ 1u, sm.abort_flag)) {
                         sm.desc[st] = cur;
                         const uint32_t bar = sm.full + 8u * st;
@@ -706,6 +712,7 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                 __syncwarp();
                 if (__any_sync(0xffffffffu, *sm.abort_flag != 0)) { aborted = true; break; }
                 ++issued;
+                if (++st == (unsigned)S) { st = 0; ph ^= 1u; }
             }
             cur = nxt;
         }
@@ -723,9 +730,9 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
         // ------------------------------------------------------------ storer
         if (lane == 0) {
             unsigned done = 0;                                // slots whose store group was committed
+            unsigned st = 0, st2 = 0;                         // slot being stored / slot being recycled, with the
+            uint32_t ph = 0, ph2 = 0;                         // phases of their barriers
             for (unsigned slot = 0; slot < n_my; ++slot) {
-                const unsigned st = slot % (unsigned)S;
-                const uint32_t ph = (slot / (unsigned)S) & 1u;
                 if (!mbar_wait(sm.full + 8u * st, ph, sm.abort_flag)) break;
                 const TileDesc d = sm.desc[st];
                 unsigned char *A = sm.stage0 + (size_t)st * P.stage_bytes;
@@ -751,11 +758,11 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                 // and every compute warp has moved past it
                 bulk_wait_read_n(P.store_lag);
                 if (slot >= (unsigned)P.store_lag) {
-                    const unsigned old = slot - (unsigned)P.store_lag;
-                    const unsigned st2 = old % (unsigned)S;
-                    if (kCompute && !mbar_wait(sm.ready + 8u * st2, (old / (unsigned)S) & 1u, sm.abort_flag)) break;
+                    if (kCompute && !mbar_wait(sm.ready + 8u * st2, ph2, sm.abort_flag)) break;
                     mbar_arrive(sm.empty + 8u * st2);
+                    if (++st2 == (unsigned)S) { st2 = 0; ph2 ^= 1u; }
                 }
+                if (++st == (unsigned)S) { st = 0; ph ^= 1u; }
             }
             bulk_wait_read<0>();
             for (unsigned slot = done > (unsigned)P.store_lag ? done - (unsigned)P.store_lag : 0u; slot < done; ++slot)
@@ -769,9 +776,11 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
         const int ct = (tid - 32) % (int)kGT;
         RotCoef rc;
         rc.rope = -1; rc.col = 0xffffffffu;
+        // the rotation table is written by the kernel launched just before this one; only these warps read it
+        if (OP == OP_COMPOSE) dependency_wait();
+        unsigned st = (unsigned)group;                        // S is a multiple of kGroups: st wraps exactly at S
+        uint32_t ph = 0;
         for (unsigned slot = (unsigned)group; slot < n_my; slot += (unsigned)kGroups) {
-            const unsigned st = slot % (unsigned)S;
-            const uint32_t ph = (slot / (unsigned)S) & 1u;
             if (!mbar_wait(sm.full + 8u * st, ph, sm.abort_flag)) break;
             const unsigned n = sm.desc[st].n;
             const unsigned flags = sm.desc[st].flags;
@@ -822,6 +831,8 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
             if (computed) fence_async_smem();
             __syncwarp();
             if (lane == 0) mbar_arrive(sm.ready + 8u * st);
+            st += (unsigned)kGroups;
+            if (st >= (unsigned)S) { st -= (unsigned)S; ph ^= 1u; }
         }
     }
     __syncthreads();
@@ -852,6 +863,7 @@ struct RopeInline { RopeParam p[kInlineOps]; };
 __global__ void kdn_rope_table_kernel(const RopeParam *params, const __grid_constant__ RopeInline inl, int n_rows, int D,
                                       float2 *table)
 {
+    release_dependents();                                  // the compose kernel may set up and start its loads now
     if (!params) params = inl.p;                           // few rows: passed as kernel parameters
     const int half = D >> 1;
     const long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x;
