@@ -320,9 +320,9 @@ def run_gpu(args) -> None:
     op_bytes = {n: op_tokens[n] * E * bytes_per_elem(INT8 if n.endswith("int8") else RAW) for n in names}
     step_bytes = float(sum(op_bytes.values()))
     reload_tokens = sum(op_tokens[n] for n in names if not n.startswith("store"))
-    kernel_of = {"store_raw": "kdn_store_kernel<0>", "retrieve_raw": "kdn_retrieve_kernel<0>",
-                 "compose_raw": "kdn_compose_kernel<2>", "store_int8": "kdn_store_kernel<2>",
-                 "retrieve_int8": "kdn_retrieve_kernel<2>", "compose_int8": "kdn_compose_kernel<3>"}
+    kernel_of = {"store_raw": "kdn_store_kernel<0, 4>", "retrieve_raw": "kdn_retrieve_kernel<0, 4>",
+                 "compose_raw": "kdn_compose_kernel<1, 4>", "store_int8": "kdn_store_kernel<2, 4>",
+                 "retrieve_int8": "kdn_retrieve_kernel<2, 4>", "compose_int8": "kdn_compose_kernel<3, 4>"}
 
     def step(sets, events=None, kinds=("store", "retrieve", "compose")):
         i = 0

@@ -185,7 +185,7 @@ Shape default_shape(int OP, bool any_coded, bool any_rot)
 {
     if (!any_coded && !any_rot) return Shape{ 32768, 4, 1, 0, 2 };
     if (OP != OP_COMPOSE || !any_rot) return Shape{ 8192, 6, 3, 2, 2 };
-    if (!any_coded) return Shape{ 8192, 6, 2, 2, 2 };
+    if (!any_coded) return Shape{ 16384, 4, 2, 1, 2 };
     return Shape{ 16384, 9, 1, 3, 2 };
 }
 
@@ -254,7 +254,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
         tile_elems = row_elems;
         if (!any_coded && !any_rot) def = Shape{ 0, 4, 8, 0, 1 };
         else if (OP == OP_STORE) def = Shape{ 0, 8, 8, 2, 2, 1 };      // two single-warp groups: a row is one warp's work
-        else def = Shape{ 0, 8, 6, 1, 2 };
+        else def = Shape{ 0, 8, 6, 2, 1, 1 };
     }
     const unsigned tpb = (unsigned)((block_elems + tile_elems - 1) / tile_elems);
 
@@ -339,6 +339,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     lp.off_b = a_bytes;
     lp.off_s = a_bytes + b_bytes;
     lp.store_lag = lag;
+    lp.reload_first = (!compute && tile_elems * 2u >= 8192u) ? 1 : 0;
 
     unsigned long long want = (unsigned long long)ctx->sm_count * (unsigned)ctas_per_sm;
     const unsigned grid = (unsigned)(tiles < want ? tiles : want);
