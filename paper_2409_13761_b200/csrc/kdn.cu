@@ -186,7 +186,7 @@ Shape default_shape(int OP, bool any_coded, bool any_rot)
     if (!any_coded && !any_rot) return Shape{ 32768, 4, 1, 0, 2 };
     if (OP != OP_COMPOSE || !any_rot) return Shape{ 8192, 6, 3, 2, 2 };
     if (!any_coded) return Shape{ 16384, 4, 2, 1, 2 };
-    return Shape{ 16384, 9, 1, 3, 2 };
+    return Shape{ 8192, 4, 4, 1, 1 };
 }
 
 // Pipeline slots: at least lag + 2, a multiple of the compute groups (a slot must always belong to the

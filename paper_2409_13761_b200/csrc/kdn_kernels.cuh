@@ -341,7 +341,7 @@ __device__ __forceinline__ void quantise_tile(const unsigned char *A, unsigned c
         // the two IEEE divides of the group are shared by its two lanes: the even lane forms a / qmax, the odd
         // lane qmax / a, and one shuffle swaps them
         const bool odd = (lane & 1u) != 0u;
-        const float mine = odd ? __fdiv_rn(qmax, a) : __fdiv_rn(a, qmax);
+        const float mine = __fdiv_rn(odd ? qmax : a, odd ? a : qmax);      // one divide per lane, operands selected first
         const float other = __shfl_xor_sync(0xffffffffu, mine, 1);
         float scale = odd ? other : mine;
         const bool ok = scale >= 1.17549435e-38f;         // smallest normal fp32; false for NaN too

@@ -189,3 +189,47 @@ def test_70b_batch_of_32_requests_each_retrieving_4_chunks_of_2048_tokens():
         dev.close()
         del dev
         torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("run_blocks", [None, 8, 1], ids=["contiguous", "runs_of_8", "fragmented"])
+def test_8b_sweep_points_block_size_32_longest_and_shortest_chunks(run_blocks):
+    """Two ends of the chunk-length sweep on the 8B shape with block_size 32: one 8192-token chunk and a batch of forty
+    128-token chunks, at three block-table fragmentations, stored and retrieved in the batched calls the sweep times."""
+    need_gib(20)
+    shape = synth.LLAMA3_8B.with_(block_size=32, n_blocks=2048)
+    dev = Device(shape)
+    try:
+        K, bs = dev.K, shape.block_size
+        layers = [0, 13, shape.n_layers - 1]
+        for T, n_req in ((8192, 1), (128, 40)):
+            nb = T // bs
+            r = nb if run_blocks is None else run_blocks
+            src = synth.make_table(n_req * nb, shape.n_blocks, r, synth.SEED_TABLES).reshape(n_req, nb)
+            dst = synth.make_table(n_req * nb, shape.n_blocks, r, synth.SEED_TABLES + 1, exclude=src.reshape(-1)).reshape(n_req, nb)
+            d_src, d_dst = dev.table(src.reshape(-1)), dev.table(dst.reshape(-1))
+            for codec in (RAW, INT8):
+                cb = K.kdn_chunk_bytes(dev.desc, T, codec)
+                big = torch.empty(n_req * cb, dtype=torch.uint8, device=dev.dev)
+                st = [K.XferOp(d_src.data_ptr() + i * nb * 4, nb, 0, K.Chunk(big.data_ptr() + i * cb, cb, T, codec)) for i in range(n_req)]
+                rt = [K.XferOp(d_dst.data_ptr() + i * nb * 4, nb, 0, K.Chunk(big.data_ptr() + i * cb, cb, T, codec)) for i in range(n_req)]
+                before = block_sums(dev)
+                dev.store(st)
+                dev.retrieve(rt)
+                assert dev.sync() == 0
+                after = block_sums(dev)
+                keep = torch.ones(shape.n_blocks, dtype=torch.bool, device=dev.dev)
+                keep[torch.from_numpy(dst.reshape(-1).astype(np.int64)).to(dev.dev)] = False
+                assert torch.equal(after[:, keep], before[:, keep])          # only destination blocks changed
+                for i in (0, n_req - 1):
+                    sp = dev.pool_np(src[i], layers)
+                    want = oracle.store(sp, np.arange(nb, dtype=np.int32), 0, T, codec)
+                    got = sub_chunk(to_np(big[i * cb:(i + 1) * cb]), shape.n_layers, T, shape.n_kv_heads, shape.head_dim, codec, layers)
+                    assert np.array_equal(got, want), (T, codec, i)
+                    ref = np.zeros_like(sp)
+                    oracle.retrieve(ref, np.arange(nb, dtype=np.int32), 0, T, codec, want)
+                    assert np.array_equal(dev.pool_np(dst[i], layers), ref), (T, codec, i)
+                del big
+    finally:
+        dev.close()
+        del dev
+        torch.cuda.empty_cache()
