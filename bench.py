@@ -179,8 +179,8 @@ class ClockSampler:
 # DRAM bytes (read + write) per launch from the committed ncu capture of a reduced case (8 chunks per
 # store/retrieve launch, 2 parts per compose launch; profiles/ncu_full_small_case_llama3_8b.md), scaled by the
 # units a bench launch processes.  Valid only for the kernel source the capture was taken from.
-NCU_KERNEL_SHA = "b9e8cd645fa7f423"
-NCU_SMALL_CASE_BYTES = {"store_raw": (536.920576e6 + 486.232576e6, 8), "retrieve_raw": (536.900608e6 + 490.784768e6, 8), "compose_raw": (268.483840e6 + 223.139840e6, 2), "store_int8": (536.966400e6 + 252.484608e6, 8), "retrieve_int8": (285.251840e6 + 483.219200e6, 8), "compose_int8": (142.698240e6 + 213.456640e6, 2)}
+NCU_KERNEL_SHA = "789bdf43c1b0116f"
+NCU_SMALL_CASE_BYTES = {"store_raw": (536.900608e6 + 485.395712e6, 8), "retrieve_raw": (536.921344e6 + 490.137088e6, 8), "compose_raw": (268.481280e6 + 221.714944e6, 2), "store_int8": (536.994048e6 + 249.219072e6, 8), "retrieve_int8": (285.334784e6 + 482.757888e6, 8), "compose_int8": (142.652160e6 + 214.158848e6, 2)}
 
 
 def measured_traffic(op: str, units: float):
