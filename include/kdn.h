@@ -4,9 +4,9 @@
  *
  * A KDN keeps precomputed KV caches apart from the serving engine and hands
  * them back on demand (paper Sec. 3.1: storage, delivery and blending
- * modules).  The engine talks to it through two calls, "store the KV cache"
- * and "retrieve the KV cache" (Sec. 3.2, "Interface with LLM serving
- * engines"), and a retrieved context may be put together from several stored
+ * modules).  The engine talks to it through two calls, one that stores a
+ * KV cache and one that retrieves it (Sec. 3.2, the paragraph on the interface
+ * with serving engines), and a retrieved context may be put together from several stored
  * pieces (Sec. 3.1 blending module; Sec. 3.2 "KV-cache blending").  This
  * library is that path between an engine's paged GPU KV pool and compact
  * per-chunk buffers:
@@ -37,7 +37,7 @@
  *   else code = round_half_even(x * (127/a)) in fp32, in [-127, 127];
  *   decode = bf16_round_nearest_even((float)code * scale).
  * int4 coding: the same with 7 in place of 127 (scale = a/7, code in [-7, 7]); a stronger codec towards the
- *   "over 10x" footprint reduction Sec. 3.2 ("KV-cache delivery") cites.
+ *   more-than-tenfold footprint reduction Sec. 3.2 ("KV-cache delivery") reports for combined techniques.
  * Key re-rotation in kdn_compose: the stored keys of a part carry rotary
  *   position embedding for positions base_pos + t; placing the part at
  *   dst_pos rotates each pair (k[i], k[i + D/2]) of every head by
@@ -80,7 +80,8 @@ typedef enum {
     KDN_E_NOMEM = 7,        /* context scratch could not be allocated */
     KDN_E_TIMEOUT = 8,      /* a bounded wait inside a kernel gave up (device) */
     KDN_E_NOTFOUND = 9,     /* kdn_index_get / kdn_index_remove: no chunk under this key */
-    KDN_E_CHECKSUM = 10     /* kdn_header_check: the payload does not match the header's checksum */
+    KDN_E_CHECKSUM = 10,    /* kdn_header_check: the payload does not match the header's checksum */
+    KDN_E_IO = 11           /* kdn_store_file / kdn_retrieve_file: a read or write of the chunk file failed or came up short */
 } kdn_status;
 
 typedef enum { KDN_CODEC_RAW_BF16 = 0, KDN_CODEC_INT8_G64 = 1, KDN_CODEC_INT4_G64 = 2 } kdn_codec;
@@ -222,6 +223,31 @@ kdn_status kdn_retrieve(kdn_ctx *ctx, int pool_id, const kdn_xfer_op *ops, int n
 kdn_status kdn_retrieve_layerwise(kdn_ctx *ctx, int pool_id, const kdn_xfer_op *ops, int n_ops, int layers_per_step,
                                   void *cuda_stream, void *side_stream, void *const *layer_ready);
 
+/* A chunk kept in a file (Sec. 3: once KV caches move out of GPU and CPU memory to disks or remote servers, the
+ * bandwidth of loading them back becomes the constraint; Sec. 3.1 delivery module).  The chunk's bytes, in the
+ * ordinary chunk layout, occupy [file_offset, file_offset + op.chunk.bytes) of the open file descriptor fd (a
+ * regular file, or anything pread / pwrite work on).  op.chunk.data and op.chunk.mem are ignored; every other
+ * field means what it means in kdn_xfer_op. */
+typedef struct {
+    kdn_xfer_op op;
+    int32_t     fd;
+    int32_t     reserved;   /* 0 */
+    int64_t     file_offset;
+} kdn_file_op;
+
+/* kdn_retrieve / kdn_store for file-backed chunks.  The bytes travel layer range by layer range through two
+ * page-locked bounce buffers (as large as the staging slabs, allocated on first use) and the staging slabs: while
+ * the calling thread reads the next range from the file, the previous one crosses the host link on side_stream and
+ * the one before that is decoded and scattered on cuda_stream.  The calling thread does the file I/O, so these
+ * calls take as long as the I/O does: kdn_retrieve_file returns when the last range has been read and enqueued (the
+ * GPU may still be working; order later work after it on cuda_stream), kdn_store_file returns when the files hold
+ * the chunks.  A failed or short read or write returns KDN_E_IO; ranges already enqueued still run.  Results are
+ * exactly those of kdn_retrieve / kdn_store on a memory-resident copy of the same bytes. */
+kdn_status kdn_retrieve_file(kdn_ctx *ctx, int pool_id, const kdn_file_op *ops, int n_ops,
+                             void *cuda_stream, void *side_stream);
+kdn_status kdn_store_file(kdn_ctx *ctx, int pool_id, const kdn_file_op *ops, int n_ops,
+                          void *cuda_stream, void *side_stream);
+
 /* Sec. 3.1 blending module: compose every request's parts into its blocks; keys of parts whose
  * part_dst_pos differs from base_pos are re-rotated (see the top of this file).  A part with equal
  * positions, and every value plane, is written exactly as kdn_retrieve writes it. */
@@ -297,8 +323,8 @@ kdn_status kdn_set_staging_bytes(kdn_ctx *ctx, size_t bytes_per_slab);
 uint64_t kdn_launch_count(const kdn_ctx *ctx);
 
 /* ------------------------------------------------------------------------------------------------
- * Storage-module shell (Sec. 3.1: the storage module "stores the KV caches keyed by various texts"; Sec. 3.2:
- * the engine stores a KV cache "with the associated text" and retrieves it "using some text").  The paper fixes
+ * Storage-module shell (Sec. 3.1: the storage module keeps KV caches under keys derived from their texts; Sec. 3.2:
+ * the engine hands over a KV cache together with its text and later asks for it by text).  The paper fixes
  * neither a key, a header nor an eviction rule; these are this library's choices.  The shell owns no chunk
  * memory: it maps keys to the caller's chunk descriptors and says which ones to drop. */
 

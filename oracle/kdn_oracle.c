@@ -54,8 +54,8 @@
  *                    select-list: compose may deliver only some tokens of a part: for each listed chunk token c
  *                    (strictly increasing) it writes position dst_pos + c and leaves the other positions alone.
  *
- *   R8  storage shell (Sec. 3.1 storage module: "stores the KV caches keyed by various texts"; Sec. 3.2 interface:
- *                    store "with the associated text", retrieve "using some text".)  key = FNV-1a 64-bit hash of the
+ *   R8  storage shell (Sec. 3.1 storage module: KV caches kept under keys derived from their texts; Sec. 3.2
+ *                    interface: a cache is stored together with its text and asked for by text.)  key = FNV-1a 64-bit hash of the
  *                    text's token ids taken as little-endian 32-bit integers; payload checksum =
  *                    sum_i ((w_i XOR 0x9E3779B9) * ((2 i + 1) mod 2^32)) mod 2^64 over the payload's little-endian
  *                    32-bit words w_i.  Neither is prescribed by the paper.
@@ -356,7 +356,7 @@ static uint16_t decoded(const uint8_t *chunk, size_t elems, int codec, size_t c)
 
 /* ------------------------------------------------------------- retrieve -- */
 
-/* Sec. 3.2 call (ii) with Sec. 3.1's "decompresses them in GPU": scatter a
+/* Sec. 3.2 call (ii) with Sec. 3.1's decompression on the GPU: scatter a
  * chunk back into the pool blocks the table names, decoding int8 (R5).  Only
  * the T addressed token slots are written. */
 int kdn_oracle_retrieve_sparse(uint16_t *pool, int L, int H, int D, int bs, int64_t nb,

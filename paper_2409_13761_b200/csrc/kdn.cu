@@ -5,6 +5,7 @@
 #include "kdn.h"
 #include "kdn_kernels.cuh"
 
+#include <cerrno>
 #include <cstdio>
 #include <cstring>
 #include <functional>
@@ -13,6 +14,8 @@
 #include <new>
 #include <utility>
 #include <vector>
+
+#include <unistd.h>
 
 using namespace kdn;
 
@@ -46,12 +49,16 @@ struct HostOp {                             // one op (or one layer range of one
     DevOp op;
     bool rotate = false;
     RopeParam rp{};
+    int fd = -1;                            // >= 0: the chunk's bytes live in this file, from file_off on
+    long long file_off = 0;
 };
 
 struct Piece {                              // host <-> slab copies belonging to a staged op
-    unsigned char *host;
+    unsigned char *host;                    // page-locked host memory, or nullptr: the piece lives in a file
     size_t slab_off;
     size_t bytes;
+    int fd;
+    long long file_off;
 };
 
 }  // namespace
@@ -71,6 +78,10 @@ struct kdn_ctx {
     cudaEvent_t slab_free[2] = { nullptr, nullptr };   // last consumer of the slab has finished
     cudaEvent_t slab_ready[2] = { nullptr, nullptr };  // the slab's producer has finished
     unsigned slab_next = 0;
+    unsigned char *bounce[2] = { nullptr, nullptr };   // page-locked mirrors of the slabs for file-backed chunks
+    cudaEvent_t bounce_done[2] = { nullptr, nullptr }; // the copies between bounce[i] and slab[i] have finished
+    bool bounce_busy[2] = { false, false };
+    std::vector<Piece> pending_writes[2];              // file pieces whose bytes are on their way into bounce[i]
     uint64_t launches = 0;
     kdn_tuning tuning{};
 };
@@ -135,6 +146,50 @@ kdn_status ensure_slabs(kdn_ctx *ctx)
         if (!ctx->slab_ready[i]) KDN_CUDA(cudaEventCreateWithFlags(&ctx->slab_ready[i], cudaEventDisableTiming));
     }
     return KDN_OK;
+}
+
+kdn_status ensure_bounce(kdn_ctx *ctx)
+{
+    for (int i = 0; i < 2; ++i) {
+        if (!ctx->bounce[i]) KDN_CUDA(cudaMallocHost((void **)&ctx->bounce[i], ctx->slab_bytes));
+        if (!ctx->bounce_done[i]) KDN_CUDA(cudaEventCreateWithFlags(&ctx->bounce_done[i], cudaEventDisableTiming));
+    }
+    return KDN_OK;
+}
+
+// Whole-range pread / pwrite (short transfers are continued, EINTR retried).
+bool read_fully(int fd, unsigned char *dst, size_t bytes, long long off)
+{
+    while (bytes) {
+        const ssize_t n = pread(fd, dst, bytes, (off_t)off);
+        if (n < 0 && errno == EINTR) continue;
+        if (n <= 0) return false;                            // error, or the file ends before the chunk does
+        dst += n; off += n; bytes -= (size_t)n;
+    }
+    return true;
+}
+bool write_fully(int fd, const unsigned char *src, size_t bytes, long long off)
+{
+    while (bytes) {
+        const ssize_t n = pwrite(fd, src, bytes, (off_t)off);
+        if (n < 0 && errno == EINTR) continue;
+        if (n <= 0) return false;
+        src += n; off += n; bytes -= (size_t)n;
+    }
+    return true;
+}
+
+// Store path: once the slab -> bounce copies of slab `s` have finished, write their pieces to the files.
+kdn_status drain_writes(kdn_ctx *ctx, unsigned s)
+{
+    if (ctx->pending_writes[s].empty()) return KDN_OK;
+    KDN_CUDA(cudaEventSynchronize(ctx->bounce_done[s]));
+    ctx->bounce_busy[s] = false;
+    bool ok = true;
+    for (const Piece &p : ctx->pending_writes[s])
+        ok = write_fully(p.fd, ctx->bounce[s] + p.slab_off, p.bytes, p.file_off) && ok;
+    ctx->pending_writes[s].clear();
+    return ok ? KDN_OK : KDN_E_IO;
 }
 
 // Largest dynamic shared-memory size already granted to each kernel on each device (setting the attribute on
@@ -406,21 +461,49 @@ kdn_status run_staged(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<
     auto flush = [&]() -> kdn_status {
         if (batch.empty()) return KDN_OK;
         const unsigned s = ctx->slab_next++ & 1u;
+        bool any_file = false;
+        for (const Piece &p : pieces) any_file |= p.host == nullptr;
+        if (any_file) {
+            kdn_status r = ensure_bounce(ctx);
+            if (r != KDN_OK) return r;
+        }
         if (OP == OP_STORE) {
+            // bounce[s] still holds file pieces of the store before last: put them into their files first
+            kdn_status r = drain_writes(ctx, s);
+            if (r != KDN_OK) return r;
             KDN_CUDA(cudaStreamWaitEvent(stream, ctx->slab_free[s], 0));
-            kdn_status r = launch_all(ctx, pool, OP, batch, stream);
+            r = launch_all(ctx, pool, OP, batch, stream);
             if (r != KDN_OK) return r;
             KDN_CUDA(cudaEventRecord(ctx->slab_ready[s], stream));
             KDN_CUDA(cudaStreamWaitEvent(side, ctx->slab_ready[s], 0));
             for (const Piece &p : pieces)
-                KDN_CUDA(cudaMemcpyAsync(p.host, ctx->slab[s] + p.slab_off, p.bytes, cudaMemcpyDeviceToHost, side));
+                KDN_CUDA(cudaMemcpyAsync(p.host ? p.host : ctx->bounce[s] + p.slab_off, ctx->slab[s] + p.slab_off, p.bytes,
+                                         cudaMemcpyDeviceToHost, side));
             KDN_CUDA(cudaEventRecord(ctx->slab_free[s], side));
+            if (any_file) {
+                KDN_CUDA(cudaEventRecord(ctx->bounce_done[s], side));
+                ctx->bounce_busy[s] = true;
+                for (const Piece &p : pieces)
+                    if (!p.host) ctx->pending_writes[s].push_back(p);
+            }
             r = between();                                       // device-resident work runs while the slab drains
             if (r != KDN_OK) return r;
         } else {
+            if (any_file) {
+                // the host reads the file pieces into bounce[s] while the GPU works on the other slab
+                if (ctx->bounce_busy[s]) KDN_CUDA(cudaEventSynchronize(ctx->bounce_done[s]));
+                ctx->bounce_busy[s] = false;
+                for (const Piece &p : pieces)
+                    if (!p.host && !read_fully(p.fd, ctx->bounce[s] + p.slab_off, p.bytes, p.file_off)) return KDN_E_IO;
+            }
             KDN_CUDA(cudaStreamWaitEvent(side, ctx->slab_free[s], 0));
             for (const Piece &p : pieces)
-                KDN_CUDA(cudaMemcpyAsync(ctx->slab[s] + p.slab_off, p.host, p.bytes, cudaMemcpyHostToDevice, side));
+                KDN_CUDA(cudaMemcpyAsync(ctx->slab[s] + p.slab_off, p.host ? p.host : ctx->bounce[s] + p.slab_off, p.bytes,
+                                         cudaMemcpyHostToDevice, side));
+            if (any_file) {
+                KDN_CUDA(cudaEventRecord(ctx->bounce_done[s], side));
+                ctx->bounce_busy[s] = true;
+            }
             KDN_CUDA(cudaEventRecord(ctx->slab_ready[s], side));
             kdn_status r = between();                            // device-resident work runs while the slab fills
             if (r != KDN_OK) return r;
@@ -466,14 +549,30 @@ kdn_status run_staged(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<
             const unsigned s = ctx->slab_next & 1u;
             sub.op.data = ctx->slab[s] + base;
             sub.op.scales = sbytes ? ctx->slab[s] + base + cbytes : nullptr;
-            pieces.push_back(Piece{ host + (size_t)l * codes_per_layer, base, cbytes });
-            if (sbytes) pieces.push_back(Piece{ host + host_codes_total + (size_t)l * scales_per_layer, base + cbytes, sbytes });
+            if (h.fd >= 0) {
+                pieces.push_back(Piece{ nullptr, base, cbytes, h.fd, h.file_off + (long long)((size_t)l * codes_per_layer) });
+                if (sbytes)
+                    pieces.push_back(Piece{ nullptr, base + cbytes, sbytes, h.fd,
+                                            h.file_off + (long long)(host_codes_total + (size_t)l * scales_per_layer) });
+            } else {
+                pieces.push_back(Piece{ host + (size_t)l * codes_per_layer, base, cbytes, -1, 0 });
+                if (sbytes)
+                    pieces.push_back(Piece{ host + host_codes_total + (size_t)l * scales_per_layer, base + cbytes, sbytes, -1, 0 });
+            }
             batch.push_back(sub);
             used = (base + cbytes + sbytes + 255) & ~(size_t)255;
             l += nl;
         }
     }
-    return flush();
+    st = flush();
+    if (OP == OP_STORE) {
+        // a store into files returns once the files hold the chunks
+        for (unsigned s = 0; s < 2; ++s) {
+            const kdn_status w = drain_writes(ctx, s);
+            if (st == KDN_OK) st = w;
+        }
+    }
+    return st;
 }
 
 // Bytes of the chunk side of one op (what crosses the host link when the chunk is host resident).
@@ -711,6 +810,10 @@ void kdn_destroy(kdn_ctx *ctx)
         if (ctx->slab_free[i]) cudaEventDestroy(ctx->slab_free[i]);
         if (ctx->slab_ready[i]) cudaEventDestroy(ctx->slab_ready[i]);
     }
+    for (int i = 0; i < 2; ++i) {
+        if (ctx->bounce[i]) cudaFreeHost(ctx->bounce[i]);
+        if (ctx->bounce_done[i]) cudaEventDestroy(ctx->bounce_done[i]);
+    }
     if (ctx->own_side) cudaStreamDestroy(ctx->own_side);
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
@@ -751,6 +854,50 @@ kdn_status kdn_store(kdn_ctx *ctx, int pool_id, const kdn_xfer_op *ops, int n_op
 kdn_status kdn_retrieve(kdn_ctx *ctx, int pool_id, const kdn_xfer_op *ops, int n_ops, void *cuda_stream, void *side_stream)
 {
     return xfer(ctx, pool_id, OP_RETRIEVE, ops, n_ops, cuda_stream, side_stream);
+}
+
+static kdn_status xfer_file(kdn_ctx *ctx, int pool_id, int OP, const kdn_file_op *ops, int n_ops, void *cuda_stream, void *side_stream)
+{
+    if (!ctx || pool_id < 0 || (size_t)pool_id >= ctx->pools.size()) return KDN_E_INVAL;
+    if (n_ops < 0 || (n_ops > 0 && !ops)) return KDN_E_INVAL;
+    const Pool &pool = ctx->pools[(size_t)pool_id];
+    const kdn_pool_desc shape = shape_of(pool);
+    kdn_status st = check_shape(&shape);
+    if (st != KDN_OK) return st;
+    for (int i = 0; i < n_ops; ++i) {
+        const kdn_xfer_op &o = ops[i].op;
+        kdn_chunk c = o.chunk;
+        c.data = (void *)(uintptr_t)16;                      // a file-backed chunk has no address to check
+        c.mem = KDN_MEM_PINNED_HOST;
+        st = check_chunk(&shape, &c);
+        if (st != KDN_OK) return st;
+        st = check_range(&shape, o.block_table, o.n_table_blocks, o.token_offset, o.chunk.n_tokens);
+        if (st != KDN_OK) return st;
+        if (ops[i].fd < 0 || ops[i].file_offset < 0) return KDN_E_INVAL;
+    }
+    if (cudaSetDevice(ctx->device) != cudaSuccess) return KDN_E_CUDA;
+    std::vector<HostOp> dev_ops, host_ops;
+    for (int i = 0; i < n_ops; ++i) {
+        const kdn_xfer_op &o = ops[i].op;
+        if (o.chunk.n_tokens == 0) continue;
+        kdn_chunk c = o.chunk;
+        c.data = nullptr;
+        HostOp h = make_host_op(pool, o.block_table, o.n_table_blocks, o.token_offset, c);
+        h.fd = ops[i].fd;
+        h.file_off = ops[i].file_offset;
+        host_ops.push_back(h);
+    }
+    return run_ops(ctx, pool_id, OP, dev_ops, host_ops, cuda_stream, side_stream);
+}
+
+kdn_status kdn_store_file(kdn_ctx *ctx, int pool_id, const kdn_file_op *ops, int n_ops, void *cuda_stream, void *side_stream)
+{
+    return xfer_file(ctx, pool_id, OP_STORE, ops, n_ops, cuda_stream, side_stream);
+}
+
+kdn_status kdn_retrieve_file(kdn_ctx *ctx, int pool_id, const kdn_file_op *ops, int n_ops, void *cuda_stream, void *side_stream)
+{
+    return xfer_file(ctx, pool_id, OP_RETRIEVE, ops, n_ops, cuda_stream, side_stream);
 }
 
 kdn_status kdn_retrieve_layerwise(kdn_ctx *ctx, int pool_id, const kdn_xfer_op *ops, int n_ops, int layers_per_step,
@@ -886,6 +1033,9 @@ kdn_status kdn_set_staging_bytes(kdn_ctx *ctx, size_t bytes_per_slab)
     for (int i = 0; i < 2; ++i) {
         if (ctx->slab[i]) KDN_CUDA(cudaFree(ctx->slab[i]));
         ctx->slab[i] = nullptr;
+        if (ctx->bounce[i]) KDN_CUDA(cudaFreeHost(ctx->bounce[i]));
+        ctx->bounce[i] = nullptr;
+        ctx->bounce_busy[i] = false;
     }
     ctx->slab_bytes = bytes_per_slab & ~(size_t)255;
     return KDN_OK;
@@ -907,6 +1057,7 @@ const char *kdn_strerror(kdn_status status)
     case KDN_E_TIMEOUT: return "a bounded wait inside a kernel expired";
     case KDN_E_NOTFOUND: return "no chunk under this key";
     case KDN_E_CHECKSUM: return "payload does not match the header's checksum";
+    case KDN_E_IO: return "reading or writing a chunk file failed";
     }
     return "unknown status";
 }

@@ -1,5 +1,5 @@
-// Storage-module shell of libkdn (paper Sec. 3.1: the storage module keeps KV caches "keyed by various texts";
-// Sec. 3.2: the engine stores a KV cache "with the associated text" and retrieves it "using some text").
+// Storage-module shell of libkdn (paper Sec. 3.1: the storage module keeps KV caches under keys derived from
+// their texts; Sec. 3.2: the engine hands over a KV cache together with its text and later asks for it by text).
 // Host side: key hash, self-describing chunk header, and an index from key to chunk with least-recently-used
 // eviction under a byte budget.  Device side: one kernel, the payload checksum.
 #include "kdn.h"

@@ -14,14 +14,14 @@ from typing import List, Optional, Sequence
 from . import build as _build
 
 KDN_OK, KDN_E_INVAL, KDN_E_SHAPE, KDN_E_ALIGN, KDN_E_RANGE, KDN_E_UNSUPPORTED, KDN_E_CUDA, KDN_E_NOMEM, \
-    KDN_E_TIMEOUT, KDN_E_NOTFOUND, KDN_E_CHECKSUM = range(11)
+    KDN_E_TIMEOUT, KDN_E_NOTFOUND, KDN_E_CHECKSUM, KDN_E_IO = range(12)
 KDN_CODEC_RAW_BF16, KDN_CODEC_INT8_G64, KDN_CODEC_INT4_G64 = 0, 1, 2
 KDN_MEM_DEVICE, KDN_MEM_PINNED_HOST = 0, 1
 
 EXPORTS = ["kdn_create", "kdn_destroy", "kdn_pool_register", "kdn_chunk_bytes", "kdn_validate_xfer",
            "kdn_validate_compose", "kdn_store", "kdn_retrieve", "kdn_compose", "kdn_status_sync",
            "kdn_set_tuning", "kdn_set_staging_bytes", "kdn_launch_count", "kdn_strerror",
-           "kdn_compose_static", "kdn_retrieve_layerwise",
+           "kdn_compose_static", "kdn_retrieve_layerwise", "kdn_store_file", "kdn_retrieve_file",
            "kdn_store_sparse", "kdn_retrieve_sparse", "kdn_compose_select",
            "kdn_key_hash", "kdn_checksum", "kdn_header_fill", "kdn_header_check", "kdn_index_create", "kdn_index_destroy",
            "kdn_index_put", "kdn_index_get", "kdn_index_remove", "kdn_index_stats"]
@@ -51,6 +51,10 @@ class kdn_compose_req(C.Structure):
 
 class kdn_sparse_op(C.Structure):
     _fields_ = [("op", kdn_xfer_op), ("keep", C.c_void_p)]
+
+
+class kdn_file_op(C.Structure):
+    _fields_ = [("op", kdn_xfer_op), ("fd", C.c_int32), ("reserved", C.c_int32), ("file_offset", C.c_int64)]
 
 
 class kdn_select(C.Structure):
@@ -106,6 +110,10 @@ def _load() -> C.CDLL:
         fn = getattr(lib, name)
         fn.restype = i32
         fn.argtypes = [vp, i32, C.POINTER(kdn_sparse_op), i32, vp, vp]
+    for name in ("kdn_store_file", "kdn_retrieve_file"):
+        fn = getattr(lib, name)
+        fn.restype = i32
+        fn.argtypes = [vp, i32, C.POINTER(kdn_file_op), i32, vp, vp]
     lib.kdn_compose_select.restype = i32
     lib.kdn_compose_select.argtypes = [vp, i32, C.POINTER(kdn_compose_req), C.POINTER(kdn_select), i32, vp, vp]
     lib.kdn_compose.restype = i32
@@ -292,6 +300,24 @@ def kdn_store_sparse(ctx, pool_id: int, ops: Sequence[XferOp], keeps: Sequence[i
 
 def kdn_retrieve_sparse(ctx, pool_id: int, ops: Sequence[XferOp], keeps: Sequence[int], stream: int = 0, side_stream: int = 0) -> None:
     _check(lib.kdn_retrieve_sparse(ctx, pool_id, sparse_array(ops, keeps), len(ops), stream, side_stream), "kdn_retrieve_sparse")
+
+
+def file_array(ops: Sequence[XferOp], fds: Sequence[int], file_offsets: Sequence[int]):
+    arr = (kdn_file_op * max(1, len(ops)))()
+    for i, (o, fd, off) in enumerate(zip(ops, fds, file_offsets)):
+        arr[i] = kdn_file_op(kdn_xfer_op(o.block_table, o.n_table_blocks, 0, o.token_offset, o.chunk.c()), int(fd), 0, int(off))
+    return arr
+
+
+def kdn_store_file(ctx, pool_id: int, ops: Sequence[XferOp], fds: Sequence[int], file_offsets: Sequence[int],
+                   stream: int = 0, side_stream: int = 0) -> None:
+    """ops[i].chunk describes the chunk (its data address is ignored); its bytes go to fds[i] at file_offsets[i]."""
+    _check(lib.kdn_store_file(ctx, pool_id, file_array(ops, fds, file_offsets), len(ops), stream, side_stream), "kdn_store_file")
+
+
+def kdn_retrieve_file(ctx, pool_id: int, ops: Sequence[XferOp], fds: Sequence[int], file_offsets: Sequence[int],
+                      stream: int = 0, side_stream: int = 0) -> None:
+    _check(lib.kdn_retrieve_file(ctx, pool_id, file_array(ops, fds, file_offsets), len(ops), stream, side_stream), "kdn_retrieve_file")
 
 
 def kdn_compose_select(ctx, pool_id: int, reqs: Sequence[ComposeReq], selects, stream: int = 0, side_stream: int = 0) -> None:

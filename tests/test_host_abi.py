@@ -39,8 +39,8 @@ def test_chunk_bytes_matches_oracle():
 
 
 def test_strerror_is_total():
-    seen = {K.kdn_strerror(s) for s in range(11)}
-    assert len(seen) == 11 and "unknown status" not in seen
+    seen = {K.kdn_strerror(s) for s in range(12)}
+    assert len(seen) == 12 and "unknown status" not in seen
     assert K.kdn_strerror(99) == "unknown status"
 
 
