@@ -442,10 +442,35 @@ def run_gpu(args) -> None:
         del buf
     torch.cuda.empty_cache()
 
+    # ---- file-backed chunks: a few chunks of the library written to and read back from one file (wall clock around
+    # the call plus the stream sync, since the calling thread does the file I/O; not part of `value`)
+    file_ops = {}
+    import tempfile
+    tmpdir = "/dev/shm" if os.path.isdir("/dev/shm") and os.access("/dev/shm", os.W_OK) else None
+    n_file = min(8, n_lib)
+    for codec, cname in ((RAW, "raw"), (INT8, "int8")):
+        cb = K.kdn_chunk_bytes(desc, T, codec)
+        with tempfile.NamedTemporaryFile(dir=tmpdir, prefix="kdn_bench_") as tf:
+            fd = tf.fileno()
+            st_ops = [K.XferOp(d_src.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(0, cb, T, codec)) for c in range(n_file)]
+            rt_ops = [K.XferOp(d_dst.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(0, cb, T, codec)) for c in range(n_file)]
+            offs = [c * cb for c in range(n_file)]
+            for name, fn, arg in (("store_file_" + cname, K.kdn_store_file, st_ops), ("retrieve_file_" + cname, K.kdn_retrieve_file, rt_ops)):
+                best = None
+                for _ in range(3):
+                    torch.cuda.synchronize()
+                    t0 = time.perf_counter()
+                    fn(ctx, pid, arg, [fd] * n_file, offs, s)
+                    assert K.kdn_status_sync(ctx, s) == K.KDN_OK
+                    dt = time.perf_counter() - t0
+                    best = dt if best is None else min(best, dt)
+                file_ops[name] = {"ms": best * 1e3, "file_gbs": n_file * cb / best / 1e9, "file_bytes": n_file * cb,
+                                  "where": "tmpfs" if tmpdir else "default temporary directory (page cache)"}
+
     if args.no_e2e:
         if rank == 0:
             print(json.dumps({"note": "profiling run, not a bench record", "ops_ms": op_ms,
-                              "ops_gbs": {n: op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 for n in names}, "int4": int4_ops, "sparse": sparse_ops, "shell": shell_ops}))
+                              "ops_gbs": {n: op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 for n in names}, "int4": int4_ops, "sparse": sparse_ops, "shell": shell_ops, "file": file_ops}))
         K.kdn_destroy(ctx)
         return
 
@@ -552,6 +577,7 @@ def run_gpu(args) -> None:
                        "bytes_per_step": step_bytes},
             "tokens_per_s_reloaded": world * reload_tokens / (sum(op_ms[n] for n in names if not n.startswith("store")) * 1e-3),
             "ops": ops, "ops_int4_not_in_value": int4_ops, "ops_keep_list_not_in_value": sparse_ops, "ops_shell_not_in_value": shell_ops,
+            "ops_file_not_in_value": file_ops,
             "roofline": {"bound": "hbm", "kernel": kernel_of[top], "op": top, "achieved": ops[top]["gbs"], "peak": peak,
                          "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": ops[top]["gbs"] / peak,
                          "frac_of_nominal_8000": ops[top]["gbs"] / 8000.0, "traffic": traffic},
