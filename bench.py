@@ -594,6 +594,9 @@ def run_gpu(args) -> None:
             b, t, dt = smp.run_pass()
             rec["cpu_baseline"] = {"value": b / dt / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
                                    "sample": smp.describe(1, b, dt), "tokens_per_s_reloaded": t / dt}
+            one = OracleSample(1, 128)                       # the same oracle on one core, on a smaller chunk
+            b1, t1, dt1 = one.run_pass()
+            rec["cpu_baseline"]["one_core"] = {"value": b1 / dt1 / 1e9, "unit": UNIT, "sample": one.describe(1, b1, dt1)}
         print(json.dumps(rec))
     K.kdn_destroy(ctx)
     if dist is not None:
