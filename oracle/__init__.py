@@ -55,6 +55,8 @@ def lib():
             L.kdn_oracle_bf16_to_f32.argtypes = [C.c_uint16]
             L.kdn_oracle_f32_to_bf16.restype = C.c_uint16
             L.kdn_oracle_f32_to_bf16.argtypes = [C.c_float]
+            L.kdn_oracle_f32_to_bf16_many.restype = None
+            L.kdn_oracle_f32_to_bf16_many.argtypes = [vp, vp, sz]
             L.kdn_oracle_f64_to_bf16.restype = C.c_uint16
             L.kdn_oracle_f64_to_bf16.argtypes = [f64]
             L.kdn_oracle_chunk_bytes.restype = sz
@@ -228,6 +230,13 @@ def dequant(q: int, scale) -> int:
 
 def f32_to_bf16(f) -> int:
     return int(lib().kdn_oracle_f32_to_bf16(float(np.float32(f))))
+
+
+def f32_to_bf16_many(f: np.ndarray) -> np.ndarray:
+    f = np.ascontiguousarray(f, dtype=np.float32)
+    out = np.empty(f.shape, dtype=np.uint16)
+    lib().kdn_oracle_f32_to_bf16_many(f.ctypes.data, out.ctypes.data, f.size)
+    return out
 
 
 def f64_to_bf16(x: float) -> int:

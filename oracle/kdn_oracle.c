@@ -106,6 +106,12 @@ uint16_t kdn_oracle_f32_to_bf16(float f)
     return (uint16_t)keep;
 }
 
+/* The same conversion for n values (so a test can sweep every fp32 bit pattern). */
+void kdn_oracle_f32_to_bf16_many(const float *f, uint16_t *out, size_t n)
+{
+    for (size_t i = 0; i < n; ++i) out[i] = kdn_oracle_f32_to_bf16(f[i]);
+}
+
 /* fp64 -> bf16, round to nearest even in ONE rounding (no trip through fp32):
  * take the bf16 at or below |x| and its upper neighbour, keep the nearer one,
  * the even one on a tie. */

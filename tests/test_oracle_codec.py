@@ -201,6 +201,27 @@ def test_f32_to_bf16_against_torch_on_rounding_classes():
         assert oracle.f32_to_bf16(f[i]) == want[i], hex(int(u[i]))
 
 
+def test_f32_to_bf16_against_torch_on_every_bit_pattern():
+    """All 2^32 fp32 bit patterns: the oracle's integer add-and-compare rounding against torch's conversion
+    (NaNs: both must give a NaN; every other pattern must match bit for bit)."""
+    from concurrent.futures import ThreadPoolExecutor
+    span = 1 << 26
+
+    def check(k):
+        u = np.arange(k * span, (k + 1) * span, dtype=np.uint64).astype(np.uint32)
+        f = u.view(np.float32)
+        got = oracle.f32_to_bf16_many(f)
+        want = torch.from_numpy(f).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
+        nan = (u & 0x7fffffff) > 0x7f800000
+        bad = (got != want) & ~nan
+        got_nan = ((got & 0x7f80) == 0x7f80) & ((got & 0x007f) != 0)
+        return int(bad.sum()), bool(np.array_equal(got_nan, nan))
+
+    with ThreadPoolExecutor(max_workers=4) as ex:
+        for bad, nans_ok in ex.map(check, range(64)):
+            assert bad == 0 and nans_ok
+
+
 def nearest_bf16_by_search(x):
     """Independent fp64 -> bf16 rounding: search the sorted table of all finite bf16 values."""
     codes = np.arange(0, 0x7f80, dtype=np.uint16)
