@@ -11,6 +11,8 @@ Array conventions (all host, C-contiguous numpy):
   chunk   uint8  [chunk_bytes]  raw: bf16 [L][2][T][H][D];
                                 int8: int8 codes [L][2][T][H][D] then fp32 scales [L][2][T][H*D/64]
                                 int4: nibbles [L][2][T][H][D/2] bytes (element 2k low, 2k+1 high) then the same scales
+                                per-channel key codecs: the same codes, then per layer fp32 k_scales [ceil(T/64)][H*D]
+                                followed by fp32 v_scales [T][H*D/64]
 """
 from __future__ import annotations
 
@@ -24,6 +26,8 @@ import numpy as np
 RAW_BF16 = 0
 INT8_G64 = 1
 INT4_G64 = 2
+INT8_KC64 = 3      # keys grouped along tokens (64 tokens of one channel), values as INT8_G64
+INT4_KC64 = 4      # the same with codes in [-7, 7]
 GROUP = 64
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -65,6 +69,8 @@ def lib():
             L.kdn_oracle_quant_group.argtypes = [vp, vp, vp]
             L.kdn_oracle_quant4_group.restype = None
             L.kdn_oracle_quant4_group.argtypes = [vp, vp, vp]
+            L.kdn_oracle_quant_channel.restype = None
+            L.kdn_oracle_quant_channel.argtypes = [vp, i32, i32, vp, vp]
             L.kdn_oracle_dequant.restype = C.c_uint16
             L.kdn_oracle_dequant.argtypes = [C.c_int8, C.c_float]
             L.kdn_oracle_rope_angle.restype = f64
@@ -221,6 +227,17 @@ def quant4_group(x_bf16: np.ndarray):
     q = np.zeros(GROUP // 2, dtype=np.uint8)
     s = np.zeros(1, dtype=np.float32)
     lib().kdn_oracle_quant4_group(_ptr(x), _ptr(q), _ptr(s))
+    return q, s[0]
+
+
+def quant_channel(x_bf16: np.ndarray, qmax: int):
+    """Encode n <= 64 bf16 bit patterns of one key channel (consecutive tokens) -> (int8 codes [n], fp32 scale)."""
+    x = np.ascontiguousarray(x_bf16, dtype=np.uint16)
+    if x.ndim != 1 or not 1 <= x.size <= GROUP:
+        raise ValueError("a channel group is 1..64 values")
+    q = np.zeros(x.size, dtype=np.int8)
+    s = np.zeros(1, dtype=np.float32)
+    lib().kdn_oracle_quant_channel(_ptr(x), x.size, int(qmax), _ptr(q), _ptr(s))
     return q, s[0]
 
 

@@ -37,6 +37,16 @@
  *                    q = clamp(round_half_even(x * inv), -7, 7); two codes per byte as two's-complement
  *                    nibbles, element 2k in the low nibble and 2k+1 in the high nibble of byte k;
  *                    chunk = nibbles[l][kv][t][head][D/2] bytes followed by the fp32 scales as in R2.
+ *   R4" per-channel key codecs (codecs 3 = int8, 4 = int4; not prescribed by the paper: Sec. 3.2 "KV-cache delivery"
+ *                    only cites quantisation among the techniques that shrink KV caches).  Keys have a few
+ *                    channels of large magnitude in every token, which a group along head_dim shares with its
+ *                    ordinary channels; grouping keys along TOKENS keeps such a channel to itself.
+ *                    K planes: group = the chunk tokens 64 g .. min(64 g + 63, T - 1) of one (l, head, d) channel;
+ *                    a = max over those tokens of |x|, then scale, inv and codes exactly as in R4 / R4' (127 or 7).
+ *                    V planes: exactly R4 / R4'.  Codes lie where R2 / R4' put them.  Scales, per layer:
+ *                    fp32 k_scales[ceil(T/64)][head*D] followed by fp32 v_scales[t][head*D/64]; layers follow
+ *                    each other; the scales follow the codes.  Decode is R5 with the element's own scale.
+ *                    Token lists (R7) are not defined for these codecs.
  *   R6  re-rotation  stored keys carry rotary position embedding at absolute
  *                    positions base_pos + t (what an engine's pool holds), so
  *                    reuse at dst_pos (Sec. 3.2 "KV-cache blending": a
@@ -80,6 +90,8 @@
 #define KDN_ORACLE_RAW_BF16 0
 #define KDN_ORACLE_INT8_G64 1
 #define KDN_ORACLE_INT4_G64 2
+#define KDN_ORACLE_INT8_KC64 3
+#define KDN_ORACLE_INT4_KC64 4
 #define KDN_ORACLE_GROUP 64
 
 /* ---------------------------------------------------------------- bf16 -- */
@@ -160,27 +172,34 @@ size_t kdn_oracle_chunk_bytes(int L, int H, int D, int T, int codec)
         if (D % KDN_ORACLE_GROUP) return 0;
         return elems / 2u + 4u * (elems / KDN_ORACLE_GROUP);
     }
+    if (codec == KDN_ORACLE_INT8_KC64 || codec == KDN_ORACLE_INT4_KC64) {
+        if (D % KDN_ORACLE_GROUP) return 0;
+        size_t hd = (size_t)H * (size_t)D;
+        size_t n_groups = ((size_t)T + KDN_ORACLE_GROUP - 1u) / KDN_ORACLE_GROUP;
+        size_t scales_per_layer = n_groups * hd + (size_t)T * hd / KDN_ORACLE_GROUP;     /* R4": K then V */
+        return (codec == KDN_ORACLE_INT4_KC64 ? elems / 2u : elems) + 4u * (size_t)L * scales_per_layer;
+    }
     return 0;
 }
 
 /* ------------------------------------------------------------ int8 codec -- */
 
 /* R4 / R4': encode one group of 64 bf16 values with codes in [-qmax, qmax] (127 or 7). */
-static void quant_group_q(const uint16_t *x_bf16, int8_t *q, float *scale_out, float qmax)
+static void quant_values_q(const uint16_t *x_bf16, int n, int8_t *q, float *scale_out, float qmax)
 {
     float a = 0.0f;
-    for (int i = 0; i < KDN_ORACLE_GROUP; ++i) {
+    for (int i = 0; i < n; ++i) {
         float v = fabsf(kdn_oracle_bf16_to_f32(x_bf16[i]));
         if (v > a) a = v;
     }
     volatile float scale = a / qmax;               /* volatile: one fp32 divide, stored as fp32 */
     if (!(scale >= FLT_MIN)) {
         *scale_out = 0.0f;
-        for (int i = 0; i < KDN_ORACLE_GROUP; ++i) q[i] = 0;
+        for (int i = 0; i < n; ++i) q[i] = 0;
         return;
     }
     volatile float inv = qmax / a;
-    for (int i = 0; i < KDN_ORACLE_GROUP; ++i) {
+    for (int i = 0; i < n; ++i) {
         volatile float prod = kdn_oracle_bf16_to_f32(x_bf16[i]) * inv;   /* one fp32 multiply */
         float r = rintf(prod);                     /* default rounding mode: ties to even */
         if (r > qmax) r = qmax;
@@ -188,6 +207,17 @@ static void quant_group_q(const uint16_t *x_bf16, int8_t *q, float *scale_out, f
         q[i] = (int8_t)(int)r;
     }
     *scale_out = scale;
+}
+
+static void quant_group_q(const uint16_t *x_bf16, int8_t *q, float *scale_out, float qmax)
+{
+    quant_values_q(x_bf16, KDN_ORACLE_GROUP, q, scale_out, qmax);
+}
+
+/* R4": encode n <= 64 values of one key channel (consecutive chunk tokens) with codes in [-qmax, qmax]. */
+void kdn_oracle_quant_channel(const uint16_t *x_bf16, int n, int qmax, int8_t *q, float *scale_out)
+{
+    quant_values_q(x_bf16, n, q, scale_out, (float)qmax);
 }
 
 void kdn_oracle_quant_group(const uint16_t *x_bf16, int8_t *q, float *scale_out)
@@ -271,7 +301,8 @@ static int check_args_list(const shape_t *s, const int32_t *table, int n_table, 
 {
     if (s->L <= 0 || s->H <= 0 || s->D <= 0 || s->bs <= 0 || s->nb <= 0) return 1;
     if (n < 0 || off < 0 || n_table < 0) return 1;
-    if (codec != KDN_ORACLE_RAW_BF16 && codec != KDN_ORACLE_INT8_G64 && codec != KDN_ORACLE_INT4_G64) return 3;
+    if (codec < KDN_ORACLE_RAW_BF16 || codec > KDN_ORACLE_INT4_KC64) return 3;
+    if ((codec == KDN_ORACLE_INT8_KC64 || codec == KDN_ORACLE_INT4_KC64) && list) return 3;   /* R4": no token lists */
     if (codec != KDN_ORACLE_RAW_BF16 && s->D % KDN_ORACLE_GROUP) return 3;
     for (int i = 0; i < n; ++i) {
         int64_t rel = list ? list[i] : i;
@@ -281,6 +312,69 @@ static int check_args_list(const shape_t *s, const int32_t *table, int n_table, 
         if (p >= (int64_t)n_table * (int64_t)s->bs) return 2;
         int32_t b = table[p / s->bs];
         if (b < 0 || (int64_t)b >= s->nb) return 4;
+    }
+    return 0;
+}
+
+/* R4": float index of the scale of chunk element (l, kv, t, head*D + d) in the scales area of a per-channel-key chunk. */
+static size_t kc_scale_index(const shape_t *s, int T, int l, int kv, int t, size_t ch)
+{
+    size_t hd = (size_t)s->H * (size_t)s->D;
+    size_t n_groups = ((size_t)T + KDN_ORACLE_GROUP - 1u) / KDN_ORACLE_GROUP;
+    size_t per_layer = n_groups * hd + (size_t)T * hd / KDN_ORACLE_GROUP;
+    if (kv == 0) return (size_t)l * per_layer + (size_t)(t / KDN_ORACLE_GROUP) * hd + ch;
+    return (size_t)l * per_layer + n_groups * hd + ((size_t)t * hd + ch) / KDN_ORACLE_GROUP;
+}
+
+static void put_code(uint8_t *chunk, int int4, size_t c, int8_t q)
+{
+    if (!int4) { ((int8_t *)chunk)[c] = q; return; }
+    uint8_t *b = chunk + c / 2u;
+    if (c & 1u) *b = (uint8_t)((*b & 0x0fu) | (((uint8_t)q & 0x0fu) << 4));
+    else *b = (uint8_t)((*b & 0xf0u) | ((uint8_t)q & 0x0fu));
+}
+
+/* R4": store with keys grouped along tokens and values grouped along head_dim. */
+static int store_kc(const shape_t *s, const uint16_t *pool, const int32_t *table, int64_t off, int T, int codec, uint8_t *chunk)
+{
+    int int4 = codec == KDN_ORACLE_INT4_KC64;
+    int qmax = int4 ? 7 : 127;
+    size_t hd = (size_t)s->H * (size_t)s->D;
+    size_t elems = (size_t)s->L * 2u * (size_t)T * hd;
+    float *scales = (float *)(chunk + (int4 ? elems / 2u : elems));
+    if (int4) memset(chunk, 0, elems / 2u);
+    for (int l = 0; l < s->L; ++l) {
+        /* keys: one group per (64-token span, channel) */
+        for (int t0 = 0; t0 < T; t0 += KDN_ORACLE_GROUP) {
+            int n = T - t0 < KDN_ORACLE_GROUP ? T - t0 : KDN_ORACLE_GROUP;
+            for (int h = 0; h < s->H; ++h)
+                for (int d = 0; d < s->D; ++d) {
+                    uint16_t x[KDN_ORACLE_GROUP];
+                    int8_t q[KDN_ORACLE_GROUP];
+                    for (int i = 0; i < n; ++i) {
+                        int64_t p = off + t0 + i;
+                        x[i] = pool[pool_index(s, l, 0, table[p / s->bs], (int)(p % s->bs), h, d)];
+                    }
+                    size_t ch = (size_t)h * (size_t)s->D + (size_t)d;
+                    kdn_oracle_quant_channel(x, n, qmax, q, scales + kc_scale_index(s, T, l, 0, t0, ch));
+                    for (int i = 0; i < n; ++i) put_code(chunk, int4, chunk_index(s, T, l, 0, t0 + i, h, d), q[i]);
+                }
+        }
+        /* values: R4 / R4' */
+        for (int t = 0; t < T; ++t) {
+            int64_t p = off + t;
+            int64_t block = table[p / s->bs];
+            int slot = (int)(p % s->bs);
+            for (int h = 0; h < s->H; ++h)
+                for (int g = 0; g < s->D / KDN_ORACLE_GROUP; ++g) {
+                    int8_t q[KDN_ORACLE_GROUP];
+                    size_t src = pool_index(s, l, 1, block, slot, h, g * KDN_ORACLE_GROUP);
+                    size_t ch = (size_t)h * (size_t)s->D + (size_t)g * KDN_ORACLE_GROUP;
+                    quant_group_q(pool + src, q, scales + kc_scale_index(s, T, l, 1, t, ch), (float)qmax);
+                    for (int i = 0; i < KDN_ORACLE_GROUP; ++i)
+                        put_code(chunk, int4, chunk_index(s, T, l, 1, t, h, g * KDN_ORACLE_GROUP + i), q[i]);
+                }
+        }
     }
     return 0;
 }
@@ -298,6 +392,8 @@ int kdn_oracle_store_sparse(const uint16_t *pool, int L, int H, int D, int bs, i
     int rc = check_args_list(&s, table, n_table, off, T, codec, keep, -1);
     if (rc) return rc;
     size_t elems = (size_t)L * 2u * (size_t)T * (size_t)H * (size_t)D;
+    if (codec == KDN_ORACLE_INT8_KC64 || codec == KDN_ORACLE_INT4_KC64)
+        return store_kc(&s, pool, table, off, T, codec, chunk);
     uint16_t *raw = (uint16_t *)chunk;
     int8_t *codes = (int8_t *)chunk;
     float *scales = (float *)(chunk + (codec == KDN_ORACLE_INT4_G64 ? elems / 2u : elems));
@@ -339,8 +435,18 @@ int kdn_oracle_store(const uint16_t *pool, int L, int H, int D, int bs, int64_t 
 }
 
 /* The stored value of chunk element c before any bf16 rounding: code and scale (raw: the bf16 itself). */
-static void stored_code(const uint8_t *chunk, size_t elems, int codec, size_t c, int *q, float *scale)
+static void stored_code(const uint8_t *chunk, size_t elems, int codec, size_t c, int *q, float *scale,
+                        const shape_t *s, int T)
 {
+    if (codec == KDN_ORACLE_INT8_KC64 || codec == KDN_ORACLE_INT4_KC64) {           /* R4" */
+        int int4 = codec == KDN_ORACLE_INT4_KC64;
+        size_t hd = (size_t)s->H * (size_t)s->D;
+        size_t ch = c % hd, row = c / hd;                  /* row = (l * 2 + kv) * T + t */
+        int t = (int)(row % (size_t)T), kv = (int)((row / (size_t)T) & 1u), l = (int)(row / (size_t)T / 2u);
+        *q = int4 ? kdn_oracle_nibble(chunk, c) : ((const int8_t *)chunk)[c];
+        *scale = ((const float *)(chunk + (int4 ? elems / 2u : elems)))[kc_scale_index(s, T, l, kv, t, ch)];
+        return;
+    }
     if (codec == KDN_ORACLE_INT8_G64) {
         *q = ((const int8_t *)chunk)[c];
         *scale = ((const float *)(chunk + elems))[c / KDN_ORACLE_GROUP];
@@ -351,12 +457,12 @@ static void stored_code(const uint8_t *chunk, size_t elems, int codec, size_t c,
 }
 
 /* R5: the bf16 a retrieve writes for chunk element c. */
-static uint16_t decoded(const uint8_t *chunk, size_t elems, int codec, size_t c)
+static uint16_t decoded(const uint8_t *chunk, size_t elems, int codec, size_t c, const shape_t *s, int T)
 {
     if (codec == KDN_ORACLE_RAW_BF16) return ((const uint16_t *)chunk)[c];
     int q;
     float scale;
-    stored_code(chunk, elems, codec, c, &q, &scale);
+    stored_code(chunk, elems, codec, c, &q, &scale, s, T);
     return kdn_oracle_dequant((int8_t)q, scale);
 }
 
@@ -383,7 +489,7 @@ int kdn_oracle_retrieve_sparse(uint16_t *pool, int L, int H, int D, int bs, int6
                     for (int d = 0; d < D; ++d) {
                         size_t c = chunk_index(&s, T, l, kv, t, h, d);
                         size_t o = pool_index(&s, l, kv, block, slot, h, d);
-                        pool[o] = decoded(chunk, elems, codec, c);
+                        pool[o] = decoded(chunk, elems, codec, c, &s, T);
                     }
             }
     return 0;
@@ -448,7 +554,7 @@ int kdn_oracle_compose_select(uint16_t *pool, int L, int H, int D, int bs, int64
                             for (int d = 0; d < D; ++d) {
                                 size_t c = chunk_index(&s, T, l, kv, t, h, d);
                                 size_t o = pool_index(&s, l, kv, block, slot, h, d);
-                                pool[o] = decoded(chunks[j], elems, codec, c);
+                                pool[o] = decoded(chunks[j], elems, codec, c, &s, T);
                                 if (kv == 0 && kref) {
                                     size_t r = (((size_t)l * (size_t)P + (size_t)p) * (size_t)H + (size_t)h) * (size_t)D + (size_t)d;
                                     kref[r] = (double)kdn_oracle_bf16_to_f32(pool[o]);
@@ -467,8 +573,8 @@ int kdn_oracle_compose_select(uint16_t *pool, int L, int H, int D, int bs, int64
                             } else {
                                 int qu, qw;
                                 float su, sw;
-                                stored_code(chunks[j], elems, codec, cu, &qu, &su);
-                                stored_code(chunks[j], elems, codec, cw, &qw, &sw);
+                                stored_code(chunks[j], elems, codec, cu, &qu, &su, &s, T);
+                                stored_code(chunks[j], elems, codec, cw, &qw, &sw, &s, T);
                                 u = (double)qu * (double)su;
                                 w = (double)qw * (double)sw;
                             }
