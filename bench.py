@@ -38,13 +38,14 @@ WORKLOAD = ("llama3-8b KV (L32 H8 D128 bf16, block_size 16, 16384-block pool): s
             "compose 10x1024 tokens (+256-token suffix), raw bf16 and int8-g64, fully fragmented tables")
 N_CHUNKS, CHUNK_TOKENS = 64, 512
 N_PARTS, PART_TOKENS, SUFFIX_TOKENS = 10, 1024, 256
-RAW, INT8, INT4 = 0, 1, 2
+RAW, INT8, INT4, INT8KC, INT4KC = 0, 1, 2, 3, 4
 FALLBACK_HBM_GBS = 6650.0
 
 
 def bytes_per_elem(codec: int) -> float:
     """Algorithmic bytes per KV element moved by one op: bf16 on the pool side + the chunk side."""
-    return {RAW: 4.0, INT8: 2.0 + 1.0 + 4.0 / 64.0, INT4: 2.0 + 0.5 + 4.0 / 64.0}[codec]
+    return {RAW: 4.0, INT8: 2.0 + 1.0 + 4.0 / 64.0, INT4: 2.0 + 0.5 + 4.0 / 64.0,
+            INT8KC: 2.0 + 1.0 + 4.0 / 64.0, INT4KC: 2.0 + 0.5 + 4.0 / 64.0}[codec]
 
 
 # ------------------------------------------------------------------------------------ CPU oracle leg --
@@ -412,6 +413,46 @@ def run_gpu(args) -> None:
     del i4
     torch.cuda.empty_cache()
 
+    # ---- per-channel key codecs (keys grouped along tokens; timed on their own, not part of `value`), and what they
+    # buy: the error of the stored keys, over all channels and over the channels without the x20 outlier gain
+    kc_ops = {}
+
+    def key_error_db(codec_id, ops_set):
+        """Retrieve chunk 0 and compare layer 0's keys with their source blocks: signal-to-noise ratio in dB."""
+        K.kdn_store(ctx, pid, ops_set["store"][:1], s)
+        K.kdn_retrieve(ctx, pid, [K.XferOp(d_dst.data_ptr(), bpc, 0, ops_set["store"][0].chunk)], s)
+        assert K.kdn_status_sync(ctx, s) == K.KDN_OK
+        x = k[0][d_src[:bpc].long()].float().reshape(-1, shape.row_elems)
+        y = k[0][d_dst[:bpc].long()].float().reshape(-1, shape.row_elems)
+        ordinary = (synth.outlier_gain(shape)[0, 0].reshape(-1) == 1).to(dev)
+        snr = lambda a, b: float(10 * torch.log10((a * a).mean() / ((a - b) ** 2).mean()))
+        return {"all_channels": snr(x, y), "ordinary_channels": snr(x[:, ordinary], y[:, ordinary])}
+
+    quality = {"int4_g64": key_error_db(INT4, make_sets(False, codecs=(INT4,))[INT4]),
+               "int8_g64": key_error_db(INT8, dev_sets[INT8])}
+    for codec, cname in ((INT8KC, "int8kc"), (INT4KC, "int4kc")):
+        kc = make_sets(False, codecs=(codec,))[codec]
+        K.kdn_store(ctx, pid, kc["part_store"], s)
+        for name, fn, arg in (("store_" + cname, K.kdn_store, kc["store"]), ("retrieve_" + cname, K.kdn_retrieve, kc["retrieve"]),
+                              ("compose_" + cname, K.kdn_compose, kc["reqs"])):
+            for _ in range(3):
+                fn(ctx, pid, arg, s)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            reps = max(1, min(args.steps, 20))
+            a.record(stream)
+            for _ in range(reps):
+                fn(ctx, pid, arg, s)
+            b.record(stream)
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / reps
+            nbytes = tokens_of[name.split("_")[0]] * E * bytes_per_elem(codec)
+            kc_ops[name] = {"ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9, "tokens_per_s": tokens_of[name.split("_")[0]] / (ms * 1e-3)}
+        assert K.kdn_status_sync(ctx, s) == K.KDN_OK
+        quality[cname] = key_error_db(codec, kc)
+        del kc
+        torch.cuda.empty_cache()
+    kc_ops["stored_key_snr_db"] = quality
+
     # ---- keep-lists: every chunk holds a seeded random half of its span's tokens (timed on its own, not in `value`)
     sparse_ops = {}
     rng = np.random.default_rng(synth.SEED_ASSIGN)
@@ -470,7 +511,7 @@ def run_gpu(args) -> None:
     if args.no_e2e:
         if rank == 0:
             print(json.dumps({"note": "profiling run, not a bench record", "ops_ms": op_ms,
-                              "ops_gbs": {n: op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 for n in names}, "int4": int4_ops, "sparse": sparse_ops, "shell": shell_ops, "file": file_ops}))
+                              "ops_gbs": {n: op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 for n in names}, "int4": int4_ops, "sparse": sparse_ops, "shell": shell_ops, "file": file_ops, "kc": kc_ops}))
         K.kdn_destroy(ctx)
         return
 
@@ -577,7 +618,7 @@ def run_gpu(args) -> None:
                        "bytes_per_step": step_bytes},
             "tokens_per_s_reloaded": world * reload_tokens / (sum(op_ms[n] for n in names if not n.startswith("store")) * 1e-3),
             "ops": ops, "ops_int4_not_in_value": int4_ops, "ops_keep_list_not_in_value": sparse_ops, "ops_shell_not_in_value": shell_ops,
-            "ops_file_not_in_value": file_ops,
+            "ops_file_not_in_value": file_ops, "ops_per_channel_key_codecs_not_in_value": kc_ops,
             "roofline": {"bound": "hbm", "kernel": kernel_of[top], "op": top, "achieved": ops[top]["gbs"], "peak": peak,
                          "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": ops[top]["gbs"] / peak,
                          "frac_of_nominal_8000": ops[top]["gbs"] / 8000.0, "traffic": traffic},

@@ -38,6 +38,15 @@
  *   decode = bf16_round_nearest_even((float)code * scale).
  * int4 coding: the same with 7 in place of 127 (scale = a/7, code in [-7, 7]); a stronger codec towards the
  *   more-than-tenfold footprint reduction Sec. 3.2 ("KV-cache delivery") reports for combined techniques.
+ * Per-channel key codecs (KDN_CODEC_INT8_KC64, KDN_CODEC_INT4_KC64; the paper prescribes no codec): keys carry a few
+ *   channels of large magnitude in every token; a group along head_dim makes its ordinary channels share the step of
+ *   such a channel.  These codecs group the KEYS along tokens instead -- the chunk tokens 64g .. 64g+63 of one
+ *   (layer, head, channel) form a group -- and code the values as the G64 codecs do.  Codes lie as in
+ *   INT8_G64 / INT4_G64; the scales that follow them are, per layer, fp32 k_scales[ceil(T/64)][H*D] and then
+ *   fp32 v_scales[T][H*D/64].  Same bytes per element as the G64 codecs when T is a multiple of 64.
+ *   They need block_size to divide 64 and the chunk's first token to sit at the start of a block (token_offset, or
+ *   part_dst_pos in kdn_compose, a multiple of block_size), else KDN_E_UNSUPPORTED; token lists, kdn_compose_static
+ *   and pools with more than about 1600 elements per token row are not supported with them.
  * Key re-rotation in kdn_compose: the stored keys of a part carry rotary
  *   position embedding for positions base_pos + t; placing the part at
  *   dst_pos rotates each pair (k[i], k[i + D/2]) of every head by
@@ -84,7 +93,8 @@ typedef enum {
     KDN_E_IO = 11           /* kdn_store_file / kdn_retrieve_file: a read or write of the chunk file failed or came up short */
 } kdn_status;
 
-typedef enum { KDN_CODEC_RAW_BF16 = 0, KDN_CODEC_INT8_G64 = 1, KDN_CODEC_INT4_G64 = 2 } kdn_codec;
+typedef enum { KDN_CODEC_RAW_BF16 = 0, KDN_CODEC_INT8_G64 = 1, KDN_CODEC_INT4_G64 = 2,
+               KDN_CODEC_INT8_KC64 = 3, KDN_CODEC_INT4_KC64 = 4 } kdn_codec;
 typedef enum { KDN_MEM_DEVICE = 0, KDN_MEM_PINNED_HOST = 1 } kdn_mem;
 
 /* An engine's paged KV pool (Sec. 3.2 names vLLM's paged memory).  k_layers and v_layers are HOST

@@ -109,10 +109,29 @@ kdn_status check_shape(const kdn_pool_desc *p)
     return KDN_OK;
 }
 
+bool is_kc(int codec) { return codec == KDN_CODEC_INT8_KC64 || codec == KDN_CODEC_INT4_KC64; }
+bool is_int4(int codec) { return codec == KDN_CODEC_INT4_G64 || codec == KDN_CODEC_INT4_KC64; }
+
+// fp32 scales one layer of a chunk holds (0 for raw bf16).
+size_t scales_per_layer(size_t row, size_t T, int codec)
+{
+    if (codec == KDN_CODEC_RAW_BF16) return 0;
+    if (is_kc(codec)) return (T + 63) / 64 * row + T * row / 64;         // key scales per channel, then value scales
+    return 2 * T * row / 64;
+}
+
+// The per-channel key codecs group 64 consecutive chunk tokens; a pool block must lie inside one group.
+kdn_status check_kc(const kdn_pool_desc *p, const kdn_chunk *c, int64_t pos)
+{
+    if (!is_kc(c->codec) || c->n_tokens == 0) return KDN_OK;
+    if (64 % p->block_size || pos % p->block_size) return KDN_E_UNSUPPORTED;
+    return KDN_OK;
+}
+
 kdn_status check_chunk(const kdn_pool_desc *p, const kdn_chunk *c)
 {
     if (c->n_tokens < 0) return KDN_E_INVAL;
-    if (c->codec != KDN_CODEC_RAW_BF16 && c->codec != KDN_CODEC_INT8_G64 && c->codec != KDN_CODEC_INT4_G64) return KDN_E_INVAL;
+    if (c->codec < KDN_CODEC_RAW_BF16 || c->codec > KDN_CODEC_INT4_KC64) return KDN_E_INVAL;
     if (c->mem != KDN_MEM_DEVICE && c->mem != KDN_MEM_PINNED_HOST) return KDN_E_INVAL;
     if (c->codec != KDN_CODEC_RAW_BF16 && p->head_dim % 64) return KDN_E_UNSUPPORTED;
     if (c->bytes != kdn_chunk_bytes(p, c->n_tokens, c->codec)) return KDN_E_SHAPE;
@@ -313,9 +332,10 @@ kdn_status launch_tiles(int OP, int groups, int gw, unsigned grid, size_t smem, 
 kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *hops, int n, cudaStream_t stream)
 {
     if (n <= 0) return KDN_OK;
-    bool any_coded = false, any_rot = false, any_list = false, all_list = true;
+    bool any_coded = false, any_rot = false, any_list = false, all_list = true, any_kc = false;
     for (int i = 0; i < n; ++i) {
         any_coded |= hops[i].op.codec != KDN_CODEC_RAW_BF16;
+        any_kc |= is_kc(hops[i].op.codec);
         any_rot |= hops[i].rotate;
         any_list |= hops[i].op.list_mode != 0;
         all_list &= hops[i].op.list_mode != 0;
@@ -327,6 +347,9 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     unsigned unit = 8;
     if (any_coded) unit = lcm_u(unit, 64);
     if (any_rot) unit = lcm_u(unit, (unsigned)pool.D);
+    // decoding a key tile of a per-channel key codec takes one scale per channel: such tiles are whole token rows
+    const bool kc_decode = any_kc && OP != OP_STORE;
+    if (kc_decode) unit = lcm_u(unit, row_elems);
     Shape def = default_shape(OP, any_coded, any_rot);
     int tile_bytes = ctx->tuning.tile_bytes > 0 ? ctx->tuning.tile_bytes : def.tile_bytes;
     unsigned tile_elems = (unsigned)tile_bytes / 2u / unit * unit;
@@ -348,7 +371,8 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
 
     const unsigned a_bytes = (tile_elems * 2u + 127u) & ~127u;
     const unsigned b_bytes = compute ? ((tile_elems + 127u) & ~127u) : 0u;
-    const unsigned s_bytes = compute ? ((tile_elems / 16u + 127u) & ~127u) : 0u;
+    unsigned s_bytes = compute ? ((tile_elems / 16u + 127u) & ~127u) : 0u;
+    if (kc_decode && s_bytes < row_elems * 4u) s_bytes = (row_elems * 4u + 127u) & ~127u;   // one scale per channel
     const unsigned stage_bytes = a_bytes + b_bytes + s_bytes;
     int groups = 0;
     if (compute) groups = ctx->tuning.compute_groups > 0 ? ctx->tuning.compute_groups : def.groups;
@@ -375,6 +399,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
 
     unsigned long long tiles = 0;
     int n_rope = 0;
+    int kc_layers = 0, kc_groups = 0;                      // grid of the key-plane store kernel (0: not needed)
     for (int i = 0; i < n; ++i) {
         DevOp op = hops[i].op;
         op.tile_begin = (unsigned)tiles;
@@ -383,8 +408,16 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
             h_rope[n_rope] = hops[i].rp;
             op.rope = n_rope++;
         }
+        if (OP == OP_STORE && is_kc(op.codec)) {
+            // the tile pipeline codes the value planes; the key planes go through kdn_store_kc_kernel below
+            op.kv_sel = 2;
+            if (op.nl > kc_layers) kc_layers = op.nl;
+            const int g = (op.T + 63) / 64;
+            if (g > kc_groups) kc_groups = g;
+        }
         h_ops[i] = op;
-        tiles += (unsigned long long)op.nl * 2ull * (op.list_mode ? (unsigned long long)op.n_list : (unsigned long long)op.nblk * tpb);
+        tiles += (unsigned long long)op.nl * (op.kv_sel ? 1ull : 2ull) *
+                 (op.list_mode ? (unsigned long long)op.n_list : (unsigned long long)op.nblk * tpb);
         if (tiles > kMaxTilesPerLaunch) return KDN_E_UNSUPPORTED;
     }
     if (tiles == 0) return KDN_OK;
@@ -429,6 +462,32 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     lp.store_lag = lag;
     lp.reload_first = (!compute && tile_elems * 2u >= 8192u) ? 1 : 0;
 
+    if (kc_groups > 0) {
+        // key planes of the per-channel key codecs: one CTA per (64-token group, layer, op)
+        const size_t kc_smem = kc_smem_bytes(row_elems);
+        if (kc_smem > smem_limit) return KDN_E_UNSUPPORTED;
+        KcLaunch kp{};
+        kp.ops = inl ? nullptr : slot->d_ops;
+        kp.n_ops = n;
+        kp.k_layers = pool.d_k;
+        kp.n_blocks = pool.nb;
+        kp.bs = pool.bs;
+        kp.row_elems = row_elems;
+        kp.status = ctx->d_status;
+        if (inl) std::memcpy(kp.inline_ops, lp.inline_ops, sizeof(DevOp) * (size_t)n);
+        {
+            std::lock_guard<std::mutex> lock(g_attr_mutex);
+            size_t &granted = g_attr_granted[std::make_pair(ctx->device, (const void *)kdn_store_kc_kernel)];
+            if (granted < kc_smem) {
+                KDN_CUDA(cudaFuncSetAttribute(kdn_store_kc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kc_smem));
+                granted = kc_smem;
+            }
+        }
+        kdn_store_kc_kernel<<<dim3((unsigned)kc_groups, (unsigned)kc_layers, (unsigned)n), kKcThreads, kc_smem, stream>>>(kp);
+        KDN_CUDA(cudaGetLastError());
+        ctx->launches++;
+    }
+
     unsigned long long want = (unsigned long long)ctx->sm_count * (unsigned)ctas_per_sm;
     const unsigned grid = (unsigned)(tiles < want ? tiles : want);
     const int gw = ctx->tuning.group_warps > 0 ? ctx->tuning.group_warps : def.gw;
@@ -470,8 +529,7 @@ HostOp make_host_op(const Pool &pool, const int32_t *table, int32_t n_table, int
     h.op.nl = pool.L;
     h.op.pos_end = (long long)n_table * pool.bs;
     const size_t elems = (size_t)pool.L * 2u * (size_t)c.n_tokens * (size_t)pool.H * (size_t)pool.D;
-    if (c.codec == KDN_CODEC_INT8_G64) h.op.scales = (unsigned char *)c.data + elems;
-    if (c.codec == KDN_CODEC_INT4_G64) h.op.scales = (unsigned char *)c.data + elems / 2u;
+    if (c.codec != KDN_CODEC_RAW_BF16) h.op.scales = (unsigned char *)c.data + (is_int4(c.codec) ? elems / 2u : elems);
     return h;
 }
 
@@ -554,9 +612,9 @@ kdn_status run_staged(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<
         const size_t T = (size_t)h.op.T;
         if (T == 0) continue;
         const bool coded = h.op.codec != KDN_CODEC_RAW_BF16;
-        const size_t codes_per_layer = h.op.codec == KDN_CODEC_INT4_G64 ? T * row : 2 * T * row * (coded ? 1 : 2);
-        const size_t scales_per_layer = coded ? 2 * T * (row / 64) * 4 : 0;
-        const size_t per_layer = ((codes_per_layer + 255) & ~(size_t)255) + ((scales_per_layer + 255) & ~(size_t)255);
+        const size_t codes_per_layer = is_int4(h.op.codec) ? T * row : 2 * T * row * (coded ? 1 : 2);
+        const size_t scale_bytes_per_layer = scales_per_layer(row, T, h.op.codec) * 4;
+        const size_t per_layer = ((codes_per_layer + 255) & ~(size_t)255) + ((scale_bytes_per_layer + 255) & ~(size_t)255);
         if (per_layer > ctx->slab_bytes) return KDN_E_UNSUPPORTED;
         unsigned char *host = h.op.data;
         const size_t host_codes_total = (size_t)pool.L * codes_per_layer;
@@ -574,7 +632,7 @@ kdn_status run_staged(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<
             // a piece is laid out exactly like a chunk of nl layers: codes, then scales
             const size_t base = used;
             const size_t cbytes = (size_t)nl * codes_per_layer;
-            const size_t sbytes = (size_t)nl * scales_per_layer;
+            const size_t sbytes = (size_t)nl * scale_bytes_per_layer;
             HostOp sub = h;
             sub.op.l0 = l;
             sub.op.nl = nl;
@@ -585,11 +643,11 @@ kdn_status run_staged(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<
                 pieces.push_back(Piece{ nullptr, base, cbytes, h.fd, h.file_off + (long long)((size_t)l * codes_per_layer) });
                 if (sbytes)
                     pieces.push_back(Piece{ nullptr, base + cbytes, sbytes, h.fd,
-                                            h.file_off + (long long)(host_codes_total + (size_t)l * scales_per_layer) });
+                                            h.file_off + (long long)(host_codes_total + (size_t)l * scale_bytes_per_layer) });
             } else {
                 pieces.push_back(Piece{ host + (size_t)l * codes_per_layer, base, cbytes, -1, 0 });
                 if (sbytes)
-                    pieces.push_back(Piece{ host + host_codes_total + (size_t)l * scales_per_layer, base + cbytes, sbytes, -1, 0 });
+                    pieces.push_back(Piece{ host + host_codes_total + (size_t)l * scale_bytes_per_layer, base + cbytes, sbytes, -1, 0 });
             }
             batch.push_back(sub);
             used = (base + cbytes + sbytes + 255) & ~(size_t)255;
@@ -612,7 +670,8 @@ size_t chunk_side_bytes(const Pool &pool, const HostOp &h)
 {
     const size_t elems = (size_t)h.op.nl * 2u * (size_t)h.op.T * (size_t)pool.H * (size_t)pool.D;
     if (h.op.codec == KDN_CODEC_RAW_BF16) return elems * 2u;
-    return (h.op.codec == KDN_CODEC_INT4_G64 ? elems / 2u : elems) + elems / 64u * 4u;
+    return (is_int4(h.op.codec) ? elems / 2u : elems) +
+           (size_t)h.op.nl * scales_per_layer((size_t)pool.H * (size_t)pool.D, (size_t)h.op.T, h.op.codec) * 4u;
 }
 
 kdn_status run_ops(kdn_ctx *ctx, int pool_id, int OP, std::vector<HostOp> &dev_ops, std::vector<HostOp> &host_ops,
@@ -663,8 +722,8 @@ HostOp layer_range(const Pool &pool, const HostOp &h, int l0, int nl)
     sub.op.l0 = l0;
     sub.op.nl = nl;
     if (h.op.codec != KDN_CODEC_RAW_BF16) {
-        sub.op.data = h.op.data + (size_t)l0 * (h.op.codec == KDN_CODEC_INT4_G64 ? plane / 2u : plane);
-        sub.op.scales = h.op.scales + (size_t)l0 * (plane / 64u) * 4u;
+        sub.op.data = h.op.data + (size_t)l0 * (is_int4(h.op.codec) ? plane / 2u : plane);
+        sub.op.scales = h.op.scales + (size_t)l0 * scales_per_layer((size_t)pool.H * (size_t)pool.D, (size_t)h.op.T, h.op.codec) * 4u;
     } else {
         sub.op.data = h.op.data + (size_t)l0 * plane * 2u;
     }
@@ -708,6 +767,7 @@ kdn_status xfer_sparse(kdn_ctx *ctx, int pool_id, int OP, const kdn_sparse_op *o
         const kdn_xfer_op &o = ops[i].op;
         st = check_chunk(&shape, &o.chunk);
         if (st != KDN_OK) return st;
+        if (is_kc(o.chunk.codec)) return KDN_E_UNSUPPORTED;      // a keep-list breaks up the 64-token key groups
         if (o.n_table_blocks < 0 || o.token_offset < 0) return KDN_E_INVAL;
         if (o.chunk.n_tokens > 0 && (!o.block_table || !ops[i].keep)) return KDN_E_INVAL;
         // the listed tokens are distinct positions below the end of the table, so there cannot be more of them
@@ -738,6 +798,12 @@ size_t kdn_chunk_bytes(const kdn_pool_desc *pool, int32_t n_tokens, int32_t code
     if (codec == KDN_CODEC_RAW_BF16) return elems * 2u;
     if (codec == KDN_CODEC_INT8_G64) return pool->head_dim % 64 ? 0 : elems + elems / 64u * 4u;
     if (codec == KDN_CODEC_INT4_G64) return pool->head_dim % 64 ? 0 : elems / 2u + elems / 64u * 4u;
+    if (is_kc(codec)) {
+        if (pool->head_dim % 64) return 0;
+        const size_t row = (size_t)pool->n_kv_heads * (size_t)pool->head_dim;
+        return (codec == KDN_CODEC_INT4_KC64 ? elems / 2u : elems) +
+               4u * (size_t)pool->n_layers * scales_per_layer(row, (size_t)n_tokens, codec);
+    }
     return 0;
 }
 
@@ -750,6 +816,8 @@ kdn_status kdn_validate_xfer(const kdn_pool_desc *pool, const kdn_xfer_op *ops, 
         st = check_chunk(pool, &ops[i].chunk);
         if (st != KDN_OK) return st;
         st = check_range(pool, ops[i].block_table, ops[i].n_table_blocks, ops[i].token_offset, ops[i].chunk.n_tokens);
+        if (st != KDN_OK) return st;
+        st = check_kc(pool, &ops[i].chunk, ops[i].token_offset);
         if (st != KDN_OK) return st;
     }
     return KDN_OK;
@@ -769,6 +837,8 @@ kdn_status kdn_validate_compose(const kdn_pool_desc *pool, const kdn_compose_req
             st = check_chunk(pool, &q.parts[j]);
             if (st != KDN_OK) return st;
             st = check_range(pool, q.block_table, q.n_table_blocks, q.part_dst_pos[j], q.parts[j].n_tokens);
+            if (st != KDN_OK) return st;
+            st = check_kc(pool, &q.parts[j], q.part_dst_pos[j]);
             if (st != KDN_OK) return st;
             rotates |= q.parts[j].n_tokens > 0 && q.part_dst_pos[j] != q.parts[j].base_pos;
         }
@@ -905,6 +975,8 @@ static kdn_status xfer_file(kdn_ctx *ctx, int pool_id, int OP, const kdn_file_op
         if (st != KDN_OK) return st;
         st = check_range(&shape, o.block_table, o.n_table_blocks, o.token_offset, o.chunk.n_tokens);
         if (st != KDN_OK) return st;
+        st = check_kc(&shape, &o.chunk, o.token_offset);
+        if (st != KDN_OK) return st;
         if (ops[i].fd < 0 || ops[i].file_offset < 0) return KDN_E_INVAL;
     }
     if (cudaSetDevice(ctx->device) != cudaSuccess) return KDN_E_CUDA;
@@ -1013,6 +1085,7 @@ static kdn_status compose_impl(kdn_ctx *ctx, int pool_id, const kdn_compose_req 
             if (selects && selects[r].part_select && selects[r].part_select[j]) {
                 if (!selects[r].part_n_select || selects[r].part_n_select[j] < 0 || selects[r].part_n_select[j] > c.n_tokens)
                     return KDN_E_INVAL;
+                if (is_kc(c.codec)) return KDN_E_UNSUPPORTED;           // select-lists are not defined for these codecs
                 if (selects[r].part_n_select[j] == 0) continue;          // nothing of this part is delivered
                 h.op.list = selects[r].part_select[j];
                 h.op.n_list = selects[r].part_n_select[j];
@@ -1162,6 +1235,7 @@ extern "C" kdn_status kdn_compose_static(int device, const kdn_pool_desc *pool, 
         for (int j = 0; j < reqs[r].n_parts; ++j) {
             if (reqs[r].parts[j].n_tokens == 0) continue;
             if (reqs[r].parts[j].mem != KDN_MEM_DEVICE) return KDN_E_UNSUPPORTED;
+            if (is_kc(reqs[r].parts[j].codec)) return KDN_E_UNSUPPORTED;
             ++n_parts;
         }
         if (n_parts > KDN_STATIC_MAX_PARTS) return KDN_E_UNSUPPORTED;

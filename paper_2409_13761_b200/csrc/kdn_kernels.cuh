@@ -35,7 +35,8 @@ constexpr int kMaxStages = 32;
 constexpr int kMaxStoreLag = 16;          // most bulk-store groups allowed to be still reading shared memory
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
-enum : uint32_t { TF_CODED = 1u, TF_ROTATE = 2u, TF_SCALES_PLAIN = 4u, TF_INT4 = 8u };   // TF_CODED: int8 or int4
+enum : uint32_t { TF_CODED = 1u, TF_ROTATE = 2u, TF_SCALES_PLAIN = 4u, TF_INT4 = 8u,   // TF_CODED: int8 or int4
+                  TF_KCHAN = 16u };   // key tile of a per-channel key codec: one scale per channel, row_elems of them
 enum : int { OP_STORE = 0, OP_RETRIEVE = 1, OP_COMPOSE = 2 };
 
 // Status values mirrored from kdn.h (kept numeric here so device code has no host header).
@@ -47,7 +48,7 @@ struct __align__(16) DevOp {
     unsigned char *data;      // layers [l0, l0 + nl) of the chunk: raw bf16, or int8 codes
     long long off;            // request position of chunk token 0
     int T;                    // tokens
-    int codec;                // 0 raw bf16, 1 int8 group-64, 2 int4 group-64
+    int codec;                // 0 raw bf16, 1 int8 group-64, 2 int4 group-64, 3 / 4 int8 / int4 with per-channel key groups
     int j0;                   // first logical block touched: off / block_size
     int nblk;                 // logical blocks touched
     unsigned tile_begin;      // index of this op's first tile in the launch
@@ -60,7 +61,9 @@ struct __align__(16) DevOp {
     int list_mode;            // 0: every token; 1 keep-list: chunk token i <-> off + list[i];
                               // 2 select-list: chunk token list[i] <-> off + list[i]
     long long pos_end;        // request positions >= pos_end are outside the block table
-    long long reserved;
+    int kv_sel;               // 0: key and value planes; 2: value planes only (the keys of a per-channel key codec are
+                              // stored by kdn_store_kc_kernel)
+    int reserved;
 };
 static_assert(sizeof(DevOp) == 96, "DevOp is copied as 96-byte records");
 
@@ -102,7 +105,7 @@ struct __align__(16) TileDesc {
     unsigned n;                   // elements; 0: nothing to do
     unsigned flags;
     int rope;
-    int reserved;
+    unsigned sbytes;              // bytes of scales that belong to the tile (coded tiles)
 };
 
 // ------------------------------------------------------------------ PTX --
@@ -455,6 +458,43 @@ __device__ __forceinline__ void dequantise4_tile(const unsigned char *B, const f
     }
 }
 
+// Two consecutive fp32 values of shared memory as a packed pair.
+__device__ __forceinline__ f32x2 lds_f32x2(const float *p)
+{
+    const uint2 v = lds64(p);
+    return pack2_bits(v.x, v.y);
+}
+
+// Decode a key tile of a per-channel key codec: n codes at B (whole token rows of row_elems channels), one scale per
+// channel at S, bf16 to A.  One item is 8 consecutive channels of one token.
+template <bool kInt4>
+__device__ __forceinline__ void dequantise_kc_tile(const unsigned char *B, const float *S, unsigned char *A,
+                                                   unsigned n, unsigned row_elems, int ct, unsigned gthreads)
+{
+    const unsigned nitems = n >> 3;
+    const f32x2 minus_bias = pack2(-8388736.0f, -8388736.0f);
+    const f32x2 minus_bias4 = pack2(-8388616.0f, -8388616.0f);
+    for (unsigned v = (unsigned)ct; v < nitems; v += gthreads) {
+        const unsigned e = v << 3;
+        const unsigned ch = e - (e / row_elems) * row_elems;
+        f32x2 f[4];
+        if (kInt4) {
+            nibbles_to_f32x2(*reinterpret_cast<const uint32_t *>(B + (e >> 1)), minus_bias4, f);
+        } else {
+            const uint2 c = lds64(B + e);
+            const uint32_t w0 = c.x ^ 0x80808080u, w1 = c.y ^ 0x80808080u;
+            f[0] = codes_to_f32x2<0>(w0, minus_bias); f[1] = codes_to_f32x2<2>(w0, minus_bias);
+            f[2] = codes_to_f32x2<0>(w1, minus_bias); f[3] = codes_to_f32x2<2>(w1, minus_bias);
+        }
+        uint4 o;
+        o.x = pack_bf16x2(mul2(f[0], lds_f32x2(S + ch)));
+        o.y = pack_bf16x2(mul2(f[1], lds_f32x2(S + ch + 2)));
+        o.z = pack_bf16x2(mul2(f[2], lds_f32x2(S + ch + 4)));
+        o.w = pack_bf16x2(mul2(f[3], lds_f32x2(S + ch + 6)));
+        sts128(A + (size_t)e * 2u, o);
+    }
+}
+
 // Rotation coefficients a thread keeps in registers: (cos, sin, -sin) for 8 consecutive frequencies,
 // as four packed pairs each.
 struct RotCoef {
@@ -494,9 +534,11 @@ __device__ __forceinline__ void rotate8(const f32x2 *u, const f32x2 *w, const Ro
 // Rotate a tile of whole head rows (n a multiple of D, D a multiple of 16).  One work item is 8
 // frequencies of one head row: elements [col, col+8) and [D/2 + col, D/2 + col + 8).
 // kCodec = 0: bf16 at A, in place.  kCodec = 1 / 2: int8 / int4 codes at B and scales at S -> bf16 at A.
-template <int kCodec>
+// kChan: the codes carry one scale per channel (S[channel], row_elems of them) instead of one per 64 elements.
+template <int kCodec, bool kChan = false>
 __device__ __forceinline__ void rotate_tile(unsigned char *A, const unsigned char *B, const float *S, unsigned n,
-                                            unsigned D, const float2 *table, int rope, RotCoef &rc, int ct, unsigned gthreads)
+                                            unsigned D, const float2 *table, int rope, RotCoef &rc, int ct, unsigned gthreads,
+                                            unsigned row_elems = 0)
 {
     const unsigned half = D >> 1;
     const unsigned per_row = D >> 4;                      // work items per head row
@@ -510,26 +552,33 @@ __device__ __forceinline__ void rotate_tile(unsigned char *A, const unsigned cha
         load_coef(rc, table, rope, col, half);
         const unsigned e_lo = r * D + col, e_hi = e_lo + half;
         f32x2 u[4], w[4];
-        if (kCodec == 2) {
-            const uint32_t cl = *reinterpret_cast<const uint32_t *>(B + (e_lo >> 1));
-            const uint32_t ch = *reinterpret_cast<const uint32_t *>(B + (e_hi >> 1));
-            const float sl = S[e_lo >> 6], sh = S[e_hi >> 6];
-            const f32x2 sl2 = pack2(sl, sl), sh2 = pack2(sh, sh);
-            const f32x2 minus_bias4 = pack2(-8388616.0f, -8388616.0f);
-            nibbles_to_f32x2(cl, minus_bias4, u);
-            nibbles_to_f32x2(ch, minus_bias4, w);
+        if (kCodec != 0) {
+            if (kCodec == 2) {
+                const f32x2 minus_bias4 = pack2(-8388616.0f, -8388616.0f);
+                nibbles_to_f32x2(*reinterpret_cast<const uint32_t *>(B + (e_lo >> 1)), minus_bias4, u);
+                nibbles_to_f32x2(*reinterpret_cast<const uint32_t *>(B + (e_hi >> 1)), minus_bias4, w);
+            } else {
+                const uint2 cl = lds64(B + e_lo), ch = lds64(B + e_hi);
+                const uint32_t l0 = cl.x ^ 0x80808080u, l1 = cl.y ^ 0x80808080u;
+                const uint32_t h0 = ch.x ^ 0x80808080u, h1 = ch.y ^ 0x80808080u;
+                u[0] = codes_to_f32x2<0>(l0, minus_bias); u[1] = codes_to_f32x2<2>(l0, minus_bias);
+                u[2] = codes_to_f32x2<0>(l1, minus_bias); u[3] = codes_to_f32x2<2>(l1, minus_bias);
+                w[0] = codes_to_f32x2<0>(h0, minus_bias); w[1] = codes_to_f32x2<2>(h0, minus_bias);
+                w[2] = codes_to_f32x2<0>(h1, minus_bias); w[3] = codes_to_f32x2<2>(h1, minus_bias);
+            }
+            if (kChan) {
+                const unsigned c_lo = e_lo - (e_lo / row_elems) * row_elems, c_hi = c_lo + half;
 #pragma unroll
-            for (int k = 0; k < 4; ++k) { u[k] = mul2(u[k], sl2); w[k] = mul2(w[k], sh2); }
-        } else if (kCodec == 1) {
-            const uint2 cl = lds64(B + e_lo), ch = lds64(B + e_hi);
-            const float sl = S[e_lo >> 6], sh = S[e_hi >> 6];
-            const f32x2 sl2 = pack2(sl, sl), sh2 = pack2(sh, sh);
-            const uint32_t l0 = cl.x ^ 0x80808080u, l1 = cl.y ^ 0x80808080u;
-            const uint32_t h0 = ch.x ^ 0x80808080u, h1 = ch.y ^ 0x80808080u;
-            u[0] = mul2(codes_to_f32x2<0>(l0, minus_bias), sl2); u[1] = mul2(codes_to_f32x2<2>(l0, minus_bias), sl2);
-            u[2] = mul2(codes_to_f32x2<0>(l1, minus_bias), sl2); u[3] = mul2(codes_to_f32x2<2>(l1, minus_bias), sl2);
-            w[0] = mul2(codes_to_f32x2<0>(h0, minus_bias), sh2); w[1] = mul2(codes_to_f32x2<2>(h0, minus_bias), sh2);
-            w[2] = mul2(codes_to_f32x2<0>(h1, minus_bias), sh2); w[3] = mul2(codes_to_f32x2<2>(h1, minus_bias), sh2);
+                for (int k = 0; k < 4; ++k) {
+                    u[k] = mul2(u[k], lds_f32x2(S + c_lo + 2 * k));
+                    w[k] = mul2(w[k], lds_f32x2(S + c_hi + 2 * k));
+                }
+            } else {
+                const float sl = S[e_lo >> 6], sh = S[e_hi >> 6];
+                const f32x2 sl2 = pack2(sl, sl), sh2 = pack2(sh, sh);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) { u[k] = mul2(u[k], sl2); w[k] = mul2(w[k], sh2); }
+            }
         } else {
             const uint4 xl = lds128(A + (size_t)e_lo * 2u), xh = lds128(A + (size_t)e_hi * 2u);
             u[0] = bf16x2_to_f32x2(xl.x); u[1] = bf16x2_to_f32x2(xl.y); u[2] = bf16x2_to_f32x2(xl.z); u[3] = bf16x2_to_f32x2(xl.w);
@@ -549,7 +598,7 @@ __device__ __forceinline__ void rotate_tile(unsigned char *A, const unsigned cha
 template <int OP>
 __device__ __forceinline__ void decode_tile(const Launch &P, unsigned g, TileDesc &d)
 {
-    d.n = 0; d.flags = 0; d.rope = -1; d.reserved = 0;
+    d.n = 0; d.flags = 0; d.rope = -1; d.sbytes = 0;
     d.g_pool = 0; d.g_chunk = 0; d.g_scales = 0;
     if (g >= P.n_tiles) return;                             // lanes past this CTA's last tile
     const DevOp *ops = P.ops ? P.ops : P.inline_ops;       // global memory, or the kernel's parameter space
@@ -574,7 +623,7 @@ __device__ __forceinline__ void decode_tile(const Launch &P, unsigned g, TileDes
         if (rel < 0 || p >= op.pos_end || c >= op.T) { atomicCAS(P.status, 0, kStatusRange); return; }
         id_index = p / P.bs;
         pool_elem = (unsigned long long)(p - id_index * P.bs) * P.row_elems;
-        ce = ((unsigned long long)plane * op.T + (unsigned long long)c) * P.row_elems;
+        ce = (unsigned long long)c * P.row_elems;          // inside the plane; the plane is added below
         n = P.row_elems;
     } else {
         const unsigned per_plane = (unsigned)op.nblk * P.tpb;
@@ -593,22 +642,43 @@ __device__ __forceinline__ void decode_tile(const Launch &P, unsigned g, TileDes
         n = (unsigned)((run - e0) < (unsigned long long)P.tile_elems ? (run - e0) : P.tile_elems);
         id_index = (long long)op.j0 + j;
         pool_elem = (unsigned long long)(p_lo - blk_start) * P.row_elems + e0;
-        ce = ((unsigned long long)plane * op.T + (unsigned long long)(p_lo - op.off)) * P.row_elems + e0;
+        ce = (unsigned long long)(p_lo - op.off) * P.row_elems + e0;     // inside the plane
     }
-    const int kv = (int)(plane & 1u);
-    const int l = op.l0 + (int)(plane >> 1);
+    const int kv = op.kv_sel ? op.kv_sel - 1 : (int)(plane & 1u);
+    const unsigned li = op.kv_sel ? plane : plane >> 1;     // layer index inside the op's layer range
+    const int l = op.l0 + (int)li;
     const long long id = __ldg(op.table + id_index);
     if (id < 0 || id >= P.n_blocks) { atomicCAS(P.status, 0, kStatusRange); return; }
     const unsigned char *base = reinterpret_cast<const unsigned char *>(kv ? P.v_layers[l] : P.k_layers[l]);
     d.g_pool = (unsigned long long)(base + ((unsigned long long)id * P.bs * P.row_elems + pool_elem) * 2ull);
+    const unsigned long long ce_plane = ce;                                   // element offset inside the plane
+    ce += ((unsigned long long)li * 2ull + (unsigned long long)kv) * (unsigned long long)op.T * P.row_elems;
     if (op.codec == 0) {
         d.g_chunk = (unsigned long long)(op.data + ce * 2ull);
     } else {
         d.flags |= TF_CODED;
-        if (op.codec == 2) { d.flags |= TF_INT4; d.g_chunk = (unsigned long long)(op.data + (ce >> 1)); }
+        if (op.codec == 2 || op.codec == 4) { d.flags |= TF_INT4; d.g_chunk = (unsigned long long)(op.data + (ce >> 1)); }
         else d.g_chunk = (unsigned long long)(op.data + ce);
-        d.g_scales = (unsigned long long)(op.scales + (ce >> 6) * 4ull);
-        if ((d.g_scales & 15ull) || ((n >> 6) & 3u)) d.flags |= TF_SCALES_PLAIN;
+        if (op.codec >= 3) {
+            // per layer: key scales [ceil(T / 64)][row_elems], then value scales [T][row_elems / 64]
+            const unsigned long long n_groups = ((unsigned long long)op.T + 63ull) >> 6;
+            const unsigned long long per_layer = n_groups * P.row_elems + (((unsigned long long)op.T * P.row_elems) >> 6);
+            if (kv == 0) {
+                // the tile is whole token rows of one 64-token group (the host sees to both)
+                d.flags |= TF_KCHAN;
+                d.g_scales = (unsigned long long)(op.scales + ((unsigned long long)li * per_layer +
+                                                               ((ce_plane / P.row_elems) >> 6) * P.row_elems) * 4ull);
+                d.sbytes = P.row_elems * 4u;
+            } else {
+                d.g_scales = (unsigned long long)(op.scales + ((unsigned long long)li * per_layer + n_groups * P.row_elems +
+                                                               (ce_plane >> 6)) * 4ull);
+                d.sbytes = n >> 4;
+            }
+        } else {
+            d.g_scales = (unsigned long long)(op.scales + (ce >> 6) * 4ull);
+            d.sbytes = n >> 4;
+        }
+        if ((d.g_scales & 15ull) || (d.sbytes & 15u)) d.flags |= TF_SCALES_PLAIN;
     }
     if (OP == OP_COMPOSE && kv == 0 && op.rope >= 0) { d.flags |= TF_ROTATE; d.rope = op.rope; }
     d.n = n;
@@ -707,9 +777,9 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                                 mbar_arrive_expect_tx(bar, code_bytes);
                                 bulk_g2s(smem_u32(A + P.off_b), (const void *)cur.g_chunk, code_bytes, bar);
                             } else {
-                                mbar_arrive_expect_tx(bar, code_bytes + (cur.n >> 4));
+                                mbar_arrive_expect_tx(bar, code_bytes + cur.sbytes);
                                 bulk_g2s(smem_u32(A + P.off_b), (const void *)cur.g_chunk, code_bytes, bar);
-                                bulk_g2s(smem_u32(A + P.off_s), (const void *)cur.g_scales, cur.n >> 4, bar);
+                                bulk_g2s(smem_u32(A + P.off_s), (const void *)cur.g_scales, cur.sbytes, bar);
                             }
                         }
                     }
@@ -750,7 +820,7 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                         if (d.flags & TF_CODED) {
                             bulk_s2g((void *)d.g_chunk, smem_u32(A + P.off_b), (d.flags & TF_INT4) ? d.n >> 1 : d.n);
                             if (!(d.flags & TF_SCALES_PLAIN))
-                                bulk_s2g((void *)d.g_scales, smem_u32(A + P.off_s), d.n >> 4);
+                                bulk_s2g((void *)d.g_scales, smem_u32(A + P.off_s), d.sbytes);
                         } else {
                             bulk_s2g((void *)d.g_chunk, smem_u32(A), d.n * 2u);
                         }
@@ -824,10 +894,19 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                 } else if (flags & TF_CODED) {
                     if (flags & TF_SCALES_PLAIN) {
                         const float *gs = reinterpret_cast<const float *>(sm.desc[st].g_scales);
-                        for (unsigned i = (unsigned)ct; i < (n >> 6); i += kGT) Sc[i] = __ldg(gs + i);
+                        for (unsigned i = (unsigned)ct; i < (sm.desc[st].sbytes >> 2); i += kGT) Sc[i] = __ldg(gs + i);
                         group_bar_sync(group, kGT);
                     }
-                    if (OP == OP_COMPOSE && (flags & TF_ROTATE)) {
+                    if (flags & TF_KCHAN) {
+                        if (OP == OP_COMPOSE && (flags & TF_ROTATE)) {
+                            if (flags & TF_INT4) rotate_tile<2, true>(A, B, Sc, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct, kGT, P.row_elems);
+                            else rotate_tile<1, true>(A, B, Sc, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct, kGT, P.row_elems);
+                        } else if (flags & TF_INT4) {
+                            dequantise_kc_tile<true>(B, Sc, A, n, P.row_elems, ct, kGT);
+                        } else {
+                            dequantise_kc_tile<false>(B, Sc, A, n, P.row_elems, ct, kGT);
+                        }
+                    } else if (OP == OP_COMPOSE && (flags & TF_ROTATE)) {
                         if (flags & TF_INT4) rotate_tile<2>(A, B, Sc, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct, kGT);
                         else rotate_tile<1>(A, B, Sc, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct, kGT);
                     } else if (flags & TF_INT4) {
@@ -872,6 +951,175 @@ kdn_retrieve_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_RETRIEV
 template <int kGroups, int kGW>
 __global__ void __launch_bounds__(threads_for(kGroups, kGW))
 kdn_compose_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_COMPOSE, kGroups, kGW>(P); }
+
+// ------------------------------------------------ keys of the per-channel key codecs --
+
+// Storing the key planes of a per-channel key codec needs, for every channel, the largest magnitude over 64 tokens
+// before the first code can be formed, so it does not fit the streaming tile pipeline.  One CTA takes one
+// (op, layer, 64-token group): the group's token rows (64 x row_elems bf16, contiguous per pool block) are brought into
+// shared memory with bulk copies; pass 1 reduces |x| per channel over four token slices; one thread per eight
+// channels combines the slices, forms scale and reciprocal (two IEEE divides per channel) and writes the scales;
+// pass 2 codes each element with its channel's reciprocal and writes the codes straight to the chunk.
+// The host guarantees: block_size divides 64, the op's token offset is a multiple of block_size, row_elems % 64 == 0.
+// Shared memory: 64 * row_elems * 2 (rows) + 4 * row_elems * 2 (slice maxima) + row_elems * 4 (reciprocals) + 16.
+struct KcLaunch {
+    const DevOp *ops;         // device array, or nullptr: inline_ops
+    int n_ops;
+    void *const *k_layers;
+    long long n_blocks;
+    int bs;
+    unsigned row_elems;
+    int *status;
+    DevOp inline_ops[kInlineOps];
+};
+
+constexpr int kKcThreads = 512;
+constexpr unsigned kKcSlices = 4;                          // token slices of 16 tokens in pass 1 and pass 2
+__host__ __device__ inline size_t kc_smem_bytes(unsigned row_elems)
+{
+    return (size_t)64 * row_elems * 2u + (size_t)kKcSlices * row_elems * 2u + (size_t)row_elems * 4u + 16u;
+}
+
+__global__ void __launch_bounds__(kKcThreads) kdn_store_kc_kernel(const __grid_constant__ KcLaunch P)
+{
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const DevOp *ops = P.ops ? P.ops : P.inline_ops;
+    const DevOp op = ops[blockIdx.z];
+    if (op.codec < 3) return;
+    const unsigned g = blockIdx.x, li = blockIdx.y;
+    const unsigned n_groups = ((unsigned)op.T + 63u) >> 6;
+    if (g >= n_groups || li >= (unsigned)op.nl) return;
+    const bool int4 = op.codec == 4;
+    const float qmax = int4 ? 7.0f : 127.0f;
+    const unsigned RE = P.row_elems;
+    const unsigned t0 = g << 6;
+    const unsigned n_tok = (unsigned)op.T - t0 < 64u ? (unsigned)op.T - t0 : 64u;
+
+    unsigned char *X = smem_raw;                                             // [n_tok][RE] bf16
+    unsigned char *pmax = X + (size_t)64 * RE * 2u;                          // [kKcSlices][RE] bf16 magnitudes
+    float *inv = reinterpret_cast<float *>(pmax + (size_t)kKcSlices * RE * 2u);   // [RE]
+    unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(reinterpret_cast<unsigned char *>(inv) + (size_t)RE * 4u);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bar_mem + 1);
+    const uint32_t bar = smem_u32(bar_mem);
+    const int tid = (int)threadIdx.x;
+
+    if (tid == 0) {
+        mbar_init(bar, 1u);
+        *abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        fence_async_smem();
+        // the group's rows, block by block (a block's tokens are contiguous in the pool)
+        const unsigned char *base = reinterpret_cast<const unsigned char *>(P.k_layers[op.l0 + (int)li]);
+        const long long first_block = (op.off + (long long)t0) / P.bs;
+        bool bad = false;
+        for (unsigned t = 0; t < n_tok && !bad; t += (unsigned)P.bs) {
+            const long long id = __ldg(op.table + first_block + t / (unsigned)P.bs);
+            if (id < 0 || id >= P.n_blocks) bad = true;
+        }
+        if (bad) {
+            atomicCAS(P.status, 0, kStatusRange);
+            *abort_flag = 1;                                                  // nothing is loaded, nothing is written
+        } else {
+            mbar_arrive_expect_tx(bar, n_tok * RE * 2u);
+            for (unsigned t = 0; t < n_tok; t += (unsigned)P.bs) {
+                const unsigned k = n_tok - t < (unsigned)P.bs ? n_tok - t : (unsigned)P.bs;
+                const long long id = __ldg(op.table + first_block + t / (unsigned)P.bs);
+                const unsigned char *src = base + (unsigned long long)id * P.bs * RE * 2ull;
+                // pieces of at most 32 KiB
+                const unsigned bytes = k * RE * 2u;
+                for (unsigned o = 0; o < bytes; o += 32768u)
+                    bulk_g2s(smem_u32(X + (size_t)t * RE * 2u + o), src + o, bytes - o < 32768u ? bytes - o : 32768u, bar);
+            }
+        }
+    }
+    __syncthreads();
+    if (*abort_flag) return;
+    const bool landed = mbar_wait(bar, 0u, abort_flag);
+    if (!__syncthreads_and(landed)) {                                         // all threads leave together
+        if (tid == 0) atomicCAS(P.status, 0, kStatusTimeout);
+        return;
+    }
+
+    const unsigned octets = RE >> 3;
+    const unsigned items = octets * kKcSlices;
+    // pass 1: per (eight channels, token slice) the largest magnitudes, as packed bf16 pairs
+    for (unsigned it = (unsigned)tid; it < items; it += (unsigned)kKcThreads) {
+        const unsigned q = it / octets, o = it - q * octets;
+        const unsigned ta = q * 16u, tb = ta + 16u < n_tok ? ta + 16u : n_tok;
+        uint32_t m0 = 0u, m1 = 0u, m2 = 0u, m3 = 0u;
+        for (unsigned t = ta; t < tb; ++t) {
+            const uint4 x = lds128(X + ((size_t)t * RE + (size_t)o * 8u) * 2u);
+            m0 = maxabs_bf16x2(m0, x.x); m1 = maxabs_bf16x2(m1, x.y);
+            m2 = maxabs_bf16x2(m2, x.z); m3 = maxabs_bf16x2(m3, x.w);
+        }
+        sts128(pmax + ((size_t)q * RE + (size_t)o * 8u) * 2u, make_uint4(m0, m1, m2, m3));
+    }
+    __syncthreads();
+    // scales: one thread per eight channels
+    const unsigned long long per_layer = (unsigned long long)n_groups * RE + (((unsigned long long)op.T * RE) >> 6);
+    float *g_scales = reinterpret_cast<float *>(op.scales) + (unsigned long long)li * per_layer + (unsigned long long)g * RE;
+    for (unsigned o = (unsigned)tid; o < octets; o += (unsigned)kKcThreads) {
+        uint32_t m[4] = { 0u, 0u, 0u, 0u };
+        for (unsigned q = 0; q < kKcSlices; ++q) {
+            const uint4 x = lds128(pmax + ((size_t)q * RE + (size_t)o * 8u) * 2u);
+            m[0] = maxabs_bf16x2(m[0], x.x); m[1] = maxabs_bf16x2(m[1], x.y);
+            m[2] = maxabs_bf16x2(m[2], x.z); m[3] = maxabs_bf16x2(m[3], x.w);
+        }
+        float sc[8], iv[8];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+            const float a_lo = __uint_as_float((m[k] << 16) & 0x7fffffffu), a_hi = __uint_as_float(m[k] & 0x7fff0000u);
+            float s_lo = __fdiv_rn(a_lo, qmax), s_hi = __fdiv_rn(a_hi, qmax);
+            const bool ok_lo = s_lo >= 1.17549435e-38f, ok_hi = s_hi >= 1.17549435e-38f;
+            sc[2 * k] = ok_lo ? s_lo : 0.0f;
+            sc[2 * k + 1] = ok_hi ? s_hi : 0.0f;
+            iv[2 * k] = ok_lo ? __fdiv_rn(qmax, a_lo) : 0.0f;
+            iv[2 * k + 1] = ok_hi ? __fdiv_rn(qmax, a_hi) : 0.0f;
+        }
+        // a layer's scales start wherever the previous layer's end: only 4-byte alignment is certain
+        float *gsp = g_scales + (size_t)o * 8u;
+        if ((reinterpret_cast<unsigned long long>(gsp) & 15ull) == 0ull) {
+            float4 *gs = reinterpret_cast<float4 *>(gsp);
+            gs[0] = make_float4(sc[0], sc[1], sc[2], sc[3]);
+            gs[1] = make_float4(sc[4], sc[5], sc[6], sc[7]);
+        } else {
+#pragma unroll
+            for (int k = 0; k < 8; ++k) gsp[k] = sc[k];
+        }
+        float4 *is = reinterpret_cast<float4 *>(inv + (size_t)o * 8u);
+        is[0] = make_float4(iv[0], iv[1], iv[2], iv[3]);
+        is[1] = make_float4(iv[4], iv[5], iv[6], iv[7]);
+    }
+    __syncthreads();
+    // pass 2: codes
+    const f32x2 magic2 = pack2(12582912.0f, 12582912.0f);
+    const f32x2 one2 = pack2(1.0f, 1.0f);
+    const unsigned long long plane_elem = ((unsigned long long)li * 2ull * (unsigned long long)op.T + t0) * RE;   // K plane, token t0
+    for (unsigned it = (unsigned)tid; it < items; it += (unsigned)kKcThreads) {
+        const unsigned q = it / octets, o = it - q * octets;
+        const unsigned ta = q * 16u, tb = ta + 16u < n_tok ? ta + 16u : n_tok;
+        const f32x2 i0 = lds_f32x2(inv + o * 8u), i1 = lds_f32x2(inv + o * 8u + 2u);
+        const f32x2 i2 = lds_f32x2(inv + o * 8u + 4u), i3 = lds_f32x2(inv + o * 8u + 6u);
+        for (unsigned t = ta; t < tb; ++t) {
+            const uint4 x = lds128(X + ((size_t)t * RE + (size_t)o * 8u) * 2u);
+            uint32_t r[8];
+            unpack2_bits(add2_unfused(mul2(bf16x2_to_f32x2(x.x), i0), magic2, one2), r[0], r[1]);
+            unpack2_bits(add2_unfused(mul2(bf16x2_to_f32x2(x.y), i1), magic2, one2), r[2], r[3]);
+            unpack2_bits(add2_unfused(mul2(bf16x2_to_f32x2(x.z), i2), magic2, one2), r[4], r[5]);
+            unpack2_bits(add2_unfused(mul2(bf16x2_to_f32x2(x.w), i3), magic2, one2), r[6], r[7]);
+            uint2 c;
+            c.x = pack_codes4(r[0], r[1], r[2], r[3]);
+            c.y = pack_codes4(r[4], r[5], r[6], r[7]);
+            const unsigned long long e = plane_elem + (unsigned long long)t * RE + (unsigned long long)o * 8u;
+            if (int4) {
+                const uint32_t a0 = c.x & 0x0f0f0f0fu, a1 = c.y & 0x0f0f0f0fu;
+                *reinterpret_cast<uint32_t *>(op.data + (e >> 1)) = __byte_perm(a0 | (a0 >> 4), a1 | (a1 >> 4), 0x6420);
+            } else {
+                *reinterpret_cast<uint2 *>(op.data + e) = c;
+            }
+        }
+    }
+}
 
 // Rotation table: row r, frequency i -> (cos, sin) of delta_r * theta_r^(-2i/D), evaluated in fp64 and
 // rounded once to fp32 (an fp32 angle would lose more than half a bf16 ulp at large position shifts).

@@ -15,7 +15,7 @@ from . import build as _build
 
 KDN_OK, KDN_E_INVAL, KDN_E_SHAPE, KDN_E_ALIGN, KDN_E_RANGE, KDN_E_UNSUPPORTED, KDN_E_CUDA, KDN_E_NOMEM, \
     KDN_E_TIMEOUT, KDN_E_NOTFOUND, KDN_E_CHECKSUM, KDN_E_IO = range(12)
-KDN_CODEC_RAW_BF16, KDN_CODEC_INT8_G64, KDN_CODEC_INT4_G64 = 0, 1, 2
+KDN_CODEC_RAW_BF16, KDN_CODEC_INT8_G64, KDN_CODEC_INT4_G64, KDN_CODEC_INT8_KC64, KDN_CODEC_INT4_KC64 = 0, 1, 2, 3, 4
 KDN_MEM_DEVICE, KDN_MEM_PINNED_HOST = 0, 1
 
 EXPORTS = ["kdn_create", "kdn_destroy", "kdn_pool_register", "kdn_chunk_bytes", "kdn_validate_xfer",

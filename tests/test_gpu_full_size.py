@@ -53,7 +53,7 @@ def test_8b_store_then_retrieve_64_chunks_of_512_tokens():
         d_src, d_dst = dev.table(src.reshape(-1)), dev.table(dst.reshape(-1))
         sample = [0, 29, 63]
         layers = list(range(shape.n_layers))
-        for codec in (RAW, INT8, INT4):
+        for codec in (RAW, INT8, INT4, oracle.INT4_KC64):
             cb = dev.K.kdn_chunk_bytes(dev.desc, T, codec)
             big = torch.empty(n_req * cb, dtype=torch.uint8, device=dev.dev)
             K = dev.K
