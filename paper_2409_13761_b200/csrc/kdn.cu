@@ -265,6 +265,22 @@ kdn_status launch_kernel(K kernel, int threads, unsigned grid, size_t smem, cuda
             granted = smem;
         }
     }
+    {
+        // the pipeline is written for CTAs that are all resident at once: never launch more than fit
+        static std::map<std::pair<std::pair<int, const void *>, size_t>, int> resident;
+        int device = 0;
+        KDN_CUDA(cudaGetDevice(&device));
+        std::lock_guard<std::mutex> lock(g_attr_mutex);
+        int &per_sm = resident[std::make_pair(std::make_pair(device, (const void *)kernel), smem)];
+        if (per_sm == 0) {
+            KDN_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem));
+            if (per_sm < 1) return KDN_E_UNSUPPORTED;
+        }
+        int sms = 0;
+        KDN_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
+        const unsigned long long cap = (unsigned long long)per_sm * (unsigned long long)sms;
+        if (grid > cap) grid = (unsigned)cap;
+    }
     if (overlap) {
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3(grid);
@@ -351,6 +367,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     const bool kc_decode = any_kc && OP != OP_STORE;
     if (kc_decode) unit = lcm_u(unit, row_elems);
     Shape def = default_shape(OP, any_coded, any_rot);
+    if (kc_decode) def = Shape{ 16384, 4, 2, 1, 1 };      // larger tiles: a key tile also loads a whole row of scales
     int tile_bytes = ctx->tuning.tile_bytes > 0 ? ctx->tuning.tile_bytes : def.tile_bytes;
     unsigned tile_elems = (unsigned)tile_bytes / 2u / unit * unit;
     if (tile_elems < unit) tile_elems = unit;

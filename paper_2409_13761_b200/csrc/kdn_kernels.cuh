@@ -30,6 +30,18 @@ constexpr int kLoaderWarp = 0;
 constexpr int kMaxGroups = 8;                 // compute groups per CTA; group g owns slots g, g + G, ...
 // A compute group is kGW warps (4 for ordinary tiles, 1 for row-sized tiles) that work together on one tile.
 __host__ __device__ constexpr int threads_for(int groups, int group_warps) { return 32 + groups * group_warps * 32 + 32; }  // loader + compute + storer
+// The launch shapes count on several CTAs per SM (eight of the two-single-warp-group form, three of the two-group
+// form, ...): every instantiation is held to about 64 registers a thread.
+__host__ __device__ constexpr int min_ctas_for(int groups, int group_warps)
+{
+    return 1024 / threads_for(groups, group_warps) > 0 ? 1024 / threads_for(groups, group_warps) : 1;
+}
+// The rotation needs more registers (eight frequencies of coefficients per thread) and its shapes fewer CTAs: four of
+// the one-group form, two of the two-group form.
+__host__ __device__ constexpr int min_ctas_for_compose(int groups, int group_warps)
+{
+    return group_warps != 4 ? min_ctas_for(groups, group_warps) : groups == 0 ? 16 : groups == 1 ? 4 : groups == 2 ? 2 : 1;
+}
 constexpr int kThreadsCopy = 64;                             // loader + storer
 constexpr int kMaxStages = 32;
 constexpr int kMaxStoreLag = 16;          // most bulk-store groups allowed to be still reading shared memory
@@ -939,17 +951,17 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
 // every waiter visits a barrier once per phase (a parity wait cannot tell phases two apart).
 // Sec. 3.2 call (i) store, Sec. 3.1 storage module: paged pool -> chunk, optional int8 coding.
 template <int kGroups, int kGW>
-__global__ void __launch_bounds__(threads_for(kGroups, kGW))
+__global__ void __launch_bounds__(threads_for(kGroups, kGW), min_ctas_for(kGroups, kGW))
 kdn_store_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_STORE, kGroups, kGW>(P); }
 
 // Sec. 3.2 call (ii) retrieve, Sec. 3.1 delivery module (decompression on the GPU): chunk -> pool.
 template <int kGroups, int kGW>
-__global__ void __launch_bounds__(threads_for(kGroups, kGW))
+__global__ void __launch_bounds__(threads_for(kGroups, kGW), min_ctas_for(kGroups, kGW))
 kdn_retrieve_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_RETRIEVE, kGroups, kGW>(P); }
 
 // Sec. 3.1 blending module: parts -> request blocks at new positions, keys re-rotated.
 template <int kGroups, int kGW>
-__global__ void __launch_bounds__(threads_for(kGroups, kGW))
+__global__ void __launch_bounds__(threads_for(kGroups, kGW), min_ctas_for_compose(kGroups, kGW))
 kdn_compose_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_COMPOSE, kGroups, kGW>(P); }
 
 // ------------------------------------------------ keys of the per-channel key codecs --
