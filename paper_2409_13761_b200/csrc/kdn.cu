@@ -481,9 +481,18 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
 
     if (kc_groups > 0) {
         // key planes of the per-channel key codecs: one CTA per (64-token group, layer, op)
-        const size_t kc_smem = kc_smem_bytes(row_elems);
+        // channels per CTA: at most 256 (36 KiB of shared memory, six CTAs per SM), a multiple of eight that divides the row
+        unsigned n_split = 1;
+        while (row_elems / n_split > 256u && row_elems % (n_split * 2u * 8u) == 0u) n_split *= 2u;
+        const unsigned cols = row_elems / n_split;
+        const size_t kc_smem = kc_smem_bytes(cols);
         if (kc_smem > smem_limit) return KDN_E_UNSUPPORTED;
+        unsigned kc_threads = (cols / 8u * kKcSlices + 31u) & ~31u;
+        if (kc_threads > 512u) kc_threads = 512u;
+        if (kc_threads < 64u) kc_threads = 64u;
         KcLaunch kp{};
+        kp.cols = cols;
+        kp.n_split = n_split;
         kp.ops = inl ? nullptr : slot->d_ops;
         kp.n_ops = n;
         kp.k_layers = pool.d_k;
@@ -500,7 +509,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
                 granted = kc_smem;
             }
         }
-        kdn_store_kc_kernel<<<dim3((unsigned)kc_groups, (unsigned)kc_layers, (unsigned)n), kKcThreads, kc_smem, stream>>>(kp);
+        kdn_store_kc_kernel<<<dim3((unsigned)kc_groups * n_split, (unsigned)kc_layers, (unsigned)n), kc_threads, kc_smem, stream>>>(kp);
         KDN_CUDA(cudaGetLastError());
         ctx->launches++;
     }

@@ -968,12 +968,15 @@ kdn_compose_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_COMPOSE,
 
 // Storing the key planes of a per-channel key codec needs, for every channel, the largest magnitude over 64 tokens
 // before the first code can be formed, so it does not fit the streaming tile pipeline.  One CTA takes one
-// (op, layer, 64-token group): the group's token rows (64 x row_elems bf16, contiguous per pool block) are brought into
-// shared memory with bulk copies; pass 1 reduces |x| per channel over four token slices; one thread per eight
-// channels combines the slices, forms scale and reciprocal (two IEEE divides per channel) and writes the scales;
-// pass 2 codes each element with its channel's reciprocal and writes the codes straight to the chunk.
-// The host guarantees: block_size divides 64, the op's token offset is a multiple of block_size, row_elems % 64 == 0.
-// Shared memory: 64 * row_elems * 2 (rows) + 4 * row_elems * 2 (slice maxima) + row_elems * 4 (reciprocals) + 16.
+// (op, layer, 64-token group, slice of `cols` channels): the slice of the group's token rows is brought into shared
+// memory with bulk copies (one per token row; one per pool block when the slice is the whole row); pass 1 reduces
+// |x| per channel over four token slices; one thread per eight channels combines them, forms scale and reciprocal
+// (two IEEE divides per channel) and writes the scales; pass 2 codes each element with its channel's reciprocal
+// and writes the codes straight to the chunk.  Several CTAs share an SM (the host picks `cols` so that they fit), so
+// one CTA's loads overlap the arithmetic of the others.
+// The host guarantees: block_size divides 64, the op's token offset is a multiple of block_size, row_elems % 64 == 0,
+// cols % 8 == 0 and cols divides row_elems.
+// Shared memory: 64 * cols * 2 (rows) + 4 * cols * 2 (slice maxima) + cols * 4 (reciprocals) + 16.
 struct KcLaunch {
     const DevOp *ops;         // device array, or nullptr: inline_ops
     int n_ops;
@@ -981,66 +984,93 @@ struct KcLaunch {
     long long n_blocks;
     int bs;
     unsigned row_elems;
+    unsigned cols;            // channels per CTA
+    unsigned n_split;         // row_elems / cols
     int *status;
     DevOp inline_ops[kInlineOps];
 };
 
-constexpr int kKcThreads = 512;
 constexpr unsigned kKcSlices = 4;                          // token slices of 16 tokens in pass 1 and pass 2
-__host__ __device__ inline size_t kc_smem_bytes(unsigned row_elems)
+__host__ __device__ inline size_t kc_smem_bytes(unsigned cols)
 {
-    return (size_t)64 * row_elems * 2u + (size_t)kKcSlices * row_elems * 2u + (size_t)row_elems * 4u + 16u;
+    return (size_t)64 * cols * 2u + (size_t)kKcSlices * cols * 2u + (size_t)cols * 4u + 16u;
 }
 
-__global__ void __launch_bounds__(kKcThreads) kdn_store_kc_kernel(const __grid_constant__ KcLaunch P)
+__global__ void __launch_bounds__(512) kdn_store_kc_kernel(const __grid_constant__ KcLaunch P)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const DevOp *ops = P.ops ? P.ops : P.inline_ops;
     const DevOp op = ops[blockIdx.z];
     if (op.codec < 3) return;
-    const unsigned g = blockIdx.x, li = blockIdx.y;
+    const unsigned g = blockIdx.x / P.n_split, part = blockIdx.x - g * P.n_split, li = blockIdx.y;
     const unsigned n_groups = ((unsigned)op.T + 63u) >> 6;
     if (g >= n_groups || li >= (unsigned)op.nl) return;
     const bool int4 = op.codec == 4;
     const float qmax = int4 ? 7.0f : 127.0f;
-    const unsigned RE = P.row_elems;
+    const unsigned RE = P.row_elems, C = P.cols, c0 = part * C;
     const unsigned t0 = g << 6;
     const unsigned n_tok = (unsigned)op.T - t0 < 64u ? (unsigned)op.T - t0 : 64u;
 
-    unsigned char *X = smem_raw;                                             // [n_tok][RE] bf16
-    unsigned char *pmax = X + (size_t)64 * RE * 2u;                          // [kKcSlices][RE] bf16 magnitudes
-    float *inv = reinterpret_cast<float *>(pmax + (size_t)kKcSlices * RE * 2u);   // [RE]
-    unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(reinterpret_cast<unsigned char *>(inv) + (size_t)RE * 4u);
+    unsigned char *X = smem_raw;                                             // [n_tok][C] bf16
+    unsigned char *pmax = X + (size_t)64 * C * 2u;                           // [kKcSlices][C] bf16 magnitudes
+    float *inv = reinterpret_cast<float *>(pmax + (size_t)kKcSlices * C * 2u);    // [C]
+    unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(reinterpret_cast<unsigned char *>(inv) + (size_t)C * 4u);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bar_mem + 1);
     const uint32_t bar = smem_u32(bar_mem);
     const int tid = (int)threadIdx.x;
+    const int nthreads = (int)blockDim.x;
 
     if (tid == 0) {
         mbar_init(bar, 1u);
         *abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
-        // the group's rows, block by block (a block's tokens are contiguous in the pool)
+    }
+    __syncthreads();
+    if (tid < 32) {
+        // warp 0 brings the rows in: lane r takes token rows r and r + 32
         const unsigned char *base = reinterpret_cast<const unsigned char *>(P.k_layers[op.l0 + (int)li]);
         const long long first_block = (op.off + (long long)t0) / P.bs;
+        long long id[2] = { 0, 0 };
         bool bad = false;
-        for (unsigned t = 0; t < n_tok && !bad; t += (unsigned)P.bs) {
-            const long long id = __ldg(op.table + first_block + t / (unsigned)P.bs);
-            if (id < 0 || id >= P.n_blocks) bad = true;
+#pragma unroll
+        for (int k = 0; k < 2; ++k) {
+            const unsigned t = (unsigned)tid + 32u * (unsigned)k;
+            if (t < n_tok) {
+                id[k] = __ldg(op.table + first_block + t / (unsigned)P.bs);
+                if (id[k] < 0 || id[k] >= P.n_blocks) bad = true;
+            }
         }
-        if (bad) {
-            atomicCAS(P.status, 0, kStatusRange);
-            *abort_flag = 1;                                                  // nothing is loaded, nothing is written
+        if (__any_sync(0xffffffffu, bad)) {
+            if (tid == 0) {
+                atomicCAS(P.status, 0, kStatusRange);
+                *abort_flag = 1;                                              // nothing is loaded, nothing is written
+            }
         } else {
-            mbar_arrive_expect_tx(bar, n_tok * RE * 2u);
-            for (unsigned t = 0; t < n_tok; t += (unsigned)P.bs) {
-                const unsigned k = n_tok - t < (unsigned)P.bs ? n_tok - t : (unsigned)P.bs;
-                const long long id = __ldg(op.table + first_block + t / (unsigned)P.bs);
-                const unsigned char *src = base + (unsigned long long)id * P.bs * RE * 2ull;
-                // pieces of at most 32 KiB
-                const unsigned bytes = k * RE * 2u;
-                for (unsigned o = 0; o < bytes; o += 32768u)
-                    bulk_g2s(smem_u32(X + (size_t)t * RE * 2u + o), src + o, bytes - o < 32768u ? bytes - o : 32768u, bar);
+            if (tid == 0) mbar_arrive_expect_tx(bar, n_tok * C * 2u);
+            __syncwarp();
+            if (P.n_split == 1u) {
+                // the whole row: a block's tokens are contiguous in the pool, one copy per block (pieces <= 32 KiB)
+                if (tid == 0) {
+                    for (unsigned t = 0; t < n_tok; t += (unsigned)P.bs) {
+                        const unsigned k = n_tok - t < (unsigned)P.bs ? n_tok - t : (unsigned)P.bs;
+                        const long long b = __ldg(op.table + first_block + t / (unsigned)P.bs);
+                        const unsigned char *src = base + (unsigned long long)b * P.bs * RE * 2ull;
+                        const unsigned bytes = k * RE * 2u;
+                        for (unsigned o = 0; o < bytes; o += 32768u)
+                            bulk_g2s(smem_u32(X + (size_t)t * RE * 2u + o), src + o, bytes - o < 32768u ? bytes - o : 32768u, bar);
+                    }
+                }
+            } else {
+#pragma unroll
+                for (int k = 0; k < 2; ++k) {
+                    const unsigned t = (unsigned)tid + 32u * (unsigned)k;
+                    if (t < n_tok) {
+                        const unsigned slot = (unsigned)((op.off + (long long)t0 + t) % P.bs);
+                        const unsigned char *src = base + (((unsigned long long)id[k] * P.bs + slot) * RE + c0) * 2ull;
+                        bulk_g2s(smem_u32(X + (size_t)t * C * 2u), src, C * 2u, bar);
+                    }
+                }
             }
         }
     }
@@ -1052,28 +1082,28 @@ __global__ void __launch_bounds__(kKcThreads) kdn_store_kc_kernel(const __grid_c
         return;
     }
 
-    const unsigned octets = RE >> 3;
+    const unsigned octets = C >> 3;
     const unsigned items = octets * kKcSlices;
     // pass 1: per (eight channels, token slice) the largest magnitudes, as packed bf16 pairs
-    for (unsigned it = (unsigned)tid; it < items; it += (unsigned)kKcThreads) {
+    for (unsigned it = (unsigned)tid; it < items; it += (unsigned)nthreads) {
         const unsigned q = it / octets, o = it - q * octets;
         const unsigned ta = q * 16u, tb = ta + 16u < n_tok ? ta + 16u : n_tok;
         uint32_t m0 = 0u, m1 = 0u, m2 = 0u, m3 = 0u;
         for (unsigned t = ta; t < tb; ++t) {
-            const uint4 x = lds128(X + ((size_t)t * RE + (size_t)o * 8u) * 2u);
+            const uint4 x = lds128(X + ((size_t)t * C + (size_t)o * 8u) * 2u);
             m0 = maxabs_bf16x2(m0, x.x); m1 = maxabs_bf16x2(m1, x.y);
             m2 = maxabs_bf16x2(m2, x.z); m3 = maxabs_bf16x2(m3, x.w);
         }
-        sts128(pmax + ((size_t)q * RE + (size_t)o * 8u) * 2u, make_uint4(m0, m1, m2, m3));
+        sts128(pmax + ((size_t)q * C + (size_t)o * 8u) * 2u, make_uint4(m0, m1, m2, m3));
     }
     __syncthreads();
     // scales: one thread per eight channels
     const unsigned long long per_layer = (unsigned long long)n_groups * RE + (((unsigned long long)op.T * RE) >> 6);
-    float *g_scales = reinterpret_cast<float *>(op.scales) + (unsigned long long)li * per_layer + (unsigned long long)g * RE;
-    for (unsigned o = (unsigned)tid; o < octets; o += (unsigned)kKcThreads) {
+    float *g_scales = reinterpret_cast<float *>(op.scales) + (unsigned long long)li * per_layer + (unsigned long long)g * RE + c0;
+    for (unsigned o = (unsigned)tid; o < octets; o += (unsigned)nthreads) {
         uint32_t m[4] = { 0u, 0u, 0u, 0u };
         for (unsigned q = 0; q < kKcSlices; ++q) {
-            const uint4 x = lds128(pmax + ((size_t)q * RE + (size_t)o * 8u) * 2u);
+            const uint4 x = lds128(pmax + ((size_t)q * C + (size_t)o * 8u) * 2u);
             m[0] = maxabs_bf16x2(m[0], x.x); m[1] = maxabs_bf16x2(m[1], x.y);
             m[2] = maxabs_bf16x2(m[2], x.z); m[3] = maxabs_bf16x2(m[3], x.w);
         }
@@ -1106,14 +1136,14 @@ __global__ void __launch_bounds__(kKcThreads) kdn_store_kc_kernel(const __grid_c
     // pass 2: codes
     const f32x2 magic2 = pack2(12582912.0f, 12582912.0f);
     const f32x2 one2 = pack2(1.0f, 1.0f);
-    const unsigned long long plane_elem = ((unsigned long long)li * 2ull * (unsigned long long)op.T + t0) * RE;   // K plane, token t0
-    for (unsigned it = (unsigned)tid; it < items; it += (unsigned)kKcThreads) {
+    const unsigned long long plane_elem = ((unsigned long long)li * 2ull * (unsigned long long)op.T + t0) * RE + c0;   // K plane, token t0
+    for (unsigned it = (unsigned)tid; it < items; it += (unsigned)nthreads) {
         const unsigned q = it / octets, o = it - q * octets;
         const unsigned ta = q * 16u, tb = ta + 16u < n_tok ? ta + 16u : n_tok;
         const f32x2 i0 = lds_f32x2(inv + o * 8u), i1 = lds_f32x2(inv + o * 8u + 2u);
         const f32x2 i2 = lds_f32x2(inv + o * 8u + 4u), i3 = lds_f32x2(inv + o * 8u + 6u);
         for (unsigned t = ta; t < tb; ++t) {
-            const uint4 x = lds128(X + ((size_t)t * RE + (size_t)o * 8u) * 2u);
+            const uint4 x = lds128(X + ((size_t)t * C + (size_t)o * 8u) * 2u);
             uint32_t r[8];
             unpack2_bits(add2_unfused(mul2(bf16x2_to_f32x2(x.x), i0), magic2, one2), r[0], r[1]);
             unpack2_bits(add2_unfused(mul2(bf16x2_to_f32x2(x.y), i1), magic2, one2), r[2], r[3]);
