@@ -31,7 +31,7 @@ def test_chunk_bytes_matches_oracle():
     for (L, H, D) in [(2, 2, 64), (32, 8, 128), (80, 8, 128), (1, 3, 8), (4, 1, 192), (2, 2, 96)]:
         d = K.pool_desc(L, H, D, 16, 64)
         for T in (0, 1, 17, 512, 2048):
-            for codec in (0, 1, 2):
+            for codec in (0, 1, 2, 3, 4):
                 assert K.kdn_chunk_bytes(d, T, codec) == oracle.chunk_bytes(L, H, D, T, codec), (L, H, D, T, codec)
     d = K.pool_desc(2, 2, 64, 16, 64)
     assert K.kdn_chunk_bytes(d, -1, 0) == 0
@@ -74,6 +74,19 @@ def test_validate_xfer_status_codes():
     assert K.kdn_validate_xfer(d96, [op]) == K.KDN_E_UNSUPPORTED                      # int8 needs head_dim % 64 == 0
     assert K.kdn_validate_xfer(K.pool_desc(2, 1, 4, 16, 64), [good_op(d)]) == K.KDN_E_ALIGN   # row of 8 bytes
     assert K.kdn_validate_xfer(K.pool_desc(0, 2, 64, 16, 64), []) == K.KDN_E_INVAL
+
+
+def test_validate_per_channel_key_codecs():
+    d = K.pool_desc(2, 2, 64, 16, 64)
+    for codec in (K.KDN_CODEC_INT8_KC64, K.KDN_CODEC_INT4_KC64):
+        assert K.kdn_validate_xfer(d, [good_op(d, T=20, off=0, codec=codec)]) == K.KDN_OK
+        assert K.kdn_validate_xfer(d, [good_op(d, T=10, off=16, codec=codec)]) == K.KDN_OK
+        assert K.kdn_validate_xfer(d, [good_op(d, T=20, off=3, codec=codec)]) == K.KDN_E_UNSUPPORTED     # not at a block start
+        assert K.kdn_validate_xfer(d, [good_op(d, T=0, off=3, n_table=1, codec=codec)]) == K.KDN_OK      # nothing to move
+    d3 = K.pool_desc(2, 2, 64, 3, 64)                                                                     # 3 does not divide 64
+    assert K.kdn_validate_xfer(d3, [good_op(d3, T=5, off=0, n_table=2, codec=K.KDN_CODEC_INT8_KC64)]) == K.KDN_E_UNSUPPORTED
+    d96 = K.pool_desc(2, 2, 96, 16, 64)                                                                   # head_dim % 64 != 0
+    assert K.kdn_chunk_bytes(d96, 4, K.KDN_CODEC_INT4_KC64) == 0
 
 
 def test_validate_compose_status_codes():
