@@ -180,8 +180,8 @@ class ClockSampler:
 # DRAM bytes (read + write) per launch from the committed ncu capture of a reduced case (8 chunks per
 # store/retrieve launch, 2 parts per compose launch; profiles/ncu_full_small_case_llama3_8b.md), scaled by the
 # units a bench launch processes.  Valid only for the kernel source the capture was taken from.
-NCU_KERNEL_SHA = "789bdf43c1b0116f"
-NCU_SMALL_CASE_BYTES = {"store_raw": (536.900608e6 + 485.395712e6, 8), "retrieve_raw": (536.921344e6 + 490.137088e6, 8), "compose_raw": (268.481280e6 + 221.714944e6, 2), "store_int8": (536.994048e6 + 249.219072e6, 8), "retrieve_int8": (285.334784e6 + 482.757888e6, 8), "compose_int8": (142.652160e6 + 214.158848e6, 2)}
+NCU_KERNEL_SHA = "f5ad9033593bf17b"
+NCU_SMALL_CASE_BYTES = {"store_raw": (536.918528e6 + 488.908544e6, 8), "retrieve_raw": (537.000192e6 + 493.293568e6, 8), "compose_raw": (268.492544e6 + 224.466176e6, 2), "store_int8": (536.922880e6 + 248.801536e6, 8), "retrieve_int8": (285.255680e6 + 482.879232e6, 8), "compose_int8": (142.663424e6 + 214.256896e6, 2)}
 
 
 def measured_traffic(op: str, units: float):
