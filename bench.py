@@ -418,7 +418,10 @@ def run_gpu(args) -> None:
     kc_ops = {}
 
     def key_error_db(codec_id, ops_set):
-        """Retrieve chunk 0 and compare layer 0's keys with their source blocks: signal-to-noise ratio in dB."""
+        """Retrieve chunk 0 and compare layer 0's keys with their source blocks: signal-to-noise ratio in dB.
+        Only where source and destination tables are disjoint (the 8B workload)."""
+        if not W["exclusive"]:
+            return None
         K.kdn_store(ctx, pid, ops_set["store"][:1], s)
         K.kdn_retrieve(ctx, pid, [K.XferOp(d_dst.data_ptr(), bpc, 0, ops_set["store"][0].chunk)], s)
         assert K.kdn_status_sync(ctx, s) == K.KDN_OK
@@ -482,6 +485,26 @@ def run_gpu(args) -> None:
         assert K.kdn_status_sync(ctx, s) == K.KDN_OK
         del buf
     torch.cuda.empty_cache()
+
+    # ---- one chunk per call: what a single retrieve costs (CUDA events around 50 back-to-back calls; not in `value`)
+    single_ops = {}
+    for codec, cname in ((RAW, "raw"), (INT8, "int8")):
+        one = dev_sets[codec]["retrieve"][:1]
+        for _ in range(5):
+            K.kdn_retrieve(ctx, pid, one, s)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        a.record(stream)
+        for _ in range(50):
+            K.kdn_retrieve(ctx, pid, one, s)
+        b.record(stream)
+        host_us = (time.perf_counter() - t0) / 50 * 1e6
+        torch.cuda.synchronize()
+        us = a.elapsed_time(b) / 50 * 1e3
+        nbytes = T * E * bytes_per_elem(codec)
+        single_ops["retrieve_one_chunk_" + cname] = {"us_per_call": us, "host_us_per_call": host_us, "gbs": nbytes / us / 1e3,
+                                                      "tokens": T, "bytes_moved": nbytes}
 
     # ---- file-backed chunks: a few chunks of the library written to and read back from one file (wall clock around
     # the call plus the stream sync, since the calling thread does the file I/O; not part of `value`)
@@ -618,7 +641,7 @@ def run_gpu(args) -> None:
                        "bytes_per_step": step_bytes},
             "tokens_per_s_reloaded": world * reload_tokens / (sum(op_ms[n] for n in names if not n.startswith("store")) * 1e-3),
             "ops": ops, "ops_int4_not_in_value": int4_ops, "ops_keep_list_not_in_value": sparse_ops, "ops_shell_not_in_value": shell_ops,
-            "ops_file_not_in_value": file_ops, "ops_per_channel_key_codecs_not_in_value": kc_ops,
+            "ops_file_not_in_value": file_ops, "ops_single_chunk_not_in_value": single_ops, "ops_per_channel_key_codecs_not_in_value": kc_ops,
             "roofline": {"bound": "hbm", "kernel": kernel_of[top], "op": top, "achieved": ops[top]["gbs"], "peak": peak,
                          "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": ops[top]["gbs"] / peak,
                          "frac_of_nominal_8000": ops[top]["gbs"] / 8000.0, "traffic": traffic},
