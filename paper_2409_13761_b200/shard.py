@@ -27,6 +27,19 @@ def shard_range(n: int, rank: int, world: int) -> range:
     return range(start, start + base + (1 if rank < extra else 0))
 
 
+def head_range(n_kv_heads: int, rank: int, world: int) -> range:
+    """The KV heads one rank of a tensor-parallel group holds: a contiguous, equal share.
+
+    Under tensor parallelism every rank's pool holds ``n_kv_heads / world`` heads of every block, and the rank stores,
+    retrieves and composes its own slice of every chunk with an ordinary pool descriptor of that many heads: a coding
+    group (64 elements along head_dim, or 64 tokens of one channel) never spans two heads, so the ranks' results are
+    exactly the head slices of the unsharded result and nothing is exchanged."""
+    if world < 1 or not 0 <= rank < world or n_kv_heads % world:
+        raise ValueError("the KV heads must divide evenly over the ranks")
+    per = n_kv_heads // world
+    return range(rank * per, (rank + 1) * per)
+
+
 def max_over_ranks(values: Sequence[float], device="cpu", group=None) -> list:
     """Element-wise maximum of a list of floats over all ranks (identity when not initialised)."""
     import torch.distributed as dist

@@ -66,3 +66,27 @@ def test_two_gloo_ranks_shard_chunks_without_any_exchange(tmp_path):
     for c, ch in got.items():                                       # and identical to the single-process result
         tab = np.random.default_rng(100 + c).permutation(64)[:2].astype(np.int32)
         assert np.array_equal(ch, oracle.store(pool, tab, 0, 8, oracle.INT8_G64))
+
+
+@pytest.mark.parametrize("codec", [oracle.RAW_BF16, oracle.INT8_G64, oracle.INT4_G64, oracle.INT8_KC64, oracle.INT4_KC64])
+def test_head_sharded_ranks_reproduce_the_unsharded_result(codec):
+    """Tensor-parallel sharding: each rank stores and retrieves its own heads with an ordinary descriptor; put side by
+    side along the head axis, the ranks' pools equal the pool of the unsharded retrieve (no exchange step)."""
+    shape = synth.TOY.with_(n_kv_heads=4, n_blocks=24, block_size=16)
+    k, v = synth.make_pool(shape, seed=17)
+    pool = synth.pool_to_numpy(k, v)
+    src, dst = np.arange(6, dtype=np.int32), np.arange(10, 16, dtype=np.int32)
+    off, T = 16, 70
+    full = np.zeros_like(pool)
+    oracle.retrieve(full, dst, off, T, codec, oracle.store(pool, src, off, T, codec))
+    world = 2
+    parts = []
+    for rank in range(world):
+        hs = shard.head_range(shape.n_kv_heads, rank, world)
+        mine = np.ascontiguousarray(pool[:, :, :, :, hs.start:hs.stop])
+        out = np.zeros_like(mine)
+        oracle.retrieve(out, dst, off, T, codec, oracle.store(mine, src, off, T, codec))
+        parts.append(out)
+    assert np.array_equal(np.concatenate(parts, axis=4), full)
+    with pytest.raises(ValueError):
+        shard.head_range(4, 0, 3)
