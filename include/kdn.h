@@ -45,8 +45,8 @@
  *   INT8_G64 / INT4_G64; the scales that follow them are, per layer, fp32 k_scales[ceil(T/64)][H*D] and then
  *   fp32 v_scales[T][H*D/64].  Same bytes per element as the G64 codecs when T is a multiple of 64.
  *   They need block_size to divide 64 and the chunk's first token to sit at the start of a block (token_offset, or
- *   part_dst_pos in kdn_compose, a multiple of block_size), else KDN_E_UNSUPPORTED; token lists, kdn_compose_static
- *   and pools with more than about 1600 elements per token row are not supported with them.
+ *   part_dst_pos in kdn_compose, a multiple of block_size), else KDN_E_UNSUPPORTED; token lists and kdn_compose_static
+ *   are not supported with them (KDN_E_UNSUPPORTED).
  * Key re-rotation in kdn_compose: the stored keys of a part carry rotary
  *   position embedding for positions base_pos + t; placing the part at
  *   dst_pos rotates each pair (k[i], k[i + D/2]) of every head by
