@@ -52,7 +52,43 @@ def lib():
     global _lib
     with _lock:
         if _lib is None:
-            L = C.CDLL(build())
+            _lib = _declare(C.CDLL(build()))
+    return _lib
+
+
+class use_library:
+    """Context manager for the pins' own self-check: run the wrappers of this module against another build of the
+    oracle (a copy with a planted mistake), then put the real one back."""
+
+    def __init__(self, path: str):
+        self.path = path
+
+    def __enter__(self):
+        global _lib
+        lib()
+        self.saved = _lib
+        _lib = _declare(C.CDLL(self.path))
+        return self
+
+    def __exit__(self, *exc):
+        global _lib
+        _lib = self.saved
+        return False
+
+
+def compile_source(source_text: str, out_path: str) -> str:
+    """Compile oracle source given as text (same flags as build()) to out_path."""
+    src = out_path + ".c"
+    with open(src, "w") as fh:
+        fh.write(source_text)
+    subprocess.run(["gcc", "-std=c99", "-O2", "-ffp-contract=off", "-fno-fast-math", "-fPIC", "-shared", "-w",
+                    "-o", out_path, src, "-lm"], check=True)
+    return out_path
+
+
+def _declare(L):
+    if True:
+        if True:
             i32, i64, f64, sz = C.c_int, C.c_int64, C.c_double, C.c_size_t
             vp = C.c_void_p
             L.kdn_oracle_bf16_to_f32.restype = C.c_float
@@ -99,8 +135,7 @@ def lib():
             L.kdn_oracle_key_hash.argtypes = [vp, sz]
             L.kdn_oracle_checksum.restype = C.c_uint64
             L.kdn_oracle_checksum.argtypes = [vp, sz]
-            _lib = L
-    return _lib
+    return L
 
 
 def _ptr(a: np.ndarray):
