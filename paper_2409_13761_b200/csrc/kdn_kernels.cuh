@@ -970,8 +970,8 @@ kdn_compose_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_COMPOSE,
 // before the first code can be formed, so it does not fit the streaming tile pipeline.  One CTA takes one
 // (op, layer, 64-token group, slice of `cols` channels): the slice of the group's token rows is brought into shared
 // memory with bulk copies (one per token row; one per pool block when the slice is the whole row); pass 1 reduces
-// |x| per channel over four token slices; one thread per eight channels combines them, forms scale and reciprocal
-// (two IEEE divides per channel) and writes the scales; pass 2 codes each element with its channel's reciprocal
+// |x| per channel over four token slices; one thread per channel combines them, forms scale and reciprocal
+// (two IEEE divides) and writes the scale; pass 2 codes each element with its channel's reciprocal
 // and writes the codes straight to the chunk.  Several CTAs share an SM (the host picks `cols` so that they fit), so
 // one CTA's loads overlap the arithmetic of the others.
 // The host guarantees: block_size divides 64, the op's token offset is a multiple of block_size, row_elems % 64 == 0,
@@ -1097,40 +1097,21 @@ __global__ void __launch_bounds__(512) kdn_store_kc_kernel(const __grid_constant
         sts128(pmax + ((size_t)q * C + (size_t)o * 8u) * 2u, make_uint4(m0, m1, m2, m3));
     }
     __syncthreads();
-    // scales: one thread per eight channels
+    // scales: one thread per channel (a layer's scales start wherever the previous layer's end, so only 4-byte
+    // alignment is certain: plain fp32 stores, consecutive channels on consecutive threads)
     const unsigned long long per_layer = (unsigned long long)n_groups * RE + (((unsigned long long)op.T * RE) >> 6);
     float *g_scales = reinterpret_cast<float *>(op.scales) + (unsigned long long)li * per_layer + (unsigned long long)g * RE + c0;
-    for (unsigned o = (unsigned)tid; o < octets; o += (unsigned)nthreads) {
-        uint32_t m[4] = { 0u, 0u, 0u, 0u };
+    for (unsigned ch = (unsigned)tid; ch < C; ch += (unsigned)nthreads) {
+        unsigned short mx = 0;
         for (unsigned q = 0; q < kKcSlices; ++q) {
-            const uint4 x = lds128(pmax + ((size_t)q * C + (size_t)o * 8u) * 2u);
-            m[0] = maxabs_bf16x2(m[0], x.x); m[1] = maxabs_bf16x2(m[1], x.y);
-            m[2] = maxabs_bf16x2(m[2], x.z); m[3] = maxabs_bf16x2(m[3], x.w);
+            const unsigned short v = *reinterpret_cast<const unsigned short *>(pmax + ((size_t)q * C + ch) * 2u) & 0x7fffu;
+            mx = v > mx ? v : mx;                                             // magnitudes of bf16 order like their bit patterns
         }
-        float sc[8], iv[8];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-            const float a_lo = __uint_as_float((m[k] << 16) & 0x7fffffffu), a_hi = __uint_as_float(m[k] & 0x7fff0000u);
-            float s_lo = __fdiv_rn(a_lo, qmax), s_hi = __fdiv_rn(a_hi, qmax);
-            const bool ok_lo = s_lo >= 1.17549435e-38f, ok_hi = s_hi >= 1.17549435e-38f;
-            sc[2 * k] = ok_lo ? s_lo : 0.0f;
-            sc[2 * k + 1] = ok_hi ? s_hi : 0.0f;
-            iv[2 * k] = ok_lo ? __fdiv_rn(qmax, a_lo) : 0.0f;
-            iv[2 * k + 1] = ok_hi ? __fdiv_rn(qmax, a_hi) : 0.0f;
-        }
-        // a layer's scales start wherever the previous layer's end: only 4-byte alignment is certain
-        float *gsp = g_scales + (size_t)o * 8u;
-        if ((reinterpret_cast<unsigned long long>(gsp) & 15ull) == 0ull) {
-            float4 *gs = reinterpret_cast<float4 *>(gsp);
-            gs[0] = make_float4(sc[0], sc[1], sc[2], sc[3]);
-            gs[1] = make_float4(sc[4], sc[5], sc[6], sc[7]);
-        } else {
-#pragma unroll
-            for (int k = 0; k < 8; ++k) gsp[k] = sc[k];
-        }
-        float4 *is = reinterpret_cast<float4 *>(inv + (size_t)o * 8u);
-        is[0] = make_float4(iv[0], iv[1], iv[2], iv[3]);
-        is[1] = make_float4(iv[4], iv[5], iv[6], iv[7]);
+        const float a = __uint_as_float((uint32_t)mx << 16);
+        const float sc = __fdiv_rn(a, qmax);
+        const bool ok = sc >= 1.17549435e-38f;                                // smallest normal fp32; false for NaN too
+        g_scales[ch] = ok ? sc : 0.0f;
+        inv[ch] = ok ? __fdiv_rn(qmax, a) : 0.0f;
     }
     __syncthreads();
     // pass 2: codes
