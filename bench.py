@@ -180,8 +180,8 @@ class ClockSampler:
 # DRAM bytes (read + write) per launch from the committed ncu capture of a reduced case (8 chunks per
 # store/retrieve launch, 2 parts per compose launch; profiles/ncu_full_small_case_llama3_8b.md), scaled by the
 # units a bench launch processes.  Valid only for the kernel source the capture was taken from.
-NCU_KERNEL_SHA = "f5ad9033593bf17b"
-NCU_SMALL_CASE_BYTES = {"store_raw": (536.918528e6 + 488.908544e6, 8), "retrieve_raw": (537.000192e6 + 493.293568e6, 8), "compose_raw": (268.492544e6 + 224.466176e6, 2), "store_int8": (536.922880e6 + 248.801536e6, 8), "retrieve_int8": (285.255680e6 + 482.879232e6, 8), "compose_int8": (142.663424e6 + 214.256896e6, 2)}
+NCU_KERNEL_SHA = "87ac4bdc4bfba822"
+NCU_SMALL_CASE_BYTES = {"store_raw": (536.904960e6 + 487.936512e6, 8), "retrieve_raw": (536.927232e6 + 490.151680e6, 8), "compose_raw": (268.491776e6 + 222.266368e6, 2), "store_int8": (536.923136e6 + 248.528896e6, 8), "retrieve_int8": (285.255936e6 + 482.943488e6, 8), "compose_int8": (142.667776e6 + 214.036992e6, 2)}
 
 
 def measured_traffic(op: str, units: float):
