@@ -12,6 +12,11 @@ group-64 codec:
               the ten parts re-rotated, a 256-token suffix left untouched              (one call)
 `value` is algorithmic GB/s over the step with every buffer resident in HBM; `e2e` is the same step with the
 chunks in page-locked host memory, so every byte crosses the host link inside the timed region.
+The same run then times, outside `value`: both ends of the chunk-length sweep (128- and 8192-token chunks, block_size
+16 and 32, both codecs, fully fragmented tables) and the largest configuration, Llama-3-70B-shaped KV (80 layers,
+library of 16 x 2048-token chunks, 32 requests x 4 chunks filling the 80 GiB pool, four of the retrievals reading
+their chunk from page-locked host memory on a side stream).  `roofline.per_op` lists every op of both workloads as
+[GB/s, fraction of the nominal 8000 GB/s], from the median CUDA-event time of the op over the timed steps.
 With --impl reference the CPU oracle is timed instead, on a bounded sample of the same workload.
 The line printed last on stdout is the JSON record.
 """
@@ -177,9 +182,9 @@ class ClockSampler:
                 "power_w_max": max(pw) if pw else None, "samples": len(sm), "reasons": sorted(reasons)}
 
 
-# DRAM bytes (read + write) per launch from the committed ncu capture of a reduced case (8 chunks per
-# store/retrieve launch, 2 parts per compose launch; profiles/ncu_full_small_case_llama3_8b.md), scaled by the
-# units a bench launch processes.  Valid only for the kernel source the capture was taken from.
+# DRAM bytes (read + write) per launch from a profiler capture of a reduced case (8 chunks per store/retrieve
+# launch, 2 parts per compose launch), scaled by the units a bench launch processes: every byte is touched once,
+# so traffic grows in proportion.  Valid only for the kernel source the capture was taken from (its hash).
 NCU_KERNEL_SHA = "87ac4bdc4bfba822"
 NCU_SMALL_CASE_BYTES = {"store_raw": (536.904960e6 + 487.936512e6, 8), "retrieve_raw": (536.927232e6 + 490.151680e6, 8), "compose_raw": (268.491776e6 + 222.266368e6, 2), "store_int8": (536.923136e6 + 248.528896e6, 8), "retrieve_int8": (285.255936e6 + 482.943488e6, 8), "compose_int8": (142.667776e6 + 214.036992e6, 2)}
 
@@ -205,132 +210,131 @@ def measured_hbm_peak():
         return FALLBACK_HBM_GBS, "fallback"
 
 
-def make_workload(args, synth):
-    """Sizes of one step.  llama3-8b is the benchmark workload; llama3-70b is the batched-retrieve configuration."""
-    if args.workload == "llama3-70b":
+def make_workload(name, args, synth):
+    """Sizes of one step.  llama3-8b is the workload `value` is measured on; llama3-70b is the batched configuration."""
+    if name == "llama3-70b":
         shape = synth.LLAMA3_70B
         assign = synth.assign_chunks(32, 4, 16)                       # 32 requests x 4 chunks out of a library of 16
-        w = dict(name="llama3-70b", shape=shape, lib=16, chunk_tokens=2048, retr=assign.reshape(-1), part_lib=16,
-                 part_tokens=2048, reqs=[list(map(int, row)) for row in assign], suffix=0, exclusive=False,
-                 text=("llama3-70b KV (L80 H8 D128 bf16, block_size 16, 16384-block pool): store a library of 16x2048 "
-                       "tokens, retrieve 32 requests x 4 chunks (fills the pool), compose the same 32x4 at cumulative "
-                       "offsets; raw bf16 and int8-g64, fully fragmented tables"))
-    else:
-        shape = synth.LLAMA3_8B
-        n_chunks, n_parts = args.chunks or N_CHUNKS, args.parts or N_PARTS
-        if args.pool_blocks:
-            shape = shape.with_(n_blocks=args.pool_blocks)
-        w = dict(name="llama3-8b", shape=shape, lib=n_chunks, chunk_tokens=CHUNK_TOKENS, retr=np.arange(n_chunks),
-                 part_lib=n_parts, part_tokens=PART_TOKENS, reqs=[list(range(n_parts))], suffix=SUFFIX_TOKENS,
-                 exclusive=True, text=WORKLOAD)
-        if args.pool_blocks or args.chunks or args.parts:
-            w["text"] = "REDUCED (%d chunks, %d parts, %d blocks): not the bench workload" % (n_chunks, n_parts, shape.n_blocks)
+        return dict(name="llama3-70b", shape=shape, lib=16, chunk_tokens=2048, retr=assign.reshape(-1), part_lib=16,
+                    part_tokens=2048, reqs=[list(map(int, row)) for row in assign], suffix=0, exclusive=False,
+                    text=("llama3-70b KV (L80 H8 D128 bf16, block_size 16, 16384-block pool): store a library of 16x2048 "
+                          "tokens, retrieve 32 requests x 4 chunks (fills the pool), compose the same 32x4 at cumulative "
+                          "offsets; raw bf16 and int8-g64, fully fragmented tables"))
+    shape = synth.LLAMA3_8B
+    n_chunks, n_parts = args.chunks or N_CHUNKS, args.parts or N_PARTS
+    if args.pool_blocks:
+        shape = shape.with_(n_blocks=args.pool_blocks)
+    w = dict(name="llama3-8b", shape=shape, lib=n_chunks, chunk_tokens=CHUNK_TOKENS, retr=np.arange(n_chunks),
+             part_lib=n_parts, part_tokens=PART_TOKENS, reqs=[list(range(n_parts))], suffix=SUFFIX_TOKENS,
+             exclusive=True, text=WORKLOAD)
+    if args.pool_blocks or args.chunks or args.parts:
+        w["text"] = "REDUCED (%d chunks, %d parts, %d blocks): not the bench workload" % (n_chunks, n_parts, shape.n_blocks)
     return w
 
 
-def run_gpu(args) -> None:
-    import torch
-    from paper_2409_13761_b200 import kdn as K, shard, synth
+NAMES = ["store_raw", "retrieve_raw", "compose_raw", "store_int8", "retrieve_int8", "compose_int8"]
 
-    rank, world, local = shard.rank_env()
-    dist = None
-    if world > 1 or "TORCHELASTIC_RUN_ID" in os.environ:        # launched by torch.distributed.run, even with one rank
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
-    torch.cuda.set_device(local)
-    dev = torch.device("cuda", local)
-    W = make_workload(args, synth)
-    shape = W["shape"]
-    T, PT, bs = W["chunk_tokens"], W["part_tokens"], shape.block_size
-    n_lib, n_retr, n_plib = W["lib"], len(W["retr"]), W["part_lib"]
-    n_parts_total = sum(len(r) for r in W["reqs"])
 
-    # ---- inputs (untimed): pool, tables, chunk buffers; every rank has its own copy of the same workload
-    k, v = synth.make_pool(shape, dev, seed=synth.SEED_VALUES + rank)
-    ctx = K.kdn_create(local)
-    desc = K.pool_desc(shape.n_layers, shape.n_kv_heads, shape.head_dim, shape.block_size, shape.n_blocks,
-                       [t.data_ptr() for t in k], [t.data_ptr() for t in v])
-    pid = K.kdn_pool_register(ctx, desc)
-    stream = torch.cuda.Stream(device=dev)
-    s = stream.cuda_stream
-    bpc, bpp = T // bs, PT // bs
-    req_blocks = [(len(r) * PT + W["suffix"]) // bs for r in W["reqs"]]
-    taken = np.zeros(0, dtype=np.int64)
+class Leg:
+    """One workload on one GPU: the pool, a library context, block tables, and the op lists of a step."""
 
-    def table(n, seed):
-        nonlocal taken
-        t = synth.make_table(n, shape.n_blocks, 1, seed, exclude=taken if W["exclusive"] else None)
+    def __init__(self, W, rank, local):
+        import torch
+        from paper_2409_13761_b200 import kdn as K, synth
+        self.torch, self.K, self.synth, self.W = torch, K, synth, W
+        self.dev = dev = torch.device("cuda", local)
+        self.local = local
+        shape = self.shape = W["shape"]
+        self.T, self.PT, self.bs = W["chunk_tokens"], W["part_tokens"], shape.block_size
+        self.n_lib, self.n_retr, self.n_plib = W["lib"], len(W["retr"]), W["part_lib"]
+        self.n_parts_total = sum(len(r) for r in W["reqs"])
+        # inputs (untimed): every rank has its own copy of the same workload
+        self.k, self.v = synth.make_pool(shape, dev, seed=synth.SEED_VALUES + rank)
+        self.ctx = K.kdn_create(local)
+        self.desc = K.pool_desc(shape.n_layers, shape.n_kv_heads, shape.head_dim, shape.block_size, shape.n_blocks,
+                                [t.data_ptr() for t in self.k], [t.data_ptr() for t in self.v])
+        self.pid = K.kdn_pool_register(self.ctx, self.desc)
+        self.stream = torch.cuda.Stream(device=dev)
+        self.s = self.stream.cuda_stream
+        self.bpc, self.bpp = self.T // self.bs, self.PT // self.bs
+        self.req_blocks = [(len(r) * self.PT + W["suffix"]) // self.bs for r in W["reqs"]]
+        self._taken = np.zeros(0, dtype=np.int64)
+        self.d_src = self._table(self.n_lib * self.bpc, synth.SEED_TABLES)        # where the library chunks are gathered from
+        self.d_dst = self._table(self.n_retr * self.bpc, synth.SEED_TABLES + 1)   # where retrievals land
+        self.d_part_src = self._table(self.n_plib * self.bpp, synth.SEED_TABLES + 2)
+        self.d_req = self._table(sum(self.req_blocks), synth.SEED_TABLES + 3)     # all composed requests, back to back
+        E = self.E = shape.elems_per_token
+        self.tokens_of = {"store": self.n_lib * self.T, "retrieve": self.n_retr * self.T, "compose": self.n_parts_total * self.PT}
+        self.op_tokens = {n: self.tokens_of[n.split("_")[0]] for n in NAMES}
+        self.op_bytes = {n: self.op_tokens[n] * E * bytes_per_elem(INT8 if n.endswith("int8") else RAW) for n in NAMES}
+        self.step_bytes = float(sum(self.op_bytes.values()))
+        self.reload_tokens = sum(self.op_tokens[n] for n in NAMES if not n.startswith("store"))
+        self.kernels = {}
+
+    def _table(self, n, seed):
+        W, shape = self.W, self.shape
+        t = self.synth.make_table(n, shape.n_blocks, 1, seed, exclude=self._taken if W["exclusive"] else None)
         if W["exclusive"]:
-            taken = np.concatenate([taken, t])
-        return torch.from_numpy(t).to(dev)
+            self._taken = np.concatenate([self._taken, t])
+        return self.torch.from_numpy(t).to(self.dev)
 
-    d_src = table(n_lib * bpc, synth.SEED_TABLES)                 # where the library chunks are gathered from
-    d_dst = table(n_retr * bpc, synth.SEED_TABLES + 1)            # where retrievals land
-    d_part_src = table(n_plib * bpp, synth.SEED_TABLES + 2)
-    d_req = table(sum(req_blocks), synth.SEED_TABLES + 3)         # all composed requests, back to back
-    i32 = 4
-
-    def make_sets(pinned_lib, pinned_retr=(), codecs=(RAW, INT8)):
+    def make_sets(self, pinned_lib, pinned_retr=(), codecs=(RAW, INT8)):
         """Chunk buffers and the op lists of one step, per codec.  pinned_lib: the whole library lives in page-locked
         host memory; pinned_retr: only these retrievals read a host copy of their chunk."""
+        K, torch, W, dev, desc = self.K, self.torch, self.W, self.dev, self.desc
+        T, PT, bpc, bpp, i32 = self.T, self.PT, self.bpc, self.bpp, 4
         sets = {}
         for codec in codecs:
             cb, pb = K.kdn_chunk_bytes(desc, T, codec), K.kdn_chunk_bytes(desc, PT, codec)
             if pinned_lib:
-                chunks = torch.empty(n_lib * cb, dtype=torch.uint8).pin_memory()
-                parts = torch.empty(n_plib * pb, dtype=torch.uint8).pin_memory()
+                chunks = torch.empty(self.n_lib * cb, dtype=torch.uint8).pin_memory()
+                parts = torch.empty(self.n_plib * pb, dtype=torch.uint8).pin_memory()
                 mem = K.KDN_MEM_PINNED_HOST
             else:
-                chunks = torch.empty(n_lib * cb, dtype=torch.uint8, device=dev)
-                parts = torch.empty(n_plib * pb, dtype=torch.uint8, device=dev)
+                chunks = torch.empty(self.n_lib * cb, dtype=torch.uint8, device=dev)
+                parts = torch.empty(self.n_plib * pb, dtype=torch.uint8, device=dev)
                 mem = K.KDN_MEM_DEVICE
             host_copy = {}
             for r in pinned_retr:
                 c = int(W["retr"][r])
                 if c not in host_copy:
                     host_copy[c] = torch.empty(cb, dtype=torch.uint8).pin_memory()
-            st_ops = [K.XferOp(d_src.data_ptr() + c * bpc * i32, bpc, 0,
-                               K.Chunk(chunks.data_ptr() + c * cb, cb, T, codec, mem)) for c in range(n_lib)]
+            st_ops = [K.XferOp(self.d_src.data_ptr() + c * bpc * i32, bpc, 0,
+                               K.Chunk(chunks.data_ptr() + c * cb, cb, T, codec, mem)) for c in range(self.n_lib)]
             rt_ops = []
             for r, c in enumerate(W["retr"]):
                 c = int(c)
                 ch = (K.Chunk(host_copy[c].data_ptr(), cb, T, codec, K.KDN_MEM_PINNED_HOST) if r in pinned_retr
                       else K.Chunk(chunks.data_ptr() + c * cb, cb, T, codec, mem))
-                rt_ops.append(K.XferOp(d_dst.data_ptr() + r * bpc * i32, bpc, 0, ch))
-            part_store = [K.XferOp(d_part_src.data_ptr() + j * bpp * i32, bpp, 0,
-                                   K.Chunk(parts.data_ptr() + j * pb, pb, PT, codec, mem)) for j in range(n_plib)]
+                rt_ops.append(K.XferOp(self.d_dst.data_ptr() + r * bpc * i32, bpc, 0, ch))
+            part_store = [K.XferOp(self.d_part_src.data_ptr() + j * bpp * i32, bpp, 0,
+                                   K.Chunk(parts.data_ptr() + j * pb, pb, PT, codec, mem)) for j in range(self.n_plib)]
             reqs, first = [], 0
-            for ids, nb_req in zip(W["reqs"], req_blocks):
-                reqs.append(K.ComposeReq(d_req.data_ptr() + first * i32, nb_req,
+            for ids, nb_req in zip(W["reqs"], self.req_blocks):
+                reqs.append(K.ComposeReq(self.d_req.data_ptr() + first * i32, nb_req,
                                          [K.Chunk(parts.data_ptr() + j * pb, pb, PT, codec, mem, 0) for j in ids],
-                                         [i * PT for i in range(len(ids))], shape.rope_theta))
+                                         [i * PT for i in range(len(ids))], self.shape.rope_theta))
                 first += nb_req
             sets[codec] = dict(chunks=chunks, parts=parts, host_copy=host_copy, store=st_ops, retrieve=rt_ops,
                                part_store=part_store, reqs=reqs)
         return sets
 
-    dev_sets = make_sets(False)
-    for codec in (RAW, INT8):                      # fill the compose parts once (untimed)
-        K.kdn_store(ctx, pid, dev_sets[codec]["part_store"], s)
-    assert K.kdn_status_sync(ctx, s) == K.KDN_OK
+    def fill_parts(self, sets, codecs=(RAW, INT8)):
+        for codec in codecs:                      # the compose parts are stored once (untimed)
+            self.K.kdn_store(self.ctx, self.pid, sets[codec]["part_store"], self.s)
+        self.check()
 
-    names = ["store_raw", "retrieve_raw", "compose_raw", "store_int8", "retrieve_int8", "compose_int8"]
-    E = shape.elems_per_token
-    tokens_of = {"store": n_lib * T, "retrieve": n_retr * T, "compose": n_parts_total * PT}
-    op_tokens = {n: tokens_of[n.split("_")[0]] for n in names}
-    op_bytes = {n: op_tokens[n] * E * bytes_per_elem(INT8 if n.endswith("int8") else RAW) for n in names}
-    step_bytes = float(sum(op_bytes.values()))
-    reload_tokens = sum(op_tokens[n] for n in names if not n.startswith("store"))
-    kernel_of = {"store_raw": "kdn_store_kernel<0, 4>", "retrieve_raw": "kdn_retrieve_kernel<0, 4>",
-                 "compose_raw": "kdn_compose_kernel<1, 4>", "store_int8": "kdn_store_kernel<2, 4>",
-                 "retrieve_int8": "kdn_retrieve_kernel<2, 4>", "compose_int8": "kdn_compose_kernel<3, 4>"}
+    def check(self):
+        st = self.K.kdn_status_sync(self.ctx, self.s)
+        assert st == self.K.KDN_OK, self.K.kdn_strerror(st)
 
-    def step(sets, events=None, kinds=("store", "retrieve", "compose")):
+    def step(self, sets, events=None, kinds=("store", "retrieve", "compose"), note_kernels=False):
+        K, ctx, pid, s = self.K, self.ctx, self.pid, self.s
         i = 0
-        for codec in (RAW, INT8):
+        for codec, cname in ((RAW, "raw"), (INT8, "int8")):
             for kind in ("store", "retrieve", "compose"):
                 if events is not None:
-                    events[i].record(stream)
+                    events[i].record(self.stream)
                 if kind not in kinds:
                     pass
                 elif kind == "store":
@@ -339,154 +343,146 @@ def run_gpu(args) -> None:
                     K.kdn_retrieve(ctx, pid, sets[codec]["retrieve"], s)
                 else:
                     K.kdn_compose(ctx, pid, sets[codec]["reqs"], s)
+                if note_kernels and kind in kinds:
+                    self.kernels[kind + "_" + cname] = K.kdn_last_launch(ctx)      # the instantiation the library chose
                 i += 1
         if events is not None:
-            events[i].record(stream)
+            events[i].record(self.stream)
 
-    def barrier():
-        if dist is not None:
-            dist.barrier()
+    def time_steps(self, sets, steps, warmup, barrier, sample_clocks=True):
+        """`steps` timed passes after `warmup` untimed ones.  Returns total ms, per-op ms (median over the steps of the
+        CUDA-event time of each op), kernels launched, clocks."""
+        torch, K = self.torch, self.K
+        self.step(sets, note_kernels=True)
+        for _ in range(max(0, warmup - 1)):
+            self.step(sets)
+        self.check()
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(NAMES) + 1)] for _ in range(steps)]
+        try:                                            # address the GPU by UUID: indices shift under CUDA_VISIBLE_DEVICES
+            gpu_id = "GPU-" + str(torch.cuda.get_device_properties(self.local).uuid)
+        except Exception:
+            gpu_id = str(self.local)
+        sampler = ClockSampler(gpu_id) if sample_clocks else None
+        barrier()
+        if sampler:
+            sampler.start()
+        launches0 = K.kdn_launch_count(self.ctx)
+        t_begin, t_end = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        t_begin.record(self.stream)
+        for it in range(steps):
+            self.step(sets, ev[it])
+        t_end.record(self.stream)
+        barrier()
+        clocks = sampler.stop() if sampler else None
+        launches = K.kdn_launch_count(self.ctx) - launches0
+        self.check()
+        per_op = {n: [ev[it][i].elapsed_time(ev[it][i + 1]) for it in range(steps)] for i, n in enumerate(NAMES)}
+        op_ms = {n: float(np.median(per_op[n])) for n in NAMES}
+        return t_begin.elapsed_time(t_end), op_ms, int(launches), clocks
+
+    def timed(self, fn, reps, warm=3):
+        """Mean CUDA-event milliseconds of `reps` back-to-back calls of fn() after `warm` untimed ones."""
+        torch = self.torch
+        for _ in range(warm):
+            fn()
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record(self.stream)
+        for _ in range(reps):
+            fn()
+        b.record(self.stream)
         torch.cuda.synchronize()
+        return a.elapsed_time(b) / reps
 
-    # ---- device-resident timing
-    for _ in range(args.warmup):
-        step(dev_sets)
-    assert K.kdn_status_sync(ctx, s) == K.KDN_OK
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(len(names) + 1)] for _ in range(args.steps)]
-    try:                                            # address the GPU by UUID: indices shift under CUDA_VISIBLE_DEVICES
-        gpu_id = "GPU-" + str(torch.cuda.get_device_properties(local).uuid)
-    except Exception:
-        gpu_id = str(local)
-    sampler = ClockSampler(gpu_id)
-    barrier()
-    sampler.start()
-    launches0 = K.kdn_launch_count(ctx)
-    t_begin = torch.cuda.Event(enable_timing=True)
-    t_end = torch.cuda.Event(enable_timing=True)
-    t_begin.record(stream)
-    for it in range(args.steps):
-        step(dev_sets, ev[it])
-    t_end.record(stream)
-    barrier()
-    clocks = sampler.stop()
-    launches = K.kdn_launch_count(ctx) - launches0
-    status = K.kdn_status_sync(ctx, s)
-    assert status == K.KDN_OK, K.kdn_strerror(status)
-    elapsed_ms = t_begin.elapsed_time(t_end)
-    op_ms = {n: float(np.mean([ev[it][i].elapsed_time(ev[it][i + 1]) for it in range(args.steps)]))
-             for i, n in enumerate(names)}
+    def close(self):
+        self.torch.cuda.synchronize()
+        self.K.kdn_destroy(self.ctx)
+        self.ctx = None
+        self.k = self.v = None
+        self.d_src = self.d_dst = self.d_part_src = self.d_req = None
+        self.torch.cuda.empty_cache()
 
-    # ---- storage shell: payload checksum over the raw chunk library (read-only stream; not part of `value`)
+
+def extras_8b(leg, dev_sets, reps):
+    """Widenings beyond the benchmark step, each timed on its own on the 8B workload (none is part of `value`)."""
+    torch, K, synth = leg.torch, leg.K, leg.synth
+    ctx, pid, s, dev, desc, shape, W = leg.ctx, leg.pid, leg.s, leg.dev, leg.desc, leg.shape, leg.W
+    T, E, bpc, i32, n_lib = leg.T, leg.E, leg.bpc, 4, leg.n_lib
+    out = {}
+
+    # storage shell: payload checksum over the raw chunk library (a read-only stream)
     lib_buf = dev_sets[RAW]["chunks"]
     csum_out = torch.zeros(1, dtype=torch.int64, device=dev)
-    for _ in range(3):
-        K.kdn_checksum(local, lib_buf.data_ptr(), lib_buf.numel(), csum_out.data_ptr(), s)
-    a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    reps = max(1, min(args.steps, 20))
-    a.record(stream)
-    for _ in range(reps):
-        K.kdn_checksum(local, lib_buf.data_ptr(), lib_buf.numel(), csum_out.data_ptr(), s)
-    b.record(stream)
-    torch.cuda.synchronize()
-    shell_ops = {"checksum_raw_library": {"ms": a.elapsed_time(b) / reps, "bytes": lib_buf.numel(),
-                                          "gbs": lib_buf.numel() / (a.elapsed_time(b) / reps * 1e-3) / 1e9}}
+    ms = leg.timed(lambda: K.kdn_checksum(leg.local, lib_buf.data_ptr(), lib_buf.numel(), csum_out.data_ptr(), s), reps)
+    out["ops_shell_not_in_value"] = {"checksum_raw_library": {"ms": ms, "bytes": lib_buf.numel(), "gbs": lib_buf.numel() / (ms * 1e-3) / 1e9}}
 
-    # ---- the int4 codec (a widening beyond the benchmark step; timed on its own, not part of `value`)
+    def three(sets, codec, cname, dst):
+        leg.K.kdn_store(ctx, pid, sets["part_store"], s)
+        for name, fn, arg in (("store_" + cname, K.kdn_store, sets["store"]), ("retrieve_" + cname, K.kdn_retrieve, sets["retrieve"]),
+                              ("compose_" + cname, K.kdn_compose, sets["reqs"])):
+            ms = leg.timed(lambda: fn(ctx, pid, arg, s), reps)
+            tok = leg.tokens_of[name.split("_")[0]]
+            nbytes = tok * E * bytes_per_elem(codec)
+            dst[name] = {"ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9, "tokens_per_s": tok / (ms * 1e-3),
+                         "kernel": K.kdn_last_launch(ctx)["kernel"]}
+        leg.check()
+
+    # the int4 codec
     int4_ops = {}
-    i4 = make_sets(False, codecs=(INT4,))[INT4]
-    K.kdn_store(ctx, pid, i4["part_store"], s)
-    for name, fn, arg in (("store_int4", K.kdn_store, i4["store"]), ("retrieve_int4", K.kdn_retrieve, i4["retrieve"]),
-                          ("compose_int4", K.kdn_compose, i4["reqs"])):
-        for _ in range(3):
-            fn(ctx, pid, arg, s)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        reps = max(1, min(args.steps, 20))
-        a.record(stream)
-        for _ in range(reps):
-            fn(ctx, pid, arg, s)
-        b.record(stream)
-        torch.cuda.synchronize()
-        ms = a.elapsed_time(b) / reps
-        nbytes = tokens_of[name.split("_")[0]] * E * bytes_per_elem(INT4)
-        int4_ops[name] = {"ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9, "tokens_per_s": tokens_of[name.split("_")[0]] / (ms * 1e-3)}
-    assert K.kdn_status_sync(ctx, s) == K.KDN_OK
-    del i4
-    torch.cuda.empty_cache()
+    i4 = leg.make_sets(False, codecs=(INT4,))[INT4]
+    three(i4, INT4, "int4", int4_ops)
+    out["ops_int4_not_in_value"] = int4_ops
 
-    # ---- per-channel key codecs (keys grouped along tokens; timed on their own, not part of `value`), and what they
-    # buy: the error of the stored keys, over all channels and over the channels without the x20 outlier gain
-    kc_ops = {}
-
-    def key_error_db(codec_id, ops_set):
-        """Retrieve chunk 0 and compare layer 0's keys with their source blocks: signal-to-noise ratio in dB.
-        Only where source and destination tables are disjoint (the 8B workload)."""
+    # per-channel key codecs, and what they buy: the error of the stored keys, over all channels and over the channels
+    # without the x20 outlier gain
+    def key_error_db(ops_set):
+        """Retrieve chunk 0 and compare layer 0's keys with their source blocks: signal-to-noise ratio in dB."""
         if not W["exclusive"]:
             return None
         K.kdn_store(ctx, pid, ops_set["store"][:1], s)
-        K.kdn_retrieve(ctx, pid, [K.XferOp(d_dst.data_ptr(), bpc, 0, ops_set["store"][0].chunk)], s)
-        assert K.kdn_status_sync(ctx, s) == K.KDN_OK
-        x = k[0][d_src[:bpc].long()].float().reshape(-1, shape.row_elems)
-        y = k[0][d_dst[:bpc].long()].float().reshape(-1, shape.row_elems)
+        K.kdn_retrieve(ctx, pid, [K.XferOp(leg.d_dst.data_ptr(), bpc, 0, ops_set["store"][0].chunk)], s)
+        leg.check()
+        x = leg.k[0][leg.d_src[:bpc].long()].float().reshape(-1, shape.row_elems)
+        y = leg.k[0][leg.d_dst[:bpc].long()].float().reshape(-1, shape.row_elems)
         ordinary = (synth.outlier_gain(shape)[0, 0].reshape(-1) == 1).to(dev)
         snr = lambda a, b: float(10 * torch.log10((a * a).mean() / ((a - b) ** 2).mean()))
         return {"all_channels": snr(x, y), "ordinary_channels": snr(x[:, ordinary], y[:, ordinary])}
 
-    quality = {"int4_g64": key_error_db(INT4, make_sets(False, codecs=(INT4,))[INT4]),
-               "int8_g64": key_error_db(INT8, dev_sets[INT8])}
+    kc_ops = {}
+    quality = {"int4_g64": key_error_db(i4), "int8_g64": key_error_db(dev_sets[INT8])}
+    del i4
+    torch.cuda.empty_cache()
     for codec, cname in ((INT8KC, "int8kc"), (INT4KC, "int4kc")):
-        kc = make_sets(False, codecs=(codec,))[codec]
-        K.kdn_store(ctx, pid, kc["part_store"], s)
-        for name, fn, arg in (("store_" + cname, K.kdn_store, kc["store"]), ("retrieve_" + cname, K.kdn_retrieve, kc["retrieve"]),
-                              ("compose_" + cname, K.kdn_compose, kc["reqs"])):
-            for _ in range(3):
-                fn(ctx, pid, arg, s)
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            reps = max(1, min(args.steps, 20))
-            a.record(stream)
-            for _ in range(reps):
-                fn(ctx, pid, arg, s)
-            b.record(stream)
-            torch.cuda.synchronize()
-            ms = a.elapsed_time(b) / reps
-            nbytes = tokens_of[name.split("_")[0]] * E * bytes_per_elem(codec)
-            kc_ops[name] = {"ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9, "tokens_per_s": tokens_of[name.split("_")[0]] / (ms * 1e-3)}
-        assert K.kdn_status_sync(ctx, s) == K.KDN_OK
-        quality[cname] = key_error_db(codec, kc)
+        kc = leg.make_sets(False, codecs=(codec,))[codec]
+        three(kc, codec, cname, kc_ops)
+        quality[cname] = key_error_db(kc)
         del kc
         torch.cuda.empty_cache()
     kc_ops["stored_key_snr_db"] = quality
+    out["ops_per_channel_key_codecs_not_in_value"] = kc_ops
 
-    # ---- keep-lists: every chunk holds a seeded random half of its span's tokens (timed on its own, not in `value`)
+    # keep-lists: every chunk holds a seeded random half of its span's tokens
     sparse_ops = {}
     rng = np.random.default_rng(synth.SEED_ASSIGN)
     n_keep = T // 2
     keep_np = np.stack([np.sort(rng.choice(T, n_keep, replace=False)) for _ in range(n_lib)]).astype(np.int32)
     d_keep = torch.from_numpy(keep_np).to(dev)
-    for codec, cname in ((RAW, "raw"), (INT8, "int8")):
+    for codec, cname in ((RAW, "raw"), (INT8, "int8"), (INT4, "int4")):
         cb = K.kdn_chunk_bytes(desc, n_keep, codec)
         buf = torch.empty(n_lib * cb, dtype=torch.uint8, device=dev)
         keeps = [d_keep.data_ptr() + c * n_keep * i32 for c in range(n_lib)]
-        st_ops = [K.XferOp(d_src.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(buf.data_ptr() + c * cb, cb, n_keep, codec)) for c in range(n_lib)]
-        rt_ops = [K.XferOp(d_dst.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(buf.data_ptr() + c * cb, cb, n_keep, codec)) for c in range(n_lib)]
+        st_ops = [K.XferOp(leg.d_src.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(buf.data_ptr() + c * cb, cb, n_keep, codec)) for c in range(n_lib)]
+        rt_ops = [K.XferOp(leg.d_dst.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(buf.data_ptr() + c * cb, cb, n_keep, codec)) for c in range(n_lib)]
         for name, fn, arg in (("store_sparse_" + cname, K.kdn_store_sparse, st_ops), ("retrieve_sparse_" + cname, K.kdn_retrieve_sparse, rt_ops)):
-            for _ in range(3):
-                fn(ctx, pid, arg, keeps, s)
-            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            reps = max(1, min(args.steps, 20))
-            a.record(stream)
-            for _ in range(reps):
-                fn(ctx, pid, arg, keeps, s)
-            b.record(stream)
-            torch.cuda.synchronize()
-            ms = a.elapsed_time(b) / reps
+            ms = leg.timed(lambda: fn(ctx, pid, arg, keeps, s), reps)
             nbytes = n_lib * n_keep * E * bytes_per_elem(codec)
             sparse_ops[name] = {"ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9, "tokens_per_s": n_lib * n_keep / (ms * 1e-3),
                                 "kept": "%d of %d tokens per chunk, seeded random" % (n_keep, T)}
-        assert K.kdn_status_sync(ctx, s) == K.KDN_OK
+        leg.check()
         del buf
     torch.cuda.empty_cache()
+    out["ops_keep_list_not_in_value"] = sparse_ops
 
-    # ---- one chunk per call: what a single retrieve costs (CUDA events around 50 back-to-back calls; not in `value`)
+    # one chunk per call: what a single retrieve costs (CUDA events around 50 back-to-back calls)
     single_ops = {}
     for codec, cname in ((RAW, "raw"), (INT8, "int8")):
         one = dev_sets[codec]["retrieve"][:1]
@@ -495,113 +491,87 @@ def run_gpu(args) -> None:
         a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         torch.cuda.synchronize()
         t0 = time.perf_counter()
-        a.record(stream)
+        a.record(leg.stream)
         for _ in range(50):
             K.kdn_retrieve(ctx, pid, one, s)
-        b.record(stream)
+        b.record(leg.stream)
         host_us = (time.perf_counter() - t0) / 50 * 1e6
         torch.cuda.synchronize()
         us = a.elapsed_time(b) / 50 * 1e3
         nbytes = T * E * bytes_per_elem(codec)
-        single_ops["retrieve_one_chunk_" + cname] = {"us_per_call": us, "host_us_per_call": host_us, "gbs": nbytes / us / 1e3,
+        single_ops["retrieve_one_chunk_" + cname] = {"us_per_call": us, "host_us_per_call_through_python": host_us, "gbs": nbytes / us / 1e3,
                                                       "tokens": T, "bytes_moved": nbytes}
+    out["ops_single_chunk_not_in_value"] = single_ops
 
-    # ---- file-backed chunks: a few chunks of the library written to and read back from one file (wall clock around
-    # the call plus the stream sync, since the calling thread does the file I/O; not part of `value`)
+    # file-backed chunks: a few chunks of the library written to and read back from files (wall clock around the call
+    # plus the stream sync, since the calling thread does the file I/O)
     file_ops = {}
     import tempfile
     tmpdir = "/dev/shm" if os.path.isdir("/dev/shm") and os.access("/dev/shm", os.W_OK) else None
     n_file = min(8, n_lib)
     for codec, cname in ((RAW, "raw"), (INT8, "int8")):
         cb = K.kdn_chunk_bytes(desc, T, codec)
-        with tempfile.NamedTemporaryFile(dir=tmpdir, prefix="kdn_bench_") as tf:
-            fd = tf.fileno()
-            st_ops = [K.XferOp(d_src.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(0, cb, T, codec)) for c in range(n_file)]
-            rt_ops = [K.XferOp(d_dst.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(0, cb, T, codec)) for c in range(n_file)]
-            offs = [c * cb for c in range(n_file)]
-            for name, fn, arg in (("store_file_" + cname, K.kdn_store_file, st_ops), ("retrieve_file_" + cname, K.kdn_retrieve_file, rt_ops)):
-                best = None
-                for _ in range(3):
-                    torch.cuda.synchronize()
-                    t0 = time.perf_counter()
-                    fn(ctx, pid, arg, [fd] * n_file, offs, s)
-                    assert K.kdn_status_sync(ctx, s) == K.KDN_OK
-                    dt = time.perf_counter() - t0
-                    best = dt if best is None else min(best, dt)
-                file_ops[name] = {"ms": best * 1e3, "file_gbs": n_file * cb / best / 1e9, "file_bytes": n_file * cb,
-                                  "where": "tmpfs" if tmpdir else "default temporary directory (page cache)"}
+        st_ops = [K.XferOp(leg.d_src.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(0, cb, T, codec)) for c in range(n_file)]
+        rt_ops = [K.XferOp(leg.d_dst.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(0, cb, T, codec)) for c in range(n_file)]
+        for layout in ("one_file", "file_per_chunk"):
+            files = [tempfile.NamedTemporaryFile(dir=tmpdir, prefix="kdn_bench_") for _ in range(1 if layout == "one_file" else n_file)]
+            try:
+                fds = [files[0].fileno()] * n_file if layout == "one_file" else [f.fileno() for f in files]
+                offs = [c * cb for c in range(n_file)] if layout == "one_file" else [0] * n_file
+                for name, fn, arg in (("store_file_" + cname, K.kdn_store_file, st_ops), ("retrieve_file_" + cname, K.kdn_retrieve_file, rt_ops)):
+                    best = None
+                    for _ in range(3):
+                        torch.cuda.synchronize()
+                        t0 = time.perf_counter()
+                        fn(ctx, pid, arg, fds, offs, s)
+                        leg.check()
+                        dt = time.perf_counter() - t0
+                        best = dt if best is None else min(best, dt)
+                    file_ops[name + "_" + layout] = {"ms": best * 1e3, "file_gbs": n_file * cb / best / 1e9, "file_bytes": n_file * cb,
+                                                     "where": "tmpfs" if tmpdir else "default temporary directory (page cache)"}
+            finally:
+                for f in files:
+                    f.close()
+    out["ops_file_not_in_value"] = file_ops
+    return out
 
-    if args.no_e2e:
-        if rank == 0:
-            print(json.dumps({"note": "profiling run, not a bench record", "ops_ms": op_ms,
-                              "ops_gbs": {n: op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 for n in names}, "int4": int4_ops, "sparse": sparse_ops, "shell": shell_ops, "file": file_ops, "kc": kc_ops}))
-        K.kdn_destroy(ctx)
-        return
 
-    # ---- end to end: chunks in page-locked host memory, every byte crosses the host link inside the timed region
-    e2e_steps = max(1, min(args.steps, args.e2e_steps))
-    if W["name"] == "llama3-8b":
-        # the whole step with the entire library on the host
-        del dev_sets
-        torch.cuda.empty_cache()
-        host_sets = make_sets(True)
-        e2e_kinds = ("store", "retrieve", "compose")
-        for codec in (RAW, INT8):
-            K.kdn_store(ctx, pid, host_sets[codec]["part_store"], s)
-        e2e_bytes = step_bytes
-        d2h = sum(K.kdn_chunk_bytes(desc, T, c) * n_lib for c in (RAW, INT8)) + 4
-        h2d = sum(K.kdn_chunk_bytes(desc, T, c) * n_retr + K.kdn_chunk_bytes(desc, PT, c) * n_parts_total for c in (RAW, INT8))
-        e2e_what = "whole step, every chunk in page-locked host memory"
-    else:
-        # the batched retrieve with four of its chunks on the host, copied in on the side stream while the
-        # device-resident retrievals run
-        pinned_retr = (5, 50, 90, 120)
-        host_sets = make_sets(False, pinned_retr)
-        for codec in (RAW, INT8):
-            host_sets[codec]["chunks"].copy_(dev_sets[codec]["chunks"])
-            for c, hb in host_sets[codec]["host_copy"].items():
-                cb = hb.numel()
-                hb.copy_(dev_sets[codec]["chunks"][c * cb:(c + 1) * cb])
-        e2e_kinds = ("retrieve",)
-        e2e_bytes = op_bytes["retrieve_raw"] + op_bytes["retrieve_int8"]
-        d2h = 4
-        h2d = sum(K.kdn_chunk_bytes(desc, T, c) * len(pinned_retr) for c in (RAW, INT8))
-        e2e_what = "batched retrieve, 4 of %d chunks in page-locked host memory (side stream)" % n_retr
-    assert K.kdn_status_sync(ctx, s) == K.KDN_OK
-    step(host_sets, kinds=e2e_kinds)
-    assert K.kdn_status_sync(ctx, s) == K.KDN_OK
-    layerwise = None
-    if W["name"] != "llama3-8b":
-        # layer-wise delivery of one host-resident chunk: when is the first layer range usable, when the last?
-        layerwise = {}
-        r0 = pinned_retr[0]
-        for codec, cname in ((RAW, "raw"), (INT8, "int8")):
-            op = [host_sets[codec]["retrieve"][r0]]
-            for mode, lps in (("whole", shape.n_layers), ("by_8_layers", 8)):
-                evs = [torch.cuda.Event(enable_timing=True) for _ in range(shape.n_layers)]
-                t_start = torch.cuda.Event(enable_timing=True)
-                for e in evs + [t_start]:
-                    e.record(stream)
-                torch.cuda.synchronize()
-                K.kdn_retrieve_layerwise(ctx, pid, op, lps, s, 0, [e.cuda_event for e in evs])   # warm
-                torch.cuda.synchronize()
-                t_start.record(stream)
-                K.kdn_retrieve_layerwise(ctx, pid, op, lps, s, 0, [e.cuda_event for e in evs])
-                torch.cuda.synchronize()
-                layerwise["%s_%s" % (cname, mode)] = {"first_layers_ready_ms": t_start.elapsed_time(evs[min(lps, shape.n_layers) - 1]),
-                                                      "all_layers_ready_ms": t_start.elapsed_time(evs[-1]),
-                                                      "chunk_bytes": K.kdn_chunk_bytes(desc, T, codec)}
-        assert K.kdn_status_sync(ctx, s) == K.KDN_OK
-    barrier()
-    t0 = time.perf_counter()
-    for _ in range(e2e_steps):
-        step(host_sets, kinds=e2e_kinds)
-        st = K.kdn_status_sync(ctx, s)            # the step's result is read back: device status + all copies landed
-        assert st == K.KDN_OK
-    barrier()
-    e2e_ms = (time.perf_counter() - t0) * 1e3
+def sweep_extract(leg, reps):
+    """Both ends of the chunk-length sweep on the 8B pool: chunk length {128, 8192} x block_size {16, 32} x codec {raw,
+    int8-g64}, fully fragmented tables, store and retrieve, each point batching enough distinct chunks to move >= 2 GiB."""
+    torch, K, synth = leg.torch, leg.K, leg.synth
+    shape, dev, s = leg.shape, leg.dev, leg.s
+    E = leg.E
+    arena = torch.empty((2 << 30) + (256 << 20), dtype=torch.uint8, device=dev)
+    points = []
+    for bs in (16, 32):
+        nb = shape.n_blocks * shape.block_size // bs
+        desc = K.pool_desc(shape.n_layers, shape.n_kv_heads, shape.head_dim, bs, nb,
+                           [t.data_ptr() for t in leg.k], [t.data_ptr() for t in leg.v])      # same memory, other block size
+        pid = K.kdn_pool_register(leg.ctx, desc)
+        for T in (128, 8192):
+            for codec in (RAW, INT8):
+                bpe = bytes_per_elem(codec)
+                n = max(1, -(-(2 << 30) // int(T * E * bpe)))
+                cb = K.kdn_chunk_bytes(desc, T, codec)
+                blocks = -(-T // bs)
+                src = synth.make_table(n * blocks, nb, 1, synth.SEED_TABLES)
+                dst = synth.make_table(n * blocks, nb, 1, synth.SEED_TABLES + 1, exclude=src)
+                d_src, d_dst = torch.from_numpy(src).to(dev), torch.from_numpy(dst).to(dev)
+                row = {"block_size": bs, "chunk_tokens": T, "codec": "int8" if codec else "raw", "chunks": n}
+                for name, fn, tab in (("store", K.kdn_store, d_src), ("retrieve", K.kdn_retrieve, d_dst)):
+                    ops = [K.XferOp(tab.data_ptr() + i * blocks * 4, blocks, 0, K.Chunk(arena.data_ptr() + i * cb, cb, T, codec)) for i in range(n)]
+                    ms = leg.timed(lambda: fn(leg.ctx, pid, ops, s), reps)
+                    row[name + "_gbs"] = n * T * E * bpe / (ms * 1e-3) / 1e9
+                leg.check()
+                points.append(row)
+    del arena
+    torch.cuda.empty_cache()
+    return points
 
-    # ---- host-link ceiling, same run: one large pinned cudaMemcpyAsync each way
+
+def host_link_peak(torch, stream, dev):
+    """Host-link ceiling of this run: one 1 GiB pinned cudaMemcpyAsync each way, best of 5."""
     probe = torch.empty(1 << 30, dtype=torch.uint8).pin_memory()
     dprobe = torch.empty(1 << 30, dtype=torch.uint8, device=dev)
     link = {}
@@ -616,41 +586,214 @@ def run_gpu(args) -> None:
             torch.cuda.synchronize()
             best = max(best, probe.numel() / (a.elapsed_time(b) * 1e-3) / 1e9)
         link[name + "_gbs"] = best
+    return link
+
+
+def leg_70b(args, rank, local, barrier, steps):
+    """The batched 70B configuration: device-resident timing of the six ops, then the batched retrieve with four of its
+    chunks in page-locked host memory (side stream) and the layer-wise delivery of one host-resident chunk."""
+    import torch
+    from paper_2409_13761_b200 import synth
+    W = make_workload("llama3-70b", args, synth)
+    leg = Leg(W, rank, local)
+    K = leg.K
+    dev_sets = leg.make_sets(False)
+    leg.fill_parts(dev_sets)
+    elapsed_ms, op_ms, launches, _ = leg.time_steps(dev_sets, steps, 3, barrier, sample_clocks=False)
+    res = {"workload": W["text"], "steps": steps, "ms_per_step": elapsed_ms / steps, "op_ms": op_ms,
+           "op_bytes": dict(leg.op_bytes), "op_tokens": dict(leg.op_tokens), "kernels": dict(leg.kernels),
+           "launches": launches, "step_bytes": leg.step_bytes}
+    if not args.no_e2e:
+        pinned_retr = (5, 50, 90, 120)
+        host_sets = leg.make_sets(False, pinned_retr)
+        for codec in (RAW, INT8):
+            host_sets[codec]["chunks"].copy_(dev_sets[codec]["chunks"])
+            for c, hb in host_sets[codec]["host_copy"].items():
+                cb = hb.numel()
+                hb.copy_(dev_sets[codec]["chunks"][c * cb:(c + 1) * cb])
+        del dev_sets
+        torch.cuda.empty_cache()
+        leg.step(host_sets, kinds=("retrieve",))
+        leg.check()
+        n_e2e = max(1, min(steps, args.e2e_steps))
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(n_e2e):
+            leg.step(host_sets, kinds=("retrieve",))
+            leg.check()                                   # the step's result is read back: device status + all copies landed
+        barrier()
+        ms = (time.perf_counter() - t0) * 1e3 / n_e2e
+        h2d = sum(K.kdn_chunk_bytes(leg.desc, leg.T, c) * len(pinned_retr) for c in (RAW, INT8))
+        res["side_stream"] = {"what": "batched retrieve, 4 of %d chunks in page-locked host memory (side stream), raw + int8" % leg.n_retr,
+                              "ms_per_step": ms, "h2d_bytes_per_step": int(h2d), "host_link_gbs": h2d / (ms * 1e-3) / 1e9,
+                              "gbs": (leg.op_bytes["retrieve_raw"] + leg.op_bytes["retrieve_int8"]) / (ms * 1e-3) / 1e9}
+        # layer-wise delivery of one host-resident chunk: when is the first layer range usable, when the last?
+        layerwise = {}
+        shape = leg.shape
+        for codec, cname in ((RAW, "raw"), (INT8, "int8")):
+            op = [host_sets[codec]["retrieve"][pinned_retr[0]]]
+            for mode, lps in (("whole", shape.n_layers), ("by_8_layers", 8)):
+                evs = [torch.cuda.Event(enable_timing=True) for _ in range(shape.n_layers)]
+                t_start = torch.cuda.Event(enable_timing=True)
+                for e in evs + [t_start]:
+                    e.record(leg.stream)
+                torch.cuda.synchronize()
+                K.kdn_retrieve_layerwise(leg.ctx, leg.pid, op, lps, leg.s, 0, [e.cuda_event for e in evs])   # warm
+                torch.cuda.synchronize()
+                t_start.record(leg.stream)
+                K.kdn_retrieve_layerwise(leg.ctx, leg.pid, op, lps, leg.s, 0, [e.cuda_event for e in evs])
+                torch.cuda.synchronize()
+                layerwise["%s_%s" % (cname, mode)] = {"first_layers_ready_ms": t_start.elapsed_time(evs[min(lps, shape.n_layers) - 1]),
+                                                      "all_layers_ready_ms": t_start.elapsed_time(evs[-1]),
+                                                      "chunk_bytes": K.kdn_chunk_bytes(leg.desc, leg.T, codec)}
+        leg.check()
+        res["layerwise_one_host_chunk"] = layerwise
+        res["host_link_peak"] = host_link_peak(torch, leg.stream, leg.dev)
+        del host_sets
+    leg.close()
+    return res
+
+
+def run_gpu(args) -> None:
+    import torch
+    from paper_2409_13761_b200 import kdn as K, shard, synth
+
+    rank, world, local = shard.rank_env()
+    dist = None
+    if world > 1 or "TORCHELASTIC_RUN_ID" in os.environ:        # launched by torch.distributed.run, even with one rank
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    if args.workload == "llama3-70b":                           # the 70B configuration on its own
+        res = leg_70b(args, rank, local, barrier, args.steps)
+        if rank == 0:
+            peak, peak_kind = measured_hbm_peak()
+            res["op_gbs"] = {n: res["op_bytes"][n] / (res["op_ms"][n] * 1e-3) / 1e9 for n in NAMES}
+            res["note"] = "llama3-70b leg on its own, not a bench record"
+            print(json.dumps(res))
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    W = make_workload("llama3-8b", args, synth)
+    leg = Leg(W, rank, local)
+    shape, T, PT, E = leg.shape, leg.T, leg.PT, leg.E
+    ctx, pid, s, desc = leg.ctx, leg.pid, leg.s, leg.desc
+    n_lib, n_retr, n_parts_total = leg.n_lib, leg.n_retr, leg.n_parts_total
+    dev_sets = leg.make_sets(False)
+    leg.fill_parts(dev_sets)
+
+    # ---- device-resident timing: the step `value` is measured on
+    elapsed_ms, op_ms, launches, clocks = leg.time_steps(dev_sets, args.steps, args.warmup, barrier)
+    reps = max(1, min(args.steps, 20))
+    extras = extras_8b(leg, dev_sets, reps)
+    full = not (args.pool_blocks or args.chunks or args.parts)
+    sweep_points = sweep_extract(leg, min(reps, 10)) if full and not args.no_sweep else None
+
+    if args.no_e2e:
+        if rank == 0:
+            print(json.dumps({"note": "profiling run, not a bench record", "ops_ms": op_ms, "kernels": leg.kernels,
+                              "ops_gbs": {n: leg.op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 for n in NAMES}, **extras,
+                              "sweep_extract": sweep_points}))
+        leg.close()
+        return
+
+    # ---- end to end: the whole step with the entire library in page-locked host memory, so every byte crosses the
+    # host link inside the timed region
+    e2e_steps = max(1, min(args.steps, args.e2e_steps))
+    del dev_sets
+    torch.cuda.empty_cache()
+    host_sets = leg.make_sets(True)
+    leg.fill_parts(host_sets)
+    d2h = sum(K.kdn_chunk_bytes(desc, T, c) * n_lib for c in (RAW, INT8)) + 4
+    h2d = sum(K.kdn_chunk_bytes(desc, T, c) * n_retr + K.kdn_chunk_bytes(desc, PT, c) * n_parts_total for c in (RAW, INT8))
+    leg.step(host_sets)
+    leg.check()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        leg.step(host_sets)
+        leg.check()                                   # the step's result is read back: device status + all copies landed
+    barrier()
+    e2e_ms = (time.perf_counter() - t0) * 1e3
+    link = host_link_peak(torch, leg.stream, dev)
+    step_bytes, op_bytes, op_tokens, reload_tokens, kernels = leg.step_bytes, leg.op_bytes, leg.op_tokens, leg.reload_tokens, dict(leg.kernels)
+    del host_sets
+    leg.close()
+
+    # ---- the largest configuration: the batched 70B workload (not part of `value`; its per-op figures go into the
+    # roofline table below)
+    r70 = None
+    if full and not args.no_70b:
+        r70 = leg_70b(args, rank, local, barrier, max(3, min(args.steps, 10)))
 
     # ---- reduce over ranks (max time), print on rank 0
-    times = shard.max_over_ranks([elapsed_ms, e2e_ms] + [op_ms[n] for n in names], device=dev)
+    vals = [elapsed_ms, e2e_ms] + [op_ms[n] for n in NAMES] + ([r70["op_ms"][n] for n in NAMES] if r70 else [])
+    times = shard.max_over_ranks(vals, device=dev)
     elapsed_ms, e2e_ms = float(times[0]), float(times[1])
-    op_ms = {n: float(times[2 + i]) for i, n in enumerate(names)}
+    op_ms = {n: float(times[2 + i]) for i, n in enumerate(NAMES)}
+    if r70:
+        r70["op_ms"] = {n: float(times[2 + len(NAMES) + i]) for i, n in enumerate(NAMES)}
     if rank == 0:
         peak, peak_kind = measured_hbm_peak()
         ms_per_step = elapsed_ms / args.steps
         value = shard.job_throughput(step_bytes, world, ms_per_step * 1e-3) / 1e9
-        ops = {n: {"ms": op_ms[n], "gbs": op_bytes[n] / (op_ms[n] * 1e-3) / 1e9,
-                   "frac_of_%s_copy_peak" % peak_kind: op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 / peak,
-                   "frac_of_8000": op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 / 8000.0,
-                   "tokens_per_s": op_tokens[n] / (op_ms[n] * 1e-3), "kernel": kernel_of[n]} for n in names}
-        top = max(names, key=lambda n: op_ms[n])
+        gbs = {n: op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 for n in NAMES}
+        ops = {n: {"ms": op_ms[n], "gbs": gbs[n], "frac_of_%s_copy_peak" % peak_kind: gbs[n] / peak, "frac_of_8000": gbs[n] / 8000.0,
+                   "tokens_per_s": op_tokens[n] / (op_ms[n] * 1e-3), "kernel": kernels[n]["kernel"], "launch": kernels[n]} for n in NAMES}
+        top = max(NAMES, key=lambda n: op_ms[n])
         units = {"store": n_lib * T / CHUNK_TOKENS, "retrieve": n_retr * T / CHUNK_TOKENS,
                  "compose": n_parts_total * PT / PART_TOKENS}[top.split("_")[0]]
         traffic = measured_traffic(top, units) if shape.elems_per_token == 65536 else None
+        # every op of both workloads as [GB/s, fraction of the nominal 8000 GB/s]; median CUDA-event time per op
+        per_op = {"fractions": "of the nominal 8000 GB/s; GB/s = algorithmic bytes / median CUDA-event time of the op",
+                  "8b": {n: [round(gbs[n], 1), round(gbs[n] / 8000.0, 4)] for n in NAMES}}
+        if r70:
+            g70 = {n: r70["op_bytes"][n] / (r70["op_ms"][n] * 1e-3) / 1e9 for n in NAMES}
+            per_op["70b"] = {n: [round(g70[n], 1), round(g70[n] / 8000.0, 4)] for n in NAMES}
+            per_op["70b_ms_per_step"] = round(r70["ms_per_step"], 3)
+            if "side_stream" in r70:
+                per_op["70b_host_link"] = [round(r70["side_stream"]["host_link_gbs"], 2), round(r70["host_link_peak"]["h2d_gbs"], 2)]
+        if sweep_points:
+            for name in ("store", "retrieve"):
+                worst = min(sweep_points, key=lambda p: p[name + "_gbs"])
+                per_op["sweep_min_" + name] = [round(worst[name + "_gbs"], 1), round(worst[name + "_gbs"] / 8000.0, 4),
+                                               "T=%d bs=%d %s" % (worst["chunk_tokens"], worst["block_size"], worst["codec"])]
+            per_op["sweep_points"] = len(sweep_points)
+        frac = gbs[top] / peak
         rec = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16/int8 (fp32 codec and rotation, fp64 angles)", "data": "synthetic",
-            "config": {"workload": W["text"], "l2": "inputs larger than L2 (every op streams >= 1.9 GB once)",
-                       "bytes_per_step": step_bytes},
-            "tokens_per_s_reloaded": world * reload_tokens / (sum(op_ms[n] for n in names if not n.startswith("store")) * 1e-3),
-            "ops": ops, "ops_int4_not_in_value": int4_ops, "ops_keep_list_not_in_value": sparse_ops, "ops_shell_not_in_value": shell_ops,
-            "ops_file_not_in_value": file_ops, "ops_single_chunk_not_in_value": single_ops, "ops_per_channel_key_codecs_not_in_value": kc_ops,
-            "roofline": {"bound": "hbm", "kernel": kernel_of[top], "op": top, "achieved": ops[top]["gbs"], "peak": peak,
-                         "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": ops[top]["gbs"] / peak,
-                         "frac_of_nominal_8000": ops[top]["gbs"] / 8000.0, "traffic": traffic},
-            "e2e": {"value": world * e2e_bytes / (e2e_ms / e2e_steps * 1e-3) / 1e9, "unit": UNIT,
+            "config": {"workload": W["text"], "also_measured": "llama3-70b batch (32x4x2048 tokens) and sweep ends: roofline.per_op",
+                       "l2": "inputs larger than L2 (every op streams >= 1.9 GB once)", "bytes_per_step": step_bytes},
+            "tokens_per_s_reloaded": world * reload_tokens / (sum(op_ms[n] for n in NAMES if not n.startswith("store")) * 1e-3),
+            "roofline": {"bound": "hbm", "kernel": kernels[top]["kernel"], "op": top, "achieved": gbs[top], "peak": peak,
+                         "peak_kind": "of " + peak_kind, "unit": "GB/s", "frac": frac,
+                         "frac_of_nominal_8000": gbs[top] / 8000.0, "traffic": traffic,
+                         "traffic_source": ("profiler capture of a reduced case, scaled by the units of a launch" if traffic is not None
+                                            else "none: the kernels changed since the profiler capture (algorithmic bytes only)"),
+                         "note": ("the measured peak is a plain device copy; bulk-copy streams run a little above it, so this "
+                                  "fraction says 'at the copy ceiling', not 'headroom left'" if frac > 1.0 else None),
+                         "per_op": per_op},
+            "e2e": {"value": world * step_bytes / (e2e_ms / e2e_steps * 1e-3) / 1e9, "unit": UNIT,
                     "h2d_bytes_per_step": int(h2d), "d2h_bytes_per_step": int(d2h), "steps": e2e_steps,
-                    "ms_per_step": e2e_ms / e2e_steps, "what": e2e_what,
+                    "ms_per_step": e2e_ms / e2e_steps, "what": "whole step, every chunk in page-locked host memory",
                     "host_link_gbs": (h2d + d2h) / (e2e_ms / e2e_steps * 1e-3) / 1e9, "host_link_peak": link,
-                    "layerwise_one_host_chunk": layerwise},
+                    "llama3_70b_side_stream": (r70 or {}).get("side_stream"),
+                    "layerwise_one_host_chunk": (r70 or {}).get("layerwise_one_host_chunk")},
             "gpu_launches": int(launches), "clocks": clocks,
+            "ops": ops, "llama3_70b": ({"workload": r70["workload"], "steps": r70["steps"], "ms_per_step": r70["ms_per_step"],
+                                        "op_ms": r70["op_ms"], "kernels": {n: r70["kernels"][n]["kernel"] for n in NAMES},
+                                        "launches": r70["launches"]} if r70 else None),
+            "sweep_extract": sweep_points, **extras,
         }
         if not args.no_cpu_baseline and world == 1:
             cores = len(os.sched_getaffinity(0))
@@ -662,7 +805,6 @@ def run_gpu(args) -> None:
             b1, t1, dt1 = one.run_pass()
             rec["cpu_baseline"]["one_core"] = {"value": b1 / dt1 / 1e9, "unit": UNIT, "sample": one.describe(1, b1, dt1)}
         print(json.dumps(rec))
-    K.kdn_destroy(ctx)
     if dist is not None:
         dist.destroy_process_group()
 
@@ -739,9 +881,12 @@ def main() -> None:
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-link leg (profiling runs)")
+    ap.add_argument("--no-70b", action="store_true", help="skip the llama3-70b leg of the default run")
+    ap.add_argument("--no-sweep", action="store_true", help="skip the sweep extract of the default run")
     ap.add_argument("--sweep", action="store_true", help="chunk-length / block-size / codec / fragmentation sweep (1 GPU)")
     ap.add_argument("--workload", default="llama3-8b", choices=["llama3-8b", "llama3-70b"],
-                    help="llama3-8b is the benchmark workload; llama3-70b is the batched-retrieve configuration")
+                    help="llama3-8b (default): the benchmark run, which also times the 70B batch and the sweep ends; "
+                         "llama3-70b: only the batched 70B configuration")
     ap.add_argument("--pool-blocks", type=int, default=0, help="smaller pool for profiler captures (default 16384)")
     ap.add_argument("--chunks", type=int, default=0, help="chunks per store/retrieve batch (default 64)")
     ap.add_argument("--parts", type=int, default=0, help="parts per composed request (default 10)")

@@ -59,6 +59,17 @@
  * descriptors, a rotation table, and (on first use of pinned-host chunks) two
  * staging slabs.  It never frees or reallocates caller memory.
  *
+ * ---------------------------------------------------------- stream order --
+ * A call's work is ordered after everything enqueued on cuda_stream before it,
+ * and everything enqueued on cuda_stream after the call returns is ordered
+ * after the call's work -- including the copies between page-locked host
+ * chunks and the device that run on side_stream: a call that uses the side
+ * stream first makes it wait for cuda_stream, and a store ends by making
+ * cuda_stream wait for its device-to-host copies.  An event recorded on
+ * cuda_stream after kdn_store therefore covers the bytes in host memory, and a
+ * host chunk filled by a copy on cuda_stream can be retrieved without a host
+ * synchronisation in between.
+ *
  * ----------------------------------------------------------------- errors --
  * Argument errors are returned at once and nothing is enqueued.  Otherwise a
  * call returns after enqueueing its work; it does not wait for the GPU.
@@ -297,8 +308,9 @@ kdn_status kdn_compose(kdn_ctx *ctx, int pool_id, const kdn_compose_req *reqs, i
  * (KDN_E_RANGE for a block id outside the pool, ...), or KDN_OK.  wait == 0: the call returns after
  * enqueueing; errors found on the device by that call are then not reported.
  *
- * The first call on each device looks up the array's device address (a one-time set-up step);
- * make that first call before any stream capture begins.  All calls on a device share the one array,
+ * The first call on each device does the one-time set-up: it looks up the array's device address, loads
+ * every kernel a later call can launch and raises their shared-memory limits, so no later call meets a
+ * first-use step of the CUDA runtime.  Make that first call before any stream capture begins.  All calls on a device share the one array,
  * and it still holds the previous call's records when the next call starts: each call rewrites the
  * records it uses and clears the status word, on cuda_stream, before its kernels run.  Two calls
  * whose work can overlap on the GPU (different streams without an ordering between them) therefore
@@ -329,8 +341,24 @@ kdn_status kdn_set_tuning(kdn_ctx *ctx, const kdn_tuning *tuning);
  * on first use).  Takes effect at the next pinned-host call; frees slabs already allocated. */
 kdn_status kdn_set_staging_bytes(kdn_ctx *ctx, size_t bytes_per_slab);
 
+/* Limit, in nanoseconds, after which a wait inside the tile pipeline gives up and the launch reports KDN_E_TIMEOUT
+ * (default, and ns = 0: two seconds).  The waits that let a CTA's own copies finish before it leaves always keep the
+ * default.  Meant for exercising the error path: with a limit shorter than a memory access the next launches give up
+ * almost at once, write little or nothing, and kdn_status_sync returns KDN_E_TIMEOUT; nothing faults or hangs, and
+ * after the default is restored the context works as before. */
+kdn_status kdn_set_wait_limit_ns(kdn_ctx *ctx, uint64_t ns);
+
 /* Kernels this context has launched so far (for accounting; never reset). */
 uint64_t kdn_launch_count(const kdn_ctx *ctx);
+
+/* Shape of the context's most recent launch of the tile pipeline, for reports: op 0 store / 1 retrieve / 2 compose
+ * (the kernel is kdn_store_kernel / kdn_retrieve_kernel / kdn_compose_kernel<compute_groups, group_warps>);
+ * grid is what was asked for (the launch itself never exceeds the CTAs resident at once). */
+typedef struct {
+    int32_t  op, compute_groups, group_warps, tile_bytes, stages, ctas_per_sm, store_lag, grid, smem_bytes;
+    uint32_t n_tiles;
+} kdn_launch_info;
+kdn_status kdn_last_launch(const kdn_ctx *ctx, kdn_launch_info *out);
 
 /* ------------------------------------------------------------------------------------------------
  * Storage-module shell (Sec. 3.1: the storage module keeps KV caches under keys derived from their texts; Sec. 3.2:

@@ -87,54 +87,52 @@ def compile_source(source_text: str, out_path: str) -> str:
 
 
 def _declare(L):
-    if True:
-        if True:
-            i32, i64, f64, sz = C.c_int, C.c_int64, C.c_double, C.c_size_t
-            vp = C.c_void_p
-            L.kdn_oracle_bf16_to_f32.restype = C.c_float
-            L.kdn_oracle_bf16_to_f32.argtypes = [C.c_uint16]
-            L.kdn_oracle_f32_to_bf16.restype = C.c_uint16
-            L.kdn_oracle_f32_to_bf16.argtypes = [C.c_float]
-            L.kdn_oracle_f32_to_bf16_many.restype = None
-            L.kdn_oracle_f32_to_bf16_many.argtypes = [vp, vp, sz]
-            L.kdn_oracle_f64_to_bf16.restype = C.c_uint16
-            L.kdn_oracle_f64_to_bf16.argtypes = [f64]
-            L.kdn_oracle_chunk_bytes.restype = sz
-            L.kdn_oracle_chunk_bytes.argtypes = [i32, i32, i32, i32, i32]
-            L.kdn_oracle_quant_group.restype = None
-            L.kdn_oracle_quant_group.argtypes = [vp, vp, vp]
-            L.kdn_oracle_quant4_group.restype = None
-            L.kdn_oracle_quant4_group.argtypes = [vp, vp, vp]
-            L.kdn_oracle_quant_channel.restype = None
-            L.kdn_oracle_quant_channel.argtypes = [vp, i32, i32, vp, vp]
-            L.kdn_oracle_dequant.restype = C.c_uint16
-            L.kdn_oracle_dequant.argtypes = [C.c_int8, C.c_float]
-            L.kdn_oracle_rope_angle.restype = f64
-            L.kdn_oracle_rope_angle.argtypes = [i64, f64, i32, i32]
-            L.kdn_oracle_rotate_pair.restype = None
-            L.kdn_oracle_rotate_pair.argtypes = [f64, f64, f64, C.POINTER(f64), C.POINTER(f64)]
-            xfer = [vp, i32, i32, i32, i32, i64, vp, i32, i64, i32, i32, vp]
-            L.kdn_oracle_store.restype = i32
-            L.kdn_oracle_store.argtypes = xfer
-            L.kdn_oracle_retrieve.restype = i32
-            L.kdn_oracle_retrieve.argtypes = xfer
-            xs = [vp, i32, i32, i32, i32, i64, vp, i32, i64, i32, i32, vp, vp]
-            L.kdn_oracle_store_sparse.restype = i32
-            L.kdn_oracle_store_sparse.argtypes = xs
-            L.kdn_oracle_retrieve_sparse.restype = i32
-            L.kdn_oracle_retrieve_sparse.argtypes = xs
-            L.kdn_oracle_compose_select.restype = i32
-            L.kdn_oracle_compose_select.argtypes = [vp, i32, i32, i32, i32, i64, vp, i32, i32,
-                                                    vp, vp, vp, vp, vp, f64, vp, vp, vp, vp]
-            L.kdn_oracle_compose.restype = i32
-            L.kdn_oracle_compose.argtypes = [vp, i32, i32, i32, i32, i64, vp, i32, i32,
-                                             vp, vp, vp, vp, vp, f64, vp, vp]
-            L.kdn_oracle_fnv1a.restype = C.c_uint64
-            L.kdn_oracle_fnv1a.argtypes = [vp, sz]
-            L.kdn_oracle_key_hash.restype = C.c_uint64
-            L.kdn_oracle_key_hash.argtypes = [vp, sz]
-            L.kdn_oracle_checksum.restype = C.c_uint64
-            L.kdn_oracle_checksum.argtypes = [vp, sz]
+    i32, i64, f64, sz = C.c_int, C.c_int64, C.c_double, C.c_size_t
+    vp = C.c_void_p
+    L.kdn_oracle_bf16_to_f32.restype = C.c_float
+    L.kdn_oracle_bf16_to_f32.argtypes = [C.c_uint16]
+    L.kdn_oracle_f32_to_bf16.restype = C.c_uint16
+    L.kdn_oracle_f32_to_bf16.argtypes = [C.c_float]
+    L.kdn_oracle_f32_to_bf16_many.restype = None
+    L.kdn_oracle_f32_to_bf16_many.argtypes = [vp, vp, sz]
+    L.kdn_oracle_f64_to_bf16.restype = C.c_uint16
+    L.kdn_oracle_f64_to_bf16.argtypes = [f64]
+    L.kdn_oracle_chunk_bytes.restype = sz
+    L.kdn_oracle_chunk_bytes.argtypes = [i32, i32, i32, i32, i32]
+    L.kdn_oracle_quant_group.restype = None
+    L.kdn_oracle_quant_group.argtypes = [vp, vp, vp]
+    L.kdn_oracle_quant4_group.restype = None
+    L.kdn_oracle_quant4_group.argtypes = [vp, vp, vp]
+    L.kdn_oracle_quant_channel.restype = None
+    L.kdn_oracle_quant_channel.argtypes = [vp, i32, i32, vp, vp]
+    L.kdn_oracle_dequant.restype = C.c_uint16
+    L.kdn_oracle_dequant.argtypes = [C.c_int8, C.c_float]
+    L.kdn_oracle_rope_angle.restype = f64
+    L.kdn_oracle_rope_angle.argtypes = [i64, f64, i32, i32]
+    L.kdn_oracle_rotate_pair.restype = None
+    L.kdn_oracle_rotate_pair.argtypes = [f64, f64, f64, C.POINTER(f64), C.POINTER(f64)]
+    xfer = [vp, i32, i32, i32, i32, i64, vp, i32, i64, i32, i32, vp]
+    L.kdn_oracle_store.restype = i32
+    L.kdn_oracle_store.argtypes = xfer
+    L.kdn_oracle_retrieve.restype = i32
+    L.kdn_oracle_retrieve.argtypes = xfer
+    xs = [vp, i32, i32, i32, i32, i64, vp, i32, i64, i32, i32, vp, vp]
+    L.kdn_oracle_store_sparse.restype = i32
+    L.kdn_oracle_store_sparse.argtypes = xs
+    L.kdn_oracle_retrieve_sparse.restype = i32
+    L.kdn_oracle_retrieve_sparse.argtypes = xs
+    L.kdn_oracle_compose_select.restype = i32
+    L.kdn_oracle_compose_select.argtypes = [vp, i32, i32, i32, i32, i64, vp, i32, i32,
+                                            vp, vp, vp, vp, vp, f64, vp, vp, vp, vp]
+    L.kdn_oracle_compose.restype = i32
+    L.kdn_oracle_compose.argtypes = [vp, i32, i32, i32, i32, i64, vp, i32, i32,
+                                     vp, vp, vp, vp, vp, f64, vp, vp]
+    L.kdn_oracle_fnv1a.restype = C.c_uint64
+    L.kdn_oracle_fnv1a.argtypes = [vp, sz]
+    L.kdn_oracle_key_hash.restype = C.c_uint64
+    L.kdn_oracle_key_hash.argtypes = [vp, sz]
+    L.kdn_oracle_checksum.restype = C.c_uint64
+    L.kdn_oracle_checksum.argtypes = [vp, sz]
     return L
 
 

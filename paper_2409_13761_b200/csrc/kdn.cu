@@ -1,5 +1,5 @@
 // Host side of libkdn: the C ABI declared in include/kdn.h.  Validates arguments, turns ops into
-// 64-byte device records, and launches the tile pipeline of kdn_kernels.cuh on the caller's stream.
+// 96-byte device records, and launches the tile pipeline of kdn_kernels.cuh on the caller's stream.
 // Paper anchors: Sec. 3.2 "Interface with LLM serving engines" (store / retrieve), Sec. 3.1 (storage,
 // delivery and blending modules).
 #include "kdn.h"
@@ -9,7 +9,6 @@
 #include <cstdio>
 #include <cstring>
 #include <functional>
-#include <map>
 #include <mutex>
 #include <new>
 #include <atomic>
@@ -20,6 +19,12 @@
 #include <unistd.h>
 
 using namespace kdn;
+
+#define KDN_CUDA(call)                                                                  \
+    do {                                                                                \
+        cudaError_t e_ = (call);                                                        \
+        if (e_ != cudaSuccess) return e_ == cudaErrorMemoryAllocation ? KDN_E_NOMEM : KDN_E_CUDA; \
+    } while (0)
 
 namespace {
 
@@ -63,12 +68,45 @@ struct Piece {                              // host <-> slab copies belonging to
     long long file_off;
 };
 
+// What a launch needs to know about its device, and what it has already asked the runtime about each kernel:
+// one per context (and one per device for kdn_compose_static), so a launch takes no lock and no device query.
+// Every kernel's dynamic shared-memory limit is raised to the device's opt-in maximum the first time it is seen,
+// whatever the launch at hand needs: the value is the same for every context of the process, so contexts cannot
+// lower each other's grants.
+struct LaunchEnv {
+    int sm_count = 0;
+    int smem_optin = 0;
+    struct Entry { const void *fn; size_t smem; int threads; int per_sm; };
+    static constexpr int kEntries = 64;
+    Entry cache[kEntries];
+    int n = 0, next = 0;
+
+    // CTAs of `kernel` resident per SM at this shape (0 = does not fit); sets the kernel's attribute on first sight.
+    template <typename K>
+    kdn_status resident(K kernel, int threads, size_t smem, int *per_sm)
+    {
+        const void *fn = (const void *)kernel;
+        bool seen = false;
+        for (int i = 0; i < n; ++i) {
+            if (cache[i].fn != fn) continue;
+            seen = true;
+            if (cache[i].smem == smem && cache[i].threads == threads) { *per_sm = cache[i].per_sm; return KDN_OK; }
+        }
+        if (!seen) KDN_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, smem_optin));
+        int r = 0;
+        KDN_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&r, kernel, threads, smem));
+        Entry &e = n < kEntries ? cache[n++] : cache[next++ % kEntries];
+        e.fn = fn; e.smem = smem; e.threads = threads; e.per_sm = r;
+        *per_sm = r;
+        return KDN_OK;
+    }
+};
+
 }  // namespace
 
 struct kdn_ctx {
     int device = 0;
-    int sm_count = 0;
-    int smem_optin = 0;
+    LaunchEnv env;                          // SM count, shared-memory limit, per-kernel occupancy cache
     std::vector<Pool> pools;
     RingSlot ring[kRing];
     unsigned ring_next = 0;
@@ -86,15 +124,12 @@ struct kdn_ctx {
     std::vector<Piece> pending_writes[2];              // file pieces whose bytes are on their way into bounce[i]
     uint64_t launches = 0;
     kdn_tuning tuning{};
+    unsigned long long wait_limit_ns = kWaitLimitNs;
+    kdn_launch_info last{};                 // shape of the most recent tile-pipeline launch
+    cudaEvent_t fork = nullptr;             // orders the side stream after the caller's stream at the start of a staged call
 };
 
 namespace {
-
-#define KDN_CUDA(call)                                                                  \
-    do {                                                                                \
-        cudaError_t e_ = (call);                                                        \
-        if (e_ != cudaSuccess) return e_ == cudaErrorMemoryAllocation ? KDN_E_NOMEM : KDN_E_CUDA; \
-    } while (0)
 
 bool shape_ok(const kdn_pool_desc *p)
 {
@@ -244,43 +279,19 @@ kdn_status drain_writes(kdn_ctx *ctx, unsigned s)
     return ok ? KDN_OK : KDN_E_IO;
 }
 
-// Largest dynamic shared-memory size already granted to each kernel on each device (setting the attribute on
-// every launch costs about a microsecond of host time).
-std::mutex g_attr_mutex;
-std::map<std::pair<int, const void *>, size_t> g_attr_granted;
-
 // `overlap`: the launch may start while the kernel before it in the stream (the rotation-table kernel) still runs;
 // the warps that read that kernel's output wait for it on the device.
 template <typename K>
-kdn_status launch_kernel(K kernel, int threads, unsigned grid, size_t smem, cudaStream_t stream, const Launch &lp,
-                         bool overlap = false)
+kdn_status launch_kernel(LaunchEnv &env, K kernel, int threads, unsigned grid, size_t smem, cudaStream_t stream,
+                         const Launch &lp, bool overlap = false)
 {
-    {
-        int device = 0;
-        KDN_CUDA(cudaGetDevice(&device));
-        std::lock_guard<std::mutex> lock(g_attr_mutex);
-        size_t &granted = g_attr_granted[std::make_pair(device, (const void *)kernel)];
-        if (granted < smem) {
-            KDN_CUDA(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            granted = smem;
-        }
-    }
-    {
-        // the pipeline is written for CTAs that are all resident at once: never launch more than fit
-        static std::map<std::pair<std::pair<int, const void *>, size_t>, int> resident;
-        int device = 0;
-        KDN_CUDA(cudaGetDevice(&device));
-        std::lock_guard<std::mutex> lock(g_attr_mutex);
-        int &per_sm = resident[std::make_pair(std::make_pair(device, (const void *)kernel), smem)];
-        if (per_sm == 0) {
-            KDN_CUDA(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, threads, smem));
-            if (per_sm < 1) return KDN_E_UNSUPPORTED;
-        }
-        int sms = 0;
-        KDN_CUDA(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, device));
-        const unsigned long long cap = (unsigned long long)per_sm * (unsigned long long)sms;
-        if (grid > cap) grid = (unsigned)cap;
-    }
+    // the pipeline is written for CTAs that are all resident at once: never launch more than fit
+    int per_sm = 0;
+    kdn_status st = env.resident(kernel, threads, smem, &per_sm);
+    if (st != KDN_OK) return st;
+    if (per_sm < 1) return KDN_E_UNSUPPORTED;
+    const unsigned long long cap = (unsigned long long)per_sm * (unsigned long long)env.sm_count;
+    if (grid > cap) grid = (unsigned)cap;
     if (overlap) {
         cudaLaunchConfig_t cfg{};
         cfg.gridDim = dim3(grid);
@@ -329,14 +340,14 @@ kdn_status fit_stages(int &stages, int groups, int lag, bool shrink, unsigned st
 }
 
 // Launch the instantiation for (OP, compute groups, warps per group); groups = 0 is the pure-copy form.
-kdn_status launch_tiles(int OP, int groups, int gw, unsigned grid, size_t smem, cudaStream_t stream, const Launch &lp,
-                        bool overlap = false)
+kdn_status launch_tiles(LaunchEnv &env, int OP, int groups, int gw, unsigned grid, size_t smem, cudaStream_t stream,
+                        const Launch &lp, bool overlap = false)
 {
 #define KDN_CASE(G, W)                                                                                             \
     if (groups == G && (G == 0 || gw == W)) {                                                                      \
-        if (OP == OP_STORE) return launch_kernel(kdn_store_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp);      \
-        if (OP == OP_RETRIEVE) return launch_kernel(kdn_retrieve_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp); \
-        return launch_kernel(kdn_compose_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp, overlap);               \
+        if (OP == OP_STORE) return launch_kernel(env, kdn_store_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp);      \
+        if (OP == OP_RETRIEVE) return launch_kernel(env, kdn_retrieve_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp); \
+        return launch_kernel(env, kdn_compose_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp, overlap);               \
     }
     KDN_CASE(0, 4) KDN_CASE(1, 4) KDN_CASE(2, 4) KDN_CASE(3, 4) KDN_CASE(4, 4) KDN_CASE(6, 4)
     KDN_CASE(2, 1) KDN_CASE(4, 1) KDN_CASE(8, 1)
@@ -396,7 +407,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     const int lag = ctx->tuning.store_lag > 0 ? ctx->tuning.store_lag : def.lag;
     int ctas_per_sm = ctx->tuning.ctas_per_sm > 0 ? ctx->tuning.ctas_per_sm : def.ctas_per_sm;
     int stages = ctx->tuning.stages > 0 ? ctx->tuning.stages : def.stages;
-    const size_t smem_limit = (size_t)ctx->smem_optin;
+    const size_t smem_limit = (size_t)ctx->env.smem_optin;
     kdn_status fit = fit_stages(stages, groups, lag, ctx->tuning.stages <= 0, stage_bytes, ctas_per_sm, smem_limit);
     if (fit != KDN_OK) return fit;
     const size_t smem = smem_bytes(stages, stage_bytes);
@@ -478,6 +489,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     lp.off_s = a_bytes + b_bytes;
     lp.store_lag = lag;
     lp.reload_first = (!compute && tile_elems * 2u >= 8192u) ? 1 : 0;
+    lp.wait_limit_ns = ctx->wait_limit_ns;
 
     if (kc_groups > 0) {
         // key planes of the per-channel key codecs: one CTA per (64-token group, layer, op)
@@ -502,24 +514,32 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
         kp.status = ctx->d_status;
         if (inl) std::memcpy(kp.inline_ops, lp.inline_ops, sizeof(DevOp) * (size_t)n);
         {
-            std::lock_guard<std::mutex> lock(g_attr_mutex);
-            size_t &granted = g_attr_granted[std::make_pair(ctx->device, (const void *)kdn_store_kc_kernel)];
-            if (granted < kc_smem) {
-                KDN_CUDA(cudaFuncSetAttribute(kdn_store_kc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kc_smem));
-                granted = kc_smem;
-            }
+            int per_sm = 0;                                  // first sight of the kernel raises its shared-memory limit
+            kdn_status r = ctx->env.resident(kdn_store_kc_kernel, (int)kc_threads, kc_smem, &per_sm);
+            if (r != KDN_OK) return r;
+            if (per_sm < 1) return KDN_E_UNSUPPORTED;
         }
         kdn_store_kc_kernel<<<dim3((unsigned)kc_groups * n_split, (unsigned)kc_layers, (unsigned)n), kc_threads, kc_smem, stream>>>(kp);
         KDN_CUDA(cudaGetLastError());
         ctx->launches++;
     }
 
-    unsigned long long want = (unsigned long long)ctx->sm_count * (unsigned)ctas_per_sm;
+    unsigned long long want = (unsigned long long)ctx->env.sm_count * (unsigned)ctas_per_sm;
     const unsigned grid = (unsigned)(tiles < want ? tiles : want);
     const int gw = ctx->tuning.group_warps > 0 ? ctx->tuning.group_warps : def.gw;
-    kdn_status st = launch_tiles(OP, groups, gw, grid, smem, stream, lp, OP == OP_COMPOSE && n_rope > 0);
+    kdn_status st = launch_tiles(ctx->env, OP, groups, gw, grid, smem, stream, lp, OP == OP_COMPOSE && n_rope > 0);
     if (st != KDN_OK) return st;
     ctx->launches++;
+    ctx->last.op = OP;
+    ctx->last.compute_groups = groups;
+    ctx->last.group_warps = groups ? gw : 4;
+    ctx->last.tile_bytes = (int32_t)(tile_elems * 2u);
+    ctx->last.stages = stages;
+    ctx->last.ctas_per_sm = ctas_per_sm;
+    ctx->last.store_lag = lag;
+    ctx->last.grid = (int32_t)grid;
+    ctx->last.smem_bytes = (int32_t)smem;
+    ctx->last.n_tiles = (uint32_t)tiles;
     if (slot) {
         KDN_CUDA(cudaEventRecord(slot->done, stream));
         slot->used = true;
@@ -735,8 +755,22 @@ kdn_status run_ops(kdn_ctx *ctx, int pool_id, int OP, std::vector<HostOp> &dev_o
         // would queue on the copy engine behind the slab transfer in flight and hold the launch back by a whole slab.
         return launch_all(ctx, pool, OP, share, stream, (size_t)kInlineOps);
     };
+    // Fork: the side stream's copies come after everything already queued on the caller's stream (a copy that filled
+    // the pinned chunk, an earlier store into it through another side stream).
+    if (!ctx->fork) KDN_CUDA(cudaEventCreateWithFlags(&ctx->fork, cudaEventDisableTiming));
+    KDN_CUDA(cudaEventRecord(ctx->fork, stream));
+    KDN_CUDA(cudaStreamWaitEvent(side, ctx->fork, 0));
     kdn_status st = run_staged(ctx, pool, OP, host_ops, stream, side, between);
     while (st == KDN_OK && next < dev_ops.size()) st = between();
+    // Join: a store's device-to-host copies run on the side stream; the caller's stream waits for them, so that an
+    // event or a synchronisation on cuda_stream covers the whole call.  (Retrieve and compose end with kernels on
+    // cuda_stream that already waited for their copies.)
+    if (OP == OP_STORE)
+        for (int i = 0; i < 2; ++i)
+            if (ctx->slab_free[i]) {
+                const cudaError_t e = cudaStreamWaitEvent(stream, ctx->slab_free[i], 0);
+                if (e != cudaSuccess && st == KDN_OK) st = KDN_E_CUDA;
+            }
     return st;
 }
 
@@ -898,8 +932,8 @@ kdn_status kdn_create(kdn_ctx **out, int device)
     int major = 0;
     if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device) != cudaSuccess) return fail(KDN_E_CUDA);
     if (major < 10) return fail(KDN_E_UNSUPPORTED);       // the kernels are built for sm_100a only
-    if (cudaDeviceGetAttribute(&ctx->sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return fail(KDN_E_CUDA);
-    if (cudaDeviceGetAttribute(&ctx->smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess) return fail(KDN_E_CUDA);
+    if (cudaDeviceGetAttribute(&ctx->env.sm_count, cudaDevAttrMultiProcessorCount, device) != cudaSuccess) return fail(KDN_E_CUDA);
+    if (cudaDeviceGetAttribute(&ctx->env.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device) != cudaSuccess) return fail(KDN_E_CUDA);
     if (cudaMalloc((void **)&ctx->d_status, sizeof(int)) != cudaSuccess) return fail(KDN_E_NOMEM);
     if (cudaMemset(ctx->d_status, 0, sizeof(int)) != cudaSuccess) return fail(KDN_E_CUDA);
     if (cudaMallocHost((void **)&ctx->h_status, sizeof(int)) != cudaSuccess) return fail(KDN_E_NOMEM);
@@ -942,6 +976,7 @@ void kdn_destroy(kdn_ctx *ctx)
         if (ctx->bounce[i]) cudaFreeHost(ctx->bounce[i]);
         if (ctx->bounce_done[i]) cudaEventDestroy(ctx->bounce_done[i]);
     }
+    if (ctx->fork) cudaEventDestroy(ctx->fork);
     if (ctx->own_side) cudaStreamDestroy(ctx->own_side);
     if (ctx->d_status) cudaFree(ctx->d_status);
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
@@ -1151,7 +1186,7 @@ kdn_status kdn_set_tuning(kdn_ctx *ctx, const kdn_tuning *tuning)
     if (tuning->compute_groups < 0) return KDN_E_INVAL;
     if (tuning->compute_groups > kMaxGroups) return KDN_E_UNSUPPORTED;
     if (tuning->group_warps != 0 && tuning->group_warps != 1 && tuning->group_warps != 4) return KDN_E_UNSUPPORTED;
-    if (tuning->tile_bytes > ctx->smem_optin) return KDN_E_UNSUPPORTED;
+    if (tuning->tile_bytes > ctx->env.smem_optin) return KDN_E_UNSUPPORTED;
     ctx->tuning = *tuning;
     return KDN_OK;
 }
@@ -1172,7 +1207,21 @@ kdn_status kdn_set_staging_bytes(kdn_ctx *ctx, size_t bytes_per_slab)
     return KDN_OK;
 }
 
+kdn_status kdn_set_wait_limit_ns(kdn_ctx *ctx, uint64_t ns)
+{
+    if (!ctx) return KDN_E_INVAL;
+    ctx->wait_limit_ns = ns ? (unsigned long long)ns : kWaitLimitNs;
+    return KDN_OK;
+}
+
 uint64_t kdn_launch_count(const kdn_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+kdn_status kdn_last_launch(const kdn_ctx *ctx, kdn_launch_info *out)
+{
+    if (!ctx || !out) return KDN_E_INVAL;
+    *out = ctx->last;
+    return KDN_OK;
+}
 
 const char *kdn_strerror(kdn_status status)
 {
@@ -1220,8 +1269,7 @@ static_assert(kStOffTable - kStOffRope == sizeof(RopeParam) * KDN_STATIC_MAX_PAR
 
 struct StaticDev {
     unsigned char *base = nullptr;          // device address of g_static_scratch on this device
-    int sm_count = 0;
-    int smem_optin = 0;
+    LaunchEnv env;
 };
 StaticDev g_static_dev[kStMaxDevices];
 std::mutex g_static_mutex;
@@ -1236,11 +1284,21 @@ kdn_status static_setup(int device, StaticDev **out)
         int major = 0;
         KDN_CUDA(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device));
         if (major < 10) return KDN_E_UNSUPPORTED;
-        KDN_CUDA(cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, device));
-        KDN_CUDA(cudaDeviceGetAttribute(&d.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device));
+        KDN_CUDA(cudaDeviceGetAttribute(&d.env.sm_count, cudaDevAttrMultiProcessorCount, device));
+        KDN_CUDA(cudaDeviceGetAttribute(&d.env.smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, device));
         void *ptr = nullptr;
         KDN_CUDA(cudaGetSymbolAddress(&ptr, g_static_scratch));
         if (!ptr) return KDN_E_CUDA;
+        // Load every kernel a later call can launch and raise its shared-memory limit now, so that no later call
+        // meets a first-use step of the runtime: the three compose forms the built-in shapes use (pure copy, decoding
+        // without rotation, rotation) and the rotation-table kernel.
+        int per_sm = 0;
+        kdn_status st = d.env.resident(kdn_compose_kernel<0, 4>, threads_for(0, 4), 1024, &per_sm);
+        if (st == KDN_OK) st = d.env.resident(kdn_compose_kernel<1, 4>, threads_for(1, 4), 1024, &per_sm);
+        if (st == KDN_OK) st = d.env.resident(kdn_compose_kernel<2, 4>, threads_for(2, 4), 1024, &per_sm);
+        if (st != KDN_OK) return st;
+        cudaFuncAttributes fa{};
+        KDN_CUDA(cudaFuncGetAttributes(&fa, kdn_rope_table_kernel));
         d.base = (unsigned char *)ptr;
     }
     *out = &d;
@@ -1314,7 +1372,7 @@ extern "C" kdn_status kdn_compose_static(int device, const kdn_pool_desc *pool, 
     const unsigned stage_bytes = a_bytes + b_bytes + s_bytes;
     const int ctas_per_sm = def.ctas_per_sm;
     int stages = def.stages;
-    const size_t smem_limit = (size_t)sd->smem_optin;
+    const size_t smem_limit = (size_t)sd->env.smem_optin;
     st = fit_stages(stages, def.groups, def.lag, true, stage_bytes, ctas_per_sm, smem_limit);
     if (st != KDN_OK) return st;
     const size_t smem = smem_bytes(stages, stage_bytes);
@@ -1373,14 +1431,19 @@ extern "C" kdn_status kdn_compose_static(int device, const kdn_pool_desc *pool, 
         lp.off_b = a_bytes;
         lp.off_s = a_bytes + b_bytes;
         lp.store_lag = def.lag;
-        const unsigned long long want = (unsigned long long)sd->sm_count * (unsigned)ctas_per_sm;
+        const unsigned long long want = (unsigned long long)sd->env.sm_count * (unsigned)ctas_per_sm;
         const unsigned grid = (unsigned)(tiles < want ? tiles : want);
-        st = launch_tiles(OP_COMPOSE, def.groups, def.gw, grid, smem, stream, lp);
+        lp.wait_limit_ns = kWaitLimitNs;
+        {
+            std::lock_guard<std::mutex> lock(g_static_mutex);     // the per-device occupancy cache is shared by all callers
+            st = launch_tiles(sd->env, OP_COMPOSE, def.groups, def.gw, grid, smem, stream, lp);
+        }
         if (st != KDN_OK) return st;
     }
     if (!wait) return KDN_OK;
-    KDN_CUDA(cudaStreamSynchronize(stream));
+    // the status word comes back on the caller's stream: no other stream of the process is involved
     int dev_status = 0;
-    KDN_CUDA(cudaMemcpy(&dev_status, sd->base, sizeof(int), cudaMemcpyDeviceToHost));
+    KDN_CUDA(cudaMemcpyAsync(&dev_status, sd->base, sizeof(int), cudaMemcpyDeviceToHost, stream));
+    KDN_CUDA(cudaStreamSynchronize(stream));
     return (dev_status >= KDN_OK && dev_status <= KDN_E_TIMEOUT) ? (kdn_status)dev_status : KDN_E_CUDA;
 }

@@ -45,7 +45,7 @@ __host__ __device__ constexpr int min_ctas_for_compose(int groups, int group_war
 constexpr int kThreadsCopy = 64;                             // loader + storer
 constexpr int kMaxStages = 32;
 constexpr int kMaxStoreLag = 16;          // most bulk-store groups allowed to be still reading shared memory
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // default limit of a pipeline wait, and the limit of every drain wait
 
 enum : uint32_t { TF_CODED = 1u, TF_ROTATE = 2u, TF_SCALES_PLAIN = 4u, TF_INT4 = 8u,   // TF_CODED: int8 or int4
                   TF_KCHAN = 16u };   // key tile of a per-channel key codec: one scale per channel, row_elems of them
@@ -107,6 +107,7 @@ struct Launch {
     int store_lag;            // bulk-store groups that may still be reading shared memory (1..kMaxStoreLag)
     int reload_first;         // copy form: after recycling a slot the storer lets the loader queue the reload
                               // before it queues the next store (see the storer loop)
+    unsigned long long wait_limit_ns;   // a pipeline wait gives up after this long (the drain waits keep kWaitLimitNs)
     DevOp inline_ops[kInlineOps];
 };
 
@@ -163,21 +164,22 @@ __device__ __forceinline__ bool mbar_try_wait_parked(uint32_t bar, uint32_t pari
     return ok != 0;
 }
 // Bounded wait: true when the phase completed; false when the CTA is aborting or the limit passed.
-__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+__device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                            unsigned long long limit_ns = kWaitLimitNs)
 {
-    unsigned long long t0 = global_timer_ns();
-    for (uint32_t n = 1;; ++n) {
-        if (mbar_try_wait_parked(bar, parity, 20000u)) return true;
-        if ((n & 15u) == 0u) {
-            if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) { *abort_flag = 1; return false; }
-        }
+    const unsigned long long t0 = global_timer_ns();
+    const uint32_t hint = limit_ns < 20000ull ? (uint32_t)limit_ns : 20000u;   // never park for longer than the limit
+    for (;;) {
+        if (mbar_try_wait_parked(bar, parity, hint)) return true;
+        if (*abort_flag) return false;
+        if (global_timer_ns() - t0 > limit_ns) { *abort_flag = 1; return false; }
     }
 }
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int *abort_flag,
+                                          unsigned long long limit_ns = kWaitLimitNs)
 {
     if (mbar_try_wait(bar, parity)) return true;
-    return mbar_wait_slow(bar, parity, abort_flag);
+    return mbar_wait_slow(bar, parity, abort_flag, limit_ns);
 }
 // Bulk async copy global -> this CTA's shared memory, completion counted on an mbarrier.
 // (No cluster is launched: the CTA's own shared window is the cluster window.)
@@ -770,8 +772,10 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
             decode_tile<OP>(P, base + 32u + lane < n_my ? bid + (base + 32u + lane) * grid : 0xffffffffu, nxt);
             const unsigned cnt = n_my - base < 32u ? n_my - base : 32u;
             for (unsigned t = 0; t < cnt; ++t) {
+                bool ok = true;                               // lane t: the slot was free and the tile's copies are queued
                 if ((unsigned)lane == t) {
-                    if (mbar_wait(sm.empty + 8u * st, ph ^ 1u, sm.abort_flag)) {
+                    ok = mbar_wait(sm.empty + 8u * st, ph ^ 1u, sm.abort_flag, P.wait_limit_ns);
+                    if (ok) {
                         sm.desc[st] = cur;
                         const uint32_t bar = sm.full + 8u * st;
                         unsigned char *A = sm.stage0 + (size_t)st * P.stage_bytes;
@@ -796,8 +800,12 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                         }
                     }
                 }
-                __syncwarp();
-                if (__any_sync(0xffffffffu, *sm.abort_flag != 0)) { aborted = true; break; }
+                if (__any_sync(0xffffffffu, !ok || *sm.abort_flag != 0)) {
+                    // a tile queued just before the CTA gave up still counts: the drain below has to wait for it
+                    if (__shfl_sync(0xffffffffu, ok ? 1 : 0, (int)t)) ++issued;
+                    aborted = true;
+                    break;
+                }
                 ++issued;
                 if (lane == 0) *sm.issued = issued;
                 if (++st == (unsigned)S) { st = 0; ph ^= 1u; }
@@ -821,13 +829,13 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
             unsigned st = 0, st2 = 0;                         // slot being stored / slot being recycled, with the
             uint32_t ph = 0, ph2 = 0;                         // phases of their barriers
             for (unsigned slot = 0; slot < n_my; ++slot) {
-                if (!mbar_wait(sm.full + 8u * st, ph, sm.abort_flag)) break;
+                if (!mbar_wait(sm.full + 8u * st, ph, sm.abort_flag, P.wait_limit_ns)) break;
                 const TileDesc d = sm.desc[st];
                 unsigned char *A = sm.stage0 + (size_t)st * P.stage_bytes;
                 if (d.n != 0u) {
                     const bool computed = kCompute && (OP == OP_STORE ? (d.flags & TF_CODED) != 0u
                                                                        : (d.flags & (TF_CODED | TF_ROTATE)) != 0u);
-                    if (computed && !mbar_wait(sm.ready + 8u * st, ph, sm.abort_flag)) break;
+                    if (computed && !mbar_wait(sm.ready + 8u * st, ph, sm.abort_flag, P.wait_limit_ns)) break;
                     if (OP == OP_STORE) {
                         if (d.flags & TF_CODED) {
                             bulk_s2g((void *)d.g_chunk, smem_u32(A + P.off_b), (d.flags & TF_INT4) ? d.n >> 1 : d.n);
@@ -846,7 +854,7 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                 // and every compute warp has moved past it
                 bulk_wait_read_n(P.store_lag);
                 if (slot >= (unsigned)P.store_lag) {
-                    if (kCompute && !mbar_wait(sm.ready + 8u * st2, ph2, sm.abort_flag)) break;
+                    if (kCompute && !mbar_wait(sm.ready + 8u * st2, ph2, sm.abort_flag, P.wait_limit_ns)) break;
                     mbar_arrive(sm.empty + 8u * st2);
                     if (++st2 == (unsigned)S) { st2 = 0; ph2 ^= 1u; }
                     // The SM works through its bulk copies in the order they were queued, and a store holds the
@@ -880,7 +888,7 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
         unsigned st = (unsigned)group;                        // S is a multiple of kGroups: st wraps exactly at S
         uint32_t ph = 0;
         for (unsigned slot = (unsigned)group; slot < n_my; slot += (unsigned)kGroups) {
-            if (!mbar_wait(sm.full + 8u * st, ph, sm.abort_flag)) break;
+            if (!mbar_wait(sm.full + 8u * st, ph, sm.abort_flag, P.wait_limit_ns)) break;
             const unsigned n = sm.desc[st].n;
             const unsigned flags = sm.desc[st].flags;
             unsigned char *A = sm.stage0 + (size_t)st * P.stage_bytes;
@@ -1078,7 +1086,13 @@ __global__ void __launch_bounds__(512) kdn_store_kc_kernel(const __grid_constant
     if (*abort_flag) return;
     const bool landed = mbar_wait(bar, 0u, abort_flag);
     if (!__syncthreads_and(landed)) {                                         // all threads leave together
-        if (tid == 0) atomicCAS(P.status, 0, kStatusTimeout);
+        if (tid == 0) {
+            atomicCAS(P.status, 0, kStatusTimeout);
+            // one more bounded wait, so that the CTA does not leave while a copy into its shared memory is in flight
+            const unsigned long long t0 = global_timer_ns();
+            while (!mbar_try_wait(bar, 0u))
+                if (global_timer_ns() - t0 > kWaitLimitNs) break;
+        }
         return;
     }
 

@@ -20,7 +20,7 @@ KDN_MEM_DEVICE, KDN_MEM_PINNED_HOST = 0, 1
 
 EXPORTS = ["kdn_create", "kdn_destroy", "kdn_pool_register", "kdn_chunk_bytes", "kdn_validate_xfer",
            "kdn_validate_compose", "kdn_store", "kdn_retrieve", "kdn_compose", "kdn_status_sync",
-           "kdn_set_tuning", "kdn_set_staging_bytes", "kdn_launch_count", "kdn_strerror",
+           "kdn_set_tuning", "kdn_set_staging_bytes", "kdn_set_wait_limit_ns", "kdn_launch_count", "kdn_last_launch", "kdn_strerror",
            "kdn_compose_static", "kdn_retrieve_layerwise", "kdn_store_file", "kdn_retrieve_file",
            "kdn_store_sparse", "kdn_retrieve_sparse", "kdn_compose_select",
            "kdn_key_hash", "kdn_checksum", "kdn_header_fill", "kdn_header_check", "kdn_index_create", "kdn_index_destroy",
@@ -71,6 +71,12 @@ class kdn_chunk_header(C.Structure):
 class kdn_index_info(C.Structure):
     _fields_ = [("capacity_bytes", C.c_size_t), ("bytes", C.c_size_t), ("entries", C.c_size_t),
                 ("hits", C.c_uint64), ("misses", C.c_uint64), ("evictions", C.c_uint64)]
+
+
+class kdn_launch_info(C.Structure):
+    _fields_ = [("op", C.c_int32), ("compute_groups", C.c_int32), ("group_warps", C.c_int32), ("tile_bytes", C.c_int32),
+                ("stages", C.c_int32), ("ctas_per_sm", C.c_int32), ("store_lag", C.c_int32), ("grid", C.c_int32),
+                ("smem_bytes", C.c_int32), ("n_tiles", C.c_uint32)]
 
 
 class kdn_tuning(C.Structure):
@@ -126,8 +132,12 @@ def _load() -> C.CDLL:
     lib.kdn_set_tuning.argtypes = [vp, C.POINTER(kdn_tuning)]
     lib.kdn_set_staging_bytes.restype = i32
     lib.kdn_set_staging_bytes.argtypes = [vp, C.c_size_t]
+    lib.kdn_set_wait_limit_ns.restype = i32
+    lib.kdn_set_wait_limit_ns.argtypes = [vp, C.c_uint64]
     lib.kdn_launch_count.restype = C.c_uint64
     lib.kdn_launch_count.argtypes = [vp]
+    lib.kdn_last_launch.restype = i32
+    lib.kdn_last_launch.argtypes = [vp, C.POINTER(kdn_launch_info)]
     lib.kdn_key_hash.restype = C.c_uint64
     lib.kdn_key_hash.argtypes = [vp, C.c_size_t]
     lib.kdn_checksum.restype = i32
@@ -359,8 +369,21 @@ def kdn_set_staging_bytes(ctx, bytes_per_slab: int) -> None:
     _check(lib.kdn_set_staging_bytes(ctx, int(bytes_per_slab)), "kdn_set_staging_bytes")
 
 
+def kdn_set_wait_limit_ns(ctx, ns: int) -> None:
+    _check(lib.kdn_set_wait_limit_ns(ctx, int(ns)), "kdn_set_wait_limit_ns")
+
+
 def kdn_launch_count(ctx) -> int:
     return int(lib.kdn_launch_count(ctx))
+
+
+def kdn_last_launch(ctx) -> dict:
+    """Shape of the most recent tile-pipeline launch, with the kernel's name as the profiler prints it."""
+    info = kdn_launch_info()
+    _check(lib.kdn_last_launch(ctx, C.byref(info)), "kdn_last_launch")
+    d = {name: int(getattr(info, name)) for name, _ in kdn_launch_info._fields_}
+    d["kernel"] = "kdn_%s_kernel<%d, %d>" % (("store", "retrieve", "compose")[d["op"]], d["compute_groups"], d["group_warps"])
+    return d
 
 
 # ------------------------------------------------------------------------ storage-module shell --

@@ -465,3 +465,79 @@ def test_layerwise_retrieve_equals_retrieve_and_events_order_layers(codec):
             K.kdn_retrieve_layerwise(dev.ctx, dev.pool_id, ops, 0, dev.stream.cuda_stream)
     finally:
         dev.close()
+
+
+@pytest.mark.parametrize("codec", [RAW, INT8])
+def test_staged_calls_are_ordered_on_the_callers_stream(codec):
+    """Host-resident chunks move on a side stream, but the call is ordered on cuda_stream alone: (a) an event recorded
+    on cuda_stream after a store covers the bytes in page-locked memory, even when the caller's side stream is busy;
+    (b) a page-locked chunk filled by a copy on cuda_stream is retrieved without a host synchronisation in between."""
+    shape = synth.TOY.with_(n_layers=6, n_kv_heads=4, head_dim=64, block_size=16, n_blocks=128)
+    dev = Device(shape, seed=77)
+    try:
+        K = dev.K
+        K.kdn_set_staging_bytes(dev.ctx, 1024 * 1024)          # one layer of 400 tokens is 400 KiB raw
+        host = dev.pool_np()
+        perm = np.random.default_rng(8).permutation(128).astype(np.int32)
+        T = 400
+        want = oracle.store(host, perm[:26], 9, T, codec)
+        ballast = torch.empty(1 << 28, dtype=torch.uint8, device=dev.dev)
+        # (a) the caller's own side stream is kept busy, so the copies out of the slabs start late
+        side = torch.cuda.Stream(device=dev.dev)
+        hbuf = dev.chunk_buf(T, codec, pinned=True, fill=0)
+        with torch.cuda.stream(side):
+            for _ in range(8):
+                ballast.fill_(1)
+        K.kdn_store(dev.ctx, dev.pool_id, [dev.op(dev.table(perm[:26]), 9, hbuf, T, codec)], dev.stream.cuda_stream, side.cuda_stream)
+        ev = torch.cuda.Event()
+        ev.record(dev.stream)
+        ev.synchronize()                                        # nothing else is waited for
+        assert np.array_equal(hbuf.numpy(), want)
+        torch.cuda.synchronize()
+        # (b) the chunk reaches page-locked memory by a copy queued on cuda_stream behind other work
+        hbuf2 = dev.chunk_buf(T, codec, pinned=True, fill=0)
+        staged = torch.from_numpy(want).to(dev.dev)
+        torch.cuda.synchronize()
+        with torch.cuda.stream(dev.stream):
+            for _ in range(8):
+                ballast.fill_(2)
+            hbuf2.copy_(staged, non_blocking=True)
+        dev.retrieve([dev.op(dev.table(perm[40:66]), 2, hbuf2, T, codec)])
+        assert dev.sync() == 0
+        ref = host.copy()
+        oracle.retrieve(ref, perm[40:66], 2, T, codec, want)
+        assert np.array_equal(dev.pool_np(), ref)
+    finally:
+        dev.close()
+
+
+@pytest.mark.parametrize("codec", [RAW, INT8])
+def test_a_wait_that_runs_out_is_reported_and_the_context_recovers(codec):
+    """Every wait inside the tile pipeline is bounded.  With the bound set below the latency of a memory access the
+    launch gives up at once: the call returns, kdn_status_sync reports KDN_E_TIMEOUT, no CTA leaves with a copy in
+    flight, and once the default bound is back the same context gives bit-exact results."""
+    shape = synth.TOY.with_(n_layers=2, n_kv_heads=4, head_dim=64, block_size=16, n_blocks=64)
+    dev = Device(shape, seed=5)
+    try:
+        K = dev.K
+        host = dev.pool_np()
+        tab = np.random.default_rng(4).permutation(64)[:20].astype(np.int32)
+        T, off = 300, 5
+        buf = dev.chunk_buf(T, codec)
+        K.kdn_set_wait_limit_ns(dev.ctx, 40)
+        dev.store([dev.op(dev.table(tab), off, buf, T, codec)])
+        assert dev.sync() == K.KDN_E_TIMEOUT
+        assert dev.sync() == 0                                  # the status word was cleared by the read
+        assert np.array_equal(dev.pool_np(), host)              # a store never writes the pool
+        K.kdn_set_wait_limit_ns(dev.ctx, 0)                     # back to the default
+        dev.store([dev.op(dev.table(tab), off, buf, T, codec)])
+        assert dev.sync() == 0
+        assert np.array_equal(to_np(buf), oracle.store(host, tab, off, T, codec))
+        dst = np.random.default_rng(5).permutation(64)[:20].astype(np.int32)
+        dev.retrieve([dev.op(dev.table(dst), off, buf, T, codec)])
+        assert dev.sync() == 0
+        ref = host.copy()
+        oracle.retrieve(ref, dst, off, T, codec, oracle.store(host, tab, off, T, codec))
+        assert np.array_equal(dev.pool_np(), ref)
+    finally:
+        dev.close()
