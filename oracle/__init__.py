@@ -13,6 +13,9 @@ Array conventions (all host, C-contiguous numpy):
                                 int4: nibbles [L][2][T][H][D/2] bytes (element 2k low, 2k+1 high) then the same scales
                                 per-channel key codecs: the same codes, then per layer fp32 k_scales [ceil(T/64)][H*D]
                                 followed by fp32 v_scales [T][H*D/64]
+                                token-delta Rice codecs: uint64 seg_off[S+1], fp32 scales[S][H*D], uint8 lens[S][H*D],
+                                uint8 params[S][H*D], then the segments' bit streams (see td_layout); the array has
+                                the worst-case capacity, td_used_bytes() of it are defined
 """
 from __future__ import annotations
 
@@ -28,6 +31,8 @@ INT8_G64 = 1
 INT4_G64 = 2
 INT8_KC64 = 3      # keys grouped along tokens (64 tokens of one channel), values as INT8_G64
 INT4_KC64 = 4      # the same with codes in [-7, 7]
+INT8_TD64 = 5      # K and V grouped along tokens, each group's codes as a Rice-coded sub-stream (direct or token delta)
+INT4_TD64 = 6      # the same with codes in [-7, 7]
 GROUP = 64
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
@@ -105,6 +110,20 @@ def _declare(L):
     L.kdn_oracle_quant4_group.argtypes = [vp, vp, vp]
     L.kdn_oracle_quant_channel.restype = None
     L.kdn_oracle_quant_channel.argtypes = [vp, i32, i32, vp, vp]
+    L.kdn_oracle_td_layout.restype = i32
+    L.kdn_oracle_td_layout.argtypes = [i32, i32, i32, i32, i32, vp]
+    L.kdn_oracle_td_max_len.restype = i32
+    L.kdn_oracle_td_max_len.argtypes = [i32]
+    L.kdn_oracle_zigzag.restype = C.c_uint
+    L.kdn_oracle_zigzag.argtypes = [i32]
+    L.kdn_oracle_unzigzag.restype = i32
+    L.kdn_oracle_unzigzag.argtypes = [C.c_uint]
+    L.kdn_oracle_rice_bits.restype = i32
+    L.kdn_oracle_rice_bits.argtypes = [C.c_uint, i32, i32]
+    L.kdn_oracle_td_encode_channel.restype = None
+    L.kdn_oracle_td_encode_channel.argtypes = [vp, i32, i32, vp, C.POINTER(i32), C.POINTER(i32)]
+    L.kdn_oracle_td_decode_channel.restype = None
+    L.kdn_oracle_td_decode_channel.argtypes = [vp, i32, i32, i32, vp]
     L.kdn_oracle_dequant.restype = C.c_uint16
     L.kdn_oracle_dequant.argtypes = [C.c_int8, C.c_float]
     L.kdn_oracle_rope_angle.restype = f64
@@ -272,6 +291,56 @@ def quant_channel(x_bf16: np.ndarray, qmax: int):
     s = np.zeros(1, dtype=np.float32)
     lib().kdn_oracle_quant_channel(_ptr(x), x.size, int(qmax), _ptr(q), _ptr(s))
     return q, s[0]
+
+
+def td_layout(L: int, H: int, D: int, T: int, codec: int) -> dict:
+    """Byte offsets of the regions of a token-delta chunk: segments, scales, lens, params, streams, capacity."""
+    out = (C.c_size_t * 6)()
+    if lib().kdn_oracle_td_layout(L, H, D, T, codec, out):
+        raise ValueError("shape or codec not codable")
+    return dict(zip(("segments", "scales", "lens", "params", "streams", "capacity"), [int(x) for x in out]))
+
+
+def td_used_bytes(chunk: np.ndarray, L: int, H: int, D: int, T: int, codec: int) -> int:
+    """The bytes of a stored token-delta chunk that are defined: seg_off[S]."""
+    lay = td_layout(L, H, D, T, codec)
+    return int(np.ascontiguousarray(chunk[:8 * (lay["segments"] + 1)]).view(np.uint64)[lay["segments"]])
+
+
+def td_max_len(qmax: int) -> int:
+    return int(lib().kdn_oracle_td_max_len(int(qmax)))
+
+
+def zigzag(e: int) -> int:
+    return int(lib().kdn_oracle_zigzag(int(e)))
+
+
+def unzigzag(u: int) -> int:
+    return int(lib().kdn_oracle_unzigzag(int(u)))
+
+
+def rice_bits(u: int, k: int, raw_bits: int) -> int:
+    return int(lib().kdn_oracle_rice_bits(int(u), int(k), int(raw_bits)))
+
+
+def td_encode_channel(q, qmax: int):
+    """Encode the n <= 64 codes of one group -> (bytes, param = mode * 8 + k)."""
+    q = np.ascontiguousarray(q, dtype=np.int8)
+    if q.ndim != 1 or not 1 <= q.size <= GROUP:
+        raise ValueError("a group is 1..64 codes")
+    out = np.zeros(td_max_len(qmax), dtype=np.uint8)
+    n, p = C.c_int(0), C.c_int(0)
+    lib().kdn_oracle_td_encode_channel(_ptr(q), q.size, int(qmax), _ptr(out), C.byref(n), C.byref(p))
+    return out[:n.value].copy(), p.value
+
+
+def td_decode_channel(data, param: int, n: int, qmax: int) -> np.ndarray:
+    buf = np.zeros(td_max_len(qmax) + 8, dtype=np.uint8)
+    data = np.ascontiguousarray(data, dtype=np.uint8)
+    buf[:data.size] = data
+    q = np.zeros(n, dtype=np.int8)
+    lib().kdn_oracle_td_decode_channel(_ptr(buf), int(param), int(n), int(qmax), _ptr(q))
+    return q
 
 
 def dequant(q: int, scale) -> int:

@@ -47,6 +47,32 @@
  *                    fp32 k_scales[ceil(T/64)][head*D] followed by fp32 v_scales[t][head*D/64]; layers follow
  *                    each other; the scales follow the codes.  Decode is R5 with the element's own scale.
  *                    Token lists (R7) are not defined for these codecs.
+ *   R9  token-delta Rice codecs (codecs 5 = int8, 6 = int4; not prescribed by the paper: Sec. 3.2 "KV-cache delivery"
+ *                    cites a scheme that quantises a KV cache and then encodes it into binary strings, and reports
+ *                    more than tenfold reductions for combined techniques.  This is this library's own bitstream.)
+ *                    Quantisation: K AND V planes are grouped along tokens as the keys of R4" are: group = the chunk
+ *                    tokens 64 g .. min(64 g + 63, T - 1) of one (l, kv, head, d) channel; scale, inv and codes as in
+ *                    R4 / R4' (127 or 7).  A group's codes q_0 .. q_{n-1} become one SUB-STREAM of n symbols:
+ *                      mode 0 (direct):       e_t = q_t
+ *                      mode 1 (token delta):  e_t = q_t - q_{t-1}, with q_{-1} = 0
+ *                      zigzag:                u_t = 2 e_t if e_t >= 0, else -2 e_t - 1
+ *                      Rice code, parameter k in 0..7: quo = u >> k; if quo < 15: quo one-bits, a zero-bit, then
+ *                      the k low bits of u, high bit first; else (escape): 15 one-bits, then u in `raw` bits, high
+ *                      bit first, raw = 9 (int8: u <= 508) or 5 (int4: u <= 28).
+ *                    Bits fill bytes from the most significant bit down; the sub-stream ends on a byte boundary,
+ *                    padded with zero bits.  The encoder takes the (mode, k) with the fewest total bits, the first
+ *                    such in the order (0,0), (0,1), .., (0,7), (1,0), .., (1,7); param = mode * 8 + k.  A sub-stream
+ *                    is never longer than 72 bytes (int8: mode 0, k = 7 costs at most 9 bits a symbol) or 40 bytes
+ *                    (int4: mode 0, k = 3 costs at most 5).
+ *                    Chunk: S = 2 L ceil(T/64) segments, segment (l, kv, g) has index (2 l + kv) ceil(T/64) + g and
+ *                    R = head * D channels.  uint64 seg_off[S + 1] (padded to 16 bytes), fp32 scales[S][R],
+ *                    uint8 lens[S][R] (bytes of each sub-stream), uint8 params[S][R], then the segments' streams:
+ *                    segment s starts at byte seg_off[s] (a multiple of 16; seg_off[0] = the end of params), holds
+ *                    its R sub-streams back to back in channel order, and is padded with zero bytes to 16;
+ *                    seg_off[S] = the bytes the chunk uses.  A chunk buffer has the worst-case capacity
+ *                    fixed part + S * R * (72 or 40); bytes past seg_off[S] are not defined.
+ *                    Decode: undo Rice, zigzag and the delta, then R5 with the channel's scale.  Token lists (R7)
+ *                    are not defined for these codecs.
  *   R6  re-rotation  stored keys carry rotary position embedding at absolute
  *                    positions base_pos + t (what an engine's pool holds), so
  *                    reuse at dst_pos (Sec. 3.2 "KV-cache blending": a
@@ -85,6 +111,7 @@
 #include <math.h>
 #include <stddef.h>
 #include <stdint.h>
+#include <stdlib.h>
 #include <string.h>
 
 #define KDN_ORACLE_RAW_BF16 0
@@ -92,6 +119,8 @@
 #define KDN_ORACLE_INT4_G64 2
 #define KDN_ORACLE_INT8_KC64 3
 #define KDN_ORACLE_INT4_KC64 4
+#define KDN_ORACLE_INT8_TD64 5
+#define KDN_ORACLE_INT4_TD64 6
 #define KDN_ORACLE_GROUP 64
 
 /* ---------------------------------------------------------------- bf16 -- */
@@ -158,6 +187,8 @@ uint16_t kdn_oracle_f64_to_bf16(double x)
 
 /* --------------------------------------------------------------- sizes -- */
 
+int kdn_oracle_td_layout(int L, int H, int D, int T, int codec, size_t *out);
+
 /* R2: bytes of one chunk of T tokens.  0 when the codec cannot hold the shape. */
 size_t kdn_oracle_chunk_bytes(int L, int H, int D, int T, int codec)
 {
@@ -178,6 +209,11 @@ size_t kdn_oracle_chunk_bytes(int L, int H, int D, int T, int codec)
         size_t n_groups = ((size_t)T + KDN_ORACLE_GROUP - 1u) / KDN_ORACLE_GROUP;
         size_t scales_per_layer = n_groups * hd + (size_t)T * hd / KDN_ORACLE_GROUP;     /* R4": K then V */
         return (codec == KDN_ORACLE_INT4_KC64 ? elems / 2u : elems) + 4u * (size_t)L * scales_per_layer;
+    }
+    if (codec == KDN_ORACLE_INT8_TD64 || codec == KDN_ORACLE_INT4_TD64) {
+        size_t lay[6];
+        if (kdn_oracle_td_layout(L, H, D, T, codec, lay)) return 0;
+        return lay[5];                                       /* R9: worst-case capacity */
     }
     return 0;
 }
@@ -248,6 +284,121 @@ uint16_t kdn_oracle_dequant(int8_t q, float scale)
     return kdn_oracle_f32_to_bf16(prod);
 }
 
+/* ------------------------------------------- token-delta Rice codecs (R9) -- */
+
+static int td_is(int codec) { return codec == KDN_ORACLE_INT8_TD64 || codec == KDN_ORACLE_INT4_TD64; }
+static int td_qmax(int codec) { return codec == KDN_ORACLE_INT8_TD64 ? 127 : 7; }
+static int td_raw_bits(int qmax) { return qmax == 127 ? 9 : 5; }           /* bits that hold the largest symbol, 4 qmax */
+
+/* R9: longest sub-stream in bytes. */
+int kdn_oracle_td_max_len(int qmax) { return qmax == 127 ? 72 : 40; }
+
+/* R9: byte offsets of a chunk's regions: out[0] = S (segments), out[1] = scales, out[2] = lens, out[3] = params,
+ * out[4] = first segment's streams (the end of the fixed part), out[5] = capacity.  Non-zero: shape not codable. */
+int kdn_oracle_td_layout(int L, int H, int D, int T, int codec, size_t *out)
+{
+    if (!td_is(codec) || L <= 0 || H <= 0 || D <= 0 || T < 0 || D % KDN_ORACLE_GROUP) return 3;
+    size_t G = ((size_t)T + KDN_ORACLE_GROUP - 1u) / KDN_ORACLE_GROUP;
+    size_t S = 2u * (size_t)L * G, R = (size_t)H * (size_t)D;
+    out[0] = S;
+    out[1] = (8u * (S + 1u) + 15u) / 16u * 16u;
+    out[2] = out[1] + 4u * S * R;
+    out[3] = out[2] + S * R;
+    out[4] = out[3] + S * R;
+    out[5] = out[4] + S * ((R * (size_t)kdn_oracle_td_max_len(td_qmax(codec)) + 15u) / 16u * 16u);
+    return 0;
+}
+
+unsigned kdn_oracle_zigzag(int e) { return e >= 0 ? 2u * (unsigned)e : 2u * (unsigned)(-e) - 1u; }
+int kdn_oracle_unzigzag(unsigned u) { return (u & 1u) ? -(int)((u + 1u) / 2u) : (int)(u / 2u); }
+
+/* R9: bits one symbol costs. */
+int kdn_oracle_rice_bits(unsigned u, int k, int raw_bits)
+{
+    unsigned quo = u >> k;
+    return quo < 15u ? (int)quo + 1 + k : 15 + raw_bits;
+}
+
+/* Bit `pos` of a byte string, counted from the most significant bit of byte 0. */
+static void put_bit(uint8_t *buf, size_t *pos, unsigned bit)
+{
+    if (bit) buf[*pos / 8u] |= (uint8_t)(0x80u >> (*pos % 8u));
+    ++*pos;
+}
+static unsigned get_bit(const uint8_t *buf, size_t *pos)
+{
+    unsigned bit = (buf[*pos / 8u] >> (7u - *pos % 8u)) & 1u;
+    ++*pos;
+    return bit;
+}
+
+static void rice_put(uint8_t *buf, size_t *pos, unsigned u, int k, int raw_bits)
+{
+    unsigned quo = u >> k;
+    if (quo < 15u) {
+        for (unsigned i = 0; i < quo; ++i) put_bit(buf, pos, 1u);
+        put_bit(buf, pos, 0u);
+        for (int b = k - 1; b >= 0; --b) put_bit(buf, pos, (u >> b) & 1u);
+    } else {
+        for (int i = 0; i < 15; ++i) put_bit(buf, pos, 1u);
+        for (int b = raw_bits - 1; b >= 0; --b) put_bit(buf, pos, (u >> b) & 1u);
+    }
+}
+
+static unsigned rice_get(const uint8_t *buf, size_t *pos, int k, int raw_bits)
+{
+    unsigned quo = 0;
+    while (quo < 15u && get_bit(buf, pos)) ++quo;             /* stops after the zero-bit, or after 15 one-bits */
+    unsigned u = 0;
+    if (quo < 15u) {
+        for (int b = 0; b < k; ++b) u = (u << 1) | get_bit(buf, pos);
+        return (quo << k) | u;
+    }
+    for (int b = 0; b < raw_bits; ++b) u = (u << 1) | get_bit(buf, pos);
+    return u;
+}
+
+/* R9: the symbol of code t of a group under `mode`. */
+static unsigned td_symbol(const int8_t *q, int t, int mode)
+{
+    int prev = (mode == 1 && t > 0) ? q[t - 1] : 0;
+    return kdn_oracle_zigzag((int)q[t] - prev);
+}
+
+/* R9: encode the n <= 64 codes of one group into out (at least kdn_oracle_td_max_len(qmax) bytes, zeroed here).
+ * *len_out = bytes used, *param_out = mode * 8 + k. */
+void kdn_oracle_td_encode_channel(const int8_t *q, int n, int qmax, uint8_t *out, int *len_out, int *param_out)
+{
+    int raw_bits = td_raw_bits(qmax);
+    long best_bits = -1;
+    int best_mode = 0, best_k = 0;
+    for (int mode = 0; mode < 2; ++mode)
+        for (int k = 0; k < 8; ++k) {
+            long bits = 0;
+            for (int t = 0; t < n; ++t) bits += kdn_oracle_rice_bits(td_symbol(q, t, mode), k, raw_bits);
+            if (best_bits < 0 || bits < best_bits) { best_bits = bits; best_mode = mode; best_k = k; }
+        }
+    memset(out, 0, (size_t)kdn_oracle_td_max_len(qmax));
+    size_t pos = 0;
+    for (int t = 0; t < n; ++t) rice_put(out, &pos, td_symbol(q, t, best_mode), best_k, raw_bits);
+    *len_out = (int)((pos + 7u) / 8u);
+    *param_out = best_mode * 8 + best_k;
+}
+
+/* R9: decode n codes of one group. */
+void kdn_oracle_td_decode_channel(const uint8_t *in, int param, int n, int qmax, int8_t *q)
+{
+    int mode = param >> 3, k = param & 7, raw_bits = td_raw_bits(qmax);
+    size_t pos = 0;
+    int prev = 0;
+    for (int t = 0; t < n; ++t) {
+        int e = kdn_oracle_unzigzag(rice_get(in, &pos, k, raw_bits));
+        int v = mode == 1 ? prev + e : e;
+        q[t] = (int8_t)v;
+        prev = v;
+    }
+}
+
 /* ------------------------------------------------------------- rotation -- */
 
 /* R6: angle of frequency index i (0 <= i < D/2) for a position shift delta. */
@@ -301,8 +452,9 @@ static int check_args_list(const shape_t *s, const int32_t *table, int n_table, 
 {
     if (s->L <= 0 || s->H <= 0 || s->D <= 0 || s->bs <= 0 || s->nb <= 0) return 1;
     if (n < 0 || off < 0 || n_table < 0) return 1;
-    if (codec < KDN_ORACLE_RAW_BF16 || codec > KDN_ORACLE_INT4_KC64) return 3;
+    if (codec < KDN_ORACLE_RAW_BF16 || codec > KDN_ORACLE_INT4_TD64) return 3;
     if ((codec == KDN_ORACLE_INT8_KC64 || codec == KDN_ORACLE_INT4_KC64) && list) return 3;   /* R4": no token lists */
+    if (td_is(codec) && list) return 3;                                                       /* R9: no token lists */
     if (codec != KDN_ORACLE_RAW_BF16 && s->D % KDN_ORACLE_GROUP) return 3;
     for (int i = 0; i < n; ++i) {
         int64_t rel = list ? list[i] : i;
@@ -379,6 +531,79 @@ static int store_kc(const shape_t *s, const uint16_t *pool, const int32_t *table
     return 0;
 }
 
+/* R9: store with K and V grouped along tokens, every group's codes written as a Rice-coded sub-stream. */
+static int store_td(const shape_t *s, const uint16_t *pool, const int32_t *table, int64_t off, int T, int codec, uint8_t *chunk)
+{
+    int qmax = td_qmax(codec);
+    size_t lay[6];
+    if (kdn_oracle_td_layout(s->L, s->H, s->D, T, codec, lay)) return 3;
+    size_t R = (size_t)s->H * (size_t)s->D;
+    int G = (T + KDN_ORACLE_GROUP - 1) / KDN_ORACLE_GROUP;
+    uint64_t *seg_off = (uint64_t *)chunk;
+    float *scales = (float *)(chunk + lay[1]);
+    uint8_t *lens = chunk + lay[2], *params = chunk + lay[3];
+    size_t cursor = lay[4];                                  /* where the next sub-stream goes */
+    memset(chunk, 0, lay[4]);
+    for (int l = 0; l < s->L; ++l)
+        for (int kv = 0; kv < 2; ++kv)
+            for (int g = 0; g < G; ++g) {
+                size_t seg = ((size_t)l * 2u + (size_t)kv) * (size_t)G + (size_t)g;
+                int t0 = g * KDN_ORACLE_GROUP;
+                int n = T - t0 < KDN_ORACLE_GROUP ? T - t0 : KDN_ORACLE_GROUP;
+                seg_off[seg] = (uint64_t)cursor;
+                for (int h = 0; h < s->H; ++h)
+                    for (int d = 0; d < s->D; ++d) {
+                        uint16_t x[KDN_ORACLE_GROUP];
+                        int8_t q[KDN_ORACLE_GROUP];
+                        uint8_t bytes[72];
+                        int len, param;
+                        for (int i = 0; i < n; ++i) {
+                            int64_t p = off + t0 + i;
+                            x[i] = pool[pool_index(s, l, kv, table[p / s->bs], (int)(p % s->bs), h, d)];
+                        }
+                        size_t ch = (size_t)h * (size_t)s->D + (size_t)d;
+                        kdn_oracle_quant_channel(x, n, qmax, q, scales + seg * R + ch);
+                        kdn_oracle_td_encode_channel(q, n, qmax, bytes, &len, &param);
+                        lens[seg * R + ch] = (uint8_t)len;
+                        params[seg * R + ch] = (uint8_t)param;
+                        memcpy(chunk + cursor, bytes, (size_t)len);
+                        cursor += (size_t)len;
+                    }
+                while (cursor % 16u) chunk[cursor++] = 0;    /* a segment ends on a 16-byte boundary */
+            }
+    seg_off[(size_t)s->L * 2u * (size_t)G] = (uint64_t)cursor;
+    return 0;
+}
+
+/* R9: all codes of a token-delta chunk as plain int8 codes[l][kv][t][head][d] (malloc'ed; NULL when out of memory). */
+static int8_t *td_unpack(const shape_t *s, int T, int codec, const uint8_t *chunk)
+{
+    size_t lay[6];
+    if (kdn_oracle_td_layout(s->L, s->H, s->D, T, codec, lay)) return NULL;
+    size_t R = (size_t)s->H * (size_t)s->D;
+    int G = (T + KDN_ORACLE_GROUP - 1) / KDN_ORACLE_GROUP;
+    const uint64_t *seg_off = (const uint64_t *)chunk;
+    const uint8_t *lens = chunk + lay[2], *params = chunk + lay[3];
+    int8_t *codes = (int8_t *)malloc((size_t)s->L * 2u * (size_t)T * R + 1u);
+    if (!codes) return NULL;
+    for (int l = 0; l < s->L; ++l)
+        for (int kv = 0; kv < 2; ++kv)
+            for (int g = 0; g < G; ++g) {
+                size_t seg = ((size_t)l * 2u + (size_t)kv) * (size_t)G + (size_t)g;
+                int t0 = g * KDN_ORACLE_GROUP;
+                int n = T - t0 < KDN_ORACLE_GROUP ? T - t0 : KDN_ORACLE_GROUP;
+                size_t cursor = (size_t)seg_off[seg];
+                for (size_t ch = 0; ch < R; ++ch) {
+                    int8_t q[KDN_ORACLE_GROUP];
+                    kdn_oracle_td_decode_channel(chunk + cursor, params[seg * R + ch], n, td_qmax(codec), q);
+                    for (int i = 0; i < n; ++i)
+                        codes[(((size_t)l * 2u + (size_t)kv) * (size_t)T + (size_t)(t0 + i)) * R + ch] = q[i];
+                    cursor += lens[seg * R + ch];
+                }
+            }
+    return codes;
+}
+
 /* ---------------------------------------------------------------- store -- */
 
 /* Sec. 3.2 call (i): gather T tokens starting at request position `off` out
@@ -394,6 +619,7 @@ int kdn_oracle_store_sparse(const uint16_t *pool, int L, int H, int D, int bs, i
     size_t elems = (size_t)L * 2u * (size_t)T * (size_t)H * (size_t)D;
     if (codec == KDN_ORACLE_INT8_KC64 || codec == KDN_ORACLE_INT4_KC64)
         return store_kc(&s, pool, table, off, T, codec, chunk);
+    if (td_is(codec)) return store_td(&s, pool, table, off, T, codec, chunk);
     uint16_t *raw = (uint16_t *)chunk;
     int8_t *codes = (int8_t *)chunk;
     float *scales = (float *)(chunk + (codec == KDN_ORACLE_INT4_G64 ? elems / 2u : elems));
@@ -436,8 +662,19 @@ int kdn_oracle_store(const uint16_t *pool, int L, int H, int D, int bs, int64_t 
 
 /* The stored value of chunk element c before any bf16 rounding: code and scale (raw: the bf16 itself). */
 static void stored_code(const uint8_t *chunk, size_t elems, int codec, size_t c, int *q, float *scale,
-                        const shape_t *s, int T)
+                        const shape_t *s, int T, const int8_t *unpacked)
 {
+    if (td_is(codec)) {                                    /* R9: codes from td_unpack, one scale per (segment, channel) */
+        size_t lay[6];
+        kdn_oracle_td_layout(s->L, s->H, s->D, T, codec, lay);
+        size_t hd = (size_t)s->H * (size_t)s->D;
+        size_t ch = c % hd, row = c / hd;                  /* row = (l * 2 + kv) * T + t */
+        size_t t = row % (size_t)T, plane = row / (size_t)T;
+        size_t G = ((size_t)T + KDN_ORACLE_GROUP - 1u) / KDN_ORACLE_GROUP;
+        *q = unpacked[c];
+        *scale = ((const float *)(chunk + lay[1]))[(plane * G + t / KDN_ORACLE_GROUP) * hd + ch];
+        return;
+    }
     if (codec == KDN_ORACLE_INT8_KC64 || codec == KDN_ORACLE_INT4_KC64) {           /* R4" */
         int int4 = codec == KDN_ORACLE_INT4_KC64;
         size_t hd = (size_t)s->H * (size_t)s->D;
@@ -457,12 +694,13 @@ static void stored_code(const uint8_t *chunk, size_t elems, int codec, size_t c,
 }
 
 /* R5: the bf16 a retrieve writes for chunk element c. */
-static uint16_t decoded(const uint8_t *chunk, size_t elems, int codec, size_t c, const shape_t *s, int T)
+static uint16_t decoded(const uint8_t *chunk, size_t elems, int codec, size_t c, const shape_t *s, int T,
+                        const int8_t *unpacked)
 {
     if (codec == KDN_ORACLE_RAW_BF16) return ((const uint16_t *)chunk)[c];
     int q;
     float scale;
-    stored_code(chunk, elems, codec, c, &q, &scale, s, T);
+    stored_code(chunk, elems, codec, c, &q, &scale, s, T, unpacked);
     return kdn_oracle_dequant((int8_t)q, scale);
 }
 
@@ -479,6 +717,11 @@ int kdn_oracle_retrieve_sparse(uint16_t *pool, int L, int H, int D, int bs, int6
     int rc = check_args_list(&s, table, n_table, off, T, codec, keep, -1);
     if (rc) return rc;
     size_t elems = (size_t)L * 2u * (size_t)T * (size_t)H * (size_t)D;
+    int8_t *unpacked = NULL;
+    if (td_is(codec) && T > 0) {
+        unpacked = td_unpack(&s, T, codec, chunk);
+        if (!unpacked) return 6;
+    }
     for (int l = 0; l < L; ++l)
         for (int kv = 0; kv < 2; ++kv)
             for (int t = 0; t < T; ++t) {
@@ -489,9 +732,10 @@ int kdn_oracle_retrieve_sparse(uint16_t *pool, int L, int H, int D, int bs, int6
                     for (int d = 0; d < D; ++d) {
                         size_t c = chunk_index(&s, T, l, kv, t, h, d);
                         size_t o = pool_index(&s, l, kv, block, slot, h, d);
-                        pool[o] = decoded(chunk, elems, codec, c, &s, T);
+                        pool[o] = decoded(chunk, elems, codec, c, &s, T, unpacked);
                     }
             }
+    free(unpacked);
     return 0;
 }
 
@@ -541,6 +785,11 @@ int kdn_oracle_compose_select(uint16_t *pool, int L, int H, int D, int bs, int64
         const uint16_t *raw = (const uint16_t *)chunks[j];
         const int32_t *sel = part_sel ? part_sel[j] : NULL;
         int n_deliver = sel ? part_nsel[j] : T;
+        int8_t *unpacked = NULL;
+        if (td_is(codec) && T > 0) {
+            unpacked = td_unpack(&s, T, codec, chunks[j]);
+            if (!unpacked) return 6;
+        }
         for (int l = 0; l < L; ++l)
             for (int kv = 0; kv < 2; ++kv)
                 for (int i_sel = 0; i_sel < n_deliver; ++i_sel) {
@@ -554,7 +803,7 @@ int kdn_oracle_compose_select(uint16_t *pool, int L, int H, int D, int bs, int64
                             for (int d = 0; d < D; ++d) {
                                 size_t c = chunk_index(&s, T, l, kv, t, h, d);
                                 size_t o = pool_index(&s, l, kv, block, slot, h, d);
-                                pool[o] = decoded(chunks[j], elems, codec, c, &s, T);
+                                pool[o] = decoded(chunks[j], elems, codec, c, &s, T, unpacked);
                                 if (kv == 0 && kref) {
                                     size_t r = (((size_t)l * (size_t)P + (size_t)p) * (size_t)H + (size_t)h) * (size_t)D + (size_t)d;
                                     kref[r] = (double)kdn_oracle_bf16_to_f32(pool[o]);
@@ -573,8 +822,8 @@ int kdn_oracle_compose_select(uint16_t *pool, int L, int H, int D, int bs, int64
                             } else {
                                 int qu, qw;
                                 float su, sw;
-                                stored_code(chunks[j], elems, codec, cu, &qu, &su, &s, T);
-                                stored_code(chunks[j], elems, codec, cw, &qw, &sw, &s, T);
+                                stored_code(chunks[j], elems, codec, cu, &qu, &su, &s, T, unpacked);
+                                stored_code(chunks[j], elems, codec, cw, &qw, &sw, &s, T, unpacked);
                                 u = (double)qu * (double)su;
                                 w = (double)qw * (double)sw;
                             }
@@ -597,6 +846,7 @@ int kdn_oracle_compose_select(uint16_t *pool, int L, int H, int D, int bs, int64
                         }
                     }
                 }
+        free(unpacked);
     }
     return 0;
 }

@@ -44,6 +44,22 @@ MUTANTS = [
      "kdn_oracle_quant_channel(x, 1, qmax, q, scales + kc_scale_index(s, T, l, 0, t0, ch)); for (int i = 1; i < n; ++i) q[i] = q[0];",
      ["test_oracle_kc"]),
     ("checksum_weights", "2u * (uint32_t)i + 1u", "(uint32_t)i + 1u", ["test_oracle_shell"]),
+    # the token-delta Rice codecs
+    ("bits_from_the_low_end", "if (bit) buf[*pos / 8u] |= (uint8_t)(0x80u >> (*pos % 8u));", "if (bit) buf[*pos / 8u] |= (uint8_t)(1u << (*pos % 8u));",
+     ["test_oracle_td"]),
+    ("zigzag_signs_swapped", "return e >= 0 ? 2u * (unsigned)e : 2u * (unsigned)(-e) - 1u;", "return e > 0 ? 2u * (unsigned)e - 1u : 2u * (unsigned)(-e);",
+     ["test_oracle_td"]),
+    ("delta_from_two_tokens_back", "int prev = (mode == 1 && t > 0) ? q[t - 1] : 0;", "int prev = (mode == 1 && t > 1) ? q[t - 2] : 0;", ["test_oracle_td"]),
+    ("escape_one_late", "if (quo < 15u) {\n        for (unsigned i = 0; i < quo; ++i) put_bit(buf, pos, 1u);",
+     "if (quo < 16u) {\n        for (unsigned i = 0; i < quo; ++i) put_bit(buf, pos, 1u);", ["test_oracle_td"]),
+    ("remainder_low_bit_first", "for (int b = k - 1; b >= 0; --b) put_bit(buf, pos, (u >> b) & 1u);", "for (int b = 0; b < k; ++b) put_bit(buf, pos, (u >> b) & 1u);",
+     ["test_oracle_td"]),
+    ("last_minimum_wins", "if (best_bits < 0 || bits < best_bits) {", "if (best_bits < 0 || bits <= best_bits) {", ["test_oracle_td"]),
+    ("segments_not_aligned", "while (cursor % 16u) chunk[cursor++] = 0;", "while (cursor % 4u) chunk[cursor++] = 0;", ["test_oracle_td"]),
+    ("values_keep_head_dim_groups", "x[i] = pool[pool_index(s, l, kv, table[p / s->bs], (int)(p % s->bs), h, d)];\n                        }\n                        size_t ch = (size_t)h * (size_t)s->D + (size_t)d;\n                        kdn_oracle_quant_channel(x, n, qmax, q, scales + seg * R + ch);",
+     "x[i] = pool[pool_index(s, l, 0, table[p / s->bs], (int)(p % s->bs), h, d)];\n                        }\n                        size_t ch = (size_t)h * (size_t)s->D + (size_t)d;\n                        kdn_oracle_quant_channel(x, n, qmax, q, scales + seg * R + ch);",
+     ["test_oracle_td"]),
+    ("decoder_forgets_the_running_code", "int v = mode == 1 ? prev + e : e;", "int v = mode == 1 && t == 1 ? prev + e : e;", ["test_oracle_td"]),
 ]
 
 

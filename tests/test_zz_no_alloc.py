@@ -202,8 +202,9 @@ free1, _ = torch.cuda.mem_get_info()
 st = K.kdn_compose_static(0, desc, [K.ComposeReq(table.data_ptr(), 3, [K.Chunk(chunk.data_ptr(), chunk.numel() * 2, T, 0, 0, 9)], [5], 1e4)], 0, True)
 assert st == K.KDN_OK, st
 free2, _ = torch.cuda.mem_get_info()
-# delta 0 call: a plain scatter, checked here by hand (position p -> table[p // bs], slot p %% bs)
-st = K.kdn_compose_static(0, desc, [K.ComposeReq(table.data_ptr(), 3, [K.Chunk(chunk.data_ptr(), chunk.numel() * 2, T, 0)], [5], 1e4)], 0, True)
+# a part placed where its keys were computed (base_pos = dst_pos = 5): a plain scatter, checked here by hand
+# (position p -> block table[p // bs], slot p %% bs)
+st = K.kdn_compose_static(0, desc, [K.ComposeReq(table.data_ptr(), 3, [K.Chunk(chunk.data_ptr(), chunk.numel() * 2, T, 0, 0, 5)], [5], 1e4)], 0, True)
 assert st == K.KDN_OK, st
 tab = [7, 3, 30]
 for l in range(L):
