@@ -47,6 +47,24 @@
  *   They need block_size to divide 64 and the chunk's first token to sit at the start of a block (token_offset, or
  *   part_dst_pos in kdn_compose, a multiple of block_size), else KDN_E_UNSUPPORTED; token lists and kdn_compose_static
  *   are not supported with them (KDN_E_UNSUPPORTED).
+ * Token-delta Rice codecs (KDN_CODEC_INT8_TD64, KDN_CODEC_INT4_TD64; Sec. 3.2 "KV-cache delivery" cites a scheme that
+ *   quantises a KV cache and then encodes it into binary strings, and reports more than tenfold smaller caches when
+ *   such techniques are combined; the paper prescribes no bitstream, this one is this library's).  Keys AND values
+ *   are grouped along tokens as the keys of the per-channel key codecs are (chunk tokens 64g .. 64g+63 of one
+ *   (layer, K|V, head, channel); codes in [-127, 127] or [-7, 7]).  The n <= 64 codes q_t of a group become one
+ *   sub-stream of n symbols: e_t = q_t (mode 0) or e_t = q_t - q_{t-1} with q_{-1} = 0 (mode 1); u_t = 2 e_t for
+ *   e_t >= 0, else -2 e_t - 1; Rice code with parameter k in 0..7: quo = u >> k; quo < 15: quo one-bits, a zero-bit, the
+ *   k low bits of u from the highest down; else 15 one-bits and u in 9 (int8) or 5 (int4) bits.  Bits fill bytes from
+ *   the most significant bit down; a sub-stream ends on a byte boundary (zero padded).  The store picks, per
+ *   sub-stream, the (mode, k) with the fewest bits, the first such in the order (0,0) .. (0,7), (1,0) .. (1,7).
+ *   Chunk of T tokens: S = 2 L ceil(T/64) segments, segment (l, kv, g) has index (2l + kv) ceil(T/64) + g and
+ *   R = H*D channels:  uint64 seg_off[S+1] (padded to 16 bytes) | fp32 scales[S][R] | uint8 lens[S][R] (bytes of each
+ *   sub-stream) | uint8 params[S][R] (mode*8 + k) | segment streams.  Segment s starts at byte seg_off[s] (a multiple of
+ *   16), holds its R sub-streams back to back in channel order and is zero padded to 16 bytes; seg_off[S] = the bytes
+ *   the chunk uses, which is what has to be kept or sent.  kdn_chunk_bytes gives the worst-case CAPACITY (a sub-stream
+ *   never exceeds 72 or 40 bytes) and chunk.bytes must equal it; bytes past seg_off[S] are not written and not read
+ *   (up to 15 beyond it may be read, never past the capacity).  kdn_td_layout gives the offsets.
+ *   Same restrictions as the per-channel key codecs, and KDN_MEM_DEVICE chunks only (KDN_E_UNSUPPORTED otherwise).
  * Key re-rotation in kdn_compose: the stored keys of a part carry rotary
  *   position embedding for positions base_pos + t; placing the part at
  *   dst_pos rotates each pair (k[i], k[i + D/2]) of every head by
@@ -105,7 +123,8 @@ typedef enum {
 } kdn_status;
 
 typedef enum { KDN_CODEC_RAW_BF16 = 0, KDN_CODEC_INT8_G64 = 1, KDN_CODEC_INT4_G64 = 2,
-               KDN_CODEC_INT8_KC64 = 3, KDN_CODEC_INT4_KC64 = 4 } kdn_codec;
+               KDN_CODEC_INT8_KC64 = 3, KDN_CODEC_INT4_KC64 = 4,
+               KDN_CODEC_INT8_TD64 = 5, KDN_CODEC_INT4_TD64 = 6 } kdn_codec;
 typedef enum { KDN_MEM_DEVICE = 0, KDN_MEM_PINNED_HOST = 1 } kdn_mem;
 
 /* An engine's paged KV pool (Sec. 3.2 names vLLM's paged memory).  k_layers and v_layers are HOST
@@ -209,6 +228,15 @@ kdn_status kdn_pool_register(kdn_ctx *ctx, const kdn_pool_desc *pool, int *pool_
 /* Bytes of one chunk of n_tokens tokens for this pool's shape; 0 if the codec cannot hold the
  * shape.  Pure host arithmetic; reads only the shape fields of *pool. */
 size_t kdn_chunk_bytes(const kdn_pool_desc *pool, int32_t n_tokens, int32_t codec);
+
+/* Byte offsets of the regions of a token-delta Rice chunk of n_tokens tokens (see the top of this file): the
+ * number of segments S, where scales, lens, params and the first segment's streams begin, and the capacity
+ * (= kdn_chunk_bytes).  After a store, the uint64 at byte 8*S of the chunk is the number of bytes in use.
+ * Pure host arithmetic.  KDN_E_UNSUPPORTED for other codecs or head_dim % 64 != 0. */
+typedef struct {
+    uint64_t segments, scales_offset, lens_offset, params_offset, streams_offset, capacity;
+} kdn_td_layout_info;
+kdn_status kdn_td_layout(const kdn_pool_desc *pool, int32_t n_tokens, int32_t codec, kdn_td_layout_info *out);
 
 /* Host-side argument check shared by kdn_store / kdn_retrieve (same status they would return);
  * touches no device.  Pointers are only compared and tested for alignment, never dereferenced,

@@ -11,7 +11,7 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libkdn.so")
 SOURCES = [os.path.join(CSRC, "kdn.cu"), os.path.join(CSRC, "kdn_shell.cu")]
-DEPS = SOURCES + [os.path.join(CSRC, "kdn_kernels.cuh"), os.path.join(ROOT, "include", "kdn.h")]
+DEPS = SOURCES + [os.path.join(CSRC, "kdn_kernels.cuh"), os.path.join(CSRC, "kdn_td.cuh"), os.path.join(ROOT, "include", "kdn.h")]
 
 
 def nvcc_path() -> str:

@@ -4,6 +4,7 @@
 // delivery and blending modules).
 #include "kdn.h"
 #include "kdn_kernels.cuh"
+#include "kdn_td.cuh"
 
 #include <cerrno>
 #include <cstdio>
@@ -146,6 +147,7 @@ kdn_status check_shape(const kdn_pool_desc *p)
 
 bool is_kc(int codec) { return codec == KDN_CODEC_INT8_KC64 || codec == KDN_CODEC_INT4_KC64; }
 bool is_int4(int codec) { return codec == KDN_CODEC_INT4_G64 || codec == KDN_CODEC_INT4_KC64; }
+bool is_td(int codec) { return codec == KDN_CODEC_INT8_TD64 || codec == KDN_CODEC_INT4_TD64; }
 
 // fp32 scales one layer of a chunk holds (0 for raw bf16).
 size_t scales_per_layer(size_t row, size_t T, int codec)
@@ -158,7 +160,7 @@ size_t scales_per_layer(size_t row, size_t T, int codec)
 // The per-channel key codecs group 64 consecutive chunk tokens; a pool block must lie inside one group.
 kdn_status check_kc(const kdn_pool_desc *p, const kdn_chunk *c, int64_t pos)
 {
-    if (!is_kc(c->codec) || c->n_tokens == 0) return KDN_OK;
+    if ((!is_kc(c->codec) && !is_td(c->codec)) || c->n_tokens == 0) return KDN_OK;
     if (64 % p->block_size || pos % p->block_size) return KDN_E_UNSUPPORTED;
     return KDN_OK;
 }
@@ -166,10 +168,11 @@ kdn_status check_kc(const kdn_pool_desc *p, const kdn_chunk *c, int64_t pos)
 kdn_status check_chunk(const kdn_pool_desc *p, const kdn_chunk *c)
 {
     if (c->n_tokens < 0) return KDN_E_INVAL;
-    if (c->codec < KDN_CODEC_RAW_BF16 || c->codec > KDN_CODEC_INT4_KC64) return KDN_E_INVAL;
+    if (c->codec < KDN_CODEC_RAW_BF16 || c->codec > KDN_CODEC_INT4_TD64) return KDN_E_INVAL;
     if (c->mem != KDN_MEM_DEVICE && c->mem != KDN_MEM_PINNED_HOST) return KDN_E_INVAL;
     if (c->codec != KDN_CODEC_RAW_BF16 && p->head_dim % 64) return KDN_E_UNSUPPORTED;
     if (c->bytes != kdn_chunk_bytes(p, c->n_tokens, c->codec)) return KDN_E_SHAPE;
+    if (is_td(c->codec) && c->mem != KDN_MEM_DEVICE) return KDN_E_UNSUPPORTED;   // variable-length chunks are not staged
     if (c->n_tokens > 0) {
         if (!c->data) return KDN_E_INVAL;
         if ((uintptr_t)c->data % 16) return KDN_E_ALIGN;
@@ -355,6 +358,20 @@ kdn_status launch_tiles(LaunchEnv &env, int OP, int groups, int gw, unsigned gri
     return KDN_E_UNSUPPORTED;
 }
 
+// The rotation table of a launch lives in a ring slot; make it large enough.
+kdn_status ensure_table(RingSlot *slot, int n_rope, int half)
+{
+    if (slot->table_rows_cap >= (size_t)n_rope && slot->table_half == half) return KDN_OK;
+    KDN_CUDA(cudaEventSynchronize(slot->done));
+    if (slot->d_table) KDN_CUDA(cudaFree(slot->d_table));
+    slot->d_table = nullptr;
+    const size_t rows = (size_t)n_rope < 64 ? 64 : (size_t)n_rope;
+    KDN_CUDA(cudaMalloc((void **)&slot->d_table, rows * (size_t)half * sizeof(float2)));
+    slot->table_rows_cap = rows;
+    slot->table_half = half;
+    return KDN_OK;
+}
+
 // Tile one batch of host ops (at most kMaxOpsPerLaunch, all on the device side) and launch it.
 kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *hops, int n, cudaStream_t stream)
 {
@@ -453,14 +470,9 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     if (!inl) KDN_CUDA(cudaMemcpyAsync(slot->d_ops, slot->h_ops, sizeof(DevOp) * (size_t)n, cudaMemcpyHostToDevice, stream));
     const int half = pool.D / 2;
     if (n_rope) {
-        if (slot->table_rows_cap < (size_t)n_rope || slot->table_half != half) {
-            KDN_CUDA(cudaEventSynchronize(slot->done));
-            if (slot->d_table) KDN_CUDA(cudaFree(slot->d_table));
-            slot->d_table = nullptr;
-            size_t rows = (size_t)n_rope < 64 ? 64 : (size_t)n_rope;
-            KDN_CUDA(cudaMalloc((void **)&slot->d_table, rows * (size_t)half * sizeof(float2)));
-            slot->table_rows_cap = rows;
-            slot->table_half = half;
+        {
+            kdn_status r = ensure_table(slot, n_rope, half);
+            if (r != KDN_OK) return r;
         }
         if (!inl) KDN_CUDA(cudaMemcpyAsync(slot->d_rope, slot->h_rope, sizeof(RopeParam) * (size_t)n_rope, cudaMemcpyHostToDevice, stream));
         const long long total = (long long)n_rope * half;
@@ -547,9 +559,120 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     return KDN_OK;
 }
 
+// Ops whose chunk is in a token-delta Rice codec: at most kInlineOps per launch, their records travel as kernel
+// parameters.  Store is three launches (plan, scan, encode), retrieve and compose one (plus the rotation table).
+kdn_status launch_td(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *hops, int n, cudaStream_t stream)
+{
+    const unsigned row_elems = (unsigned)pool.H * (unsigned)pool.D;
+    // channels per CTA: a multiple of 16 that divides the row, whole heads when keys are re-rotated, 256 if possible
+    bool any_rot = false;
+    for (int i = 0; i < n; ++i) any_rot |= hops[i].rotate;
+    const unsigned unit = any_rot ? lcm_u(16u, (unsigned)pool.D) : 16u;
+    unsigned n_split = 1;
+    while (row_elems / n_split > 256u && row_elems % (n_split * 2u) == 0u && (row_elems / (n_split * 2u)) % unit == 0u) n_split *= 2u;
+    const unsigned cols = row_elems / n_split;
+    if (cols % 16u || cols > 1024u) return KDN_E_UNSUPPORTED;
+    unsigned threads = (cols + 31u) & ~31u;                  // one thread per channel in the coding loops
+    if (threads < 64u) threads = 64u;
+    if (threads > 512u) return KDN_E_UNSUPPORTED;
+    const size_t smem_limit = (size_t)ctx->env.smem_optin;
+
+    for (int first = 0; first < n; first += kInlineOps) {
+        const int m = n - first < kInlineOps ? n - first : kInlineOps;
+        TdLaunch tp{};
+        RopeInline rope_inl{};
+        int n_rope = 0, max_groups = 0, max_layers = 0;
+        for (int i = 0; i < m; ++i) {
+            DevOp op = hops[first + i].op;
+            op.rope = -1;
+            if (hops[first + i].rotate) {
+                rope_inl.p[n_rope] = hops[first + i].rp;
+                op.rope = n_rope++;
+            }
+            tp.inline_ops[i] = op;
+            const int g = (op.T + 63) / 64;
+            if (g > max_groups) max_groups = g;
+            if (op.nl > max_layers) max_layers = op.nl;
+        }
+        if (max_groups == 0 || max_layers == 0) continue;
+        tp.ops = nullptr;
+        tp.n_ops = m;
+        tp.k_layers = pool.d_k;
+        tp.v_layers = pool.d_v;
+        tp.n_blocks = pool.nb;
+        tp.bs = pool.bs;
+        tp.D = pool.D;
+        tp.L = pool.L;
+        tp.row_elems = row_elems;
+        tp.cols = cols;
+        tp.n_split = n_split;
+        tp.status = ctx->d_status;
+        const dim3 grid((unsigned)max_groups * n_split, (unsigned)max_layers * 2u, (unsigned)m);
+        int per_sm = 0;
+        if (OP == OP_STORE) {
+            const size_t smem_plan = td_store_smem_bytes(cols, false), smem_enc = td_store_smem_bytes(cols, true);
+            if (smem_enc > smem_limit) return KDN_E_UNSUPPORTED;
+            kdn_status r = ctx->env.resident(kdn_td_plan_kernel, (int)threads, smem_plan, &per_sm);
+            if (r == KDN_OK && per_sm >= 1) r = ctx->env.resident(kdn_td_encode_kernel, (int)threads, smem_enc, &per_sm);
+            if (r != KDN_OK) return r;
+            if (per_sm < 1) return KDN_E_UNSUPPORTED;
+            kdn_td_plan_kernel<<<grid, threads, smem_plan, stream>>>(tp);
+            KDN_CUDA(cudaGetLastError());
+            kdn_td_scan_kernel<<<(unsigned)m, 256, 0, stream>>>(tp);
+            KDN_CUDA(cudaGetLastError());
+            kdn_td_encode_kernel<<<grid, threads, smem_enc, stream>>>(tp);
+            KDN_CUDA(cudaGetLastError());
+            ctx->launches += 3;
+        } else {
+            const size_t smem = td_decode_smem_bytes(cols);
+            if (smem > smem_limit) return KDN_E_UNSUPPORTED;
+            RingSlot *slot = nullptr;
+            if (n_rope) {
+                slot = &ctx->ring[ctx->ring_next++ % kRing];
+                if (slot->used) KDN_CUDA(cudaEventSynchronize(slot->done));
+                kdn_status r = ensure_table(slot, n_rope, pool.D / 2);
+                if (r != KDN_OK) return r;
+                const long long total = (long long)n_rope * (pool.D / 2);
+                kdn_rope_table_kernel<<<(unsigned)((total + 127) / 128), 128, 0, stream>>>(nullptr, rope_inl, n_rope, pool.D, slot->d_table);
+                KDN_CUDA(cudaGetLastError());
+                ctx->launches++;
+                tp.rope = slot->d_table;
+            }
+            kdn_status r = OP == OP_COMPOSE ? ctx->env.resident(kdn_td_decode_kernel<true>, (int)threads, smem, &per_sm)
+                                            : ctx->env.resident(kdn_td_decode_kernel<false>, (int)threads, smem, &per_sm);
+            if (r != KDN_OK) return r;
+            if (per_sm < 1) return KDN_E_UNSUPPORTED;
+            if (OP == OP_COMPOSE) kdn_td_decode_kernel<true><<<grid, threads, smem, stream>>>(tp);
+            else kdn_td_decode_kernel<false><<<grid, threads, smem, stream>>>(tp);
+            KDN_CUDA(cudaGetLastError());
+            ctx->launches++;
+            if (slot) {
+                KDN_CUDA(cudaEventRecord(slot->done, stream));
+                slot->used = true;
+            }
+        }
+    }
+    return KDN_OK;
+}
+
 kdn_status launch_all(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<HostOp> &hops, cudaStream_t stream,
                       size_t max_ops = kMaxOpsPerLaunch)
 {
+    bool any_td = false;
+    for (const HostOp &h : hops) any_td |= is_td(h.op.codec);
+    if (any_td) {
+        // token-delta chunks go through their own kernels; everything else through the tile pipeline
+        std::vector<HostOp> td, rest;
+        for (const HostOp &h : hops) (is_td(h.op.codec) ? td : rest).push_back(h);
+        kdn_status st = launch_td(ctx, pool, OP, td.data(), (int)td.size(), stream);
+        if (st != KDN_OK) return st;
+        for (size_t i = 0; i < rest.size(); i += max_ops) {
+            size_t n = rest.size() - i < max_ops ? rest.size() - i : max_ops;
+            st = launch_batch(ctx, pool, OP, rest.data() + i, (int)n, stream);
+            if (st != KDN_OK) return st;
+        }
+        return KDN_OK;
+    }
     for (size_t i = 0; i < hops.size(); i += max_ops) {
         size_t n = hops.size() - i < max_ops ? hops.size() - i : max_ops;
         kdn_status st = launch_batch(ctx, pool, OP, hops.data() + i, (int)n, stream);
@@ -575,7 +698,7 @@ HostOp make_host_op(const Pool &pool, const int32_t *table, int32_t n_table, int
     h.op.nl = pool.L;
     h.op.pos_end = (long long)n_table * pool.bs;
     const size_t elems = (size_t)pool.L * 2u * (size_t)c.n_tokens * (size_t)pool.H * (size_t)pool.D;
-    if (c.codec != KDN_CODEC_RAW_BF16) h.op.scales = (unsigned char *)c.data + (is_int4(c.codec) ? elems / 2u : elems);
+    if (c.codec != KDN_CODEC_RAW_BF16 && !is_td(c.codec)) h.op.scales = (unsigned char *)c.data + (is_int4(c.codec) ? elems / 2u : elems);
     return h;
 }
 
@@ -781,6 +904,7 @@ HostOp layer_range(const Pool &pool, const HostOp &h, int l0, int nl)
     const size_t plane = 2u * (size_t)h.op.T * (size_t)pool.H * (size_t)pool.D;     // elements of one layer
     sub.op.l0 = l0;
     sub.op.nl = nl;
+    if (is_td(h.op.codec)) return sub;                      // segments are found through the chunk's own offset table
     if (h.op.codec != KDN_CODEC_RAW_BF16) {
         sub.op.data = h.op.data + (size_t)l0 * (is_int4(h.op.codec) ? plane / 2u : plane);
         sub.op.scales = h.op.scales + (size_t)l0 * scales_per_layer((size_t)pool.H * (size_t)pool.D, (size_t)h.op.T, h.op.codec) * 4u;
@@ -827,7 +951,7 @@ kdn_status xfer_sparse(kdn_ctx *ctx, int pool_id, int OP, const kdn_sparse_op *o
         const kdn_xfer_op &o = ops[i].op;
         st = check_chunk(&shape, &o.chunk);
         if (st != KDN_OK) return st;
-        if (is_kc(o.chunk.codec)) return KDN_E_UNSUPPORTED;      // a keep-list breaks up the 64-token key groups
+        if (is_kc(o.chunk.codec) || is_td(o.chunk.codec)) return KDN_E_UNSUPPORTED;   // a keep-list breaks up the 64-token groups
         if (o.n_table_blocks < 0 || o.token_offset < 0) return KDN_E_INVAL;
         if (o.chunk.n_tokens > 0 && (!o.block_table || !ops[i].keep)) return KDN_E_INVAL;
         // the listed tokens are distinct positions below the end of the table, so there cannot be more of them
@@ -858,6 +982,10 @@ size_t kdn_chunk_bytes(const kdn_pool_desc *pool, int32_t n_tokens, int32_t code
     if (codec == KDN_CODEC_RAW_BF16) return elems * 2u;
     if (codec == KDN_CODEC_INT8_G64) return pool->head_dim % 64 ? 0 : elems + elems / 64u * 4u;
     if (codec == KDN_CODEC_INT4_G64) return pool->head_dim % 64 ? 0 : elems / 2u + elems / 64u * 4u;
+    if (is_td(codec)) {
+        if (pool->head_dim % 64) return 0;
+        return (size_t)td_layout(pool->n_layers, (unsigned)(pool->n_kv_heads * pool->head_dim), n_tokens, codec).capacity;
+    }
     if (is_kc(codec)) {
         if (pool->head_dim % 64) return 0;
         const size_t row = (size_t)pool->n_kv_heads * (size_t)pool->head_dim;
@@ -865,6 +993,16 @@ size_t kdn_chunk_bytes(const kdn_pool_desc *pool, int32_t n_tokens, int32_t code
                4u * (size_t)pool->n_layers * scales_per_layer(row, (size_t)n_tokens, codec);
     }
     return 0;
+}
+
+kdn_status kdn_td_layout(const kdn_pool_desc *pool, int32_t n_tokens, int32_t codec, kdn_td_layout_info *out)
+{
+    if (!shape_ok(pool) || n_tokens < 0 || !out) return KDN_E_INVAL;
+    if (!is_td(codec) || pool->head_dim % 64) return KDN_E_UNSUPPORTED;
+    const TdLayout t = td_layout(pool->n_layers, (unsigned)(pool->n_kv_heads * pool->head_dim), n_tokens, codec);
+    out->segments = t.S; out->scales_offset = t.scales; out->lens_offset = t.lens; out->params_offset = t.params;
+    out->streams_offset = t.streams; out->capacity = t.capacity;
+    return KDN_OK;
 }
 
 kdn_status kdn_validate_xfer(const kdn_pool_desc *pool, const kdn_xfer_op *ops, int n_ops)
@@ -1146,7 +1284,7 @@ static kdn_status compose_impl(kdn_ctx *ctx, int pool_id, const kdn_compose_req 
             if (selects && selects[r].part_select && selects[r].part_select[j]) {
                 if (!selects[r].part_n_select || selects[r].part_n_select[j] < 0 || selects[r].part_n_select[j] > c.n_tokens)
                     return KDN_E_INVAL;
-                if (is_kc(c.codec)) return KDN_E_UNSUPPORTED;           // select-lists are not defined for these codecs
+                if (is_kc(c.codec) || is_td(c.codec)) return KDN_E_UNSUPPORTED;   // select-lists are not defined for these codecs
                 if (selects[r].part_n_select[j] == 0) continue;          // nothing of this part is delivered
                 h.op.list = selects[r].part_select[j];
                 h.op.n_list = selects[r].part_n_select[j];
@@ -1319,7 +1457,7 @@ extern "C" kdn_status kdn_compose_static(int device, const kdn_pool_desc *pool, 
         for (int j = 0; j < reqs[r].n_parts; ++j) {
             if (reqs[r].parts[j].n_tokens == 0) continue;
             if (reqs[r].parts[j].mem != KDN_MEM_DEVICE) return KDN_E_UNSUPPORTED;
-            if (is_kc(reqs[r].parts[j].codec)) return KDN_E_UNSUPPORTED;
+            if (is_kc(reqs[r].parts[j].codec) || is_td(reqs[r].parts[j].codec)) return KDN_E_UNSUPPORTED;
             ++n_parts;
         }
         if (n_parts > KDN_STATIC_MAX_PARTS) return KDN_E_UNSUPPORTED;

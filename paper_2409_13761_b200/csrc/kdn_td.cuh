@@ -336,6 +336,7 @@ __global__ void __launch_bounds__(256) kdn_td_scan_kernel(const __grid_constant_
         unsigned long long run = lay.streams;
         for (int i = 0; i < 256; ++i) { const unsigned long long v = part[i]; part[i] = run; run += v; }
         seg_off[0] = lay.streams;
+        if ((lay.S + 1ull) & 1ull) seg_off[lay.S + 1ull] = 0ull;             // the table is padded to 16 bytes with zeros
     }
     __syncthreads();
     unsigned long long run = part[tid];

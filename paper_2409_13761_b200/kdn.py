@@ -16,10 +16,11 @@ from . import build as _build
 KDN_OK, KDN_E_INVAL, KDN_E_SHAPE, KDN_E_ALIGN, KDN_E_RANGE, KDN_E_UNSUPPORTED, KDN_E_CUDA, KDN_E_NOMEM, \
     KDN_E_TIMEOUT, KDN_E_NOTFOUND, KDN_E_CHECKSUM, KDN_E_IO = range(12)
 KDN_CODEC_RAW_BF16, KDN_CODEC_INT8_G64, KDN_CODEC_INT4_G64, KDN_CODEC_INT8_KC64, KDN_CODEC_INT4_KC64 = 0, 1, 2, 3, 4
+KDN_CODEC_INT8_TD64, KDN_CODEC_INT4_TD64 = 5, 6
 KDN_MEM_DEVICE, KDN_MEM_PINNED_HOST = 0, 1
 
 EXPORTS = ["kdn_create", "kdn_destroy", "kdn_pool_register", "kdn_chunk_bytes", "kdn_validate_xfer",
-           "kdn_validate_compose", "kdn_store", "kdn_retrieve", "kdn_compose", "kdn_status_sync",
+           "kdn_validate_compose", "kdn_td_layout", "kdn_store", "kdn_retrieve", "kdn_compose", "kdn_status_sync",
            "kdn_set_tuning", "kdn_set_staging_bytes", "kdn_set_wait_limit_ns", "kdn_launch_count", "kdn_last_launch", "kdn_strerror",
            "kdn_compose_static", "kdn_retrieve_layerwise", "kdn_store_file", "kdn_retrieve_file",
            "kdn_store_sparse", "kdn_retrieve_sparse", "kdn_compose_select",
@@ -73,6 +74,10 @@ class kdn_index_info(C.Structure):
                 ("hits", C.c_uint64), ("misses", C.c_uint64), ("evictions", C.c_uint64)]
 
 
+class kdn_td_layout_info(C.Structure):
+    _fields_ = [(n, C.c_uint64) for n in ("segments", "scales_offset", "lens_offset", "params_offset", "streams_offset", "capacity")]
+
+
 class kdn_launch_info(C.Structure):
     _fields_ = [("op", C.c_int32), ("compute_groups", C.c_int32), ("group_warps", C.c_int32), ("tile_bytes", C.c_int32),
                 ("stages", C.c_int32), ("ctas_per_sm", C.c_int32), ("store_lag", C.c_int32), ("grid", C.c_int32),
@@ -102,6 +107,8 @@ def _load() -> C.CDLL:
     lib.kdn_pool_register.argtypes = [vp, C.POINTER(kdn_pool_desc), C.POINTER(i32)]
     lib.kdn_chunk_bytes.restype = C.c_size_t
     lib.kdn_chunk_bytes.argtypes = [C.POINTER(kdn_pool_desc), C.c_int32, C.c_int32]
+    lib.kdn_td_layout.restype = i32
+    lib.kdn_td_layout.argtypes = [C.POINTER(kdn_pool_desc), C.c_int32, C.c_int32, C.POINTER(kdn_td_layout_info)]
     lib.kdn_validate_xfer.restype = i32
     lib.kdn_validate_xfer.argtypes = [C.POINTER(kdn_pool_desc), C.POINTER(kdn_xfer_op), i32]
     lib.kdn_validate_compose.restype = i32
@@ -268,6 +275,13 @@ def kdn_pool_register(ctx, desc: kdn_pool_desc) -> int:
 
 def kdn_chunk_bytes(desc: kdn_pool_desc, n_tokens: int, codec: int) -> int:
     return int(lib.kdn_chunk_bytes(C.byref(desc), int(n_tokens), int(codec)))
+
+
+def kdn_td_layout(desc: kdn_pool_desc, n_tokens: int, codec: int) -> dict:
+    """Region offsets of a token-delta Rice chunk: segments, scales_offset, lens_offset, params_offset, streams_offset, capacity."""
+    info = kdn_td_layout_info()
+    _check(lib.kdn_td_layout(C.byref(desc), int(n_tokens), int(codec), C.byref(info)), "kdn_td_layout")
+    return {name: int(getattr(info, name)) for name, _ in kdn_td_layout_info._fields_}
 
 
 def kdn_validate_xfer(desc: kdn_pool_desc, ops: Sequence[XferOp]) -> int:

@@ -167,3 +167,36 @@ def compact_table(table: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:
     """(unique physical blocks, table rewritten to index into them) for streaming a pool subset."""
     uniq, inv = np.unique(table, return_inverse=True)
     return uniq.astype(np.int64), inv.astype(np.int32)
+
+
+def correlated_tokens(shape: KVShape, n_tokens: int, rho: float, seed: int, device="cpu", outliers: bool = True) -> torch.Tensor:
+    """bf16 [L][2][n_tokens][H][D]: every channel a stationary first-order autoregressive sequence along tokens,
+    x_t = rho x_{t-1} + sqrt(1 - rho^2) eps_t with eps ~ N(0, 1) (so x_t ~ N(0, 1) and neighbouring tokens correlate
+    with coefficient rho; rho = 0 is the uncorrelated input of make_pool), times the channel gain of outlier_gain."""
+    dev = torch.device(device)
+    g = torch.Generator(device=dev).manual_seed(seed)
+    L, H, D = shape.n_layers, shape.n_kv_heads, shape.head_dim
+    eps = torch.randn((n_tokens, L * 2 * H * D), generator=g, device=dev, dtype=torch.float32)
+    if rho != 0.0:
+        # x = M eps with M[t][s] = rho^(t-s) sqrt(1 - rho^2) for 0 < s <= t and M[t][0] = rho^t
+        t = torch.arange(n_tokens, device=dev, dtype=torch.float64)
+        m = torch.tril(torch.pow(torch.tensor(float(rho), dtype=torch.float64, device=dev), (t[:, None] - t[None, :]).clamp(min=0)))
+        m[:, 1:] *= float(np.sqrt(1.0 - rho * rho))
+        eps = m.to(torch.float32) @ eps
+    x = eps.reshape(n_tokens, L, 2, H, D).permute(1, 2, 0, 3, 4)
+    if outliers:
+        x = x * outlier_gain(shape).to(dev)[:, :, None]
+    return x.to(torch.bfloat16).contiguous()
+
+
+def place_tokens(k_layers: Sequence[torch.Tensor], v_layers: Sequence[torch.Tensor], table: np.ndarray, token_offset: int,
+                 x: torch.Tensor) -> None:
+    """Write x [L][2][T][H][D] into the pool at request positions token_offset + t of the request whose block table is
+    ``table`` (input generation only: this is where a serving engine's prefill would have put the tokens)."""
+    bs = k_layers[0].shape[1]
+    pos = token_offset + np.arange(x.shape[2])
+    blocks = torch.as_tensor(np.asarray(table, dtype=np.int64)[pos // bs], device=k_layers[0].device)
+    slots = torch.as_tensor(pos % bs, device=k_layers[0].device)
+    for l in range(len(k_layers)):
+        k_layers[l][blocks, slots] = x[l, 0].to(k_layers[l].device)
+        v_layers[l][blocks, slots] = x[l, 1].to(v_layers[l].device)

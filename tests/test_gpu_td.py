@@ -1,0 +1,205 @@
+"""GPU parity of the token-delta Rice codecs (codecs 5 and 6) against the CPU oracle, through the C ABI.
+
+store: the bytes a chunk uses are bit-identical to the oracle's chunk, and nothing past them is written;
+retrieve: the pool is bit-identical to the oracle's; compose: values and unrotated keys bit-identical, re-rotated
+keys within the rotation tolerance.  Inputs are uncorrelated and token-correlated (so that both coding modes occur),
+with zero, constant, extreme and saw-tooth channels planted (flushed scales, the shortest and the longest
+sub-streams, the escape code)."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from paper_2409_13761_b200 import synth
+from harness import Device, to_np, check_rotated_keys
+
+pytestmark = pytest.mark.gpu
+RAW, INT8 = oracle.RAW_BF16, oracle.INT8_G64
+TD8, TD4 = oracle.INT8_TD64, oracle.INT4_TD64
+
+SHAPES = [
+    synth.TOY,                                                                                  # rows of 128: one slice
+    synth.TOY.with_(n_layers=2, n_kv_heads=8, head_dim=128, block_size=16, n_blocks=96),        # rows of 1024: four slices
+    synth.TOY.with_(n_layers=1, n_kv_heads=3, head_dim=192, block_size=32, n_blocks=40),        # rows of 576: slices of 144
+    synth.TOY.with_(n_layers=3, n_kv_heads=1, head_dim=64, block_size=4, n_blocks=128),         # rows of 64, tiny blocks
+]
+IDS = ["H%dD%dbs%d" % (s.n_kv_heads, s.head_dim, s.block_size) for s in SHAPES]
+
+
+def bf16_bits(x):
+    return (np.asarray(x, dtype=np.float32).view(np.uint32) >> 16).astype(np.uint16)
+
+
+def make_pool_np(shape, table, off, T, rho, seed):
+    """A pool whose request positions off .. off+T-1 (through `table`) hold token-correlated values with planted
+    special channels; the rest is the ordinary uncorrelated fill."""
+    k, v = synth.make_pool(shape, "cpu", seed=seed)
+    x = synth.correlated_tokens(shape, T, rho, seed + 1)
+    xb = x.view(torch.int16).numpy().view(np.uint16).copy()                 # [L][2][T][H][D]
+    big = bf16_bits([3.0])[0]
+    xb[0, 0, :, 0, 0] = 0                                                    # an all-zero channel: scale 0
+    xb[0, 1, :, 0, 1] = bf16_bits([1e-40])[0]                                # a subnormal channel: flushed
+    xb[0, 0, :, 0, 2] = big                                                  # constant: delta mode, one bit a token
+    xb[0, 1, :, 0, 3] = np.where(np.arange(T) % 2 == 0, big, big | 0x8000)   # +max, -max: the longest sub-streams
+    xb[0, 0, :, 0, 4] = np.where(np.arange(T) % 64 == 0, big, 0)             # one spike per group
+    xb[0, 0, 1::3, 0, 5] = 0x8000                                            # negative zeros among ordinary values
+    synth.place_tokens(k, v, table, off, torch.from_numpy(xb.view(np.int16)).view(torch.bfloat16))
+    return synth.pool_to_numpy(k, v)
+
+
+def used_bytes(K, desc, buf, T, codec):
+    lay = K.kdn_td_layout(desc, T, codec)
+    head = to_np(buf[:8 * (lay["segments"] + 1)]).view(np.uint64)
+    return int(head[lay["segments"]]), lay
+
+
+@pytest.mark.parametrize("shape", SHAPES, ids=IDS)
+@pytest.mark.parametrize("codec", [TD8, TD4], ids=["int8td", "int4td"])
+@pytest.mark.parametrize("rho", [0.0, 0.97])
+def test_store_retrieve_compose_against_the_oracle(shape, codec, rho):
+    bs = shape.block_size
+    rng = np.random.default_rng(17)
+    perm = rng.permutation(shape.n_blocks).astype(np.int32)
+    cases = [(150, 0), (64, bs), (37, 2 * bs)]                              # ragged last group, one full group, a short one
+    nb_src = max(-(-(off + T) // bs) for T, off in cases)
+    src = perm[:nb_src]
+    pool = make_pool_np(shape, src, 0, nb_src * bs, rho, seed=31)
+    dev = Device(shape, pool_np=pool)
+    try:
+        K = dev.K
+        for T, off in cases:
+            want = oracle.store(pool, src, off, T, codec)
+            buf = dev.chunk_buf(T, codec)
+            dev.store([dev.op(dev.table(src), off, buf, T, codec)])
+            assert dev.sync() == 0
+            used, lay = used_bytes(K, dev.desc, buf, T, codec)
+            assert lay["capacity"] == buf.numel() == want.size
+            assert used == oracle.td_used_bytes(want, shape.n_layers, shape.n_kv_heads, shape.head_dim, T, codec)
+            got = to_np(buf)
+            assert np.array_equal(got[:used], want[:used])
+            assert np.all(got[used:] == 0xA5)                                # nothing past the bytes in use is written
+            # retrieve into other blocks
+            nb = -(-(off + T) // bs)
+            dst = perm[nb_src:nb_src + nb]
+            before = dev.pool_np()
+            dev.retrieve([dev.op(dev.table(dst), off, buf, T, codec)])
+            assert dev.sync() == 0
+            ref = before.copy()
+            oracle.retrieve(ref, dst, off, T, codec, want)
+            assert np.array_equal(dev.pool_np(), ref)
+            # compose at another block-aligned position, keys re-rotated (chunks of different base positions)
+            if shape.head_dim % 16 == 0 and (shape.n_kv_heads * shape.head_dim <= 512 or 256 % shape.head_dim == 0):
+                rt = perm[nb_src + nb:nb_src + nb + nb + 2]
+                dpos = 2 * bs
+                before = dev.pool_np()
+                dev.compose([K.ComposeReq(dev.table(rt).data_ptr(), len(rt), [dev.chunk(buf, T, codec, 7)], [dpos], shape.rope_theta)])
+                assert dev.sync() == 0
+                ref = before.copy()
+                kref, kmag = oracle.compose(ref, rt, [(want, T, codec, 7, dpos)], shape.rope_theta, want_ref=True)
+                got_pool = dev.pool_np()
+                p = dpos + np.arange(T)
+                rot = np.zeros(got_pool.shape, dtype=bool)
+                rot[:, 0, rt[p // bs], p % bs] = True
+                assert np.array_equal(got_pool[~rot], ref[~rot])
+                check_rotated_keys(got_pool[:, 0, rt[p // bs], p % bs], kref[:, dpos:dpos + T], kmag[:, dpos:dpos + T],
+                                   ref[:, 0, rt[p // bs], p % bs])
+    finally:
+        dev.close()
+
+
+def test_mixed_batch_and_many_ops():
+    """One call carrying token-delta chunks of both widths next to raw and int8 chunks, more ops than one launch holds."""
+    shape = synth.TOY.with_(n_layers=2, n_kv_heads=2, head_dim=64, block_size=16, n_blocks=512)
+    dev = Device(shape, seed=23)
+    try:
+        K = dev.K
+        host = dev.pool_np()
+        rng = np.random.default_rng(5)
+        n = 45
+        codecs = [(TD8, TD4, RAW, INT8)[i % 4] for i in range(n)]
+        Ts = [int(rng.integers(1, 130)) for _ in range(n)]
+        tabs = [rng.permutation(512)[:9].astype(np.int32) for _ in range(n)]
+        bufs = [dev.chunk_buf(T, c) for T, c in zip(Ts, codecs)]
+        dev.store([dev.op(dev.table(t), 0, b, T, c) for t, b, T, c in zip(tabs, bufs, Ts, codecs)])
+        assert dev.sync() == 0
+        wants = []
+        for t, b, T, c in zip(tabs, bufs, Ts, codecs):
+            want = oracle.store(host, t, 0, T, c)
+            wants.append(want)
+            got = to_np(b)
+            if c in (TD8, TD4):
+                used = oracle.td_used_bytes(want, 2, 2, 64, T, c)
+                assert np.array_equal(got[:used], want[:used])
+            else:
+                assert np.array_equal(got, want)
+        # retrieve all of them into disjoint destinations in one call
+        dst = rng.permutation(512).astype(np.int32)[:n * 9].reshape(n, 9)
+        dev.retrieve([dev.op(dev.table(d), 0, b, T, c) for d, b, T, c in zip(dst, bufs, Ts, codecs)])
+        assert dev.sync() == 0
+        ref = host.copy()
+        for d, w, T, c in zip(dst, wants, Ts, codecs):
+            oracle.retrieve(ref, d, 0, T, c, w)
+        assert np.array_equal(dev.pool_np(), ref)
+    finally:
+        dev.close()
+
+
+def test_layerwise_retrieve_of_a_token_delta_chunk():
+    shape = synth.TOY.with_(n_layers=5, n_kv_heads=2, head_dim=64, block_size=16, n_blocks=64)
+    dev = Device(shape, seed=29)
+    try:
+        K = dev.K
+        host = dev.pool_np()
+        perm = np.random.default_rng(2).permutation(64).astype(np.int32)
+        T = 100
+        buf = dev.chunk_buf(T, TD4)
+        dev.store([dev.op(dev.table(perm[:7]), 0, buf, T, TD4)])
+        assert dev.sync() == 0
+        K.kdn_retrieve_layerwise(dev.ctx, dev.pool_id, [dev.op(dev.table(perm[10:17]), 0, buf, T, TD4)], 2, dev.stream.cuda_stream)
+        assert dev.sync() == 0
+        ref = host.copy()
+        oracle.retrieve(ref, perm[10:17], 0, T, TD4, oracle.store(host, perm[:7], 0, T, TD4))
+        assert np.array_equal(dev.pool_np(), ref)
+    finally:
+        dev.close()
+
+
+def test_refusals_and_damaged_chunks():
+    shape = synth.TOY.with_(n_layers=1, n_kv_heads=2, head_dim=64, block_size=16, n_blocks=64)
+    dev = Device(shape, seed=3)
+    try:
+        K = dev.K
+        tab = dev.table(np.arange(8, dtype=np.int32))
+        T = 64
+        buf = dev.chunk_buf(T, TD8)
+        for bad in (lambda: dev.store([dev.op(tab, 3, buf, T, TD8)]),                       # first token not at a block start
+                    lambda: dev.store([dev.op(tab, 0, dev.chunk_buf(T, TD8, pinned=True), T, TD8)]),   # host-resident chunk
+                    lambda: K.kdn_store_sparse(dev.ctx, dev.pool_id, [dev.op(tab, 0, buf, T, TD8)], [tab.data_ptr()], dev.stream.cuda_stream)):
+            with pytest.raises(K.KdnError) as e:
+                bad()
+            assert e.value.status == K.KDN_E_UNSUPPORTED
+        st = K.kdn_compose_static(0, dev.desc, [K.ComposeReq(tab.data_ptr(), 8, [dev.chunk(buf, T, TD8)], [0], 1e4)], dev.stream.cuda_stream)
+        assert st == K.KDN_E_UNSUPPORTED
+        assert K.kdn_chunk_bytes(K.pool_desc(1, 2, 80, 16, 64), T, TD8) == 0            # head_dim not a multiple of 64
+        # a damaged chunk is reported, never followed: lengths that cannot be, and an offset outside the chunk
+        dev.store([dev.op(tab, 0, buf, T, TD8)])
+        assert dev.sync() == 0
+        host = dev.pool_np()
+        lay = K.kdn_td_layout(dev.desc, T, TD8)
+        good = buf.clone()
+        buf[lay["lens_offset"]:lay["lens_offset"] + 128] = 255
+        dev.retrieve([dev.op(dev.table(np.arange(8, dtype=np.int32) + 20), 0, buf, T, TD8)])
+        assert dev.sync() == K.KDN_E_RANGE
+        buf.copy_(good)
+        buf[:8].copy_(torch.from_numpy(np.array([lay["capacity"] + 4096], dtype=np.uint64).view(np.uint8)).to(dev.dev))
+        dev.retrieve([dev.op(dev.table(np.arange(8, dtype=np.int32) + 20), 0, buf, T, TD8)])
+        assert dev.sync() == K.KDN_E_RANGE
+        buf.copy_(good)
+        dev.retrieve([dev.op(dev.table(np.arange(8, dtype=np.int32) + 40), 0, buf, T, TD8)])
+        assert dev.sync() == 0
+        ref = host.copy()
+        oracle.retrieve(ref, np.arange(8, dtype=np.int32) + 40, 0, T, TD8, oracle.store(host, np.arange(8, dtype=np.int32), 0, T, TD8))
+        got = dev.pool_np()
+        assert np.array_equal(got[:, :, 40:], ref[:, :, 40:]) and np.array_equal(got[:, :, :20], ref[:, :, :20])
+    finally:
+        dev.close()

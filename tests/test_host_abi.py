@@ -31,7 +31,7 @@ def test_chunk_bytes_matches_oracle():
     for (L, H, D) in [(2, 2, 64), (32, 8, 128), (80, 8, 128), (1, 3, 8), (4, 1, 192), (2, 2, 96)]:
         d = K.pool_desc(L, H, D, 16, 64)
         for T in (0, 1, 17, 512, 2048):
-            for codec in (0, 1, 2, 3, 4):
+            for codec in (0, 1, 2, 3, 4, 5, 6):
                 assert K.kdn_chunk_bytes(d, T, codec) == oracle.chunk_bytes(L, H, D, T, codec), (L, H, D, T, codec)
     d = K.pool_desc(2, 2, 64, 16, 64)
     assert K.kdn_chunk_bytes(d, -1, 0) == 0
@@ -58,7 +58,7 @@ def test_validate_xfer_status_codes():
     assert K.kdn_validate_xfer(d, [good_op(d, data=0x10008)]) == K.KDN_E_ALIGN
     assert K.kdn_validate_xfer(d, [good_op(d, data=0)]) == K.KDN_E_INVAL
     assert K.kdn_validate_xfer(d, [good_op(d, table=0)]) == K.KDN_E_INVAL
-    assert K.kdn_validate_xfer(d, [good_op(d, codec=5)]) == K.KDN_E_INVAL
+    assert K.kdn_validate_xfer(d, [good_op(d, codec=7)]) == K.KDN_E_INVAL
     op = good_op(d)
     op.chunk.bytes += 2
     assert K.kdn_validate_xfer(d, [op]) == K.KDN_E_SHAPE
@@ -78,7 +78,7 @@ def test_validate_xfer_status_codes():
 
 def test_validate_per_channel_key_codecs():
     d = K.pool_desc(2, 2, 64, 16, 64)
-    for codec in (K.KDN_CODEC_INT8_KC64, K.KDN_CODEC_INT4_KC64):
+    for codec in (K.KDN_CODEC_INT8_KC64, K.KDN_CODEC_INT4_KC64, K.KDN_CODEC_INT8_TD64, K.KDN_CODEC_INT4_TD64):
         assert K.kdn_validate_xfer(d, [good_op(d, T=20, off=0, codec=codec)]) == K.KDN_OK
         assert K.kdn_validate_xfer(d, [good_op(d, T=10, off=16, codec=codec)]) == K.KDN_OK
         assert K.kdn_validate_xfer(d, [good_op(d, T=20, off=3, codec=codec)]) == K.KDN_E_UNSUPPORTED     # not at a block start
