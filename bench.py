@@ -43,7 +43,7 @@ WORKLOAD = ("llama3-8b KV (L32 H8 D128 bf16, block_size 16, 16384-block pool): s
             "compose 10x1024 tokens (+256-token suffix), raw bf16 and int8-g64, fully fragmented tables")
 N_CHUNKS, CHUNK_TOKENS = 64, 512
 N_PARTS, PART_TOKENS, SUFFIX_TOKENS = 10, 1024, 256
-RAW, INT8, INT4, INT8KC, INT4KC = 0, 1, 2, 3, 4
+RAW, INT8, INT4, INT8KC, INT4KC, INT8TD, INT4TD = 0, 1, 2, 3, 4, 5, 6
 FALLBACK_HBM_GBS = 6650.0
 
 
@@ -533,6 +533,44 @@ def extras_8b(leg, dev_sets, reps):
                 for f in files:
                     f.close()
     out["ops_file_not_in_value"] = file_ops
+
+    # token-delta Rice codecs (quantise, then entropy-code along tokens): how small the chunks get and how fast they are
+    # stored and decoded, on inputs whose neighbouring tokens correlate with coefficient rho (rho = 0: the ordinary
+    # uncorrelated input, the worst case for this codec).  This leg rewrites the library's source blocks, so it runs last.
+    td = {}
+    n_td = min(n_lib, 32)
+    bf16_bytes = n_td * T * E * 2
+    for rho in (0.0, 0.9, 0.99):
+        for c in range(n_td):
+            x = synth.correlated_tokens(shape, T, rho, synth.SEED_VALUES + 100 + c, dev)
+            synth.place_tokens(leg.k, leg.v, leg.d_src[c * bpc:(c + 1) * bpc].cpu().numpy(), 0, x)
+        del x
+        for codec, cname in ((INT8TD, "int8td"), (INT4TD, "int4td")):
+            cb = K.kdn_chunk_bytes(desc, T, codec)
+            lay = K.kdn_td_layout(desc, T, codec)
+            buf = torch.empty(n_td * cb, dtype=torch.uint8, device=dev)
+            st_ops = [K.XferOp(leg.d_src.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(buf.data_ptr() + c * cb, cb, T, codec)) for c in range(n_td)]
+            rt_ops = [K.XferOp(leg.d_dst.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(buf.data_ptr() + c * cb, cb, T, codec)) for c in range(n_td)]
+            reqs = [K.ComposeReq(leg.d_dst.data_ptr() + c * bpc * i32, bpc, [K.Chunk(buf.data_ptr() + c * cb, cb, T, codec, K.KDN_MEM_DEVICE, 4096)],
+                                 [0], shape.rope_theta) for c in range(n_td)]
+            ms_store = leg.timed(lambda: K.kdn_store(ctx, pid, st_ops, s), min(reps, 5), warm=2)
+            leg.check()
+            used = sum(int(buf[c * cb + 8 * lay["segments"]:c * cb + 8 * lay["segments"] + 8].view(torch.int64).item()) for c in range(n_td))
+            ms_retr = leg.timed(lambda: K.kdn_retrieve(ctx, pid, rt_ops, s), min(reps, 5), warm=2)
+            ms_comp = leg.timed(lambda: K.kdn_compose(ctx, pid, reqs, s), min(reps, 5), warm=2)
+            leg.check()
+            moved = used + bf16_bytes                        # coded bytes on the chunk side, bf16 on the pool side
+            td["%s_rho_%s" % (cname, rho)] = {
+                "chunk_bytes_used": used, "bits_per_element": 8.0 * used / (n_td * T * E), "smaller_than_bf16_by": bf16_bytes / used,
+                "store_ms": ms_store, "store_gbs": moved / (ms_store * 1e-3) / 1e9,
+                "retrieve_ms": ms_retr, "retrieve_gbs": moved / (ms_retr * 1e-3) / 1e9, "retrieve_tokens_per_s": n_td * T / (ms_retr * 1e-3),
+                "compose_ms": ms_comp, "compose_gbs": moved / (ms_comp * 1e-3) / 1e9,
+                "retrieve_frac_of_8000": moved / (ms_retr * 1e-3) / 1e9 / 8000.0}
+            del buf
+        torch.cuda.empty_cache()
+    td["what"] = ("%d chunks x %d tokens; GB/s counts the bytes the chunks use plus the bf16 bytes on the pool side; "
+                  "rho = correlation of neighbouring tokens in the synthetic input" % (n_td, T))
+    out["ops_token_delta_rice_not_in_value"] = td
     return out
 
 

@@ -43,5 +43,30 @@ def build(force: bool = False, verbose: bool = False) -> str:
     return LIB
 
 
+def cuda_home() -> str:
+    return os.path.dirname(os.path.dirname(nvcc_path()))
+
+
+def build_example(name: str, out_dir: str) -> str:
+    """Compile examples/<name>.c (plain C99 against include/kdn.h) and link it with libkdn.so; returns the executable."""
+    build()
+    src = os.path.join(HERE, "examples", name + ".c")
+    exe = os.path.join(out_dir, name)
+    cc = shutil.which("gcc") or shutil.which("cc")
+    if not cc:
+        raise RuntimeError("no C compiler found")
+    cuda = cuda_home()
+    subprocess.run([cc, "-std=c99", "-O2", "-Wall", "-I", os.path.join(ROOT, "include"), "-I", os.path.join(cuda, "include"),
+                    src, "-o", exe, "-L", HERE, "-lkdn", "-L", os.path.join(cuda, "lib64"), "-lcudart",
+                    "-Wl,-rpath," + HERE, "-Wl,-rpath," + os.path.join(cuda, "lib64")], check=True)
+    return exe
+
+
+def example_env() -> dict:
+    env = dict(os.environ)
+    env["LD_LIBRARY_PATH"] = HERE + os.pathsep + os.path.join(cuda_home(), "lib64") + os.pathsep + env.get("LD_LIBRARY_PATH", "")
+    return env
+
+
 if __name__ == "__main__":
     print(build(force="--force" in sys.argv, verbose="-v" in sys.argv))

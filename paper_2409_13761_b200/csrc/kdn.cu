@@ -33,6 +33,7 @@ constexpr int kRing = 8;                   // launches that may be queued before
 constexpr int kMaxOpsPerLaunch = 4096;
 constexpr unsigned kMaxTilesPerLaunch = 0x7fff0000u;
 constexpr size_t kDefaultSlabBytes = (size_t)256 << 20;
+constexpr unsigned kTdCols = 128;           // channels per CTA of the token-delta kernels
 
 struct Pool {
     int L, H, D, bs;
@@ -328,7 +329,8 @@ Shape default_shape(int OP, bool any_coded, bool any_rot)
 
 // Pipeline slots: at least lag + 2, a multiple of the compute groups (a slot must always belong to the
 // same group), and, unless the caller fixed the count, few enough for ctas_per_sm CTAs to share an SM.
-kdn_status fit_stages(int &stages, int groups, int lag, bool shrink, unsigned stage_bytes, int ctas_per_sm, size_t smem_limit)
+kdn_status fit_stages(int &stages, int groups, int lag, bool shrink, unsigned stage_bytes, int ctas_per_sm, size_t smem_limit,
+                      int rows_per_tile = 1)
 {
     const int g = groups > 0 ? groups : 1;
     if (stages > kMaxStages) stages = kMaxStages;
@@ -337,9 +339,9 @@ kdn_status fit_stages(int &stages, int groups, int lag, bool shrink, unsigned st
     stages = stages / g * g;
     if (shrink)
         while (stages - g >= min_stages &&
-               smem_bytes(stages, stage_bytes) * (size_t)ctas_per_sm > smem_limit - 1024u * (size_t)ctas_per_sm)
+               smem_bytes(stages, stage_bytes, rows_per_tile) * (size_t)ctas_per_sm > smem_limit - 1024u * (size_t)ctas_per_sm)
             stages -= g;
-    return smem_bytes(stages, stage_bytes) > smem_limit ? KDN_E_UNSUPPORTED : KDN_OK;
+    return smem_bytes(stages, stage_bytes, rows_per_tile) > smem_limit ? KDN_E_UNSUPPORTED : KDN_OK;
 }
 
 // Launch the instantiation for (OP, compute groups, warps per group); groups = 0 is the pure-copy form.
@@ -404,11 +406,23 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     // a token-list op moves one token row per tile: the tile must hold a row; a launch of only such ops uses
     // row-sized slots and as many of them as fit, to keep enough bytes in flight
     if (any_list && tile_elems < row_elems) tile_elems = row_elems;
+    int rows_per_tile = 1;
     if (all_list) {
         // row-sized tiles are bound by the per-CTA loader and storer, not by bytes in flight per CTA: measured on
         // the 8B shape (2 KiB rows), throughput grows with CTAs per SM up to 8 (copy form 3.0 -> 6.4 TB/s)
         tile_elems = row_elems;
-        if (!any_coded && !any_rot) def = Shape{ 0, 4, 8, 0, 1 };
+        bool all_keep = true;
+        for (int i = 0; i < n; ++i) all_keep &= hops[i].op.list_mode == 1;
+        const int want_rows = ctx->tuning.tile_bytes > 0 ? ctx->tuning.tile_bytes / 2 / (int)row_elems : 2048 / (int)row_elems;
+        if (any_coded && !any_rot && all_keep && want_rows >= 2 && (unsigned long long)pool.nb * (unsigned)pool.bs < 0xffffffffull) {
+            // coded keep-list launches: a tile takes several listed rows -- neighbours in the chunk, so its codes and
+            // scales move with one copy each, and rows that are neighbours in the pool share a copy too.  From a sweep on
+            // the 8B shape with half of the tokens kept: two 1024-element rows per tile, five CTAs per SM with two
+            // single-warp groups each, one store in flight (int8 5.1 -> 5.9 TB/s, int4 4.0 -> 4.9)
+            rows_per_tile = want_rows > kMaxRowsPerTile ? kMaxRowsPerTile : want_rows;
+            tile_elems = (unsigned)rows_per_tile * row_elems;
+            def = Shape{ 0, 6, 5, 2, 1, 1 };
+        } else if (!any_coded && !any_rot) def = Shape{ 0, 4, 8, 0, 1 };
         else if (OP == OP_STORE) def = Shape{ 0, 8, 8, 2, 2, 1 };      // two single-warp groups: a row is one warp's work
         else def = Shape{ 0, 8, 6, 2, 1, 1 };
     }
@@ -425,9 +439,9 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     int ctas_per_sm = ctx->tuning.ctas_per_sm > 0 ? ctx->tuning.ctas_per_sm : def.ctas_per_sm;
     int stages = ctx->tuning.stages > 0 ? ctx->tuning.stages : def.stages;
     const size_t smem_limit = (size_t)ctx->env.smem_optin;
-    kdn_status fit = fit_stages(stages, groups, lag, ctx->tuning.stages <= 0, stage_bytes, ctas_per_sm, smem_limit);
+    kdn_status fit = fit_stages(stages, groups, lag, ctx->tuning.stages <= 0, stage_bytes, ctas_per_sm, smem_limit, rows_per_tile);
     if (fit != KDN_OK) return fit;
-    const size_t smem = smem_bytes(stages, stage_bytes);
+    const size_t smem = smem_bytes(stages, stage_bytes, rows_per_tile);
 
     // Few ops travel as kernel parameters; otherwise through a ring slot (pinned staging + device copy).  A ring
     // slot is also what owns the rotation table.
@@ -462,7 +476,8 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
         }
         h_ops[i] = op;
         tiles += (unsigned long long)op.nl * (op.kv_sel ? 1ull : 2ull) *
-                 (op.list_mode ? (unsigned long long)op.n_list : (unsigned long long)op.nblk * tpb);
+                 (op.list_mode ? ((unsigned long long)op.n_list + (unsigned)rows_per_tile - 1ull) / (unsigned)rows_per_tile
+                               : (unsigned long long)op.nblk * tpb);
         if (tiles > kMaxTilesPerLaunch) return KDN_E_UNSUPPORTED;
     }
     if (tiles == 0) return KDN_OK;
@@ -502,6 +517,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     lp.store_lag = lag;
     lp.reload_first = (!compute && tile_elems * 2u >= 8192u) ? 1 : 0;
     lp.wait_limit_ns = ctx->wait_limit_ns;
+    lp.rows_per_tile = rows_per_tile;
 
     if (kc_groups > 0) {
         // key planes of the per-channel key codecs: one CTA per (64-token group, layer, op)
@@ -564,12 +580,13 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
 kdn_status launch_td(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *hops, int n, cudaStream_t stream)
 {
     const unsigned row_elems = (unsigned)pool.H * (unsigned)pool.D;
-    // channels per CTA: a multiple of 16 that divides the row, whole heads when keys are re-rotated, 256 if possible
+    // channels per CTA: a multiple of 16 that divides the row, whole heads when keys are re-rotated, kTdCols if possible
+    // (small slices: many CTAs share an SM, and each one's loads, decoding and stores overlap the others')
     bool any_rot = false;
     for (int i = 0; i < n; ++i) any_rot |= hops[i].rotate;
     const unsigned unit = any_rot ? lcm_u(16u, (unsigned)pool.D) : 16u;
     unsigned n_split = 1;
-    while (row_elems / n_split > 256u && row_elems % (n_split * 2u) == 0u && (row_elems / (n_split * 2u)) % unit == 0u) n_split *= 2u;
+    while (row_elems / n_split > kTdCols && row_elems % (n_split * 2u) == 0u && (row_elems / (n_split * 2u)) % unit == 0u) n_split *= 2u;
     const unsigned cols = row_elems / n_split;
     if (cols % 16u || cols > 1024u) return KDN_E_UNSUPPORTED;
     unsigned threads = (cols + 31u) & ~31u;                  // one thread per channel in the coding loops
@@ -1572,6 +1589,7 @@ extern "C" kdn_status kdn_compose_static(int device, const kdn_pool_desc *pool, 
         const unsigned long long want = (unsigned long long)sd->env.sm_count * (unsigned)ctas_per_sm;
         const unsigned grid = (unsigned)(tiles < want ? tiles : want);
         lp.wait_limit_ns = kWaitLimitNs;
+        lp.rows_per_tile = 1;
         {
             std::lock_guard<std::mutex> lock(g_static_mutex);     // the per-device occupancy cache is shared by all callers
             st = launch_tiles(sd->env, OP_COMPOSE, def.groups, def.gw, grid, smem, stream, lp);

@@ -40,7 +40,7 @@ __host__ __device__ constexpr int min_ctas_for(int groups, int group_warps)
 // the one-group form, two of the two-group form.
 __host__ __device__ constexpr int min_ctas_for_compose(int groups, int group_warps)
 {
-    return group_warps != 4 ? min_ctas_for(groups, group_warps) : groups == 0 ? 16 : groups == 1 ? 4 : groups == 2 ? 2 : 1;
+    return group_warps != 4 ? min_ctas_for(groups, group_warps) : groups == 0 ? 8 : groups == 1 ? 4 : groups == 2 ? 2 : 1;
 }
 constexpr int kThreadsCopy = 64;                             // loader + storer
 constexpr int kMaxStages = 32;
@@ -48,7 +48,9 @@ constexpr int kMaxStoreLag = 16;          // most bulk-store groups allowed to b
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // default limit of a pipeline wait, and the limit of every drain wait
 
 enum : uint32_t { TF_CODED = 1u, TF_ROTATE = 2u, TF_SCALES_PLAIN = 4u, TF_INT4 = 8u,   // TF_CODED: int8 or int4
-                  TF_KCHAN = 16u };   // key tile of a per-channel key codec: one scale per channel, row_elems of them
+                  TF_KCHAN = 16u,     // key tile of a per-channel key codec: one scale per channel, row_elems of them
+                  TF_ROWS = 32u };    // several listed token rows: contiguous in the chunk, rows[] says where each sits in the pool
+constexpr int kMaxRowsPerTile = 4;
 enum : int { OP_STORE = 0, OP_RETRIEVE = 1, OP_COMPOSE = 2 };
 
 // Status values mirrored from kdn.h (kept numeric here so device code has no host header).
@@ -108,6 +110,7 @@ struct Launch {
     int reload_first;         // copy form: after recycling a slot the storer lets the loader queue the reload
                               // before it queues the next store (see the storer loop)
     unsigned long long wait_limit_ns;   // a pipeline wait gives up after this long (the drain waits keep kWaitLimitNs)
+    int rows_per_tile;        // keep-list ops: listed token rows per tile (1: one row per tile)
     DevOp inline_ops[kInlineOps];
 };
 
@@ -119,7 +122,11 @@ struct __align__(16) TileDesc {
     unsigned flags;
     int rope;
     unsigned sbytes;              // bytes of scales that belong to the tile (coded tiles)
+    unsigned runs;                // TF_ROWS: nibble r = how many rows the copy that starts at row r covers (0: row r rides
+                                  // along with an earlier one); rows that are neighbours in the pool share one copy.  The
+                                  // rows' places in the pool plane travel beside the descriptor in shared memory.
 };
+static_assert(sizeof(TileDesc) == 48, "TileDesc is copied with 128-bit accesses");
 
 // ------------------------------------------------------------------ PTX --
 
@@ -609,11 +616,12 @@ __device__ __forceinline__ void rotate_tile(unsigned char *A, const unsigned cha
 
 // Address resolution (request position -> block-table entry -> pool address) and chunk addressing
 // for tile g.  Records KDN_E_RANGE and yields an empty tile for a block id outside the pool.
+// rows_out: shared memory for the token-row indices of a several-row tile (TF_ROWS); untouched otherwise.
 template <int OP>
-__device__ __forceinline__ void decode_tile(const Launch &P, unsigned g, TileDesc &d)
+__device__ __forceinline__ void decode_tile(const Launch &P, unsigned g, TileDesc &d, unsigned *rows_out)
 {
     d.n = 0; d.flags = 0; d.rope = -1; d.sbytes = 0;
-    d.g_pool = 0; d.g_chunk = 0; d.g_scales = 0;
+    d.g_pool = 0; d.g_chunk = 0; d.g_scales = 0; d.runs = 0;
     if (g >= P.n_tiles) return;                             // lanes past this CTA's last tile
     const DevOp *ops = P.ops ? P.ops : P.inline_ops;       // global memory, or the kernel's parameter space
     int lo = 0, hi = P.n_ops - 1;
@@ -627,7 +635,55 @@ __device__ __forceinline__ void decode_tile(const Launch &P, unsigned g, TileDes
     long long id_index;                                     // block-table entry of the tile
     unsigned long long pool_elem;                           // element offset of the tile inside its pool block
     unsigned long long ce;                                  // element offset of the tile inside the chunk
-    if (op.list_mode != 0) {
+    bool many_rows = false;
+    if (op.list_mode == 1 && P.rows_per_tile > 1) {
+        // keep-list: up to rows_per_tile consecutive listed tokens per tile; they are consecutive chunk tokens, and
+        // each sits wherever its own block-table entry says
+        const unsigned rpt = (unsigned)P.rows_per_tile;
+        const unsigned tpp = ((unsigned)op.n_list + rpt - 1u) / rpt;
+        plane = gl / tpp;
+        const unsigned i0 = (gl - plane * tpp) * rpt;
+        const unsigned nr = (unsigned)op.n_list - i0 < rpt ? (unsigned)op.n_list - i0 : rpt;
+        bool bad = false;
+        unsigned rows[kMaxRowsPerTile];
+#pragma unroll
+        for (int r = 0; r < kMaxRowsPerTile; ++r) {
+            rows[r] = 0u;
+            if ((unsigned)r < nr) {
+                const long long rel = __ldg(op.list + i0 + (unsigned)r);
+                const long long p = op.off + rel;
+                if (rel < 0 || p >= op.pos_end || (long long)(i0 + (unsigned)r) >= op.T) { bad = true; continue; }
+                const long long bi = p / P.bs;
+                const long long id = __ldg(op.table + bi);
+                if (id < 0 || id >= P.n_blocks) { bad = true; continue; }
+                rows[r] = (unsigned)(id * P.bs + (p - bi * P.bs));
+            }
+        }
+        if (bad) { atomicCAS(P.status, 0, kStatusRange); return; }          // the whole tile is skipped
+        // runs of rows that are neighbours in the pool, worked out back to front (all indices are compile-time: the
+        // arrays stay in registers)
+        unsigned len[kMaxRowsPerTile + 1];
+        len[kMaxRowsPerTile] = 0u;
+        unsigned runs = 0u;
+#pragma unroll
+        for (int r = kMaxRowsPerTile - 1; r >= 0; --r) {
+            const bool next_joins = r + 1 < kMaxRowsPerTile && (unsigned)(r + 1) < nr && rows[r + 1 < kMaxRowsPerTile ? r + 1 : r] == rows[r] + 1u;
+            len[r] = (unsigned)r < nr ? 1u + (next_joins ? len[r + 1] : 0u) : 0u;
+        }
+#pragma unroll
+        for (int r = 0; r < kMaxRowsPerTile; ++r) {
+            const bool joins_prev = r > 0 && rows[r] == rows[r > 0 ? r - 1 : 0] + 1u;
+            if (!joins_prev) runs |= len[r] << (4 * r);
+        }
+        *reinterpret_cast<uint4 *>(rows_out) = make_uint4(rows[0], rows[1], rows[2], rows[3]);
+        d.runs = runs;
+        d.flags |= TF_ROWS;
+        many_rows = true;
+        id_index = 0;
+        pool_elem = 0;
+        ce = (unsigned long long)i0 * P.row_elems;
+        n = nr * P.row_elems;
+    } else if (op.list_mode != 0) {
         // one listed token (one row of H * D elements) per tile
         plane = gl / (unsigned)op.n_list;
         const unsigned i = gl - plane * (unsigned)op.n_list;
@@ -661,10 +717,14 @@ __device__ __forceinline__ void decode_tile(const Launch &P, unsigned g, TileDes
     const int kv = op.kv_sel ? op.kv_sel - 1 : (int)(plane & 1u);
     const unsigned li = op.kv_sel ? plane : plane >> 1;     // layer index inside the op's layer range
     const int l = op.l0 + (int)li;
-    const long long id = __ldg(op.table + id_index);
-    if (id < 0 || id >= P.n_blocks) { atomicCAS(P.status, 0, kStatusRange); return; }
     const unsigned char *base = reinterpret_cast<const unsigned char *>(kv ? P.v_layers[l] : P.k_layers[l]);
-    d.g_pool = (unsigned long long)(base + ((unsigned long long)id * P.bs * P.row_elems + pool_elem) * 2ull);
+    if (many_rows) {
+        d.g_pool = (unsigned long long)base;
+    } else {
+        const long long id = __ldg(op.table + id_index);
+        if (id < 0 || id >= P.n_blocks) { atomicCAS(P.status, 0, kStatusRange); d.flags = 0; return; }
+        d.g_pool = (unsigned long long)(base + ((unsigned long long)id * P.bs * P.row_elems + pool_elem) * 2ull);
+    }
     const unsigned long long ce_plane = ce;                                   // element offset inside the plane
     ce += ((unsigned long long)li * 2ull + (unsigned long long)kv) * (unsigned long long)op.T * P.row_elems;
     if (op.codec == 0) {
@@ -704,6 +764,8 @@ struct Smem {
     unsigned char *stage0;
     uint32_t full, empty, ready;      // shared addresses of the barrier arrays (8 bytes per stage)
     TileDesc *desc;
+    unsigned *rows_stage;             // [stages][4]: token-row indices of the several-row tile in each slot
+    unsigned *rows_ahead;             // [2][32][4]: the same for the tiles the loader has decoded but not yet queued
     volatile int *abort_flag;
     volatile unsigned *issued;        // tiles whose loads the loader has queued so far
 };
@@ -719,15 +781,20 @@ __device__ __forceinline__ Smem carve(const Launch &P, unsigned char *smem)
     p += 24u * (size_t)P.stages;
     p = (unsigned char *)(((uintptr_t)p + 15u) & ~(uintptr_t)15u);
     s.desc = reinterpret_cast<TileDesc *>(p);
-    s.abort_flag = reinterpret_cast<volatile int *>(p + sizeof(TileDesc) * (size_t)P.stages);
+    p += sizeof(TileDesc) * (size_t)P.stages;
+    s.rows_stage = reinterpret_cast<unsigned *>(p);          // both areas exist only in launches with several-row tiles
+    s.rows_ahead = s.rows_stage + 4u * (size_t)P.stages;
+    if (P.rows_per_tile > 1) p += 16u * (size_t)P.stages + 16u * 64u;
+    s.abort_flag = reinterpret_cast<volatile int *>(p);
     s.issued = reinterpret_cast<volatile unsigned *>(s.abort_flag + 1);
     return s;
 }
 
 // Bytes of shared memory a launch needs (host mirrors this).
-__host__ __device__ inline size_t smem_bytes(int stages, unsigned stage_bytes)
+__host__ __device__ inline size_t smem_bytes(int stages, unsigned stage_bytes, int rows_per_tile = 1)
 {
-    return (size_t)stages * stage_bytes + 24u * (size_t)stages + 16u + sizeof(TileDesc) * (size_t)stages + 16u;
+    return (size_t)stages * stage_bytes + 24u * (size_t)stages + 16u + sizeof(TileDesc) * (size_t)stages + 16u +
+           (rows_per_tile > 1 ? 16u * (size_t)stages + 16u * 64u : 0u);
 }
 
 template <int OP, int kGroups, int kGW>
@@ -766,10 +833,12 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
         uint32_t ph = 0;                                      // barriers (flips every time the slots wrap around)
         bool aborted = false;
         TileDesc cur;
-        decode_tile<OP>(P, (unsigned)lane < n_my ? bid + (unsigned)lane * grid : 0xffffffffu, cur);
+        unsigned ahead = 0;                                   // which half of rows_ahead holds the rows of `cur`
+        decode_tile<OP>(P, (unsigned)lane < n_my ? bid + (unsigned)lane * grid : 0xffffffffu, cur, sm.rows_ahead + (size_t)lane * 4u);
         for (unsigned base = 0; base < n_my && !aborted; base += 32u) {
             TileDesc nxt;
-            decode_tile<OP>(P, base + 32u + lane < n_my ? bid + (base + 32u + lane) * grid : 0xffffffffu, nxt);
+            decode_tile<OP>(P, base + 32u + lane < n_my ? bid + (base + 32u + lane) * grid : 0xffffffffu, nxt,
+                            sm.rows_ahead + ((size_t)(ahead ^ 1u) * 32u + (size_t)lane) * 4u);
             const unsigned cnt = n_my - base < 32u ? n_my - base : 32u;
             for (unsigned t = 0; t < cnt; ++t) {
                 bool ok = true;                               // lane t: the slot was free and the tile's copies are queued
@@ -777,13 +846,29 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                     ok = mbar_wait(sm.empty + 8u * st, ph ^ 1u, sm.abort_flag, P.wait_limit_ns);
                     if (ok) {
                         sm.desc[st] = cur;
+                        if (OP != OP_STORE && (cur.flags & TF_ROWS))       // the storer scatters the rows
+                            *reinterpret_cast<uint4 *>(sm.rows_stage + (size_t)st * 4u) =
+                                *reinterpret_cast<const uint4 *>(sm.rows_ahead + ((size_t)ahead * 32u + (size_t)lane) * 4u);
                         const uint32_t bar = sm.full + 8u * st;
                         unsigned char *A = sm.stage0 + (size_t)st * P.stage_bytes;
                         if (cur.n == 0u) {
                             mbar_arrive(bar);
                         } else if (OP == OP_STORE) {
                             mbar_arrive_expect_tx(bar, cur.n * 2u);
-                            bulk_g2s(smem_u32(A), (const void *)cur.g_pool, cur.n * 2u, bar);
+                            if (cur.flags & TF_ROWS) {
+                                // one copy per run of rows that are neighbours in the pool
+                                const unsigned rb = P.row_elems * 2u;
+                                const uint4 rv = *reinterpret_cast<const uint4 *>(sm.rows_ahead + ((size_t)ahead * 32u + (size_t)lane) * 4u);
+                                const unsigned rows[kMaxRowsPerTile] = { rv.x, rv.y, rv.z, rv.w };
+#pragma unroll
+                                for (int r = 0; r < kMaxRowsPerTile; ++r) {
+                                    const unsigned len = (cur.runs >> (4 * r)) & 15u;
+                                    if (len) bulk_g2s(smem_u32(A + (size_t)r * rb), (const void *)(cur.g_pool + (unsigned long long)rows[r] * rb),
+                                                      len * rb, bar);
+                                }
+                            } else {
+                                bulk_g2s(smem_u32(A), (const void *)cur.g_pool, cur.n * 2u, bar);
+                            }
                         } else if (!(cur.flags & TF_CODED)) {
                             mbar_arrive_expect_tx(bar, cur.n * 2u);
                             bulk_g2s(smem_u32(A), (const void *)cur.g_chunk, cur.n * 2u, bar);
@@ -811,6 +896,7 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                 if (++st == (unsigned)S) { st = 0; ph ^= 1u; }
             }
             cur = nxt;
+            ahead ^= 1u;
         }
         if (aborted && lane == 0) {
             atomicCAS(P.status, 0, kStatusTimeout);
@@ -843,6 +929,15 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                                 bulk_s2g((void *)d.g_scales, smem_u32(A + P.off_s), d.sbytes);
                         } else {
                             bulk_s2g((void *)d.g_chunk, smem_u32(A), d.n * 2u);
+                        }
+                    } else if (d.flags & TF_ROWS) {
+                        const unsigned rb = P.row_elems * 2u;
+                        const uint4 rv = *reinterpret_cast<const uint4 *>(sm.rows_stage + (size_t)st * 4u);
+                        const unsigned rows[kMaxRowsPerTile] = { rv.x, rv.y, rv.z, rv.w };
+#pragma unroll
+                        for (int r = 0; r < kMaxRowsPerTile; ++r) {
+                            const unsigned len = (d.runs >> (4 * r)) & 15u;
+                            if (len) bulk_s2g((void *)(d.g_pool + (unsigned long long)rows[r] * rb), smem_u32(A + (size_t)r * rb), len * rb);
                         }
                     } else {
                         bulk_s2g((void *)d.g_pool, smem_u32(A), d.n * 2u);

@@ -64,12 +64,19 @@ __host__ __device__ inline size_t td_store_smem_bytes(unsigned cols, bool encode
     return (size_t)64 * cols * 2u + (size_t)kKcSlices * cols * 2u + (size_t)cols * 4u +
            (encode ? (size_t)cols * 72u + 32u : 0u) + 256u + 16u;
 }
-// Shared memory of the decode kernel: bf16 rows (the stream bytes land in the same area first), codes, scales,
-// lens / offsets, barrier.
+// Shared memory of the decode kernel: the slice's stream bytes as they lie in the chunk, the same sub-streams
+// interleaved word by word (so that the 32 lanes of a warp read 32 different banks), codes, scales, offsets, barrier.
+// The bf16 rows reuse the two stream areas once the codes are complete.
+constexpr unsigned kTdWords = 19;                           // 32-bit words per interleaved sub-stream: 72 bytes, and the word after
+__host__ __device__ inline size_t td_decode_packed_bytes(unsigned cols) { return ((size_t)cols * 72u + 128u + 127u) & ~(size_t)127u; }
+__host__ __device__ inline size_t td_decode_front_bytes(unsigned cols)
+{
+    const size_t a = (size_t)64 * cols * 2u, s = td_decode_packed_bytes(cols) + (size_t)kTdWords * cols * 4u;
+    return a > s ? a : s;
+}
 __host__ __device__ inline size_t td_decode_smem_bytes(unsigned cols)
 {
-    const size_t a = (size_t)64 * cols * 2u, s = (size_t)cols * 72u + 512u;
-    return (a > s ? a : s) + (size_t)64 * cols + (size_t)cols * 4u + (size_t)cols * 4u + 256u + 16u;
+    return td_decode_front_bytes(cols) + (size_t)64 * cols + (size_t)cols * 4u + 256u + 16u;
 }
 
 // Bits of one Rice code word.
@@ -456,13 +463,12 @@ __global__ void __launch_bounds__(512) kdn_td_decode_kernel(const __grid_constan
     const unsigned C = P.cols, RE = P.row_elems;
     const int codec = s.op.codec;
     const unsigned raw_bits = (unsigned)td_raw_bits(codec);
-    const size_t a_bytes = (size_t)64 * C * 2u, s_bytes = (size_t)C * 72u + 512u;
 
-    unsigned char *A = smem_raw;                                         // bf16 rows; first the slice's stream bytes
-    unsigned char *B = A + (a_bytes > s_bytes ? a_bytes : s_bytes);      // codes [n_tok][C]
+    unsigned char *A = smem_raw;                                         // bf16 rows; first the slice's stream bytes ...
+    uint32_t *I = reinterpret_cast<uint32_t *>(A + td_decode_packed_bytes(C));   // ... and the interleaved sub-streams [word][C]
+    unsigned char *B = A + td_decode_front_bytes(C);                     // codes [n_tok][C]
     float *Sc = reinterpret_cast<float *>(B + (size_t)64 * C);           // scales [C]
-    unsigned *offs = reinterpret_cast<unsigned *>(Sc + C);               // per channel: byte offset << 8 | param
-    unsigned *scratch = offs + C;                                        // 64 words
+    unsigned *scratch = reinterpret_cast<unsigned *>(Sc + C);            // 64 words
     unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(reinterpret_cast<unsigned char *>(scratch) + 256u);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bar_mem + 1);
     const uint32_t bar = smem_u32(bar_mem);
@@ -482,8 +488,9 @@ __global__ void __launch_bounds__(512) kdn_td_decode_kernel(const __grid_constan
     td_block_scan(before, scratch, &total_before);                        // (its barriers also publish the mbarrier)
     const unsigned my_len = tid < C ? lens[s.c0 + tid] : 0u;               // blockDim.x >= C
     const unsigned my_off = td_block_scan(my_len, scratch, &total_slice);
+    unsigned param = 0;
     if (tid < C) {
-        offs[tid] = (my_off << 8) | s.op.data[lay.params + row + s.c0 + tid];
+        param = s.op.data[lay.params + row + s.c0 + tid];
         Sc[tid] = reinterpret_cast<const float *>(s.op.data + lay.scales)[row + s.c0 + tid];
     }
     const unsigned long long seg_begin = reinterpret_cast<const unsigned long long *>(s.op.data)[s.seg];
@@ -519,36 +526,43 @@ __global__ void __launch_bounds__(512) kdn_td_decode_kernel(const __grid_constan
     }
     // one thread per channel: Rice, zigzag, delta -> codes
     if (tid < C) {
-        const unsigned o = offs[tid];
-        const unsigned mode = (o >> 3) & 1u, k = o & 7u;
-        const uint32_t addr = smem_u32(A) + shift + (o >> 8);
-        uint32_t wp = addr & ~3u;
-        const unsigned skip = (addr & 3u) * 8u;
-        uint32_t w;
-        asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w) : "r"(wp));
-        unsigned long long buf = ((unsigned long long)td_be(w) << 32) << skip;
-        int nb = 32 - (int)skip;
-        wp += 4u;
-        int prev = 0;
-        unsigned char *bp = B + tid;
-        for (unsigned t = 0; t < s.n_tok; ++t) {
-            if (nb <= 32) {
-                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w) : "r"(wp));
-                buf |= (unsigned long long)td_be(w) << (32 - nb);
-                nb += 32;
-                wp += 4u;
+        const unsigned mode_mask = (param & 8u) ? 0xffffffffu : 0u, k = param & 7u;
+        // the sub-stream, as big-endian words, into column tid of the interleaved area: word j of every channel sits in
+        // one row, so a warp's loads below never meet in a bank wherever each lane is in its stream
+        {
+            const uint32_t addr = smem_u32(A) + shift + my_off;
+            const uint32_t al = addr & ~3u;
+            const unsigned sh8 = (addr & 3u) * 8u;
+            // (a length no sub-stream can have means a damaged chunk: reported, and clamped so that nothing leaves the area)
+            if (my_len > td_max_len(codec)) atomicCAS(P.status, 0, kStatusRange);
+            const unsigned len_c = my_len < td_max_len(codec) ? my_len : td_max_len(codec);
+            const unsigned nw = ((len_c + 3u) >> 2) + 1u;                 // the window below looks one word past the last bit
+            uint32_t x0, x1;
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(x0) : "r"(al));
+            for (unsigned j = 0; j < nw; ++j) {
+                asm volatile("ld.shared.u32 %0, [%1];" : "=r"(x1) : "r"(al + 4u * (j + 1u)));
+                I[(size_t)j * C + tid] = td_be(__funnelshift_r(x0, x1, sh8));
+                x0 = x1;
             }
-            const uint32_t hi = (uint32_t)(buf >> 32);
+        }
+        const uint32_t *col = I + tid;
+        unsigned bp = 0;                                                  // bits consumed so far
+        int prev = 0;
+        unsigned char *out = B + tid;
+#pragma unroll 4
+        for (unsigned t = 0; t < s.n_tok; ++t) {
+            const unsigned wi = (bp >> 5) < kTdWords - 2u ? (bp >> 5) : kTdWords - 2u;   // a damaged stream cannot run off the area
+            const uint32_t *wp = col + (size_t)wi * C;
+            const uint32_t hi = __funnelshift_l(wp[C], wp[0], bp);       // the next 32 bits of the stream
             const unsigned ones = (unsigned)__clz((int)~hi);
-            unsigned u, len;
-            if (ones < 15u) { u = (ones << k) | (((hi << (ones + 1u)) >> 1) >> (31u - k)); len = ones + 1u + k; }
-            else { u = (hi << 15) >> (32u - raw_bits); len = 15u + raw_bits; }
-            buf <<= len;
-            nb -= (int)len;
+            unsigned u = (ones << k) | (((hi << (ones + 1u)) >> 1) >> (31u - k));
+            unsigned len = ones + 1u + k;
+            if (ones >= 15u) { u = (hi << 15) >> (32u - raw_bits); len = 15u + raw_bits; }
+            bp += len;
             const int e = (int)(u >> 1) ^ -(int)(u & 1u);
-            const int q = mode ? prev + e : e;
+            const int q = e + (prev & (int)mode_mask);
             prev = q;
-            bp[(size_t)t * C] = (unsigned char)q;
+            out[(size_t)t * C] = (unsigned char)q;
         }
     }
     __syncthreads();                                                      // codes complete, stream bytes no longer read

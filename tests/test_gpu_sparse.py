@@ -131,3 +131,71 @@ def test_list_entries_outside_the_table_are_reported_not_faulted():
         assert dev.sync() == 0
     finally:
         dev.close()
+
+
+@pytest.mark.parametrize("codec", [INT8, INT4])
+def test_coded_keep_lists_take_several_rows_per_tile(codec):
+    """Coded keep-list launches put several listed rows in a tile (two of 1024 elements, up to four shorter ones) and move rows that are neighbours in the pool with
+    one copy: lists with runs of every length, over a contiguous and over a scattered block table (runs that cross a
+    block boundary stay one copy only where the blocks are neighbours too), list lengths that leave a ragged last tile,
+    and a mixed batch with a raw op."""
+    shape = synth.TOY.with_(n_layers=2, n_kv_heads=8, head_dim=128, block_size=8, n_blocks=128)
+    dev = Device(shape, seed=61)
+    try:
+        K = dev.K
+        bs = shape.block_size
+        rng = np.random.default_rng(codec)
+        host = dev.pool_np()
+        span = 10 * bs
+        contiguous = (np.arange(10) + 50).astype(np.int32)
+        scattered = rng.permutation(50)[:10].astype(np.int32)
+        runs = np.array([0, 1, 2, 3, 5, 6, 8, 10, 11, 12, 13, 14, 15, 16, 17, 20, 23, 24, 30, 31, 32, 33, 34, 41, 47, 48, 49, 50, 51, 52, 79])
+        lists = [runs, np.arange(span), np.sort(rng.choice(span, 37, replace=False)), np.array([7, 8]), np.arange(3) * 9]
+        ops, keeps, wants, bufs = [], [], [], []
+        for tab in (contiguous, scattered):
+            for keep in lists:
+                c = codec
+                b = dev.chunk_buf(len(keep), c)
+                ops.append(dev.op(dev.table(tab), 0, b, len(keep), c))
+                keeps.append(dev_list(dev, keep).data_ptr())
+                wants.append(oracle.store(host, tab, 0, len(keep), c, keep=keep))
+                bufs.append(b)
+        raw_keep = np.array([1, 2, 3, 40])
+        rb = dev.chunk_buf(4, RAW)
+        ops.append(dev.op(dev.table(scattered), 0, rb, 4, RAW))
+        keeps.append(dev_list(dev, raw_keep).data_ptr())
+        wants.append(oracle.store(host, scattered, 0, 4, RAW, keep=raw_keep))
+        bufs.append(rb)
+        K.kdn_store_sparse(dev.ctx, dev.pool_id, ops, keeps, dev.stream.cuda_stream)
+        assert dev.sync() == 0
+        assert K.kdn_last_launch(dev.ctx)["tile_bytes"] == 2 * 1024 * 2            # two rows of 1024 elements
+        for b, w in zip(bufs, wants):
+            assert np.array_equal(to_np(b), w)
+        # retrieve each chunk into its own destination blocks: neighbouring blocks for the first, scattered for the rest
+        ref = host.copy()
+        all_keeps = lists + lists + [raw_keep]
+        free = rng.permutation(np.setdiff1d(np.arange(128), np.arange(60, 70)))
+        for i, (b, w, keep) in enumerate(zip(bufs, wants, all_keeps)):
+            dtab = (np.arange(10) + 60).astype(np.int32) if i == 0 else free[(i % 11) * 10:(i % 11) * 10 + 10].astype(np.int32)
+            c = RAW if i == len(bufs) - 1 else codec
+            K.kdn_retrieve_sparse(dev.ctx, dev.pool_id, [dev.op(dev.table(dtab), 0, b, len(keep), c)], [keeps[i]], dev.stream.cuda_stream)
+            oracle.retrieve(ref, dtab, 0, len(keep), c, w, keep=keep)
+        assert dev.sync() == 0
+        assert np.array_equal(dev.pool_np(), ref)
+        # a listed position outside the table: reported; the tile that holds it is skipped, the other tiles are written
+        keep_bad = np.array([0, 1, 2, 3, 4, 5, 6, 200], dtype=np.int32)
+        b = dev.chunk_buf(8, codec, fill=0xA5)
+        K.kdn_store_sparse(dev.ctx, dev.pool_id, [dev.op(dev.table(contiguous), 0, b, 8, codec)], [dev_list(dev, keep_bad).data_ptr()],
+                           dev.stream.cuda_stream)
+        assert dev.sync() == K.KDN_E_RANGE
+        L, R = shape.n_layers, shape.n_kv_heads * shape.head_dim
+        rows_per_tile = K.kdn_last_launch(dev.ctx)["tile_bytes"] // 2 // R
+        n_ok = 7 // rows_per_tile * rows_per_tile                                   # the tiles before the one with the bad entry
+        good = oracle.store(ref, contiguous, 0, n_ok, codec, keep=keep_bad[:n_ok])      # ref: the pool as the retrieves left it
+        got = to_np(b)
+        per_tok = R // 2 if codec == INT4 else R
+        codes = got[:L * 2 * 8 * per_tok].reshape(L * 2, 8, per_tok)
+        gcodes = good[:L * 2 * n_ok * per_tok].reshape(L * 2, n_ok, per_tok)
+        assert np.array_equal(codes[:, :n_ok], gcodes) and np.all(codes[:, n_ok:] == 0xA5)
+    finally:
+        dev.close()
