@@ -402,18 +402,22 @@ class Leg:
         self.torch.cuda.empty_cache()
 
 
-def extras_8b(leg, dev_sets, reps):
+EXTRAS = ("shell", "int4", "kc", "sparse", "single", "file", "td")
+
+
+def extras_8b(leg, dev_sets, reps, which=EXTRAS):
     """Widenings beyond the benchmark step, each timed on its own on the 8B workload (none is part of `value`)."""
     torch, K, synth = leg.torch, leg.K, leg.synth
     ctx, pid, s, dev, desc, shape, W = leg.ctx, leg.pid, leg.s, leg.dev, leg.desc, leg.shape, leg.W
     T, E, bpc, i32, n_lib = leg.T, leg.E, leg.bpc, 4, leg.n_lib
     out = {}
 
-    # storage shell: payload checksum over the raw chunk library (a read-only stream)
-    lib_buf = dev_sets[RAW]["chunks"]
-    csum_out = torch.zeros(1, dtype=torch.int64, device=dev)
-    ms = leg.timed(lambda: K.kdn_checksum(leg.local, lib_buf.data_ptr(), lib_buf.numel(), csum_out.data_ptr(), s), reps)
-    out["ops_shell_not_in_value"] = {"checksum_raw_library": {"ms": ms, "bytes": lib_buf.numel(), "gbs": lib_buf.numel() / (ms * 1e-3) / 1e9}}
+    if "shell" in which:
+        # storage shell: payload checksum over the raw chunk library (a read-only stream)
+        lib_buf = dev_sets[RAW]["chunks"]
+        csum_out = torch.zeros(1, dtype=torch.int64, device=dev)
+        ms = leg.timed(lambda: K.kdn_checksum(leg.local, lib_buf.data_ptr(), lib_buf.numel(), csum_out.data_ptr(), s), reps)
+        out["ops_shell_not_in_value"] = {"checksum_raw_library": {"ms": ms, "bytes": lib_buf.numel(), "gbs": lib_buf.numel() / (ms * 1e-3) / 1e9}}
 
     def three(sets, codec, cname, dst):
         leg.K.kdn_store(ctx, pid, sets["part_store"], s)
@@ -426,151 +430,177 @@ def extras_8b(leg, dev_sets, reps):
                          "kernel": K.kdn_last_launch(ctx)["kernel"]}
         leg.check()
 
-    # the int4 codec
-    int4_ops = {}
-    i4 = leg.make_sets(False, codecs=(INT4,))[INT4]
-    three(i4, INT4, "int4", int4_ops)
-    out["ops_int4_not_in_value"] = int4_ops
-
-    # per-channel key codecs, and what they buy: the error of the stored keys, over all channels and over the channels
-    # without the x20 outlier gain
-    def key_error_db(ops_set):
-        """Retrieve chunk 0 and compare layer 0's keys with their source blocks: signal-to-noise ratio in dB."""
-        if not W["exclusive"]:
-            return None
-        K.kdn_store(ctx, pid, ops_set["store"][:1], s)
-        K.kdn_retrieve(ctx, pid, [K.XferOp(leg.d_dst.data_ptr(), bpc, 0, ops_set["store"][0].chunk)], s)
-        leg.check()
-        x = leg.k[0][leg.d_src[:bpc].long()].float().reshape(-1, shape.row_elems)
-        y = leg.k[0][leg.d_dst[:bpc].long()].float().reshape(-1, shape.row_elems)
-        ordinary = (synth.outlier_gain(shape)[0, 0].reshape(-1) == 1).to(dev)
-        snr = lambda a, b: float(10 * torch.log10((a * a).mean() / ((a - b) ** 2).mean()))
-        return {"all_channels": snr(x, y), "ordinary_channels": snr(x[:, ordinary], y[:, ordinary])}
-
-    kc_ops = {}
-    quality = {"int4_g64": key_error_db(i4), "int8_g64": key_error_db(dev_sets[INT8])}
-    del i4
-    torch.cuda.empty_cache()
-    for codec, cname in ((INT8KC, "int8kc"), (INT4KC, "int4kc")):
-        kc = leg.make_sets(False, codecs=(codec,))[codec]
-        three(kc, codec, cname, kc_ops)
-        quality[cname] = key_error_db(kc)
-        del kc
+    if "int4" in which:
+        # the int4 codec
+        int4_ops = {}
+        i4 = leg.make_sets(False, codecs=(INT4,))[INT4]
+        three(i4, INT4, "int4", int4_ops)
+        del i4
         torch.cuda.empty_cache()
-    kc_ops["stored_key_snr_db"] = quality
-    out["ops_per_channel_key_codecs_not_in_value"] = kc_ops
+        out["ops_int4_not_in_value"] = int4_ops
 
-    # keep-lists: every chunk holds a seeded random half of its span's tokens
-    sparse_ops = {}
-    rng = np.random.default_rng(synth.SEED_ASSIGN)
-    n_keep = T // 2
-    keep_np = np.stack([np.sort(rng.choice(T, n_keep, replace=False)) for _ in range(n_lib)]).astype(np.int32)
-    d_keep = torch.from_numpy(keep_np).to(dev)
-    for codec, cname in ((RAW, "raw"), (INT8, "int8"), (INT4, "int4")):
-        cb = K.kdn_chunk_bytes(desc, n_keep, codec)
-        buf = torch.empty(n_lib * cb, dtype=torch.uint8, device=dev)
-        keeps = [d_keep.data_ptr() + c * n_keep * i32 for c in range(n_lib)]
-        st_ops = [K.XferOp(leg.d_src.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(buf.data_ptr() + c * cb, cb, n_keep, codec)) for c in range(n_lib)]
-        rt_ops = [K.XferOp(leg.d_dst.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(buf.data_ptr() + c * cb, cb, n_keep, codec)) for c in range(n_lib)]
-        for name, fn, arg in (("store_sparse_" + cname, K.kdn_store_sparse, st_ops), ("retrieve_sparse_" + cname, K.kdn_retrieve_sparse, rt_ops)):
-            ms = leg.timed(lambda: fn(ctx, pid, arg, keeps, s), reps)
-            nbytes = n_lib * n_keep * E * bytes_per_elem(codec)
-            sparse_ops[name] = {"ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9, "tokens_per_s": n_lib * n_keep / (ms * 1e-3),
-                                "kept": "%d of %d tokens per chunk, seeded random" % (n_keep, T)}
-        leg.check()
-        del buf
-    torch.cuda.empty_cache()
-    out["ops_keep_list_not_in_value"] = sparse_ops
-
-    # one chunk per call: what a single retrieve costs (CUDA events around 50 back-to-back calls)
-    single_ops = {}
-    for codec, cname in ((RAW, "raw"), (INT8, "int8")):
-        one = dev_sets[codec]["retrieve"][:1]
-        for _ in range(5):
-            K.kdn_retrieve(ctx, pid, one, s)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        t0 = time.perf_counter()
-        a.record(leg.stream)
-        for _ in range(50):
-            K.kdn_retrieve(ctx, pid, one, s)
-        b.record(leg.stream)
-        host_us = (time.perf_counter() - t0) / 50 * 1e6
-        torch.cuda.synchronize()
-        us = a.elapsed_time(b) / 50 * 1e3
-        nbytes = T * E * bytes_per_elem(codec)
-        single_ops["retrieve_one_chunk_" + cname] = {"us_per_call": us, "host_us_per_call_through_python": host_us, "gbs": nbytes / us / 1e3,
-                                                      "tokens": T, "bytes_moved": nbytes}
-    out["ops_single_chunk_not_in_value"] = single_ops
-
-    # file-backed chunks: a few chunks of the library written to and read back from files (wall clock around the call
-    # plus the stream sync, since the calling thread does the file I/O)
-    file_ops = {}
-    import tempfile
-    tmpdir = "/dev/shm" if os.path.isdir("/dev/shm") and os.access("/dev/shm", os.W_OK) else None
-    n_file = min(8, n_lib)
-    for codec, cname in ((RAW, "raw"), (INT8, "int8")):
-        cb = K.kdn_chunk_bytes(desc, T, codec)
-        st_ops = [K.XferOp(leg.d_src.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(0, cb, T, codec)) for c in range(n_file)]
-        rt_ops = [K.XferOp(leg.d_dst.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(0, cb, T, codec)) for c in range(n_file)]
-        for layout in ("one_file", "file_per_chunk"):
-            files = [tempfile.NamedTemporaryFile(dir=tmpdir, prefix="kdn_bench_") for _ in range(1 if layout == "one_file" else n_file)]
-            try:
-                fds = [files[0].fileno()] * n_file if layout == "one_file" else [f.fileno() for f in files]
-                offs = [c * cb for c in range(n_file)] if layout == "one_file" else [0] * n_file
-                for name, fn, arg in (("store_file_" + cname, K.kdn_store_file, st_ops), ("retrieve_file_" + cname, K.kdn_retrieve_file, rt_ops)):
-                    best = None
-                    for _ in range(3):
-                        torch.cuda.synchronize()
-                        t0 = time.perf_counter()
-                        fn(ctx, pid, arg, fds, offs, s)
-                        leg.check()
-                        dt = time.perf_counter() - t0
-                        best = dt if best is None else min(best, dt)
-                    file_ops[name + "_" + layout] = {"ms": best * 1e3, "file_gbs": n_file * cb / best / 1e9, "file_bytes": n_file * cb,
-                                                     "where": "tmpfs" if tmpdir else "default temporary directory (page cache)"}
-            finally:
-                for f in files:
-                    f.close()
-    out["ops_file_not_in_value"] = file_ops
-
-    # token-delta Rice codecs (quantise, then entropy-code along tokens): how small the chunks get and how fast they are
-    # stored and decoded, on inputs whose neighbouring tokens correlate with coefficient rho (rho = 0: the ordinary
-    # uncorrelated input, the worst case for this codec).  This leg rewrites the library's source blocks, so it runs last.
-    td = {}
-    n_td = min(n_lib, 32)
-    bf16_bytes = n_td * T * E * 2
-    for rho in (0.0, 0.9, 0.99):
-        for c in range(n_td):
-            x = synth.correlated_tokens(shape, T, rho, synth.SEED_VALUES + 100 + c, dev)
-            synth.place_tokens(leg.k, leg.v, leg.d_src[c * bpc:(c + 1) * bpc].cpu().numpy(), 0, x)
-        del x
-        for codec, cname in ((INT8TD, "int8td"), (INT4TD, "int4td")):
-            cb = K.kdn_chunk_bytes(desc, T, codec)
-            lay = K.kdn_td_layout(desc, T, codec)
-            buf = torch.empty(n_td * cb, dtype=torch.uint8, device=dev)
-            st_ops = [K.XferOp(leg.d_src.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(buf.data_ptr() + c * cb, cb, T, codec)) for c in range(n_td)]
-            rt_ops = [K.XferOp(leg.d_dst.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(buf.data_ptr() + c * cb, cb, T, codec)) for c in range(n_td)]
-            reqs = [K.ComposeReq(leg.d_dst.data_ptr() + c * bpc * i32, bpc, [K.Chunk(buf.data_ptr() + c * cb, cb, T, codec, K.KDN_MEM_DEVICE, 4096)],
-                                 [0], shape.rope_theta) for c in range(n_td)]
-            ms_store = leg.timed(lambda: K.kdn_store(ctx, pid, st_ops, s), min(reps, 5), warm=2)
+    if "kc" in which:
+        # per-channel key codecs, and what they buy: the error of the stored keys, over all channels and over the channels
+        # without the x20 outlier gain
+        def key_error_db(ops_set):
+            """Retrieve chunk 0 and compare layer 0's keys with their source blocks: signal-to-noise ratio in dB."""
+            if not W["exclusive"]:
+                return None
+            K.kdn_store(ctx, pid, ops_set["store"][:1], s)
+            K.kdn_retrieve(ctx, pid, [K.XferOp(leg.d_dst.data_ptr(), bpc, 0, ops_set["store"][0].chunk)], s)
             leg.check()
-            used = sum(int(buf[c * cb + 8 * lay["segments"]:c * cb + 8 * lay["segments"] + 8].view(torch.int64).item()) for c in range(n_td))
-            ms_retr = leg.timed(lambda: K.kdn_retrieve(ctx, pid, rt_ops, s), min(reps, 5), warm=2)
-            ms_comp = leg.timed(lambda: K.kdn_compose(ctx, pid, reqs, s), min(reps, 5), warm=2)
+            x = leg.k[0][leg.d_src[:bpc].long()].float().reshape(-1, shape.row_elems)
+            y = leg.k[0][leg.d_dst[:bpc].long()].float().reshape(-1, shape.row_elems)
+            ordinary = (synth.outlier_gain(shape)[0, 0].reshape(-1) == 1).to(dev)
+            snr = lambda a, b: float(10 * torch.log10((a * a).mean() / ((a - b) ** 2).mean()))
+            return {"all_channels": snr(x, y), "ordinary_channels": snr(x[:, ordinary], y[:, ordinary])}
+
+        kc_ops = {}
+        i4q = leg.make_sets(False, codecs=(INT4,))[INT4]
+        quality = {"int4_g64": key_error_db(i4q), "int8_g64": key_error_db(dev_sets[INT8])}
+        del i4q
+        torch.cuda.empty_cache()
+        for codec, cname in ((INT8KC, "int8kc"), (INT4KC, "int4kc")):
+            kc = leg.make_sets(False, codecs=(codec,))[codec]
+            three(kc, codec, cname, kc_ops)
+            quality[cname] = key_error_db(kc)
+            del kc
+            torch.cuda.empty_cache()
+        kc_ops["stored_key_snr_db"] = quality
+        out["ops_per_channel_key_codecs_not_in_value"] = kc_ops
+
+    if "sparse" in which:
+        # keep-lists: every chunk holds a seeded random half of its span's tokens
+        sparse_ops = {}
+        rng = np.random.default_rng(synth.SEED_ASSIGN)
+        n_keep = T // 2
+        keep_np = np.stack([np.sort(rng.choice(T, n_keep, replace=False)) for _ in range(n_lib)]).astype(np.int32)
+        d_keep = torch.from_numpy(keep_np).to(dev)
+        for codec, cname in ((RAW, "raw"), (INT8, "int8"), (INT4, "int4")):
+            cb = K.kdn_chunk_bytes(desc, n_keep, codec)
+            buf = torch.empty(n_lib * cb, dtype=torch.uint8, device=dev)
+            keeps = [d_keep.data_ptr() + c * n_keep * i32 for c in range(n_lib)]
+            st_ops = [K.XferOp(leg.d_src.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(buf.data_ptr() + c * cb, cb, n_keep, codec)) for c in range(n_lib)]
+            rt_ops = [K.XferOp(leg.d_dst.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(buf.data_ptr() + c * cb, cb, n_keep, codec)) for c in range(n_lib)]
+            for name, fn, arg in (("store_sparse_" + cname, K.kdn_store_sparse, st_ops), ("retrieve_sparse_" + cname, K.kdn_retrieve_sparse, rt_ops)):
+                ms = leg.timed(lambda: fn(ctx, pid, arg, keeps, s), reps)
+                nbytes = n_lib * n_keep * E * bytes_per_elem(codec)
+                sparse_ops[name] = {"ms": ms, "gbs": nbytes / (ms * 1e-3) / 1e9, "tokens_per_s": n_lib * n_keep / (ms * 1e-3),
+                                    "kept": "%d of %d tokens per chunk, seeded random" % (n_keep, T)}
             leg.check()
-            moved = used + bf16_bytes                        # coded bytes on the chunk side, bf16 on the pool side
-            td["%s_rho_%s" % (cname, rho)] = {
-                "chunk_bytes_used": used, "bits_per_element": 8.0 * used / (n_td * T * E), "smaller_than_bf16_by": bf16_bytes / used,
-                "store_ms": ms_store, "store_gbs": moved / (ms_store * 1e-3) / 1e9,
-                "retrieve_ms": ms_retr, "retrieve_gbs": moved / (ms_retr * 1e-3) / 1e9, "retrieve_tokens_per_s": n_td * T / (ms_retr * 1e-3),
-                "compose_ms": ms_comp, "compose_gbs": moved / (ms_comp * 1e-3) / 1e9,
-                "retrieve_frac_of_8000": moved / (ms_retr * 1e-3) / 1e9 / 8000.0}
             del buf
         torch.cuda.empty_cache()
-    td["what"] = ("%d chunks x %d tokens; GB/s counts the bytes the chunks use plus the bf16 bytes on the pool side; "
-                  "rho = correlation of neighbouring tokens in the synthetic input" % (n_td, T))
-    out["ops_token_delta_rice_not_in_value"] = td
+        out["ops_keep_list_not_in_value"] = sparse_ops
+
+    if "single" in which:
+        # one chunk per call: what a single retrieve costs (CUDA events around back-to-back calls, each call another chunk
+        # of the library into its own blocks, so nothing is served from L2)
+        single_ops = {}
+        for codec, cname in ((RAW, "raw"), (INT8, "int8")):
+            ones = [K.xfer_array([op]) for op in dev_sets[codec]["retrieve"]]
+            n_calls = 2 * len(ones)
+            for arr in ones[:8]:
+                K.lib.kdn_retrieve(ctx, pid, arr, 1, s, 0)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            a.record(leg.stream)
+            for i in range(n_calls):
+                K.lib.kdn_retrieve(ctx, pid, ones[i % len(ones)], 1, s, 0)
+            b.record(leg.stream)
+            host_us = (time.perf_counter() - t0) / n_calls * 1e6
+            torch.cuda.synchronize()
+            leg.check()
+            us = a.elapsed_time(b) / n_calls * 1e3
+            nbytes = T * E * bytes_per_elem(codec)
+            single_ops["retrieve_one_chunk_" + cname] = {"us_per_call": us, "host_us_per_call_through_ctypes": host_us, "gbs": nbytes / us / 1e3,
+                                                          "frac_of_8000": nbytes / us / 1e3 / 8000.0, "tokens": T, "bytes_moved": nbytes}
+        # the same call from plain C (the example program: one raw chunk, 200 calls): host time per call without Python
+        try:
+            import re
+            import tempfile
+            from paper_2409_13761_b200 import build as _build
+            with tempfile.TemporaryDirectory() as td_:
+                exe = _build.build_example("single_chunk", td_)
+                res = subprocess.run([exe], capture_output=True, text=True, timeout=300, env=_build.example_env())
+            m = re.search(r"ok host_us=([0-9.]+) device_us=([0-9.]+) gbs=([0-9.]+)", res.stdout)
+            single_ops["from_c_example"] = ({"host_us_per_call": float(m.group(1)), "device_us_per_call": float(m.group(2)),
+                                             "gbs": float(m.group(3)), "note": "one chunk re-read every call (half of it may sit in L2)"}
+                                            if m else {"error": (res.stdout + res.stderr)[-300:]})
+        except Exception as exc:                      # no C compiler on the box: the ctypes figure stands alone
+            single_ops["from_c_example"] = {"error": str(exc)[:200]}
+        out["ops_single_chunk_not_in_value"] = single_ops
+
+    if "file" in which:
+        # file-backed chunks: a few chunks of the library written to and read back from files (wall clock around the call
+        # plus the stream sync, since the calling thread does the file I/O)
+        file_ops = {}
+        import tempfile
+        tmpdir = "/dev/shm" if os.path.isdir("/dev/shm") and os.access("/dev/shm", os.W_OK) else None
+        n_file = min(8, n_lib)
+        for codec, cname in ((RAW, "raw"), (INT8, "int8")):
+            cb = K.kdn_chunk_bytes(desc, T, codec)
+            st_ops = [K.XferOp(leg.d_src.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(0, cb, T, codec)) for c in range(n_file)]
+            rt_ops = [K.XferOp(leg.d_dst.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(0, cb, T, codec)) for c in range(n_file)]
+            for layout in ("one_file", "file_per_chunk"):
+                files = [tempfile.NamedTemporaryFile(dir=tmpdir, prefix="kdn_bench_") for _ in range(1 if layout == "one_file" else n_file)]
+                try:
+                    fds = [files[0].fileno()] * n_file if layout == "one_file" else [f.fileno() for f in files]
+                    offs = [c * cb for c in range(n_file)] if layout == "one_file" else [0] * n_file
+                    for name, fn, arg in (("store_file_" + cname, K.kdn_store_file, st_ops), ("retrieve_file_" + cname, K.kdn_retrieve_file, rt_ops)):
+                        best = None
+                        for _ in range(3):
+                            torch.cuda.synchronize()
+                            t0 = time.perf_counter()
+                            fn(ctx, pid, arg, fds, offs, s)
+                            leg.check()
+                            dt = time.perf_counter() - t0
+                            best = dt if best is None else min(best, dt)
+                        file_ops[name + "_" + layout] = {"ms": best * 1e3, "file_gbs": n_file * cb / best / 1e9, "file_bytes": n_file * cb,
+                                                         "where": "tmpfs" if tmpdir else "default temporary directory (page cache)"}
+                finally:
+                    for f in files:
+                        f.close()
+        out["ops_file_not_in_value"] = file_ops
+
+    if "td" in which:
+        # token-delta Rice codecs (quantise, then entropy-code along tokens): how small the chunks get and how fast they are
+        # stored and decoded, on inputs whose neighbouring tokens correlate with coefficient rho (rho = 0: the ordinary
+        # uncorrelated input, the worst case for this codec).  This leg rewrites the library's source blocks, so it runs last.
+        td = {}
+        n_td = min(n_lib, 32)
+        bf16_bytes = n_td * T * E * 2
+        for rho in (0.0, 0.9, 0.99):
+            for c in range(n_td):
+                x = synth.correlated_tokens(shape, T, rho, synth.SEED_VALUES + 100 + c, dev)
+                synth.place_tokens(leg.k, leg.v, leg.d_src[c * bpc:(c + 1) * bpc].cpu().numpy(), 0, x)
+            del x
+            for codec, cname in ((INT8TD, "int8td"), (INT4TD, "int4td")):
+                cb = K.kdn_chunk_bytes(desc, T, codec)
+                lay = K.kdn_td_layout(desc, T, codec)
+                buf = torch.empty(n_td * cb, dtype=torch.uint8, device=dev)
+                st_ops = [K.XferOp(leg.d_src.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(buf.data_ptr() + c * cb, cb, T, codec)) for c in range(n_td)]
+                rt_ops = [K.XferOp(leg.d_dst.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(buf.data_ptr() + c * cb, cb, T, codec)) for c in range(n_td)]
+                reqs = [K.ComposeReq(leg.d_dst.data_ptr() + c * bpc * i32, bpc, [K.Chunk(buf.data_ptr() + c * cb, cb, T, codec, K.KDN_MEM_DEVICE, 4096)],
+                                     [0], shape.rope_theta) for c in range(n_td)]
+                ms_store = leg.timed(lambda: K.kdn_store(ctx, pid, st_ops, s), min(reps, 5), warm=2)
+                leg.check()
+                used = sum(int(buf[c * cb + 8 * lay["segments"]:c * cb + 8 * lay["segments"] + 8].view(torch.int64).item()) for c in range(n_td))
+                ms_retr = leg.timed(lambda: K.kdn_retrieve(ctx, pid, rt_ops, s), min(reps, 5), warm=2)
+                ms_comp = leg.timed(lambda: K.kdn_compose(ctx, pid, reqs, s), min(reps, 5), warm=2)
+                leg.check()
+                moved = used + bf16_bytes                        # coded bytes on the chunk side, bf16 on the pool side
+                td["%s_rho_%s" % (cname, rho)] = {
+                    "chunk_bytes_used": used, "bits_per_element": 8.0 * used / (n_td * T * E), "smaller_than_bf16_by": bf16_bytes / used,
+                    "store_ms": ms_store, "store_gbs": moved / (ms_store * 1e-3) / 1e9,
+                    "retrieve_ms": ms_retr, "retrieve_gbs": moved / (ms_retr * 1e-3) / 1e9, "retrieve_tokens_per_s": n_td * T / (ms_retr * 1e-3),
+                    "compose_ms": ms_comp, "compose_gbs": moved / (ms_comp * 1e-3) / 1e9,
+                    "retrieve_frac_of_8000": moved / (ms_retr * 1e-3) / 1e9 / 8000.0}
+                del buf
+            torch.cuda.empty_cache()
+        td["what"] = ("%d chunks x %d tokens; GB/s counts the bytes the chunks use plus the bf16 bytes on the pool side; "
+                      "rho = correlation of neighbouring tokens in the synthetic input" % (n_td, T))
+        out["ops_token_delta_rice_not_in_value"] = td
     return out
 
 
@@ -731,7 +761,7 @@ def run_gpu(args) -> None:
     # ---- device-resident timing: the step `value` is measured on
     elapsed_ms, op_ms, launches, clocks = leg.time_steps(dev_sets, args.steps, args.warmup, barrier)
     reps = max(1, min(args.steps, 20))
-    extras = extras_8b(leg, dev_sets, reps)
+    extras = extras_8b(leg, dev_sets, reps, tuple(x for x in args.extras.split(",") if x))
     full = not (args.pool_blocks or args.chunks or args.parts)
     sweep_points = sweep_extract(leg, min(reps, 10)) if full and not args.no_sweep else None
 
@@ -919,6 +949,7 @@ def main() -> None:
     ap.add_argument("--e2e-steps", type=int, default=4)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true", help="skip the host-link leg (profiling runs)")
+    ap.add_argument("--extras", default=",".join(EXTRAS), help="which of the legs outside `value` to run: " + ",".join(EXTRAS))
     ap.add_argument("--no-70b", action="store_true", help="skip the llama3-70b leg of the default run")
     ap.add_argument("--no-sweep", action="store_true", help="skip the sweep extract of the default run")
     ap.add_argument("--sweep", action="store_true", help="chunk-length / block-size / codec / fragmentation sweep (1 GPU)")

@@ -34,6 +34,7 @@ constexpr int kMaxOpsPerLaunch = 4096;
 constexpr unsigned kMaxTilesPerLaunch = 0x7fff0000u;
 constexpr size_t kDefaultSlabBytes = (size_t)256 << 20;
 constexpr unsigned kTdCols = 128;           // channels per CTA of the token-delta kernels
+constexpr unsigned kKcCols = 256;           // channels per CTA of the key-plane store of the per-channel key codecs
 
 struct Pool {
     int L, H, D, bs;
@@ -191,6 +192,14 @@ kdn_status check_range(const kdn_pool_desc *p, const int32_t *table, int32_t n_t
 
 unsigned gcd_u(unsigned a, unsigned b) { while (b) { unsigned t = a % b; a = b; b = t; } return a; }
 unsigned lcm_u(unsigned a, unsigned b) { return a / gcd_u(a, b) * b; }
+
+// Make `device` current; the runtime's own switch costs a fraction of a microsecond even when nothing changes.
+kdn_status use_device(int device)
+{
+    int cur = -1;
+    if (cudaGetDevice(&cur) == cudaSuccess && cur == device) return KDN_OK;
+    return cudaSetDevice(device) == cudaSuccess ? KDN_OK : KDN_E_CUDA;
+}
 
 kdn_status ensure_side(kdn_ctx *ctx)
 {
@@ -350,8 +359,8 @@ kdn_status launch_tiles(LaunchEnv &env, int OP, int groups, int gw, unsigned gri
 {
 #define KDN_CASE(G, W)                                                                                             \
     if (groups == G && (G == 0 || gw == W)) {                                                                      \
-        if (OP == OP_STORE) return launch_kernel(env, kdn_store_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp);      \
-        if (OP == OP_RETRIEVE) return launch_kernel(env, kdn_retrieve_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp); \
+        if (OP == OP_STORE) return launch_kernel(env, kdn_store_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp, overlap);      \
+        if (OP == OP_RETRIEVE) return launch_kernel(env, kdn_retrieve_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp, overlap); \
         return launch_kernel(env, kdn_compose_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp, overlap);               \
     }
     KDN_CASE(0, 4) KDN_CASE(1, 4) KDN_CASE(2, 4) KDN_CASE(3, 4) KDN_CASE(4, 4) KDN_CASE(6, 4)
@@ -523,7 +532,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
         // key planes of the per-channel key codecs: one CTA per (64-token group, layer, op)
         // channels per CTA: at most 256 (36 KiB of shared memory, six CTAs per SM), a multiple of eight that divides the row
         unsigned n_split = 1;
-        while (row_elems / n_split > 256u && row_elems % (n_split * 2u * 8u) == 0u) n_split *= 2u;
+        while (row_elems / n_split > kKcCols && row_elems % (n_split * 2u * 8u) == 0u) n_split *= 2u;
         const unsigned cols = row_elems / n_split;
         const size_t kc_smem = kc_smem_bytes(cols);
         if (kc_smem > smem_limit) return KDN_E_UNSUPPORTED;
@@ -555,7 +564,10 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     unsigned long long want = (unsigned long long)ctx->env.sm_count * (unsigned)ctas_per_sm;
     const unsigned grid = (unsigned)(tiles < want ? tiles : want);
     const int gw = ctx->tuning.group_warps > 0 ? ctx->tuning.group_warps : def.gw;
-    kdn_status st = launch_tiles(ctx->env, OP, groups, gw, grid, smem, stream, lp, OP == OP_COMPOSE && n_rope > 0);
+    // Every launch of the pipeline is a programmatic dependent launch.  After the rotation-table kernel only the warps
+    // that read the table wait for it; otherwise every thread waits for the kernel before it, whatever that was.
+    lp.wait_all = (OP == OP_COMPOSE && n_rope > 0) ? 0 : 1;
+    kdn_status st = launch_tiles(ctx->env, OP, groups, gw, grid, smem, stream, lp, true);
     if (st != KDN_OK) return st;
     ctx->launches++;
     ctx->last.op = OP;
@@ -655,12 +667,20 @@ kdn_status launch_td(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *hops,
                 ctx->launches++;
                 tp.rope = slot->d_table;
             }
-            kdn_status r = OP == OP_COMPOSE ? ctx->env.resident(kdn_td_decode_kernel<true>, (int)threads, smem, &per_sm)
-                                            : ctx->env.resident(kdn_td_decode_kernel<false>, (int)threads, smem, &per_sm);
-            if (r != KDN_OK) return r;
-            if (per_sm < 1) return KDN_E_UNSUPPORTED;
-            if (OP == OP_COMPOSE) kdn_td_decode_kernel<true><<<grid, threads, smem, stream>>>(tp);
-            else kdn_td_decode_kernel<false><<<grid, threads, smem, stream>>>(tp);
+            kdn_status r = KDN_OK;
+#define KDN_TD_DECODE(COMPOSE, COLS)                                                                        \
+            {                                                                                               \
+                r = ctx->env.resident(kdn_td_decode_kernel<COMPOSE, COLS>, (int)threads, smem, &per_sm);    \
+                if (r != KDN_OK) return r;                                                                  \
+                if (per_sm < 1) return KDN_E_UNSUPPORTED;                                                   \
+                kdn_td_decode_kernel<COMPOSE, COLS><<<grid, threads, smem, stream>>>(tp);                   \
+            }
+            if (cols == kTdCols && threads == kTdCols) {
+                if (OP == OP_COMPOSE) KDN_TD_DECODE(true, kTdCols) else KDN_TD_DECODE(false, kTdCols)
+            } else {
+                if (OP == OP_COMPOSE) KDN_TD_DECODE(true, 0) else KDN_TD_DECODE(false, 0)
+            }
+#undef KDN_TD_DECODE
             KDN_CUDA(cudaGetLastError());
             ctx->launches++;
             if (slot) {
@@ -945,7 +965,12 @@ kdn_status xfer(kdn_ctx *ctx, int pool_id, int OP, const kdn_xfer_op *ops, int n
     const kdn_pool_desc shape = shape_of(pool);
     kdn_status st = kdn_validate_xfer(&shape, ops, n_ops);
     if (st != KDN_OK) return st;
-    if (cudaSetDevice(ctx->device) != cudaSuccess) return KDN_E_CUDA;
+    if (use_device(ctx->device) != KDN_OK) return KDN_E_CUDA;
+    if (n_ops == 1 && ops[0].chunk.mem == KDN_MEM_DEVICE && ops[0].chunk.n_tokens > 0 && !is_td(ops[0].chunk.codec)) {
+        // one device-resident chunk, the call a serving engine makes per request: no lists to build
+        const HostOp h = make_host_op(pool, ops[0].block_table, ops[0].n_table_blocks, ops[0].token_offset, ops[0].chunk);
+        return launch_batch(ctx, pool, OP, &h, 1, (cudaStream_t)cuda_stream);
+    }
     std::vector<HostOp> dev_ops, host_ops;
     for (int i = 0; i < n_ops; ++i) {
         if (ops[i].chunk.n_tokens == 0) continue;
@@ -1590,6 +1615,7 @@ extern "C" kdn_status kdn_compose_static(int device, const kdn_pool_desc *pool, 
         const unsigned grid = (unsigned)(tiles < want ? tiles : want);
         lp.wait_limit_ns = kWaitLimitNs;
         lp.rows_per_tile = 1;
+        lp.wait_all = 0;
         {
             std::lock_guard<std::mutex> lock(g_static_mutex);     // the per-device occupancy cache is shared by all callers
             st = launch_tiles(sd->env, OP_COMPOSE, def.groups, def.gw, grid, smem, stream, lp);

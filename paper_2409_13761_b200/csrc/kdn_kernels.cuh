@@ -111,6 +111,9 @@ struct Launch {
                               // before it queues the next store (see the storer loop)
     unsigned long long wait_limit_ns;   // a pipeline wait gives up after this long (the drain waits keep kWaitLimitNs)
     int rows_per_tile;        // keep-list ops: listed token rows per tile (1: one row per tile)
+    int wait_all;             // the launch may start while the kernel before it in the stream still runs (programmatic
+                              // dependent launch): every thread waits for that kernel before it touches global memory.
+                              // 0: only the warps that read the rotation table wait (the kernel before is the table kernel)
     DevOp inline_ops[kInlineOps];
 };
 
@@ -507,11 +510,14 @@ __device__ __forceinline__ void dequantise_kc_tile(const unsigned char *B, const
             f[0] = codes_to_f32x2<0>(w0, minus_bias); f[1] = codes_to_f32x2<2>(w0, minus_bias);
             f[2] = codes_to_f32x2<0>(w1, minus_bias); f[3] = codes_to_f32x2<2>(w1, minus_bias);
         }
+        // the item's eight scales as two 128-bit loads: consecutive threads are 32 bytes apart, which 128-bit loads
+        // take without a bank conflict (64-bit loads at that stride meet eight to a bank)
+        const uint4 s0 = lds128(S + ch), s1 = lds128(S + ch + 4);
         uint4 o;
-        o.x = pack_bf16x2(mul2(f[0], lds_f32x2(S + ch)));
-        o.y = pack_bf16x2(mul2(f[1], lds_f32x2(S + ch + 2)));
-        o.z = pack_bf16x2(mul2(f[2], lds_f32x2(S + ch + 4)));
-        o.w = pack_bf16x2(mul2(f[3], lds_f32x2(S + ch + 6)));
+        o.x = pack_bf16x2(mul2(f[0], pack2_bits(s0.x, s0.y)));
+        o.y = pack_bf16x2(mul2(f[1], pack2_bits(s0.z, s0.w)));
+        o.z = pack_bf16x2(mul2(f[2], pack2_bits(s1.x, s1.y)));
+        o.w = pack_bf16x2(mul2(f[3], pack2_bits(s1.z, s1.w)));
         sts128(A + (size_t)e * 2u, o);
     }
 }
@@ -589,11 +595,12 @@ __device__ __forceinline__ void rotate_tile(unsigned char *A, const unsigned cha
             }
             if (kChan) {
                 const unsigned c_lo = e_lo - (e_lo / row_elems) * row_elems, c_hi = c_lo + half;
-#pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                    u[k] = mul2(u[k], lds_f32x2(S + c_lo + 2 * k));
-                    w[k] = mul2(w[k], lds_f32x2(S + c_hi + 2 * k));
-                }
+                const uint4 a0 = lds128(S + c_lo), a1 = lds128(S + c_lo + 4);     // 128-bit loads: no bank conflicts at this stride
+                const uint4 b0 = lds128(S + c_hi), b1 = lds128(S + c_hi + 4);
+                u[0] = mul2(u[0], pack2_bits(a0.x, a0.y)); u[1] = mul2(u[1], pack2_bits(a0.z, a0.w));
+                u[2] = mul2(u[2], pack2_bits(a1.x, a1.y)); u[3] = mul2(u[3], pack2_bits(a1.z, a1.w));
+                w[0] = mul2(w[0], pack2_bits(b0.x, b0.y)); w[1] = mul2(w[1], pack2_bits(b0.z, b0.w));
+                w[2] = mul2(w[2], pack2_bits(b1.x, b1.y)); w[3] = mul2(w[3], pack2_bits(b1.z, b1.w));
             } else {
                 const float sl = S[e_lo >> 6], sh = S[e_hi >> 6];
                 const f32x2 sl2 = pack2(sl, sl), sh2 = pack2(sh, sh);
@@ -803,6 +810,9 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
     constexpr bool kCompute = kGroups > 0;
     constexpr unsigned kGT = (unsigned)kGW * 32u;           // threads of one compute group
     extern __shared__ __align__(128) unsigned char smem_raw[];
+    // The next launch of this library in the stream may be scheduled as this kernel's CTAs leave, set up its barriers
+    // and then wait (below) for this kernel to finish: back-to-back calls lose no time between kernels.
+    release_dependents();
     const Smem sm = carve(P, smem_raw);
     const int S = P.stages;
     const int tid = (int)threadIdx.x;
@@ -821,6 +831,7 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
         fence_async_smem();
     }
     __syncthreads();
+    if (P.wait_all) dependency_wait();                      // returns at once when the launch was an ordinary one
 
     const unsigned grid = gridDim.x, bid = blockIdx.x;
     const unsigned n_my = P.n_tiles > bid ? (P.n_tiles - bid + grid - 1u) / grid : 0u;

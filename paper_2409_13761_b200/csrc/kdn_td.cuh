@@ -454,13 +454,15 @@ __global__ void __launch_bounds__(512) kdn_td_encode_kernel(const __grid_constan
 // Big-endian view of a little-endian word: the stream's first byte in the top bits.
 __device__ __forceinline__ uint32_t td_be(uint32_t w) { return __byte_perm(w, 0u, 0x0123); }
 
-template <bool kCompose>
-__global__ void __launch_bounds__(512) kdn_td_decode_kernel(const __grid_constant__ TdLaunch P)
+// kCols: channels per CTA when known at compile time (the usual slice; every stride in the decoding loop is then an
+// immediate), 0: taken from the launch record.
+template <bool kCompose, unsigned kCols>
+__global__ void __launch_bounds__(kCols ? kCols : 512) kdn_td_decode_kernel(const __grid_constant__ TdLaunch P)
 {
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const TdSlice s = td_slice(P);
     if (!s.valid) return;
-    const unsigned C = P.cols, RE = P.row_elems;
+    const unsigned C = kCols ? kCols : P.cols, RE = P.row_elems;
     const int codec = s.op.codec;
     const unsigned raw_bits = (unsigned)td_raw_bits(codec);
 
@@ -526,7 +528,7 @@ __global__ void __launch_bounds__(512) kdn_td_decode_kernel(const __grid_constan
     }
     // one thread per channel: Rice, zigzag, delta -> codes
     if (tid < C) {
-        const unsigned mode_mask = (param & 8u) ? 0xffffffffu : 0u, k = param & 7u;
+        const unsigned k = param & 7u;
         // the sub-stream, as big-endian words, into column tid of the interleaved area: word j of every channel sits in
         // one row, so a warp's loads below never meet in a bank wherever each lane is in its stream
         {
@@ -545,24 +547,36 @@ __global__ void __launch_bounds__(512) kdn_td_decode_kernel(const __grid_constan
                 x0 = x1;
             }
         }
-        const uint32_t *col = I + tid;
+        // 32-bit shared addresses throughout: column tid of the interleaved words, column tid of the code tile
+        const uint32_t col = smem_u32(I) + tid * 4u, row_b = C * 4u;
+        uint32_t out = smem_u32(B) + tid;
+        const unsigned k1 = k + 1u, kpow = 1u << k, krem = 32u - k;
+        const bool delta = (param & 8u) != 0u;
         unsigned bp = 0;                                                  // bits consumed so far
         int prev = 0;
-        unsigned char *out = B + tid;
 #pragma unroll 4
         for (unsigned t = 0; t < s.n_tok; ++t) {
             const unsigned wi = (bp >> 5) < kTdWords - 2u ? (bp >> 5) : kTdWords - 2u;   // a damaged stream cannot run off the area
-            const uint32_t *wp = col + (size_t)wi * C;
-            const uint32_t hi = __funnelshift_l(wp[C], wp[0], bp);       // the next 32 bits of the stream
+            const uint32_t a = col + wi * row_b;
+            uint32_t w0, w1;
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w0) : "r"(a));
+            asm volatile("ld.shared.u32 %0, [%1];" : "=r"(w1) : "r"(a + row_b));
+            const uint32_t hi = __funnelshift_l(w1, w0, bp);             // the next 32 bits of the stream
             const unsigned ones = (unsigned)__clz((int)~hi);
-            unsigned u = (ones << k) | (((hi << (ones + 1u)) >> 1) >> (31u - k));
-            unsigned len = ones + 1u + k;
-            if (ones >= 15u) { u = (hi << 15) >> (32u - raw_bits); len = 15u + raw_bits; }
+            // quo ones, a zero, k bits: the k bits are the top of hi << (ones + 1); a shift by 32 (k = 0) gives 0 in PTX
+            unsigned rem;
+            asm("shr.b32 %0, %1, %2;" : "=r"(rem) : "r"(hi << (ones + 1u)), "r"(krem));
+            unsigned u = ones * kpow + rem;
+            unsigned len = ones + k1;
+            if (__builtin_expect(ones >= 15u, 0)) { u = (hi << 15) >> (32u - raw_bits); len = 15u + raw_bits; }   // the escape: rare
             bp += len;
-            const int e = (int)(u >> 1) ^ -(int)(u & 1u);
-            const int q = e + (prev & (int)mode_mask);
+            int sgn;
+            asm("bfe.s32 %0, %1, 0, 1;" : "=r"(sgn) : "r"(u));           // -(u & 1)
+            int q = (int)(u >> 1) ^ sgn;
+            if (delta) q += prev;
             prev = q;
-            out[(size_t)t * C] = (unsigned char)q;
+            asm volatile("st.shared.u8 [%0], %1;" :: "r"(out), "r"(q) : "memory");
+            out += C;
         }
     }
     __syncthreads();                                                      // codes complete, stream bytes no longer read
