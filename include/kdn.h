@@ -64,7 +64,11 @@
  *   the chunk uses, which is what has to be kept or sent.  kdn_chunk_bytes gives the worst-case CAPACITY (a sub-stream
  *   never exceeds 72 or 40 bytes) and chunk.bytes must equal it; bytes past seg_off[S] are not written and not read
  *   (up to 15 beyond it may be read, never past the capacity).  kdn_td_layout gives the offsets.
- *   Same restrictions as the per-channel key codecs, and KDN_MEM_DEVICE chunks only (KDN_E_UNSUPPORTED otherwise).
+ *   Same restrictions as the per-channel key codecs.  kdn_store writes KDN_MEM_DEVICE chunks only (the size of the
+ *   result is not known before the kernels have run); kdn_retrieve and kdn_compose also take KDN_MEM_PINNED_HOST
+ *   chunks: the library reads seg_off[S] from host memory and copies just the bytes in use over the host link (a
+ *   chunk whose bytes in use exceed a staging slab, or whose offset table no store can have written, is refused).
+ *   Files (kdn_*_file) are not supported.
  * Key re-rotation in kdn_compose: the stored keys of a part carry rotary
  *   position embedding for positions base_pos + t; placing the part at
  *   dst_pos rotates each pair (k[i], k[i + D/2]) of every head by

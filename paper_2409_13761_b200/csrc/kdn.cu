@@ -17,6 +17,8 @@
 #include <utility>
 #include <vector>
 
+#include <sys/mman.h>
+#include <sys/stat.h>
 #include <unistd.h>
 
 using namespace kdn;
@@ -174,7 +176,6 @@ kdn_status check_chunk(const kdn_pool_desc *p, const kdn_chunk *c)
     if (c->mem != KDN_MEM_DEVICE && c->mem != KDN_MEM_PINNED_HOST) return KDN_E_INVAL;
     if (c->codec != KDN_CODEC_RAW_BF16 && p->head_dim % 64) return KDN_E_UNSUPPORTED;
     if (c->bytes != kdn_chunk_bytes(p, c->n_tokens, c->codec)) return KDN_E_SHAPE;
-    if (is_td(c->codec) && c->mem != KDN_MEM_DEVICE) return KDN_E_UNSUPPORTED;   // variable-length chunks are not staged
     if (c->n_tokens > 0) {
         if (!c->data) return KDN_E_INVAL;
         if ((uintptr_t)c->data % 16) return KDN_E_ALIGN;
@@ -248,27 +249,56 @@ bool write_fully(int fd, const unsigned char *src, size_t bytes, long long off)
     return true;
 }
 
+// Write through a shared mapping of the file: buffered writes to ONE file take its inode lock exclusively, so
+// parallel pwrite()s queue up behind each other (measured: 5 GB/s however many threads); stores through a mapping
+// only meet at the page level.  The file must already be long enough.  False: the descriptor cannot be mapped.
+bool write_mapped(int fd, const unsigned char *src, size_t bytes, long long off)
+{
+    static const long long page = sysconf(_SC_PAGESIZE) > 0 ? sysconf(_SC_PAGESIZE) : 4096;
+    const long long a = off / page * page;
+    const size_t d = (size_t)(off - a);
+    void *m = mmap(nullptr, bytes + d, PROT_READ | PROT_WRITE, MAP_SHARED | MAP_POPULATE, fd, (off_t)a);
+    if (m == MAP_FAILED) return false;
+    std::memcpy((unsigned char *)m + d, src, bytes);
+    munmap(m, bytes + d);
+    return true;
+}
+
 // Move the file pieces among `pieces` between their files and `bounce` (write = bounce -> file).  One thread copies
 // out of the page cache at 5-6 GB/s, a tenth of the host link, so the pieces are cut into slices of kIoSlice bytes
 // and up to kIoThreads threads work through them.
 constexpr size_t kIoSlice = (size_t)4 << 20;
-constexpr unsigned kIoThreads = 8;
+constexpr unsigned kIoThreads = 16;
 bool file_io(const std::vector<Piece> &pieces, unsigned char *bounce, bool write)
 {
-    struct Slice { int fd; unsigned char *mem; size_t bytes; long long off; };
+    struct Slice { int fd; unsigned char *mem; size_t bytes; long long off; bool mapped; };
     std::vector<Slice> slices;
     for (const Piece &p : pieces) {
         if (p.host) continue;
+        bool mapped = false;
+        if (write) {
+            // a regular file is grown to its final length first (a mapping cannot reach past the end), then written
+            // through mappings; anything else (or a failure to grow) takes pwrite()
+            struct stat sb;
+            if (fstat(p.fd, &sb) == 0 && S_ISREG(sb.st_mode)) {
+                const long long end = p.file_off + (long long)p.bytes;
+                mapped = sb.st_size >= end || ftruncate(p.fd, (off_t)end) == 0;
+            }
+        }
         for (size_t o = 0; o < p.bytes; o += kIoSlice)
             slices.push_back(Slice{ p.fd, bounce + p.slab_off + o, p.bytes - o < kIoSlice ? p.bytes - o : kIoSlice,
-                                    p.file_off + (long long)o });
+                                    p.file_off + (long long)o, mapped });
     }
     std::atomic<size_t> next{ 0 };
     std::atomic<bool> ok{ true };
     auto work = [&]() {
         for (size_t i = next.fetch_add(1); i < slices.size(); i = next.fetch_add(1)) {
             const Slice &c = slices[i];
-            if (!(write ? write_fully(c.fd, c.mem, c.bytes, c.off) : read_fully(c.fd, c.mem, c.bytes, c.off))) ok = false;
+            if (write) {
+                if (!(c.mapped && write_mapped(c.fd, c.mem, c.bytes, c.off)) && !write_fully(c.fd, c.mem, c.bytes, c.off)) ok = false;
+            } else if (!read_fully(c.fd, c.mem, c.bytes, c.off)) {
+                ok = false;
+            }
         }
     };
     const unsigned n_threads = slices.size() < kIoThreads ? (unsigned)slices.size() : kIoThreads;
@@ -735,6 +765,8 @@ HostOp make_host_op(const Pool &pool, const int32_t *table, int32_t n_table, int
     h.op.nl = pool.L;
     h.op.pos_end = (long long)n_table * pool.bs;
     const size_t elems = (size_t)pool.L * 2u * (size_t)c.n_tokens * (size_t)pool.H * (size_t)pool.D;
+    if (is_td(c.codec))       // token lists do not exist for these codecs: pos_end carries the bytes the kernels may read
+        h.op.pos_end = (long long)td_layout(pool.L, (unsigned)pool.H * (unsigned)pool.D, c.n_tokens, c.codec).capacity;
     if (c.codec != KDN_CODEC_RAW_BF16 && !is_td(c.codec)) h.op.scales = (unsigned char *)c.data + (is_int4(c.codec) ? elems / 2u : elems);
     return h;
 }
@@ -880,6 +912,56 @@ size_t chunk_side_bytes(const Pool &pool, const HostOp &h)
            (size_t)h.op.nl * scales_per_layer((size_t)pool.H * (size_t)pool.D, (size_t)h.op.T, h.op.codec) * 4u;
 }
 
+// Retrieve / compose from token-delta chunks in page-locked host memory: the bytes each chunk uses (its own offset
+// table says how many) are copied into a staging slab on the side stream, as many chunks as fit, and decoded from there
+// while the next slab fills.
+kdn_status run_td_host(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector<HostOp> &hops, cudaStream_t stream, cudaStream_t side)
+{
+    kdn_status st = ensure_slabs(ctx);
+    if (st != KDN_OK) return st;
+    const unsigned row_elems = (unsigned)pool.H * (unsigned)pool.D;
+    std::vector<HostOp> batch;
+    std::vector<Piece> pieces;
+    size_t fill = 0;
+    auto flush = [&]() -> kdn_status {
+        if (batch.empty()) return KDN_OK;
+        const unsigned s = ctx->slab_next++ & 1u;
+        KDN_CUDA(cudaStreamWaitEvent(side, ctx->slab_free[s], 0));
+        for (const Piece &p : pieces)
+            KDN_CUDA(cudaMemcpyAsync(ctx->slab[s] + p.slab_off, p.host, p.bytes, cudaMemcpyHostToDevice, side));
+        KDN_CUDA(cudaEventRecord(ctx->slab_ready[s], side));
+        KDN_CUDA(cudaStreamWaitEvent(stream, ctx->slab_ready[s], 0));
+        for (HostOp &h : batch) h.op.data = ctx->slab[s] + (size_t)(uintptr_t)h.op.data;      // offsets become addresses
+        kdn_status r = launch_td(ctx, pool, OP, batch.data(), (int)batch.size(), stream);
+        if (r != KDN_OK) return r;
+        KDN_CUDA(cudaEventRecord(ctx->slab_free[s], stream));
+        batch.clear();
+        pieces.clear();
+        fill = 0;
+        return KDN_OK;
+    };
+    for (const HostOp &h : hops) {
+        const TdLayout lay = td_layout(pool.L, row_elems, h.op.T, h.op.codec);
+        const unsigned long long *seg_off = reinterpret_cast<const unsigned long long *>(h.op.data);   // host memory: readable here
+        const unsigned long long used = seg_off[lay.S];
+        bool stored = used >= lay.streams && used <= lay.capacity && !(used & 15ull) && seg_off[0] == lay.streams;
+        for (unsigned long long i = 0; stored && i < lay.S; ++i) stored = seg_off[i] <= seg_off[i + 1];
+        if (!stored) return KDN_E_SHAPE;                     // not a chunk a store has written
+        if (used > ctx->slab_bytes) return KDN_E_UNSUPPORTED;
+        if (fill + used > ctx->slab_bytes) {
+            st = flush();
+            if (st != KDN_OK) return st;
+        }
+        pieces.push_back(Piece{ h.op.data, fill, (size_t)used, -1, 0 });
+        HostOp sub = h;
+        sub.op.data = (unsigned char *)(uintptr_t)fill;      // offset inside the slab until the slab is known
+        sub.op.pos_end = (long long)used;                    // the slab holds no more of the chunk than this
+        batch.push_back(sub);
+        fill = (fill + (size_t)used + 255) & ~(size_t)255;
+    }
+    return flush();
+}
+
 kdn_status run_ops(kdn_ctx *ctx, int pool_id, int OP, std::vector<HostOp> &dev_ops, std::vector<HostOp> &host_ops,
                    void *cuda_stream, void *side_stream)
 {
@@ -891,6 +973,21 @@ kdn_status run_ops(kdn_ctx *ctx, int pool_id, int OP, std::vector<HostOp> &dev_o
         kdn_status st = ensure_side(ctx);
         if (st != KDN_OK) return st;
         side = ctx->own_side;
+    }
+    // Host-resident token-delta chunks travel whole (only the bytes they use), apart from the layer-range staging
+    std::vector<HostOp> td_host;
+    for (size_t i = 0; i < host_ops.size();) {
+        if (is_td(host_ops[i].op.codec)) { td_host.push_back(host_ops[i]); host_ops.erase(host_ops.begin() + (long)i); }
+        else ++i;
+    }
+    if (!td_host.empty()) {
+        if (OP == OP_STORE) return KDN_E_UNSUPPORTED;        // the size of the result is not known before the kernels ran
+        if (!ctx->fork) KDN_CUDA(cudaEventCreateWithFlags(&ctx->fork, cudaEventDisableTiming));
+        KDN_CUDA(cudaEventRecord(ctx->fork, stream));
+        KDN_CUDA(cudaStreamWaitEvent(side, ctx->fork, 0));
+        kdn_status st = run_td_host(ctx, pool, OP, td_host, stream, side);
+        if (st != KDN_OK) return st;
+        if (host_ops.empty()) return launch_all(ctx, pool, OP, dev_ops, stream);
     }
     // Host-resident chunks cross the link slab by slab.  The device-resident ops of the same call are cut into about
     // as many launches as there are slab hand-overs and enqueued between them, so the GPU works on them while the
@@ -1218,6 +1315,7 @@ static kdn_status xfer_file(kdn_ctx *ctx, int pool_id, int OP, const kdn_file_op
         if (st != KDN_OK) return st;
         st = check_kc(&shape, &o.chunk, o.token_offset);
         if (st != KDN_OK) return st;
+        if (is_td(o.chunk.codec)) return KDN_E_UNSUPPORTED;      // variable-length chunks are not staged through files
         if (ops[i].fd < 0 || ops[i].file_offset < 0) return KDN_E_INVAL;
     }
     if (cudaSetDevice(ctx->device) != cudaSuccess) return KDN_E_CUDA;

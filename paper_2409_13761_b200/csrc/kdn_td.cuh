@@ -500,7 +500,9 @@ __global__ void __launch_bounds__(kCols ? kCols : 512) kdn_td_decode_kernel(cons
     const unsigned shift = (unsigned)(((unsigned long long)s.op.data + src) & 15ull);
     const unsigned bytes_al = (shift + total_slice + 15u) & ~15u;
     // a damaged chunk must not send a copy outside the chunk or outside the staging area
-    const bool sane = total_slice <= C * td_max_len(codec) && src >= lay.streams && src - shift + bytes_al <= lay.capacity;
+    // (op.pos_end: the bytes of the chunk that exist at op.data -- its capacity, or what a staging slab holds of it)
+    const unsigned long long have = (unsigned long long)s.op.pos_end < lay.capacity ? (unsigned long long)s.op.pos_end : lay.capacity;
+    const bool sane = total_slice <= C * td_max_len(codec) && src >= lay.streams && src - shift + bytes_al <= have;
     if (tid == 0) {
         if (!sane) {
             atomicCAS(P.status, 0, kStatusRange);

@@ -173,7 +173,7 @@ def test_refusals_and_damaged_chunks():
         T = 64
         buf = dev.chunk_buf(T, TD8)
         for bad in (lambda: dev.store([dev.op(tab, 3, buf, T, TD8)]),                       # first token not at a block start
-                    lambda: dev.store([dev.op(tab, 0, dev.chunk_buf(T, TD8, pinned=True), T, TD8)]),   # host-resident chunk
+                    lambda: dev.store([dev.op(tab, 0, dev.chunk_buf(T, TD8, pinned=True), T, TD8)]),   # store into host memory
                     lambda: K.kdn_store_sparse(dev.ctx, dev.pool_id, [dev.op(tab, 0, buf, T, TD8)], [tab.data_ptr()], dev.stream.cuda_stream)):
             with pytest.raises(K.KdnError) as e:
                 bad()
@@ -201,5 +201,63 @@ def test_refusals_and_damaged_chunks():
         oracle.retrieve(ref, np.arange(8, dtype=np.int32) + 40, 0, T, TD8, oracle.store(host, np.arange(8, dtype=np.int32), 0, T, TD8))
         got = dev.pool_np()
         assert np.array_equal(got[:, :, 40:], ref[:, :, 40:]) and np.array_equal(got[:, :, :20], ref[:, :, :20])
+    finally:
+        dev.close()
+
+
+@pytest.mark.parametrize("codec", [TD8, TD4], ids=["int8td", "int4td"])
+def test_retrieve_and_compose_from_page_locked_host_chunks(codec):
+    """Delivery of compressed chunks (the point of coding them): token-delta chunks kept in page-locked host memory are
+    retrieved and composed; only the bytes each chunk uses cross the host link, through staging slabs that hold a few
+    chunks at a time, in a call that also carries device-resident chunks."""
+    shape = synth.TOY.with_(n_layers=3, n_kv_heads=2, head_dim=64, block_size=16, n_blocks=256)
+    perm = np.random.default_rng(12).permutation(256).astype(np.int32)
+    pool = make_pool_np(shape, perm[:40], 0, 640, 0.9, seed=77)
+    dev = Device(shape, pool_np=pool)
+    try:
+        K = dev.K
+        Ts = [200, 64, 130, 37, 256]
+        srcs, off = [], 0
+        for T in Ts:
+            nb = -(-T // 16)
+            srcs.append(perm[off:off + nb])
+            off += nb
+        wants = [oracle.store(pool, t, 0, T, codec) for t, T in zip(srcs, Ts)]
+        dbufs = [dev.chunk_buf(T, codec) for T in Ts]
+        dev.store([dev.op(dev.table(t), 0, b, T, codec) for t, b, T in zip(srcs, dbufs, Ts)])
+        assert dev.sync() == 0
+        hbufs = []
+        for b, w, T in zip(dbufs, wants, Ts):
+            used = oracle.td_used_bytes(w, 3, 2, 64, T, codec)
+            h = dev.chunk_buf(T, codec, pinned=True, fill=0x5A)
+            h[:used].copy_(b[:used])                                   # only the bytes in use are kept
+            hbufs.append(h)
+        torch.cuda.synchronize()
+        K.kdn_set_staging_bytes(dev.ctx, 512 * 1024)                      # two or three of the chunks at a time
+        dsts = [perm[60 + 20 * i:60 + 20 * i + 17] for i in range(len(Ts))]
+        ops = [dev.op(dev.table(d), 0, (hbufs[i] if i != 2 else dbufs[i]), T, codec) for i, (d, T) in enumerate(zip(dsts, Ts))]
+        dev.retrieve(ops)
+        assert dev.sync() == 0
+        ref = pool.copy()
+        for d, w, T in zip(dsts, wants, Ts):
+            oracle.retrieve(ref, d, 0, T, codec, w)
+        assert np.array_equal(dev.pool_np(), ref)
+        # compose two host-resident parts into one request, the second one re-rotated
+        rt = perm[200:230]
+        dev.compose([K.ComposeReq(dev.table(rt).data_ptr(), 30, [dev.chunk(hbufs[0], 200, codec, 0), dev.chunk(hbufs[4], 256, codec, 0)],
+                                  [0, 208], shape.rope_theta)])
+        assert dev.sync() == 0
+        kref, kmag = oracle.compose(ref, rt, [(wants[0], 200, codec, 0, 0), (wants[4], 256, codec, 0, 208)], shape.rope_theta, want_ref=True)
+        got = dev.pool_np()
+        p = 208 + np.arange(256)
+        rot = np.zeros(got.shape, dtype=bool)
+        rot[:, 0, rt[p // 16], p % 16] = True
+        assert np.array_equal(got[~rot], ref[~rot])
+        check_rotated_keys(got[:, 0, rt[p // 16], p % 16], kref[:, 208:464], kmag[:, 208:464], ref[:, 0, rt[p // 16], p % 16])
+        # a host buffer no store has written is refused, not followed
+        junk = dev.chunk_buf(64, codec, pinned=True, fill=0xFF)
+        with pytest.raises(K.KdnError) as e:
+            dev.retrieve([dev.op(dev.table(dsts[0]), 0, junk, 64, codec)])
+        assert e.value.status == K.KDN_E_SHAPE
     finally:
         dev.close()
