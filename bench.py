@@ -589,13 +589,33 @@ def extras_8b(leg, dev_sets, reps, which=EXTRAS):
                 ms_retr = leg.timed(lambda: K.kdn_retrieve(ctx, pid, rt_ops, s), min(reps, 5), warm=2)
                 ms_comp = leg.timed(lambda: K.kdn_compose(ctx, pid, reqs, s), min(reps, 5), warm=2)
                 leg.check()
+                # delivery from page-locked host memory: the chunks packed back to back, only their bytes in use (wall
+                # clock around the call and the status read, as in the end-to-end leg)
+                useds = [int(buf[c * cb + 8 * lay["segments"]:c * cb + 8 * lay["segments"] + 8].view(torch.int64).item()) for c in range(n_td)]
+                starts = np.concatenate([[0], np.cumsum([(u + 255) // 256 * 256 for u in useds])])
+                arena = torch.empty(int(starts[-1]), dtype=torch.uint8).pin_memory()
+                for c in range(n_td):
+                    arena[int(starts[c]):int(starts[c]) + useds[c]].copy_(buf[c * cb:c * cb + useds[c]])
+                torch.cuda.synchronize()
+                h_ops = [K.XferOp(leg.d_dst.data_ptr() + c * bpc * i32, bpc, 0,
+                                  K.Chunk(arena.data_ptr() + int(starts[c]), cb, T, codec, K.KDN_MEM_PINNED_HOST)) for c in range(n_td)]
+                K.kdn_retrieve(ctx, pid, h_ops, s)
+                leg.check()
+                t0 = time.perf_counter()
+                for _ in range(3):
+                    K.kdn_retrieve(ctx, pid, h_ops, s)
+                    leg.check()
+                host_ms = (time.perf_counter() - t0) / 3 * 1e3
+                del arena
                 moved = used + bf16_bytes                        # coded bytes on the chunk side, bf16 on the pool side
                 td["%s_rho_%s" % (cname, rho)] = {
                     "chunk_bytes_used": used, "bits_per_element": 8.0 * used / (n_td * T * E), "smaller_than_bf16_by": bf16_bytes / used,
                     "store_ms": ms_store, "store_gbs": moved / (ms_store * 1e-3) / 1e9,
                     "retrieve_ms": ms_retr, "retrieve_gbs": moved / (ms_retr * 1e-3) / 1e9, "retrieve_tokens_per_s": n_td * T / (ms_retr * 1e-3),
                     "compose_ms": ms_comp, "compose_gbs": moved / (ms_comp * 1e-3) / 1e9,
-                    "retrieve_frac_of_8000": moved / (ms_retr * 1e-3) / 1e9 / 8000.0}
+                    "retrieve_frac_of_8000": moved / (ms_retr * 1e-3) / 1e9 / 8000.0,
+                    "from_host_ms": host_ms, "from_host_link_gbs": used / (host_ms * 1e-3) / 1e9,
+                    "from_host_bf16_gbs_delivered": bf16_bytes / (host_ms * 1e-3) / 1e9}
                 del buf
             torch.cuda.empty_cache()
         td["what"] = ("%d chunks x %d tokens; GB/s counts the bytes the chunks use plus the bf16 bytes on the pool side; "

@@ -249,45 +249,44 @@ bool write_fully(int fd, const unsigned char *src, size_t bytes, long long off)
     return true;
 }
 
-// Write through a shared mapping of the file: buffered writes to ONE file take its inode lock exclusively, so
-// parallel pwrite()s queue up behind each other (measured: 5 GB/s however many threads); stores through a mapping
-// only meet at the page level.  The file must already be long enough.  False: the descriptor cannot be mapped.
-bool write_mapped(int fd, const unsigned char *src, size_t bytes, long long off)
-{
-    static const long long page = sysconf(_SC_PAGESIZE) > 0 ? sysconf(_SC_PAGESIZE) : 4096;
-    const long long a = off / page * page;
-    const size_t d = (size_t)(off - a);
-    void *m = mmap(nullptr, bytes + d, PROT_READ | PROT_WRITE, MAP_SHARED | MAP_POPULATE, fd, (off_t)a);
-    if (m == MAP_FAILED) return false;
-    std::memcpy((unsigned char *)m + d, src, bytes);
-    munmap(m, bytes + d);
-    return true;
-}
-
 // Move the file pieces among `pieces` between their files and `bounce` (write = bounce -> file).  One thread copies
 // out of the page cache at 5-6 GB/s, a tenth of the host link, so the pieces are cut into slices of kIoSlice bytes
 // and up to kIoThreads threads work through them.
+// Writes go through a shared mapping of the file where that is possible: buffered writes to ONE file take its inode
+// lock exclusively, so parallel pwrite()s queue up behind each other (measured: 5 GB/s however many threads), while
+// stores through a mapping only meet at the page level.  Each piece is mapped once by the calling thread and unmapped
+// once after the workers are done (an unmap per slice made every worker interrupt all the others to flush their
+// address translations).  A regular file is grown to its final length first: a mapping cannot reach past the end.
 constexpr size_t kIoSlice = (size_t)4 << 20;
 constexpr unsigned kIoThreads = 16;
 bool file_io(const std::vector<Piece> &pieces, unsigned char *bounce, bool write)
 {
-    struct Slice { int fd; unsigned char *mem; size_t bytes; long long off; bool mapped; };
+    static const long long page = sysconf(_SC_PAGESIZE) > 0 ? sysconf(_SC_PAGESIZE) : 4096;
+    struct Slice { int fd; unsigned char *mem; size_t bytes; long long off; unsigned char *mapped; };
+    struct Mapping { void *base; size_t bytes; };
     std::vector<Slice> slices;
+    std::vector<Mapping> mappings;
     for (const Piece &p : pieces) {
         if (p.host) continue;
-        bool mapped = false;
+        unsigned char *mapped = nullptr;                     // where the piece's first byte sits in the mapping, if any
         if (write) {
-            // a regular file is grown to its final length first (a mapping cannot reach past the end), then written
-            // through mappings; anything else (or a failure to grow) takes pwrite()
             struct stat sb;
             if (fstat(p.fd, &sb) == 0 && S_ISREG(sb.st_mode)) {
                 const long long end = p.file_off + (long long)p.bytes;
-                mapped = sb.st_size >= end || ftruncate(p.fd, (off_t)end) == 0;
+                if (sb.st_size >= end || ftruncate(p.fd, (off_t)end) == 0) {
+                    const long long a = p.file_off / page * page;
+                    const size_t d = (size_t)(p.file_off - a);
+                    void *m = mmap(nullptr, p.bytes + d, PROT_READ | PROT_WRITE, MAP_SHARED, p.fd, (off_t)a);
+                    if (m != MAP_FAILED) {
+                        mappings.push_back(Mapping{ m, p.bytes + d });
+                        mapped = (unsigned char *)m + d;
+                    }
+                }
             }
         }
         for (size_t o = 0; o < p.bytes; o += kIoSlice)
             slices.push_back(Slice{ p.fd, bounce + p.slab_off + o, p.bytes - o < kIoSlice ? p.bytes - o : kIoSlice,
-                                    p.file_off + (long long)o, mapped });
+                                    p.file_off + (long long)o, mapped ? mapped + o : nullptr });
     }
     std::atomic<size_t> next{ 0 };
     std::atomic<bool> ok{ true };
@@ -295,7 +294,8 @@ bool file_io(const std::vector<Piece> &pieces, unsigned char *bounce, bool write
         for (size_t i = next.fetch_add(1); i < slices.size(); i = next.fetch_add(1)) {
             const Slice &c = slices[i];
             if (write) {
-                if (!(c.mapped && write_mapped(c.fd, c.mem, c.bytes, c.off)) && !write_fully(c.fd, c.mem, c.bytes, c.off)) ok = false;
+                if (c.mapped) std::memcpy(c.mapped, c.mem, c.bytes);
+                else if (!write_fully(c.fd, c.mem, c.bytes, c.off)) ok = false;
             } else if (!read_fully(c.fd, c.mem, c.bytes, c.off)) {
                 ok = false;
             }
@@ -308,6 +308,7 @@ bool file_io(const std::vector<Piece> &pieces, unsigned char *bounce, bool write
     }
     work();
     for (std::thread &t : helpers) t.join();
+    for (const Mapping &m : mappings) munmap(m.base, m.bytes);
     return ok;
 }
 

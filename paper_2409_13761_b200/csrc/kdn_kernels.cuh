@@ -491,16 +491,28 @@ __device__ __forceinline__ f32x2 lds_f32x2(const float *p)
 
 // Decode a key tile of a per-channel key codec: n codes at B (whole token rows of row_elems channels), one scale per
 // channel at S, bf16 to A.  One item is 8 consecutive channels of one token.
-template <bool kInt4>
+// kKeep: keep a thread's eight scales in registers from item to item (not in the compose kernels, whose rotation
+// path already fills their register budget).
+template <bool kInt4, bool kKeep = true>
 __device__ __forceinline__ void dequantise_kc_tile(const unsigned char *B, const float *S, unsigned char *A,
                                                    unsigned n, unsigned row_elems, int ct, unsigned gthreads)
 {
     const unsigned nitems = n >> 3;
     const f32x2 minus_bias = pack2(-8388736.0f, -8388736.0f);
     const f32x2 minus_bias4 = pack2(-8388616.0f, -8388616.0f);
+    // A thread's items are gthreads * 8 elements apart; where that is a whole number of rows (1024-element rows, four
+    // warps) every item of the thread has the same eight channels, and their scales are loaded once, not once per item.
+    unsigned have_ch = 0xffffffffu;
+    f32x2 sc[4];
     for (unsigned v = (unsigned)ct; v < nitems; v += gthreads) {
         const unsigned e = v << 3;
         const unsigned ch = e - (e / row_elems) * row_elems;
+        if (!kKeep || ch != have_ch) {
+            const uint4 s0 = lds128(S + ch), s1 = lds128(S + ch + 4);
+            sc[0] = pack2_bits(s0.x, s0.y); sc[1] = pack2_bits(s0.z, s0.w);
+            sc[2] = pack2_bits(s1.x, s1.y); sc[3] = pack2_bits(s1.z, s1.w);
+            have_ch = ch;
+        }
         f32x2 f[4];
         if (kInt4) {
             nibbles_to_f32x2(*reinterpret_cast<const uint32_t *>(B + (e >> 1)), minus_bias4, f);
@@ -510,14 +522,11 @@ __device__ __forceinline__ void dequantise_kc_tile(const unsigned char *B, const
             f[0] = codes_to_f32x2<0>(w0, minus_bias); f[1] = codes_to_f32x2<2>(w0, minus_bias);
             f[2] = codes_to_f32x2<0>(w1, minus_bias); f[3] = codes_to_f32x2<2>(w1, minus_bias);
         }
-        // the item's eight scales as two 128-bit loads: consecutive threads are 32 bytes apart, which 128-bit loads
-        // take without a bank conflict (64-bit loads at that stride meet eight to a bank)
-        const uint4 s0 = lds128(S + ch), s1 = lds128(S + ch + 4);
         uint4 o;
-        o.x = pack_bf16x2(mul2(f[0], pack2_bits(s0.x, s0.y)));
-        o.y = pack_bf16x2(mul2(f[1], pack2_bits(s0.z, s0.w)));
-        o.z = pack_bf16x2(mul2(f[2], pack2_bits(s1.x, s1.y)));
-        o.w = pack_bf16x2(mul2(f[3], pack2_bits(s1.z, s1.w)));
+        o.x = pack_bf16x2(mul2(f[0], sc[0]));
+        o.y = pack_bf16x2(mul2(f[1], sc[1]));
+        o.z = pack_bf16x2(mul2(f[2], sc[2]));
+        o.w = pack_bf16x2(mul2(f[3], sc[3]));
         sts128(A + (size_t)e * 2u, o);
     }
 }
@@ -595,8 +604,8 @@ __device__ __forceinline__ void rotate_tile(unsigned char *A, const unsigned cha
             }
             if (kChan) {
                 const unsigned c_lo = e_lo - (e_lo / row_elems) * row_elems, c_hi = c_lo + half;
-                const uint4 a0 = lds128(S + c_lo), a1 = lds128(S + c_lo + 4);     // 128-bit loads: no bank conflicts at this stride
-                const uint4 b0 = lds128(S + c_hi), b1 = lds128(S + c_hi + 4);
+                const uint4 a0 = lds128(S + c_lo), a1 = lds128(S + c_lo + 4);     // 128-bit loads: two lanes to a bank at worst
+                const uint4 b0 = lds128(S + c_hi), b1 = lds128(S + c_hi + 4);     // (kept per item: caching sixteen scales spills)
                 u[0] = mul2(u[0], pack2_bits(a0.x, a0.y)); u[1] = mul2(u[1], pack2_bits(a0.z, a0.w));
                 u[2] = mul2(u[2], pack2_bits(a1.x, a1.y)); u[3] = mul2(u[3], pack2_bits(a1.z, a1.w));
                 w[0] = mul2(w[0], pack2_bits(b0.x, b0.y)); w[1] = mul2(w[1], pack2_bits(b0.z, b0.w));
@@ -1028,9 +1037,9 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                             if (flags & TF_INT4) rotate_tile<2, true>(A, B, Sc, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct, kGT, P.row_elems);
                             else rotate_tile<1, true>(A, B, Sc, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct, kGT, P.row_elems);
                         } else if (flags & TF_INT4) {
-                            dequantise_kc_tile<true>(B, Sc, A, n, P.row_elems, ct, kGT);
+                            dequantise_kc_tile<true, OP != OP_COMPOSE>(B, Sc, A, n, P.row_elems, ct, kGT);
                         } else {
-                            dequantise_kc_tile<false>(B, Sc, A, n, P.row_elems, ct, kGT);
+                            dequantise_kc_tile<false, OP != OP_COMPOSE>(B, Sc, A, n, P.row_elems, ct, kGT);
                         }
                     } else if (OP == OP_COMPOSE && (flags & TF_ROTATE)) {
                         if (flags & TF_INT4) rotate_tile<2>(A, B, Sc, n, (unsigned)P.D, P.rope, sm.desc[st].rope, rc, ct, kGT);

@@ -59,10 +59,12 @@ __host__ __device__ inline TdLayout td_layout(int L, unsigned row_elems, int T, 
 
 // Shared memory of the store kernels: token rows, slice maxima, reciprocals, the stream staging area (encode only),
 // small per-warp scratch, barrier.
+// (the plan kernel keeps a table of code-word lengths in place of the staging area: 512 symbols x 8 parameters x 16 bits)
+constexpr unsigned kTdCostEntries = 512;
 __host__ __device__ inline size_t td_store_smem_bytes(unsigned cols, bool encode)
 {
     return (size_t)64 * cols * 2u + (size_t)kKcSlices * cols * 2u + (size_t)cols * 4u +
-           (encode ? (size_t)cols * 72u + 32u : 0u) + 256u + 16u;
+           (encode ? (size_t)cols * 72u + 32u : (size_t)kTdCostEntries * 16u) + 256u + 16u;
 }
 // Shared memory of the decode kernel: the slice's stream bytes as they lie in the chunk, the same sub-streams
 // interleaved word by word (so that the 32 lanes of a warp read 32 different banks), codes, scales, offsets, barrier.
@@ -85,7 +87,7 @@ __device__ __forceinline__ unsigned td_cost(unsigned u, unsigned k, unsigned esc
     const unsigned quo = u >> k;
     return quo < 15u ? quo + 1u + k : esc_bits;
 }
-__device__ __forceinline__ unsigned td_zigzag(int e) { return e >= 0 ? 2u * (unsigned)e : 2u * (unsigned)(-e) - 1u; }
+__device__ __forceinline__ unsigned td_zigzag(int e) { return ((unsigned)e << 1) ^ (unsigned)(e >> 31); }   // 2e, or -2e - 1 for e < 0
 
 // round_half_even(x * inv) as the low byte of the sum with 1.5 * 2^23: two separately rounded fp32 operations.
 __device__ __forceinline__ int td_code(unsigned short x_bf16, float inv)
@@ -249,7 +251,8 @@ __global__ void __launch_bounds__(512) kdn_td_plan_kernel(const __grid_constant_
     unsigned char *X = smem_raw;
     unsigned char *pmax = X + (size_t)64 * C * 2u;
     float *inv = reinterpret_cast<float *>(pmax + (size_t)kKcSlices * C * 2u);
-    unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(reinterpret_cast<unsigned char *>(inv) + (size_t)C * 4u + 256u);
+    uint4 *cost = reinterpret_cast<uint4 *>(reinterpret_cast<unsigned char *>(inv) + (size_t)C * 4u);   // [symbol]: 8 lengths x 16 bits
+    unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(reinterpret_cast<unsigned char *>(cost) + (size_t)kTdCostEntries * 16u + 256u);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bar_mem + 1);
     const uint32_t bar = smem_u32(bar_mem);
     const unsigned tid = threadIdx.x;
@@ -265,6 +268,14 @@ __global__ void __launch_bounds__(512) kdn_td_plan_kernel(const __grid_constant_
         if (!td_load_slice(X, bar, base, s.op.table, s.op.off + (long long)(s.g << 6), s.n_tok, P.bs, P.n_blocks, RE, C, s.c0,
                            P.n_split == 1u, P.status) && tid == 0)
             *abort_flag = 1;
+    }
+    // while the rows are on their way: the length of every symbol's code word under every parameter, k = 0 .. 7 as
+    // eight 16-bit fields (a sub-stream's total stays below 2^16, so whole words can be added up field by field)
+    for (unsigned u = tid; u < kTdCostEntries; u += blockDim.x) {
+        unsigned c[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) c[k] = td_cost(u, (unsigned)k, esc_bits);
+        cost[u] = make_uint4(c[0] | (c[1] << 16), c[2] | (c[3] << 16), c[4] | (c[5] << 16), c[6] | (c[7] << 16));
     }
     __syncthreads();
     if (*abort_flag) return;
@@ -284,17 +295,17 @@ __global__ void __launch_bounds__(512) kdn_td_plan_kernel(const __grid_constant_
     // one thread per channel: the cost in bits of every (mode, k), then the first minimum
     for (unsigned ch = tid; ch < C; ch += blockDim.x) {
         const float iv = inv[ch];
-        unsigned b0[8], b1[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) { b0[k] = 0u; b1[k] = 0u; }
+        uint4 a0 = make_uint4(0u, 0u, 0u, 0u), a1 = a0;                     // mode 0 / mode 1 totals, packed like the table
         int prev = 0;
         for (unsigned t = 0; t < s.n_tok; ++t) {
             const int q = td_code(*reinterpret_cast<const unsigned short *>(X + ((size_t)t * C + ch) * 2u), iv);
-            const unsigned u0 = td_zigzag(q), u1 = td_zigzag(q - prev);
+            const uint4 c0 = cost[td_zigzag(q)], c1 = cost[td_zigzag(q - prev)];      // symbols are at most 4 * 127 < 512
             prev = q;
-#pragma unroll
-            for (int k = 0; k < 8; ++k) { b0[k] += td_cost(u0, (unsigned)k, esc_bits); b1[k] += td_cost(u1, (unsigned)k, esc_bits); }
+            a0.x += c0.x; a0.y += c0.y; a0.z += c0.z; a0.w += c0.w;
+            a1.x += c1.x; a1.y += c1.y; a1.z += c1.z; a1.w += c1.w;
         }
+        const unsigned b0[8] = { a0.x & 0xffffu, a0.x >> 16, a0.y & 0xffffu, a0.y >> 16, a0.z & 0xffffu, a0.z >> 16, a0.w & 0xffffu, a0.w >> 16 };
+        const unsigned b1[8] = { a1.x & 0xffffu, a1.x >> 16, a1.y & 0xffffu, a1.y >> 16, a1.z & 0xffffu, a1.z >> 16, a1.w & 0xffffu, a1.w >> 16 };
         unsigned best = b0[0], param = 0u;
 #pragma unroll
         for (int k = 1; k < 8; ++k) if (b0[k] < best) { best = b0[k]; param = (unsigned)k; }
@@ -588,7 +599,7 @@ __global__ void __launch_bounds__(kCols ? kCols : 512) kdn_td_decode_kernel(cons
         rc.rope = -1; rc.col = 0xffffffffu;
         rotate_tile<1, true>(A, B, Sc, n, (unsigned)P.D, P.rope, s.op.rope, rc, (int)tid, blockDim.x, C);
     } else {
-        dequantise_kc_tile<false>(B, Sc, A, n, C, (int)tid, blockDim.x);
+        dequantise_kc_tile<false, !kCompose>(B, Sc, A, n, C, (int)tid, blockDim.x);
     }
     fence_async_smem();
     __syncthreads();
