@@ -59,12 +59,13 @@ __host__ __device__ inline TdLayout td_layout(int L, unsigned row_elems, int T, 
 
 // Shared memory of the store kernels: token rows, slice maxima, reciprocals, the stream staging area (encode only),
 // small per-warp scratch, barrier.
-// (the plan kernel keeps a table of code-word lengths in place of the staging area: 512 symbols x 8 parameters x 16 bits)
-constexpr unsigned kTdCostEntries = 512;
+// (the plan kernel keeps two tables of code-word lengths in place of the staging area, each replicated so that the
+// lanes of a warp never meet in a bank: 64 entries x 32 copies x 4 bytes and 64 entries x 16 copies x 8 bytes)
+constexpr unsigned kTdCostBytes = 64u * 32u * 4u + 64u * 16u * 8u + 64u * 4u + 64u * 8u;   // the copies, and one set of entries to copy from
 __host__ __device__ inline size_t td_store_smem_bytes(unsigned cols, bool encode)
 {
     return (size_t)64 * cols * 2u + (size_t)kKcSlices * cols * 2u + (size_t)cols * 4u +
-           (encode ? (size_t)cols * 72u + 32u : (size_t)kTdCostEntries * 16u) + 256u + 16u;
+           (encode ? (size_t)cols * 72u + 32u : (size_t)kTdCostBytes) + 256u + 16u;
 }
 // Shared memory of the decode kernel: the slice's stream bytes as they lie in the chunk, the same sub-streams
 // interleaved word by word (so that the 32 lanes of a warp read 32 different banks), codes, scales, offsets, barrier.
@@ -88,6 +89,9 @@ __device__ __forceinline__ unsigned td_cost(unsigned u, unsigned k, unsigned esc
     return quo < 15u ? quo + 1u + k : esc_bits;
 }
 __device__ __forceinline__ unsigned td_zigzag(int e) { return ((unsigned)e << 1) ^ (unsigned)(e >> 31); }   // 2e, or -2e - 1 for e < 0
+
+// Big-endian view of a little-endian word: the stream's first byte in the top bits.
+__device__ __forceinline__ uint32_t td_be(uint32_t w) { return __byte_perm(w, 0u, 0x0123); }
 
 // round_half_even(x * inv) as the low byte of the sum with 1.5 * 2^23: two separately rounded fp32 operations.
 __device__ __forceinline__ int td_code(unsigned short x_bf16, float inv)
@@ -251,8 +255,11 @@ __global__ void __launch_bounds__(512) kdn_td_plan_kernel(const __grid_constant_
     unsigned char *X = smem_raw;
     unsigned char *pmax = X + (size_t)64 * C * 2u;
     float *inv = reinterpret_cast<float *>(pmax + (size_t)kKcSlices * C * 2u);
-    uint4 *cost = reinterpret_cast<uint4 *>(reinterpret_cast<unsigned char *>(inv) + (size_t)C * 4u);   // [symbol]: 8 lengths x 16 bits
-    unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(reinterpret_cast<unsigned char *>(cost) + (size_t)kTdCostEntries * 16u + 256u);
+    // code-word lengths as 8-bit fields.  lo[min(u, 60)][lane]: k = 0, 1, 2 (from u = 60 on all three are the escape);
+    // hi[u >> 3][lane / 2]: k = 3 .. 7 (their quotients are functions of u >> 3).  One copy per lane / pair of lanes.
+    uint32_t *lo_tab = reinterpret_cast<uint32_t *>(reinterpret_cast<unsigned char *>(inv) + (size_t)C * 4u);
+    uint2 *hi_tab = reinterpret_cast<uint2 *>(lo_tab + 64u * 32u);
+    unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(reinterpret_cast<unsigned char *>(lo_tab) + (size_t)kTdCostBytes + 256u);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bar_mem + 1);
     const uint32_t bar = smem_u32(bar_mem);
     const unsigned tid = threadIdx.x;
@@ -269,13 +276,22 @@ __global__ void __launch_bounds__(512) kdn_td_plan_kernel(const __grid_constant_
                            P.n_split == 1u, P.status) && tid == 0)
             *abort_flag = 1;
     }
-    // while the rows are on their way: the length of every symbol's code word under every parameter, k = 0 .. 7 as
-    // eight 16-bit fields (a sub-stream's total stays below 2^16, so whole words can be added up field by field)
-    for (unsigned u = tid; u < kTdCostEntries; u += blockDim.x) {
-        unsigned c[8];
-#pragma unroll
-        for (int k = 0; k < 8; ++k) c[k] = td_cost(u, (unsigned)k, esc_bits);
-        cost[u] = make_uint4(c[0] | (c[1] << 16), c[2] | (c[3] << 16), c[4] | (c[5] << 16), c[6] | (c[7] << 16));
+    // while the rows are on their way: fill the tables -- every entry is worked out once, then copied
+    {
+        uint32_t *lo_one = reinterpret_cast<uint32_t *>(hi_tab + 64u * 16u);
+        uint2 *hi_one = reinterpret_cast<uint2 *>(lo_one + 64u);
+        for (unsigned i = tid; i < 128u; i += blockDim.x) {
+            if (i < 64u) {
+                lo_one[i] = td_cost(i, 0u, esc_bits) | (td_cost(i, 1u, esc_bits) << 8) | (td_cost(i, 2u, esc_bits) << 16);
+            } else {
+                const unsigned u = (i - 64u) << 3;
+                hi_one[i - 64u] = make_uint2(td_cost(u, 3u, esc_bits) | (td_cost(u, 4u, esc_bits) << 8) | (td_cost(u, 5u, esc_bits) << 16) |
+                                             (td_cost(u, 6u, esc_bits) << 24), td_cost(u, 7u, esc_bits));
+            }
+        }
+        __syncthreads();
+        for (unsigned i = tid; i < 64u * 32u; i += blockDim.x) lo_tab[i] = lo_one[i >> 5];
+        for (unsigned i = tid; i < 64u * 16u; i += blockDim.x) hi_tab[i] = hi_one[i >> 4];
     }
     __syncthreads();
     if (*abort_flag) return;
@@ -292,20 +308,37 @@ __global__ void __launch_bounds__(512) kdn_td_plan_kernel(const __grid_constant_
     const TdLayout lay = td_layout(P.L, RE, s.op.T, codec);
     const unsigned long long row = (unsigned long long)s.seg * RE + s.c0;
     td_channel_scales(X, pmax, inv, reinterpret_cast<float *>(s.op.data + lay.scales) + row, s.n_tok, C, qmax);
-    // one thread per channel: the cost in bits of every (mode, k), then the first minimum
+    // one thread per channel: the cost in bits of every (mode, k), then the first minimum.  Lengths are at most 24, so
+    // the 8-bit fields hold eight symbols' worth; after every eight symbols they are spread into 16-bit fields.
     for (unsigned ch = tid; ch < C; ch += blockDim.x) {
         const float iv = inv[ch];
-        uint4 a0 = make_uint4(0u, 0u, 0u, 0u), a1 = a0;                     // mode 0 / mode 1 totals, packed like the table
+        const uint32_t *lo_l = lo_tab + (tid & 31u);
+        const uint2 *hi_l = hi_tab + ((tid & 31u) >> 1);
+        unsigned w02[2] = { 0u, 0u }, w1[2] = { 0u, 0u }, w35[2] = { 0u, 0u }, w46[2] = { 0u, 0u }, w7[2] = { 0u, 0u };
         int prev = 0;
-        for (unsigned t = 0; t < s.n_tok; ++t) {
-            const int q = td_code(*reinterpret_cast<const unsigned short *>(X + ((size_t)t * C + ch) * 2u), iv);
-            const uint4 c0 = cost[td_zigzag(q)], c1 = cost[td_zigzag(q - prev)];      // symbols are at most 4 * 127 < 512
-            prev = q;
-            a0.x += c0.x; a0.y += c0.y; a0.z += c0.z; a0.w += c0.w;
-            a1.x += c1.x; a1.y += c1.y; a1.z += c1.z; a1.w += c1.w;
+        for (unsigned t0 = 0; t0 < s.n_tok; t0 += 8u) {
+            unsigned al[2] = { 0u, 0u }, ah[2] = { 0u, 0u };
+            const unsigned t1 = t0 + 8u < s.n_tok ? t0 + 8u : s.n_tok;
+            for (unsigned t = t0; t < t1; ++t) {
+                const int q = td_code(*reinterpret_cast<const unsigned short *>(X + ((size_t)t * C + ch) * 2u), iv);
+                const unsigned u[2] = { td_zigzag(q), td_zigzag(q - prev) };        // at most 4 * 127 < 512
+                prev = q;
+#pragma unroll
+                for (int m = 0; m < 2; ++m) {
+                    al[m] += lo_l[(u[m] < 60u ? u[m] : 60u) << 5];
+                    const uint2 h = hi_l[(u[m] >> 3) << 4];
+                    ah[m] += h.x;
+                    w7[m] += h.y;
+                }
+            }
+#pragma unroll
+            for (int m = 0; m < 2; ++m) {
+                w02[m] += al[m] & 0x00ff00ffu; w1[m] += (al[m] >> 8) & 0x00ff00ffu;
+                w35[m] += ah[m] & 0x00ff00ffu; w46[m] += (ah[m] >> 8) & 0x00ff00ffu;
+            }
         }
-        const unsigned b0[8] = { a0.x & 0xffffu, a0.x >> 16, a0.y & 0xffffu, a0.y >> 16, a0.z & 0xffffu, a0.z >> 16, a0.w & 0xffffu, a0.w >> 16 };
-        const unsigned b1[8] = { a1.x & 0xffffu, a1.x >> 16, a1.y & 0xffffu, a1.y >> 16, a1.z & 0xffffu, a1.z >> 16, a1.w & 0xffffu, a1.w >> 16 };
+        const unsigned b0[8] = { w02[0] & 0xffffu, w1[0] & 0xffffu, w02[0] >> 16, w35[0] & 0xffffu, w46[0] & 0xffffu, w35[0] >> 16, w46[0] >> 16, w7[0] };
+        const unsigned b1[8] = { w02[1] & 0xffffu, w1[1] & 0xffffu, w02[1] >> 16, w35[1] & 0xffffu, w46[1] & 0xffffu, w35[1] >> 16, w46[1] >> 16, w7[1] };
         unsigned best = b0[0], param = 0u;
 #pragma unroll
         for (int k = 1; k < 8; ++k) if (b0[k] < best) { best = b0[k]; param = (unsigned)k; }
@@ -420,28 +453,40 @@ __global__ void __launch_bounds__(512) kdn_td_encode_kernel(const __grid_constan
         }
         return;
     }
-    td_channel_scales(X, pmax, inv, nullptr, s.n_tok, C, qmax);
+    // the staging area starts out as zeros: sub-streams are OR-ed into it a 32-bit word at a time, since the first and
+    // the last word of a sub-stream also hold bits of its neighbours
+    for (unsigned i = tid; i < (C * 72u + 32u) / 16u; i += blockDim.x) sts128(stage + (size_t)i * 16u, make_uint4(0u, 0u, 0u, 0u));
+    td_channel_scales(X, pmax, inv, nullptr, s.n_tok, C, qmax);                 // (its barriers also publish the zeros)
     if (tid < C) {
         const unsigned param = s.op.data[lay.params + row + s.c0 + tid];
-        const unsigned mode = param >> 3, k = param & 7u;
+        const bool delta = (param & 8u) != 0u;
+        const unsigned k = param & 7u, kmask = (1u << k) - 1u, k1 = k + 1u;
         const float iv = inv[tid];
-        unsigned char *out = stage + shift + my_off;
+        const uint32_t addr = smem_u32(stage) + shift + my_off;          // first byte of the sub-stream
+        uint32_t wp = addr & ~3u;                                         // the word it starts in ...
+        unsigned nb = (addr & 3u) * 8u;                                   // ... after this many bits that are not its own
         unsigned long long acc = 0;
-        unsigned nb = 0, pos = 0;
         int prev = 0;
         for (unsigned t = 0; t < s.n_tok; ++t) {
             const int q = td_code(*reinterpret_cast<const unsigned short *>(X + ((size_t)t * C + tid) * 2u), iv);
-            const unsigned u = td_zigzag(mode ? q - prev : q);
+            const unsigned u = td_zigzag(delta ? q - prev : q);
             prev = q;
             const unsigned quo = u >> k;
-            unsigned w, len;
-            if (quo < 15u) { w = (((1u << quo) - 1u) << (k + 1u)) | (u & ((1u << k) - 1u)); len = quo + 1u + k; }
-            else { w = (0x7fffu << raw_bits) | u; len = 15u + raw_bits; }
+            unsigned w = (((1u << quo) - 1u) << k1) | (u & kmask), len = quo + k1;
+            if (__builtin_expect(quo >= 15u, 0)) { w = (0x7fffu << raw_bits) | u; len = 15u + raw_bits; }
             acc = (acc << len) | w;
             nb += len;
-            while (nb >= 8u && pos < my_len) { out[pos++] = (unsigned char)(acc >> (nb - 8u)); nb -= 8u; }
+            if (nb >= 32u) {                                              // a full word: bytes in stream order, first byte lowest
+                nb -= 32u;
+                const uint32_t word = td_be((uint32_t)(acc >> nb));
+                asm volatile("red.shared.or.b32 [%0], %1;" :: "r"(wp), "r"(word) : "memory");
+                wp += 4u;
+            }
         }
-        if (nb > 0u && pos < my_len) out[pos++] = (unsigned char)(acc << (8u - nb));
+        if (nb > 0u) {
+            const uint32_t word = td_be((uint32_t)(acc << (32u - nb)));
+            asm volatile("red.shared.or.b32 [%0], %1;" :: "r"(wp), "r"(word) : "memory");
+        }
     }
     // the last slice of a segment also writes the zero bytes that pad the segment to 16
     unsigned pad = 0;
@@ -462,8 +507,6 @@ __global__ void __launch_bounds__(512) kdn_td_encode_kernel(const __grid_constan
 
 // ----------------------------------------------------------------------------------- retrieve / compose --
 
-// Big-endian view of a little-endian word: the stream's first byte in the top bits.
-__device__ __forceinline__ uint32_t td_be(uint32_t w) { return __byte_perm(w, 0u, 0x0123); }
 
 // kCols: channels per CTA when known at compile time (the usual slice; every stride in the decoding loop is then an
 // immediate), 0: taken from the launch record.
