@@ -251,3 +251,79 @@ def test_8b_sweep_points_block_size_32_longest_and_shortest_chunks(run_blocks):
         dev.close()
         del dev
         torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("codec", [oracle.INT8_TD64, oracle.INT4_TD64], ids=["int8td", "int4td"])
+def test_8b_token_delta_store_and_retrieve_16_chunks_of_512_tokens(codec):
+    """The token-delta Rice codecs at the 8B shape, in the batched calls the benchmark times, on token-correlated input:
+    the bytes in use of every chunk are consistent (offset table monotone, 16-byte aligned, equal to the lengths' sums),
+    sampled chunks and layers equal the oracle's segment for segment (scales, lengths, parameters, streams), and the
+    retrieved blocks equal the oracle's; blocks that are no destination keep their bits."""
+    need_gib(50)
+    shape = synth.LLAMA3_8B
+    dev = Device(shape)
+    try:
+        K = dev.K
+        n_req, T, bs = 16, 512, shape.block_size
+        nb = T // bs
+        L, H, D = shape.n_layers, shape.n_kv_heads, shape.head_dim
+        R, G = H * D, T // 64
+        src = synth.make_table(n_req * nb, shape.n_blocks, 1, synth.SEED_TABLES).reshape(n_req, nb)
+        dst = synth.make_table(n_req * nb, shape.n_blocks, 1, synth.SEED_TABLES + 1, exclude=src.reshape(-1)).reshape(n_req, nb)
+        for i in range(n_req):                                               # neighbouring tokens correlate (rho 0.9 / 0.99)
+            synth.place_tokens(dev.k, dev.v, src[i], 0, synth.correlated_tokens(shape, T, 0.9 if i % 2 else 0.99, 500 + i, dev.dev))
+        d_src, d_dst = dev.table(src.reshape(-1)), dev.table(dst.reshape(-1))
+        cb = K.kdn_chunk_bytes(dev.desc, T, codec)
+        lay = K.kdn_td_layout(dev.desc, T, codec)
+        S = lay["segments"]
+        big = torch.full((n_req * cb,), 0xA5, dtype=torch.uint8, device=dev.dev)
+        st = [K.XferOp(d_src.data_ptr() + i * nb * 4, nb, 0, K.Chunk(big.data_ptr() + i * cb, cb, T, codec)) for i in range(n_req)]
+        rt = [K.XferOp(d_dst.data_ptr() + i * nb * 4, nb, 0, K.Chunk(big.data_ptr() + i * cb, cb, T, codec)) for i in range(n_req)]
+        before = block_sums(dev)
+        dev.store(st)
+        assert dev.sync() == 0
+        assert torch.equal(block_sums(dev), before)
+        dev.retrieve(rt)
+        assert dev.sync() == 0
+        after = block_sums(dev)
+        keep = torch.ones(shape.n_blocks, dtype=torch.bool, device=dev.dev)
+        keep[torch.from_numpy(dst.reshape(-1).astype(np.int64)).to(dev.dev)] = False
+        assert torch.equal(after[:, keep], before[:, keep])
+        layers = [0, 17, 31]
+        total_used = 0
+        for i in range(n_req):
+            head = to_np(big[i * cb:i * cb + lay["streams_offset"]])
+            seg_off = head[:8 * (S + 1)].view(np.uint64).astype(np.int64)
+            lens = head[lay["lens_offset"]:lay["params_offset"]].reshape(S, R)
+            sizes = (lens.astype(np.int64).sum(axis=1) + 15) // 16 * 16
+            assert seg_off[0] == lay["streams_offset"] and np.array_equal(np.diff(seg_off), sizes)
+            assert lens.max() <= (72 if codec == oracle.INT8_TD64 else 40)
+            total_used += int(seg_off[S])
+            assert torch.all(big[i * cb + int(seg_off[S]):(i + 1) * cb] == 0xA5)       # nothing past the bytes in use
+            if i not in (0, 7, 15):
+                continue
+            sp = dev.pool_np(src[i], layers)
+            want = oracle.store(sp, np.arange(nb, dtype=np.int32), 0, T, codec)
+            wl = oracle.td_layout(len(layers), H, D, T, codec)
+            w_off = want[:8 * (wl["segments"] + 1)].view(np.uint64).astype(np.int64)
+            got = to_np(big[i * cb:i * cb + int(seg_off[S])])
+            for j, l in enumerate(layers):
+                for kv in range(2):
+                    for g in range(G):
+                        s_full, s_sub = (2 * l + kv) * G + g, (2 * j + kv) * G + g
+                        for region, width in (("scales", 4), ("lens", 1), ("params", 1)):
+                            a = got[lay[region + "_offset"] + s_full * R * width:lay[region + "_offset"] + (s_full + 1) * R * width]
+                            b = want[wl[region] + s_sub * R * width:wl[region] + (s_sub + 1) * R * width]
+                            assert np.array_equal(a, b), (i, l, kv, g, region)
+                        n = int(w_off[s_sub + 1] - w_off[s_sub])
+                        assert n == int(seg_off[s_full + 1] - seg_off[s_full])
+                        assert np.array_equal(got[seg_off[s_full]:seg_off[s_full] + n], want[w_off[s_sub]:w_off[s_sub] + n]), (i, l, kv, g)
+            ref = np.zeros_like(sp)
+            oracle.retrieve(ref, np.arange(nb, dtype=np.int32), 0, T, codec, want)
+            assert np.array_equal(dev.pool_np(dst[i], layers), ref), (codec, i)
+        bits = 8.0 * total_used / (n_req * T * shape.elems_per_token)
+        assert bits < (8.0 if codec == oracle.INT8_TD64 else 3.8)              # correlated input: smaller than the fixed-rate code
+    finally:
+        dev.close()
+        del dev
+        torch.cuda.empty_cache()
