@@ -1113,7 +1113,8 @@ struct KcLaunch {
     DevOp inline_ops[kInlineOps];
 };
 
-constexpr unsigned kKcSlices = 4;                          // token slices of 16 tokens in pass 1 and pass 2
+constexpr unsigned kKcSlices = 4;                          // token slices in pass 1 and pass 2
+constexpr unsigned kKcTok = 64u / kKcSlices;              // tokens per slice
 __host__ __device__ inline size_t kc_smem_bytes(unsigned cols)
 {
     return (size_t)64 * cols * 2u + (size_t)kKcSlices * cols * 2u + (size_t)cols * 4u + 16u;
@@ -1216,7 +1217,7 @@ __global__ void __launch_bounds__(512) kdn_store_kc_kernel(const __grid_constant
     // pass 1: per (eight channels, token slice) the largest magnitudes, as packed bf16 pairs
     for (unsigned it = (unsigned)tid; it < items; it += (unsigned)nthreads) {
         const unsigned q = it / octets, o = it - q * octets;
-        const unsigned ta = q * 16u, tb = ta + 16u < n_tok ? ta + 16u : n_tok;
+        const unsigned ta = q * kKcTok, tb = ta + kKcTok < n_tok ? ta + kKcTok : n_tok;
         uint32_t m0 = 0u, m1 = 0u, m2 = 0u, m3 = 0u;
         for (unsigned t = ta; t < tb; ++t) {
             const uint4 x = lds128(X + ((size_t)t * C + (size_t)o * 8u) * 2u);
@@ -1249,7 +1250,7 @@ __global__ void __launch_bounds__(512) kdn_store_kc_kernel(const __grid_constant
     const unsigned long long plane_elem = ((unsigned long long)li * 2ull * (unsigned long long)op.T + t0) * RE + c0;   // K plane, token t0
     for (unsigned it = (unsigned)tid; it < items; it += (unsigned)nthreads) {
         const unsigned q = it / octets, o = it - q * octets;
-        const unsigned ta = q * 16u, tb = ta + 16u < n_tok ? ta + 16u : n_tok;
+        const unsigned ta = q * kKcTok, tb = ta + kKcTok < n_tok ? ta + kKcTok : n_tok;
         const f32x2 i0 = lds_f32x2(inv + o * 8u), i1 = lds_f32x2(inv + o * 8u + 2u);
         const f32x2 i2 = lds_f32x2(inv + o * 8u + 4u), i3 = lds_f32x2(inv + o * 8u + 6u);
         for (unsigned t = ta; t < tb; ++t) {

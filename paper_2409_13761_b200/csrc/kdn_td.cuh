@@ -190,7 +190,7 @@ __device__ __forceinline__ void td_channel_scales(const unsigned char *X, unsign
     const unsigned octets = C >> 3, items = octets * kKcSlices;
     for (unsigned it = tid; it < items; it += nthreads) {
         const unsigned q = it / octets, o = it - q * octets;
-        const unsigned ta = q * 16u, tb = ta + 16u < n_tok ? ta + 16u : n_tok;
+        const unsigned ta = q * kKcTok, tb = ta + kKcTok < n_tok ? ta + kKcTok : n_tok;
         uint32_t m0 = 0u, m1 = 0u, m2 = 0u, m3 = 0u;
         for (unsigned t = ta; t < tb; ++t) {
             const uint4 x = lds128(X + ((size_t)t * C + (size_t)o * 8u) * 2u);
