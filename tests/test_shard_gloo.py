@@ -68,7 +68,8 @@ def test_two_gloo_ranks_shard_chunks_without_any_exchange(tmp_path):
         assert np.array_equal(ch, oracle.store(pool, tab, 0, 8, oracle.INT8_G64))
 
 
-@pytest.mark.parametrize("codec", [oracle.RAW_BF16, oracle.INT8_G64, oracle.INT4_G64, oracle.INT8_KC64, oracle.INT4_KC64])
+@pytest.mark.parametrize("codec", [oracle.RAW_BF16, oracle.INT8_G64, oracle.INT4_G64, oracle.INT8_KC64, oracle.INT4_KC64,
+                                   oracle.INT8_TD64, oracle.INT4_TD64])
 def test_head_sharded_ranks_reproduce_the_unsharded_result(codec):
     """Tensor-parallel sharding: each rank stores and retrieves its own heads with an ordinary descriptor; put side by
     side along the head axis, the ranks' pools equal the pool of the unsharded retrieve (no exchange step)."""
