@@ -855,6 +855,22 @@ def run_gpu(args) -> None:
                 per_op["sweep_min_" + name] = [round(worst[name + "_gbs"], 1), round(worst[name + "_gbs"] / 8000.0, 4),
                                                "T=%d bs=%d %s" % (worst["chunk_tokens"], worst["block_size"], worst["codec"])]
             per_op["sweep_points"] = len(sweep_points)
+        # the widenings of the 8B leg in the same compact form (outside `value`)
+        wide = {}
+        for key in ("ops_int4_not_in_value", "ops_per_channel_key_codecs_not_in_value", "ops_keep_list_not_in_value"):
+            for n, v in (extras.get(key) or {}).items():
+                if isinstance(v, dict) and "gbs" in v:
+                    wide[n] = [round(v["gbs"], 1), round(v["gbs"] / 8000.0, 4)]
+        for n, v in (extras.get("ops_single_chunk_not_in_value") or {}).items():
+            if isinstance(v, dict) and "gbs" in v:
+                wide[n] = [round(v["gbs"], 1), round(v["gbs"] / 8000.0, 4)]
+        for n, v in (extras.get("ops_token_delta_rice_not_in_value") or {}).items():
+            if isinstance(v, dict) and "retrieve_gbs" in v:
+                wide["td_" + n] = {"x_smaller": round(v["smaller_than_bf16_by"], 2), "store": round(v["store_gbs"], 1),
+                                   "retrieve": round(v["retrieve_gbs"], 1), "compose": round(v["compose_gbs"], 1),
+                                   "host_bf16_gbs": round(v["from_host_bf16_gbs_delivered"], 1)}
+        if wide:
+            per_op["widenings_8b"] = wide
         frac = gbs[top] / peak
         rec = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

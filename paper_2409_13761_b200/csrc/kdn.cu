@@ -438,6 +438,14 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     if (kc_decode) unit = lcm_u(unit, row_elems);
     Shape def = default_shape(OP, any_coded, any_rot);
     if (kc_decode) def = Shape{ 16384, 4, 2, 1, 1 };      // larger tiles: a key tile also loads a whole row of scales
+    if (!compute && !any_list) {
+        // a small copy launch (one chunk per call) is mostly pipeline fill and drain: half-size tiles in six slots start
+        // storing sooner and end on a shorter tail (one 512-token 8B chunk: 24.8 -> 24.2 us); batched launches keep the
+        // larger tiles, which are worth 1 % there
+        unsigned long long bytes = 0;
+        for (int i = 0; i < n; ++i) bytes += (unsigned long long)hops[i].op.nl * 4ull * (unsigned long long)hops[i].op.T * row_elems;
+        if (bytes / 32768ull < 48ull * (unsigned long long)ctx->env.sm_count) def = Shape{ 16384, 6, 1, 0, 2 };
+    }
     int tile_bytes = ctx->tuning.tile_bytes > 0 ? ctx->tuning.tile_bytes : def.tile_bytes;
     unsigned tile_elems = (unsigned)tile_bytes / 2u / unit * unit;
     if (tile_elems < unit) tile_elems = unit;
