@@ -614,6 +614,11 @@ def extras_8b(leg, dev_sets, reps, which=EXTRAS):
                     "retrieve_ms": ms_retr, "retrieve_gbs": moved / (ms_retr * 1e-3) / 1e9, "retrieve_tokens_per_s": n_td * T / (ms_retr * 1e-3),
                     "compose_ms": ms_comp, "compose_gbs": moved / (ms_comp * 1e-3) / 1e9,
                     "retrieve_frac_of_8000": moved / (ms_retr * 1e-3) / 1e9 / 8000.0,
+                    # the decoder is bound by the integer ALU pipe, not by HBM: 148 SMs x 4 schedulers x one ALU-pipe
+                    # instruction every other cycle x 1.965 GHz x 32 lanes, at about 20 such operations per symbol
+                    "retrieve_roofline": {"bound": "alu", "unit": "symbols/s", "achieved": n_td * T * E / (ms_retr * 1e-3),
+                                          "peak": 148 * 4 * 0.5 * 1.965e9 * 32 / 20.0,
+                                          "frac": n_td * T * E / (ms_retr * 1e-3) / (148 * 4 * 0.5 * 1.965e9 * 32 / 20.0)},
                     "from_host_ms": host_ms, "from_host_link_gbs": used / (host_ms * 1e-3) / 1e9,
                     "from_host_bf16_gbs_delivered": bf16_bytes / (host_ms * 1e-3) / 1e9}
                 del buf

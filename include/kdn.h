@@ -90,7 +90,9 @@
  * cuda_stream wait for its device-to-host copies.  An event recorded on
  * cuda_stream after kdn_store therefore covers the bytes in host memory, and a
  * host chunk filled by a copy on cuda_stream can be retrieved without a host
- * synchronisation in between.
+ * synchronisation in between.  (The library's kernels let a kernel that is launched behind them with CUDA's
+ * programmatic stream serialisation start early; such a kernel has to call cudaGridDependencySynchronize before it
+ * reads what the call wrote.  Ordinary launches, copies, events and synchronisations are ordered as usual.)
  *
  * ----------------------------------------------------------------- errors --
  * Argument errors are returned at once and nothing is enqueued.  Otherwise a
