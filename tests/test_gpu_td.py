@@ -254,6 +254,19 @@ def test_retrieve_and_compose_from_page_locked_host_chunks(codec):
         rot[:, 0, rt[p // 16], p % 16] = True
         assert np.array_equal(got[~rot], ref[~rot])
         check_rotated_keys(got[:, 0, rt[p // 16], p % 16], kref[:, 208:464], kmag[:, 208:464], ref[:, 0, rt[p // 16], p % 16])
+        # layer-wise delivery of a host-resident chunk (every step brings the chunk's bytes over again: correct, not fast)
+        before = dev.pool_np()
+        lw = perm[232:249]
+        K.kdn_retrieve_layerwise(dev.ctx, dev.pool_id, [dev.op(dev.table(lw), 0, hbufs[3], Ts[3], codec)], 2, dev.stream.cuda_stream)
+        assert dev.sync() == 0
+        oracle.retrieve(before, lw, 0, Ts[3], codec, wants[3])
+        assert np.array_equal(dev.pool_np(), before)
+        # files are not a home for these chunks
+        import tempfile
+        with tempfile.TemporaryFile() as tf:
+            with pytest.raises(K.KdnError) as e:
+                K.kdn_retrieve_file(dev.ctx, dev.pool_id, [dev.op(dev.table(lw), 0, dbufs[3], Ts[3], codec)], [tf.fileno()], [0], dev.stream.cuda_stream)
+            assert e.value.status == K.KDN_E_UNSUPPORTED
         # a host buffer no store has written is refused, not followed
         junk = dev.chunk_buf(64, codec, pinned=True, fill=0xFF)
         with pytest.raises(K.KdnError) as e:
