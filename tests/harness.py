@@ -94,7 +94,7 @@ def bf16_ulp_distance(a_bits: np.ndarray, b_bits: np.ndarray) -> np.ndarray:
     return np.abs(key(a_bits) - key(b_bits))
 
 
-def check_rotated_keys(got_bits: np.ndarray, kref: np.ndarray, kmag: np.ndarray, oracle_bits: np.ndarray):
+def check_rotated_keys(got_bits: np.ndarray, kref: np.ndarray, kmag: np.ndarray, oracle_bits: np.ndarray, min_equal=0.995):
     """Tolerance for re-rotated keys.
 
     |got - ref64| <= 2^-8 |ref64| + 2^-21 (|u| + |w|): one bf16 ulp relative to the fp64 result, plus a
@@ -115,5 +115,5 @@ def check_rotated_keys(got_bits: np.ndarray, kref: np.ndarray, kmag: np.ndarray,
     solid = np.abs(kref) >= 2.0 ** -12 * kmag
     assert d[solid].max(initial=0) <= 1, "rotated key differs from the rounded fp64 result by %d bf16 steps" % int(d[solid].max())
     frac_equal = float((d == 0).mean())
-    assert frac_equal > 0.995, "only %.4f of rotated keys equal the rounded fp64 result" % frac_equal
+    assert frac_equal > min_equal, "only %.4f of rotated keys equal the rounded fp64 result" % frac_equal
     return frac_equal
