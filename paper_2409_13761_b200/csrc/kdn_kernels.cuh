@@ -114,6 +114,9 @@ struct Launch {
     int wait_all;             // the launch may start while the kernel before it in the stream still runs (programmatic
                               // dependent launch): every thread waits for that kernel before it touches global memory.
                               // 0: only the warps that read the rotation table wait (the kernel before is the table kernel)
+    float one;                // 1.0f, as a launch parameter: the coding loops form "product + constant" as
+                              // fma(product, one, constant), and with a multiplier the assembler cannot see there
+                              // is nothing it could contract with the multiply before it (the codecs round twice)
     DevOp inline_ops[kInlineOps];
 };
 
@@ -310,11 +313,22 @@ __device__ __forceinline__ f32x2 fma2(f32x2 a, f32x2 b, f32x2 c)
 }
 // p + c with its own rounding when p is a product.  The assembler contracts a packed multiply whose only
 // use is a packed add into one fused multiply-add (measured: it does so even though both carry .rn, unlike
-// the scalar forms), which would round x * inv + c once instead of twice.  Written as fma(p, 1, c) the sum
-// is the same correctly rounded p + c and there is nothing left to contract.
+// the scalar forms), which would round x * inv + c once instead of twice.  Written as fma(p, one, c) with
+// one = 1.0f arriving as a launch parameter the sum is the same correctly rounded p + c, and a multiplier
+// whose value the assembler does not know leaves it nothing to contract (with a literal 1.0f it folded the
+// multiply away again in one of the kernels: codes at exact ties came out one step off).
 __device__ __forceinline__ f32x2 add2_unfused(f32x2 p, f32x2 c, f32x2 one) { return fma2(p, one, c); }
 // The two bf16 halves of w as a packed fp32 pair (exact).
 __device__ __forceinline__ f32x2 bf16x2_to_f32x2(uint32_t w) { return pack2_bits(w << 16, w & 0xffff0000u); }
+// The same through the mixed-precision add of sm_100 (bf16 + fp32 -> fp32; x + (-0) = x for every x, signed zeros and
+// subnormals included): the widening leaves the integer pipe, which the coding loops load most.
+__device__ __forceinline__ f32x2 bf16x2_widen(uint32_t w)
+{
+    f32x2 d;
+    asm("{ .reg .b16 l, h; .reg .f32 fl, fh; mov.b32 {l, h}, %1; add.rn.f32.bf16 fl, l, %2; add.rn.f32.bf16 fh, h, %2;"
+        " mov.b64 %0, {fl, fh}; }" : "=l"(d) : "r"(w), "f"(-0.0f));
+    return d;
+}
 // max(|a|, |b|) on both bf16 halves; the sign of the result is meaningless.
 __device__ __forceinline__ uint32_t maxabs_bf16x2(uint32_t a, uint32_t b)
 {
@@ -323,15 +337,29 @@ __device__ __forceinline__ uint32_t maxabs_bf16x2(uint32_t a, uint32_t b)
     return d;
 }
 
-// Rounding trick used by quantise_tile: round_half_even(x * inv) is the low byte of the fp32 sum of the
-// (already rounded) product with 1.5 * 2^23.  For |x * inv| < 2^22 the adder itself rounds the sum to an
-// integer, ties to even, and the low mantissa bits are the two's-complement integer.  The product and the
-// sum are two separately rounded fp32 operations, as the codec's definition requires.
-__device__ __forceinline__ uint32_t pack_codes4(uint32_t r0, uint32_t r1, uint32_t r2, uint32_t r3)
+// Rounding trick used by quantise_tile: round_half_even(x * inv) sits in the low mantissa bits of the fp32 sum of the
+// (already rounded) product with 1.5 * 2^23 + bias.  For |x * inv| < 2^22 the adder itself rounds the sum to an
+// integer, ties to even (the bias is even, so ties fall the same way), and the mantissa holds code + bias.  The
+// product and the sum are two separately rounded fp32 operations, as the codec's definition requires.
+// Codes are then gathered in the floating-point pipe, exactly: with r = M + bias + code (M = 1.5 * 2^23) of two
+// element pairs, (r_b - M) * 256 + r_a = M + (code_a + bias) + 256 (code_b + bias) in each half, no carries since
+// 0 < code + bias < 256.  For int8 (bias 128) one byte permute interleaves the two halves' 16-bit fields and one XOR
+// takes the bias off; for int4 (bias 8) the odd half is added in shifted by one nibble first.
+__device__ __forceinline__ f32x2 gather2(f32x2 ra, f32x2 rb, f32x2 minus_m, f32x2 k256)
 {
-    uint32_t a = __byte_perm(r0, r1, 0x0040);             // r0.b0, r1.b0
-    uint32_t b = __byte_perm(r2, r3, 0x0040);
-    return __byte_perm(a, b, 0x5410);
+    return fma2(add2(rb, minus_m), k256, ra);
+}
+__device__ __forceinline__ uint32_t codes4_from(f32x2 t)        // int8: t = gather2 of pairs (0,1) and (2,3)
+{
+    uint32_t lo, hi;
+    unpack2_bits(t, lo, hi);
+    return __byte_perm(lo, hi, 0x5140) ^ 0x80808080u;
+}
+__device__ __forceinline__ uint32_t nibbles4_from(f32x2 t)      // int4: four nibbles in the low 16 bits, biased
+{
+    uint32_t lo, hi;
+    unpack2_bits(t, lo, hi);
+    return hi * 16u + lo;
 }
 // Encode n elements (a multiple of 64) of bf16 at A into int8 codes at B and one fp32 scale per 64
 // elements (to shared S, or straight to global when the destination is not 16-byte aligned).
@@ -341,7 +369,7 @@ __device__ __forceinline__ uint32_t pack_codes4(uint32_t r0, uint32_t r1, uint32
 // kInt4: codes in [-7, 7], two per byte (element 2k in the low nibble), 16 bytes per lane instead of 32.
 template <bool kInt4>
 __device__ __forceinline__ void quantise_tile(const unsigned char *A, unsigned char *B, float *S, float *g_scales,
-                                              unsigned n, int ct, unsigned gthreads)
+                                              unsigned n, int ct, unsigned gthreads, float one)
 {
     const float qmax = kInt4 ? 7.0f : 127.0f;
     const unsigned nhalf = n >> 5;                         // 32-element half groups
@@ -376,27 +404,26 @@ __device__ __forceinline__ void quantise_tile(const unsigned char *A, unsigned c
         scale = ok ? scale : 0.0f;
         if (act) {
             const f32x2 inv2 = pack2(inv, inv);
-            const f32x2 magic2 = pack2(12582912.0f, 12582912.0f);
-            const f32x2 one2 = pack2(1.0f, 1.0f);
+            const float magic = 12582912.0f + (kInt4 ? 8.0f : 128.0f);
+            const f32x2 magic2 = pack2(magic, magic);
+            const f32x2 minus_m2 = pack2(-12582912.0f, -12582912.0f);
+            const f32x2 k256 = pack2(256.0f, 256.0f);
+            const f32x2 one2 = pack2(one, one);
             unsigned char *dst = B + (size_t)h * (kInt4 ? 16u : 32u);
             uint32_t nib[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-                // per pair: one rounded product, one rounded sum with 1.5 * 2^23 (see above)
-                uint32_t r[8];
-                unpack2_bits(add2_unfused(mul2(bf16x2_to_f32x2(x[j].x), inv2), magic2, one2), r[0], r[1]);
-                unpack2_bits(add2_unfused(mul2(bf16x2_to_f32x2(x[j].y), inv2), magic2, one2), r[2], r[3]);
-                unpack2_bits(add2_unfused(mul2(bf16x2_to_f32x2(x[j].z), inv2), magic2, one2), r[4], r[5]);
-                unpack2_bits(add2_unfused(mul2(bf16x2_to_f32x2(x[j].w), inv2), magic2, one2), r[6], r[7]);
-                uint2 q;
-                q.x = pack_codes4(r[0], r[1], r[2], r[3]);
-                q.y = pack_codes4(r[4], r[5], r[6], r[7]);
+                // per pair: one rounded product, one rounded sum with 1.5 * 2^23 + bias (see above)
+                const f32x2 r01 = add2_unfused(mul2(bf16x2_widen(x[j].x), inv2), magic2, one2);
+                const f32x2 r23 = add2_unfused(mul2(bf16x2_widen(x[j].y), inv2), magic2, one2);
+                const f32x2 r45 = add2_unfused(mul2(bf16x2_widen(x[j].z), inv2), magic2, one2);
+                const f32x2 r67 = add2_unfused(mul2(bf16x2_widen(x[j].w), inv2), magic2, one2);
+                const f32x2 ta = gather2(r01, r23, minus_m2, k256), tb = gather2(r45, r67, minus_m2, k256);
                 if (kInt4) {
-                    // low nibbles of the eight code bytes -> four bytes: byte k = code 2k | code 2k+1 << 4
-                    const uint32_t t0 = q.x & 0x0f0f0f0fu, t1 = q.y & 0x0f0f0f0fu;
-                    nib[j] = __byte_perm(t0 | (t0 >> 4), t1 | (t1 >> 4), 0x6420);
+                    // byte k = code 2k | code 2k+1 << 4
+                    nib[j] = __byte_perm(nibbles4_from(ta), nibbles4_from(tb), 0x5410) ^ 0x88888888u;
                 } else {
-                    sts64(dst + (((unsigned)j + rot) & 3u) * 8u, q);
+                    sts64(dst + (((unsigned)j + rot) & 3u) * 8u, make_uint2(codes4_from(ta), codes4_from(tb)));
                 }
             }
             if (kInt4) {
@@ -1018,11 +1045,11 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                         // that size (no loop, no tail predicates): about a quarter fewer instructions
                         constexpr unsigned kOnePass = kGT * 32u;
                         if (flags & TF_INT4) {
-                            if (n == kOnePass) quantise_tile<true>(A, B, Sc, gs, kOnePass, ct, kGT);
-                            else quantise_tile<true>(A, B, Sc, gs, n, ct, kGT);
+                            if (n == kOnePass) quantise_tile<true>(A, B, Sc, gs, kOnePass, ct, kGT, P.one);
+                            else quantise_tile<true>(A, B, Sc, gs, n, ct, kGT, P.one);
                         } else {
-                            if (n == kOnePass) quantise_tile<false>(A, B, Sc, gs, kOnePass, ct, kGT);
-                            else quantise_tile<false>(A, B, Sc, gs, n, ct, kGT);
+                            if (n == kOnePass) quantise_tile<false>(A, B, Sc, gs, kOnePass, ct, kGT, P.one);
+                            else quantise_tile<false>(A, B, Sc, gs, n, ct, kGT, P.one);
                         }
                         computed = true;
                     }
@@ -1110,6 +1137,7 @@ struct KcLaunch {
     unsigned cols;            // channels per CTA
     unsigned n_split;         // row_elems / cols
     int *status;
+    float one;                // 1.0f (see Launch::one)
     DevOp inline_ops[kInlineOps];
 };
 
@@ -1245,8 +1273,11 @@ __global__ void __launch_bounds__(512) kdn_store_kc_kernel(const __grid_constant
     }
     __syncthreads();
     // pass 2: codes
-    const f32x2 magic2 = pack2(12582912.0f, 12582912.0f);
-    const f32x2 one2 = pack2(1.0f, 1.0f);
+    const float magic = 12582912.0f + (int4 ? 8.0f : 128.0f);
+    const f32x2 magic2 = pack2(magic, magic);
+    const f32x2 minus_m2 = pack2(-12582912.0f, -12582912.0f);
+    const f32x2 k256 = pack2(256.0f, 256.0f);
+    const f32x2 one2 = pack2(P.one, P.one);
     const unsigned long long plane_elem = ((unsigned long long)li * 2ull * (unsigned long long)op.T + t0) * RE + c0;   // K plane, token t0
     for (unsigned it = (unsigned)tid; it < items; it += (unsigned)nthreads) {
         const unsigned q = it / octets, o = it - q * octets;
@@ -1255,21 +1286,16 @@ __global__ void __launch_bounds__(512) kdn_store_kc_kernel(const __grid_constant
         const f32x2 i2 = lds_f32x2(inv + o * 8u + 4u), i3 = lds_f32x2(inv + o * 8u + 6u);
         for (unsigned t = ta; t < tb; ++t) {
             const uint4 x = lds128(X + ((size_t)t * C + (size_t)o * 8u) * 2u);
-            uint32_t r[8];
-            unpack2_bits(add2_unfused(mul2(bf16x2_to_f32x2(x.x), i0), magic2, one2), r[0], r[1]);
-            unpack2_bits(add2_unfused(mul2(bf16x2_to_f32x2(x.y), i1), magic2, one2), r[2], r[3]);
-            unpack2_bits(add2_unfused(mul2(bf16x2_to_f32x2(x.z), i2), magic2, one2), r[4], r[5]);
-            unpack2_bits(add2_unfused(mul2(bf16x2_to_f32x2(x.w), i3), magic2, one2), r[6], r[7]);
-            uint2 c;
-            c.x = pack_codes4(r[0], r[1], r[2], r[3]);
-            c.y = pack_codes4(r[4], r[5], r[6], r[7]);
+            const f32x2 r01 = add2_unfused(mul2(bf16x2_widen(x.x), i0), magic2, one2);
+            const f32x2 r23 = add2_unfused(mul2(bf16x2_widen(x.y), i1), magic2, one2);
+            const f32x2 r45 = add2_unfused(mul2(bf16x2_widen(x.z), i2), magic2, one2);
+            const f32x2 r67 = add2_unfused(mul2(bf16x2_widen(x.w), i3), magic2, one2);
+            const f32x2 ga = gather2(r01, r23, minus_m2, k256), gb = gather2(r45, r67, minus_m2, k256);
             const unsigned long long e = plane_elem + (unsigned long long)t * RE + (unsigned long long)o * 8u;
-            if (int4) {
-                const uint32_t a0 = c.x & 0x0f0f0f0fu, a1 = c.y & 0x0f0f0f0fu;
-                *reinterpret_cast<uint32_t *>(op.data + (e >> 1)) = __byte_perm(a0 | (a0 >> 4), a1 | (a1 >> 4), 0x6420);
-            } else {
-                *reinterpret_cast<uint2 *>(op.data + e) = c;
-            }
+            if (int4)
+                *reinterpret_cast<uint32_t *>(op.data + (e >> 1)) = __byte_perm(nibbles4_from(ga), nibbles4_from(gb), 0x5410) ^ 0x88888888u;
+            else
+                *reinterpret_cast<uint2 *>(op.data + e) = make_uint2(codes4_from(ga), codes4_from(gb));
         }
     }
 }
