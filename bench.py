@@ -663,6 +663,49 @@ def sweep_extract(leg, reps):
     return points
 
 
+def shard_extract(leg, reps):
+    """The 8B pool seen by one rank of a head-sharded (tensor-parallel) engine: 4, 2 and 1 of the 8 KV heads per GPU,
+    i.e. token rows of 512, 256 and 128 elements and pool blocks of 16, 8 and 4 KiB (the same memory registered with
+    fewer heads and more blocks).  Store, retrieve and compose of 512-token chunks, raw and int8-g64, fully fragmented
+    tables, enough chunks per launch to move 2 GiB on the pool side."""
+    torch, K, synth = leg.torch, leg.K, leg.synth
+    shape, dev, s = leg.shape, leg.dev, leg.s
+    arena = torch.empty((2 << 30) + (256 << 20), dtype=torch.uint8, device=dev)
+    T, bs, points = 512, shape.block_size, []
+    for heads in (4, 2, 1):
+        k = shape.n_kv_heads // heads
+        nb = shape.n_blocks * k
+        E = shape.elems_per_token // k
+        desc = K.pool_desc(shape.n_layers, heads, shape.head_dim, bs, nb,
+                           [t.data_ptr() for t in leg.k], [t.data_ptr() for t in leg.v])      # same memory, narrower rows
+        pid = K.kdn_pool_register(leg.ctx, desc)
+        blocks = T // bs
+        for codec in (RAW, INT8):
+            bpe = bytes_per_elem(codec)
+            n = max(1, (2 << 30) // int(T * E * 2))
+            cb = K.kdn_chunk_bytes(desc, T, codec)
+            src = synth.make_table(n * blocks, nb, 1, synth.SEED_TABLES)
+            dst = synth.make_table(n * blocks, nb, 1, synth.SEED_TABLES + 1, exclude=src)
+            d_src, d_dst = torch.from_numpy(src).to(dev), torch.from_numpy(dst).to(dev)
+            chunk = lambda i, base=0: K.Chunk(arena.data_ptr() + i * cb, cb, T, codec, K.KDN_MEM_DEVICE, base)
+            st = [K.XferOp(d_src.data_ptr() + i * blocks * 4, blocks, 0, chunk(i)) for i in range(n)]
+            rt = [K.XferOp(d_dst.data_ptr() + i * blocks * 4, blocks, 0, chunk(i)) for i in range(n)]
+            rq = [K.ComposeReq(d_dst.data_ptr(), n * blocks, [chunk(i) for i in range(n)], [i * T for i in range(n)], shape.rope_theta)]
+            row = {"kv_heads_per_gpu": heads, "row_elems": heads * shape.head_dim, "block_bytes": bs * heads * shape.head_dim * 2,
+                   "codec": "int8" if codec else "raw", "chunks": n}
+            for name, fn in (("store", lambda: K.kdn_store(leg.ctx, pid, st, s)), ("retrieve", lambda: K.kdn_retrieve(leg.ctx, pid, rt, s)),
+                             ("compose", lambda: K.kdn_compose(leg.ctx, pid, rq, s))):
+                for _ in range(8):                        # every ring slot of the context has sized its rotation table
+                    fn()
+                ms = leg.timed(fn, reps)
+                row[name + "_gbs"] = n * T * E * bpe / (ms * 1e-3) / 1e9
+            leg.check()
+            points.append(row)
+    del arena
+    torch.cuda.empty_cache()
+    return points
+
+
 def host_link_peak(torch, stream, dev):
     """Host-link ceiling of this run: one 1 GiB pinned cudaMemcpyAsync each way, best of 5."""
     probe = torch.empty(1 << 30, dtype=torch.uint8).pin_memory()
@@ -789,12 +832,13 @@ def run_gpu(args) -> None:
     extras = extras_8b(leg, dev_sets, reps, tuple(x for x in args.extras.split(",") if x))
     full = not (args.pool_blocks or args.chunks or args.parts)
     sweep_points = sweep_extract(leg, min(reps, 10)) if full and not args.no_sweep else None
+    shard_points = shard_extract(leg, min(reps, 10)) if full and not args.no_sweep else None
 
     if args.no_e2e:
         if rank == 0:
             print(json.dumps({"note": "profiling run, not a bench record", "ops_ms": op_ms, "kernels": leg.kernels,
                               "ops_gbs": {n: leg.op_bytes[n] / (op_ms[n] * 1e-3) / 1e9 for n in NAMES}, **extras,
-                              "sweep_extract": sweep_points}))
+                              "sweep_extract": sweep_points, "head_sharded_shapes": shard_points}))
         leg.close()
         return
 
@@ -860,6 +904,11 @@ def run_gpu(args) -> None:
                 per_op["sweep_min_" + name] = [round(worst[name + "_gbs"], 1), round(worst[name + "_gbs"] / 8000.0, 4),
                                                "T=%d bs=%d %s" % (worst["chunk_tokens"], worst["block_size"], worst["codec"])]
             per_op["sweep_points"] = len(sweep_points)
+        if shard_points:
+            for name in ("store", "retrieve", "compose"):
+                worst = min(shard_points, key=lambda p: p[name + "_gbs"])
+                per_op["head_shard_min_" + name] = [round(worst[name + "_gbs"], 1), round(worst[name + "_gbs"] / 8000.0, 4),
+                                                    "%d of 8 KV heads per GPU, %s" % (worst["kv_heads_per_gpu"], worst["codec"])]
         # the widenings of the 8B leg in the same compact form (outside `value`)
         wide = {}
         for key in ("ops_int4_not_in_value", "ops_per_channel_key_codecs_not_in_value", "ops_keep_list_not_in_value"):
@@ -881,7 +930,7 @@ def run_gpu(args) -> None:
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
             "dtype": "bf16/int8 (fp32 codec and rotation, fp64 angles)", "data": "synthetic",
-            "config": {"workload": W["text"], "also_measured": "llama3-70b batch (32x4x2048 tokens) and sweep ends: roofline.per_op",
+            "config": {"workload": W["text"], "also_measured": "llama3-70b batch (32x4x2048 tokens), sweep ends and head-sharded pool shapes: roofline.per_op",
                        "l2": "inputs larger than L2 (every op streams >= 1.9 GB once)", "bytes_per_step": step_bytes},
             "tokens_per_s_reloaded": world * reload_tokens / (sum(op_ms[n] for n in NAMES if not n.startswith("store")) * 1e-3),
             "roofline": {"bound": "hbm", "kernel": kernels[top]["kernel"], "op": top, "achieved": gbs[top], "peak": peak,
@@ -902,7 +951,7 @@ def run_gpu(args) -> None:
             "ops": ops, "llama3_70b": ({"workload": r70["workload"], "steps": r70["steps"], "ms_per_step": r70["ms_per_step"],
                                         "op_ms": r70["op_ms"], "kernels": {n: r70["kernels"][n]["kernel"] for n in NAMES},
                                         "launches": r70["launches"]} if r70 else None),
-            "sweep_extract": sweep_points, **extras,
+            "sweep_extract": sweep_points, "head_sharded_shapes": shard_points, **extras,
         }
         if not args.no_cpu_baseline and world == 1:
             cores = len(os.sched_getaffinity(0))

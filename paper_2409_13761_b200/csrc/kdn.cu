@@ -481,7 +481,41 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
         else def = Shape{ 0, 8, 6, 2, 1, 1 };
     }
     const unsigned tpb = (unsigned)((block_elems + tile_elems - 1) / tile_elems);
-
+    if (!any_list && !kc_decode && ctx->tuning.tile_bytes <= 0) {
+        // A pool block smaller than the tile the shape was tuned for (few KV heads per GPU under tensor parallelism, or
+        // a small block_size) caps the tile at the block.  From sweeps on the 8B shape with 4, 2 and 1 KV heads:
+        // the copy form keeps the same bytes in flight per SM with more CTAs, then more slots (one head, 4 KiB blocks:
+        // 1.9 -> 6.3 TB/s); the coding forms give a tile of 4 KiB or less to one warp instead of four (int8 store /
+        // retrieve 4.2 / 4.6 -> 5.8 / 5.7, compose 3.8 -> 5.4); a rotation-only compose takes six slots in as many CTAs
+        // as fit (2.7 -> 6.2); a coded compose whose every tile needs its own table entry takes six slots (5.6 -> 6.2).
+        const unsigned tb = tile_elems * 2u;
+        const bool capped = tb < (unsigned)def.tile_bytes;
+        if (!compute) {
+            if (capped) {
+                const unsigned in_flight = (unsigned)def.tile_bytes * (unsigned)def.stages * (unsigned)def.ctas_per_sm;
+                unsigned ctas = (unsigned)def.tile_bytes / tb * (unsigned)def.ctas_per_sm;
+                if (ctas > 8u) ctas = 8u;
+                unsigned st = in_flight / (ctas * tb);
+                if (st < (unsigned)def.stages) st = (unsigned)def.stages;
+                if (st > 16u) st = 16u;
+                def.ctas_per_sm = (int)ctas;
+                def.stages = (int)st;
+            }
+        } else if (!any_rot) {
+            if (tb <= 4096u) def = Shape{ 0, 8, 4, 2, def.lag, 1 };
+        } else if (!any_coded) {
+            if (capped) {
+                unsigned ctas = (unsigned)ctx->env.smem_optin / (6u * tb + 1024u);
+                if (ctas > 6u) ctas = 6u;
+                if (ctas < 1u) ctas = 1u;
+                def = Shape{ 0, 6, (int)ctas, 1, 1 };
+            }
+        } else if (tb <= 4096u) {
+            def = Shape{ 0, 8, 8, 2, 1, 1 };
+        } else if (tpb == 1u) {
+            def = Shape{ 0, 6, 3, 1, 1 };
+        }
+    }
     const unsigned a_bytes = (tile_elems * 2u + 127u) & ~127u;
     const unsigned b_bytes = compute ? ((tile_elems + 127u) & ~127u) : 0u;
     unsigned s_bytes = compute ? ((tile_elems / 16u + 127u) & ~127u) : 0u;
@@ -582,7 +616,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
         const unsigned cols = row_elems / n_split;
         const size_t kc_smem = kc_smem_bytes(cols);
         if (kc_smem > smem_limit) return KDN_E_UNSUPPORTED;
-        unsigned kc_threads = (cols / 8u * kKcSlices + 31u) & ~31u;
+        unsigned kc_threads = (cols / 8u + 7u) / 8u * 32u;       // a warp per 64 channels
         if (kc_threads > 512u) kc_threads = 512u;
         if (kc_threads < 64u) kc_threads = 64u;
         KcLaunch kp{};

@@ -1145,7 +1145,7 @@ constexpr unsigned kKcSlices = 4;                          // token slices in pa
 constexpr unsigned kKcTok = 64u / kKcSlices;              // tokens per slice
 __host__ __device__ inline size_t kc_smem_bytes(unsigned cols)
 {
-    return (size_t)64 * cols * 2u + (size_t)kKcSlices * cols * 2u + (size_t)cols * 4u + 16u;
+    return (size_t)64 * cols * 2u + 16u;                   // the tile, the barrier and the abort word
 }
 
 __global__ void __launch_bounds__(512) kdn_store_kc_kernel(const __grid_constant__ KcLaunch P)
@@ -1164,13 +1164,10 @@ __global__ void __launch_bounds__(512) kdn_store_kc_kernel(const __grid_constant
     const unsigned n_tok = (unsigned)op.T - t0 < 64u ? (unsigned)op.T - t0 : 64u;
 
     unsigned char *X = smem_raw;                                             // [n_tok][C] bf16
-    unsigned char *pmax = X + (size_t)64 * C * 2u;                           // [kKcSlices][C] bf16 magnitudes
-    float *inv = reinterpret_cast<float *>(pmax + (size_t)kKcSlices * C * 2u);    // [C]
-    unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(reinterpret_cast<unsigned char *>(inv) + (size_t)C * 4u);
+    unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(X + (size_t)64 * C * 2u);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bar_mem + 1);
     const uint32_t bar = smem_u32(bar_mem);
     const int tid = (int)threadIdx.x;
-    const int nthreads = (int)blockDim.x;
 
     if (tid == 0) {
         mbar_init(bar, 1u);
@@ -1240,63 +1237,82 @@ __global__ void __launch_bounds__(512) kdn_store_kc_kernel(const __grid_constant
         return;
     }
 
+    // From here on the warps do not meet again: a warp owns 64 channels (eight octets) for all 64 tokens, lane (j, q)
+    // takes octet j of them in token quarter q.  The group's largest magnitudes meet through two shuffles, each lane
+    // forms the scale and the reciprocal of two of its octet's channels, and four more shuffles hand every lane the
+    // reciprocals of all eight.
     const unsigned octets = C >> 3;
-    const unsigned items = octets * kKcSlices;
-    // pass 1: per (eight channels, token slice) the largest magnitudes, as packed bf16 pairs
-    for (unsigned it = (unsigned)tid; it < items; it += (unsigned)nthreads) {
-        const unsigned q = it / octets, o = it - q * octets;
-        const unsigned ta = q * kKcTok, tb = ta + kKcTok < n_tok ? ta + kKcTok : n_tok;
-        uint32_t m0 = 0u, m1 = 0u, m2 = 0u, m3 = 0u;
-        for (unsigned t = ta; t < tb; ++t) {
-            const uint4 x = lds128(X + ((size_t)t * C + (size_t)o * 8u) * 2u);
-            m0 = maxabs_bf16x2(m0, x.x); m1 = maxabs_bf16x2(m1, x.y);
-            m2 = maxabs_bf16x2(m2, x.z); m3 = maxabs_bf16x2(m3, x.w);
+    const unsigned lane = (unsigned)tid & 31u, j = lane & 7u, q = lane >> 3;
+    const unsigned o = ((unsigned)tid >> 5) * 8u + j;
+    const bool act = o < octets;
+    const unsigned ta = q * kKcTok, tb = ta + kKcTok < n_tok ? ta + kKcTok : n_tok;
+    const unsigned char *Xo = X + (size_t)o * 16u;
+    // pass 1: the largest magnitudes of the lane's octet over its tokens, as packed bf16 pairs
+    uint32_t m0 = 0u, m1 = 0u, m2 = 0u, m3 = 0u;
+    if (act) {
+        if (n_tok == 64u) {                                                   // a full group: a fixed trip count, loads batched
+#pragma unroll
+            for (unsigned i = 0; i < kKcTok; ++i) {
+                const uint4 x = lds128(Xo + (size_t)(ta + i) * C * 2u);
+                m0 = maxabs_bf16x2(m0, x.x); m1 = maxabs_bf16x2(m1, x.y);
+                m2 = maxabs_bf16x2(m2, x.z); m3 = maxabs_bf16x2(m3, x.w);
+            }
+        } else {
+            for (unsigned t = ta; t < tb; ++t) {
+                const uint4 x = lds128(Xo + (size_t)t * C * 2u);
+                m0 = maxabs_bf16x2(m0, x.x); m1 = maxabs_bf16x2(m1, x.y);
+                m2 = maxabs_bf16x2(m2, x.z); m3 = maxabs_bf16x2(m3, x.w);
+            }
         }
-        sts128(pmax + ((size_t)q * C + (size_t)o * 8u) * 2u, make_uint4(m0, m1, m2, m3));
     }
-    __syncthreads();
-    // scales: one thread per channel (a layer's scales start wherever the previous layer's end, so only 4-byte
-    // alignment is certain: plain fp32 stores, consecutive channels on consecutive threads)
-    const unsigned long long per_layer = (unsigned long long)n_groups * RE + (((unsigned long long)op.T * RE) >> 6);
-    float *g_scales = reinterpret_cast<float *>(op.scales) + (unsigned long long)li * per_layer + (unsigned long long)g * RE + c0;
-    for (unsigned ch = (unsigned)tid; ch < C; ch += (unsigned)nthreads) {
-        unsigned short mx = 0;
-        for (unsigned q = 0; q < kKcSlices; ++q) {
-            const unsigned short v = *reinterpret_cast<const unsigned short *>(pmax + ((size_t)q * C + ch) * 2u) & 0x7fffu;
-            mx = v > mx ? v : mx;                                             // magnitudes of bf16 order like their bit patterns
-        }
-        const float a = __uint_as_float((uint32_t)mx << 16);
-        const float sc = __fdiv_rn(a, qmax);
-        const bool ok = sc >= 1.17549435e-38f;                                // smallest normal fp32; false for NaN too
-        g_scales[ch] = ok ? sc : 0.0f;
-        inv[ch] = ok ? __fdiv_rn(qmax, a) : 0.0f;
+#pragma unroll
+    for (int d = 8; d <= 16; d <<= 1) {
+        m0 = maxabs_bf16x2(m0, __shfl_xor_sync(0xffffffffu, m0, d)); m1 = maxabs_bf16x2(m1, __shfl_xor_sync(0xffffffffu, m1, d));
+        m2 = maxabs_bf16x2(m2, __shfl_xor_sync(0xffffffffu, m2, d)); m3 = maxabs_bf16x2(m3, __shfl_xor_sync(0xffffffffu, m3, d));
     }
-    __syncthreads();
+    // scales of channels 2q and 2q + 1 of the octet (a layer's scales start wherever the previous layer's end, so only
+    // 4-byte alignment is certain: plain fp32 stores)
+    const uint32_t mq = q == 0u ? m0 : q == 1u ? m1 : q == 2u ? m2 : m3;
+    const float a_lo = __uint_as_float((mq & 0x7fffu) << 16), a_hi = __uint_as_float(mq & 0x7fff0000u);
+    const float sc_lo = __fdiv_rn(a_lo, qmax), sc_hi = __fdiv_rn(a_hi, qmax);
+    const bool ok_lo = sc_lo >= 1.17549435e-38f, ok_hi = sc_hi >= 1.17549435e-38f;   // smallest normal fp32; false for NaN too
+    const float inv_lo = ok_lo ? __fdiv_rn(qmax, a_lo) : 0.0f, inv_hi = ok_hi ? __fdiv_rn(qmax, a_hi) : 0.0f;
+    if (act) {
+        const unsigned long long per_layer = (unsigned long long)n_groups * RE + (((unsigned long long)op.T * RE) >> 6);
+        float *g_scales = reinterpret_cast<float *>(op.scales) + (unsigned long long)li * per_layer + (unsigned long long)g * RE + c0 + o * 8u + q * 2u;
+        g_scales[0] = ok_lo ? sc_lo : 0.0f;
+        g_scales[1] = ok_hi ? sc_hi : 0.0f;
+    }
+    const f32x2 i0 = pack2(__shfl_sync(0xffffffffu, inv_lo, (int)j), __shfl_sync(0xffffffffu, inv_hi, (int)j));
+    const f32x2 i1 = pack2(__shfl_sync(0xffffffffu, inv_lo, (int)j + 8), __shfl_sync(0xffffffffu, inv_hi, (int)j + 8));
+    const f32x2 i2 = pack2(__shfl_sync(0xffffffffu, inv_lo, (int)j + 16), __shfl_sync(0xffffffffu, inv_hi, (int)j + 16));
+    const f32x2 i3 = pack2(__shfl_sync(0xffffffffu, inv_lo, (int)j + 24), __shfl_sync(0xffffffffu, inv_hi, (int)j + 24));
+    if (!act) return;
     // pass 2: codes
     const float magic = 12582912.0f + (int4 ? 8.0f : 128.0f);
     const f32x2 magic2 = pack2(magic, magic);
     const f32x2 minus_m2 = pack2(-12582912.0f, -12582912.0f);
     const f32x2 k256 = pack2(256.0f, 256.0f);
     const f32x2 one2 = pack2(P.one, P.one);
-    const unsigned long long plane_elem = ((unsigned long long)li * 2ull * (unsigned long long)op.T + t0) * RE + c0;   // K plane, token t0
-    for (unsigned it = (unsigned)tid; it < items; it += (unsigned)nthreads) {
-        const unsigned q = it / octets, o = it - q * octets;
-        const unsigned ta = q * kKcTok, tb = ta + kKcTok < n_tok ? ta + kKcTok : n_tok;
-        const f32x2 i0 = lds_f32x2(inv + o * 8u), i1 = lds_f32x2(inv + o * 8u + 2u);
-        const f32x2 i2 = lds_f32x2(inv + o * 8u + 4u), i3 = lds_f32x2(inv + o * 8u + 6u);
-        for (unsigned t = ta; t < tb; ++t) {
-            const uint4 x = lds128(X + ((size_t)t * C + (size_t)o * 8u) * 2u);
-            const f32x2 r01 = add2_unfused(mul2(bf16x2_widen(x.x), i0), magic2, one2);
-            const f32x2 r23 = add2_unfused(mul2(bf16x2_widen(x.y), i1), magic2, one2);
-            const f32x2 r45 = add2_unfused(mul2(bf16x2_widen(x.z), i2), magic2, one2);
-            const f32x2 r67 = add2_unfused(mul2(bf16x2_widen(x.w), i3), magic2, one2);
-            const f32x2 ga = gather2(r01, r23, minus_m2, k256), gb = gather2(r45, r67, minus_m2, k256);
-            const unsigned long long e = plane_elem + (unsigned long long)t * RE + (unsigned long long)o * 8u;
-            if (int4)
-                *reinterpret_cast<uint32_t *>(op.data + (e >> 1)) = __byte_perm(nibbles4_from(ga), nibbles4_from(gb), 0x5410) ^ 0x88888888u;
-            else
-                *reinterpret_cast<uint2 *>(op.data + e) = make_uint2(codes4_from(ga), codes4_from(gb));
-        }
+    const unsigned long long plane_elem = ((unsigned long long)li * 2ull * (unsigned long long)op.T + t0) * RE + c0 + o * 8u;   // K plane, token t0
+    auto code_row = [&](unsigned t) {
+        const uint4 x = lds128(Xo + (size_t)t * C * 2u);
+        const f32x2 r01 = add2_unfused(mul2(bf16x2_widen(x.x), i0), magic2, one2);
+        const f32x2 r23 = add2_unfused(mul2(bf16x2_widen(x.y), i1), magic2, one2);
+        const f32x2 r45 = add2_unfused(mul2(bf16x2_widen(x.z), i2), magic2, one2);
+        const f32x2 r67 = add2_unfused(mul2(bf16x2_widen(x.w), i3), magic2, one2);
+        const f32x2 ga = gather2(r01, r23, minus_m2, k256), gb = gather2(r45, r67, minus_m2, k256);
+        const unsigned long long e = plane_elem + (unsigned long long)t * RE;
+        if (int4)
+            *reinterpret_cast<uint32_t *>(op.data + (e >> 1)) = __byte_perm(nibbles4_from(ga), nibbles4_from(gb), 0x5410) ^ 0x88888888u;
+        else
+            *reinterpret_cast<uint2 *>(op.data + e) = make_uint2(codes4_from(ga), codes4_from(gb));
+    };
+    if (n_tok == 64u) {
+#pragma unroll 4
+        for (unsigned i = 0; i < kKcTok; ++i) code_row(ta + i);
+    } else {
+        for (unsigned t = ta; t < tb; ++t) code_row(t);
     }
 }
 
