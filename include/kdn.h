@@ -352,9 +352,11 @@ kdn_status kdn_compose(kdn_ctx *ctx, int pool_id, const kdn_compose_req *reqs, i
 kdn_status kdn_compose_static(int device, const kdn_pool_desc *pool, const kdn_compose_req *reqs, int n_reqs,
                               void *cuda_stream, int wait);
 
-/* kdn_store / kdn_retrieve for chunks that hold only the tokens of a keep-list (see kdn_sparse_op).  One tile per
- * listed token row; list entries that point outside the block table are skipped and reported as KDN_E_RANGE by
- * kdn_status_sync.  kdn_retrieve_sparse writes exactly the listed positions. */
+/* kdn_store / kdn_retrieve for chunks that hold only the tokens of a keep-list (see kdn_sparse_op).  A tile takes
+ * one listed token row or several that follow one another in the list (up to 16); a list entry that points outside
+ * the block table is reported as KDN_E_RANGE by kdn_status_sync and nothing is moved for it, nor, possibly, for the
+ * rows that share its tile: after that error neither the chunk (store) nor the listed positions (retrieve) are to be
+ * used.  kdn_retrieve_sparse writes the listed positions and nothing else. */
 kdn_status kdn_store_sparse(kdn_ctx *ctx, int pool_id, const kdn_sparse_op *ops, int n_ops,
                             void *cuda_stream, void *side_stream);
 kdn_status kdn_retrieve_sparse(kdn_ctx *ctx, int pool_id, const kdn_sparse_op *ops, int n_ops,
@@ -386,11 +388,14 @@ kdn_status kdn_set_wait_limit_ns(kdn_ctx *ctx, uint64_t ns);
 uint64_t kdn_launch_count(const kdn_ctx *ctx);
 
 /* Shape of the context's most recent launch of the tile pipeline, for reports: op 0 store / 1 retrieve / 2 compose
- * (the kernel is kdn_store_kernel / kdn_retrieve_kernel / kdn_compose_kernel<compute_groups, group_warps>);
- * grid is what was asked for (the launch itself never exceeds the CTAs resident at once). */
+ * (the kernel is kdn_store_kernel / kdn_retrieve_kernel / kdn_compose_kernel<compute_groups, group_warps>, or, with
+ * rows_kernel = 1, kdn_store_rows_kernel / kdn_retrieve_rows_kernel: tiles of up to 16 token rows, which keep-lists over
+ * short rows and dense coded ops on pool blocks of 2 KiB or less are given); rows_per_tile: token rows per tile of a
+ * keep-list launch (1 otherwise); grid is what was asked for (the launch itself never exceeds the CTAs resident at once). */
 typedef struct {
     int32_t  op, compute_groups, group_warps, tile_bytes, stages, ctas_per_sm, store_lag, grid, smem_bytes;
     uint32_t n_tiles;
+    int32_t  rows_per_tile, rows_kernel;
 } kdn_launch_info;
 kdn_status kdn_last_launch(const kdn_ctx *ctx, kdn_launch_info *out);
 

@@ -370,7 +370,7 @@ Shape default_shape(int OP, bool any_coded, bool any_rot)
 // Pipeline slots: at least lag + 2, a multiple of the compute groups (a slot must always belong to the
 // same group), and, unless the caller fixed the count, few enough for ctas_per_sm CTAs to share an SM.
 kdn_status fit_stages(int &stages, int groups, int lag, bool shrink, unsigned stage_bytes, int ctas_per_sm, size_t smem_limit,
-                      int rows_per_tile = 1)
+                      int rows_per_tile = 1, bool wide = false)
 {
     const int g = groups > 0 ? groups : 1;
     if (stages > kMaxStages) stages = kMaxStages;
@@ -379,20 +379,32 @@ kdn_status fit_stages(int &stages, int groups, int lag, bool shrink, unsigned st
     stages = stages / g * g;
     if (shrink)
         while (stages - g >= min_stages &&
-               smem_bytes(stages, stage_bytes, rows_per_tile) * (size_t)ctas_per_sm > smem_limit - 1024u * (size_t)ctas_per_sm)
+               smem_bytes(stages, stage_bytes, rows_per_tile, wide) * (size_t)ctas_per_sm > smem_limit - 1024u * (size_t)ctas_per_sm)
             stages -= g;
-    return smem_bytes(stages, stage_bytes, rows_per_tile) > smem_limit ? KDN_E_UNSUPPORTED : KDN_OK;
+    return smem_bytes(stages, stage_bytes, rows_per_tile, wide) > smem_limit ? KDN_E_UNSUPPORTED : KDN_OK;
 }
 
 // Launch the instantiation for (OP, compute groups, warps per group); groups = 0 is the pure-copy form.
 kdn_status launch_tiles(LaunchEnv &env, int OP, int groups, int gw, unsigned grid, size_t smem, cudaStream_t stream,
-                        const Launch &lp, bool overlap = false)
+                        const Launch &lp, bool overlap = false, bool wide = false)
 {
 #define KDN_CASE(G, W)                                                                                             \
     if (groups == G && (G == 0 || gw == W)) {                                                                      \
         if (OP == OP_STORE) return launch_kernel(env, kdn_store_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp, overlap);      \
         if (OP == OP_RETRIEVE) return launch_kernel(env, kdn_retrieve_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp, overlap); \
         return launch_kernel(env, kdn_compose_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp, overlap);               \
+    }
+    if (wide) {
+        // tiles of up to 16 token rows: the kernels that keep the row indices in shared memory (store and retrieve, copy
+        // form and two single-warp groups)
+#define KDN_ROWS_CASE(G, W)                                                                                        \
+        if (groups == G && (G == 0 || gw == W)) {                                                                  \
+            if (OP == OP_STORE) return launch_kernel(env, kdn_store_rows_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp, overlap);       \
+            if (OP == OP_RETRIEVE) return launch_kernel(env, kdn_retrieve_rows_kernel<G, W>, threads_for(G, W), grid, smem, stream, lp, overlap); \
+        }
+        KDN_ROWS_CASE(0, 4) KDN_ROWS_CASE(2, 1)
+#undef KDN_ROWS_CASE
+        return KDN_E_UNSUPPORTED;
     }
     KDN_CASE(0, 4) KDN_CASE(1, 4) KDN_CASE(2, 4) KDN_CASE(3, 4) KDN_CASE(4, 4) KDN_CASE(6, 4)
     KDN_CASE(2, 1) KDN_CASE(4, 1) KDN_CASE(8, 1)
@@ -429,6 +441,22 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     }
     const bool compute = any_coded || any_rot;
     const unsigned row_elems = (unsigned)pool.H * (unsigned)pool.D;
+    // Pool blocks of 2 KiB or less (block_size 1 or 2 with whole rows, a few tokens of one KV head): a coding tile that stops
+    // at the end of its block is far too small.  Such launches run as keep-list launches over the implied list 0, 1, 2, ...
+    // (list_mode 3): a tile then takes several token rows, wherever their blocks are, and rows that are neighbours in the
+    // pool still share a copy (8B shape, block_size 1: int8 store / retrieve 3.5 / 3.7 -> TB/s of the keep-list form).
+    std::vector<HostOp> as_rows;
+    if (any_coded && !any_rot && !any_list && !any_kc && (OP == OP_STORE || OP == OP_RETRIEVE) && ctx->tuning.tile_bytes <= 0 &&
+        (unsigned long long)pool.bs * row_elems * 2ull <= 2048ull) {
+        as_rows.assign(hops, hops + n);
+        for (HostOp &h : as_rows) {
+            h.op.list_mode = 3;
+            h.op.n_list = h.op.T;
+            h.op.list = nullptr;
+        }
+        hops = as_rows.data();
+        any_list = all_list = true;
+    }
 
     // tile size: whole 16-byte units; whole 64-element groups with int8 / int4; whole head rows with rotation
     unsigned unit = 8;
@@ -466,14 +494,19 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
         // the 8B shape (2 KiB rows), throughput grows with CTAs per SM up to 8 (copy form 3.0 -> 6.4 TB/s)
         tile_elems = row_elems;
         bool all_keep = true;
-        for (int i = 0; i < n; ++i) all_keep &= hops[i].op.list_mode == 1;
+        for (int i = 0; i < n; ++i) all_keep &= hops[i].op.list_mode == 1 || hops[i].op.list_mode == 3;
         const int want_rows = ctx->tuning.tile_bytes > 0 ? ctx->tuning.tile_bytes / 2 / (int)row_elems : 2048 / (int)row_elems;
-        if (any_coded && !any_rot && all_keep && want_rows >= 2 && (unsigned long long)pool.nb * (unsigned)pool.bs < 0xffffffffull) {
+        if (!any_coded && !any_rot && all_keep && want_rows >= 2 && row_elems < 1024u && (unsigned long long)pool.nb * (unsigned)pool.bs < 0xffffffffull) {
+            // copy form on rows shorter than 2 KiB (few KV heads per GPU): several rows per tile as well
+            rows_per_tile = want_rows > kWideRowsPerTile ? kWideRowsPerTile : want_rows;
+            tile_elems = (unsigned)rows_per_tile * row_elems;
+            def = Shape{ 0, 4, 8, 0, 1 };
+        } else if (any_coded && !any_rot && all_keep && want_rows >= 2 && (unsigned long long)pool.nb * (unsigned)pool.bs < 0xffffffffull) {
             // coded keep-list launches: a tile takes several listed rows -- neighbours in the chunk, so its codes and
             // scales move with one copy each, and rows that are neighbours in the pool share a copy too.  From a sweep on
             // the 8B shape with half of the tokens kept: two 1024-element rows per tile, five CTAs per SM with two
             // single-warp groups each, one store in flight (int8 5.1 -> 5.9 TB/s, int4 4.0 -> 4.9)
-            rows_per_tile = want_rows > kMaxRowsPerTile ? kMaxRowsPerTile : want_rows;
+            rows_per_tile = want_rows > kWideRowsPerTile ? kWideRowsPerTile : want_rows;
             tile_elems = (unsigned)rows_per_tile * row_elems;
             def = Shape{ 0, 6, 5, 2, 1, 1 };
         } else if (!any_coded && !any_rot) def = Shape{ 0, 4, 8, 0, 1 };
@@ -531,9 +564,11 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     int ctas_per_sm = ctx->tuning.ctas_per_sm > 0 ? ctx->tuning.ctas_per_sm : def.ctas_per_sm;
     int stages = ctx->tuning.stages > 0 ? ctx->tuning.stages : def.stages;
     const size_t smem_limit = (size_t)ctx->env.smem_optin;
-    kdn_status fit = fit_stages(stages, groups, lag, ctx->tuning.stages <= 0, stage_bytes, ctas_per_sm, smem_limit, rows_per_tile);
+    // more than four rows per tile, and dense ops run as rows, go to the kernels built for that
+    const bool wide = rows_per_tile > kMaxRowsPerTile || !as_rows.empty();
+    kdn_status fit = fit_stages(stages, groups, lag, ctx->tuning.stages <= 0, stage_bytes, ctas_per_sm, smem_limit, rows_per_tile, wide);
     if (fit != KDN_OK) return fit;
-    const size_t smem = smem_bytes(stages, stage_bytes, rows_per_tile);
+    const size_t smem = smem_bytes(stages, stage_bytes, rows_per_tile, wide);
 
     // Few ops travel as kernel parameters; otherwise through a ring slot (pinned staging + device copy).  A ring
     // slot is also what owns the rotation table.
@@ -652,7 +687,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     // Every launch of the pipeline is a programmatic dependent launch.  After the rotation-table kernel only the warps
     // that read the table wait for it; otherwise every thread waits for the kernel before it, whatever that was.
     lp.wait_all = (OP == OP_COMPOSE && n_rope > 0) ? 0 : 1;
-    kdn_status st = launch_tiles(ctx->env, OP, groups, gw, grid, smem, stream, lp, true);
+    kdn_status st = launch_tiles(ctx->env, OP, groups, gw, grid, smem, stream, lp, true, wide);
     if (st != KDN_OK) return st;
     ctx->launches++;
     ctx->last.op = OP;
@@ -665,6 +700,8 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     ctx->last.grid = (int32_t)grid;
     ctx->last.smem_bytes = (int32_t)smem;
     ctx->last.n_tiles = (uint32_t)tiles;
+    ctx->last.rows_per_tile = rows_per_tile;
+    ctx->last.rows_kernel = wide ? 1 : 0;
     if (slot) {
         KDN_CUDA(cudaEventRecord(slot->done, stream));
         slot->used = true;

@@ -50,7 +50,10 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;   // default limit of
 enum : uint32_t { TF_CODED = 1u, TF_ROTATE = 2u, TF_SCALES_PLAIN = 4u, TF_INT4 = 8u,   // TF_CODED: int8 or int4
                   TF_KCHAN = 16u,     // key tile of a per-channel key codec: one scale per channel, row_elems of them
                   TF_ROWS = 32u };    // several listed token rows: contiguous in the chunk, rows[] says where each sits in the pool
-constexpr int kMaxRowsPerTile = 4;
+constexpr int kMaxRowsPerTile = 4;         // several-row tiles of the ordinary kernels
+constexpr int kWideRowsPerTile = 16;       // ... of the kernels built for short rows (kWide)
+constexpr unsigned kRowsAheadStride = 20;  // kWide: words per lane in the decoded-ahead row area (128-bit stores by 32 lanes at
+                                           // this stride spread over all banks)
 enum : int { OP_STORE = 0, OP_RETRIEVE = 1, OP_COMPOSE = 2 };
 
 // Status values mirrored from kdn.h (kept numeric here so device code has no host header).
@@ -73,7 +76,8 @@ struct __align__(16) DevOp {
     const int32_t *list;      // device token list (list_mode != 0): relative request positions, increasing
     int n_list;               // listed tokens
     int list_mode;            // 0: every token; 1 keep-list: chunk token i <-> off + list[i];
-                              // 2 select-list: chunk token list[i] <-> off + list[i]
+                              // 2 select-list: chunk token list[i] <-> off + list[i]; 3 (kWide kernels only): keep-list
+                              // 0, 1, 2, ... with no list in memory: a dense op whose tiles take whole token rows
     long long pos_end;        // request positions >= pos_end are outside the block table
     int kv_sel;               // 0: key and value planes; 2: value planes only (the keys of a per-channel key codec are
                               // stored by kdn_store_kc_kernel)
@@ -131,6 +135,8 @@ struct __align__(16) TileDesc {
     unsigned runs;                // TF_ROWS: nibble r = how many rows the copy that starts at row r covers (0: row r rides
                                   // along with an earlier one); rows that are neighbours in the pool share one copy.  The
                                   // rows' places in the pool plane travel beside the descriptor in shared memory.
+                                  // kWide kernels: bit r (r < 16) = a copy starts at row r and runs up to the next set bit;
+                                  // bits 16..20 = rows in the tile.
 };
 static_assert(sizeof(TileDesc) == 48, "TileDesc is copied with 128-bit accesses");
 
@@ -660,7 +666,7 @@ __device__ __forceinline__ void rotate_tile(unsigned char *A, const unsigned cha
 // Address resolution (request position -> block-table entry -> pool address) and chunk addressing
 // for tile g.  Records KDN_E_RANGE and yields an empty tile for a block id outside the pool.
 // rows_out: shared memory for the token-row indices of a several-row tile (TF_ROWS); untouched otherwise.
-template <int OP>
+template <int OP, bool kWide = false>
 __device__ __forceinline__ void decode_tile(const Launch &P, unsigned g, TileDesc &d, unsigned *rows_out)
 {
     d.n = 0; d.flags = 0; d.rope = -1; d.sbytes = 0;
@@ -679,7 +685,51 @@ __device__ __forceinline__ void decode_tile(const Launch &P, unsigned g, TileDes
     unsigned long long pool_elem;                           // element offset of the tile inside its pool block
     unsigned long long ce;                                  // element offset of the tile inside the chunk
     bool many_rows = false;
-    if (op.list_mode == 1 && P.rows_per_tile > 1) {
+    if (kWide && (op.list_mode == 1 || op.list_mode == 3)) {
+        // kWide: every keep-list tile goes this way, whatever its row count
+        const unsigned rpt = (unsigned)P.rows_per_tile;
+        const unsigned tpp = ((unsigned)op.n_list + rpt - 1u) / rpt;
+        plane = gl / tpp;
+        const unsigned i0 = (gl - plane * tpp) * rpt;
+        const unsigned nr = (unsigned)op.n_list - i0 < rpt ? (unsigned)op.n_list - i0 : rpt;
+        bool bad = false;
+        unsigned starts = 0u, prev = 0u;
+        // four rows at a time, so that their look-ups are in flight together; the indices go to shared memory
+        auto resolve4 = [&](unsigned r0) {
+            unsigned rows4[4] = { 0u, 0u, 0u, 0u };
+#pragma unroll
+            for (unsigned k = 0; k < 4u; ++k) {
+                const unsigned r = r0 + k;
+                if (r < nr) {
+                    const long long rel = op.list_mode == 3 ? (long long)(i0 + r) : (long long)__ldg(op.list + i0 + r);
+                    const long long p = op.off + rel;
+                    unsigned row = 0u;
+                    if (rel < 0 || p >= op.pos_end || (long long)(i0 + r) >= op.T) {
+                        bad = true;
+                    } else {
+                        const long long bi = p / P.bs;
+                        const long long id = __ldg(op.table + bi);
+                        if (id < 0 || id >= P.n_blocks) bad = true;
+                        else row = (unsigned)(id * P.bs + (p - bi * P.bs));
+                    }
+                    if (r == 0u || row != prev + 1u) starts |= 1u << r;
+                    prev = row;
+                    rows4[k] = row;
+                }
+            }
+            *reinterpret_cast<uint4 *>(rows_out + r0) = make_uint4(rows4[0], rows4[1], rows4[2], rows4[3]);
+        };
+        resolve4(0u);                                       // tiles of up to four rows end here
+        for (unsigned r0 = 4u; r0 < nr; r0 += 4u) resolve4(r0);
+        if (bad) { atomicCAS(P.status, 0, kStatusRange); return; }          // the whole tile is skipped
+        d.runs = starts | (nr << 16);
+        d.flags |= TF_ROWS;
+        many_rows = true;
+        id_index = 0;
+        pool_elem = 0;
+        ce = (unsigned long long)i0 * P.row_elems;
+        n = nr * P.row_elems;
+    } else if (op.list_mode == 1 && P.rows_per_tile > 1) {
         // keep-list: up to rows_per_tile consecutive listed tokens per tile; they are consecutive chunk tokens, and
         // each sits wherever its own block-table entry says
         const unsigned rpt = (unsigned)P.rows_per_tile;
@@ -730,7 +780,7 @@ __device__ __forceinline__ void decode_tile(const Launch &P, unsigned g, TileDes
         // one listed token (one row of H * D elements) per tile
         plane = gl / (unsigned)op.n_list;
         const unsigned i = gl - plane * (unsigned)op.n_list;
-        const long long rel = __ldg(op.list + i);
+        const long long rel = __ldg(op.list + i);                        // (list_mode 3 never comes here: kWide kernels only)
         const long long c = op.list_mode == 2 ? rel : (long long)i;      // chunk token
         const long long p = op.off + rel;
         if (rel < 0 || p >= op.pos_end || c >= op.T) { atomicCAS(P.status, 0, kStatusRange); return; }
@@ -813,6 +863,7 @@ struct Smem {
     volatile unsigned *issued;        // tiles whose loads the loader has queued so far
 };
 
+template <bool kWide>
 __device__ __forceinline__ Smem carve(const Launch &P, unsigned char *smem)
 {
     Smem s;
@@ -826,21 +877,27 @@ __device__ __forceinline__ Smem carve(const Launch &P, unsigned char *smem)
     s.desc = reinterpret_cast<TileDesc *>(p);
     p += sizeof(TileDesc) * (size_t)P.stages;
     s.rows_stage = reinterpret_cast<unsigned *>(p);          // both areas exist only in launches with several-row tiles
-    s.rows_ahead = s.rows_stage + 4u * (size_t)P.stages;
-    if (P.rows_per_tile > 1) p += 16u * (size_t)P.stages + 16u * 64u;
+    if constexpr (kWide) {
+        s.rows_ahead = s.rows_stage + (size_t)kWideRowsPerTile * (size_t)P.stages;
+        p += 4u * ((size_t)kWideRowsPerTile * (size_t)P.stages + 64u * kRowsAheadStride);
+    } else {
+        s.rows_ahead = s.rows_stage + 4u * (size_t)P.stages;
+        if (P.rows_per_tile > 1) p += 16u * (size_t)P.stages + 16u * 64u;
+    }
     s.abort_flag = reinterpret_cast<volatile int *>(p);
     s.issued = reinterpret_cast<volatile unsigned *>(s.abort_flag + 1);
     return s;
 }
 
 // Bytes of shared memory a launch needs (host mirrors this).
-__host__ __device__ inline size_t smem_bytes(int stages, unsigned stage_bytes, int rows_per_tile = 1)
+__host__ __device__ inline size_t smem_bytes(int stages, unsigned stage_bytes, int rows_per_tile = 1, bool wide = false)
 {
     return (size_t)stages * stage_bytes + 24u * (size_t)stages + 16u + sizeof(TileDesc) * (size_t)stages + 16u +
-           (rows_per_tile > 1 ? 16u * (size_t)stages + 16u * 64u : 0u);
+           (wide ? 4u * ((size_t)kWideRowsPerTile * (size_t)stages + 64u * kRowsAheadStride)
+                 : rows_per_tile > 1 ? 16u * (size_t)stages + 16u * 64u : 0u);
 }
 
-template <int OP, int kGroups, int kGW>
+template <int OP, int kGroups, int kGW, bool kWide = false>
 __device__ __forceinline__ void tile_pipeline(const Launch &P)
 {
     constexpr bool kCompute = kGroups > 0;
@@ -849,7 +906,7 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
     // The next launch of this library in the stream may be scheduled as this kernel's CTAs leave, set up its barriers
     // and then wait (below) for this kernel to finish: back-to-back calls lose no time between kernels.
     release_dependents();
-    const Smem sm = carve(P, smem_raw);
+    const Smem sm = carve<kWide>(P, smem_raw);
     const int S = P.stages;
     const int tid = (int)threadIdx.x;
     const int warp = tid >> 5;
@@ -881,11 +938,12 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
         bool aborted = false;
         TileDesc cur;
         unsigned ahead = 0;                                   // which half of rows_ahead holds the rows of `cur`
-        decode_tile<OP>(P, (unsigned)lane < n_my ? bid + (unsigned)lane * grid : 0xffffffffu, cur, sm.rows_ahead + (size_t)lane * 4u);
+        constexpr unsigned kAheadStride = kWide ? kRowsAheadStride : 4u;
+        decode_tile<OP, kWide>(P, (unsigned)lane < n_my ? bid + (unsigned)lane * grid : 0xffffffffu, cur, sm.rows_ahead + (size_t)lane * kAheadStride);
         for (unsigned base = 0; base < n_my && !aborted; base += 32u) {
             TileDesc nxt;
-            decode_tile<OP>(P, base + 32u + lane < n_my ? bid + (base + 32u + lane) * grid : 0xffffffffu, nxt,
-                            sm.rows_ahead + ((size_t)(ahead ^ 1u) * 32u + (size_t)lane) * 4u);
+            decode_tile<OP, kWide>(P, base + 32u + lane < n_my ? bid + (base + 32u + lane) * grid : 0xffffffffu, nxt,
+                                   sm.rows_ahead + ((size_t)(ahead ^ 1u) * 32u + (size_t)lane) * kAheadStride);
             const unsigned cnt = n_my - base < 32u ? n_my - base : 32u;
             for (unsigned t = 0; t < cnt; ++t) {
                 bool ok = true;                               // lane t: the slot was free and the tile's copies are queued
@@ -893,6 +951,14 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                     ok = mbar_wait(sm.empty + 8u * st, ph ^ 1u, sm.abort_flag, P.wait_limit_ns);
                     if (ok) {
                         sm.desc[st] = cur;
+                        if constexpr (kWide) {
+                            if (OP != OP_STORE && (cur.flags & TF_ROWS)) {                 // the storer scatters the rows
+                                const unsigned *my_rows = sm.rows_ahead + ((size_t)ahead * 32u + (size_t)lane) * kRowsAheadStride;
+                                const unsigned nr = cur.runs >> 16;
+                                for (unsigned b = 0; b < nr; b += 4u)
+                                    sts128(sm.rows_stage + (size_t)st * kWideRowsPerTile + b, lds128(my_rows + b));
+                            }
+                        } else
                         if (OP != OP_STORE && (cur.flags & TF_ROWS))       // the storer scatters the rows
                             *reinterpret_cast<uint4 *>(sm.rows_stage + (size_t)st * 4u) =
                                 *reinterpret_cast<const uint4 *>(sm.rows_ahead + ((size_t)ahead * 32u + (size_t)lane) * 4u);
@@ -902,7 +968,24 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                             mbar_arrive(bar);
                         } else if (OP == OP_STORE) {
                             mbar_arrive_expect_tx(bar, cur.n * 2u);
-                            if (cur.flags & TF_ROWS) {
+                            if (kWide && (cur.flags & TF_ROWS)) {
+                                const unsigned rb = P.row_elems * 2u;
+                                const unsigned *my_rows = sm.rows_ahead + ((size_t)ahead * 32u + (size_t)lane) * kRowsAheadStride;
+                                const unsigned nr = cur.runs >> 16;
+                                const unsigned starts = (cur.runs & 0xffffu) | (1u << nr);      // a stop bit behind the last row
+                                for (unsigned b = 0; b < nr; b += 4u) {
+                                    const uint4 rv = lds128(my_rows + b);
+                                    const unsigned rows4[4] = { rv.x, rv.y, rv.z, rv.w };
+#pragma unroll
+                                    for (unsigned k = 0; k < 4u; ++k) {
+                                        const unsigned r = b + k;
+                                        if (r < nr && ((starts >> r) & 1u)) {
+                                            const unsigned len = (unsigned)__ffs((int)(starts >> (r + 1u)));     // rows up to the next start
+                                            bulk_g2s(smem_u32(A + (size_t)r * rb), (const void *)(cur.g_pool + (unsigned long long)rows4[k] * rb), len * rb, bar);
+                                        }
+                                    }
+                                }
+                            } else if (cur.flags & TF_ROWS) {
                                 // one copy per run of rows that are neighbours in the pool
                                 const unsigned rb = P.row_elems * 2u;
                                 const uint4 rv = *reinterpret_cast<const uint4 *>(sm.rows_ahead + ((size_t)ahead * 32u + (size_t)lane) * 4u);
@@ -976,6 +1059,23 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
                                 bulk_s2g((void *)d.g_scales, smem_u32(A + P.off_s), d.sbytes);
                         } else {
                             bulk_s2g((void *)d.g_chunk, smem_u32(A), d.n * 2u);
+                        }
+                    } else if (kWide && (d.flags & TF_ROWS)) {
+                        const unsigned rb = P.row_elems * 2u;
+                        const unsigned *rows = sm.rows_stage + (size_t)st * kWideRowsPerTile;
+                        const unsigned nr = d.runs >> 16;
+                        const unsigned starts = (d.runs & 0xffffu) | (1u << nr);
+                        for (unsigned b = 0; b < nr; b += 4u) {
+                            const uint4 rv = lds128(rows + b);
+                            const unsigned rows4[4] = { rv.x, rv.y, rv.z, rv.w };
+#pragma unroll
+                            for (unsigned k = 0; k < 4u; ++k) {
+                                const unsigned r = b + k;
+                                if (r < nr && ((starts >> r) & 1u)) {
+                                    const unsigned len = (unsigned)__ffs((int)(starts >> (r + 1u)));
+                                    bulk_s2g((void *)(d.g_pool + (unsigned long long)rows4[k] * rb), smem_u32(A + (size_t)r * rb), len * rb);
+                                }
+                            }
                         }
                     } else if (d.flags & TF_ROWS) {
                         const unsigned rb = P.row_elems * 2u;
@@ -1103,6 +1203,15 @@ __device__ __forceinline__ void tile_pipeline(const Launch &P)
 template <int kGroups, int kGW>
 __global__ void __launch_bounds__(threads_for(kGroups, kGW), min_ctas_for(kGroups, kGW))
 kdn_store_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_STORE, kGroups, kGW>(P); }
+
+// Store and retrieve for launches whose tiles take up to 16 token rows (keep-lists over short rows, dense ops on very
+// small pool blocks): the row indices stay in shared memory.  Built apart so that the ordinary kernels keep their registers.
+template <int kGroups, int kGW>
+__global__ void __launch_bounds__(threads_for(kGroups, kGW), min_ctas_for(kGroups, kGW))
+kdn_store_rows_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_STORE, kGroups, kGW, true>(P); }
+template <int kGroups, int kGW>
+__global__ void __launch_bounds__(threads_for(kGroups, kGW), min_ctas_for(kGroups, kGW))
+kdn_retrieve_rows_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_RETRIEVE, kGroups, kGW, true>(P); }
 
 // Sec. 3.2 call (ii) retrieve, Sec. 3.1 delivery module (decompression on the GPU): chunk -> pool.
 template <int kGroups, int kGW>

@@ -81,7 +81,7 @@ class kdn_td_layout_info(C.Structure):
 class kdn_launch_info(C.Structure):
     _fields_ = [("op", C.c_int32), ("compute_groups", C.c_int32), ("group_warps", C.c_int32), ("tile_bytes", C.c_int32),
                 ("stages", C.c_int32), ("ctas_per_sm", C.c_int32), ("store_lag", C.c_int32), ("grid", C.c_int32),
-                ("smem_bytes", C.c_int32), ("n_tiles", C.c_uint32)]
+                ("smem_bytes", C.c_int32), ("n_tiles", C.c_uint32), ("rows_per_tile", C.c_int32), ("rows_kernel", C.c_int32)]
 
 
 class kdn_tuning(C.Structure):
@@ -396,7 +396,8 @@ def kdn_last_launch(ctx) -> dict:
     info = kdn_launch_info()
     _check(lib.kdn_last_launch(ctx, C.byref(info)), "kdn_last_launch")
     d = {name: int(getattr(info, name)) for name, _ in kdn_launch_info._fields_}
-    d["kernel"] = "kdn_%s_kernel<%d, %d>" % (("store", "retrieve", "compose")[d["op"]], d["compute_groups"], d["group_warps"])
+    d["kernel"] = "kdn_%s%s_kernel<%d, %d>" % (("store", "retrieve", "compose")[d["op"]], "_rows" if d["rows_kernel"] else "",
+                                               d["compute_groups"], d["group_warps"])
     return d
 
 

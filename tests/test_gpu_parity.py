@@ -541,3 +541,47 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_recovers(codec):
         assert np.array_equal(dev.pool_np(), ref)
     finally:
         dev.close()
+
+
+@pytest.mark.parametrize("codec", [INT8, INT4])
+@pytest.mark.parametrize("bs,heads,head_dim", [(1, 8, 128), (2, 2, 128), (1, 2, 64), (4, 1, 64)])
+def test_coded_ops_on_pool_blocks_of_2_kib_or_less_run_as_token_rows(codec, bs, heads, head_dim):
+    """Pool blocks of at most 2 KiB: a coding tile that ends with its block would be tiny, so the launch takes whole
+    token rows, several per tile, wherever their blocks are.  Same bytes, same pool as any other dense op."""
+    shape = synth.TOY.with_(n_layers=2, n_kv_heads=heads, head_dim=head_dim, block_size=bs, n_blocks=2048)
+    dev = Device(shape, seed=83)
+    try:
+        K = dev.K
+        rng = np.random.default_rng(bs * 10 + codec)
+        host = dev.pool_np()
+        perm = rng.permutation(2048).astype(np.int32)
+        ops, metas, used = [], [], 0
+        for T, off in ((150, 0), (64, 3), (1, 0), (37, 5 * bs + 1), (257, 2)):
+            nb = -(-(off + T) // bs)
+            tab = perm[used:used + nb]
+            used += nb
+            buf = dev.chunk_buf(T, codec)
+            ops.append(dev.op(dev.table(tab), off, buf, T, codec))
+            metas.append((tab, off, T, buf))
+        dev.store(ops)
+        assert dev.sync() == 0
+        assert "rows" in K.kdn_last_launch(dev.ctx)["kernel"]
+        wants = [oracle.store(host, tab, off, T, codec) for tab, off, T, _ in metas]
+        for (tab, off, T, buf), want in zip(metas, wants):
+            assert np.array_equal(to_np(buf), want), (T, off)
+        assert np.array_equal(dev.pool_np(), host)
+        ref = host.copy()
+        rops = []
+        for (tab, off, T, buf), want in zip(metas, wants):
+            off2 = off + 1
+            nb = -(-(off2 + T) // bs)
+            dtab = perm[used:used + nb]
+            used += nb
+            rops.append(dev.op(dev.table(dtab), off2, buf, T, codec))
+            oracle.retrieve(ref, dtab, off2, T, codec, want)
+        dev.retrieve(rops)
+        assert dev.sync() == 0
+        assert "rows" in K.kdn_last_launch(dev.ctx)["kernel"]
+        assert np.array_equal(dev.pool_np(), ref)
+    finally:
+        dev.close()
