@@ -316,25 +316,40 @@ __global__ void __launch_bounds__(512) kdn_td_plan_kernel(const __grid_constant_
         const uint2 *hi_l = hi_tab + ((tid & 31u) >> 1);
         unsigned w02[2] = { 0u, 0u }, w1[2] = { 0u, 0u }, w35[2] = { 0u, 0u }, w46[2] = { 0u, 0u }, w7[2] = { 0u, 0u };
         int prev = 0;
-        for (unsigned t0 = 0; t0 < s.n_tok; t0 += 8u) {
-            unsigned al[2] = { 0u, 0u }, ah[2] = { 0u, 0u };
-            const unsigned t1 = t0 + 8u < s.n_tok ? t0 + 8u : s.n_tok;
-            for (unsigned t = t0; t < t1; ++t) {
-                const int q = td_code(*reinterpret_cast<const unsigned short *>(X + ((size_t)t * C + ch) * 2u), iv);
-                const unsigned u[2] = { td_zigzag(q), td_zigzag(q - prev) };        // at most 4 * 127 < 512
-                prev = q;
+        unsigned al[2], ah[2];
+        auto symbol = [&](unsigned t) {
+            const int q = td_code(*reinterpret_cast<const unsigned short *>(X + ((size_t)t * C + ch) * 2u), iv);
+            const unsigned u[2] = { td_zigzag(q), td_zigzag(q - prev) };        // at most 4 * 127 < 512
+            prev = q;
 #pragma unroll
-                for (int m = 0; m < 2; ++m) {
-                    al[m] += lo_l[(u[m] < 60u ? u[m] : 60u) << 5];
-                    const uint2 h = hi_l[(u[m] >> 3) << 4];
-                    ah[m] += h.x;
-                    w7[m] += h.y;
-                }
+            for (int m = 0; m < 2; ++m) {
+                al[m] += lo_l[(u[m] < 60u ? u[m] : 60u) << 5];
+                const uint2 h = hi_l[(u[m] >> 3) << 4];
+                ah[m] += h.x;
+                w7[m] += h.y;
             }
+        };
+        auto widen = [&]() {
 #pragma unroll
             for (int m = 0; m < 2; ++m) {
                 w02[m] += al[m] & 0x00ff00ffu; w1[m] += (al[m] >> 8) & 0x00ff00ffu;
                 w35[m] += ah[m] & 0x00ff00ffu; w46[m] += (ah[m] >> 8) & 0x00ff00ffu;
+            }
+        };
+        if (s.n_tok == 64u) {                                   // a full group: fixed trip counts, eight symbols unrolled
+#pragma unroll 1
+            for (unsigned t0 = 0; t0 < 64u; t0 += 8u) {
+                al[0] = al[1] = ah[0] = ah[1] = 0u;
+#pragma unroll
+                for (unsigned k = 0; k < 8u; ++k) symbol(t0 + k);
+                widen();
+            }
+        } else {
+            for (unsigned t0 = 0; t0 < s.n_tok; t0 += 8u) {
+                al[0] = al[1] = ah[0] = ah[1] = 0u;
+                const unsigned t1 = t0 + 8u < s.n_tok ? t0 + 8u : s.n_tok;
+                for (unsigned t = t0; t < t1; ++t) symbol(t);
+                widen();
             }
         }
         const unsigned b0[8] = { w02[0] & 0xffffu, w1[0] & 0xffffu, w02[0] >> 16, w35[0] & 0xffffu, w46[0] & 0xffffu, w35[0] >> 16, w46[0] >> 16, w7[0] };
@@ -467,6 +482,7 @@ __global__ void __launch_bounds__(512) kdn_td_encode_kernel(const __grid_constan
         unsigned nb = (addr & 3u) * 8u;                                   // ... after this many bits that are not its own
         unsigned long long acc = 0;
         int prev = 0;
+#pragma unroll 4
         for (unsigned t = 0; t < s.n_tok; ++t) {
             const int q = td_code(*reinterpret_cast<const unsigned short *>(X + ((size_t)t * C + tid) * 2u), iv);
             const unsigned u = td_zigzag(delta ? q - prev : q);
