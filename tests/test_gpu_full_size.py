@@ -327,3 +327,59 @@ def test_8b_token_delta_store_and_retrieve_16_chunks_of_512_tokens(codec):
         dev.close()
         del dev
         torch.cuda.empty_cache()
+
+
+@pytest.mark.parametrize("heads", [1, 2])
+def test_8b_pool_of_one_rank_of_a_head_sharded_engine(heads):
+    """What one rank of a tensor-parallel engine holds of the 8B shape: `heads` of the 8 KV heads, i.e. pool blocks of
+    4 or 8 KiB, in the launch configuration the benchmark's head-sharded leg times (512-token chunks, 2 GiB per launch,
+    fully fragmented tables).  Store then retrieve, raw and int8: pool blocks other than the destinations keep their
+    bits, raw is the identity, sampled chunks are checked element by element against the oracle."""
+    need_gib(24)
+    shape = synth.LLAMA3_8B.with_(n_kv_heads=heads, n_blocks=32768)
+    dev = Device(shape)
+    try:
+        K = dev.K
+        T, bs = 512, shape.block_size
+        nb = T // bs
+        n_req = (2 << 30) // (T * shape.elems_per_token * 2)
+        src = synth.make_table(n_req * nb, shape.n_blocks, 1, synth.SEED_TABLES).reshape(n_req, nb)
+        dst = synth.make_table(n_req * nb, shape.n_blocks, 1, synth.SEED_TABLES + 1, exclude=src.reshape(-1)).reshape(n_req, nb)
+        d_src, d_dst = dev.table(src.reshape(-1)), dev.table(dst.reshape(-1))
+        layers = list(range(shape.n_layers))
+        for codec in (RAW, INT8):
+            cb = K.kdn_chunk_bytes(dev.desc, T, codec)
+            big = torch.empty(n_req * cb, dtype=torch.uint8, device=dev.dev)
+            st = [K.XferOp(d_src.data_ptr() + i * nb * 4, nb, 0, K.Chunk(big.data_ptr() + i * cb, cb, T, codec)) for i in range(n_req)]
+            rt = [K.XferOp(d_dst.data_ptr() + i * nb * 4, nb, 0, K.Chunk(big.data_ptr() + i * cb, cb, T, codec)) for i in range(n_req)]
+            before = block_sums(dev)
+            dev.store(st)
+            assert dev.sync() == 0
+            info = K.kdn_last_launch(dev.ctx)
+            assert info["tile_bytes"] == bs * heads * shape.head_dim * 2            # a tile is one pool block
+            assert codec != RAW or info["ctas_per_sm"] >= 4                          # ... and in the copy form more CTAs keep the bytes in flight
+            assert torch.equal(block_sums(dev), before)
+            dev.retrieve(rt)
+            assert dev.sync() == 0
+            after = block_sums(dev)
+            keep = torch.ones(shape.n_blocks, dtype=torch.bool, device=dev.dev)
+            keep[torch.from_numpy(dst.reshape(-1).astype(np.int64)).to(dev.dev)] = False
+            assert torch.equal(after[:, keep], before[:, keep])
+            if codec == RAW:
+                si = torch.from_numpy(src.reshape(-1).astype(np.int64)).to(dev.dev)
+                di = torch.from_numpy(dst.reshape(-1).astype(np.int64)).to(dev.dev)
+                for t in dev.k + dev.v:
+                    assert torch.equal(t.index_select(0, si), t.index_select(0, di))
+            for i in (0, n_req // 3, n_req - 1):
+                sp = dev.pool_np(src[i], layers)
+                want = oracle.store(sp, np.arange(nb, dtype=np.int32), 0, T, codec)
+                assert np.array_equal(to_np(big[i * cb:(i + 1) * cb]), want), (codec, i)
+                ref = np.zeros_like(sp)
+                oracle.retrieve(ref, np.arange(nb, dtype=np.int32), 0, T, codec, want)
+                assert np.array_equal(dev.pool_np(dst[i], layers), ref), (codec, i)
+            del big
+            torch.cuda.empty_cache()
+    finally:
+        dev.close()
+        del dev
+        torch.cuda.empty_cache()
