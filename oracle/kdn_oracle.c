@@ -71,8 +71,11 @@
  *                    its R sub-streams back to back in channel order, and is padded with zero bytes to 16;
  *                    seg_off[S] = the bytes the chunk uses.  A chunk buffer has the worst-case capacity
  *                    fixed part + S * R * (72 or 40); bytes past seg_off[S] are not defined.
- *                    Decode: undo Rice, zigzag and the delta, then R5 with the channel's scale.  Token lists (R7)
- *                    are not defined for these codecs.
+ *                    Decode: undo Rice, zigzag and the delta, then R5 with the channel's scale.  With a keep-list
+ *                    (R7) the chunk's tokens are the listed ones: groups are 64 consecutive CHUNK tokens and mode 1
+ *                    differences a code from that of the listed token before it (the combination the paper's Sec. 3.2
+ *                    "KV-cache delivery" points to: drop tokens, then code what is left).  Select-lists are not
+ *                    defined for these codecs.
  *   R6  re-rotation  stored keys carry rotary position embedding at absolute
  *                    positions base_pos + t (what an engine's pool holds), so
  *                    reuse at dst_pos (Sec. 3.2 "KV-cache blending": a
@@ -454,7 +457,7 @@ static int check_args_list(const shape_t *s, const int32_t *table, int n_table, 
     if (n < 0 || off < 0 || n_table < 0) return 1;
     if (codec < KDN_ORACLE_RAW_BF16 || codec > KDN_ORACLE_INT4_TD64) return 3;
     if ((codec == KDN_ORACLE_INT8_KC64 || codec == KDN_ORACLE_INT4_KC64) && list) return 3;   /* R4": no token lists */
-    if (td_is(codec) && list) return 3;                                                       /* R9: no token lists */
+    if (td_is(codec) && list && list_bound >= 0) return 3;                                    /* R9: keep-lists only */
     if (codec != KDN_ORACLE_RAW_BF16 && s->D % KDN_ORACLE_GROUP) return 3;
     for (int i = 0; i < n; ++i) {
         int64_t rel = list ? list[i] : i;
@@ -532,7 +535,8 @@ static int store_kc(const shape_t *s, const uint16_t *pool, const int32_t *table
 }
 
 /* R9: store with K and V grouped along tokens, every group's codes written as a Rice-coded sub-stream. */
-static int store_td(const shape_t *s, const uint16_t *pool, const int32_t *table, int64_t off, int T, int codec, uint8_t *chunk)
+static int store_td(const shape_t *s, const uint16_t *pool, const int32_t *table, int64_t off, int T, int codec,
+                    const int32_t *keep, uint8_t *chunk)
 {
     int qmax = td_qmax(codec);
     size_t lay[6];
@@ -558,7 +562,7 @@ static int store_td(const shape_t *s, const uint16_t *pool, const int32_t *table
                         uint8_t bytes[72];
                         int len, param;
                         for (int i = 0; i < n; ++i) {
-                            int64_t p = off + t0 + i;
+                            int64_t p = off + (keep ? keep[t0 + i] : t0 + i);             /* R7: the listed tokens */
                             x[i] = pool[pool_index(s, l, kv, table[p / s->bs], (int)(p % s->bs), h, d)];
                         }
                         size_t ch = (size_t)h * (size_t)s->D + (size_t)d;
@@ -619,7 +623,7 @@ int kdn_oracle_store_sparse(const uint16_t *pool, int L, int H, int D, int bs, i
     size_t elems = (size_t)L * 2u * (size_t)T * (size_t)H * (size_t)D;
     if (codec == KDN_ORACLE_INT8_KC64 || codec == KDN_ORACLE_INT4_KC64)
         return store_kc(&s, pool, table, off, T, codec, chunk);
-    if (td_is(codec)) return store_td(&s, pool, table, off, T, codec, chunk);
+    if (td_is(codec)) return store_td(&s, pool, table, off, T, codec, keep, chunk);
     uint16_t *raw = (uint16_t *)chunk;
     int8_t *codes = (int8_t *)chunk;
     float *scales = (float *)(chunk + (codec == KDN_ORACLE_INT4_G64 ? elems / 2u : elems));

@@ -261,11 +261,58 @@ def test_retrieve_and_compose_equal_the_per_channel_key_codec_on_keys(codec, kc)
     assert np.array_equal(ka[:, 5:5 + T], kb[:, 5:5 + T])
 
 
-def test_token_lists_are_refused():
+@pytest.mark.parametrize("codec", [TD8, TD4])
+def test_keep_list_chunk_is_the_chunk_of_the_listed_tokens(codec):
+    """A keep-list chunk (R9 with R7) is, byte for byte, the dense chunk of a pool in which the listed tokens sit side by
+    side: groups are 64 consecutive CHUNK tokens and a difference is taken from the listed token before.  Walked by hand
+    as well: every group's codes are the per-channel quantiser's of the listed rows.  Retrieve writes the listed
+    positions, each with what the dense retrieve of the compacted pool gives, and nothing else."""
+    shape = synth.TOY.with_(n_layers=2, n_kv_heads=2, head_dim=64, block_size=4, n_blocks=64)
+    k, v = synth.make_pool(shape, "cpu", seed=27)
+    pool = synth.pool_to_numpy(k, v)
+    L, H, D, bs = shape.n_layers, shape.n_kv_heads, shape.head_dim, shape.block_size
+    rng = np.random.default_rng(4)
+    table = rng.permutation(64)[:40].astype(np.int32)                     # 160 positions
+    off = 3
+    keep = np.sort(rng.choice(150, 100, replace=False)).astype(np.int32)  # two groups: 64 + 36 chunk tokens
+    T = len(keep)
+    chunk = oracle.store(pool, table, off, T, codec, keep=keep)
+    # the same tokens side by side in another pool, stored densely
+    pos = off + keep
+    packed = np.zeros_like(pool)
+    ptab = np.arange(-(-T // bs), dtype=np.int32)
+    t = np.arange(T)
+    packed[:, :, ptab[t // bs], t % bs] = pool[:, :, table[pos // bs], pos % bs]
+    assert np.array_equal(chunk, oracle.store(packed, ptab, 0, T, codec))
+    groups, used = walk_chunk(chunk, L, H, D, T, codec)
+    x = pool[:, :, table[pos // bs], pos % bs].reshape(L, 2, T, H * D)
+    for (l, kv, g, ch), (scale, codes) in groups.items():
+        q, sc = oracle.quant_channel(x[l, kv, 64 * g:64 * g + 64, ch], QMAX[codec])
+        assert np.float32(sc).view(np.uint32) == np.float32(scale).view(np.uint32) and list(q) == codes
+    # with every position listed the list changes nothing
+    assert np.array_equal(oracle.store(pool, table, off, 150, codec, keep=np.arange(150)), oracle.store(pool, table, off, 150, codec))
+    # retrieve
+    dtab = rng.permutation(64)[:40].astype(np.int32)
+    got = np.full_like(pool, 0x1234)
+    oracle.retrieve(got, dtab, off, T, codec, chunk, keep=keep)
+    dense = np.zeros_like(pool)
+    oracle.retrieve(dense, ptab, 0, T, codec, chunk)
+    want = np.full_like(pool, 0x1234)
+    want[:, :, dtab[pos // bs], pos % bs] = dense[:, :, ptab[t // bs], t % bs]
+    assert np.array_equal(got, want)
+
+
+def test_select_lists_are_refused():
+    """Select-lists (compose of some tokens of a part) are not defined for these codecs; a keep-list that is not
+    strictly increasing is refused as for every codec."""
     k, v = synth.make_pool(synth.TOY, "cpu")
     pool = synth.pool_to_numpy(k, v)
+    tab = np.arange(4, dtype=np.int32)
+    chunk = oracle.store(pool, tab, 0, 8, TD8)
     with pytest.raises(ValueError):
-        oracle.store(pool, np.arange(4, dtype=np.int32), 0, 3, TD8, keep=[0, 2, 5])
+        oracle.compose(pool.copy(), tab, [(chunk, 8, TD8, 0, 0)], 10000.0, select=[[0, 2, 5]])
+    with pytest.raises(ValueError):
+        oracle.store(pool, tab, 0, 3, TD8, keep=[0, 5, 2])
 
 
 def ar1(rng, n_tokens, n_channels, rho):
