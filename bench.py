@@ -622,6 +622,29 @@ def extras_8b(leg, dev_sets, reps, which=EXTRAS):
                     "from_host_ms": host_ms, "from_host_link_gbs": used / (host_ms * 1e-3) / 1e9,
                     "from_host_bf16_gbs_delivered": bf16_bytes / (host_ms * 1e-3) / 1e9}
                 del buf
+                if codec == INT4TD:
+                    # the same chunks holding only half of their tokens (a seeded random keep-list per chunk): token dropping
+                    # and coding together, against the bf16 bytes of the whole span
+                    n_keep = T // 2
+                    rng = np.random.default_rng(11)
+                    keep = torch.from_numpy(np.stack([np.sort(rng.choice(T, n_keep, replace=False)) for _ in range(n_td)]).astype(np.int32)).to(dev)
+                    keeps = [keep.data_ptr() + c * n_keep * i32 for c in range(n_td)]
+                    cbk = K.kdn_chunk_bytes(desc, n_keep, codec)
+                    layk = K.kdn_td_layout(desc, n_keep, codec)
+                    bufk = torch.empty(n_td * cbk, dtype=torch.uint8, device=dev)
+                    sk = [K.XferOp(leg.d_src.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(bufk.data_ptr() + c * cbk, cbk, n_keep, codec)) for c in range(n_td)]
+                    rk = [K.XferOp(leg.d_dst.data_ptr() + c * bpc * i32, bpc, 0, K.Chunk(bufk.data_ptr() + c * cbk, cbk, n_keep, codec)) for c in range(n_td)]
+                    ms_sk = leg.timed(lambda: K.kdn_store_sparse(ctx, pid, sk, keeps, s), min(reps, 5), warm=2)
+                    leg.check()
+                    usedk = sum(int(bufk[c * cbk + 8 * layk["segments"]:c * cbk + 8 * layk["segments"] + 8].view(torch.int64).item()) for c in range(n_td))
+                    ms_rk = leg.timed(lambda: K.kdn_retrieve_sparse(ctx, pid, rk, keeps, s), min(reps, 5), warm=2)
+                    leg.check()
+                    td["%s_rho_%s" % (cname, rho)]["half_of_the_tokens_kept"] = {
+                        "chunk_bytes_used": usedk, "bits_per_kept_element": 8.0 * usedk / (n_td * n_keep * E),
+                        "smaller_than_bf16_of_the_whole_span_by": bf16_bytes / usedk,
+                        "store_ms": ms_sk, "retrieve_ms": ms_rk, "retrieve_kept_tokens_per_s": n_td * n_keep / (ms_rk * 1e-3),
+                        "retrieve_gbs": (usedk + bf16_bytes / 2) / (ms_rk * 1e-3) / 1e9}
+                    del bufk, keep
             torch.cuda.empty_cache()
         td["what"] = ("%d chunks x %d tokens; GB/s counts the bytes the chunks use plus the bf16 bytes on the pool side; "
                       "rho = correlation of neighbouring tokens in the synthetic input" % (n_td, T))
@@ -923,6 +946,8 @@ def run_gpu(args) -> None:
                 wide["td_" + n] = {"x_smaller": round(v["smaller_than_bf16_by"], 2), "store": round(v["store_gbs"], 1),
                                    "retrieve": round(v["retrieve_gbs"], 1), "compose": round(v["compose_gbs"], 1),
                                    "host_bf16_gbs": round(v["from_host_bf16_gbs_delivered"], 1)}
+                if "half_of_the_tokens_kept" in v:
+                    wide["td_" + n]["x_smaller_with_half_of_the_tokens_kept"] = round(v["half_of_the_tokens_kept"]["smaller_than_bf16_of_the_whole_span_by"], 2)
         if wide:
             per_op["widenings_8b"] = wide
         frac = gbs[top] / peak

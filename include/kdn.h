@@ -64,7 +64,11 @@
  *   the chunk uses, which is what has to be kept or sent.  kdn_chunk_bytes gives the worst-case CAPACITY (a sub-stream
  *   never exceeds 72 or 40 bytes) and chunk.bytes must equal it; bytes past seg_off[S] are not written and not read
  *   (up to 15 beyond it may be read, never past the capacity).  kdn_td_layout gives the offsets.
- *   Same restrictions as the per-channel key codecs.  kdn_store writes KDN_MEM_DEVICE chunks only (the size of the
+ *   Same restrictions as the per-channel key codecs, except for keep-lists: kdn_store_sparse and kdn_retrieve_sparse
+ *   take these codecs (the chunk then codes the LISTED tokens: groups are 64 consecutive chunk tokens, mode 1 differences
+ *   a code from that of the listed token before it; no rule on token_offset or block_size, every row is found through
+ *   its own table entry).  Dropping half of the tokens and coding the rest is what brings a chunk below a tenth of its
+ *   span's bf16 bytes on token-correlated input.  kdn_store writes KDN_MEM_DEVICE chunks only (the size of the
  *   result is not known before the kernels have run); kdn_retrieve and kdn_compose also take KDN_MEM_PINNED_HOST
  *   chunks: the library reads seg_off[S] from host memory and copies just the bytes in use over the host link (a
  *   chunk whose bytes in use exceed a staging slab, or whose offset table no store can have written, is refused).

@@ -857,8 +857,8 @@ HostOp make_host_op(const Pool &pool, const int32_t *table, int32_t n_table, int
     h.op.nl = pool.L;
     h.op.pos_end = (long long)n_table * pool.bs;
     const size_t elems = (size_t)pool.L * 2u * (size_t)c.n_tokens * (size_t)pool.H * (size_t)pool.D;
-    if (is_td(c.codec))       // token lists do not exist for these codecs: pos_end carries the bytes the kernels may read
-        h.op.pos_end = (long long)td_layout(pool.L, (unsigned)pool.H * (unsigned)pool.D, c.n_tokens, c.codec).capacity;
+    if (is_td(c.codec))       // these codecs keep their scales inside the chunk: the field points behind the bytes that exist
+        h.op.scales = (unsigned char *)c.data + td_layout(pool.L, (unsigned)pool.H * (unsigned)pool.D, c.n_tokens, c.codec).capacity;
     if (c.codec != KDN_CODEC_RAW_BF16 && !is_td(c.codec)) h.op.scales = (unsigned char *)c.data + (is_int4(c.codec) ? elems / 2u : elems);
     return h;
 }
@@ -1023,7 +1023,10 @@ kdn_status run_td_host(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector
             KDN_CUDA(cudaMemcpyAsync(ctx->slab[s] + p.slab_off, p.host, p.bytes, cudaMemcpyHostToDevice, side));
         KDN_CUDA(cudaEventRecord(ctx->slab_ready[s], side));
         KDN_CUDA(cudaStreamWaitEvent(stream, ctx->slab_ready[s], 0));
-        for (HostOp &h : batch) h.op.data = ctx->slab[s] + (size_t)(uintptr_t)h.op.data;      // offsets become addresses
+        for (HostOp &h : batch) {                                                             // offsets become addresses
+            h.op.data = ctx->slab[s] + (size_t)(uintptr_t)h.op.data;
+            h.op.scales = ctx->slab[s] + (size_t)(uintptr_t)h.op.scales;
+        }
         kdn_status r = launch_td(ctx, pool, OP, batch.data(), (int)batch.size(), stream);
         if (r != KDN_OK) return r;
         KDN_CUDA(cudaEventRecord(ctx->slab_free[s], stream));
@@ -1047,7 +1050,7 @@ kdn_status run_td_host(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector
         pieces.push_back(Piece{ h.op.data, fill, (size_t)used, -1, 0 });
         HostOp sub = h;
         sub.op.data = (unsigned char *)(uintptr_t)fill;      // offset inside the slab until the slab is known
-        sub.op.pos_end = (long long)used;                    // the slab holds no more of the chunk than this
+        sub.op.scales = (unsigned char *)(uintptr_t)(fill + (size_t)used);   // the slab holds no more of the chunk than this
         batch.push_back(sub);
         fill = (fill + (size_t)used + 255) & ~(size_t)255;
     }
@@ -1182,7 +1185,8 @@ kdn_status xfer_sparse(kdn_ctx *ctx, int pool_id, int OP, const kdn_sparse_op *o
         const kdn_xfer_op &o = ops[i].op;
         st = check_chunk(&shape, &o.chunk);
         if (st != KDN_OK) return st;
-        if (is_kc(o.chunk.codec) || is_td(o.chunk.codec)) return KDN_E_UNSUPPORTED;   // a keep-list breaks up the 64-token groups
+        if (is_kc(o.chunk.codec)) return KDN_E_UNSUPPORTED;   // a keep-list breaks up the 64-token groups of the key planes
+        // (the token-delta codecs group the chunk's own tokens, listed or not)
         if (o.n_table_blocks < 0 || o.token_offset < 0) return KDN_E_INVAL;
         if (o.chunk.n_tokens > 0 && (!o.block_table || !ops[i].keep)) return KDN_E_INVAL;
         // the listed tokens are distinct positions below the end of the table, so there cannot be more of them

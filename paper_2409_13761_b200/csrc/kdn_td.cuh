@@ -130,22 +130,35 @@ __device__ __forceinline__ unsigned td_block_scan(unsigned v, unsigned *scratch,
     return r;
 }
 
+// Request position of row t of group g of an op: off + 64 g + t, or, for a keep-list op, off + list[64 g + t].
+// Returns -1 for a list entry that is negative or points past the block table.
+__device__ __forceinline__ long long td_row_pos(const DevOp &op, unsigned g, unsigned t)
+{
+    const unsigned i = (g << 6) + t;
+    if (op.list_mode == 0) return op.off + (long long)i;
+    const long long rel = __ldg(op.list + i);
+    const long long p = op.off + rel;
+    return (rel < 0 || p >= op.pos_end) ? -1ll : p;
+}
+
 // Bring the slice [c0, c0 + C) of the n_tok token rows of one group (request positions pos0 ..) of a pool plane
 // into X[n_tok][C] with bulk copies counted on `bar`.  Warp 0 calls this; returns false (and records KDN_E_RANGE)
 // when a block id lies outside the pool, in which case nothing was issued.
-__device__ __forceinline__ bool td_load_slice(unsigned char *X, uint32_t bar, const unsigned char *base, const int32_t *table,
-                                              long long pos0, unsigned n_tok, int bs, long long n_blocks, unsigned RE,
+__device__ __forceinline__ bool td_load_slice(unsigned char *X, uint32_t bar, const unsigned char *base, const DevOp &op, unsigned g,
+                                              unsigned n_tok, int bs, long long n_blocks, unsigned RE,
                                               unsigned C, unsigned c0, bool whole_row, int *status)
 {
     const unsigned lane = threadIdx.x & 31u;
-    const long long first_block = pos0 / bs;
-    long long id[2] = { 0, 0 };
+    const int32_t *table = op.table;
+    long long id[2] = { 0, 0 }, pos[2] = { 0, 0 };
     bool bad = false;
 #pragma unroll
     for (int k = 0; k < 2; ++k) {
         const unsigned t = lane + 32u * (unsigned)k;
         if (t < n_tok) {
-            id[k] = __ldg(table + first_block + t / (unsigned)bs);
+            pos[k] = td_row_pos(op, g, t);
+            if (pos[k] < 0) { bad = true; continue; }
+            id[k] = __ldg(table + pos[k] / bs);
             if (id[k] < 0 || id[k] >= n_blocks) bad = true;
         }
     }
@@ -155,9 +168,11 @@ __device__ __forceinline__ bool td_load_slice(unsigned char *X, uint32_t bar, co
     }
     if (lane == 0) mbar_arrive_expect_tx(bar, n_tok * C * 2u);
     __syncwarp();
-    if (whole_row) {
-        // a block's tokens are contiguous in the pool: one copy per block (pieces <= 32 KiB)
+    if (whole_row && op.list_mode == 0) {
+        // a block's tokens are contiguous in the pool: one copy per block (pieces <= 32 KiB); the host sees to it that
+        // the group starts at a block start
         if (lane == 0) {
+            const long long first_block = (op.off + (long long)(g << 6)) / bs;
             for (unsigned t = 0; t < n_tok; t += (unsigned)bs) {
                 const unsigned k = n_tok - t < (unsigned)bs ? n_tok - t : (unsigned)bs;
                 const long long b = __ldg(table + first_block + t / (unsigned)bs);
@@ -172,9 +187,10 @@ __device__ __forceinline__ bool td_load_slice(unsigned char *X, uint32_t bar, co
         for (int k = 0; k < 2; ++k) {
             const unsigned t = lane + 32u * (unsigned)k;
             if (t < n_tok) {
-                const unsigned slot = (unsigned)((pos0 + t) % bs);
+                const unsigned slot = (unsigned)(pos[k] % bs);
                 const unsigned char *src = base + (((unsigned long long)id[k] * bs + slot) * RE + c0) * 2ull;
-                bulk_g2s(smem_u32(X + (size_t)t * C * 2u), src, C * 2u, bar);
+                for (unsigned o = 0; o < C * 2u; o += 32768u)              // (a slice is at most 1024 channels: one piece)
+                    bulk_g2s(smem_u32(X + (size_t)t * C * 2u + o), src + o, C * 2u - o < 32768u ? C * 2u - o : 32768u, bar);
             }
         }
     }
@@ -272,7 +288,7 @@ __global__ void __launch_bounds__(512) kdn_td_plan_kernel(const __grid_constant_
     __syncthreads();
     if (tid < 32) {
         const unsigned char *base = reinterpret_cast<const unsigned char *>((s.kv ? P.v_layers : P.k_layers)[s.op.l0 + (int)s.li]);
-        if (!td_load_slice(X, bar, base, s.op.table, s.op.off + (long long)(s.g << 6), s.n_tok, P.bs, P.n_blocks, RE, C, s.c0,
+        if (!td_load_slice(X, bar, base, s.op, s.g, s.n_tok, P.bs, P.n_blocks, RE, C, s.c0,
                            P.n_split == 1u, P.status) && tid == 0)
             *abort_flag = 1;
     }
@@ -439,7 +455,7 @@ __global__ void __launch_bounds__(512) kdn_td_encode_kernel(const __grid_constan
     __syncthreads();
     if (tid < 32) {
         const unsigned char *base = reinterpret_cast<const unsigned char *>((s.kv ? P.v_layers : P.k_layers)[s.op.l0 + (int)s.li]);
-        if (!td_load_slice(X, bar, base, s.op.table, s.op.off + (long long)(s.g << 6), s.n_tok, P.bs, P.n_blocks, RE, C, s.c0,
+        if (!td_load_slice(X, bar, base, s.op, s.g, s.n_tok, P.bs, P.n_blocks, RE, C, s.c0,
                            P.n_split == 1u, P.status) && tid == 0)
             *abort_flag = 1;
     }
@@ -570,8 +586,10 @@ __global__ void __launch_bounds__(kCols ? kCols : 512) kdn_td_decode_kernel(cons
     const unsigned shift = (unsigned)(((unsigned long long)s.op.data + src) & 15ull);
     const unsigned bytes_al = (shift + total_slice + 15u) & ~15u;
     // a damaged chunk must not send a copy outside the chunk or outside the staging area
-    // (op.pos_end: the bytes of the chunk that exist at op.data -- its capacity, or what a staging slab holds of it)
-    const unsigned long long have = (unsigned long long)s.op.pos_end < lay.capacity ? (unsigned long long)s.op.pos_end : lay.capacity;
+    // (op.scales, which these codecs have no other use for, points behind the bytes of the chunk that exist at op.data:
+    // its capacity, or what a staging slab holds of it)
+    const unsigned long long exist = (unsigned long long)(s.op.scales - s.op.data);
+    const unsigned long long have = exist < lay.capacity ? exist : lay.capacity;
     const bool sane = total_slice <= C * td_max_len(codec) && src >= lay.streams && src - shift + bytes_al <= have;
     if (tid == 0) {
         if (!sane) {
@@ -665,23 +683,24 @@ __global__ void __launch_bounds__(kCols ? kCols : 512) kdn_td_decode_kernel(cons
     // rows -> pool blocks
     if (tid < 32) {
         unsigned char *base = reinterpret_cast<unsigned char *>((s.kv ? P.v_layers : P.k_layers)[s.op.l0 + (int)s.li]);
-        const long long pos0 = s.op.off + (long long)(s.g << 6);
-        const long long first_block = pos0 / P.bs;
-        long long id[2] = { 0, 0 };
+        long long id[2] = { 0, 0 }, pos[2] = { 0, 0 };
         bool bad = false;
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
             const unsigned t = tid + 32u * (unsigned)k;
             if (t < s.n_tok) {
-                id[k] = __ldg(s.op.table + first_block + t / (unsigned)P.bs);
+                pos[k] = td_row_pos(s.op, s.g, t);
+                if (pos[k] < 0) { bad = true; continue; }
+                id[k] = __ldg(s.op.table + pos[k] / P.bs);
                 if (id[k] < 0 || id[k] >= P.n_blocks) bad = true;
             }
         }
         if (__any_sync(0xffffffffu, bad)) {
             if (tid == 0) atomicCAS(P.status, 0, kStatusRange);        // nothing of this slice is written
         } else {
-            if (P.n_split == 1u) {
+            if (P.n_split == 1u && s.op.list_mode == 0) {
                 if (tid == 0) {
+                    const long long first_block = (s.op.off + (long long)(s.g << 6)) / P.bs;
                     for (unsigned t = 0; t < s.n_tok; t += (unsigned)P.bs) {
                         const unsigned k = s.n_tok - t < (unsigned)P.bs ? s.n_tok - t : (unsigned)P.bs;
                         const long long b = __ldg(s.op.table + first_block + t / (unsigned)P.bs);
@@ -696,7 +715,7 @@ __global__ void __launch_bounds__(kCols ? kCols : 512) kdn_td_decode_kernel(cons
                 for (int k = 0; k < 2; ++k) {
                     const unsigned t = tid + 32u * (unsigned)k;
                     if (t < s.n_tok) {
-                        const unsigned slot = (unsigned)((pos0 + t) % P.bs);
+                        const unsigned slot = (unsigned)(pos[k] % P.bs);
                         unsigned char *d = base + (((unsigned long long)id[k] * P.bs + slot) * RE + s.c0) * 2ull;
                         bulk_s2g(d, smem_u32(A + (size_t)t * C * 2u), C * 2u);
                     }

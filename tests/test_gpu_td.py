@@ -174,7 +174,8 @@ def test_refusals_and_damaged_chunks():
         buf = dev.chunk_buf(T, TD8)
         for bad in (lambda: dev.store([dev.op(tab, 3, buf, T, TD8)]),                       # first token not at a block start
                     lambda: dev.store([dev.op(tab, 0, dev.chunk_buf(T, TD8, pinned=True), T, TD8)]),   # store into host memory
-                    lambda: K.kdn_store_sparse(dev.ctx, dev.pool_id, [dev.op(tab, 0, buf, T, TD8)], [tab.data_ptr()], dev.stream.cuda_stream)):
+                    lambda: K.kdn_compose_select(dev.ctx, dev.pool_id, [K.ComposeReq(tab.data_ptr(), 8, [dev.chunk(buf, T, TD8)], [0], 1e4)],
+                                                 [[(tab.data_ptr(), 4)]], dev.stream.cuda_stream)):   # select-lists
             with pytest.raises(K.KdnError) as e:
                 bad()
             assert e.value.status == K.KDN_E_UNSUPPORTED
@@ -272,5 +273,60 @@ def test_retrieve_and_compose_from_page_locked_host_chunks(codec):
         with pytest.raises(K.KdnError) as e:
             dev.retrieve([dev.op(dev.table(dsts[0]), 0, junk, 64, codec)])
         assert e.value.status == K.KDN_E_SHAPE
+    finally:
+        dev.close()
+
+
+@pytest.mark.parametrize("shape", SHAPES, ids=IDS)
+@pytest.mark.parametrize("codec", [TD8, TD4], ids=["int8td", "int4td"])
+def test_keep_list_chunks_against_the_oracle(shape, codec):
+    """Keep-lists with the token-delta codecs: the chunk codes the listed tokens (groups of 64 chunk tokens, differences
+    along the listed tokens), wherever they sit in the request -- no alignment rule.  Store bytes, retrieve into other
+    blocks (device and page-locked host chunk), and a list entry outside the table."""
+    bs = shape.block_size
+    rng = np.random.default_rng(23 + codec)
+    perm = rng.permutation(shape.n_blocks).astype(np.int32)
+    span, off = 200, 3
+    nb = -(-(off + span) // bs)
+    src, dst = perm[:nb], perm[nb:2 * nb]
+    pool = make_pool_np(shape, src, off, span, 0.95, seed=41)
+    dev = Device(shape, pool_np=pool)
+    try:
+        K = dev.K
+        lists = [np.sort(rng.choice(span, 100, replace=False)), np.arange(span), np.array([7]), np.arange(0, span, 3), np.arange(64) + 5]
+        ops, keeps, wants, bufs = [], [], [], []
+        for keep in lists:
+            keep = keep.astype(np.int32)
+            b = dev.chunk_buf(len(keep), codec)
+            d_keep = dev.table(keep)
+            ops.append(dev.op(dev.table(src), off, b, len(keep), codec))
+            keeps.append(d_keep.data_ptr())
+            wants.append(oracle.store(pool, src, off, len(keep), codec, keep=keep))
+            bufs.append(b)
+        K.kdn_store_sparse(dev.ctx, dev.pool_id, ops, keeps, dev.stream.cuda_stream)
+        assert dev.sync() == 0
+        for b, w, keep in zip(bufs, wants, lists):
+            used = oracle.td_used_bytes(w, shape.n_layers, shape.n_kv_heads, shape.head_dim, len(keep), codec)
+            got = to_np(b)
+            assert np.array_equal(got[:used], w[:used]) and np.all(got[used:] == 0xA5), len(keep)
+        assert np.array_equal(dev.pool_np(), pool)
+        ref = pool.copy()
+        for i, (b, w, keep) in enumerate(zip(bufs, wants, lists)):
+            src_buf = b
+            if i % 2 == 1:                                                       # every other chunk from page-locked host memory
+                src_buf = dev.chunk_buf(len(keep), codec, pinned=True)
+                src_buf.copy_(b.cpu())
+            K.kdn_retrieve_sparse(dev.ctx, dev.pool_id, [dev.op(dev.table(dst), off, src_buf, len(keep), codec)], [keeps[i]], dev.stream.cuda_stream)
+            assert dev.sync() == 0
+            oracle.retrieve(ref, dst, off, len(keep), codec, w, keep=keep.astype(np.int32))
+            assert np.array_equal(dev.pool_np(), ref), i
+        bad = np.array([0, 1, 2, nb * bs], dtype=np.int32)                        # the last entry points past the table
+        b = dev.chunk_buf(4, codec)
+        K.kdn_store_sparse(dev.ctx, dev.pool_id, [dev.op(dev.table(src), 0, b, 4, codec)], [dev.table(bad).data_ptr()], dev.stream.cuda_stream)
+        assert dev.sync() == K.KDN_E_RANGE
+        K.kdn_retrieve_sparse(dev.ctx, dev.pool_id, [dev.op(dev.table(dst), 0, bufs[2], 1, codec)], [dev.table(np.array([nb * bs + 5], dtype=np.int32)).data_ptr()],
+                              dev.stream.cuda_stream)
+        assert dev.sync() == K.KDN_E_RANGE
+        assert np.array_equal(dev.pool_np(), ref)
     finally:
         dev.close()
