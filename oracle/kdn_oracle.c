@@ -46,7 +46,8 @@
  *                    V planes: exactly R4 / R4'.  Codes lie where R2 / R4' put them.  Scales, per layer:
  *                    fp32 k_scales[ceil(T/64)][head*D] followed by fp32 v_scales[t][head*D/64]; layers follow
  *                    each other; the scales follow the codes.  Decode is R5 with the element's own scale.
- *                    Token lists (R7) are not defined for these codecs.
+ *                    With a keep-list (R7) the chunk's tokens are the listed ones and a key group is 64 consecutive
+ *                    CHUNK tokens, as for R9; select-lists are not defined for these codecs.
  *   R9  token-delta Rice codecs (codecs 5 = int8, 6 = int4; not prescribed by the paper: Sec. 3.2 "KV-cache delivery"
  *                    cites a scheme that quantises a KV cache and then encodes it into binary strings, and reports
  *                    more than tenfold reductions for combined techniques.  This is this library's own bitstream.)
@@ -456,7 +457,7 @@ static int check_args_list(const shape_t *s, const int32_t *table, int n_table, 
     if (s->L <= 0 || s->H <= 0 || s->D <= 0 || s->bs <= 0 || s->nb <= 0) return 1;
     if (n < 0 || off < 0 || n_table < 0) return 1;
     if (codec < KDN_ORACLE_RAW_BF16 || codec > KDN_ORACLE_INT4_TD64) return 3;
-    if ((codec == KDN_ORACLE_INT8_KC64 || codec == KDN_ORACLE_INT4_KC64) && list) return 3;   /* R4": no token lists */
+    if ((codec == KDN_ORACLE_INT8_KC64 || codec == KDN_ORACLE_INT4_KC64) && list && list_bound >= 0) return 3;   /* R4": keep-lists only */
     if (td_is(codec) && list && list_bound >= 0) return 3;                                    /* R9: keep-lists only */
     if (codec != KDN_ORACLE_RAW_BF16 && s->D % KDN_ORACLE_GROUP) return 3;
     for (int i = 0; i < n; ++i) {
@@ -490,7 +491,8 @@ static void put_code(uint8_t *chunk, int int4, size_t c, int8_t q)
 }
 
 /* R4": store with keys grouped along tokens and values grouped along head_dim. */
-static int store_kc(const shape_t *s, const uint16_t *pool, const int32_t *table, int64_t off, int T, int codec, uint8_t *chunk)
+static int store_kc(const shape_t *s, const uint16_t *pool, const int32_t *table, int64_t off, int T, int codec,
+                    const int32_t *keep, uint8_t *chunk)
 {
     int int4 = codec == KDN_ORACLE_INT4_KC64;
     int qmax = int4 ? 7 : 127;
@@ -507,7 +509,7 @@ static int store_kc(const shape_t *s, const uint16_t *pool, const int32_t *table
                     uint16_t x[KDN_ORACLE_GROUP];
                     int8_t q[KDN_ORACLE_GROUP];
                     for (int i = 0; i < n; ++i) {
-                        int64_t p = off + t0 + i;
+                        int64_t p = off + (keep ? keep[t0 + i] : t0 + i);                 /* R7: the listed tokens */
                         x[i] = pool[pool_index(s, l, 0, table[p / s->bs], (int)(p % s->bs), h, d)];
                     }
                     size_t ch = (size_t)h * (size_t)s->D + (size_t)d;
@@ -517,7 +519,7 @@ static int store_kc(const shape_t *s, const uint16_t *pool, const int32_t *table
         }
         /* values: R4 / R4' */
         for (int t = 0; t < T; ++t) {
-            int64_t p = off + t;
+            int64_t p = off + (keep ? keep[t] : t);
             int64_t block = table[p / s->bs];
             int slot = (int)(p % s->bs);
             for (int h = 0; h < s->H; ++h)
@@ -622,7 +624,7 @@ int kdn_oracle_store_sparse(const uint16_t *pool, int L, int H, int D, int bs, i
     if (rc) return rc;
     size_t elems = (size_t)L * 2u * (size_t)T * (size_t)H * (size_t)D;
     if (codec == KDN_ORACLE_INT8_KC64 || codec == KDN_ORACLE_INT4_KC64)
-        return store_kc(&s, pool, table, off, T, codec, chunk);
+        return store_kc(&s, pool, table, off, T, codec, keep, chunk);
     if (td_is(codec)) return store_td(&s, pool, table, off, T, codec, keep, chunk);
     uint16_t *raw = (uint16_t *)chunk;
     int8_t *codes = (int8_t *)chunk;

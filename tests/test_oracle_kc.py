@@ -182,9 +182,41 @@ def test_compose_rotates_the_unrounded_stored_key(codec, base, qmax):
 
 
 @pytest.mark.parametrize("codec,base,qmax", KC)
-def test_token_lists_are_refused(codec, base, qmax):
-    shape = synth.TOY.with_(n_blocks=8)
-    k, v = synth.make_pool(shape, "cpu", seed=1)
+def test_keep_list_chunk_is_the_chunk_of_the_listed_tokens(codec, base, qmax):
+    """A keep-list chunk is, byte for byte, the dense chunk of a pool in which the listed tokens sit side by side (key
+    groups are 64 consecutive CHUNK tokens), its codes and scales are the second formulation's on the listed rows, and
+    retrieve writes the listed positions with what the dense retrieve of that pool gives, nothing else.  Select-lists
+    stay refused."""
+    shape = synth.TOY.with_(n_layers=2, n_kv_heads=2, head_dim=64, block_size=4, n_blocks=64)
+    k, v = synth.make_pool(shape, "cpu", seed=29)
     pool = synth.pool_to_numpy(k, v)
+    L, H, D, bs = shape.n_layers, shape.n_kv_heads, shape.head_dim, shape.block_size
+    rng = np.random.default_rng(6)
+    table = rng.permutation(64)[:40].astype(np.int32)
+    off = 2
+    keep = np.sort(rng.choice(150, 100, replace=False)).astype(np.int32)
+    T = len(keep)
+    chunk = oracle.store(pool, table, off, T, codec, keep=keep)
+    pos = off + keep
+    t = np.arange(T)
+    ptab = np.arange(-(-T // bs), dtype=np.int32)
+    packed = np.zeros_like(pool)
+    packed[:, :, ptab[t // bs], t % bs] = pool[:, :, table[pos // bs], pos % bs]
+    assert np.array_equal(chunk, oracle.store(packed, ptab, 0, T, codec))
+    codes, k_sc, _ = split_chunk(chunk, L, T, H, D, codec)
+    x = pool[:, :, table[pos // bs], pos % bs].reshape(L, 2, T, H * D)
+    for l in range(L):
+        for g in range(-(-T // 64)):
+            q, sc = second_formulation(x[l, 0, 64 * g:64 * g + 64], qmax)
+            assert np.array_equal(codes[l, 0, 64 * g:64 * g + 64], q)
+            assert np.array_equal(k_sc[l, g].view(np.uint32), sc.astype(np.float32).view(np.uint32))
+    dtab = rng.permutation(64)[:40].astype(np.int32)
+    got = np.full_like(pool, 0x1234)
+    oracle.retrieve(got, dtab, off, T, codec, chunk, keep=keep)
+    dense = np.zeros_like(pool)
+    oracle.retrieve(dense, ptab, 0, T, codec, chunk)
+    want = np.full_like(pool, 0x1234)
+    want[:, :, dtab[pos // bs], pos % bs] = dense[:, :, ptab[t // bs], t % bs]
+    assert np.array_equal(got, want)
     with pytest.raises(ValueError):
-        oracle.store(pool, np.arange(4, dtype=np.int32), 0, 3, codec, keep=[0, 2, 5])
+        oracle.compose(pool.copy(), ptab, [(chunk, T, codec, 0, 0)], 10000.0, select=[[0, 2, 5]])

@@ -60,6 +60,8 @@ MUTANTS = [
      "x[i] = pool[pool_index(s, l, 0, table[p / s->bs], (int)(p % s->bs), h, d)];\n                        }\n                        size_t ch = (size_t)h * (size_t)s->D + (size_t)d;\n                        kdn_oracle_quant_channel(x, n, qmax, q, scales + seg * R + ch);",
      ["test_oracle_td"]),
     ("decoder_forgets_the_running_code", "int v = mode == 1 ? prev + e : e;", "int v = mode == 1 && t == 1 ? prev + e : e;", ["test_oracle_td"]),
+    ("keep_list_ignored_by_the_key_groups", "int64_t p = off + (keep ? keep[t0 + i] : t0 + i);                 /* R7: the listed tokens */",
+     "int64_t p = off + t0 + i; (void)keep;", ["test_oracle_kc"]),
     ("keep_list_ignored_by_the_token_delta_store", "int64_t p = off + (keep ? keep[t0 + i] : t0 + i);", "int64_t p = off + t0 + i; (void)keep;", ["test_oracle_td"]),
     ("keep_list_restarts_in_every_group", "int64_t p = off + (keep ? keep[t0 + i] : t0 + i);", "int64_t p = off + (keep ? keep[i] + t0 : t0 + i);", ["test_oracle_td"]),
 ]
