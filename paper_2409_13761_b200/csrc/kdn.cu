@@ -495,7 +495,9 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
         tile_elems = row_elems;
         bool all_keep = true;
         for (int i = 0; i < n; ++i) all_keep &= hops[i].op.list_mode == 1 || hops[i].op.list_mode == 3;
-        const int want_rows = ctx->tuning.tile_bytes > 0 ? ctx->tuning.tile_bytes / 2 / (int)row_elems : 2048 / (int)row_elems;
+        int want_rows = ctx->tuning.tile_bytes > 0 ? ctx->tuning.tile_bytes / 2 / (int)row_elems : 2048 / (int)row_elems;
+        if (kc_decode)                                     // a key tile must lie inside one 64-token group: a power of two
+            while (want_rows & (want_rows - 1)) want_rows &= want_rows - 1;
         if (!any_coded && !any_rot && all_keep && want_rows >= 2 && row_elems < 1024u && (unsigned long long)pool.nb * (unsigned)pool.bs < 0xffffffffull) {
             // copy form on rows shorter than 2 KiB (few KV heads per GPU): several rows per tile as well
             rows_per_tile = want_rows > kWideRowsPerTile ? kWideRowsPerTile : want_rows;
@@ -1185,8 +1187,8 @@ kdn_status xfer_sparse(kdn_ctx *ctx, int pool_id, int OP, const kdn_sparse_op *o
         const kdn_xfer_op &o = ops[i].op;
         st = check_chunk(&shape, &o.chunk);
         if (st != KDN_OK) return st;
-        if (is_kc(o.chunk.codec)) return KDN_E_UNSUPPORTED;   // a keep-list breaks up the 64-token groups of the key planes
-        // (the token-delta codecs group the chunk's own tokens, listed or not)
+        // (the per-channel key and the token-delta codecs group the chunk's own tokens, listed or not; every row is found
+        // through its own table entry, so there is no rule on token_offset or block_size here)
         if (o.n_table_blocks < 0 || o.token_offset < 0) return KDN_E_INVAL;
         if (o.chunk.n_tokens > 0 && (!o.block_table || !ops[i].keep)) return KDN_E_INVAL;
         // the listed tokens are distinct positions below the end of the table, so there cannot be more of them

@@ -1225,6 +1225,18 @@ kdn_compose_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_COMPOSE,
 
 // ------------------------------------------------ keys of the per-channel key codecs --
 
+// Request position of row t of group g of an op: off + 64 g + t, or, for a keep-list op, off + list[64 g + t].
+// Returns -1 for a list entry that is negative or points past the block table.
+__device__ __forceinline__ long long group_row_pos(const DevOp &op, unsigned g, unsigned t)
+{
+    const unsigned i = (g << 6) + t;
+    if (op.list_mode == 0) return op.off + (long long)i;
+    const long long rel = __ldg(op.list + i);
+    const long long p = op.off + rel;
+    return (rel < 0 || p >= op.pos_end) ? -1ll : p;
+}
+
+
 // Storing the key planes of a per-channel key codec needs, for every channel, the largest magnitude over 64 tokens
 // before the first code can be formed, so it does not fit the streaming tile pipeline.  One CTA takes one
 // (op, layer, 64-token group, slice of `cols` channels): the slice of the group's token rows is brought into shared
@@ -1286,16 +1298,17 @@ __global__ void __launch_bounds__(512) kdn_store_kc_kernel(const __grid_constant
     }
     __syncthreads();
     if (tid < 32) {
-        // warp 0 brings the rows in: lane r takes token rows r and r + 32
+        // warp 0 brings the rows in: lane r takes token rows r and r + 32, each found through its own table entry
         const unsigned char *base = reinterpret_cast<const unsigned char *>(P.k_layers[op.l0 + (int)li]);
-        const long long first_block = (op.off + (long long)t0) / P.bs;
-        long long id[2] = { 0, 0 };
+        long long id[2] = { 0, 0 }, pos[2] = { 0, 0 };
         bool bad = false;
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
             const unsigned t = (unsigned)tid + 32u * (unsigned)k;
             if (t < n_tok) {
-                id[k] = __ldg(op.table + first_block + t / (unsigned)P.bs);
+                pos[k] = group_row_pos(op, g, t);
+                if (pos[k] < 0) { bad = true; continue; }
+                id[k] = __ldg(op.table + pos[k] / P.bs);
                 if (id[k] < 0 || id[k] >= P.n_blocks) bad = true;
             }
         }
@@ -1307,9 +1320,10 @@ __global__ void __launch_bounds__(512) kdn_store_kc_kernel(const __grid_constant
         } else {
             if (tid == 0) mbar_arrive_expect_tx(bar, n_tok * C * 2u);
             __syncwarp();
-            if (P.n_split == 1u) {
+            if (P.n_split == 1u && op.list_mode == 0) {
                 // the whole row: a block's tokens are contiguous in the pool, one copy per block (pieces <= 32 KiB)
                 if (tid == 0) {
+                    const long long first_block = (op.off + (long long)t0) / P.bs;
                     for (unsigned t = 0; t < n_tok; t += (unsigned)P.bs) {
                         const unsigned k = n_tok - t < (unsigned)P.bs ? n_tok - t : (unsigned)P.bs;
                         const long long b = __ldg(op.table + first_block + t / (unsigned)P.bs);
@@ -1324,7 +1338,7 @@ __global__ void __launch_bounds__(512) kdn_store_kc_kernel(const __grid_constant
                 for (int k = 0; k < 2; ++k) {
                     const unsigned t = (unsigned)tid + 32u * (unsigned)k;
                     if (t < n_tok) {
-                        const unsigned slot = (unsigned)((op.off + (long long)t0 + t) % P.bs);
+                        const unsigned slot = (unsigned)(pos[k] % P.bs);
                         const unsigned char *src = base + (((unsigned long long)id[k] * P.bs + slot) * RE + c0) * 2ull;
                         bulk_g2s(smem_u32(X + (size_t)t * C * 2u), src, C * 2u, bar);
                     }

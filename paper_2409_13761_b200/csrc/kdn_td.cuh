@@ -130,17 +130,6 @@ __device__ __forceinline__ unsigned td_block_scan(unsigned v, unsigned *scratch,
     return r;
 }
 
-// Request position of row t of group g of an op: off + 64 g + t, or, for a keep-list op, off + list[64 g + t].
-// Returns -1 for a list entry that is negative or points past the block table.
-__device__ __forceinline__ long long td_row_pos(const DevOp &op, unsigned g, unsigned t)
-{
-    const unsigned i = (g << 6) + t;
-    if (op.list_mode == 0) return op.off + (long long)i;
-    const long long rel = __ldg(op.list + i);
-    const long long p = op.off + rel;
-    return (rel < 0 || p >= op.pos_end) ? -1ll : p;
-}
-
 // Bring the slice [c0, c0 + C) of the n_tok token rows of one group (request positions pos0 ..) of a pool plane
 // into X[n_tok][C] with bulk copies counted on `bar`.  Warp 0 calls this; returns false (and records KDN_E_RANGE)
 // when a block id lies outside the pool, in which case nothing was issued.
@@ -156,7 +145,7 @@ __device__ __forceinline__ bool td_load_slice(unsigned char *X, uint32_t bar, co
     for (int k = 0; k < 2; ++k) {
         const unsigned t = lane + 32u * (unsigned)k;
         if (t < n_tok) {
-            pos[k] = td_row_pos(op, g, t);
+            pos[k] = group_row_pos(op, g, t);
             if (pos[k] < 0) { bad = true; continue; }
             id[k] = __ldg(table + pos[k] / bs);
             if (id[k] < 0 || id[k] >= n_blocks) bad = true;
@@ -689,7 +678,7 @@ __global__ void __launch_bounds__(kCols ? kCols : 512) kdn_td_decode_kernel(cons
         for (int k = 0; k < 2; ++k) {
             const unsigned t = tid + 32u * (unsigned)k;
             if (t < s.n_tok) {
-                pos[k] = td_row_pos(s.op, s.g, t);
+                pos[k] = group_row_pos(s.op, s.g, t);
                 if (pos[k] < 0) { bad = true; continue; }
                 id[k] = __ldg(s.op.table + pos[k] / P.bs);
                 if (id[k] < 0 || id[k] >= P.n_blocks) bad = true;

@@ -165,13 +165,71 @@ def test_what_the_codecs_do_not_support_is_refused():
             dev.close()
     dev = Device(synth.TOY.with_(n_blocks=16), seed=1)
     try:
-        for codec in KC:
+        for codec in KC:                                                   # select-lists
             b = dev.chunk_buf(5, codec)
             tab = dev.table(np.arange(4, dtype=np.int32))
-            keep = dev.table(np.arange(5, dtype=np.int32))
+            sel = dev.table(np.arange(3, dtype=np.int32))
             with pytest.raises(K.KdnError) as e:
-                K.kdn_store_sparse(dev.ctx, dev.pool_id, [dev.op(tab, 0, b, 5, codec)], [keep.data_ptr()], dev.stream.cuda_stream)
+                K.kdn_compose_select(dev.ctx, dev.pool_id, [K.ComposeReq(tab.data_ptr(), 4, [dev.chunk(b, 5, codec)], [0], 1e4)],
+                                     [[(sel.data_ptr(), 3)]], dev.stream.cuda_stream)
             assert e.value.status == K.KDN_E_UNSUPPORTED
         assert dev.sync() == 0
+    finally:
+        dev.close()
+
+
+@pytest.mark.parametrize("shape", SHAPES, ids=["H%dD%dbs%d" % (s.n_kv_heads, s.head_dim, s.block_size) for s in SHAPES])
+@pytest.mark.parametrize("codec", KC, ids=["int8kc", "int4kc"])
+def test_keep_list_chunks_against_the_oracle(shape, codec):
+    """Keep-lists with the per-channel key codecs: a key group is 64 consecutive listed tokens, wherever they sit in the
+    request (no alignment rule).  Store bytes, retrieve into other blocks (device and page-locked host chunk), a dense
+    compose of a sparsely stored chunk, and a list entry outside the table."""
+    bs = shape.block_size
+    rng = np.random.default_rng(31 + codec)
+    perm = rng.permutation(shape.n_blocks).astype(np.int32)
+    span, off = 200, 5
+    nb = -(-(off + span) // bs)
+    src, dst = perm[:nb], perm[nb:2 * nb]
+    dev = Device(shape, seed=77)
+    try:
+        K = dev.K
+        pool = dev.pool_np()
+        lists = [np.sort(rng.choice(span, 100, replace=False)), np.arange(span), np.array([7]), np.arange(0, span, 3), np.arange(64) + 5]
+        ops, keeps, wants, bufs = [], [], [], []
+        for keep in lists:
+            keep = keep.astype(np.int32)
+            b = dev.chunk_buf(len(keep), codec)
+            ops.append(dev.op(dev.table(src), off, b, len(keep), codec))
+            keeps.append(dev.table(keep).data_ptr())
+            wants.append(oracle.store(pool, src, off, len(keep), codec, keep=keep))
+            bufs.append(b)
+        K.kdn_store_sparse(dev.ctx, dev.pool_id, ops, keeps, dev.stream.cuda_stream)
+        assert dev.sync() == 0
+        for b, w, keep in zip(bufs, wants, lists):
+            assert np.array_equal(to_np(b), w), len(keep)
+        assert np.array_equal(dev.pool_np(), pool)
+        ref = pool.copy()
+        for i, (b, w, keep) in enumerate(zip(bufs, wants, lists)):
+            src_buf = b
+            if i % 2 == 1:
+                src_buf = dev.chunk_buf(len(keep), codec, pinned=True)
+                src_buf.copy_(b.cpu())
+            K.kdn_retrieve_sparse(dev.ctx, dev.pool_id, [dev.op(dev.table(dst), off, src_buf, len(keep), codec)], [keeps[i]], dev.stream.cuda_stream)
+            assert dev.sync() == 0
+            oracle.retrieve(ref, dst, off, len(keep), codec, w, keep=keep.astype(np.int32))
+            assert np.array_equal(dev.pool_np(), ref), i
+        # a sparsely stored chunk is an ordinary chunk of its own tokens: a dense retrieve at a block start places them side by side
+        if 64 % bs == 0:
+            T = len(lists[0])
+            dt = perm[2 * nb:2 * nb + -(-T // bs)]
+            dev.retrieve([dev.op(dev.table(dt), 0, bufs[0], T, codec)])
+            assert dev.sync() == 0
+            oracle.retrieve(ref, dt, 0, T, codec, wants[0])
+            assert np.array_equal(dev.pool_np(), ref)
+        bad = np.array([0, 1, 2, nb * bs], dtype=np.int32)
+        b = dev.chunk_buf(4, codec)
+        K.kdn_store_sparse(dev.ctx, dev.pool_id, [dev.op(dev.table(src), 0, b, 4, codec)], [dev.table(bad).data_ptr()], dev.stream.cuda_stream)
+        assert dev.sync() == K.KDN_E_RANGE
+        assert np.array_equal(dev.pool_np(), ref)
     finally:
         dev.close()
