@@ -47,7 +47,8 @@
  *                    fp32 k_scales[ceil(T/64)][head*D] followed by fp32 v_scales[t][head*D/64]; layers follow
  *                    each other; the scales follow the codes.  Decode is R5 with the element's own scale.
  *                    With a keep-list (R7) the chunk's tokens are the listed ones and a key group is 64 consecutive
- *                    CHUNK tokens, as for R9; select-lists are not defined for these codecs.
+ *                    CHUNK tokens, as for R9; a select-list delivers the listed chunk tokens, each decoded with its
+ *                    own scales, as for every fixed-rate codec.
  *   R9  token-delta Rice codecs (codecs 5 = int8, 6 = int4; not prescribed by the paper: Sec. 3.2 "KV-cache delivery"
  *                    cites a scheme that quantises a KV cache and then encodes it into binary strings, and reports
  *                    more than tenfold reductions for combined techniques.  This is this library's own bitstream.)
@@ -457,7 +458,6 @@ static int check_args_list(const shape_t *s, const int32_t *table, int n_table, 
     if (s->L <= 0 || s->H <= 0 || s->D <= 0 || s->bs <= 0 || s->nb <= 0) return 1;
     if (n < 0 || off < 0 || n_table < 0) return 1;
     if (codec < KDN_ORACLE_RAW_BF16 || codec > KDN_ORACLE_INT4_TD64) return 3;
-    if ((codec == KDN_ORACLE_INT8_KC64 || codec == KDN_ORACLE_INT4_KC64) && list && list_bound >= 0) return 3;   /* R4": keep-lists only */
     if (td_is(codec) && list && list_bound >= 0) return 3;                                    /* R9: keep-lists only */
     if (codec != KDN_ORACLE_RAW_BF16 && s->D % KDN_ORACLE_GROUP) return 3;
     for (int i = 0; i < n; ++i) {

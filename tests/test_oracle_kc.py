@@ -218,5 +218,28 @@ def test_keep_list_chunk_is_the_chunk_of_the_listed_tokens(codec, base, qmax):
     want = np.full_like(pool, 0x1234)
     want[:, :, dtab[pos // bs], pos % bs] = dense[:, :, ptab[t // bs], t % bs]
     assert np.array_equal(got, want)
-    with pytest.raises(ValueError):
-        oracle.compose(pool.copy(), ptab, [(chunk, T, codec, 0, 0)], 10000.0, select=[[0, 2, 5]])
+
+
+@pytest.mark.parametrize("codec,base,qmax", KC)
+def test_select_list_delivers_the_listed_tokens_of_the_full_compose(codec, base, qmax):
+    """A select-list changes which positions are written, never what is written there: the listed positions hold what
+    the compose of the whole part puts there (rotated keys included, their fp64 references too), every other position
+    keeps its bits."""
+    shape = synth.TOY.with_(n_layers=2, n_kv_heads=2, head_dim=64, block_size=4, n_blocks=64)
+    k, v = synth.make_pool(shape, "cpu", seed=30)
+    pool = synth.pool_to_numpy(k, v)
+    bs, T, dp, theta = shape.block_size, 100, 8, 10000.0
+    rng = np.random.default_rng(9)
+    table = rng.permutation(64)[:30].astype(np.int32)
+    chunk = oracle.store(pool, table, 0, T, codec)
+    rtab = rng.permutation(64)[:30].astype(np.int32)
+    sel = np.sort(rng.choice(T, 37, replace=False)).astype(np.int32)
+    full = np.full_like(pool, 0x4321)
+    kf, _ = oracle.compose(full, rtab, [(chunk, T, codec, 3, dp)], theta, want_ref=True)
+    part = np.full_like(pool, 0x4321)
+    ks, _ = oracle.compose(part, rtab, [(chunk, T, codec, 3, dp)], theta, want_ref=True, select=[sel])
+    pos = dp + sel
+    want = np.full_like(pool, 0x4321)
+    want[:, :, rtab[pos // bs], pos % bs] = full[:, :, rtab[pos // bs], pos % bs]
+    assert np.array_equal(part, want)
+    assert np.array_equal(ks[:, pos], kf[:, pos])
