@@ -45,8 +45,8 @@
  *   INT8_G64 / INT4_G64; the scales that follow them are, per layer, fp32 k_scales[ceil(T/64)][H*D] and then
  *   fp32 v_scales[T][H*D/64].  Same bytes per element as the G64 codecs when T is a multiple of 64.
  *   They need block_size to divide 64 and the chunk's first token to sit at the start of a block (token_offset, or
- *   part_dst_pos in kdn_compose, a multiple of block_size), else KDN_E_UNSUPPORTED; select-lists and kdn_compose_static
- *   are not supported with them (KDN_E_UNSUPPORTED).  Keep-lists are (kdn_store_sparse, kdn_retrieve_sparse): the chunk
+ *   part_dst_pos in kdn_compose and kdn_compose_select, a multiple of block_size), else KDN_E_UNSUPPORTED;
+ *   kdn_compose_static is not supported with them (KDN_E_UNSUPPORTED).  Keep-lists are (kdn_store_sparse, kdn_retrieve_sparse): the chunk
  *   then holds the listed tokens, a key group is 64 consecutive chunk tokens, and neither rule above applies, since
  *   every listed row is found through its own table entry.
  * Token-delta Rice codecs (KDN_CODEC_INT8_TD64, KDN_CODEC_INT4_TD64; Sec. 3.2 "KV-cache delivery" cites a scheme that

@@ -163,17 +163,47 @@ def test_what_the_codecs_do_not_support_is_refused():
                     assert e.value.status == K.KDN_E_UNSUPPORTED
         finally:
             dev.close()
-    dev = Device(synth.TOY.with_(n_blocks=16), seed=1)
+
+
+@pytest.mark.parametrize("shape", SHAPES[:3], ids=["H%dD%dbs%d" % (s.n_kv_heads, s.head_dim, s.block_size) for s in SHAPES[:3]])
+@pytest.mark.parametrize("codec", KC, ids=["int8kc", "int4kc"])
+def test_select_list_compose_against_the_oracle(shape, codec):
+    """kdn_compose_select with per-channel key chunks: two parts, one with a select-list and a position shift (keys
+    re-rotated), one delivered whole; listed positions as the oracle has them, every other position untouched."""
+    bs = shape.block_size
+    rng = np.random.default_rng(37 + codec)
+    perm = rng.permutation(shape.n_blocks).astype(np.int32)
+    T = 130
+    nb = -(-T // bs)
+    dev = Device(shape, seed=79)
     try:
-        for codec in KC:                                                   # select-lists
-            b = dev.chunk_buf(5, codec)
-            tab = dev.table(np.arange(4, dtype=np.int32))
-            sel = dev.table(np.arange(3, dtype=np.int32))
-            with pytest.raises(K.KdnError) as e:
-                K.kdn_compose_select(dev.ctx, dev.pool_id, [K.ComposeReq(tab.data_ptr(), 4, [dev.chunk(b, 5, codec)], [0], 1e4)],
-                                     [[(sel.data_ptr(), 3)]], dev.stream.cuda_stream)
-            assert e.value.status == K.KDN_E_UNSUPPORTED
+        K = dev.K
+        pool = dev.pool_np()
+        srcs = [perm[:nb], perm[nb:2 * nb]]
+        bufs = [dev.chunk_buf(T, codec) for _ in srcs]
+        dev.store([dev.op(dev.table(t), 0, b, T, codec) for t, b in zip(srcs, bufs)])
         assert dev.sync() == 0
+        wants = [oracle.store(pool, t, 0, T, codec) for t in srcs]
+        d0, d1 = 0, -(-T // 64) * 64                                       # block-aligned destinations (64 is a multiple of block_size)
+        rt = perm[2 * nb:2 * nb + -(-(d1 + T) // bs)]
+        sel = np.sort(rng.choice(T, 41, replace=False)).astype(np.int32)
+        d_sel = dev.table(sel)
+        before = dev.pool_np()
+        K.kdn_compose_select(dev.ctx, dev.pool_id,
+                             [K.ComposeReq(dev.table(rt).data_ptr(), len(rt), [dev.chunk(bufs[0], T, codec, 9), dev.chunk(bufs[1], T, codec, d1)],
+                                           [d0, d1], shape.rope_theta)],
+                             [[(d_sel.data_ptr(), len(sel)), None]], dev.stream.cuda_stream)
+        assert dev.sync() == 0
+        ref = before.copy()
+        kref, kmag = oracle.compose(ref, rt, [(wants[0], T, codec, 9, d0), (wants[1], T, codec, d1, d1)], shape.rope_theta,
+                                    want_ref=True, select=[sel, None])
+        got = dev.pool_np()
+        p = d0 + sel
+        rot = np.zeros(got.shape, dtype=bool)
+        rot[:, 0, rt[p // bs], p % bs] = True
+        assert np.array_equal(got[~rot], ref[~rot])
+        check_rotated_keys(got[:, 0, rt[p // bs], p % bs], kref[:, p], kmag[:, p], ref[:, 0, rt[p // bs], p % bs],
+                           min_equal=0.995 if got[:, 0, rt[p // bs], p % bs].size >= 8192 else 0.95)
     finally:
         dev.close()
 
