@@ -76,8 +76,8 @@
  *                    Decode: undo Rice, zigzag and the delta, then R5 with the channel's scale.  With a keep-list
  *                    (R7) the chunk's tokens are the listed ones: groups are 64 consecutive CHUNK tokens and mode 1
  *                    differences a code from that of the listed token before it (the combination the paper's Sec. 3.2
- *                    "KV-cache delivery" points to: drop tokens, then code what is left).  Select-lists are not
- *                    defined for these codecs.
+ *                    "KV-cache delivery" points to: drop tokens, then code what is left).  A select-list delivers
+ *                    the listed chunk tokens of the decoded chunk, as for every codec.
  *   R6  re-rotation  stored keys carry rotary position embedding at absolute
  *                    positions base_pos + t (what an engine's pool holds), so
  *                    reuse at dst_pos (Sec. 3.2 "KV-cache blending": a
@@ -458,7 +458,6 @@ static int check_args_list(const shape_t *s, const int32_t *table, int n_table, 
     if (s->L <= 0 || s->H <= 0 || s->D <= 0 || s->bs <= 0 || s->nb <= 0) return 1;
     if (n < 0 || off < 0 || n_table < 0) return 1;
     if (codec < KDN_ORACLE_RAW_BF16 || codec > KDN_ORACLE_INT4_TD64) return 3;
-    if (td_is(codec) && list && list_bound >= 0) return 3;                                    /* R9: keep-lists only */
     if (codec != KDN_ORACLE_RAW_BF16 && s->D % KDN_ORACLE_GROUP) return 3;
     for (int i = 0; i < n; ++i) {
         int64_t rel = list ? list[i] : i;

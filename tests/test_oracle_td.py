@@ -302,17 +302,30 @@ def test_keep_list_chunk_is_the_chunk_of_the_listed_tokens(codec):
     assert np.array_equal(got, want)
 
 
-def test_select_lists_are_refused():
-    """Select-lists (compose of some tokens of a part) are not defined for these codecs; a keep-list that is not
-    strictly increasing is refused as for every codec."""
-    k, v = synth.make_pool(synth.TOY, "cpu")
+@pytest.mark.parametrize("codec", [TD8, TD4])
+def test_select_list_delivers_the_listed_tokens_of_the_full_compose(codec):
+    """A select-list changes which positions are written, never what is written there (re-rotated keys and their fp64
+    references included); a keep-list that is not strictly increasing is refused as for every codec."""
+    shape = synth.TOY.with_(n_layers=2, n_kv_heads=2, head_dim=64, block_size=4, n_blocks=64)
+    k, v = synth.make_pool(shape, "cpu", seed=32)
     pool = synth.pool_to_numpy(k, v)
-    tab = np.arange(4, dtype=np.int32)
-    chunk = oracle.store(pool, tab, 0, 8, TD8)
+    bs, T, dp, theta = shape.block_size, 100, 8, 10000.0
+    rng = np.random.default_rng(10)
+    table = rng.permutation(64)[:30].astype(np.int32)
+    chunk = oracle.store(pool, table, 0, T, codec)
+    rtab = rng.permutation(64)[:30].astype(np.int32)
+    sel = np.sort(rng.choice(T, 37, replace=False)).astype(np.int32)
+    full = np.full_like(pool, 0x4321)
+    kf, _ = oracle.compose(full, rtab, [(chunk, T, codec, 3, dp)], theta, want_ref=True)
+    part = np.full_like(pool, 0x4321)
+    ks, _ = oracle.compose(part, rtab, [(chunk, T, codec, 3, dp)], theta, want_ref=True, select=[sel])
+    pos = dp + sel
+    want = np.full_like(pool, 0x4321)
+    want[:, :, rtab[pos // bs], pos % bs] = full[:, :, rtab[pos // bs], pos % bs]
+    assert np.array_equal(part, want)
+    assert np.array_equal(ks[:, pos], kf[:, pos])
     with pytest.raises(ValueError):
-        oracle.compose(pool.copy(), tab, [(chunk, 8, TD8, 0, 0)], 10000.0, select=[[0, 2, 5]])
-    with pytest.raises(ValueError):
-        oracle.store(pool, tab, 0, 3, TD8, keep=[0, 5, 2])
+        oracle.store(pool, table, 0, 3, codec, keep=[0, 5, 2])
 
 
 def ar1(rng, n_tokens, n_channels, rho):
