@@ -66,7 +66,8 @@
  *   the chunk uses, which is what has to be kept or sent.  kdn_chunk_bytes gives the worst-case CAPACITY (a sub-stream
  *   never exceeds 72 or 40 bytes) and chunk.bytes must equal it; bytes past seg_off[S] are not written and not read
  *   (up to 15 beyond it may be read, never past the capacity).  kdn_td_layout gives the offsets.
- *   Same restrictions as the per-channel key codecs, except for keep-lists: kdn_store_sparse and kdn_retrieve_sparse
+ *   Same restrictions as the per-channel key codecs (kdn_compose_select included: whole groups are decoded, the listed
+ *   rows delivered, a group without a listed token skipped), and the same freedom for keep-lists: kdn_store_sparse and kdn_retrieve_sparse
  *   take these codecs (the chunk then codes the LISTED tokens: groups are 64 consecutive chunk tokens, mode 1 differences
  *   a code from that of the listed token before it; no rule on token_offset or block_size, every row is found through
  *   its own table entry).  Dropping half of the tokens and coding the rest is what brings a chunk below a tenth of its

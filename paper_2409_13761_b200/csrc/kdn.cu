@@ -1522,7 +1522,6 @@ static kdn_status compose_impl(kdn_ctx *ctx, int pool_id, const kdn_compose_req 
             if (selects && selects[r].part_select && selects[r].part_select[j]) {
                 if (!selects[r].part_n_select || selects[r].part_n_select[j] < 0 || selects[r].part_n_select[j] > c.n_tokens)
                     return KDN_E_INVAL;
-                if (is_td(c.codec)) return KDN_E_UNSUPPORTED;            // select-lists are not defined for the token-delta codecs
                 if (selects[r].part_n_select[j] == 0) continue;          // nothing of this part is delivered
                 h.op.list = selects[r].part_select[j];
                 h.op.n_list = selects[r].part_n_select[j];

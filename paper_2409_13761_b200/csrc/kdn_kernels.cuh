@@ -1230,7 +1230,7 @@ kdn_compose_kernel(const __grid_constant__ Launch P) { tile_pipeline<OP_COMPOSE,
 __device__ __forceinline__ long long group_row_pos(const DevOp &op, unsigned g, unsigned t)
 {
     const unsigned i = (g << 6) + t;
-    if (op.list_mode == 0) return op.off + (long long)i;
+    if (op.list_mode != 1) return op.off + (long long)i;      // (a select-list chooses among the chunk's tokens, it does not move them)
     const long long rel = __ldg(op.list + i);
     const long long p = op.off + rel;
     return (rel < 0 || p >= op.pos_end) ? -1ll : p;

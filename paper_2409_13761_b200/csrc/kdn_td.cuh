@@ -130,6 +130,17 @@ __device__ __forceinline__ unsigned td_block_scan(unsigned v, unsigned *scratch,
     return r;
 }
 
+// First index of the increasing list whose entry is >= key (n when there is none).  At most 32 steps.
+__device__ __forceinline__ unsigned td_lower_bound(const int32_t *list, unsigned n, long long key)
+{
+    unsigned lo = 0, hi = n;
+    while (lo < hi) {
+        const unsigned mid = (lo + hi) >> 1;
+        if ((long long)__ldg(list + mid) < key) lo = mid + 1u; else hi = mid;
+    }
+    return lo;
+}
+
 // Bring the slice [c0, c0 + C) of the n_tok token rows of one group (request positions pos0 ..) of a pool plane
 // into X[n_tok][C] with bulk copies counted on `bar`.  Warp 0 calls this; returns false (and records KDN_E_RANGE)
 // when a block id lies outside the pool, in which case nothing was issued.
@@ -556,13 +567,18 @@ __global__ void __launch_bounds__(kCols ? kCols : 512) kdn_td_decode_kernel(cons
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         fence_async_smem();
     }
+    // a select-list (compose): which of its entries fall into this group?  Two threads look; none: nothing to do here
+    const bool selecting = kCompose && s.op.list_mode == 2;
+    if (selecting && tid < 2u) scratch[40u + tid] = td_lower_bound(s.op.list, (unsigned)s.op.n_list, ((long long)s.g + tid) << 6);
     const TdLayout lay = td_layout(P.L, RE, s.op.T, codec);
     const unsigned long long row = (unsigned long long)s.seg * RE;
     const unsigned char *lens = s.op.data + lay.lens + row;
     unsigned before = 0;
     for (unsigned c = tid; c < s.c0; c += blockDim.x) before += lens[c];
     unsigned total_before, total_slice;
-    td_block_scan(before, scratch, &total_before);                        // (its barriers also publish the mbarrier)
+    td_block_scan(before, scratch, &total_before);                        // (its barriers also publish the mbarrier and the two indices)
+    const unsigned sel_lo = selecting ? scratch[40] : 0u, sel_hi = selecting ? scratch[41] : 0u;
+    if (selecting && sel_lo >= sel_hi) return;                            // every thread alike, and no copy has been started
     const unsigned my_len = tid < C ? lens[s.c0 + tid] : 0u;               // blockDim.x >= C
     const unsigned my_off = td_block_scan(my_len, scratch, &total_slice);
     unsigned param = 0;
@@ -673,12 +689,24 @@ __global__ void __launch_bounds__(kCols ? kCols : 512) kdn_td_decode_kernel(cons
     if (tid < 32) {
         unsigned char *base = reinterpret_cast<unsigned char *>((s.kv ? P.v_layers : P.k_layers)[s.op.l0 + (int)s.li]);
         long long id[2] = { 0, 0 }, pos[2] = { 0, 0 };
+        unsigned row_t[2] = { tid, tid + 32u };                       // which row of the group lane k writes (64: none)
         bool bad = false;
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
-            const unsigned t = tid + 32u * (unsigned)k;
-            if (t < s.n_tok) {
-                pos[k] = group_row_pos(s.op, s.g, t);
+            if (selecting) {
+                // the group's listed tokens, at most 64 of them: lane k takes entry sel_lo + tid + 32 k
+                const unsigned idx = sel_lo + tid + 32u * (unsigned)k;
+                row_t[k] = 64u;
+                if (idx < sel_hi) {
+                    const long long c = (long long)__ldg(s.op.list + idx) - ((long long)s.g << 6);
+                    if (c < 0 || c >= (long long)s.n_tok) bad = true;      // (a list that is not increasing)
+                    else row_t[k] = (unsigned)c;
+                }
+            } else if (row_t[k] >= s.n_tok) {
+                row_t[k] = 64u;
+            }
+            if (row_t[k] < 64u) {
+                pos[k] = group_row_pos(s.op, s.g, row_t[k]);
                 if (pos[k] < 0) { bad = true; continue; }
                 id[k] = __ldg(s.op.table + pos[k] / P.bs);
                 if (id[k] < 0 || id[k] >= P.n_blocks) bad = true;
@@ -702,8 +730,8 @@ __global__ void __launch_bounds__(kCols ? kCols : 512) kdn_td_decode_kernel(cons
             } else {
 #pragma unroll
                 for (int k = 0; k < 2; ++k) {
-                    const unsigned t = tid + 32u * (unsigned)k;
-                    if (t < s.n_tok) {
+                    const unsigned t = row_t[k];
+                    if (t < 64u) {
                         const unsigned slot = (unsigned)(pos[k] % P.bs);
                         unsigned char *d = base + (((unsigned long long)id[k] * P.bs + slot) * RE + s.c0) * 2ull;
                         bulk_s2g(d, smem_u32(A + (size_t)t * C * 2u), C * 2u);

@@ -173,9 +173,7 @@ def test_refusals_and_damaged_chunks():
         T = 64
         buf = dev.chunk_buf(T, TD8)
         for bad in (lambda: dev.store([dev.op(tab, 3, buf, T, TD8)]),                       # first token not at a block start
-                    lambda: dev.store([dev.op(tab, 0, dev.chunk_buf(T, TD8, pinned=True), T, TD8)]),   # store into host memory
-                    lambda: K.kdn_compose_select(dev.ctx, dev.pool_id, [K.ComposeReq(tab.data_ptr(), 8, [dev.chunk(buf, T, TD8)], [0], 1e4)],
-                                                 [[(tab.data_ptr(), 4)]], dev.stream.cuda_stream)):   # select-lists
+                    lambda: dev.store([dev.op(tab, 0, dev.chunk_buf(T, TD8, pinned=True), T, TD8)])):  # store into host memory
             with pytest.raises(K.KdnError) as e:
                 bad()
             assert e.value.status == K.KDN_E_UNSUPPORTED
@@ -328,5 +326,52 @@ def test_keep_list_chunks_against_the_oracle(shape, codec):
                               dev.stream.cuda_stream)
         assert dev.sync() == K.KDN_E_RANGE
         assert np.array_equal(dev.pool_np(), ref)
+    finally:
+        dev.close()
+
+
+@pytest.mark.parametrize("shape", [SHAPES[0], SHAPES[1], SHAPES[3]], ids=[IDS[0], IDS[1], IDS[3]])   # (rows of 576 are too wide to rotate)
+@pytest.mark.parametrize("codec", [TD8, TD4], ids=["int8td", "int4td"])
+def test_select_list_compose_against_the_oracle(shape, codec):
+    """kdn_compose_select with token-delta chunks: the decoder still decodes whole groups, but only the listed rows leave
+    it, and a group without a listed token is not decoded at all.  One part with a list that skips the middle group and
+    a position shift (keys re-rotated), one from page-locked host memory delivered whole, one with a single listed token."""
+    bs = shape.block_size
+    rng = np.random.default_rng(43 + codec)
+    perm = rng.permutation(shape.n_blocks).astype(np.int32)
+    T = 170                                                               # three groups: 64 + 64 + 42
+    nb = -(-T // bs)
+    span = -(-T // 64) * 64
+    pool = make_pool_np(shape, perm[:nb], 0, T, 0.9, seed=47)
+    dev = Device(shape, pool_np=pool)
+    try:
+        K = dev.K
+        buf = dev.chunk_buf(T, codec)
+        dev.store([dev.op(dev.table(perm[:nb]), 0, buf, T, codec)])
+        assert dev.sync() == 0
+        want = oracle.store(pool, perm[:nb], 0, T, codec)
+        hbuf = dev.chunk_buf(T, codec, pinned=True)
+        hbuf.copy_(buf.cpu())
+        rt = perm[nb:nb + 3 * span // bs + 1]
+        sel_a = np.concatenate([np.sort(rng.choice(64, 20, replace=False)), 128 + np.sort(rng.choice(42, 11, replace=False))]).astype(np.int32)
+        sel_c = np.array([65], dtype=np.int32)
+        d_a, d_c = dev.table(sel_a), dev.table(sel_c)
+        before = dev.pool_np()
+        K.kdn_compose_select(dev.ctx, dev.pool_id,
+                             [K.ComposeReq(dev.table(rt).data_ptr(), len(rt),
+                                           [dev.chunk(buf, T, codec, 7), dev.chunk(hbuf, T, codec, span), dev.chunk(buf, T, codec, 0)],
+                                           [0, span, 2 * span], shape.rope_theta)],
+                             [[(d_a.data_ptr(), len(sel_a)), None, (d_c.data_ptr(), 1)]], dev.stream.cuda_stream)
+        assert dev.sync() == 0
+        ref = before.copy()
+        kref, kmag = oracle.compose(ref, rt, [(want, T, codec, 7, 0), (want, T, codec, span, span), (want, T, codec, 0, 2 * span)],
+                                    shape.rope_theta, want_ref=True, select=[sel_a, None, sel_c])
+        got = dev.pool_np()
+        p = np.concatenate([sel_a, 2 * span + sel_c])                      # the re-rotated positions
+        rot = np.zeros(got.shape, dtype=bool)
+        rot[:, 0, rt[p // bs], p % bs] = True
+        assert np.array_equal(got[~rot], ref[~rot])
+        g = got[:, 0, rt[p // bs], p % bs]
+        check_rotated_keys(g, kref[:, p], kmag[:, p], ref[:, 0, rt[p // bs], p % bs], min_equal=0.995 if g.size >= 8192 else 0.95)
     finally:
         dev.close()
