@@ -336,6 +336,7 @@ def test_select_list_compose_against_the_oracle(shape, codec):
     """kdn_compose_select with token-delta chunks: the decoder still decodes whole groups, but only the listed rows leave
     it, and a group without a listed token is not decoded at all.  One part with a list that skips the middle group and
     a position shift (keys re-rotated), one from page-locked host memory delivered whole, one with a single listed token."""
+    shape = shape.with_(n_blocks=max(shape.n_blocks, 256))
     bs = shape.block_size
     rng = np.random.default_rng(43 + codec)
     perm = rng.permutation(shape.n_blocks).astype(np.int32)
