@@ -185,8 +185,8 @@ class ClockSampler:
 # DRAM bytes (read + write) per launch from a profiler capture of a reduced case (8 chunks per store/retrieve
 # launch, 2 parts per compose launch), scaled by the units a bench launch processes: every byte is touched once,
 # so traffic grows in proportion.  Valid only for the kernel source the capture was taken from (its hash).
-NCU_KERNEL_SHA = "607ff67e0cb3ea48"
-NCU_SMALL_CASE_BYTES = {"store_raw": (536.920832e6 + 487.979520e6, 8), "retrieve_raw": (537.022976e6 + 490.659840e6, 8), "compose_raw": (268.505344e6 + 222.629376e6, 2), "store_int8": (536.936960e6 + 250.894336e6, 8), "retrieve_int8": (285.353472e6 + 482.643968e6, 8), "compose_int8": (142.675200e6 + 213.902080e6, 2)}
+NCU_KERNEL_SHA = "d5c5296358235c98"
+NCU_SMALL_CASE_BYTES = {"store_raw": (536.921344e6 + 486.536960e6, 8), "retrieve_raw": (536.920832e6 + 491.426816e6, 8), "compose_raw": (268.572928e6 + 222.653952e6, 2), "store_int8": (536.936704e6 + 251.162112e6, 8), "retrieve_int8": (285.271040e6 + 484.859904e6, 8), "compose_int8": (142.711552e6 + 214.546944e6, 2)}
 
 
 def measured_traffic(op: str, units: float):
