@@ -577,8 +577,7 @@ __global__ void __launch_bounds__(kCols ? kCols : 512) kdn_td_decode_kernel(cons
     for (unsigned c = tid; c < s.c0; c += blockDim.x) before += lens[c];
     unsigned total_before, total_slice;
     td_block_scan(before, scratch, &total_before);                        // (its barriers also publish the mbarrier and the two indices)
-    const unsigned sel_lo = selecting ? scratch[40] : 0u, sel_hi = selecting ? scratch[41] : 0u;
-    if (selecting && sel_lo >= sel_hi) return;                            // every thread alike, and no copy has been started
+    if (selecting && scratch[40] >= scratch[41]) return;                  // every thread alike, and no copy has been started
     const unsigned my_len = tid < C ? lens[s.c0 + tid] : 0u;               // blockDim.x >= C
     const unsigned my_off = td_block_scan(my_len, scratch, &total_slice);
     unsigned param = 0;
@@ -694,10 +693,11 @@ __global__ void __launch_bounds__(kCols ? kCols : 512) kdn_td_decode_kernel(cons
 #pragma unroll
         for (int k = 0; k < 2; ++k) {
             if (selecting) {
-                // the group's listed tokens, at most 64 of them: lane k takes entry sel_lo + tid + 32 k
-                const unsigned idx = sel_lo + tid + 32u * (unsigned)k;
+                // the group's listed tokens, at most 64 of them: lane k takes entry first + tid + 32 k (the two indices
+                // still sit where the search left them: the scans use the words below)
+                const unsigned idx = scratch[40] + tid + 32u * (unsigned)k;
                 row_t[k] = 64u;
-                if (idx < sel_hi) {
+                if (idx < scratch[41]) {
                     const long long c = (long long)__ldg(s.op.list + idx) - ((long long)s.g << 6);
                     if (c < 0 || c >= (long long)s.n_tok) bad = true;      // (a list that is not increasing)
                     else row_t[k] = (unsigned)c;
