@@ -511,17 +511,19 @@ def test_staged_calls_are_ordered_on_the_callers_stream(codec):
         dev.close()
 
 
-@pytest.mark.parametrize("codec", [RAW, INT8])
-def test_a_wait_that_runs_out_is_reported_and_the_context_recovers(codec):
+@pytest.mark.parametrize("codec,bs", [(RAW, 16), (INT8, 16), (INT8, 1)], ids=["raw", "int8", "int8-as-token-rows"])
+def test_a_wait_that_runs_out_is_reported_and_the_context_recovers(codec, bs):
     """Every wait inside the tile pipeline is bounded.  With the bound set below the latency of a memory access the
     launch gives up at once: the call returns, kdn_status_sync reports KDN_E_TIMEOUT, no CTA leaves with a copy in
-    flight, and once the default bound is back the same context gives bit-exact results."""
-    shape = synth.TOY.with_(n_layers=2, n_kv_heads=4, head_dim=64, block_size=16, n_blocks=64)
+    flight, and once the default bound is back the same context gives bit-exact results.  (block_size 1: the kernels
+    whose tiles take up to 16 token rows.)"""
+    nblk = 64 * 16 // bs
+    shape = synth.TOY.with_(n_layers=2, n_kv_heads=4, head_dim=64, block_size=bs, n_blocks=nblk)
     dev = Device(shape, seed=5)
     try:
         K = dev.K
         host = dev.pool_np()
-        tab = np.random.default_rng(4).permutation(64)[:20].astype(np.int32)
+        tab = np.random.default_rng(4).permutation(nblk)[:20 * 16 // bs].astype(np.int32)
         T, off = 300, 5
         buf = dev.chunk_buf(T, codec)
         K.kdn_set_wait_limit_ns(dev.ctx, 40)
@@ -533,7 +535,11 @@ def test_a_wait_that_runs_out_is_reported_and_the_context_recovers(codec):
         dev.store([dev.op(dev.table(tab), off, buf, T, codec)])
         assert dev.sync() == 0
         assert np.array_equal(to_np(buf), oracle.store(host, tab, off, T, codec))
-        dst = np.random.default_rng(5).permutation(64)[:20].astype(np.int32)
+        dst = np.random.default_rng(5).permutation(nblk)[:20 * 16 // bs].astype(np.int32)
+        K.kdn_set_wait_limit_ns(dev.ctx, 40)                    # the same for a retrieve: it may have written some rows, no more
+        dev.retrieve([dev.op(dev.table(dst), off, buf, T, codec)])
+        assert dev.sync() == K.KDN_E_TIMEOUT
+        K.kdn_set_wait_limit_ns(dev.ctx, 0)
         dev.retrieve([dev.op(dev.table(dst), off, buf, T, codec)])
         assert dev.sync() == 0
         ref = host.copy()
