@@ -384,7 +384,8 @@ kdn_status kdn_set_tuning(kdn_ctx *ctx, const kdn_tuning *tuning);
  * on first use).  Takes effect at the next pinned-host call; frees slabs already allocated. */
 kdn_status kdn_set_staging_bytes(kdn_ctx *ctx, size_t bytes_per_slab);
 
-/* Limit, in nanoseconds, after which a wait inside the tile pipeline gives up and the launch reports KDN_E_TIMEOUT
+/* Limit, in nanoseconds, after which a wait inside the tile pipeline (and the wait of a key-plane or token-delta CTA for
+ * its rows or bytes) gives up and the launch reports KDN_E_TIMEOUT
  * (default, and ns = 0: two seconds).  The waits that let a CTA's own copies finish before it leaves always keep the
  * default.  Meant for exercising the error path: with a limit shorter than a memory access the next launches give up
  * almost at once, write little or nothing, and kdn_status_sync returns KDN_E_TIMEOUT; nothing faults or hangs, and

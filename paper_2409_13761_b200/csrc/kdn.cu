@@ -662,6 +662,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
         if (kc_threads < 64u) kc_threads = 64u;
         KcLaunch kp{};
         kp.one = 1.0f;
+        kp.wait_limit_ns = ctx->wait_limit_ns;
         kp.cols = cols;
         kp.n_split = n_split;
         kp.ops = inl ? nullptr : slot->d_ops;
@@ -733,6 +734,7 @@ kdn_status launch_td(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *hops,
     for (int first = 0; first < n; first += kInlineOps) {
         const int m = n - first < kInlineOps ? n - first : kInlineOps;
         TdLaunch tp{};
+        tp.wait_limit_ns = ctx->wait_limit_ns;
         RopeInline rope_inl{};
         int n_rope = 0, max_groups = 0, max_layers = 0;
         for (int i = 0; i < m; ++i) {

@@ -1259,6 +1259,7 @@ struct KcLaunch {
     unsigned n_split;         // row_elems / cols
     int *status;
     float one;                // 1.0f (see Launch::one)
+    unsigned long long wait_limit_ns;   // the wait for the tile gives up after this long
     DevOp inline_ops[kInlineOps];
 };
 
@@ -1348,7 +1349,7 @@ __global__ void __launch_bounds__(512) kdn_store_kc_kernel(const __grid_constant
     }
     __syncthreads();
     if (*abort_flag) return;
-    const bool landed = mbar_wait(bar, 0u, abort_flag);
+    const bool landed = mbar_wait(bar, 0u, abort_flag, P.wait_limit_ns);
     if (!__syncthreads_and(landed)) {                                         // all threads leave together
         if (tid == 0) {
             atomicCAS(P.status, 0, kStatusTimeout);

@@ -33,6 +33,7 @@ struct TdLaunch {
     unsigned n_split;         // row_elems / cols
     const float2 *rope;
     int *status;
+    unsigned long long wait_limit_ns;   // a wait for a slice's bytes gives up after this long
     DevOp inline_ops[kInlineOps];
 };
 
@@ -310,8 +311,18 @@ __global__ void __launch_bounds__(512) kdn_td_plan_kernel(const __grid_constant_
         for (unsigned i = tid; i < 64u * 16u; i += blockDim.x) hi_tab[i] = hi_one[i >> 4];
     }
     __syncthreads();
-    if (*abort_flag) return;
-    const bool landed = mbar_wait(bar, 0u, abort_flag);
+    const TdLayout lay = td_layout(P.L, RE, s.op.T, codec);
+    const unsigned long long row = (unsigned long long)s.seg * RE + s.c0;
+    // a slice that is given up (a block id outside the pool, a wait that ran out) leaves lengths of zero behind: the scan
+    // and the encoder then see a consistent, if incomplete, chunk instead of whatever the buffer held before
+    auto give_up = [&]() {
+        for (unsigned ch = tid; ch < C; ch += blockDim.x) {
+            s.op.data[lay.lens + row + ch] = 0;
+            s.op.data[lay.params + row + ch] = 0;
+        }
+    };
+    if (*abort_flag) { give_up(); return; }
+    const bool landed = mbar_wait(bar, 0u, abort_flag, P.wait_limit_ns);
     if (!__syncthreads_and(landed)) {
         if (tid == 0) {
             atomicCAS(P.status, 0, kStatusTimeout);
@@ -319,10 +330,9 @@ __global__ void __launch_bounds__(512) kdn_td_plan_kernel(const __grid_constant_
             while (!mbar_try_wait(bar, 0u))
                 if (global_timer_ns() - t0 > kWaitLimitNs) break;
         }
+        give_up();
         return;
     }
-    const TdLayout lay = td_layout(P.L, RE, s.op.T, codec);
-    const unsigned long long row = (unsigned long long)s.seg * RE + s.c0;
     td_channel_scales(X, pmax, inv, reinterpret_cast<float *>(s.op.data + lay.scales) + row, s.n_tok, C, qmax);
     // one thread per channel: the cost in bits of every (mode, k), then the first minimum.  Lengths are at most 24, so
     // the 8-bit fields hold eight symbols' worth; after every eight symbols they are spread into 16-bit fields.
@@ -472,9 +482,17 @@ __global__ void __launch_bounds__(512) kdn_td_encode_kernel(const __grid_constan
     const unsigned long long seg_begin = reinterpret_cast<const unsigned long long *>(s.op.data)[s.seg];
     unsigned char *dst = s.op.data + seg_begin + total_before;
     const unsigned shift = (unsigned)((unsigned long long)dst & 15ull);                      // staging mirrors the destination's alignment
+    // the lengths are the planner's, but a planner CTA may have given up: nothing may leave the staging area or the chunk
+    // (the capacity ends on a 16-byte boundary, so the padding of a segment's last slice fits whenever its bytes do)
+    const bool sane = total_slice <= C * td_max_len(codec) && seg_begin >= lay.streams &&
+                      seg_begin + total_before + total_slice <= lay.capacity;
+    if (tid == 0 && !sane) {
+        atomicCAS(P.status, 0, kStatusRange);
+        *abort_flag = 1;
+    }
     __syncthreads();
     if (*abort_flag) return;
-    const bool landed = mbar_wait(bar, 0u, abort_flag);
+    const bool landed = mbar_wait(bar, 0u, abort_flag, P.wait_limit_ns);
     if (!__syncthreads_and(landed)) {
         if (tid == 0) {
             atomicCAS(P.status, 0, kStatusTimeout);
@@ -488,12 +506,13 @@ __global__ void __launch_bounds__(512) kdn_td_encode_kernel(const __grid_constan
     // the last word of a sub-stream also hold bits of its neighbours
     for (unsigned i = tid; i < (C * 72u + 32u) / 16u; i += blockDim.x) sts128(stage + (size_t)i * 16u, make_uint4(0u, 0u, 0u, 0u));
     td_channel_scales(X, pmax, inv, nullptr, s.n_tok, C, qmax);                 // (its barriers also publish the zeros)
-    if (tid < C) {
+    if (tid < C && my_len != 0u && my_len <= td_max_len(codec)) {       // (a length of zero: the planner gave this slice up)
         const unsigned param = s.op.data[lay.params + row + s.c0 + tid];
         const bool delta = (param & 8u) != 0u;
         const unsigned k = param & 7u, kmask = (1u << k) - 1u, k1 = k + 1u;
         const float iv = inv[tid];
         const uint32_t addr = smem_u32(stage) + shift + my_off;          // first byte of the sub-stream
+        const uint32_t wend = (addr + my_len + 3u) & ~3u;                 // no word at or past this one is this sub-stream's
         uint32_t wp = addr & ~3u;                                         // the word it starts in ...
         unsigned nb = (addr & 3u) * 8u;                                   // ... after this many bits that are not its own
         unsigned long long acc = 0;
@@ -511,11 +530,11 @@ __global__ void __launch_bounds__(512) kdn_td_encode_kernel(const __grid_constan
             if (nb >= 32u) {                                              // a full word: bytes in stream order, first byte lowest
                 nb -= 32u;
                 const uint32_t word = td_be((uint32_t)(acc >> nb));
-                asm volatile("red.shared.or.b32 [%0], %1;" :: "r"(wp), "r"(word) : "memory");
+                if (wp < wend) asm volatile("red.shared.or.b32 [%0], %1;" :: "r"(wp), "r"(word) : "memory");
                 wp += 4u;
             }
         }
-        if (nb > 0u) {
+        if (nb > 0u && wp < wend) {
             const uint32_t word = td_be((uint32_t)(acc << (32u - nb)));
             asm volatile("red.shared.or.b32 [%0], %1;" :: "r"(wp), "r"(word) : "memory");
         }
@@ -610,7 +629,7 @@ __global__ void __launch_bounds__(kCols ? kCols : 512) kdn_td_decode_kernel(cons
     }
     __syncthreads();
     if (*abort_flag) return;
-    const bool landed = mbar_wait(bar, 0u, abort_flag);
+    const bool landed = mbar_wait(bar, 0u, abort_flag, P.wait_limit_ns);
     if (!__syncthreads_and(landed)) {
         if (tid == 0) {
             atomicCAS(P.status, 0, kStatusTimeout);

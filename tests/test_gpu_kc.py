@@ -263,3 +263,32 @@ def test_keep_list_chunks_against_the_oracle(shape, codec):
         assert np.array_equal(dev.pool_np(), ref)
     finally:
         dev.close()
+
+
+@pytest.mark.parametrize("codec", KC, ids=["int8kc", "int4kc"])
+def test_a_wait_that_runs_out_in_the_key_plane_store(codec):
+    """The key-plane kernel's wait for its tile is bounded too: KDN_E_TIMEOUT, no write outside the chunk, the pool
+    untouched, and the context bit-exact again once the default bound is back."""
+    shape = synth.TOY.with_(n_layers=2, n_kv_heads=4, head_dim=64, block_size=16, n_blocks=96)
+    dev = Device(shape, seed=9)
+    try:
+        K = dev.K
+        host = dev.pool_np()
+        tab = np.random.default_rng(6).permutation(96)[:20].astype(np.int32)
+        T = 300
+        guard = 4096
+        n = K.kdn_chunk_bytes(dev.desc, T, codec)
+        arena = torch.full((n + 2 * guard,), 0x5C, dtype=torch.uint8, device=dev.dev)
+        buf = arena[guard:guard + n]
+        K.kdn_set_wait_limit_ns(dev.ctx, 40)
+        dev.store([dev.op(dev.table(tab), 0, buf, T, codec)])
+        assert dev.sync() in (0, K.KDN_E_TIMEOUT)                         # (0: every CTA found its rows landed in time)
+        assert np.array_equal(dev.pool_np(), host)
+        a = to_np(arena)
+        assert np.all(a[:guard] == 0x5C) and np.all(a[-guard:] == 0x5C)
+        K.kdn_set_wait_limit_ns(dev.ctx, 0)
+        dev.store([dev.op(dev.table(tab), 0, buf, T, codec)])
+        assert dev.sync() == 0
+        assert np.array_equal(to_np(buf), oracle.store(host, tab, 0, T, codec))
+    finally:
+        dev.close()

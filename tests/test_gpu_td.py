@@ -376,3 +376,80 @@ def test_select_list_compose_against_the_oracle(shape, codec):
         check_rotated_keys(g, kref[:, p], kmag[:, p], ref[:, 0, rt[p // bs], p % bs], min_equal=0.995 if g.size >= 8192 else 0.95)
     finally:
         dev.close()
+
+
+@pytest.mark.parametrize("codec", [TD8, TD4], ids=["int8td", "int4td"])
+def test_a_wait_that_runs_out_in_the_token_delta_kernels(codec):
+    """The waits of the planner, the encoder and the decoder are bounded like those of the tile pipeline.  With the
+    bound below the latency of a memory access a CTA whose bytes have not landed gives up: KDN_E_TIMEOUT (or, when every
+    CTA found its bytes in time, a correct result), nothing written outside the chunk (a planner CTA that gives up
+    leaves zero lengths behind, and the encoder trusts no length), the pool untouched by a store; with the default bound
+    back the same context is bit-exact again."""
+    shape = synth.TOY.with_(n_layers=2, n_kv_heads=4, head_dim=64, block_size=16, n_blocks=96)
+    dev = Device(shape, seed=9)
+    try:
+        K = dev.K
+        host = dev.pool_np()
+        tab = np.random.default_rng(6).permutation(96)[:20].astype(np.int32)
+        T = 300
+        guard = 4096
+        whole = dev.chunk_buf(T, codec)                                       # (reference size)
+        arena = torch.full((whole.numel() + 2 * guard,), 0x5C, dtype=torch.uint8, device=dev.dev)
+        buf = arena[guard:guard + whole.numel()]
+        want = oracle.store(host, tab, 0, T, codec)
+        used = oracle.td_used_bytes(want, shape.n_layers, shape.n_kv_heads, shape.head_dim, T, codec)
+        K.kdn_set_wait_limit_ns(dev.ctx, 40)
+        dev.store([dev.op(dev.table(tab), 0, buf, T, codec)])
+        st = dev.sync()
+        # (a CTA of the store kernels fills its tables before it looks for its rows, so they may all have landed by then)
+        assert st in (0, K.KDN_E_TIMEOUT)
+        assert np.array_equal(dev.pool_np(), host)
+        a = to_np(arena)
+        assert np.all(a[:guard] == 0x5C) and np.all(a[-guard:] == 0x5C)       # nothing left the chunk
+        assert st != 0 or np.array_equal(a[guard:guard + used], want[:used])
+        K.kdn_set_wait_limit_ns(dev.ctx, 0)
+        dev.store([dev.op(dev.table(tab), 0, buf, T, codec)])
+        assert dev.sync() == 0
+        assert np.array_equal(to_np(buf)[:used], want[:used])
+        dst = np.random.default_rng(7).permutation(96)[:20].astype(np.int32)
+        K.kdn_set_wait_limit_ns(dev.ctx, 40)
+        dev.retrieve([dev.op(dev.table(dst), 0, buf, T, codec)])
+        assert dev.sync() in (0, K.KDN_E_TIMEOUT)
+        K.kdn_set_wait_limit_ns(dev.ctx, 0)
+        dev.retrieve([dev.op(dev.table(dst), 0, buf, T, codec)])
+        assert dev.sync() == 0
+        ref = host.copy()
+        oracle.retrieve(ref, dst, 0, T, codec, want)
+        assert np.array_equal(dev.pool_np(), ref)
+    finally:
+        dev.close()
+
+
+@pytest.mark.parametrize("codec", [TD8, TD4], ids=["int8td", "int4td"])
+def test_a_block_id_outside_the_pool_in_a_store_is_reported_and_nothing_leaves_the_chunk(codec):
+    """The planner CTAs of the slices that meet the bad table entry give up and leave zero lengths behind; the other
+    slices of the same segments are still placed consistently: KDN_E_RANGE, no byte outside the chunk, the pool as it was."""
+    shape = synth.TOY.with_(n_layers=2, n_kv_heads=4, head_dim=64, block_size=16, n_blocks=96)
+    dev = Device(shape, seed=10)
+    try:
+        K = dev.K
+        host = dev.pool_np()
+        tab = np.random.default_rng(8).permutation(96)[:20].astype(np.int32)
+        bad = tab.copy()
+        bad[7] = 96 + 5                                                       # tokens 112 .. 127: the second group
+        T, guard = 300, 4096
+        n = K.kdn_chunk_bytes(dev.desc, T, codec)
+        arena = torch.full((n + 2 * guard,), 0xFF, dtype=torch.uint8, device=dev.dev)   # 0xFF: lengths no sub-stream can have
+        buf = arena[guard:guard + n]
+        dev.store([dev.op(dev.table(bad), 0, buf, T, codec)])
+        assert dev.sync() == K.KDN_E_RANGE
+        a = to_np(arena)
+        assert np.all(a[:guard] == 0xFF) and np.all(a[-guard:] == 0xFF)
+        assert np.array_equal(dev.pool_np(), host)
+        dev.store([dev.op(dev.table(tab), 0, buf, T, codec)])
+        assert dev.sync() == 0
+        want = oracle.store(host, tab, 0, T, codec)
+        used = oracle.td_used_bytes(want, shape.n_layers, shape.n_kv_heads, shape.head_dim, T, codec)
+        assert np.array_equal(to_np(buf)[:used], want[:used])
+    finally:
+        dev.close()
