@@ -62,11 +62,15 @@ __host__ __device__ inline TdLayout td_layout(int L, unsigned row_elems, int T, 
 // small per-warp scratch, barrier.
 // (the plan kernel keeps two tables of code-word lengths in place of the staging area, each replicated so that the
 // lanes of a warp never meet in a bank: 64 entries x 32 copies x 4 bytes and 64 entries x 16 copies x 8 bytes)
+// Behind the encoder's staging area: room for the longest thing a channel could write from the last planned byte on (64
+// symbols of 24 bits), so that a sub-stream that came out longer than planned -- the pool changed under the store --
+// garbles the chunk's bytes, which the caller has then forfeited, but never leaves the area.
+constexpr unsigned kTdStageSlack = 256u;
 constexpr unsigned kTdCostBytes = 64u * 32u * 4u + 64u * 16u * 8u + 64u * 4u + 64u * 8u;   // the copies, and one set of entries to copy from
 __host__ __device__ inline size_t td_store_smem_bytes(unsigned cols, bool encode)
 {
     return (size_t)64 * cols * 2u + (size_t)kKcSlices * cols * 2u + (size_t)cols * 4u +
-           (encode ? (size_t)cols * 72u + 32u : (size_t)kTdCostBytes) + 256u + 16u;
+           (encode ? (size_t)cols * 72u + 32u + kTdStageSlack : (size_t)kTdCostBytes) + 256u + 16u;
 }
 // Shared memory of the decode kernel: the slice's stream bytes as they lie in the chunk, the same sub-streams
 // interleaved word by word (so that the 32 lanes of a warp read 32 different banks), codes, scales, offsets, barrier.
@@ -451,7 +455,7 @@ __global__ void __launch_bounds__(512) kdn_td_encode_kernel(const __grid_constan
     unsigned char *pmax = X + (size_t)64 * C * 2u;
     float *inv = reinterpret_cast<float *>(pmax + (size_t)kKcSlices * C * 2u);
     unsigned char *stage = reinterpret_cast<unsigned char *>(inv) + (size_t)C * 4u;          // C * 72 + 32 bytes
-    unsigned *scratch = reinterpret_cast<unsigned *>(stage + (size_t)C * 72u + 32u);          // 64 words
+    unsigned *scratch = reinterpret_cast<unsigned *>(stage + (size_t)C * 72u + 32u + kTdStageSlack);   // 64 words
     unsigned long long *bar_mem = reinterpret_cast<unsigned long long *>(reinterpret_cast<unsigned char *>(scratch) + 256u);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bar_mem + 1);
     const uint32_t bar = smem_u32(bar_mem);
@@ -512,7 +516,6 @@ __global__ void __launch_bounds__(512) kdn_td_encode_kernel(const __grid_constan
         const unsigned k = param & 7u, kmask = (1u << k) - 1u, k1 = k + 1u;
         const float iv = inv[tid];
         const uint32_t addr = smem_u32(stage) + shift + my_off;          // first byte of the sub-stream
-        const uint32_t wend = (addr + my_len + 3u) & ~3u;                 // no word at or past this one is this sub-stream's
         uint32_t wp = addr & ~3u;                                         // the word it starts in ...
         unsigned nb = (addr & 3u) * 8u;                                   // ... after this many bits that are not its own
         unsigned long long acc = 0;
@@ -530,11 +533,11 @@ __global__ void __launch_bounds__(512) kdn_td_encode_kernel(const __grid_constan
             if (nb >= 32u) {                                              // a full word: bytes in stream order, first byte lowest
                 nb -= 32u;
                 const uint32_t word = td_be((uint32_t)(acc >> nb));
-                if (wp < wend) asm volatile("red.shared.or.b32 [%0], %1;" :: "r"(wp), "r"(word) : "memory");
+                asm volatile("red.shared.or.b32 [%0], %1;" :: "r"(wp), "r"(word) : "memory");
                 wp += 4u;
             }
         }
-        if (nb > 0u && wp < wend) {
+        if (nb > 0u) {
             const uint32_t word = td_be((uint32_t)(acc << (32u - nb)));
             asm volatile("red.shared.or.b32 [%0], %1;" :: "r"(wp), "r"(word) : "memory");
         }
