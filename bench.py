@@ -185,8 +185,8 @@ class ClockSampler:
 # DRAM bytes (read + write) per launch from a profiler capture of a reduced case (8 chunks per store/retrieve
 # launch, 2 parts per compose launch), scaled by the units a bench launch processes: every byte is touched once,
 # so traffic grows in proportion.  Valid only for the kernel source the capture was taken from (its hash).
-NCU_KERNEL_SHA = "d5c5296358235c98"
-NCU_SMALL_CASE_BYTES = {"store_raw": (536.921344e6 + 486.536960e6, 8), "retrieve_raw": (536.920832e6 + 491.426816e6, 8), "compose_raw": (268.572928e6 + 222.653952e6, 2), "store_int8": (536.936704e6 + 251.162112e6, 8), "retrieve_int8": (285.271040e6 + 484.859904e6, 8), "compose_int8": (142.711552e6 + 214.546944e6, 2)}
+NCU_KERNEL_SHA = "d1f836c912029be7"
+NCU_SMALL_CASE_BYTES = {"store_raw": (536.921088e6 + 488.388608e6, 8), "retrieve_raw": (536.921088e6 + 490.368768e6, 8), "compose_raw": (268.505856e6 + 223.703552e6, 2), "store_int8": (536.938240e6 + 250.342912e6, 8), "retrieve_int8": (285.271040e6 + 482.806528e6, 8), "compose_int8": (142.674944e6 + 213.722368e6, 2)}
 
 
 def measured_traffic(op: str, units: float):
