@@ -446,7 +446,9 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
     // (list_mode 3): a tile then takes several token rows, wherever their blocks are, and rows that are neighbours in the
     // pool still share a copy (8B shape, block_size 1: int8 store / retrieve 3.5 / 3.7 -> 5.2 / 5.3 TB/s).
     std::vector<HostOp> as_rows;
-    if (any_coded && !any_rot && !any_list && !any_kc && (OP == OP_STORE || OP == OP_RETRIEVE) && ctx->tuning.tile_bytes <= 0 &&
+    // (the kernels for tiles of many rows exist for the built-in shapes only: a caller-set shape keeps the ordinary kernels)
+    const bool own_shape = ctx->tuning.compute_groups > 0 || ctx->tuning.group_warps > 0;
+    if (any_coded && !any_rot && !any_list && !any_kc && (OP == OP_STORE || OP == OP_RETRIEVE) && ctx->tuning.tile_bytes <= 0 && !own_shape &&
         (unsigned long long)pool.bs * row_elems * 2ull <= 2048ull && (unsigned long long)pool.nb * (unsigned)pool.bs < 0xffffffffull) {
         as_rows.assign(hops, hops + n);
         for (HostOp &h : as_rows) {
@@ -498,6 +500,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
         int want_rows = ctx->tuning.tile_bytes > 0 ? ctx->tuning.tile_bytes / 2 / (int)row_elems : 2048 / (int)row_elems;
         if (kc_decode)                                     // a key tile must lie inside one 64-token group: a power of two
             while (want_rows & (want_rows - 1)) want_rows &= want_rows - 1;
+        if (own_shape && want_rows > kMaxRowsPerTile) want_rows = kMaxRowsPerTile;
         if (!any_coded && !any_rot && all_keep && want_rows >= 2 && row_elems < 1024u && (unsigned long long)pool.nb * (unsigned)pool.bs < 0xffffffffull) {
             // copy form on rows shorter than 2 KiB (few KV heads per GPU): several rows per tile as well
             rows_per_tile = want_rows > kWideRowsPerTile ? kWideRowsPerTile : want_rows;
