@@ -75,7 +75,8 @@
  *   result is not known before the kernels have run); kdn_retrieve and kdn_compose also take KDN_MEM_PINNED_HOST
  *   chunks: the library reads seg_off[S] from host memory and copies just the bytes in use over the host link (a
  *   chunk whose bytes in use exceed a staging slab, or whose offset table no store can have written, is refused).
- *   Files (kdn_*_file) are not supported.
+ *   kdn_retrieve_file takes them the same way (the offset table is read from the file first, then the bytes in use,
+ *   so only those need be in the file); kdn_store_file does not, for the reason kdn_store does not write host chunks.
  * Key re-rotation in kdn_compose: the stored keys of a part carry rotary
  *   position embedding for positions base_pos + t; placing the part at
  *   dst_pos rotates each pair (k[i], k[i + D/2]) of every head by

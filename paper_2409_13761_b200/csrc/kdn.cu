@@ -1025,9 +1025,24 @@ kdn_status run_td_host(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector
     auto flush = [&]() -> kdn_status {
         if (batch.empty()) return KDN_OK;
         const unsigned s = ctx->slab_next++ & 1u;
+        bool any_file = false;
+        for (const Piece &p : pieces) any_file |= p.host == nullptr;
+        if (any_file) {
+            // chunks in files: the host reads their bytes in use into the page-locked mirror of the slab first
+            kdn_status r = ensure_bounce(ctx);
+            if (r != KDN_OK) return r;
+            if (ctx->bounce_busy[s]) KDN_CUDA(cudaEventSynchronize(ctx->bounce_done[s]));
+            ctx->bounce_busy[s] = false;
+            if (!file_io(pieces, ctx->bounce[s], false)) return KDN_E_IO;
+        }
         KDN_CUDA(cudaStreamWaitEvent(side, ctx->slab_free[s], 0));
         for (const Piece &p : pieces)
-            KDN_CUDA(cudaMemcpyAsync(ctx->slab[s] + p.slab_off, p.host, p.bytes, cudaMemcpyHostToDevice, side));
+            KDN_CUDA(cudaMemcpyAsync(ctx->slab[s] + p.slab_off, p.host ? p.host : ctx->bounce[s] + p.slab_off, p.bytes,
+                                     cudaMemcpyHostToDevice, side));
+        if (any_file) {
+            KDN_CUDA(cudaEventRecord(ctx->bounce_done[s], side));
+            ctx->bounce_busy[s] = true;
+        }
         KDN_CUDA(cudaEventRecord(ctx->slab_ready[s], side));
         KDN_CUDA(cudaStreamWaitEvent(stream, ctx->slab_ready[s], 0));
         for (HostOp &h : batch) {                                                             // offsets become addresses
@@ -1044,7 +1059,15 @@ kdn_status run_td_host(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector
     };
     for (const HostOp &h : hops) {
         const TdLayout lay = td_layout(pool.L, row_elems, h.op.T, h.op.codec);
-        const unsigned long long *seg_off = reinterpret_cast<const unsigned long long *>(h.op.data);   // host memory: readable here
+        // the chunk's own offset table says how many bytes it uses: in host memory it is read in place, from a file it
+        // is read first (a short blocking read of 8 (S + 1) bytes)
+        std::vector<unsigned long long> from_file;
+        const unsigned long long *seg_off = reinterpret_cast<const unsigned long long *>(h.op.data);
+        if (h.fd >= 0) {
+            from_file.resize((size_t)lay.S + 1u);
+            if (!read_fully(h.fd, reinterpret_cast<unsigned char *>(from_file.data()), from_file.size() * 8u, h.file_off)) return KDN_E_IO;
+            seg_off = from_file.data();
+        }
         const unsigned long long used = seg_off[lay.S];
         bool stored = used >= lay.streams && used <= lay.capacity && !(used & 15ull) && seg_off[0] == lay.streams;
         for (unsigned long long i = 0; stored && i < lay.S; ++i) stored = seg_off[i] <= seg_off[i + 1];
@@ -1054,7 +1077,7 @@ kdn_status run_td_host(kdn_ctx *ctx, const Pool &pool, int OP, const std::vector
             st = flush();
             if (st != KDN_OK) return st;
         }
-        pieces.push_back(Piece{ h.op.data, fill, (size_t)used, -1, 0 });
+        pieces.push_back(h.fd >= 0 ? Piece{ nullptr, fill, (size_t)used, h.fd, h.file_off } : Piece{ h.op.data, fill, (size_t)used, -1, 0 });
         HostOp sub = h;
         sub.op.data = (unsigned char *)(uintptr_t)fill;      // offset inside the slab until the slab is known
         sub.op.scales = (unsigned char *)(uintptr_t)(fill + (size_t)used);   // the slab holds no more of the chunk than this
@@ -1418,7 +1441,8 @@ static kdn_status xfer_file(kdn_ctx *ctx, int pool_id, int OP, const kdn_file_op
         if (st != KDN_OK) return st;
         st = check_kc(&shape, &o.chunk, o.token_offset);
         if (st != KDN_OK) return st;
-        if (is_td(o.chunk.codec)) return KDN_E_UNSUPPORTED;      // variable-length chunks are not staged through files
+        // (a token-delta chunk in a file: its offset table first, then the bytes it uses; storing one is refused below,
+        // as for host memory: the size of the result is not known before the kernels have run)
         if (ops[i].fd < 0 || ops[i].file_offset < 0) return KDN_E_INVAL;
     }
     if (cudaSetDevice(ctx->device) != cudaSuccess) return KDN_E_CUDA;

@@ -5,6 +5,8 @@ retrieve: the pool is bit-identical to the oracle's; compose: values and unrotat
 keys within the rotation tolerance.  Inputs are uncorrelated and token-correlated (so that both coding modes occur),
 with zero, constant, extreme and saw-tooth channels planted (flushed scales, the shortest and the longest
 sub-streams, the escape code)."""
+import os
+
 import numpy as np
 import pytest
 import torch
@@ -209,8 +211,8 @@ def test_retrieve_and_compose_from_page_locked_host_chunks(codec):
     """Delivery of compressed chunks (the point of coding them): token-delta chunks kept in page-locked host memory are
     retrieved and composed; only the bytes each chunk uses cross the host link, through staging slabs that hold a few
     chunks at a time, in a call that also carries device-resident chunks."""
-    shape = synth.TOY.with_(n_layers=3, n_kv_heads=2, head_dim=64, block_size=16, n_blocks=256)
-    perm = np.random.default_rng(12).permutation(256).astype(np.int32)
+    shape = synth.TOY.with_(n_layers=3, n_kv_heads=2, head_dim=64, block_size=16, n_blocks=512)
+    perm = np.random.default_rng(12).permutation(512).astype(np.int32)
     pool = make_pool_np(shape, perm[:40], 0, 640, 0.9, seed=77)
     dev = Device(shape, pool_np=pool)
     try:
@@ -260,12 +262,29 @@ def test_retrieve_and_compose_from_page_locked_host_chunks(codec):
         assert dev.sync() == 0
         oracle.retrieve(before, lw, 0, Ts[3], codec, wants[3])
         assert np.array_equal(dev.pool_np(), before)
-        # files are not a home for these chunks
+        # chunks in files: only the bytes in use need be there; all five in one file at odd offsets, retrieved in one call
         import tempfile
         with tempfile.TemporaryFile() as tf:
-            with pytest.raises(K.KdnError) as e:
-                K.kdn_retrieve_file(dev.ctx, dev.pool_id, [dev.op(dev.table(lw), 0, dbufs[3], Ts[3], codec)], [tf.fileno()], [0], dev.stream.cuda_stream)
+            offs, cur = [], 24
+            for h, w, T in zip(hbufs, wants, Ts):
+                used = oracle.td_used_bytes(w, 3, 2, 64, T, codec)
+                offs.append(cur)
+                os.pwrite(tf.fileno(), h[:used].numpy().tobytes(), cur)
+                cur += used + 40
+            fdst = [perm[250 + 20 * i:250 + 20 * i + 17] for i in range(len(Ts))]
+            fops = [dev.op(dev.table(d), 0, dbufs[i], T, codec) for i, (d, T) in enumerate(zip(fdst, Ts))]   # (the data address is ignored)
+            before = dev.pool_np()
+            K.kdn_retrieve_file(dev.ctx, dev.pool_id, fops, [tf.fileno()] * len(Ts), offs, dev.stream.cuda_stream)
+            assert dev.sync() == 0
+            for d, w, T in zip(fdst, wants, Ts):
+                oracle.retrieve(before, d, 0, T, codec, w)
+            assert np.array_equal(dev.pool_np(), before)
+            with pytest.raises(K.KdnError) as e:                          # storing into a file: the size is not known beforehand
+                K.kdn_store_file(dev.ctx, dev.pool_id, [fops[0]], [tf.fileno()], [0], dev.stream.cuda_stream)
             assert e.value.status == K.KDN_E_UNSUPPORTED
+            with pytest.raises(K.KdnError) as e:                          # no offset table a store can have written at this place
+                K.kdn_retrieve_file(dev.ctx, dev.pool_id, [fops[0]], [tf.fileno()], [offs[0] + 8], dev.stream.cuda_stream)
+            assert e.value.status == K.KDN_E_SHAPE
         # a host buffer no store has written is refused, not followed
         junk = dev.chunk_buf(64, codec, pinned=True, fill=0xFF)
         with pytest.raises(K.KdnError) as e:
