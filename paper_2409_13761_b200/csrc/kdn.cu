@@ -528,7 +528,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
         // a small block_size) caps the tile at the block.  From sweeps on the 8B shape with 4, 2 and 1 KV heads:
         // the copy form keeps the same bytes in flight per SM with more CTAs, then more slots (one head, 4 KiB blocks:
         // 1.9 -> 6.3 TB/s); the coding forms give a tile of 4 KiB or less to one warp instead of four (int8 store /
-        // retrieve 4.2 / 4.6 -> 5.8 / 5.7, compose 3.8 -> 5.4); a rotation-only compose takes six slots in as many CTAs
+        // retrieve 4.2 / 4.6 -> 5.8 / 5.7, compose 3.8 -> 5.4, eight slots in four CTAs); a rotation-only compose takes six slots in as many CTAs
         // as fit (2.7 -> 6.2); a coded compose whose every tile needs its own table entry takes six slots (5.6 -> 6.2).
         const unsigned tb = tile_elems * 2u;
         const bool capped = tb < (unsigned)def.tile_bytes;
@@ -553,7 +553,7 @@ kdn_status launch_batch(kdn_ctx *ctx, const Pool &pool, int OP, const HostOp *ho
                 def = Shape{ 0, 6, (int)ctas, 1, 1 };
             }
         } else if (tb <= 4096u) {
-            def = Shape{ 0, 8, 8, 2, 1, 1 };
+            def = Shape{ 0, 8, 4, 2, 1, 1 };
         } else if (tpb == 1u) {
             def = Shape{ 0, 6, 3, 1, 1 };
         }
